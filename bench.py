@@ -1,0 +1,346 @@
+#!/usr/bin/env python
+"""Benchmark of the delayed synchronous step (ABS-SGD, arXiv 2308.15164, Algorithm 1) on B200.
+
+A "step" is one iteration of Algorithm 1 on the ResNet18-sized workload (P = 11,689,512 fp32
+parameters, W = 4 workers with b = (2,2,4,8) micro-batches): 16 accumulate launches (Step 2)
+plus one fused weighted-reduce/update launch (Step 1), run in pipelined mode so that Step 1 of
+iteration t overlaps Step 2 of iteration t+1.  The metric is algorithmic HBM bytes per second:
+
+    bytes per step = 16 * 12 * P  (accumulate: read g, read acc, write acc)
+                   + (8 * 4 + 16) * P  (fused step: read 4 acc + x + v, write x + v + 4 zeros)
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+
+With N > 1 (launched by torchrun) every rank runs an independent replica on its own GPU (the
+step has no exchange between replicas); rank 0 prints ONE JSON line with the whole-job value.
+"""
+
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import tempfile
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np  # noqa: E402
+
+METRIC = "delayed-sync iteration HBM throughput (16 accumulate + 1 fused sync step, algorithmic bytes)"
+UNIT = "GB/s"
+HBM_NOMINAL_GBS = 8000.0
+HBM_FALLBACK_GBS = 6650.0
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            d = json.load(f)
+        return dict(hbm_gbs=float(d["hbm_gbs"]), bf16_tflops=float(d["bf16_tflops"]),
+                    bf16_tflops_sustained=float(d.get("bf16_tflops_sustained", d["bf16_tflops"])), source="measured")
+    return dict(hbm_gbs=HBM_FALLBACK_GBS, bf16_tflops=1590.0, bf16_tflops_sustained=1400.0, source="fallback")
+
+
+class ClockSampler:
+    """Samples SM clock and throttle reasons with nvidia-smi while the timed region runs."""
+
+    FIELDS = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+              "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+              "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.gpu = gpu_index
+        self.proc = None
+        self.path = None
+
+    def start(self):
+        try:
+            fd, self.path = tempfile.mkstemp(suffix=".csv")
+            os.close(fd)
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--id={self.gpu}", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits",
+                 "-lms", "100"], stdout=open(self.path, "w"), stderr=subprocess.DEVNULL)
+        except Exception:
+            self.proc = None
+
+    def stop(self):
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        if self.proc is None:
+            return out
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        sm, mx, reasons = [], [], set()
+        try:
+            for line in open(self.path):
+                f = [s.strip() for s in line.split(",")]
+                if len(f) < 9:
+                    continue
+                try:
+                    sm.append(float(f[1])); mx.append(float(f[2]))
+                except ValueError:
+                    continue
+                for name, val in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), f[5:9]):
+                    if val.lower().startswith("active"):
+                        reasons.add(name)
+            os.unlink(self.path)
+        except Exception:
+            pass
+        if sm:
+            out.update(sm_mhz=float(np.median(sm)), sm_max_mhz=float(max(mx)), reasons=sorted(reasons), samples=len(sm))
+        return out
+
+
+def bytes_per_step(wl, b_row):
+    g_bytes = 2 if wl.grad_dtype == "bf16" else 4
+    calls = int(sum(b_row))
+    w_act = int(sum(1 for b in b_row if b > 0))
+    acc = calls * (g_bytes + 8) * wl.P
+    sync = (8 * w_act + 16) * wl.P
+    return acc, sync
+
+
+# ------------------------------------------------------------------------------------------
+def run_reference(args):
+    """The CPU oracle (C twin, OpenMP) timed on the host cores, same workload and metric."""
+    from paper_2308_15164_b200 import dist as D
+    from paper_2308_15164_b200 import workloads as wlm
+
+    rank, _, world = D.rank_info()
+    if rank != 0:
+        return
+    from oracle.c_oracle import AbsSgdOracleC
+
+    wl = wlm.config(2)
+    x0 = wlm.params0(wl)
+    pool = wlm.grad_pool(wl)
+    b_row = wlm.schedule(wl)[0]
+    order = wlm.call_order(b_row)
+    acc_b, sync_b = bytes_per_step(wl, b_row)
+    o = AbsSgdOracleC(x0, wl.W, wl.lr, wl.momentum, wl.weight_decay)
+    c = 0
+
+    def one_step():
+        nonlocal c
+        for (i, k) in order:
+            o.accumulate(i, pool[c % wl.pool_size]); c += 1
+        o.sync_step()
+
+    for _ in range(args.warmup):
+        one_step()
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        one_step()
+    dt = time.perf_counter() - t0
+    cores = int(os.environ.get("OMP_NUM_THREADS", os.cpu_count() or 1))
+    val = (acc_b + sync_b) * args.steps / dt / 1e9
+    line = {
+        "impl": "reference", "metric": METRIC, "value": val, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": dt / args.steps * 1e3, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+        "config": {"workload": "cfg2 resnet18-sized: P=11689512, W=4, b=(2,2,4,8), full size, every step on the host"},
+        "cpu_baseline": {"value": val, "unit": UNIT, "cores": cores, "kind": "oracle",
+                         "sample": f"{args.steps} full iterations of the workload (C oracle, OpenMP)"},
+        "e2e": {"value": val, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line), flush=True)
+
+
+# ------------------------------------------------------------------------------------------
+def run_ours(args):
+    import torch
+
+    from paper_2308_15164_b200 import binding as B
+    from paper_2308_15164_b200 import dist as D
+    from paper_2308_15164_b200 import workloads as wlm
+
+    rank, local_rank, world = D.init("nccl")
+    dev = torch.device("cuda", local_rank)
+    torch.cuda.set_device(dev)
+    peaks = measured_peaks()
+
+    wl = wlm.config(2)
+    x0 = wlm.params0(wl)
+    pool = wlm.grad_pool(wl)                      # 16 x P fp32 = 748 MB (larger than the 126 MB L2)
+    b_row = wlm.schedule(wl)[0]
+    order = wlm.call_order(b_row)
+    acc_b, sync_b = bytes_per_step(wl, b_row)
+    step_bytes = acc_b + sync_b
+    pool_d = torch.from_numpy(pool).to(dev)
+    x0_d = torch.from_numpy(x0).to(dev)
+    torch.cuda.synchronize()
+
+    def make(pipelined, host_input=False):
+        return B.AbsSgd(x0_d, wl.W, wl.lr, wl.momentum, wl.weight_decay, pipelined=pipelined, host_input=host_input)
+
+    call_idx = [0]
+    rows = [pool_d[r].data_ptr() for r in range(wl.pool_size)]      # raw device addresses of the pool rows
+
+    def one_step(eng):
+        c = call_idx[0]
+        for (i, k) in order:
+            eng.accumulate(i, rows[c % wl.pool_size]); c += 1
+        call_idx[0] = c
+        eng.sync_step()
+
+    def timed(eng, steps, warmup):
+        for _ in range(warmup):
+            one_step(eng)
+        eng.wait(); eng.synchronize()
+        D.barrier(dev)
+        torch.cuda.synchronize()
+        n0 = eng.launch_count()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        with torch.cuda.stream(eng.stream_acc):
+            e0.record()
+            for _ in range(steps):
+                one_step(eng)
+            eng.wait()                      # stream_acc waits for the last fused kernel on stream_sync
+            e1.record()
+        torch.cuda.synchronize()
+        D.barrier(dev)
+        return e0.elapsed_time(e1) / 1e3, eng.launch_count() - n0
+
+    # ---- pass 1: the timed region (pipelined, nothing instrumented) -------------------------
+    eng = make(pipelined=True)
+    sampler = ClockSampler(local_rank if "CUDA_VISIBLE_DEVICES" not in os.environ else
+                           int(os.environ["CUDA_VISIBLE_DEVICES"].split(",")[local_rank]))
+    sampler.start()
+    secs, launches = timed(eng, args.steps, args.warmup)
+    clocks = sampler.stop()
+    value, worst = D.aggregate_throughput(step_bytes * args.steps / 1e9, secs, dev)
+
+    # ---- pass 2: same region with an event pair around every launch -> per-kernel durations --
+    eng.profile(True)
+    timed(eng, args.steps, 1)
+    n_acc, ms_acc = eng.kernel_stats(B.K_ACCUMULATE)
+    n_syn, ms_syn = eng.kernel_stats(B.K_SYNC)
+    eng.profile(False)
+    eng.destroy()
+
+    # ---- pass 3: eager mode (no overlap): each kernel class alone on the GPU ------------------
+    eng = make(pipelined=False)
+    eng.profile(True)
+    timed(eng, args.steps, args.warmup)
+    n_acc_e, ms_acc_e = eng.kernel_stats(B.K_ACCUMULATE)
+    n_syn_e, ms_syn_e = eng.kernel_stats(B.K_SYNC)
+    eng.destroy()
+
+    def roof(alg_bytes, n, ms, name, note):
+        ach = alg_bytes / (ms / n / 1e3) / 1e9 if n and ms > 0 else None
+        return {"kernel": name, "bound": "hbm", "achieved": ach, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                "frac": (ach / peaks["hbm_gbs"]) if ach else None, "peak_source": "of " + peaks["source"],
+                "frac_of_nominal_8TBs": (ach / HBM_NOMINAL_GBS) if ach else None,
+                "avg_us": ms / n * 1e3 if n else None, "launches": n, "traffic": None, "how": note}
+
+    per_acc = 12 * wl.P
+    roofline = roof(per_acc, n_acc, ms_acc, "k_accumulate_f32",
+                    "CUDA events around every launch on stream_acc inside the pipelined timed region")
+    roofline_sync = roof(sync_b, n_syn, ms_syn, "k_sync<4>",
+                         "CUDA events around every launch on stream_sync inside the pipelined timed region "
+                         "(shares HBM with concurrent accumulate kernels)")
+    isolated = {"accumulate": roof(per_acc, n_acc_e, ms_acc_e, "k_accumulate_f32", "eager mode, kernel alone on the GPU"),
+                "sync": roof(sync_b, n_syn_e, ms_syn_e, "k_sync<4>", "eager mode, kernel alone on the GPU")}
+
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+        "ms_per_step": worst / args.steps * 1e3, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "f32", "data": "synthetic",
+        "config": {"workload": "cfg2 resnet18-sized: P=11689512 (62 tensors), W=4, b=(2,2,4,8), lr=0.1 mu=0.9 wd=5e-4",
+                   "mode": "pipelined (two streams)", "l2": "inputs larger than L2: gradient pool 748 MB cycled, "
+                   "accumulators 374 MB", "parallelism": f"replicas x{world}", "bytes_per_step": step_bytes},
+        "frac_of_measured_hbm": value / world / peaks["hbm_gbs"],
+        "roofline": roofline, "roofline_sync": roofline_sync, "isolated": isolated,
+        "gpu_launches": launches, "clocks": clocks,
+    }
+
+    if rank == 0:
+        line["e2e"] = run_e2e(B, wlm, wl, x0_d, pool, order, step_bytes, min(args.steps, 10))
+        line["cpu_baseline"] = run_cpu_baseline(wlm, wl, x0, pool, order, step_bytes)
+        print(json.dumps(line), flush=True)
+    D.barrier(dev)
+    D.shutdown()
+
+
+def run_e2e(B, wlm, wl, x0_d, pool, order, step_bytes, steps):
+    """Same metric through the public API with HOST buffers: every step copies its 16 gradient
+    micro-batches from pinned host memory and reads the published parameters back."""
+    import torch
+
+    pool_h = torch.from_numpy(pool).pin_memory()
+    out_h = torch.empty(wl.P, dtype=torch.float32).pin_memory()
+    eng = B.AbsSgd(x0_d, wl.W, wl.lr, wl.momentum, wl.weight_decay, pipelined=True, host_input=True)
+    c = 0
+
+    def one():
+        nonlocal c
+        for (i, k) in order:
+            eng.accumulate_host(i, pool_h[c % wl.pool_size]); c += 1
+        eng.sync_step()
+        eng.params_host(out_h.numpy())
+
+    for _ in range(2):
+        one()
+    torch.cuda.synchronize()
+    t0 = time.perf_counter()
+    for _ in range(steps):
+        one()
+    torch.cuda.synchronize()
+    dt = time.perf_counter() - t0
+    eng.destroy()
+    return {"value": step_bytes * steps / dt / 1e9, "unit": UNIT, "ms_per_step": dt / steps * 1e3, "steps": steps,
+            "h2d_bytes_per_step": len(order) * wl.P * 4, "d2h_bytes_per_step": wl.P * 4,
+            "note": "PCIe-bound: 16 gradient vectors in, parameters out, every step"}
+
+
+def run_cpu_baseline(wlm, wl, x0, pool, order, step_bytes):
+    from oracle.c_oracle import AbsSgdOracleC
+
+    o = AbsSgdOracleC(x0, wl.W, wl.lr, wl.momentum, wl.weight_decay)
+    c = 0
+
+    def one():
+        nonlocal c
+        for (i, k) in order:
+            o.accumulate(i, pool[c % wl.pool_size]); c += 1
+        o.sync_step()
+
+    one()
+    t0 = time.perf_counter()
+    n = 0
+    while n < 40 and (time.perf_counter() - t0) < 15.0:
+        one(); n += 1
+    dt = time.perf_counter() - t0
+    o.close()
+    return {"value": step_bytes * n / dt / 1e9, "unit": UNIT, "cores": int(os.environ.get("OMP_NUM_THREADS", os.cpu_count() or 1)),
+            "kind": "oracle", "ms_per_step": dt / n * 1e3,
+            "sample": f"{n} full iterations of the same workload (C oracle, OpenMP, all host cores)"}
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    args = ap.parse_args()
+    if args.warmup < 3:
+        args.warmup = 3
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

@@ -1,0 +1,202 @@
+/*
+ * abs_sgd.h -- C ABI of the delayed synchronous step of ABS-SGD on one NVIDIA B200.
+ *
+ * Method: "A Delayed Synchronous SGD Algorithm with Adaptive Batch Size for Heterogeneous
+ * GPU Clusters", arXiv 2308.15164, Algorithm 1.  Paper <-> library notation:
+ *     N workers            = W          n parameters        = P
+ *     G_t^i (accumulated)  = acc[set][i] (fp32, length P)
+ *     M_t^i (batch size)   = b_i * M_r, b_i = number of abs_accumulate* calls of worker i
+ *     learning rate gamma  = lr         compensation lambda = lambda_dc
+ * The W workers of the paper are W gradient buffers in this GPU's memory, so the "global
+ * synchronization" of Step 1 is an in-device weighted reduction; no collective is involved.
+ *
+ * One iteration t (Algorithm 1, body of the while loop):
+ *     abs_accumulate*(worker i, ...)   any number of times per worker, in any order
+ *                                      (Step 2: G_t^i += g, M_t^i += M_r; the count is not
+ *                                       preset -- the library counts calls)
+ *     abs_sync_step()                  ends the iteration: the weighted average of the
+ *                                      DELAYED gradients  Gbar_{t-1} = sum_i G_{t-1}^i / sum_i b_i
+ *                                      (Step 1) is applied to x_t, giving x_{t+1}
+ *                                      ("Update parameters"); the consumed set is cleared
+ *                                      and becomes the target of iteration t+1.
+ * Update rule (momentum and weight decay extend the paper's plain SGD; with momentum =
+ * weight_decay = 0 it is exactly x_{t+1} = x_t - lr * Gtilde_t):
+ *     Gtilde = Gbar + lambda_dc * Gbar*Gbar*(x_t - x_{t-1})         (Eq. 6; lambda_dc = 0: off)
+ *     g = Gtilde + weight_decay * x ;  v = momentum * v + g ;  x = x - lr * v
+ * If sum_i b_i = 0 for the delayed set (always at t = 0, where G_{-1} = 0) the step leaves
+ * x and v untouched; buffers and counters still swap and t still advances.
+ *
+ * Conventions
+ *   - All functions return an int status (ABS_OK or a negative ABS_E* code); none aborts,
+ *     throws or blocks the host unless stated.  Argument errors are detected before any
+ *     GPU work is enqueued.
+ *   - "dev" pointers are device memory of the current CUDA device, "host" pointers host
+ *     memory.  The caller owns every buffer it passes in (workspace, gradients, x/y,
+ *     params0) and both streams; the context owns only host state and CUDA events.
+ *   - Work is enqueued on the streams given in abs_config and follows CUDA stream order:
+ *     an input buffer must stay valid and unchanged until the work enqueued by the call
+ *     that received it has completed.
+ *   - A context is not thread-safe; use one host thread per context.
+ */
+#ifndef ABS_SGD_H_
+#define ABS_SGD_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define ABS_OK        0
+#define ABS_EINVAL   (-1)  /* null / misaligned pointer, worker >= W, P = 0, W = 0 or > 64, bad dtype or flags */
+#define ABS_ESTATE   (-2)  /* context destroyed or never initialised                                          */
+#define ABS_ECUDA    (-3)  /* a CUDA runtime call failed; abs_last_error() gives the text                     */
+#define ABS_ENOMEM   (-4)  /* workspace smaller than abs_workspace_bytes()                                    */
+#define ABS_ETIMEOUT (-5)  /* a bounded device-side wait ran out                                              */
+
+#define ABS_GRAD_F32   0u  /* abs_accumulate takes fp32 gradients */
+#define ABS_GRAD_BF16  1u  /* abs_accumulate takes bf16 gradients (widened exactly to fp32) */
+
+#define ABS_FLAG_PIPELINED  1u  /* Step 1 of iteration t runs on stream_sync, concurrently with Step 2 of t+1 */
+#define ABS_FLAG_MLP        2u  /* the flat vector is a 2-layer MLP; enables abs_accumulate_mlp               */
+#define ABS_FLAG_HOST_INPUT 4u  /* reserve staging so abs_accumulate_host may be used                         */
+
+#define ABS_MAX_WORKERS 64u
+
+/* Kernel classes, for abs_kernel_stats() and abs_set_launch(). */
+#define ABS_K_ACCUMULATE 0   /* Step 2: acc += g                                        */
+#define ABS_K_SYNC       1   /* Step 1 + update: weighted reduce, momentum SGD, clear   */
+#define ABS_K_MLP_FWD    2   /* MLP: operand cast, forward GEMM, loss gradient          */
+#define ABS_K_MLP_BWD    3   /* MLP: layer-2 backward, dZ, bias gradients               */
+#define ABS_K_MLP_DW1    4   /* MLP: dW1 = X^T dZ on tcgen05, accumulated into acc      */
+#define ABS_K_COUNT      5
+
+typedef struct abs_ctx abs_ctx;   /* opaque; host memory owned by the library */
+
+typedef struct abs_config {
+    uint64_t P;               /* number of parameters n (> 0)                                         */
+    uint32_t W;               /* number of logical workers N (1..ABS_MAX_WORKERS)                     */
+    float lr;                 /* gamma                                                                */
+    float momentum;           /* mu; 0 = the paper's plain SGD                                        */
+    float weight_decay;       /* coupled L2; 0 = the paper's plain SGD                                */
+    float lambda_dc;          /* lambda of Eq. 6; 0 disables compensation                             */
+    uint32_t grad_dtype;      /* ABS_GRAD_F32 or ABS_GRAD_BF16: element type of abs_accumulate inputs */
+    uint32_t flags;           /* ABS_FLAG_*                                                           */
+    uint32_t mlp_in, mlp_hidden, mlp_out, mlp_mb;  /* with ABS_FLAG_MLP: layer sizes and samples per
+                                 micro-batch.  Flat layout: W1 [in,hidden] row-major, b1 [hidden],
+                                 W2 [hidden,out] row-major, b2 [out]; P must equal their total.
+                                 Limits: in % 128 == 0, hidden % 128 == 0, out <= 16, mb == 64.      */
+    void *stream_acc;         /* cudaStream_t for Step 2 work (accumulation); NULL = default stream   */
+    void *stream_sync;        /* cudaStream_t for Step 1 work when ABS_FLAG_PIPELINED; must then
+                                 differ from stream_acc                                               */
+} abs_config;
+
+/* Bytes of device workspace abs_init needs for this configuration (0 if cfg is invalid).
+ * Holds: parameters x (two copies when pipelined), momentum v, the double-buffered per-worker
+ * accumulators acc[2][W][P_pad] (P_pad = P rounded up to 256 elements), device counters,
+ * and the MLP / host-input scratch when those flags are set. */
+size_t abs_workspace_bytes(const abs_config *cfg);
+
+/* Algorithm 1, "Initialization": t = 0, G_{-1}^i = 0, x_0 = params0.
+ * workspace_dev: device memory, 256-byte aligned, >= abs_workspace_bytes(cfg); used until
+ * abs_destroy.  params0_dev: P fp32 values, copied in (stream-ordered on stream_acc).
+ * Errors: ABS_EINVAL (bad cfg/pointers), ABS_ENOMEM (workspace too small), ABS_ECUDA. */
+int abs_init(abs_ctx **out, const abs_config *cfg, void *workspace_dev, size_t workspace_bytes,
+             const float *params0_dev);
+
+/* Algorithm 1, Step 2 (one reference batch of worker `worker`): G_t^i += grad, b_i += 1.
+ * grad_dev: P contiguous elements of cfg.grad_dtype, 16-byte aligned, device memory; the
+ * gradient of a micro-batch is the MEAN over its M_r samples.  Enqueued on stream_acc. */
+int abs_accumulate(abs_ctx *ctx, uint32_t worker, const void *grad_dev);
+
+/* Same as abs_accumulate for a gradient in (preferably pinned) HOST memory: copies it to
+ * the device through an internal double-buffered staging area, then accumulates.  Needs
+ * ABS_FLAG_HOST_INPUT.  grad_host must stay valid until the copy has completed (the call
+ * may return earlier when the memory is pinned). */
+int abs_accumulate_host(abs_ctx *ctx, uint32_t worker, const void *grad_host);
+
+/* Algorithm 1, Step 2 with the gradient computed here: forward and backward pass of the
+ * 2-layer ReLU MLP with mean softmax cross-entropy on one micro-batch, evaluated at the
+ * current parameters x_t, and accumulated into worker `worker`'s buffer; b_i += 1.
+ * x_dev: [mlp_mb, mlp_in] fp32 row-major; y_dev: [mlp_mb] int32 class indices in
+ * [0, mlp_out).  GEMM operands are rounded to bf16 (nearest even) with fp32 accumulation;
+ * dW1 = X^T dZ runs on the tcgen05 tensor cores and its epilogue adds into the accumulator.
+ * Needs ABS_FLAG_MLP.  Enqueued on stream_acc. */
+int abs_accumulate_mlp(abs_ctx *ctx, uint32_t worker, const float *x_dev, const int32_t *y_dev);
+
+/* Algorithm 1, Step 1 + compensation + "Update parameters" + t = t + 1 (see the file header).
+ * Without ABS_FLAG_PIPELINED the fused kernel runs on stream_acc.  With it, the call makes
+ * x_{t+1} (computed by the kernel launched one call earlier on stream_sync) visible to
+ * stream_acc, and launches the kernel for the set just filled on stream_sync, so that it
+ * overlaps the accumulation of iteration t+1.  Both modes publish the same x_1, x_2, ...
+ * Never blocks the host. */
+int abs_sync_step(abs_ctx *ctx);
+
+/* Device pointer to the published parameters x_t (P fp32).  Work enqueued on stream_acc after
+ * this call sees x_t; the pointer is valid until the next abs_sync_step.  Does not block. */
+int abs_params(abs_ctx *ctx, const float **x_dev_out);
+
+/* Copy the published parameters x_t to host memory (P fp32); blocks until the copy is done. */
+int abs_params_host(abs_ctx *ctx, float *dst_host);
+
+/* Device pointer to the momentum buffer v (P fp32) as of the published parameters.  In
+ * pipelined mode v is being rewritten by the in-flight kernel; call abs_wait first. */
+int abs_momentum(abs_ctx *ctx, const float **v_dev_out);
+
+/* Device pointer to accumulator G^worker of set `set` (0 or 1), P fp32 (inspection / parity). */
+int abs_accumulator(abs_ctx *ctx, uint32_t set, uint32_t worker, const float **acc_dev_out);
+
+/* Logical state after the calls made so far (what Algorithm 1 holds at this point):
+ * cnt_host[2][W] = b_i of both sets, *cur = index of the set the current iteration fills,
+ * *t = iteration counter.  Host-side, never blocks.  Any output pointer may be NULL. */
+int abs_counters(abs_ctx *ctx, int32_t *cnt_host, uint32_t *cur, uint64_t *t);
+
+/* The b_i that sync step number `step` (0-based, < t, at most 63 steps back) consumed, as
+ * counted ON THE DEVICE by the accumulate kernels and logged by the fused kernel before it
+ * cleared them.  b_host[W].  Blocks until the logging kernel has finished. */
+int abs_consumed(abs_ctx *ctx, uint64_t step, int32_t *b_host);
+
+/* gamma may change between iterations (Theorem 1 allows gamma_t).  The rate travels with the
+ * gradients: the value in effect when abs_sync_step ends iteration t is the one used to apply
+ * that iteration's gradients, i.e. it is the paper's gamma_{t+1} (x_{t+2} = x_{t+1} - gamma_{t+1} *
+ * Gtilde_{t+1}).  Supplying it one iteration ahead is what lets Step 1 start the moment the
+ * iteration ends; eager and pipelined mode follow the same rule. */
+int abs_set_lr(abs_ctx *ctx, float lr);
+
+/* Make stream_acc wait (on the device, not the host) for every kernel launched on
+ * stream_sync so far.  Does not publish anything new. */
+int abs_wait(abs_ctx *ctx);
+
+/* Blocks until everything enqueued so far has finished and reports the device-side status:
+ * ABS_OK, ABS_ECUDA (a stream reported an error) or ABS_ETIMEOUT (a kernel gave up a bounded
+ * wait on an mbarrier; its output tile was not written). */
+int abs_check(abs_ctx *ctx);
+
+/* Launch shape of a kernel class: CTAs per SM for the persistent grid (0 = default, -1 = one
+ * tile per CTA).  For ABS_K_MLP_DW1 the value selects the epilogue instead: 0 = TMA load + add +
+ * TMA store of the accumulator tile, 1 = TMA reduce-add. */
+int abs_set_launch(abs_ctx *ctx, int kernel_class, int ctas_per_sm);
+
+/* Per-kernel timing with CUDA events on the launching stream.  abs_profile(ctx, 1) starts
+ * recording an event pair around every launch; abs_kernel_stats() blocks until recorded
+ * work has finished and returns the number of launches and their summed duration since
+ * profiling was switched on (or last reset by abs_profile(ctx, 1)). */
+int abs_profile(abs_ctx *ctx, int enable);
+int abs_kernel_stats(abs_ctx *ctx, int kernel_class, uint64_t *launches, double *total_ms);
+
+/* Number of kernels this context has launched since abs_init. */
+uint64_t abs_launch_count(abs_ctx *ctx);
+
+/* Text of the last error on this context (never NULL; "" if none).  ctx may be NULL: then
+ * the text of the last failed abs_init on this thread. */
+const char *abs_last_error(abs_ctx *ctx);
+
+/* Waits for the context's enqueued work, releases events and host state.  The workspace
+ * is the caller's to free afterwards.  Using ctx after this returns ABS_ESTATE. */
+int abs_destroy(abs_ctx *ctx);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* ABS_SGD_H_ */

@@ -1,0 +1,233 @@
+"""ctypes binding of the C ABI declared in include/abs_sgd.h.
+
+Argument marshalling only: every step of the delayed synchronous step runs in the CUDA
+kernels of libabs_sgd.so.  PyTorch is used for device memory and stream handles.  There is
+no CPU fallback: if the shared library is missing this module raises at import.
+"""
+
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import Optional
+
+import numpy as np
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libabs_sgd.so")
+
+if not os.path.exists(LIB_PATH):
+    raise ImportError(
+        f"{LIB_PATH} not found: build it with `python -m paper_2308_15164_b200.build` "
+        "(nvcc, sm_100a).  There is no CPU fallback.")
+
+lib = ctypes.CDLL(LIB_PATH)
+
+OK, EINVAL, ESTATE, ECUDA, ENOMEM, ETIMEOUT = 0, -1, -2, -3, -4, -5
+GRAD_F32, GRAD_BF16 = 0, 1
+FLAG_PIPELINED, FLAG_MLP, FLAG_HOST_INPUT = 1, 2, 4
+K_ACCUMULATE, K_SYNC, K_MLP_FWD, K_MLP_BWD, K_MLP_DW1 = range(5)
+KERNEL_NAMES = ["accumulate", "sync", "mlp_fwd", "mlp_bwd", "mlp_dw1"]
+
+
+class AbsConfig(ctypes.Structure):
+    _fields_ = [
+        ("P", ctypes.c_uint64), ("W", ctypes.c_uint32),
+        ("lr", ctypes.c_float), ("momentum", ctypes.c_float), ("weight_decay", ctypes.c_float),
+        ("lambda_dc", ctypes.c_float),
+        ("grad_dtype", ctypes.c_uint32), ("flags", ctypes.c_uint32),
+        ("mlp_in", ctypes.c_uint32), ("mlp_hidden", ctypes.c_uint32), ("mlp_out", ctypes.c_uint32),
+        ("mlp_mb", ctypes.c_uint32),
+        ("stream_acc", ctypes.c_void_p), ("stream_sync", ctypes.c_void_p),
+    ]
+
+
+_vp, _u32, _u64 = ctypes.c_void_p, ctypes.c_uint32, ctypes.c_uint64
+_sig = {
+    "abs_workspace_bytes": (ctypes.c_size_t, [ctypes.POINTER(AbsConfig)]),
+    "abs_init": (ctypes.c_int, [ctypes.POINTER(_vp), ctypes.POINTER(AbsConfig), _vp, ctypes.c_size_t, _vp]),
+    "abs_accumulate": (ctypes.c_int, [_vp, _u32, _vp]),
+    "abs_accumulate_host": (ctypes.c_int, [_vp, _u32, _vp]),
+    "abs_accumulate_mlp": (ctypes.c_int, [_vp, _u32, _vp, _vp]),
+    "abs_sync_step": (ctypes.c_int, [_vp]),
+    "abs_params": (ctypes.c_int, [_vp, ctypes.POINTER(_vp)]),
+    "abs_params_host": (ctypes.c_int, [_vp, _vp]),
+    "abs_momentum": (ctypes.c_int, [_vp, ctypes.POINTER(_vp)]),
+    "abs_accumulator": (ctypes.c_int, [_vp, _u32, _u32, ctypes.POINTER(_vp)]),
+    "abs_counters": (ctypes.c_int, [_vp, _vp, ctypes.POINTER(_u32), ctypes.POINTER(_u64)]),
+    "abs_consumed": (ctypes.c_int, [_vp, _u64, _vp]),
+    "abs_set_lr": (ctypes.c_int, [_vp, ctypes.c_float]),
+    "abs_wait": (ctypes.c_int, [_vp]),
+    "abs_check": (ctypes.c_int, [_vp]),
+    "abs_set_launch": (ctypes.c_int, [_vp, ctypes.c_int, ctypes.c_int]),
+    "abs_profile": (ctypes.c_int, [_vp, ctypes.c_int]),
+    "abs_kernel_stats": (ctypes.c_int, [_vp, ctypes.c_int, ctypes.POINTER(_u64), ctypes.POINTER(ctypes.c_double)]),
+    "abs_launch_count": (ctypes.c_uint64, [_vp]),
+    "abs_last_error": (ctypes.c_char_p, [_vp]),
+    "abs_destroy": (ctypes.c_int, [_vp]),
+}
+for _name, (_res, _args) in _sig.items():
+    _fn = getattr(lib, _name)
+    _fn.restype = _res
+    _fn.argtypes = _args
+
+
+class AbsError(RuntimeError):
+    def __init__(self, code, text):
+        super().__init__(f"abs_sgd status {code}: {text}")
+        self.code = code
+
+
+def _ptr(t) -> int:
+    """Raw address of a torch tensor / numpy array / int."""
+    if isinstance(t, torch.Tensor):
+        return t.data_ptr()
+    if isinstance(t, np.ndarray):
+        return t.ctypes.data
+    return int(t) if t is not None else 0
+
+
+def make_config(P, W, lr, momentum=0.0, weight_decay=0.0, lambda_dc=0.0, grad_dtype=GRAD_F32, flags=0,
+                mlp=None, stream_acc=0, stream_sync=0) -> AbsConfig:
+    c = AbsConfig()
+    c.P, c.W = int(P), int(W)
+    c.lr, c.momentum, c.weight_decay, c.lambda_dc = lr, momentum, weight_decay, lambda_dc
+    c.grad_dtype, c.flags = grad_dtype, flags
+    if mlp is not None:
+        c.mlp_in, c.mlp_hidden, c.mlp_out, c.mlp_mb = mlp
+    c.stream_acc, c.stream_sync = stream_acc or None, stream_sync or None
+    return c
+
+
+def abs_workspace_bytes(cfg: AbsConfig) -> int:
+    return int(lib.abs_workspace_bytes(ctypes.byref(cfg)))
+
+
+class AbsSgd:
+    """Thin object wrapper: one method per C entry point, same names without the ``abs_`` prefix."""
+
+    def __init__(self, params0: torch.Tensor, W: int, lr: float, momentum=0.0, weight_decay=0.0, lambda_dc=0.0,
+                 grad_dtype=GRAD_F32, pipelined=False, mlp=None, host_input=False,
+                 stream_acc: Optional[torch.cuda.Stream] = None, stream_sync: Optional[torch.cuda.Stream] = None):
+        assert params0.is_cuda and params0.dtype == torch.float32 and params0.is_contiguous()
+        self.device = params0.device
+        self.P, self.W = params0.numel(), W
+        self.stream_acc = stream_acc or torch.cuda.Stream(device=self.device)
+        self.stream_sync = stream_sync or (torch.cuda.Stream(device=self.device) if pipelined else None)
+        flags = (FLAG_PIPELINED if pipelined else 0) | (FLAG_MLP if mlp else 0) | (FLAG_HOST_INPUT if host_input else 0)
+        self.cfg = make_config(self.P, W, lr, momentum, weight_decay, lambda_dc, grad_dtype, flags, mlp,
+                               self.stream_acc.cuda_stream, self.stream_sync.cuda_stream if self.stream_sync else 0)
+        nbytes = abs_workspace_bytes(self.cfg)
+        if nbytes == 0:
+            raise AbsError(EINVAL, "invalid configuration")
+        self.workspace = torch.empty(nbytes, dtype=torch.uint8, device=self.device)
+        self._h = _vp()
+        # params0 may have been produced on another stream: make it visible to stream_acc.
+        self.stream_acc.wait_stream(torch.cuda.current_stream(self.device))
+        with torch.cuda.device(self.device):
+            rc = lib.abs_init(ctypes.byref(self._h), ctypes.byref(self.cfg), self.workspace.data_ptr(), nbytes,
+                              params0.data_ptr())
+        if rc != OK:
+            raise AbsError(rc, lib.abs_last_error(None).decode())
+        self._keep = params0
+
+    def _ck(self, rc):
+        if rc != OK:
+            raise AbsError(rc, lib.abs_last_error(self._h).decode())
+
+    def accumulate(self, worker: int, grad):
+        self._ck(lib.abs_accumulate(self._h, worker, _ptr(grad)))
+
+    def accumulate_host(self, worker: int, grad_host):
+        self._ck(lib.abs_accumulate_host(self._h, worker, _ptr(grad_host)))
+
+    def accumulate_mlp(self, worker: int, x, y):
+        self._ck(lib.abs_accumulate_mlp(self._h, worker, _ptr(x), _ptr(y)))
+
+    def sync_step(self):
+        self._ck(lib.abs_sync_step(self._h))
+
+    def params(self) -> torch.Tensor:
+        """The published parameters as a tensor aliasing library memory (valid until the next sync_step)."""
+        p = _vp()
+        self._ck(lib.abs_params(self._h, ctypes.byref(p)))
+        return _alias(p.value, self.P, torch.float32, self.device)
+
+    def params_host(self, out: Optional[np.ndarray] = None) -> np.ndarray:
+        if out is None:
+            out = np.empty(self.P, dtype=np.float32)
+        self._ck(lib.abs_params_host(self._h, _ptr(out)))
+        return out
+
+    def momentum(self) -> torch.Tensor:
+        p = _vp()
+        self._ck(lib.abs_momentum(self._h, ctypes.byref(p)))
+        return _alias(p.value, self.P, torch.float32, self.device)
+
+    def accumulator(self, set_index: int, worker: int) -> torch.Tensor:
+        p = _vp()
+        self._ck(lib.abs_accumulator(self._h, set_index, worker, ctypes.byref(p)))
+        return _alias(p.value, self.P, torch.float32, self.device)
+
+    def counters(self):
+        cnt = np.zeros((2, self.W), dtype=np.int32)
+        cur, t = _u32(0), _u64(0)
+        self._ck(lib.abs_counters(self._h, cnt.ctypes.data, ctypes.byref(cur), ctypes.byref(t)))
+        return cnt, int(cur.value), int(t.value)
+
+    def consumed(self, step: int) -> np.ndarray:
+        b = np.zeros(self.W, dtype=np.int32)
+        self._ck(lib.abs_consumed(self._h, step, b.ctypes.data))
+        return b
+
+    def set_lr(self, lr: float):
+        self._ck(lib.abs_set_lr(self._h, lr))
+
+    def wait(self):
+        self._ck(lib.abs_wait(self._h))
+
+    def check(self):
+        self._ck(lib.abs_check(self._h))
+
+    def set_launch(self, kernel_class: int, ctas_per_sm: int):
+        self._ck(lib.abs_set_launch(self._h, kernel_class, ctas_per_sm))
+
+    def profile(self, enable: bool):
+        self._ck(lib.abs_profile(self._h, int(enable)))
+
+    def kernel_stats(self, kernel_class: int):
+        n, ms = _u64(0), ctypes.c_double(0.0)
+        self._ck(lib.abs_kernel_stats(self._h, kernel_class, ctypes.byref(n), ctypes.byref(ms)))
+        return int(n.value), float(ms.value)
+
+    def launch_count(self) -> int:
+        return int(lib.abs_launch_count(self._h))
+
+    def synchronize(self):
+        self.stream_acc.synchronize()
+        if self.stream_sync is not None:
+            self.stream_sync.synchronize()
+
+    def destroy(self):
+        if self._h:
+            lib.abs_destroy(self._h)
+            self._h = _vp()
+
+    def __del__(self):
+        try:
+            self.destroy()
+        except Exception:
+            pass
+
+
+def _alias(addr: int, n: int, dtype, device) -> torch.Tensor:
+    """A tensor viewing ``n`` elements of library-owned device memory at ``addr`` (no copy)."""
+    itemsize = torch.empty(0, dtype=dtype).element_size()
+
+    class _Mem:
+        __cuda_array_interface__ = {
+            "shape": (n,), "typestr": {4: "<f4", 2: "<u2"}[itemsize], "data": (addr, False), "version": 2,
+        }
+
+    return torch.as_tensor(_Mem(), device=device)

@@ -1,0 +1,595 @@
+// Host side of the C ABI: state machine of Algorithm 1 (arXiv 2308.15164), workspace carving,
+// argument checks, stream ordering of Step 1 against Step 2, kernel launches.
+#include <cmath>
+#include <cstdio>
+#include <cstring>
+#include <mutex>
+#include <string>
+#include <unordered_set>
+#include <vector>
+
+#include "abs_internal.h"
+
+using namespace abs_sgd;
+
+namespace {
+
+constexpr uint32_t kMagic = 0xAB55D6D0u;
+
+struct TimedLaunch {
+    int kernel_class;
+    cudaEvent_t start, stop;
+};
+
+size_t round_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+
+struct Layout {
+    size_t P_pad = 0;
+    size_t off_x[2] = {0, 0}, off_v = 0, off_acc = 0, off_cnt = 0, off_ticket = 0, off_log = 0;
+    size_t off_shadow[2] = {0, 0}, off_mlp = 0, off_stage[2] = {0, 0};
+    size_t total = 0;
+};
+
+bool config_ok(const abs_config* c, std::string* why) {
+    auto fail = [&](const char* m) { if (why) *why = m; return false; };
+    if (!c) return fail("config is NULL");
+    if (c->P == 0) return fail("P must be > 0");
+    if (c->W == 0 || c->W > ABS_MAX_WORKERS) return fail("W must be in 1..64");
+    if (c->grad_dtype != ABS_GRAD_F32 && c->grad_dtype != ABS_GRAD_BF16) return fail("unknown grad_dtype");
+    if (c->flags & ~(ABS_FLAG_PIPELINED | ABS_FLAG_MLP | ABS_FLAG_HOST_INPUT)) return fail("unknown flag bits");
+    if (!std::isfinite(c->lr) || !std::isfinite(c->momentum) || !std::isfinite(c->weight_decay) ||
+        !std::isfinite(c->lambda_dc))
+        return fail("lr, momentum, weight_decay and lambda_dc must be finite");
+    if ((c->flags & ABS_FLAG_PIPELINED) && c->stream_acc == c->stream_sync)
+        return fail("pipelined mode needs two different streams");
+    if (c->flags & ABS_FLAG_MLP) {
+        if (c->mlp_in == 0 || c->mlp_in % 128 || c->mlp_hidden == 0 || c->mlp_hidden % 128)
+            return fail("mlp_in and mlp_hidden must be positive multiples of 128");
+        if (c->mlp_out == 0 || c->mlp_out > 16) return fail("mlp_out must be in 1..16");
+        if (c->mlp_mb != 64) return fail("mlp_mb must be 64");
+        const uint64_t need = (uint64_t)c->mlp_in * c->mlp_hidden + c->mlp_hidden +
+                              (uint64_t)c->mlp_hidden * c->mlp_out + c->mlp_out;
+        if (need != c->P) return fail("P does not match the MLP layer sizes");
+    }
+    return true;
+}
+
+Layout make_layout(const abs_config& c) {
+    Layout L;
+    L.P_pad = round_up(c.P, kPadElems);
+    const bool pipe = c.flags & ABS_FLAG_PIPELINED;
+    size_t o = 0;
+    auto take = [&](size_t bytes) { size_t at = o; o = round_up(o + bytes, 4096); return at; };
+    L.off_x[0] = take(L.P_pad * 4);
+    L.off_x[1] = pipe ? take(L.P_pad * 4) : L.off_x[0];
+    L.off_v = take(L.P_pad * 4);
+    L.off_acc = take((size_t)2 * c.W * L.P_pad * 4);
+    L.off_cnt = take((size_t)2 * kMaxW * 4);
+    L.off_ticket = take(256);
+    L.off_log = take((size_t)kLogDepth * kMaxW * 4);
+    if (c.flags & ABS_FLAG_MLP) {
+        L.off_shadow[0] = take(L.P_pad * 2);
+        L.off_shadow[1] = pipe ? take(L.P_pad * 2) : L.off_shadow[0];
+        MlpDims d{(int)c.mlp_in, (int)c.mlp_hidden, (int)c.mlp_out, (int)c.mlp_mb};
+        L.off_mlp = take(mlp_scratch_bytes(d));
+    }
+    if (c.flags & ABS_FLAG_HOST_INPUT) {
+        const size_t es = c.grad_dtype == ABS_GRAD_BF16 ? 2 : 4;
+        L.off_stage[0] = take(L.P_pad * es);
+        L.off_stage[1] = take(L.P_pad * es);
+    }
+    L.total = o;
+    return L;
+}
+
+std::mutex g_live_mu;
+std::unordered_set<abs_ctx*> g_live;
+thread_local std::string g_init_error;
+
+}  // namespace
+
+struct abs_ctx {
+    uint32_t magic = kMagic;
+    abs_config cfg{};
+    Layout L;
+    char* ws = nullptr;
+    cudaStream_t s_acc = nullptr, s_sync = nullptr, s_copy = nullptr;
+    bool pipelined = false, mlp = false;
+    int device = 0, num_sms = 148;
+
+    // logical state of Algorithm 1 (host mirror)
+    std::vector<int32_t> h_cnt;   // [2][W]
+    uint32_t cur = 0;
+    uint64_t t = 0;
+
+    // execution state
+    int pub = 0;                  // which x buffer holds the published parameters
+    bool pending = false;         // pipelined: a fused kernel launched on s_sync is not yet published
+    int pending_out = 0;          // buffer it writes
+    float lr_now = 0.f;
+    float lr_prev_call = 0.f;     // learning rate in effect at the previous abs_sync_step call
+    float disp_scale = 0.f;       // lr of the step that produced the newest x (0 after a no-op)
+    cudaEvent_t ev_acc_done = nullptr, ev_sync_done = nullptr, ev_aux = nullptr;
+    cudaEvent_t ev_stage_free[2] = {nullptr, nullptr}, ev_stage_full[2] = {nullptr, nullptr};
+    bool stage_used[2] = {false, false};
+    int stage_next = 0;
+    int ctas_per_sm[ABS_K_COUNT] = {0, 0, 0, 0, 0};
+    MlpDims mlp_dims{0, 0, 0, 0};
+    MlpScratch mlp_scratch{};
+    std::vector<TmapBytes> acc_tmaps;   // [2][W]: TMA descriptor of each accumulator row's W1 slice
+
+    // bookkeeping
+    uint64_t launches = 0;
+    bool profiling = false;
+    std::vector<TimedLaunch> timed;
+    std::vector<cudaEvent_t> ev_pool;
+    uint64_t stat_n[ABS_K_COUNT] = {0};
+    double stat_ms[ABS_K_COUNT] = {0};
+    std::string err;
+
+    float* x(int k) const { return reinterpret_cast<float*>(ws + L.off_x[k]); }
+    float* v() const { return reinterpret_cast<float*>(ws + L.off_v); }
+    float* acc(uint32_t set, uint32_t i) const {
+        return reinterpret_cast<float*>(ws + L.off_acc) + ((size_t)set * cfg.W + i) * L.P_pad;
+    }
+    int32_t* cnt(uint32_t set, uint32_t i) const { return reinterpret_cast<int32_t*>(ws + L.off_cnt) + set * kMaxW + i; }
+    unsigned int* ticket() const { return reinterpret_cast<unsigned int*>(ws + L.off_ticket); }
+    int32_t* log_row(uint64_t step) const {
+        return reinterpret_cast<int32_t*>(ws + L.off_log) + (step % kLogDepth) * kMaxW;
+    }
+    __nv_bfloat16* shadow(int k) const { return reinterpret_cast<__nv_bfloat16*>(ws + L.off_shadow[k]); }
+};
+
+namespace {
+
+bool live(abs_ctx* c) {
+    if (!c) return false;
+    std::lock_guard<std::mutex> g(g_live_mu);
+    return g_live.count(c) != 0 && c->magic == kMagic;
+}
+
+int cuda_fail(abs_ctx* c, cudaError_t e, const char* what) {
+    char buf[256];
+    snprintf(buf, sizeof buf, "%s: %s", what, cudaGetErrorString(e));
+    c->err = buf;
+    return ABS_ECUDA;
+}
+#define CK(call)                                                   \
+    do {                                                           \
+        cudaError_t e__ = (call);                                  \
+        if (e__ != cudaSuccess) return cuda_fail(c, e__, #call);   \
+    } while (0)
+
+int invalid(abs_ctx* c, const char* msg) {
+    c->err = msg;
+    return ABS_EINVAL;
+}
+
+cudaEvent_t take_event(abs_ctx* c) {
+    if (!c->ev_pool.empty()) {
+        cudaEvent_t e = c->ev_pool.back();
+        c->ev_pool.pop_back();
+        return e;
+    }
+    cudaEvent_t e = nullptr;
+    if (cudaEventCreate(&e) != cudaSuccess) return nullptr;
+    return e;
+}
+
+// Brackets a launch with an event pair when profiling is on.
+struct Timed {
+    abs_ctx* c;
+    cudaStream_t s;
+    cudaEvent_t stop = nullptr;
+    Timed(abs_ctx* c_, int kernel_class, cudaStream_t s_) : c(c_), s(s_) {
+        if (!c->profiling) return;
+        cudaEvent_t start = take_event(c);
+        stop = take_event(c);
+        if (!start || !stop) { stop = nullptr; return; }
+        cudaEventRecord(start, s);
+        c->timed.push_back({kernel_class, start, stop});
+    }
+    ~Timed() {
+        if (stop) cudaEventRecord(stop, s);
+    }
+};
+
+int collect_timings(abs_ctx* c) {
+    for (auto& tl : c->timed) {
+        CK(cudaEventSynchronize(tl.stop));
+        float ms = 0.f;
+        CK(cudaEventElapsedTime(&ms, tl.start, tl.stop));
+        c->stat_n[tl.kernel_class] += 1;
+        c->stat_ms[tl.kernel_class] += ms;
+        c->ev_pool.push_back(tl.start);
+        c->ev_pool.push_back(tl.stop);
+    }
+    c->timed.clear();
+    return ABS_OK;
+}
+
+void mlp_mark(void* user, int kernel_class, int n);
+
+// Launch the fused Step-1 kernel on `set`, reading x[in] and writing x[out], on `stream`.
+int launch_fused(abs_ctx* c, uint32_t set, int in, int out, uint64_t log_step, cudaStream_t stream) {
+    SyncArgs a{};
+    a.x_in = c->x(in);
+    a.x_out = c->x(out);
+    a.v = c->v();
+    a.acc = c->acc(set, 0);
+    a.row_stride = c->L.P_pad;
+    a.n_vec = c->L.P_pad / 4;
+    a.W = (int)c->cfg.W;
+    a.cnt = c->cnt(set, 0);
+    a.log_row = c->log_row(log_step);
+    a.ticket = c->ticket();
+    a.lr = c->lr_now;
+    a.mu = c->cfg.momentum;
+    a.wd = c->cfg.weight_decay;
+    a.lambda_dc = c->cfg.lambda_dc;
+    a.disp_scale = c->disp_scale;
+    a.shadow = c->mlp ? c->shadow(out) : nullptr;
+    {
+        Timed tm(c, ABS_K_SYNC, stream);
+        CK(launch_sync(a, c->ctas_per_sm[ABS_K_SYNC], c->num_sms, stream));
+    }
+    c->launches += 1;
+    return ABS_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+size_t abs_workspace_bytes(const abs_config* cfg) {
+    if (!config_ok(cfg, nullptr)) return 0;
+    return make_layout(*cfg).total;
+}
+
+int abs_init(abs_ctx** out, const abs_config* cfg, void* workspace_dev, size_t workspace_bytes,
+             const float* params0_dev) {
+    g_init_error.clear();
+    if (!out) { g_init_error = "out is NULL"; return ABS_EINVAL; }
+    *out = nullptr;
+    std::string why;
+    if (!config_ok(cfg, &why)) { g_init_error = why; return ABS_EINVAL; }
+    if (!workspace_dev || (reinterpret_cast<uintptr_t>(workspace_dev) & 255)) {
+        g_init_error = "workspace must be non-NULL and 256-byte aligned";
+        return ABS_EINVAL;
+    }
+    if (!params0_dev || (reinterpret_cast<uintptr_t>(params0_dev) & 15)) {
+        g_init_error = "params0 must be non-NULL and 16-byte aligned";
+        return ABS_EINVAL;
+    }
+    Layout L = make_layout(*cfg);
+    if (workspace_bytes < L.total) { g_init_error = "workspace too small"; return ABS_ENOMEM; }
+
+    abs_ctx* c = new abs_ctx();
+    c->cfg = *cfg;
+    c->L = L;
+    c->ws = static_cast<char*>(workspace_dev);
+    c->s_acc = static_cast<cudaStream_t>(cfg->stream_acc);
+    c->s_sync = static_cast<cudaStream_t>(cfg->stream_sync);
+    c->pipelined = cfg->flags & ABS_FLAG_PIPELINED;
+    c->mlp = cfg->flags & ABS_FLAG_MLP;
+    c->h_cnt.assign((size_t)2 * cfg->W, 0);
+    c->lr_now = cfg->lr;
+    c->lr_prev_call = cfg->lr;
+
+    auto bail = [&](cudaError_t e, const char* what) {
+        cuda_fail(c, e, what);
+        g_init_error = c->err;
+        delete c;
+        return ABS_ECUDA;
+    };
+    cudaError_t e;
+    if ((e = cudaGetDevice(&c->device)) != cudaSuccess) return bail(e, "cudaGetDevice");
+    if ((e = cudaDeviceGetAttribute(&c->num_sms, cudaDevAttrMultiProcessorCount, c->device)) != cudaSuccess)
+        return bail(e, "cudaDeviceGetAttribute");
+    if ((e = cudaEventCreateWithFlags(&c->ev_acc_done, cudaEventDisableTiming)) != cudaSuccess) return bail(e, "cudaEventCreate");
+    if ((e = cudaEventCreateWithFlags(&c->ev_sync_done, cudaEventDisableTiming)) != cudaSuccess) return bail(e, "cudaEventCreate");
+    if ((e = cudaEventCreateWithFlags(&c->ev_aux, cudaEventDisableTiming)) != cudaSuccess) return bail(e, "cudaEventCreate");
+    if (cfg->flags & ABS_FLAG_HOST_INPUT) {
+        if ((e = cudaStreamCreateWithFlags(&c->s_copy, cudaStreamNonBlocking)) != cudaSuccess) return bail(e, "cudaStreamCreate");
+        for (int k = 0; k < 2; ++k) {
+            if ((e = cudaEventCreateWithFlags(&c->ev_stage_free[k], cudaEventDisableTiming)) != cudaSuccess) return bail(e, "cudaEventCreate");
+            if ((e = cudaEventCreateWithFlags(&c->ev_stage_full[k], cudaEventDisableTiming)) != cudaSuccess) return bail(e, "cudaEventCreate");
+        }
+    }
+
+    // Algorithm 1, Initialization: G_{-1}^i = 0, counters 0, v = 0, x_0 = params0.
+    const size_t state_bytes = L.off_log + (size_t)kLogDepth * kMaxW * 4;
+    if ((e = cudaMemsetAsync(c->ws, 0, state_bytes, c->s_acc)) != cudaSuccess) return bail(e, "cudaMemsetAsync");
+    if ((e = cudaMemcpyAsync(c->x(0), params0_dev, cfg->P * 4, cudaMemcpyDeviceToDevice, c->s_acc)) != cudaSuccess)
+        return bail(e, "cudaMemcpyAsync(params0)");
+    if (c->mlp) {
+        c->mlp_dims = MlpDims{(int)cfg->mlp_in, (int)cfg->mlp_hidden, (int)cfg->mlp_out, (int)cfg->mlp_mb};
+        const char* msg = nullptr;
+        if ((e = cudaMemsetAsync(c->ws + L.off_shadow[0], 0, L.P_pad * 2, c->s_acc)) != cudaSuccess) return bail(e, "cudaMemsetAsync");
+        if (c->pipelined && (e = cudaMemsetAsync(c->ws + L.off_shadow[1], 0, L.P_pad * 2, c->s_acc)) != cudaSuccess)
+            return bail(e, "cudaMemsetAsync");
+        if ((e = mlp_scratch_init(&c->mlp_scratch, c->mlp_dims, c->ws + L.off_mlp, &msg)) != cudaSuccess)
+            return bail(e, msg ? msg : "mlp_scratch_init");
+        if ((e = cudaMemsetAsync(c->mlp_scratch.status, 0, sizeof(int), c->s_acc)) != cudaSuccess) return bail(e, "cudaMemsetAsync");
+        c->acc_tmaps.resize((size_t)2 * cfg->W);
+        for (uint32_t set = 0; set < 2; ++set)
+            for (uint32_t i = 0; i < cfg->W; ++i)
+                if ((e = mlp_make_acc_tmap(&c->acc_tmaps[(size_t)set * cfg->W + i], c->mlp_dims, c->acc(set, i))) != cudaSuccess)
+                    return bail(e, "cuTensorMapEncodeTiled(accumulator)");
+        if ((e = launch_cast_bf16(c->x(0), c->shadow(0), L.P_pad, c->num_sms, c->s_acc)) != cudaSuccess)
+            return bail(e, "launch_cast_bf16");
+        c->launches += 1;
+    }
+    if (c->pipelined) {   // stream_sync must not start before the state is initialised
+        if ((e = cudaEventRecord(c->ev_aux, c->s_acc)) != cudaSuccess) return bail(e, "cudaEventRecord");
+        if ((e = cudaStreamWaitEvent(c->s_sync, c->ev_aux, 0)) != cudaSuccess) return bail(e, "cudaStreamWaitEvent");
+    }
+    {
+        std::lock_guard<std::mutex> g(g_live_mu);
+        g_live.insert(c);
+    }
+    *out = c;
+    return ABS_OK;
+}
+
+int abs_accumulate(abs_ctx* c, uint32_t worker, const void* grad_dev) {
+    if (!live(c)) return ABS_ESTATE;
+    if (worker >= c->cfg.W) return invalid(c, "worker index out of range");
+    if (!grad_dev || (reinterpret_cast<uintptr_t>(grad_dev) & 15)) return invalid(c, "gradient pointer must be non-NULL and 16-byte aligned");
+    {
+        Timed tm(c, ABS_K_ACCUMULATE, c->s_acc);
+        CK(launch_accumulate(c->acc(c->cur, worker), grad_dev, c->cfg.grad_dtype, c->cfg.P, c->cnt(c->cur, worker),
+                             c->ctas_per_sm[ABS_K_ACCUMULATE], c->num_sms, c->s_acc));
+    }
+    c->launches += 1;
+    c->h_cnt[(size_t)c->cur * c->cfg.W + worker] += 1;
+    return ABS_OK;
+}
+
+int abs_accumulate_host(abs_ctx* c, uint32_t worker, const void* grad_host) {
+    if (!live(c)) return ABS_ESTATE;
+    if (!(c->cfg.flags & ABS_FLAG_HOST_INPUT)) return invalid(c, "context was created without ABS_FLAG_HOST_INPUT");
+    if (worker >= c->cfg.W) return invalid(c, "worker index out of range");
+    if (!grad_host) return invalid(c, "gradient pointer is NULL");
+    const int k = c->stage_next;
+    c->stage_next ^= 1;
+    const size_t es = c->cfg.grad_dtype == ABS_GRAD_BF16 ? 2 : 4;
+    void* stage = c->ws + c->L.off_stage[k];
+    // The copy of micro-batch n+1 overlaps the accumulate kernel of micro-batch n.
+    if (c->stage_used[k]) CK(cudaStreamWaitEvent(c->s_copy, c->ev_stage_free[k], 0));
+    CK(cudaMemcpyAsync(stage, grad_host, c->cfg.P * es, cudaMemcpyHostToDevice, c->s_copy));
+    CK(cudaEventRecord(c->ev_stage_full[k], c->s_copy));
+    CK(cudaStreamWaitEvent(c->s_acc, c->ev_stage_full[k], 0));
+    {
+        Timed tm(c, ABS_K_ACCUMULATE, c->s_acc);
+        CK(launch_accumulate(c->acc(c->cur, worker), stage, c->cfg.grad_dtype, c->cfg.P, c->cnt(c->cur, worker),
+                             c->ctas_per_sm[ABS_K_ACCUMULATE], c->num_sms, c->s_acc));
+    }
+    CK(cudaEventRecord(c->ev_stage_free[k], c->s_acc));
+    c->stage_used[k] = true;
+    c->launches += 1;
+    c->h_cnt[(size_t)c->cur * c->cfg.W + worker] += 1;
+    return ABS_OK;
+}
+
+int abs_accumulate_mlp(abs_ctx* c, uint32_t worker, const float* x_dev, const int32_t* y_dev) {
+    if (!live(c)) return ABS_ESTATE;
+    if (!c->mlp) return invalid(c, "context was created without ABS_FLAG_MLP");
+    if (worker >= c->cfg.W) return invalid(c, "worker index out of range");
+    if (!x_dev || (reinterpret_cast<uintptr_t>(x_dev) & 15)) return invalid(c, "x pointer must be non-NULL and 16-byte aligned");
+    if (!y_dev || (reinterpret_cast<uintptr_t>(y_dev) & 3)) return invalid(c, "y pointer must be non-NULL and 4-byte aligned");
+    CK(launch_mlp_grad(c->mlp_dims, c->mlp_scratch, c->x(c->pub), c->shadow(c->pub), x_dev, y_dev,
+                       c->acc(c->cur, worker), &c->acc_tmaps[(size_t)c->cur * c->cfg.W + worker], c->cnt(c->cur, worker),
+                       c->ctas_per_sm[ABS_K_MLP_DW1], c->s_acc, mlp_mark, c));
+    c->h_cnt[(size_t)c->cur * c->cfg.W + worker] += 1;
+    return ABS_OK;
+}
+
+int abs_sync_step(abs_ctx* c) {
+    if (!live(c)) return ABS_ESTATE;
+    const uint32_t W = c->cfg.W;
+    const uint32_t d = c->cur ^ 1;   // the delayed set (filled during iteration t-1)
+    if (!c->pipelined) {
+        // Step 1 on the delayed set, in place, on stream_acc.
+        int64_t B = 0;
+        for (uint32_t i = 0; i < W; ++i) B += c->h_cnt[(size_t)d * W + i];
+        if (B > 0) {
+            // The learning rate travels with the gradients: the delayed set is applied with the
+            // rate that was in effect when its iteration ended (same rule as pipelined mode,
+            // where that kernel was already launched one call ago).
+            const float lr_call = c->lr_now;
+            c->lr_now = c->lr_prev_call;
+            int rc = launch_fused(c, d, c->pub, c->pub, c->t, c->s_acc);
+            c->lr_now = lr_call;
+            if (rc != ABS_OK) return rc;
+            c->disp_scale = c->lr_prev_call;
+        } else {
+            CK(cudaMemsetAsync(c->log_row(c->t), 0, kMaxW * 4, c->s_acc));
+            c->disp_scale = 0.f;
+        }
+    } else {
+        // Publish x_{t+1}: the kernel launched one call ago (on the set of iteration t-1).
+        if (c->pending) {
+            CK(cudaStreamWaitEvent(c->s_acc, c->ev_sync_done, 0));
+            c->pub = c->pending_out;
+            c->pending = false;
+        }
+        // Launch Step 1 for the set just filled (iteration t); it is published by the next call.
+        int64_t B = 0;
+        for (uint32_t i = 0; i < W; ++i) B += c->h_cnt[(size_t)c->cur * W + i];
+        CK(cudaEventRecord(c->ev_acc_done, c->s_acc));
+        CK(cudaStreamWaitEvent(c->s_sync, c->ev_acc_done, 0));
+        if (B > 0) {
+            const int out = c->pub ^ 1;
+            int rc = launch_fused(c, c->cur, c->pub, out, c->t + 1, c->s_sync);
+            if (rc != ABS_OK) return rc;
+            c->disp_scale = c->lr_now;
+            c->pending_out = out;
+        } else {
+            CK(cudaMemsetAsync(c->log_row(c->t + 1), 0, kMaxW * 4, c->s_sync));
+            c->disp_scale = 0.f;
+            c->pending_out = c->pub;
+        }
+        CK(cudaEventRecord(c->ev_sync_done, c->s_sync));
+        c->pending = true;
+    }
+    // Logical state (Algorithm 1: clear the consumed set, swap roles, t = t + 1).
+    for (uint32_t i = 0; i < W; ++i) c->h_cnt[(size_t)d * W + i] = 0;
+    c->lr_prev_call = c->lr_now;
+    c->cur = d;
+    c->t += 1;
+    return ABS_OK;
+}
+
+int abs_params(abs_ctx* c, const float** x_dev_out) {
+    if (!live(c)) return ABS_ESTATE;
+    if (!x_dev_out) return invalid(c, "output pointer is NULL");
+    *x_dev_out = c->x(c->pub);
+    return ABS_OK;
+}
+
+int abs_params_host(abs_ctx* c, float* dst_host) {
+    if (!live(c)) return ABS_ESTATE;
+    if (!dst_host) return invalid(c, "destination pointer is NULL");
+    CK(cudaMemcpyAsync(dst_host, c->x(c->pub), c->cfg.P * 4, cudaMemcpyDeviceToHost, c->s_acc));
+    CK(cudaStreamSynchronize(c->s_acc));
+    return ABS_OK;
+}
+
+int abs_momentum(abs_ctx* c, const float** v_dev_out) {
+    if (!live(c)) return ABS_ESTATE;
+    if (!v_dev_out) return invalid(c, "output pointer is NULL");
+    *v_dev_out = c->v();
+    return ABS_OK;
+}
+
+int abs_accumulator(abs_ctx* c, uint32_t set, uint32_t worker, const float** acc_dev_out) {
+    if (!live(c)) return ABS_ESTATE;
+    if (set > 1 || worker >= c->cfg.W || !acc_dev_out) return invalid(c, "bad set / worker / output pointer");
+    *acc_dev_out = c->acc(set, worker);
+    return ABS_OK;
+}
+
+int abs_counters(abs_ctx* c, int32_t* cnt_host, uint32_t* cur, uint64_t* t) {
+    if (!live(c)) return ABS_ESTATE;
+    if (cnt_host) memcpy(cnt_host, c->h_cnt.data(), c->h_cnt.size() * sizeof(int32_t));
+    if (cur) *cur = c->cur;
+    if (t) *t = c->t;
+    return ABS_OK;
+}
+
+int abs_consumed(abs_ctx* c, uint64_t step, int32_t* b_host) {
+    if (!live(c)) return ABS_ESTATE;
+    if (!b_host) return invalid(c, "output pointer is NULL");
+    if (step >= c->t || c->t - step >= (uint64_t)kLogDepth) return invalid(c, "step is not in the logged window");
+    if (c->pipelined) CK(cudaStreamSynchronize(c->s_sync));
+    CK(cudaStreamSynchronize(c->s_acc));
+    CK(cudaMemcpy(b_host, c->log_row(step), c->cfg.W * sizeof(int32_t), cudaMemcpyDeviceToHost));
+    return ABS_OK;
+}
+
+int abs_set_lr(abs_ctx* c, float lr) {
+    if (!live(c)) return ABS_ESTATE;
+    if (!std::isfinite(lr)) return invalid(c, "lr must be finite");
+    c->lr_now = lr;
+    return ABS_OK;
+}
+
+int abs_wait(abs_ctx* c) {
+    if (!live(c)) return ABS_ESTATE;
+    if (c->pipelined) {
+        CK(cudaEventRecord(c->ev_aux, c->s_sync));
+        CK(cudaStreamWaitEvent(c->s_acc, c->ev_aux, 0));
+    }
+    return ABS_OK;
+}
+
+int abs_check(abs_ctx* c) {
+    if (!live(c)) return ABS_ESTATE;
+    if (c->pipelined) CK(cudaStreamSynchronize(c->s_sync));
+    CK(cudaStreamSynchronize(c->s_acc));
+    if (c->mlp) {
+        int st = 0;
+        CK(cudaMemcpy(&st, c->mlp_scratch.status, sizeof(int), cudaMemcpyDeviceToHost));
+        if (st != 0) {
+            c->err = "a bounded device-side wait ran out (MLP dW1 kernel)";
+            return ABS_ETIMEOUT;
+        }
+    }
+    return ABS_OK;
+}
+
+int abs_set_launch(abs_ctx* c, int kernel_class, int ctas_per_sm) {
+    if (!live(c)) return ABS_ESTATE;
+    if (kernel_class < 0 || kernel_class >= ABS_K_COUNT || ctas_per_sm < -1 || ctas_per_sm > 64)
+        return invalid(c, "bad kernel class or CTA count");
+    c->ctas_per_sm[kernel_class] = ctas_per_sm;
+    return ABS_OK;
+}
+
+int abs_profile(abs_ctx* c, int enable) {
+    if (!live(c)) return ABS_ESTATE;
+    int rc = collect_timings(c);
+    if (rc != ABS_OK) return rc;
+    if (enable) {
+        for (int k = 0; k < ABS_K_COUNT; ++k) { c->stat_n[k] = 0; c->stat_ms[k] = 0.0; }
+    }
+    c->profiling = enable != 0;
+    return ABS_OK;
+}
+
+int abs_kernel_stats(abs_ctx* c, int kernel_class, uint64_t* launches, double* total_ms) {
+    if (!live(c)) return ABS_ESTATE;
+    if (kernel_class < 0 || kernel_class >= ABS_K_COUNT) return invalid(c, "bad kernel class");
+    int rc = collect_timings(c);
+    if (rc != ABS_OK) return rc;
+    if (launches) *launches = c->stat_n[kernel_class];
+    if (total_ms) *total_ms = c->stat_ms[kernel_class];
+    return ABS_OK;
+}
+
+uint64_t abs_launch_count(abs_ctx* c) { return live(c) ? c->launches : 0; }
+
+const char* abs_last_error(abs_ctx* c) {
+    if (!c) return g_init_error.c_str();
+    if (!live(c)) return "context is not alive";
+    return c->err.c_str();
+}
+
+int abs_destroy(abs_ctx* c) {
+    if (!live(c)) return ABS_ESTATE;
+    {
+        std::lock_guard<std::mutex> g(g_live_mu);
+        g_live.erase(c);
+    }
+    cudaStreamSynchronize(c->s_acc);
+    if (c->pipelined) cudaStreamSynchronize(c->s_sync);
+    if (c->s_copy) { cudaStreamSynchronize(c->s_copy); cudaStreamDestroy(c->s_copy); }
+    for (auto& tl : c->timed) { cudaEventDestroy(tl.start); cudaEventDestroy(tl.stop); }
+    for (auto e : c->ev_pool) cudaEventDestroy(e);
+    for (cudaEvent_t e : {c->ev_acc_done, c->ev_sync_done, c->ev_aux, c->ev_stage_free[0], c->ev_stage_free[1],
+                          c->ev_stage_full[0], c->ev_stage_full[1]})
+        if (e) cudaEventDestroy(e);
+    c->magic = 0;
+    delete c;
+    return ABS_OK;
+}
+
+}  // extern "C"
+
+namespace {
+// Called by the MLP launcher around each group of its kernels: n = 0 before, n = launches made after.
+void mlp_mark(void* user, int kernel_class, int n) {
+    abs_ctx* c = static_cast<abs_ctx*>(user);
+    c->launches += (uint64_t)n;
+    if (!c->profiling) return;
+    if (n == 0) {
+        cudaEvent_t start = take_event(c), stop = take_event(c);
+        if (!start || !stop) return;
+        cudaEventRecord(start, c->s_acc);
+        c->timed.push_back({kernel_class, start, stop});
+    } else if (!c->timed.empty() && c->timed.back().kernel_class == kernel_class) {
+        cudaEventRecord(c->timed.back().stop, c->s_acc);
+    }
+}
+}  // namespace

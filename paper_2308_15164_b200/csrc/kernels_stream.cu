@@ -1,0 +1,323 @@
+// Streaming kernels of the delayed synchronous step (arXiv 2308.15164, Algorithm 1).
+//
+//   k_accumulate_*  Step 2:  G_t^i += g ;  b_i += 1
+//   k_sync          Step 1 + Eq. 6 + "Update parameters", fused:
+//                     B = sum_i b_i ;  Gbar = (sum_i G_{t-1}^i) / B ;  compensation ;
+//                     g = Gbar + wd*x ; v = mu*v + g ; x' = x - lr*v ;
+//                     G_{t-1}^i <- 0 ; b_i <- 0 (after logging them)
+//
+// Both are pure HBM streams (about 1 flop per 4 bytes), so the design goal is bytes in flight:
+// 128-bit accesses, several independent loads per thread issued before the first use, a grid
+// that is a multiple of the SM count, and one pass over every byte (each accumulator element is
+// read once and overwritten with zero by the same thread that read it).
+#include "abs_internal.h"
+
+namespace abs_sgd {
+
+namespace {
+
+constexpr int kBlock = 256;
+
+// Read-once global loads: bypass L1, mark evict-first in L2.
+__device__ __forceinline__ float4 ld_stream(const float4* p) {
+    float4 r;
+    asm volatile("ld.global.cs.v4.f32 {%0,%1,%2,%3}, [%4];" : "=f"(r.x), "=f"(r.y), "=f"(r.z), "=f"(r.w) : "l"(p));
+    return r;
+}
+__device__ __forceinline__ uint4 ld_stream(const uint4* p) {
+    uint4 r;
+    asm volatile("ld.global.cs.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(r.x), "=r"(r.y), "=r"(r.z), "=r"(r.w) : "l"(p));
+    return r;
+}
+__device__ __forceinline__ void st_stream(float4* p, float4 v) {
+    asm volatile("st.global.cs.v4.f32 [%0], {%1,%2,%3,%4};" ::"l"(p), "f"(v.x), "f"(v.y), "f"(v.z), "f"(v.w) : "memory");
+}
+__device__ __forceinline__ float bf16_lo(uint32_t w) { return __uint_as_float(w << 16); }
+__device__ __forceinline__ float bf16_hi(uint32_t w) { return __uint_as_float(w & 0xFFFF0000u); }
+
+// ------------------------------------------------------------------------------------------
+// Step 2, fp32 gradient: 12 bytes per parameter (read g, read acc, write acc).
+// ------------------------------------------------------------------------------------------
+template <int U>
+__global__ void __launch_bounds__(kBlock) k_accumulate_f32(float* acc, const float* __restrict__ g,
+                                                           unsigned long long n_vec, unsigned long long P,
+                                                           int32_t* cnt) {
+    float4* acc4 = reinterpret_cast<float4*>(acc);
+    const float4* g4 = reinterpret_cast<const float4*>(g);
+    const unsigned long long tile = (unsigned long long)kBlock * U;
+    for (unsigned long long base = blockIdx.x * tile; base < n_vec; base += gridDim.x * tile) {
+        float4 a[U], b[U];
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            const unsigned long long idx = base + (unsigned long long)u * kBlock + threadIdx.x;
+            if (idx < n_vec) {
+                b[u] = ld_stream(g4 + idx);
+                a[u] = acc4[idx];
+            }
+        }
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            const unsigned long long idx = base + (unsigned long long)u * kBlock + threadIdx.x;
+            if (idx < n_vec) {
+                a[u].x += b[u].x; a[u].y += b[u].y; a[u].z += b[u].z; a[u].w += b[u].w;
+                acc4[idx] = a[u];
+            }
+        }
+    }
+    if (blockIdx.x == 0) {
+        const unsigned long long j = n_vec * 4 + threadIdx.x;   // ragged tail (P % 4 elements)
+        if (j < P) acc[j] += g[j];
+        if (threadIdx.x == 0) cnt[0] += 1;                      // M_t^i += M_r
+    }
+}
+
+// ------------------------------------------------------------------------------------------
+// Step 2, bf16 gradient: 10 bytes per parameter.  One 128-bit load carries 8 gradients.
+// ------------------------------------------------------------------------------------------
+template <int U>
+__global__ void __launch_bounds__(kBlock) k_accumulate_bf16(float* acc, const uint16_t* __restrict__ g,
+                                                            unsigned long long n_vec8, unsigned long long P,
+                                                            int32_t* cnt) {
+    float4* acc4 = reinterpret_cast<float4*>(acc);
+    const uint4* g8 = reinterpret_cast<const uint4*>(g);
+    const unsigned long long tile = (unsigned long long)kBlock * U;
+    for (unsigned long long base = blockIdx.x * tile; base < n_vec8; base += gridDim.x * tile) {
+        float4 a0[U], a1[U];
+        uint4 b[U];
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            const unsigned long long idx = base + (unsigned long long)u * kBlock + threadIdx.x;
+            if (idx < n_vec8) {
+                b[u] = ld_stream(g8 + idx);
+                a0[u] = acc4[2 * idx];
+                a1[u] = acc4[2 * idx + 1];
+            }
+        }
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            const unsigned long long idx = base + (unsigned long long)u * kBlock + threadIdx.x;
+            if (idx < n_vec8) {
+                a0[u].x += bf16_lo(b[u].x); a0[u].y += bf16_hi(b[u].x);
+                a0[u].z += bf16_lo(b[u].y); a0[u].w += bf16_hi(b[u].y);
+                a1[u].x += bf16_lo(b[u].z); a1[u].y += bf16_hi(b[u].z);
+                a1[u].z += bf16_lo(b[u].w); a1[u].w += bf16_hi(b[u].w);
+                acc4[2 * idx] = a0[u];
+                acc4[2 * idx + 1] = a1[u];
+            }
+        }
+    }
+    if (blockIdx.x == 0) {
+        const unsigned long long j = n_vec8 * 8 + threadIdx.x;  // ragged tail (P % 8 elements)
+        if (j < P) acc[j] += __uint_as_float((uint32_t)g[j] << 16);
+        if (threadIdx.x == 0) cnt[0] += 1;
+    }
+}
+
+// ------------------------------------------------------------------------------------------
+// Step 1 + update, fused.  (8*W_act + 16) bytes per parameter, W_act = #{i : b_i > 0}:
+// read W_act accumulators + x + v, write x' + v + W_act zeros.  Rows of idle workers
+// (b_i = 0) are neither read nor rewritten.  WT > 0: W known at compile time (all loads of a
+// vector are issued before the first add); WT == 0: any W, in chunks of 8 rows.
+// ------------------------------------------------------------------------------------------
+__device__ __forceinline__ void update_vec(float4& x, float4& v, const float4 s, const float Bf,
+                                           const SyncArgs& a) {
+    float gx = __fdiv_rn(s.x, Bf), gy = __fdiv_rn(s.y, Bf), gz = __fdiv_rn(s.z, Bf), gw = __fdiv_rn(s.w, Bf);
+    if (a.lambda_dc != 0.0f) {   // Eq. 6 with x_t - x_{t-1} = -disp_scale * v
+        const float c = -a.lambda_dc * a.disp_scale;
+        gx += c * gx * gx * v.x; gy += c * gy * gy * v.y; gz += c * gz * gz * v.z; gw += c * gw * gw * v.w;
+    }
+    gx += a.wd * x.x; gy += a.wd * x.y; gz += a.wd * x.z; gw += a.wd * x.w;
+    v.x = a.mu * v.x + gx; v.y = a.mu * v.y + gy; v.z = a.mu * v.z + gz; v.w = a.mu * v.w + gw;
+    x.x -= a.lr * v.x; x.y -= a.lr * v.y; x.z -= a.lr * v.z; x.w -= a.lr * v.w;
+}
+
+__device__ __forceinline__ void store_shadow(__nv_bfloat16* shadow, unsigned long long idx, const float4 x) {
+    __nv_bfloat162 lo = __floats2bfloat162_rn(x.x, x.y);
+    __nv_bfloat162 hi = __floats2bfloat162_rn(x.z, x.w);
+    uint2 pk;
+    pk.x = *reinterpret_cast<uint32_t*>(&lo);
+    pk.y = *reinterpret_cast<uint32_t*>(&hi);
+    reinterpret_cast<uint2*>(shadow)[idx] = pk;
+}
+
+template <int WT, int U>
+__global__ void __launch_bounds__(kBlock) k_sync(const SyncArgs a) {
+    __shared__ int s_cnt[kMaxW];
+    const int W = WT > 0 ? WT : a.W;
+    if (threadIdx.x < W) s_cnt[threadIdx.x] = a.cnt[threadIdx.x];
+    __syncthreads();
+    long long B = 0;
+    unsigned long long active = 0;
+    for (int i = 0; i < W; ++i) {
+        B += s_cnt[i];
+        if (s_cnt[i] > 0) active |= 1ull << i;
+    }
+    const float Bf = (float)B;
+
+    const float4* xin = reinterpret_cast<const float4*>(a.x_in);
+    float4* xout = reinterpret_cast<float4*>(a.x_out);
+    float4* v4 = reinterpret_cast<float4*>(a.v);
+    float4* acc4 = reinterpret_cast<float4*>(a.acc);
+    const unsigned long long rs = a.row_stride / 4;
+    const float4 zero = make_float4(0.f, 0.f, 0.f, 0.f);
+    const unsigned long long tile = (unsigned long long)kBlock * U;
+
+    if (B > 0) {
+        for (unsigned long long base = blockIdx.x * tile; base < a.n_vec; base += gridDim.x * tile) {
+            if constexpr (WT > 0) {
+                float4 r[U][WT], x[U], v[U];
+#pragma unroll
+                for (int u = 0; u < U; ++u) {
+                    const unsigned long long idx = base + (unsigned long long)u * kBlock + threadIdx.x;
+                    if (idx < a.n_vec) {
+#pragma unroll
+                        for (int i = 0; i < WT; ++i)
+                            if ((active >> i) & 1) r[u][i] = ld_stream(acc4 + i * rs + idx);
+                        x[u] = ld_stream(xin + idx);
+                        v[u] = ld_stream(v4 + idx);
+                    }
+                }
+#pragma unroll
+                for (int u = 0; u < U; ++u) {
+                    const unsigned long long idx = base + (unsigned long long)u * kBlock + threadIdx.x;
+                    if (idx < a.n_vec) {
+                        float4 s = zero;
+#pragma unroll
+                        for (int i = 0; i < WT; ++i)      // fixed worker order
+                            if ((active >> i) & 1) {
+                                s.x += r[u][i].x; s.y += r[u][i].y; s.z += r[u][i].z; s.w += r[u][i].w;
+                            }
+                        update_vec(x[u], v[u], s, Bf, a);
+                        st_stream(xout + idx, x[u]);
+                        st_stream(v4 + idx, v[u]);
+                        if (a.shadow) store_shadow(a.shadow, idx, x[u]);
+#pragma unroll
+                        for (int i = 0; i < WT; ++i)
+                            if ((active >> i) & 1) st_stream(acc4 + i * rs + idx, zero);
+                    }
+                }
+            } else {
+                const unsigned long long idx = base + threadIdx.x;   // U == 1 in the generic path
+                if (idx < a.n_vec) {
+                    float4 x = ld_stream(xin + idx), v = ld_stream(v4 + idx);
+                    float4 s = zero;
+                    for (int i0 = 0; i0 < W; i0 += 8) {
+                        float4 r[8];
+#pragma unroll
+                        for (int c = 0; c < 8; ++c)
+                            if (i0 + c < W && ((active >> (i0 + c)) & 1)) r[c] = ld_stream(acc4 + (i0 + c) * rs + idx);
+#pragma unroll
+                        for (int c = 0; c < 8; ++c)
+                            if (i0 + c < W && ((active >> (i0 + c)) & 1)) {
+                                s.x += r[c].x; s.y += r[c].y; s.z += r[c].z; s.w += r[c].w;
+                                st_stream(acc4 + (i0 + c) * rs + idx, zero);
+                            }
+                    }
+                    update_vec(x, v, s, Bf, a);
+                    st_stream(xout + idx, x);
+                    st_stream(v4 + idx, v);
+                    if (a.shadow) store_shadow(a.shadow, idx, x);
+                }
+            }
+        }
+    } else if (a.x_out != a.x_in) {
+        // Nothing to apply (sum_i b_i = 0): x_{t+1} = x_t, v unchanged.  The host normally
+        // skips the launch in this case; kept so the kernel is correct on its own.
+        for (unsigned long long idx = blockIdx.x * (unsigned long long)kBlock + threadIdx.x; idx < a.n_vec;
+             idx += (unsigned long long)gridDim.x * kBlock) {
+            const float4 x = xin[idx];
+            xout[idx] = x;
+            if (a.shadow) store_shadow(a.shadow, idx, x);
+        }
+    }
+
+    // The last CTA to finish logs the consumed b_i and clears the device counters (every CTA
+    // read them before taking its ticket).
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        __threadfence();
+        const unsigned int t = atomicAdd(a.ticket, 1u);
+        if (t == gridDim.x - 1) {
+            for (int i = 0; i < W; ++i) {
+                a.log_row[i] = s_cnt[i];
+                a.cnt[i] = 0;
+            }
+            *a.ticket = 0u;
+        }
+    }
+}
+
+__global__ void __launch_bounds__(kBlock) k_cast_bf16(const float4* __restrict__ src, __nv_bfloat16* dst,
+                                                      unsigned long long n_vec) {
+    for (unsigned long long idx = blockIdx.x * (unsigned long long)kBlock + threadIdx.x; idx < n_vec;
+         idx += (unsigned long long)gridDim.x * kBlock)
+        store_shadow(dst, idx, src[idx]);
+}
+
+inline unsigned grid_for(unsigned long long n_items, int per_cta, int ctas_per_sm, int num_sms) {
+    unsigned long long tiles = (n_items + per_cta - 1) / per_cta;
+    if (tiles == 0) tiles = 1;
+    if (ctas_per_sm > 0) {
+        const unsigned long long cap = (unsigned long long)ctas_per_sm * num_sms;
+        if (tiles > cap) tiles = cap;
+    }
+    if (tiles > 0x7FFFFFFFull) tiles = 0x7FFFFFFFull;
+    return (unsigned)tiles;
+}
+
+template <int WT, int U>
+cudaError_t launch_sync_t(const SyncArgs& a, int ctas_per_sm, int num_sms, cudaStream_t stream) {
+    const unsigned grid = grid_for(a.n_vec, kBlock * U, ctas_per_sm, num_sms);
+    k_sync<WT, U><<<grid, kBlock, 0, stream>>>(a);
+    return cudaGetLastError();
+}
+
+}  // namespace
+
+cudaError_t launch_accumulate(float* acc_row, const void* g, uint32_t grad_dtype, size_t P, int32_t* cnt,
+                              int ctas_per_sm, int num_sms, cudaStream_t stream) {
+    constexpr int U = 4;
+    if (ctas_per_sm == 0) ctas_per_sm = 8;
+    if (grad_dtype == ABS_GRAD_F32) {
+        const unsigned long long n_vec = P / 4;
+        const unsigned grid = grid_for(n_vec, kBlock * U, ctas_per_sm, num_sms);
+        k_accumulate_f32<U><<<grid, kBlock, 0, stream>>>(acc_row, static_cast<const float*>(g), n_vec, P, cnt);
+    } else {
+        const unsigned long long n_vec8 = P / 8;
+        const unsigned grid = grid_for(n_vec8, kBlock * U, ctas_per_sm, num_sms);
+        k_accumulate_bf16<U><<<grid, kBlock, 0, stream>>>(acc_row, static_cast<const uint16_t*>(g), n_vec8, P, cnt);
+    }
+    return cudaGetLastError();
+}
+
+cudaError_t launch_sync(const SyncArgs& a, int ctas_per_sm, int num_sms, cudaStream_t stream) {
+    if (ctas_per_sm == 0) ctas_per_sm = 4;
+    switch (a.W) {
+        case 1: return launch_sync_t<1, 4>(a, ctas_per_sm, num_sms, stream);
+        case 2: return launch_sync_t<2, 4>(a, ctas_per_sm, num_sms, stream);
+        case 3: return launch_sync_t<3, 2>(a, ctas_per_sm, num_sms, stream);
+        case 4: return launch_sync_t<4, 2>(a, ctas_per_sm, num_sms, stream);
+        case 5: return launch_sync_t<5, 2>(a, ctas_per_sm, num_sms, stream);
+        case 6: return launch_sync_t<6, 2>(a, ctas_per_sm, num_sms, stream);
+        case 7: return launch_sync_t<7, 1>(a, ctas_per_sm, num_sms, stream);
+        case 8: return launch_sync_t<8, 1>(a, ctas_per_sm, num_sms, stream);
+        case 9: return launch_sync_t<9, 1>(a, ctas_per_sm, num_sms, stream);
+        case 10: return launch_sync_t<10, 1>(a, ctas_per_sm, num_sms, stream);
+        case 11: return launch_sync_t<11, 1>(a, ctas_per_sm, num_sms, stream);
+        case 12: return launch_sync_t<12, 1>(a, ctas_per_sm, num_sms, stream);
+        case 13: return launch_sync_t<13, 1>(a, ctas_per_sm, num_sms, stream);
+        case 14: return launch_sync_t<14, 1>(a, ctas_per_sm, num_sms, stream);
+        case 15: return launch_sync_t<15, 1>(a, ctas_per_sm, num_sms, stream);
+        case 16: return launch_sync_t<16, 1>(a, ctas_per_sm, num_sms, stream);
+        default: return launch_sync_t<0, 1>(a, ctas_per_sm, num_sms, stream);
+    }
+}
+
+cudaError_t launch_cast_bf16(const float* src, __nv_bfloat16* dst, size_t n, int num_sms, cudaStream_t stream) {
+    const unsigned long long n_vec = n / 4;
+    const unsigned grid = grid_for(n_vec, kBlock, 8, num_sms);
+    k_cast_bf16<<<grid, kBlock, 0, stream>>>(reinterpret_cast<const float4*>(src), dst, n_vec);
+    return cudaGetLastError();
+}
+
+}  // namespace abs_sgd
