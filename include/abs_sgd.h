@@ -54,6 +54,7 @@ extern "C" {
 #define ABS_ECUDA    (-3)  /* a CUDA runtime call failed; abs_last_error() gives the text                     */
 #define ABS_ENOMEM   (-4)  /* workspace smaller than abs_workspace_bytes()                                    */
 #define ABS_ETIMEOUT (-5)  /* a bounded device-side wait ran out                                              */
+#define ABS_ELIMIT   (-6)  /* a size exceeds a fixed built-in capacity (abs_sync_step_noalloc: W > 64)        */
 
 #define ABS_GRAD_F32   0u  /* abs_accumulate takes fp32 gradients */
 #define ABS_GRAD_BF16  1u  /* abs_accumulate takes bf16 gradients (widened exactly to fp32) */
@@ -195,6 +196,39 @@ const char *abs_last_error(abs_ctx *ctx);
 /* Waits for the context's enqueued work, releases events and host state.  The workspace
  * is the caller's to free afterwards.  Using ctx after this returns ABS_ESTATE. */
 int abs_destroy(abs_ctx *ctx);
+
+/* One fused sync step on buffers the CALLER owns, for callers that cannot allocate device
+ * memory.  (No counterpart in the paper: this is a packaging variant of the kernel behind
+ * abs_sync_step, not another algorithm step.)
+ *
+ * Meant for code that runs inside someone else's memory budget -- an extension under a
+ * framework that already reserved the GPU for its own pool, a job whose device memory was
+ * carved up front, a loop that cannot afford the device-wide synchronisation of cudaMalloc /
+ * cudaFree.  The call itself allocates nothing, on the host or on the device: the few words of
+ * working memory the kernel needs (its CTA ticket and the log of consumed counts) live in a
+ * 1 KiB array built into the library, which every GPU that loads the library holds until the
+ * process exits.
+ *
+ * Computes, in place and on `stream`:  B = sum_i cnt[i];  if B > 0:
+ *     Gbar = (sum_{i: cnt[i]>0} acc[i]) / B ;  g = Gbar + weight_decay*x ;  v = momentum*v + g ;
+ *     x = x - lr*v ;  acc[i] = 0 for every i with cnt[i] > 0 ;
+ * then cnt[i] = 0 for all i.  (No compensation term, no bf16 shadow.)
+ *   x_dev, v_dev   P fp32 each, 16-byte aligned, updated in place
+ *   acc_dev        W rows of fp32, row i at acc_dev + i*row_stride, 16-byte aligned
+ *   row_stride, P  in elements; both multiples of 4, row_stride >= P
+ *   cnt_dev        W int32 device counters b_i (input, cleared on output)
+ *   stream         cudaStream_t (NULL = default stream)
+ * Limit: W <= 64 (what the built-in working memory can log); larger W returns ABS_ELIMIT and
+ * nothing is launched.  Other bad arguments return ABS_EINVAL, CUDA failures ABS_ECUDA.
+ *
+ * The first call on each device looks up the device address of the built-in array (one
+ * cudaGetSymbolAddress, no allocation); make that first call outside any stream capture.
+ * All calls on a device share the array and it keeps the previous call's contents (the call
+ * clears the word that must start at zero), so two calls whose kernels may overlap on the GPU
+ * -- different streams without an ordering between them -- race on it: order them. */
+int abs_sync_step_noalloc(float *x_dev, float *v_dev, float *acc_dev, uint64_t row_stride, uint64_t P,
+                          uint32_t W, int32_t *cnt_dev, float lr, float momentum, float weight_decay,
+                          void *stream);
 
 #ifdef __cplusplus
 }

@@ -24,7 +24,7 @@ if not os.path.exists(LIB_PATH):
 
 lib = ctypes.CDLL(LIB_PATH)
 
-OK, EINVAL, ESTATE, ECUDA, ENOMEM, ETIMEOUT = 0, -1, -2, -3, -4, -5
+OK, EINVAL, ESTATE, ECUDA, ENOMEM, ETIMEOUT, ELIMIT = 0, -1, -2, -3, -4, -5, -6
 GRAD_F32, GRAD_BF16 = 0, 1
 FLAG_PIPELINED, FLAG_MLP, FLAG_HOST_INPUT = 1, 2, 4
 K_ACCUMULATE, K_SYNC, K_MLP_FWD, K_MLP_BWD, K_MLP_DW1 = range(5)
@@ -66,6 +66,8 @@ _sig = {
     "abs_launch_count": (ctypes.c_uint64, [_vp]),
     "abs_last_error": (ctypes.c_char_p, [_vp]),
     "abs_destroy": (ctypes.c_int, [_vp]),
+    "abs_sync_step_noalloc": (ctypes.c_int, [_vp, _vp, _vp, _u64, _u64, _u32, _vp, ctypes.c_float, ctypes.c_float,
+                                             ctypes.c_float, _vp]),
 }
 for _name, (_res, _args) in _sig.items():
     _fn = getattr(lib, _name)
@@ -219,6 +221,15 @@ class AbsSgd:
             self.destroy()
         except Exception:
             pass
+
+
+def sync_step_noalloc(x: torch.Tensor, v: torch.Tensor, acc: torch.Tensor, cnt: torch.Tensor, lr: float,
+                      momentum: float = 0.0, weight_decay: float = 0.0, stream: Optional[torch.cuda.Stream] = None) -> int:
+    """abs_sync_step_noalloc on caller-owned tensors: x, v fp32 [P]; acc fp32 [W, row_stride]; cnt int32 [W].
+    Returns the status code (no exception), so callers can test for ELIMIT / EINVAL."""
+    s = stream.cuda_stream if stream is not None else torch.cuda.current_stream(x.device).cuda_stream
+    return int(lib.abs_sync_step_noalloc(x.data_ptr(), v.data_ptr(), acc.data_ptr(), acc.stride(0), x.numel(),
+                                         acc.shape[0], cnt.data_ptr(), lr, momentum, weight_decay, s))
 
 
 def _alias(addr: int, n: int, dtype, device) -> torch.Tensor:
