@@ -265,11 +265,72 @@ def run_ours(args):
     }
 
     if rank == 0:
-        line["e2e"] = run_e2e(B, wlm, wl, x0_d, pool, order, step_bytes, min(args.steps, 10))
-        line["cpu_baseline"] = run_cpu_baseline(wlm, wl, x0, pool, order, step_bytes)
+        sections = args.sections.split(",")
+        if "e2e" in sections:
+            line["e2e"] = run_e2e(B, wlm, wl, x0_d, pool, order, step_bytes, min(args.steps, 10))
+        if "cpu" in sections:
+            line["cpu_baseline"] = run_cpu_baseline(wlm, wl, x0, pool, order, step_bytes)
+        del pool_d
+        torch.cuda.empty_cache()
+        if "mlp" in sections:
+            line["mlp"] = run_mlp(B, wlm, dev, peaks)
         print(json.dumps(line), flush=True)
     D.barrier(dev)
     D.shutdown()
+
+
+def run_mlp(B, wlm, dev, peaks, iters=12):
+    """Secondary measurement on the MLP workload (3072-4096-10, W=4, b_i ~ U{1..8}): per-kernel-class
+    durations of the micro-batch gradient, and the dW1 = X^T dZ GEMM (M=3072, N=4096, K=64) as TFLOP/s
+    and as HBM GB/s -- with K = 64 it is bound by the read-modify-write of the fp32 accumulator slice."""
+    import torch
+
+    wl = wlm.config(4, T=iters)
+    d = wl.mlp
+    x0_d = torch.from_numpy(wlm.params0(wl)).to(dev)
+    xs, ys = wlm.mlp_batches(wl)
+    xs_d, ys_d = torch.from_numpy(xs).to(dev), torch.from_numpy(ys).to(dev)
+    torch.cuda.synchronize()
+    out = {"workload": "cfg4 mlp 3072-4096-10, mb=64, W=4, b_i~U{1..8}, pipelined", "iterations": iters}
+    for name, epi in (("tma_load_add_store", 0), ("tma_reduce_add", 1)):
+        eng = B.AbsSgd(x0_d, wl.W, wl.lr, wl.momentum, wl.weight_decay, pipelined=True, mlp=(d.d_in, d.d_hidden, d.d_out, d.mb))
+        eng.set_launch(B.K_MLP_DW1, epi)
+        calls = list(wlm.iter_calls(wl))
+
+        def run(profile):
+            eng.profile(profile)
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            n = 0
+            with torch.cuda.stream(eng.stream_acc):
+                e0.record()
+                for it in calls:
+                    for (i, k, c) in it:
+                        eng.accumulate_mlp(i, xs_d[c % wl.mlp_pool], ys_d[c % wl.mlp_pool]); n += 1
+                    eng.sync_step()
+                eng.wait()
+                e1.record()
+            torch.cuda.synchronize()
+            return e0.elapsed_time(e1), n
+
+        run(False)                                  # warm-up
+        ms_total, n_mb = run(False)
+        run(True)
+        stats = {nm: eng.kernel_stats(k) for nm, k in (("fwd", B.K_MLP_FWD), ("bwd", B.K_MLP_BWD), ("dw1", B.K_MLP_DW1), ("sync", B.K_SYNC))}
+        eng.check()
+        eng.destroy()
+        n_dw, ms_dw = stats["dw1"]
+        us_dw = ms_dw / n_dw * 1e3
+        flop = 2.0 * d.d_in * d.d_hidden * d.mb
+        rmw_bytes = 8.0 * d.d_in * d.d_hidden + 2.0 * d.mb * (d.d_in + d.d_hidden)
+        out[name] = {
+            "us_per_microbatch_all_kernels": ms_total / n_mb * 1e3,
+            "us_fwd": stats["fwd"][1] / max(stats["fwd"][0], 1) * 1e3, "us_bwd": stats["bwd"][1] / max(stats["bwd"][0], 1) * 1e3,
+            "us_dw1": us_dw, "us_sync": stats["sync"][1] / max(stats["sync"][0], 1) * 1e3,
+            "dw1_tflops": flop / us_dw / 1e6, "dw1_frac_of_bf16_peak_sustained": flop / us_dw / 1e6 / peaks["bf16_tflops_sustained"],
+            "dw1_hbm_gbs": rmw_bytes / us_dw / 1e3, "dw1_frac_of_hbm": rmw_bytes / us_dw / 1e3 / peaks["hbm_gbs"],
+            "microbatches": n_mb,
+        }
+    return out
 
 
 def run_e2e(B, wlm, wl, x0_d, pool, order, step_bytes, steps):
@@ -330,9 +391,11 @@ def run_cpu_baseline(wlm, wl, x0, pool, order, step_bytes):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--steps", type=int, default=1000)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--sections", default="e2e,cpu,mlp",
+                    help="extra measurements after the timed region (drop them for a profiler's launch list)")
     args = ap.parse_args()
     if args.warmup < 3:
         args.warmup = 3

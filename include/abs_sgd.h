@@ -175,8 +175,9 @@ int abs_wait(abs_ctx *ctx);
 int abs_check(abs_ctx *ctx);
 
 /* Launch shape of a kernel class: CTAs per SM for the persistent grid (0 = default, -1 = one
- * tile per CTA).  For ABS_K_MLP_DW1 the value selects the epilogue instead: 0 = TMA load + add +
- * TMA store of the accumulator tile, 1 = TMA reduce-add. */
+ * tile per CTA).  For ABS_K_MLP_DW1 the value is a bit mask of MLP kernel variants instead:
+ * bit 0 = dW1 epilogue by TMA reduce-add (default: TMA load + add + TMA store of the accumulator
+ * tile); bit 1 = forward GEMM on CUDA cores (default: tcgen05).  Results agree within rounding. */
 int abs_set_launch(abs_ctx *ctx, int kernel_class, int ctas_per_sm);
 
 /* Per-kernel timing with CUDA events on the launching stream.  abs_profile(ctx, 1) starts

@@ -308,7 +308,7 @@ int abs_init(abs_ctx** out, const abs_config* cfg, void* workspace_dev, size_t w
         if ((e = cudaMemsetAsync(c->ws + L.off_shadow[0], 0, L.P_pad * 2, c->s_acc)) != cudaSuccess) return bail(e, "cudaMemsetAsync");
         if (c->pipelined && (e = cudaMemsetAsync(c->ws + L.off_shadow[1], 0, L.P_pad * 2, c->s_acc)) != cudaSuccess)
             return bail(e, "cudaMemsetAsync");
-        if ((e = mlp_scratch_init(&c->mlp_scratch, c->mlp_dims, c->ws + L.off_mlp, &msg)) != cudaSuccess)
+        if ((e = mlp_scratch_init(&c->mlp_scratch, c->mlp_dims, c->ws + L.off_mlp, c->shadow(0), c->shadow(1), &msg)) != cudaSuccess)
             return bail(e, msg ? msg : "mlp_scratch_init");
         if ((e = cudaMemsetAsync(c->mlp_scratch.status, 0, sizeof(int), c->s_acc)) != cudaSuccess) return bail(e, "cudaMemsetAsync");
         c->acc_tmaps.resize((size_t)2 * cfg->W);
@@ -378,7 +378,7 @@ int abs_accumulate_mlp(abs_ctx* c, uint32_t worker, const float* x_dev, const in
     if (worker >= c->cfg.W) return invalid(c, "worker index out of range");
     if (!x_dev || (reinterpret_cast<uintptr_t>(x_dev) & 15)) return invalid(c, "x pointer must be non-NULL and 16-byte aligned");
     if (!y_dev || (reinterpret_cast<uintptr_t>(y_dev) & 3)) return invalid(c, "y pointer must be non-NULL and 4-byte aligned");
-    CK(launch_mlp_grad(c->mlp_dims, c->mlp_scratch, c->x(c->pub), c->shadow(c->pub), x_dev, y_dev,
+    CK(launch_mlp_grad(c->mlp_dims, c->mlp_scratch, c->x(c->pub), c->shadow(c->pub), c->pub, x_dev, y_dev,
                        c->acc(c->cur, worker), &c->acc_tmaps[(size_t)c->cur * c->cfg.W + worker], c->cnt(c->cur, worker),
                        c->ctas_per_sm[ABS_K_MLP_DW1], c->s_acc, mlp_mark, c));
     c->h_cnt[(size_t)c->cur * c->cfg.W + worker] += 1;

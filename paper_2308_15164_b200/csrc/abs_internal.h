@@ -58,20 +58,23 @@ struct MlpScratch {      // device pointers carved from the workspace (all hidde
     float* dl;           // [mb][16]              dL (fp32)
     __nv_bfloat16* dlb;  // [mb][16]              bf16(dL)
     int* status;         // device status word: ABS_ETIMEOUT if a bounded wait ran out
-    TmapBytes tmap_xt, tmap_dzt;
+    TmapBytes tmap_xt, tmap_dzt;   // dW1 operands
+    TmapBytes tmap_xb, tmap_w1[2]; // forward GEMM operands (W1 of each bf16 shadow copy)
 };
 size_t mlp_scratch_bytes(const MlpDims& d);
 // Lays the scratch out at `base` (1024-B aligned) and encodes the operand TMA descriptors (host call).
-cudaError_t mlp_scratch_init(MlpScratch* s, const MlpDims& d, void* base, const char** err);
+cudaError_t mlp_scratch_init(MlpScratch* s, const MlpDims& d, void* base, __nv_bfloat16* shadow0,
+                             __nv_bfloat16* shadow1, const char** err);
 // TMA descriptor of the W1 slice of one worker's accumulator row (fp32 [d_in][d_hidden]).
 cudaError_t mlp_make_acc_tmap(void* tmap_out, const MlpDims& d, float* acc_row);
 // Enqueues the whole micro-batch gradient; adds into acc_row (flat MLP layout) and bumps cnt.
 // shadow: bf16 copy of the published parameters (same flat layout).  x_pub: the fp32 parameters.
-// epilogue: 0 = TMA load + add + TMA store, 1 = TMA reduce-add.
+// shadow_idx: which of the two shadow copies `shadow` is.  variant: bit 0 = dW1 epilogue by TMA reduce-add
+// (else TMA load + add + TMA store); bit 1 = forward GEMM on CUDA cores (cross-check of the tcgen05 one).
 // mark(user, kernel_class, 0) is called before a kernel group, mark(user, kernel_class, n) after n launches.
 cudaError_t launch_mlp_grad(const MlpDims& d, const MlpScratch& s, const float* x_pub,
-                            const __nv_bfloat16* shadow, const float* x_dev, const int32_t* y_dev,
-                            float* acc_row, const void* acc_tmap, int32_t* cnt, int epilogue, cudaStream_t stream,
+                            const __nv_bfloat16* shadow, int shadow_idx, const float* x_dev, const int32_t* y_dev,
+                            float* acc_row, const void* acc_tmap, int32_t* cnt, int variant, cudaStream_t stream,
                             void (*mark)(void* user, int kernel_class, int n), void* user);
 
 }  // namespace abs_sgd

@@ -15,7 +15,8 @@
 //
 // Kernels (all on the caller's stream):
 //   k_cast_x      X fp32 -> bf16 in both orientations
-//   k_fwd1        Z^T partials = W1^T X^T, split over d_in
+//   k_fwd1_tcgen05  Z^T partials = W1^T X^T, split over d_in, on tcgen05 (W1 as an MN-major operand)
+//   (k_fwd1         the same on CUDA cores, kept as a cross-check selectable through abs_set_launch)
 //   k_fwd2        Z = sum of partials + b1, gate, bf16(H), per-chunk partial logits
 //   k_loss        logits, softmax, dL, db2 += ...
 //   k_bwd         dH, dZ, db1 += ..., dW2 += ..., bf16(dZ)^T, b_i += 1
@@ -69,7 +70,7 @@ __global__ void __launch_bounds__(256) k_fwd1(const __nv_bfloat16* __restrict__ 
     __shared__ float sx[KT][64 + 4];   // [k][r]
     const int h0 = blockIdx.x * 64;
     const int s = blockIdx.y;
-    const int k_per = d_in / kSplitK;
+    const int k_per = d_in / (int)gridDim.y;
     const int kbeg = s * k_per, kend = kbeg + k_per;
     const int th = threadIdx.x / 16, tr = threadIdx.x % 16;   // 16 x 16 threads, 4 h x 4 r each
     float acc[4][4] = {};
@@ -112,7 +113,7 @@ __global__ void __launch_bounds__(256) k_fwd1(const __nv_bfloat16* __restrict__ 
 __global__ void __launch_bounds__(256) k_fwd2(const float* __restrict__ zpart, const float* __restrict__ b1,
                                               const __nv_bfloat16* __restrict__ w2b, float* __restrict__ zt,
                                               __nv_bfloat16* __restrict__ hbt, float* __restrict__ lpart, int d_h,
-                                              int d_out) {
+                                              int d_out, int nsplit) {
     __shared__ float red[4][kMB][kOutPad];
     const int r = threadIdx.x % kMB, grp = threadIdx.x / kMB;
     const int h_beg = blockIdx.x * kChunkH;
@@ -121,8 +122,7 @@ __global__ void __launch_bounds__(256) k_fwd2(const float* __restrict__ zpart, c
     for (int o = 0; o < kOutPad; ++o) l[o] = 0.f;
     for (int h = h_beg + grp; h < h_beg + kChunkH; h += 4) {
         float z = 0.f;
-#pragma unroll
-        for (int s = 0; s < kSplitK; ++s) z += zpart[((size_t)s * d_h + h) * kMB + r];
+        for (int s = 0; s < nsplit; ++s) z += zpart[((size_t)s * d_h + h) * kMB + r];
         z += b1[h];
         zt[(size_t)h * kMB + r] = z;
         const __nv_bfloat16 hb = __float2bfloat16_rn(z > 0.f ? z : 0.f);
@@ -404,6 +404,143 @@ __global__ void __launch_bounds__(128) k_dw1_tcgen05(const __grid_constant__ CUt
     }
 }
 
+// ============================================================================================
+// Forward GEMM on tcgen05:  zpart[s][h][r] = sum_{k in split s} W1b[k][h] * xb[r][k]
+//   D [M = 128 hidden][N = 64 samples] += A B^T with
+//   A = W1b^T tile: stored [k][h] with h contiguous, i.e. an MN-major operand.  A TMA box of
+//       64 h x 64 k (128-byte rows, 128-byte swizzle) is exactly the canonical MN-major layout:
+//       8-k-row groups 1024 B apart (stride offset), the two 64-wide h blocks of the tile one box
+//       (8192 B) apart (leading offset).  One UMMA step (K = 16) consumes two 8-k groups: +2048 B.
+//   B = xb tile [64 samples][64 k], K-major as in the dW1 kernel.
+// One CTA per (128-hidden tile, K split); a kFwdStages-deep TMA -> MMA pipeline streams the
+// weights once.  Warp 0 lane 0 issues TMA, warp 1 lane 0 issues MMAs, all four warps store D.
+// ============================================================================================
+constexpr int kFwdStages = 6;
+constexpr int kFwdStageBytes = 2 * 8192 + 8192;   // two A boxes + one B box
+
+__device__ __forceinline__ uint64_t umma_desc_mn_sw128(uint32_t smem_addr, uint32_t lbo_bytes) {
+    uint64_t d = 0;
+    d |= (uint64_t)((smem_addr & 0x3FFFF) >> 4);
+    d |= (uint64_t)(lbo_bytes >> 4) << 16;                // leading-dim byte offset: next 64-wide MN block
+    d |= (uint64_t)(1024 >> 4) << 32;                     // stride-dim byte offset: next group of 8 k-rows
+    d |= (uint64_t)1 << 46;
+    d |= (uint64_t)2 << 61;
+    return d;
+}
+
+struct FwdSmem {
+    alignas(1024) uint8_t stage[kFwdStages][kFwdStageBytes];   // [A h0..63 | A h64..127 | B]
+    alignas(8) uint64_t full[kFwdStages];
+    uint64_t empty[kFwdStages];
+    uint64_t done;
+    uint32_t tmem_base;
+    uint32_t failed;
+};
+
+__global__ void __launch_bounds__(128) k_fwd1_tcgen05(const __grid_constant__ CUtensorMap tm_w1,
+                                                      const __grid_constant__ CUtensorMap tm_xb, float* __restrict__ zpart,
+                                                      int d_in, int d_h, int* status) {
+    extern __shared__ uint8_t smem_raw[];
+    FwdSmem& s = *reinterpret_cast<FwdSmem*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+    const int warp = threadIdx.x / 32, lane = threadIdx.x % 32;
+    const int h0 = blockIdx.x * 128;
+    const int split = blockIdx.y;
+    const int k_per = d_in / (int)gridDim.y;
+    const int kbeg = split * k_per;
+    const int nk = k_per / 64;                       // pipeline steps of 64 k
+
+    if (warp == 0) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&s.tmem_base)), "r"(64) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    if (threadIdx.x == 0) {
+        for (int i = 0; i < kFwdStages; ++i) {
+            mbar_init(&s.full[i], 1);
+            mbar_init(&s.empty[i], 1);
+        }
+        mbar_init(&s.done, 1);
+        s.failed = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    const uint32_t tmem = s.tmem_base;
+
+    if (warp == 0 && lane == 0) {                    // ---- TMA producer
+        for (int kb = 0; kb < nk; ++kb) {
+            const int st = kb % kFwdStages;
+            if (kb >= kFwdStages && !mbar_wait(&s.empty[st], ((kb / kFwdStages) - 1) & 1)) { s.failed = 1; break; }
+            mbar_expect_tx(&s.full[st], kFwdStageBytes);
+            const int k0 = kbeg + kb * 64;
+            tma_load_2d(s.stage[st], &tm_w1, h0, k0, &s.full[st]);
+            tma_load_2d(s.stage[st] + 8192, &tm_w1, h0 + 64, k0, &s.full[st]);
+            tma_load_2d(s.stage[st] + 16384, &tm_xb, k0, 0, &s.full[st]);
+        }
+    } else if (warp == 1 && lane == 0) {             // ---- MMA issuer
+        constexpr uint32_t idesc = umma_idesc_bf16(128, 64) | (1u << 15);   // A is MN-major
+        bool ok = true;
+        for (int kb = 0; kb < nk && ok; ++kb) {
+            const int st = kb % kFwdStages;
+            ok = mbar_wait(&s.full[st], (kb / kFwdStages) & 1);
+            if (!ok) break;
+            asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+            const uint32_t a0 = smem_u32(s.stage[st]);
+            const uint64_t db = umma_desc_k_sw128(a0 + 16384);
+#pragma unroll
+            for (int k = 0; k < 4; ++k) {
+                const uint64_t da = umma_desc_mn_sw128(a0 + k * 2048, 8192);
+                const uint32_t accumulate = (kb > 0 || k > 0);
+                asm volatile(
+                    "{\n .reg .pred p;\n setp.ne.b32 p, %4, 0;\n"
+                    " tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n}\n"
+                    ::"r"(tmem), "l"(da), "l"(db + 2 * k), "r"(idesc), "r"(accumulate) : "memory");
+            }
+            // frees the stage for the producer once these MMAs have read it
+            asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(&s.empty[st])) : "memory");
+        }
+        if (ok) asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(&s.done)) : "memory");
+        else s.failed = 1;
+    }
+    __syncwarp();
+
+    bool ok = mbar_wait(&s.done, 0);
+    ok = __all_sync(0xffffffffu, ok);
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    if (ok) {
+        const int h = h0 + threadIdx.x;               // TMEM lane = hidden unit
+        float* out = zpart + ((size_t)split * d_h + h) * kMB;
+#pragma unroll 1
+        for (int p = 0; p < 2; ++p) {
+            uint32_t v[32];
+            const uint32_t taddr = tmem + ((uint32_t)(warp * 32) << 16) + (uint32_t)(p * 32);
+            asm volatile(
+                "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+                "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];"
+                : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]), "=r"(v[8]),
+                  "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15]), "=r"(v[16]),
+                  "=r"(v[17]), "=r"(v[18]), "=r"(v[19]), "=r"(v[20]), "=r"(v[21]), "=r"(v[22]), "=r"(v[23]), "=r"(v[24]),
+                  "=r"(v[25]), "=r"(v[26]), "=r"(v[27]), "=r"(v[28]), "=r"(v[29]), "=r"(v[30]), "=r"(v[31])
+                : "r"(taddr) : "memory");
+            asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+            for (int j = 0; j < 8; ++j)
+                *reinterpret_cast<float4*>(out + p * 32 + 4 * j) =
+                    make_float4(__uint_as_float(v[4 * j]), __uint_as_float(v[4 * j + 1]), __uint_as_float(v[4 * j + 2]),
+                                __uint_as_float(v[4 * j + 3]));
+        }
+    } else if (threadIdx.x == 0) {
+        atomicExch(status, ABS_ETIMEOUT);
+        // bounded chance for copies still in flight to land before shared memory is released
+        for (int i = 0; i < kFwdStages; ++i) mbar_wait(&s.full[i], 0);
+    }
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    if (warp == 0) {
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(64) : "memory");
+    }
+}
+
 // ---- host helpers --------------------------------------------------------------------------
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
@@ -454,7 +591,8 @@ size_t mlp_scratch_bytes(const MlpDims& d) {
     return o;
 }
 
-cudaError_t mlp_scratch_init(MlpScratch* s, const MlpDims& d, void* base, const char** err) {
+cudaError_t mlp_scratch_init(MlpScratch* s, const MlpDims& d, void* base, __nv_bfloat16* shadow0,
+                             __nv_bfloat16* shadow1, const char** err) {
     char* p = static_cast<char*>(base);
     size_t o = 0;
     auto take = [&](size_t b) { char* at = p + o; o = align_up(o + b, 1024); return at; };
@@ -476,6 +614,22 @@ cudaError_t mlp_scratch_init(MlpScratch* s, const MlpDims& d, void* base, const 
         *err = "cuTensorMapEncodeTiled failed for the dW1 operands";
         return cudaErrorInvalidValue;
     }
+    // forward GEMM operands: W1 (bf16 shadow, [d_in][d_hidden]) in 64 x 64 boxes, xb [mb][d_in] in 64 x 64 boxes
+    if (!encode_2d(reinterpret_cast<CUtensorMap*>(&s->tmap_w1[0]), CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, shadow0, d.d_in,
+                   d.d_hidden, 64, 64) ||
+        !encode_2d(reinterpret_cast<CUtensorMap*>(&s->tmap_w1[1]), CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, shadow1, d.d_in,
+                   d.d_hidden, 64, 64) ||
+        !encode_2d(reinterpret_cast<CUtensorMap*>(&s->tmap_xb), CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, s->xb, kMB, d.d_in, kMB,
+                   64)) {
+        *err = "cuTensorMapEncodeTiled failed for the forward GEMM operands";
+        return cudaErrorInvalidValue;
+    }
+    cudaError_t e0 = cudaFuncSetAttribute(k_fwd1_tcgen05, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                          (int)sizeof(FwdSmem) + 1024);
+    if (e0 != cudaSuccess) {
+        *err = "cudaFuncSetAttribute(forward kernel)";
+        return e0;
+    }
     cudaError_t e = cudaFuncSetAttribute(k_dw1_tcgen05<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                          (int)sizeof(DwSmem) + 1024);
     if (e == cudaSuccess)
@@ -493,16 +647,26 @@ cudaError_t mlp_make_acc_tmap(void* tmap_out, const MlpDims& d, float* acc_row) 
 }
 
 cudaError_t launch_mlp_grad(const MlpDims& d, const MlpScratch& s, const float* x_pub, const __nv_bfloat16* shadow,
-                            const float* x_dev, const int32_t* y_dev, float* acc_row, const void* acc_tmap, int32_t* cnt,
-                            int variant, cudaStream_t stream, void (*mark)(void*, int, int), void* user) {
+                            int shadow_idx, const float* x_dev, const int32_t* y_dev, float* acc_row, const void* acc_tmap,
+                            int32_t* cnt, int variant, cudaStream_t stream, void (*mark)(void*, int, int), void* user) {
     const size_t o_b1 = (size_t)d.d_in * d.d_hidden, o_w2 = o_b1 + d.d_hidden, o_b2 = o_w2 + (size_t)d.d_hidden * d.d_out;
     const int n_chunks = d.d_hidden / kChunkH;
     cudaError_t e;
 
     mark(user, ABS_K_MLP_FWD, 0);
     k_cast_x<<<d.d_in / 64, 256, 0, stream>>>(x_dev, s.xb, s.xtb, d.d_in);
-    k_fwd1<<<dim3(d.d_hidden / 64, kSplitK), 256, 0, stream>>>(shadow, s.xb, s.zpart, d.d_in, d.d_hidden);
-    k_fwd2<<<n_chunks, 256, 0, stream>>>(s.zpart, x_pub + o_b1, shadow + o_w2, s.zt, s.hbt, s.lpart, d.d_hidden, d.d_out);
+    // every K split must be a whole number of 64-wide pipeline steps (d_in is a multiple of 128)
+    const int nsplit = (d.d_in % (64 * kSplitK) == 0) ? kSplitK : 2;
+    if (variant & 2) {
+        k_fwd1<<<dim3(d.d_hidden / 64, nsplit), 256, 0, stream>>>(shadow, s.xb, s.zpart, d.d_in, d.d_hidden);
+    } else {
+        const CUtensorMap* tw = reinterpret_cast<const CUtensorMap*>(&s.tmap_w1[shadow_idx]);
+        const CUtensorMap* tx = reinterpret_cast<const CUtensorMap*>(&s.tmap_xb);
+        k_fwd1_tcgen05<<<dim3(d.d_hidden / 128, nsplit), 128, sizeof(FwdSmem) + 1024, stream>>>(*tw, *tx, s.zpart, d.d_in,
+                                                                                           d.d_hidden, s.status);
+    }
+    k_fwd2<<<n_chunks, 256, 0, stream>>>(s.zpart, x_pub + o_b1, shadow + o_w2, s.zt, s.hbt, s.lpart, d.d_hidden, d.d_out,
+                                         nsplit);
     k_loss<<<1, kMB, 0, stream>>>(s.lpart, n_chunks, x_pub + o_b2, y_dev, s.dl, s.dlb, acc_row + o_b2, d.d_out);
     mark(user, ABS_K_MLP_FWD, 4);
     if ((e = cudaGetLastError()) != cudaSuccess) return e;
@@ -518,7 +682,7 @@ cudaError_t launch_mlp_grad(const MlpDims& d, const MlpScratch& s, const float* 
     const CUtensorMap* ta = reinterpret_cast<const CUtensorMap*>(&s.tmap_xt);
     const CUtensorMap* tb = reinterpret_cast<const CUtensorMap*>(&s.tmap_dzt);
     const CUtensorMap* tc = reinterpret_cast<const CUtensorMap*>(acc_tmap);
-    if (variant == 1)
+    if (variant & 1)
         k_dw1_tcgen05<true><<<grid, 128, sizeof(DwSmem) + 1024, stream>>>(*ta, *tb, *tc, s.status);
     else
         k_dw1_tcgen05<false><<<grid, 128, sizeof(DwSmem) + 1024, stream>>>(*ta, *tb, *tc, s.status);

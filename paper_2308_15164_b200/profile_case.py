@@ -1,0 +1,73 @@
+"""Small, short runs of one kernel class, sized for a profiler capture.
+
+    python -m paper_2308_15164_b200.profile_case sync       [--P 11689512] [--W 4] [--iters 3]
+    python -m paper_2308_15164_b200.profile_case accumulate [--P 11689512] [--W 4] [--iters 3] [--bf16]
+    python -m paper_2308_15164_b200.profile_case mlp        [--iters 2]
+
+Each case keeps its working set larger than the 126 MB L2 but to a few hundred MB, launches the
+kernel of interest a handful of times and exits, so that a multi-pass capture ends by itself.
+Every kernel launched here is the library's own (through the C ABI); nothing is timed.
+"""
+
+from __future__ import annotations
+
+import argparse
+import sys
+
+import numpy as np
+import torch
+
+
+def main(argv=None):
+    ap = argparse.ArgumentParser()
+    ap.add_argument("case", choices=["sync", "accumulate", "mlp"])
+    ap.add_argument("--P", type=int, default=11_689_512)
+    ap.add_argument("--W", type=int, default=4)
+    ap.add_argument("--iters", type=int, default=3)
+    ap.add_argument("--bf16", action="store_true")
+    ap.add_argument("--pipelined", action="store_true")
+    ap.add_argument("--epilogue", type=int, default=0)
+    args = ap.parse_args(argv)
+
+    from . import binding as B
+    from . import workloads as wlm
+
+    dev = torch.device("cuda:0")
+    torch.cuda.set_device(dev)
+    if args.case in ("sync", "accumulate"):
+        g = torch.Generator(device="cpu").manual_seed(0)
+        x0 = (torch.randn(args.P, generator=g) * 0.02).to(dev)
+        pool = torch.randn((4, (args.P + 7) // 8 * 8), generator=g)
+        pool = (pool.to(torch.bfloat16) if args.bf16 else pool).to(dev)
+        eng = B.AbsSgd(x0, args.W, 0.1, 0.9, 5e-4, grad_dtype=B.GRAD_BF16 if args.bf16 else B.GRAD_F32,
+                       pipelined=args.pipelined)
+        torch.cuda.synchronize()
+        c = 0
+        for _ in range(args.iters + 1):          # the first sync step has nothing to apply
+            for i in range(args.W):
+                eng.accumulate(i, pool[c % 4]); c += 1
+            eng.sync_step()
+        eng.check()
+        eng.destroy()
+    else:
+        wl = wlm.config(4)
+        d = wl.mlp
+        x0 = torch.from_numpy(wlm.params0(wl)).to(dev)
+        xs, ys = wlm.mlp_batches(wl)
+        xs_d, ys_d = torch.from_numpy(xs[:8]).to(dev), torch.from_numpy(ys[:8]).to(dev)
+        eng = B.AbsSgd(x0, wl.W, wl.lr, wl.momentum, pipelined=args.pipelined, mlp=(d.d_in, d.d_hidden, d.d_out, d.mb))
+        eng.set_launch(B.K_MLP_DW1, args.epilogue)
+        torch.cuda.synchronize()
+        c = 0
+        for _ in range(args.iters + 1):
+            for i in range(wl.W):
+                eng.accumulate_mlp(i, xs_d[c % 8], ys_d[c % 8]); c += 1
+            eng.sync_step()
+        eng.check()
+        eng.destroy()
+    print("done", args.case)
+    return 0
+
+
+if __name__ == "__main__":
+    sys.exit(main())
