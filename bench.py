@@ -290,9 +290,11 @@ def run_mlp(B, wlm, dev, peaks, iters=12):
     x0_d = torch.from_numpy(wlm.params0(wl)).to(dev)
     xs, ys = wlm.mlp_batches(wl)
     xs_d, ys_d = torch.from_numpy(xs).to(dev), torch.from_numpy(ys).to(dev)
+    xp = [xs_d[b].data_ptr() for b in range(wl.mlp_pool)]      # raw device addresses of the micro-batches
+    yp = [ys_d[b].data_ptr() for b in range(wl.mlp_pool)]
     torch.cuda.synchronize()
     out = {"workload": "cfg4 mlp 3072-4096-10, mb=64, W=4, b_i~U{1..8}, pipelined", "iterations": iters}
-    for name, epi in (("tma_load_add_store", 0), ("tma_reduce_add", 1)):
+    for name, epi in (("tma_load_add_store", 0), ("tma_reduce_add", 1), ("persistent", 4)):
         eng = B.AbsSgd(x0_d, wl.W, wl.lr, wl.momentum, wl.weight_decay, pipelined=True, mlp=(d.d_in, d.d_hidden, d.d_out, d.mb))
         eng.set_launch(B.K_MLP_DW1, epi)
         calls = list(wlm.iter_calls(wl))
@@ -305,7 +307,7 @@ def run_mlp(B, wlm, dev, peaks, iters=12):
                 e0.record()
                 for it in calls:
                     for (i, k, c) in it:
-                        eng.accumulate_mlp(i, xs_d[c % wl.mlp_pool], ys_d[c % wl.mlp_pool]); n += 1
+                        eng.accumulate_mlp(i, xp[c % wl.mlp_pool], yp[c % wl.mlp_pool]); n += 1
                     eng.sync_step()
                 eng.wait()
                 e1.record()

@@ -71,7 +71,7 @@ Layout make_layout(const abs_config& c) {
         L.off_shadow[0] = take(L.P_pad * 2);
         L.off_shadow[1] = pipe ? take(L.P_pad * 2) : L.off_shadow[0];
         MlpDims d{(int)c.mlp_in, (int)c.mlp_hidden, (int)c.mlp_out, (int)c.mlp_mb};
-        L.off_mlp = take(mlp_scratch_bytes(d));
+        L.off_mlp = take(2 * mlp_scratch_bytes(d));
     }
     if (c.flags & ABS_FLAG_HOST_INPUT) {
         const size_t es = c.grad_dtype == ABS_GRAD_BF16 ? 2 : 4;
@@ -115,7 +115,12 @@ struct abs_ctx {
     int stage_next = 0;
     int ctas_per_sm[ABS_K_COUNT] = {0, 0, 0, 0, 0};
     MlpDims mlp_dims{0, 0, 0, 0};
-    MlpScratch mlp_scratch{};
+    MlpScratch mlp_scratch[2]{};         // two sets: front part of micro-batch n+1 overlaps dW1 of micro-batch n
+    cudaStream_t s_dw = nullptr;         // internal stream of the dW1 GEMMs
+    cudaEvent_t ev_front_done[2] = {nullptr, nullptr}, ev_dw_done[2] = {nullptr, nullptr};
+    bool slot_used[2] = {false, false};
+    int mlp_slot = 0, dw_last_slot = 0;
+    bool dw_outstanding = false;         // a dW1 kernel was enqueued since stream_acc last waited for that stream
     std::vector<TmapBytes> acc_tmaps;   // [2][W]: TMA descriptor of each accumulator row's W1 slice
 
     // bookkeeping
@@ -208,7 +213,16 @@ int collect_timings(abs_ctx* c) {
     return ABS_OK;
 }
 
-void mlp_mark(void* user, int kernel_class, int n);
+void mlp_mark(void* user, int kernel_class, int n, cudaStream_t stream);
+
+// stream_acc waits (on the device) for every dW1 GEMM enqueued so far on the internal stream.
+int join_dw(abs_ctx* c) {
+    if (c->dw_outstanding) {
+        CK(cudaStreamWaitEvent(c->s_acc, c->ev_dw_done[c->dw_last_slot], 0));
+        c->dw_outstanding = false;
+    }
+    return ABS_OK;
+}
 
 // Launch the fused Step-1 kernel on `set`, reading x[in] and writing x[out], on `stream`.
 int launch_fused(abs_ctx* c, uint32_t set, int in, int out, uint64_t log_step, cudaStream_t stream) {
@@ -308,9 +322,17 @@ int abs_init(abs_ctx** out, const abs_config* cfg, void* workspace_dev, size_t w
         if ((e = cudaMemsetAsync(c->ws + L.off_shadow[0], 0, L.P_pad * 2, c->s_acc)) != cudaSuccess) return bail(e, "cudaMemsetAsync");
         if (c->pipelined && (e = cudaMemsetAsync(c->ws + L.off_shadow[1], 0, L.P_pad * 2, c->s_acc)) != cudaSuccess)
             return bail(e, "cudaMemsetAsync");
-        if ((e = mlp_scratch_init(&c->mlp_scratch, c->mlp_dims, c->ws + L.off_mlp, c->shadow(0), c->shadow(1), &msg)) != cudaSuccess)
-            return bail(e, msg ? msg : "mlp_scratch_init");
-        if ((e = cudaMemsetAsync(c->mlp_scratch.status, 0, sizeof(int), c->s_acc)) != cudaSuccess) return bail(e, "cudaMemsetAsync");
+        const size_t one = mlp_scratch_bytes(c->mlp_dims);
+        for (int k = 0; k < 2; ++k) {
+            if ((e = mlp_scratch_init(&c->mlp_scratch[k], c->mlp_dims, c->ws + L.off_mlp + k * one, c->shadow(0), c->shadow(1),
+                                      &msg)) != cudaSuccess)
+                return bail(e, msg ? msg : "mlp_scratch_init");
+            if ((e = cudaMemsetAsync(c->mlp_scratch[k].zero_from, 0, c->mlp_scratch[k].zero_bytes, c->s_acc)) != cudaSuccess)
+                return bail(e, "cudaMemsetAsync");
+            if ((e = cudaEventCreateWithFlags(&c->ev_front_done[k], cudaEventDisableTiming)) != cudaSuccess) return bail(e, "cudaEventCreate");
+            if ((e = cudaEventCreateWithFlags(&c->ev_dw_done[k], cudaEventDisableTiming)) != cudaSuccess) return bail(e, "cudaEventCreate");
+        }
+        if ((e = cudaStreamCreateWithFlags(&c->s_dw, cudaStreamNonBlocking)) != cudaSuccess) return bail(e, "cudaStreamCreate");
         c->acc_tmaps.resize((size_t)2 * cfg->W);
         for (uint32_t set = 0; set < 2; ++set)
             for (uint32_t i = 0; i < cfg->W; ++i)
@@ -336,6 +358,7 @@ int abs_accumulate(abs_ctx* c, uint32_t worker, const void* grad_dev) {
     if (!live(c)) return ABS_ESTATE;
     if (worker >= c->cfg.W) return invalid(c, "worker index out of range");
     if (!grad_dev || (reinterpret_cast<uintptr_t>(grad_dev) & 15)) return invalid(c, "gradient pointer must be non-NULL and 16-byte aligned");
+    if (int rc = join_dw(c)) return rc;
     {
         Timed tm(c, ABS_K_ACCUMULATE, c->s_acc);
         CK(launch_accumulate(c->acc(c->cur, worker), grad_dev, c->cfg.grad_dtype, c->cfg.P, c->cnt(c->cur, worker),
@@ -351,6 +374,7 @@ int abs_accumulate_host(abs_ctx* c, uint32_t worker, const void* grad_host) {
     if (!(c->cfg.flags & ABS_FLAG_HOST_INPUT)) return invalid(c, "context was created without ABS_FLAG_HOST_INPUT");
     if (worker >= c->cfg.W) return invalid(c, "worker index out of range");
     if (!grad_host) return invalid(c, "gradient pointer is NULL");
+    if (int rc = join_dw(c)) return rc;
     const int k = c->stage_next;
     c->stage_next ^= 1;
     const size_t es = c->cfg.grad_dtype == ABS_GRAD_BF16 ? 2 : 4;
@@ -378,9 +402,23 @@ int abs_accumulate_mlp(abs_ctx* c, uint32_t worker, const float* x_dev, const in
     if (worker >= c->cfg.W) return invalid(c, "worker index out of range");
     if (!x_dev || (reinterpret_cast<uintptr_t>(x_dev) & 15)) return invalid(c, "x pointer must be non-NULL and 16-byte aligned");
     if (!y_dev || (reinterpret_cast<uintptr_t>(y_dev) & 3)) return invalid(c, "y pointer must be non-NULL and 4-byte aligned");
-    CK(launch_mlp_grad(c->mlp_dims, c->mlp_scratch, c->x(c->pub), c->shadow(c->pub), c->pub, x_dev, y_dev,
-                       c->acc(c->cur, worker), &c->acc_tmaps[(size_t)c->cur * c->cfg.W + worker], c->cnt(c->cur, worker),
-                       c->ctas_per_sm[ABS_K_MLP_DW1], c->s_acc, mlp_mark, c));
+    // Two scratch sets and a second stream: the latency-bound front part (cast, forward, loss,
+    // layer-2 backward) of micro-batch n+1 runs on stream_acc while the HBM-bound dW1 GEMM of
+    // micro-batch n runs on the internal stream.  dW1 kernels stay in call order on that stream.
+    const int k = c->mlp_slot;
+    c->mlp_slot ^= 1;
+    const int variant = c->ctas_per_sm[ABS_K_MLP_DW1];
+    if (c->slot_used[k]) CK(cudaStreamWaitEvent(c->s_acc, c->ev_dw_done[k], 0));   // scratch set k is free again
+    CK(launch_mlp_front(c->mlp_dims, c->mlp_scratch[k], c->x(c->pub), c->shadow(c->pub), c->pub, x_dev, y_dev,
+                        c->acc(c->cur, worker), c->cnt(c->cur, worker), variant, c->s_acc, mlp_mark, c));
+    CK(cudaEventRecord(c->ev_front_done[k], c->s_acc));
+    CK(cudaStreamWaitEvent(c->s_dw, c->ev_front_done[k], 0));
+    CK(launch_mlp_dw1(c->mlp_dims, c->mlp_scratch[k], &c->acc_tmaps[(size_t)c->cur * c->cfg.W + worker], variant, c->s_dw,
+                      mlp_mark, c));
+    CK(cudaEventRecord(c->ev_dw_done[k], c->s_dw));
+    c->slot_used[k] = true;
+    c->dw_outstanding = true;
+    c->dw_last_slot = k;
     c->h_cnt[(size_t)c->cur * c->cfg.W + worker] += 1;
     return ABS_OK;
 }
@@ -389,6 +427,7 @@ int abs_sync_step(abs_ctx* c) {
     if (!live(c)) return ABS_ESTATE;
     const uint32_t W = c->cfg.W;
     const uint32_t d = c->cur ^ 1;   // the delayed set (filled during iteration t-1)
+    if (int rc = join_dw(c)) return rc;
     if (!c->pipelined) {
         // Step 1 on the delayed set, in place, on stream_acc.
         int64_t B = 0;
@@ -466,6 +505,7 @@ int abs_momentum(abs_ctx* c, const float** v_dev_out) {
 int abs_accumulator(abs_ctx* c, uint32_t set, uint32_t worker, const float** acc_dev_out) {
     if (!live(c)) return ABS_ESTATE;
     if (set > 1 || worker >= c->cfg.W || !acc_dev_out) return invalid(c, "bad set / worker / output pointer");
+    if (int rc = join_dw(c)) return rc;
     *acc_dev_out = c->acc(set, worker);
     return ABS_OK;
 }
@@ -497,6 +537,7 @@ int abs_set_lr(abs_ctx* c, float lr) {
 
 int abs_wait(abs_ctx* c) {
     if (!live(c)) return ABS_ESTATE;
+    if (int rc = join_dw(c)) return rc;
     if (c->pipelined) {
         CK(cudaEventRecord(c->ev_aux, c->s_sync));
         CK(cudaStreamWaitEvent(c->s_acc, c->ev_aux, 0));
@@ -507,11 +548,13 @@ int abs_wait(abs_ctx* c) {
 int abs_check(abs_ctx* c) {
     if (!live(c)) return ABS_ESTATE;
     if (c->pipelined) CK(cudaStreamSynchronize(c->s_sync));
+    if (c->s_dw) CK(cudaStreamSynchronize(c->s_dw));
     CK(cudaStreamSynchronize(c->s_acc));
     if (c->mlp) {
-        int st = 0;
-        CK(cudaMemcpy(&st, c->mlp_scratch.status, sizeof(int), cudaMemcpyDeviceToHost));
-        if (st != 0) {
+        int st = 0, st1 = 0;
+        CK(cudaMemcpy(&st, c->mlp_scratch[0].status, sizeof(int), cudaMemcpyDeviceToHost));
+        CK(cudaMemcpy(&st1, c->mlp_scratch[1].status, sizeof(int), cudaMemcpyDeviceToHost));
+        if (st != 0 || st1 != 0) {
             c->err = "a bounded device-side wait ran out (MLP dW1 kernel)";
             return ABS_ETIMEOUT;
         }
@@ -565,6 +608,9 @@ int abs_destroy(abs_ctx* c) {
     cudaStreamSynchronize(c->s_acc);
     if (c->pipelined) cudaStreamSynchronize(c->s_sync);
     if (c->s_copy) { cudaStreamSynchronize(c->s_copy); cudaStreamDestroy(c->s_copy); }
+    if (c->s_dw) { cudaStreamSynchronize(c->s_dw); cudaStreamDestroy(c->s_dw); }
+    for (cudaEvent_t e : {c->ev_front_done[0], c->ev_front_done[1], c->ev_dw_done[0], c->ev_dw_done[1]})
+        if (e) cudaEventDestroy(e);
     for (auto& tl : c->timed) { cudaEventDestroy(tl.start); cudaEventDestroy(tl.stop); }
     for (auto e : c->ev_pool) cudaEventDestroy(e);
     for (cudaEvent_t e : {c->ev_acc_done, c->ev_sync_done, c->ev_aux, c->ev_stage_free[0], c->ev_stage_free[1],
@@ -579,17 +625,17 @@ int abs_destroy(abs_ctx* c) {
 
 namespace {
 // Called by the MLP launcher around each group of its kernels: n = 0 before, n = launches made after.
-void mlp_mark(void* user, int kernel_class, int n) {
+void mlp_mark(void* user, int kernel_class, int n, cudaStream_t stream) {
     abs_ctx* c = static_cast<abs_ctx*>(user);
     c->launches += (uint64_t)n;
     if (!c->profiling) return;
     if (n == 0) {
         cudaEvent_t start = take_event(c), stop = take_event(c);
         if (!start || !stop) return;
-        cudaEventRecord(start, c->s_acc);
+        cudaEventRecord(start, stream);
         c->timed.push_back({kernel_class, start, stop});
     } else if (!c->timed.empty() && c->timed.back().kernel_class == kernel_class) {
-        cudaEventRecord(c->timed.back().stop, c->s_acc);
+        cudaEventRecord(c->timed.back().stop, stream);
     }
 }
 }  // namespace

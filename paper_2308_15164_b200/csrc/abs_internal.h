@@ -51,13 +51,16 @@ struct MlpScratch {      // device pointers carved from the workspace (all hidde
     __nv_bfloat16* xb;   // [mb][d_in]            bf16(X)
     __nv_bfloat16* xtb;  // [d_in][mb]            bf16(X)^T: K-major A operand of dW1
     float* zpart;        // [split][d_hidden][mb] split-K partial sums of the forward GEMM
-    float* zt;           // [d_hidden][mb]        pre-activations Z^T (fp32)
     __nv_bfloat16* hbt;  // [d_hidden][mb]        bf16(relu(Z))^T
     __nv_bfloat16* dzt;  // [d_hidden][mb]        bf16(dZ)^T: K-major B operand of dW1
-    float* lpart;        // [chunks][mb][16]      partial logits
-    float* dl;           // [mb][16]              dL (fp32)
+    float* lpart;        // [d_hidden/32][mb][16] partial logits per CTA of k_fwd2
+    float* gpart;        // [groups][mb][16]      partial logits per group of 8 CTAs
     __nv_bfloat16* dlb;  // [mb][16]              bf16(dL)
+    unsigned int* tickets;  // [groups + 1]       "last CTA done" tickets of the logit reduction (zero between launches)
     int* status;         // device status word: ABS_ETIMEOUT if a bounded wait ran out
+    void* zero_from;     // region that must be zero before first use (tickets + status) ...
+    size_t zero_bytes;   // ... and its size
+    int num_sms;         // SM count of the device (grid of the persistent dW1 kernel)
     TmapBytes tmap_xt, tmap_dzt;   // dW1 operands
     TmapBytes tmap_xb, tmap_w1[2]; // forward GEMM operands (W1 of each bf16 shadow copy)
 };
@@ -67,14 +70,19 @@ cudaError_t mlp_scratch_init(MlpScratch* s, const MlpDims& d, void* base, __nv_b
                              __nv_bfloat16* shadow1, const char** err);
 // TMA descriptor of the W1 slice of one worker's accumulator row (fp32 [d_in][d_hidden]).
 cudaError_t mlp_make_acc_tmap(void* tmap_out, const MlpDims& d, float* acc_row);
-// Enqueues the whole micro-batch gradient; adds into acc_row (flat MLP layout) and bumps cnt.
-// shadow: bf16 copy of the published parameters (same flat layout).  x_pub: the fp32 parameters.
-// shadow_idx: which of the two shadow copies `shadow` is.  variant: bit 0 = dW1 epilogue by TMA reduce-add
-// (else TMA load + add + TMA store); bit 1 = forward GEMM on CUDA cores (cross-check of the tcgen05 one).
-// mark(user, kernel_class, 0) is called before a kernel group, mark(user, kernel_class, n) after n launches.
-cudaError_t launch_mlp_grad(const MlpDims& d, const MlpScratch& s, const float* x_pub,
-                            const __nv_bfloat16* shadow, int shadow_idx, const float* x_dev, const int32_t* y_dev,
-                            float* acc_row, const void* acc_tmap, int32_t* cnt, int variant, cudaStream_t stream,
-                            void (*mark)(void* user, int kernel_class, int n), void* user);
+// The micro-batch gradient is enqueued in two parts so that the caller can put them on different streams:
+//   front: cast, forward GEMM, loss, layer-2 backward (writes dzt/xtb of this scratch set; adds db2, db1, dW2
+//          into acc_row; bumps cnt);   dw1: the dW1 GEMM, which reads xtb/dzt and adds into the W1 slice.
+// shadow: bf16 copy of the published parameters (same flat layout), shadow_idx: which of the two copies it is.
+// x_pub: the fp32 parameters.  variant: bit 0 = dW1 epilogue by TMA reduce-add (else TMA load + add + TMA
+// store); bit 1 = forward GEMM on CUDA cores (cross-check of the tcgen05 one); bit 2 = persistent dW1 kernel.
+// mark(user, kernel_class, 0, stream) is called before a kernel group, mark(user, kernel_class, n, stream) after
+// its n launches.
+typedef void (*MlpMark)(void* user, int kernel_class, int n, cudaStream_t stream);
+cudaError_t launch_mlp_front(const MlpDims& d, const MlpScratch& s, const float* x_pub, const __nv_bfloat16* shadow,
+                             int shadow_idx, const float* x_dev, const int32_t* y_dev, float* acc_row, int32_t* cnt,
+                             int variant, cudaStream_t stream, MlpMark mark, void* user);
+cudaError_t launch_mlp_dw1(const MlpDims& d, const MlpScratch& s, const void* acc_tmap, int variant, cudaStream_t stream,
+                           MlpMark mark, void* user);
 
 }  // namespace abs_sgd

@@ -13,15 +13,18 @@
 // K = mb = 64), K-major: A = X^T stored [d_in][64], B = dZ^T stored [d_h][64].  A 64-element
 // bf16 row is exactly one 128-byte swizzle row, so each operand tile is one TMA box.
 //
-// Kernels (all on the caller's stream):
-//   k_cast_x      X fp32 -> bf16 in both orientations
+// Kernels (five launches per micro-batch; the first four form the "front" part, the last one
+// may run on another stream):
+//   k_cast_x        X fp32 -> bf16 in both orientations
 //   k_fwd1_tcgen05  Z^T partials = W1^T X^T, split over d_in, on tcgen05 (W1 as an MN-major operand)
 //   (k_fwd1         the same on CUDA cores, kept as a cross-check selectable through abs_set_launch)
-//   k_fwd2        Z = sum of partials + b1, gate, bf16(H), per-chunk partial logits
-//   k_loss        logits, softmax, dL, db2 += ...
-//   k_bwd         dH, dZ, db1 += ..., dW2 += ..., bf16(dZ)^T, b_i += 1
-//   k_dw1_tcgen05 dW1 tile = A B^T on the 5th-gen tensor cores (TMEM accumulator); epilogue
-//                 adds the tile into the worker's accumulator slice via TMA load / TMA store.
+//   k_fwd2          Z = sum of partials + b1, bf16(H), partial logits per 32 hidden units; the last CTAs
+//                   to finish (two-level ticket) reduce the partial logits in a fixed order and compute
+//                   softmax, dL and db2
+//   k_bwd           dH, dZ, bf16(dZ)^T, db1 += ..., dW2 += ..., b_i += 1
+//   k_dw1_tcgen05   dW1 tile = A B^T on the 5th-gen tensor cores (TMEM accumulator); epilogue adds the
+//                   tile into the worker's accumulator slice via TMA load / TMA store (or TMA reduce-add)
+//   (k_dw1_persistent  the same as a persistent, warp-specialised kernel with a shared-memory ring)
 #include <cuda.h>
 
 #include <cstdio>
@@ -34,34 +37,46 @@ namespace {
 
 constexpr int kMB = 64;          // samples per micro-batch = K of the dW1 contraction
 constexpr int kOutPad = 16;      // logits / dL rows are padded to 16 columns
-constexpr int kSplitK = 4;       // forward GEMM: d_in is split into this many partial sums
-constexpr int kChunkH = 128;     // hidden units per CTA in k_fwd2 (partial-logit chunk)
+constexpr int kSplitK = 4;       // forward GEMM: d_in is split into at most this many partial sums
+constexpr int kHB = 32;          // hidden units per CTA in k_fwd2 / k_bwd
+constexpr int kGroup = 8;        // CTAs per first-level group of the logit reduction
 
 __device__ __forceinline__ float bf16_to_f(__nv_bfloat16 v) { return __bfloat162float(v); }
+__device__ __forceinline__ uint32_t pack_bf16x2(float a, float b) {
+    __nv_bfloat162 p = __floats2bfloat162_rn(a, b);
+    return *reinterpret_cast<uint32_t*>(&p);
+}
 
 // --------------------------------------------------------------------------------------------
-// X [64][d_in] fp32  ->  xb [64][d_in] bf16  and  xtb [d_in][64] bf16
+// X [64][d_in] fp32  ->  xb [64][d_in] bf16  and  xtb [d_in][64] bf16.   CTA: 16 columns.
 // --------------------------------------------------------------------------------------------
 __global__ void __launch_bounds__(256) k_cast_x(const float* __restrict__ x, __nv_bfloat16* __restrict__ xb,
                                                 __nv_bfloat16* __restrict__ xtb, int d_in) {
-    __shared__ __nv_bfloat16 tile[kMB][64 + 2];
-    const int c0 = blockIdx.x * 64;
-    for (int e = threadIdx.x; e < kMB * 64; e += 256) {
-        const int r = e / 64, c = e % 64;
-        const __nv_bfloat16 v = __float2bfloat16_rn(x[(size_t)r * d_in + c0 + c]);
-        xb[(size_t)r * d_in + c0 + c] = v;
-        tile[r][c] = v;
+    __shared__ __nv_bfloat16 tile[16][kMB + 8];
+    const int c0 = blockIdx.x * 16;
+    {
+        const int r = threadIdx.x / 4, q = threadIdx.x % 4;
+        const float4 v = *reinterpret_cast<const float4*>(x + (size_t)r * d_in + c0 + 4 * q);
+        uint2 pk;
+        pk.x = pack_bf16x2(v.x, v.y);
+        pk.y = pack_bf16x2(v.z, v.w);
+        *reinterpret_cast<uint2*>(xb + (size_t)r * d_in + c0 + 4 * q) = pk;
+        tile[4 * q + 0][r] = __float2bfloat16_rn(v.x);
+        tile[4 * q + 1][r] = __float2bfloat16_rn(v.y);
+        tile[4 * q + 2][r] = __float2bfloat16_rn(v.z);
+        tile[4 * q + 3][r] = __float2bfloat16_rn(v.w);
     }
     __syncthreads();
-    for (int e = threadIdx.x; e < kMB * 64; e += 256) {
-        const int c = e / 64, r = e % 64;
-        xtb[(size_t)(c0 + c) * kMB + r] = tile[r][c];
+    {
+        const int c = threadIdx.x / 16, r4 = (threadIdx.x % 16) * 4;
+        uint2 pk = *reinterpret_cast<const uint2*>(&tile[c][r4]);
+        *reinterpret_cast<uint2*>(xtb + (size_t)(c0 + c) * kMB + r4) = pk;
     }
 }
 
 // --------------------------------------------------------------------------------------------
-// Forward GEMM, CUDA cores:  zpart[s][h][r] = sum_{k in split s} W1b[k][h] * xb[r][k]
-// CTA tile: 64 hidden x 64 samples, 256 threads, 4x4 outputs per thread.
+// Forward GEMM, CUDA cores (cross-check):  zpart[s][h][r] = sum_{k in split s} W1b[k][h] * xb[r][k]
+// CTA tile: 64 hidden x 64 samples, 256 threads, 4x4 outputs per thread; gridDim.y = number of splits.
 // --------------------------------------------------------------------------------------------
 __global__ void __launch_bounds__(256) k_fwd1(const __nv_bfloat16* __restrict__ w1b, const __nv_bfloat16* __restrict__ xb,
                                               float* __restrict__ zpart, int d_in, int d_h) {
@@ -107,124 +122,194 @@ __global__ void __launch_bounds__(256) k_fwd1(const __nv_bfloat16* __restrict__ 
 }
 
 // --------------------------------------------------------------------------------------------
-// Z = sum_s zpart + b1 ; gate ; bf16(H) ; partial logits of this chunk of hidden units.
-// CTA: kChunkH hidden units; 256 threads = 4 groups of 64 samples.
+// k_fwd2: per CTA 32 hidden units x 64 samples.
+//   phase 1 (thread = sample r, 8 hidden units): Z = sum_s zpart + b1 ; hb = bf16(relu(Z)) -> hbt
+//   phase 2 (thread = sample r, 4 logits):        partial logits of these 32 hidden units -> lpart[cta]
+//   tail: the last CTA of each group of 8 sums the group's partials (fixed order) -> gpart[group];
+//         the last group to finish sums the group partials, adds b2, and computes
+//         dL = (softmax - onehot)/mb, bf16(dL), db2 += sum_r dL.
+// tickets[0 .. n_groups) are the group tickets, tickets[n_groups] the global one; all zero on entry
+// and reset before exit.
 // --------------------------------------------------------------------------------------------
-__global__ void __launch_bounds__(256) k_fwd2(const float* __restrict__ zpart, const float* __restrict__ b1,
-                                              const __nv_bfloat16* __restrict__ w2b, float* __restrict__ zt,
-                                              __nv_bfloat16* __restrict__ hbt, float* __restrict__ lpart, int d_h,
-                                              int d_out, int nsplit) {
-    __shared__ float red[4][kMB][kOutPad];
-    const int r = threadIdx.x % kMB, grp = threadIdx.x / kMB;
-    const int h_beg = blockIdx.x * kChunkH;
-    float l[kOutPad];
-#pragma unroll
-    for (int o = 0; o < kOutPad; ++o) l[o] = 0.f;
-    for (int h = h_beg + grp; h < h_beg + kChunkH; h += 4) {
-        float z = 0.f;
-        for (int s = 0; s < nsplit; ++s) z += zpart[((size_t)s * d_h + h) * kMB + r];
-        z += b1[h];
-        zt[(size_t)h * kMB + r] = z;
-        const __nv_bfloat16 hb = __float2bfloat16_rn(z > 0.f ? z : 0.f);
-        hbt[(size_t)h * kMB + r] = hb;
-        const float hf = bf16_to_f(hb);
-        for (int o = 0; o < d_out; ++o) l[o] = fmaf(hf, bf16_to_f(w2b[(size_t)h * d_out + o]), l[o]);
+__global__ void __launch_bounds__(256) k_fwd2(const float* __restrict__ zpart, int nsplit, const float* __restrict__ b1,
+                                              const __nv_bfloat16* __restrict__ w2b, const float* __restrict__ b2,
+                                              const int32_t* __restrict__ y, __nv_bfloat16* __restrict__ hbt,
+                                              float* lpart, float* gpart, unsigned int* tickets,
+                                              __nv_bfloat16* __restrict__ dlb, float* acc_b2, int d_h, int d_out) {
+    __shared__ float sh[kHB][kMB + 1];
+    __shared__ float sw2[kHB][kOutPad];
+    __shared__ float sl[kMB][kOutPad + 1];
+    __shared__ unsigned int s_last;
+    const int h_beg = blockIdx.x * kHB;
+    const int n_cta = gridDim.x;
+    const int n_groups = (n_cta + kGroup - 1) / kGroup;
+
+    for (int e = threadIdx.x; e < kHB * kOutPad; e += 256) {
+        const int hl = e / kOutPad, o = e % kOutPad;
+        sw2[hl][o] = o < d_out ? bf16_to_f(w2b[(size_t)(h_beg + hl) * d_out + o]) : 0.f;
     }
+    {
+        const int r = threadIdx.x % kMB, g = threadIdx.x / kMB;
+        float z[8];
 #pragma unroll
-    for (int o = 0; o < kOutPad; ++o) red[grp][r][o] = l[o];
+        for (int j = 0; j < 8; ++j) z[j] = b1[h_beg + g * 8 + j];
+        for (int s = 0; s < nsplit; ++s)
+#pragma unroll
+            for (int j = 0; j < 8; ++j) z[j] += zpart[((size_t)s * d_h + h_beg + g * 8 + j) * kMB + r];
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+            const __nv_bfloat16 hb = __float2bfloat16_rn(z[j] > 0.f ? z[j] : 0.f);
+            hbt[(size_t)(h_beg + g * 8 + j) * kMB + r] = hb;
+            sh[g * 8 + j][r] = bf16_to_f(hb);
+        }
+    }
     __syncthreads();
-    for (int e = threadIdx.x; e < kMB * kOutPad; e += 256) {
-        const int rr = e / kOutPad, o = e % kOutPad;
-        lpart[((size_t)blockIdx.x * kMB + rr) * kOutPad + o] = (red[0][rr][o] + red[1][rr][o]) + (red[2][rr][o] + red[3][rr][o]);
+    {
+        const int r = threadIdx.x / 4, og = threadIdx.x % 4;
+        float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
+#pragma unroll 8
+        for (int hl = 0; hl < kHB; ++hl) {
+            const float hv = sh[hl][r];
+            a0 = fmaf(hv, sw2[hl][4 * og + 0], a0);
+            a1 = fmaf(hv, sw2[hl][4 * og + 1], a1);
+            a2 = fmaf(hv, sw2[hl][4 * og + 2], a2);
+            a3 = fmaf(hv, sw2[hl][4 * og + 3], a3);
+        }
+        reinterpret_cast<float4*>(lpart)[(size_t)blockIdx.x * (kMB * kOutPad / 4) + threadIdx.x] = make_float4(a0, a1, a2, a3);
     }
+    // ---- first level: last CTA of the group reduces the group's partial logits
+    const int group = blockIdx.x / kGroup;
+    const int g_first = group * kGroup;
+    const int g_count = min(kGroup, n_cta - g_first);
+    __threadfence();
+    __syncthreads();
+    if (threadIdx.x == 0) s_last = (atomicAdd(&tickets[group], 1u) == (unsigned)(g_count - 1));
+    __syncthreads();
+    if (!s_last) return;
+    __threadfence();
+    {
+        float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+        for (int c = 0; c < g_count; ++c) {
+            const float4 v = __ldcg(reinterpret_cast<const float4*>(lpart) + (size_t)(g_first + c) * (kMB * kOutPad / 4) + threadIdx.x);
+            acc.x += v.x; acc.y += v.y; acc.z += v.z; acc.w += v.w;
+        }
+        reinterpret_cast<float4*>(gpart)[(size_t)group * (kMB * kOutPad / 4) + threadIdx.x] = acc;
+    }
+    // ---- second level: the last group sums all group partials and finishes the loss
+    __threadfence();
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        tickets[group] = 0u;
+        s_last = (atomicAdd(&tickets[n_groups], 1u) == (unsigned)(n_groups - 1));
+    }
+    __syncthreads();
+    if (!s_last) return;
+    __threadfence();
+    {
+        float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+        for (int c = 0; c < n_groups; ++c) {
+            const float4 v = __ldcg(reinterpret_cast<const float4*>(gpart) + (size_t)c * (kMB * kOutPad / 4) + threadIdx.x);
+            acc.x += v.x; acc.y += v.y; acc.z += v.z; acc.w += v.w;
+        }
+        const int r = threadIdx.x / 4, og = threadIdx.x % 4;
+        sl[r][4 * og + 0] = acc.x; sl[r][4 * og + 1] = acc.y; sl[r][4 * og + 2] = acc.z; sl[r][4 * og + 3] = acc.w;
+    }
+    __syncthreads();
+    if (threadIdx.x < kMB) {
+        const int r = threadIdx.x;
+        float l[kOutPad];
+        float mx = -INFINITY;
+#pragma unroll
+        for (int o = 0; o < kOutPad; ++o) {
+            l[o] = o < d_out ? sl[r][o] + b2[o] : -INFINITY;
+            mx = fmaxf(mx, l[o]);
+        }
+        float den = 0.f;
+#pragma unroll
+        for (int o = 0; o < kOutPad; ++o) {
+            l[o] = o < d_out ? expf(l[o] - mx) : 0.f;
+            den += l[o];
+        }
+        const int yr = y[r];
+#pragma unroll
+        for (int o = 0; o < kOutPad; ++o) {
+            const float g = o < d_out ? (l[o] / den - (o == yr ? 1.f : 0.f)) * (1.0f / kMB) : 0.f;
+            dlb[r * kOutPad + o] = __float2bfloat16_rn(g);
+            sl[r][o] = g;
+        }
+    }
+    __syncthreads();
+    if (threadIdx.x < d_out) {
+        float s = 0.f;
+        for (int rr = 0; rr < kMB; ++rr) s += sl[rr][threadIdx.x];
+        acc_b2[threadIdx.x] += s;
+    }
+    if (threadIdx.x == 0) tickets[n_groups] = 0u;
 }
 
 // --------------------------------------------------------------------------------------------
-// One CTA: logits = sum of chunk partials + b2 ; softmax ; dL = (p - onehot)/mb ; db2 += sum_r dL.
+// k_bwd: per CTA 32 hidden units x 64 samples.
+//   phase 1 (thread = sample r, 8 hidden units): dH = sum_o bf16(dL)[r][o] W2b[h][o]; dZ = dH * [H > 0]
+//            (H > 0 exactly when Z > 0); dzt[h][r] = bf16(dZ)
+//   phase 2 (thread = hidden unit, 2 outputs): dW2[h][o] += sum_r bf16(H)[h][r] bf16(dL)[r][o],
+//            db1[h] += sum_r dZ[h][r]   (fixed summation order over r)
 // --------------------------------------------------------------------------------------------
-__global__ void __launch_bounds__(kMB) k_loss(const float* __restrict__ lpart, int n_chunks, const float* __restrict__ b2,
-                                              const int32_t* __restrict__ y, float* __restrict__ dl,
-                                              __nv_bfloat16* __restrict__ dlb, float* acc_b2, int d_out) {
-    __shared__ float sdl[kMB][kOutPad];
-    const int r = threadIdx.x;
-    float l[kOutPad];
-    float mx = -INFINITY;
-    for (int o = 0; o < d_out; ++o) {
-        float s = 0.f;
-        for (int c = 0; c < n_chunks; ++c) s += lpart[((size_t)c * kMB + r) * kOutPad + o];
-        l[o] = s + b2[o];
-        mx = fmaxf(mx, l[o]);
+__global__ void __launch_bounds__(256) k_bwd(const __nv_bfloat16* __restrict__ hbt, const __nv_bfloat16* __restrict__ dlb,
+                                             const __nv_bfloat16* __restrict__ w2b, __nv_bfloat16* __restrict__ dzt,
+                                             float* acc_b1, float* acc_w2, int32_t* cnt, int d_out) {
+    __shared__ float sdl[kMB][kOutPad + 1];
+    __shared__ float sw2[kHB][kOutPad];
+    __shared__ float sh[kHB][kMB + 1];
+    __shared__ float sdz[kHB][kMB + 1];
+    const int h_beg = blockIdx.x * kHB;
+    for (int e = threadIdx.x; e < kMB * kOutPad; e += 256) sdl[e / kOutPad][e % kOutPad] = bf16_to_f(dlb[e]);
+    for (int e = threadIdx.x; e < kHB * kOutPad; e += 256) {
+        const int hl = e / kOutPad, o = e % kOutPad;
+        sw2[hl][o] = o < d_out ? bf16_to_f(w2b[(size_t)(h_beg + hl) * d_out + o]) : 0.f;
     }
-    float den = 0.f;
-    for (int o = 0; o < d_out; ++o) {
-        l[o] = expf(l[o] - mx);
-        den += l[o];
-    }
-    const int yr = y[r];
-    for (int o = 0; o < kOutPad; ++o) {
-        float g = 0.f;
-        if (o < d_out) g = (l[o] / den - (o == yr ? 1.f : 0.f)) * (1.0f / kMB);
-        dl[r * kOutPad + o] = g;
-        dlb[r * kOutPad + o] = __float2bfloat16_rn(g);
-        sdl[r][o] = g;
-    }
-    __syncthreads();
-    if (r < d_out) {
-        float s = 0.f;
-        for (int rr = 0; rr < kMB; ++rr) s += sdl[rr][r];
-        acc_b2[r] += s;
-    }
-}
-
-// --------------------------------------------------------------------------------------------
-// Backward through layer 2 and the ReLU, hidden-major.  CTA: 8 hidden units, 64 threads each.
-//   dH[r][h] = sum_o bf16(dL)[r][o] * W2b[h][o] ; dZ = dH * [Z > 0] ; dzt[h][r] = bf16(dZ)
-//   db1[h] += sum_r dZ ; dW2[h][o] += sum_r bf16(H)[h][r] * bf16(dL)[r][o] ; b_i += 1
-// --------------------------------------------------------------------------------------------
-__global__ void __launch_bounds__(512) k_bwd(const float* __restrict__ zt, const __nv_bfloat16* __restrict__ hbt,
-                                             const __nv_bfloat16* __restrict__ dlb, const __nv_bfloat16* __restrict__ w2b,
-                                             __nv_bfloat16* __restrict__ dzt, float* acc_b1, float* acc_w2, int32_t* cnt,
-                                             int d_out) {
-    __shared__ float sdl[kMB][kOutPad];
-    __shared__ float red[8][2][kOutPad + 1];
-    for (int e = threadIdx.x; e < kMB * kOutPad; e += 512) sdl[e / kOutPad][e % kOutPad] = bf16_to_f(dlb[e]);
-    __syncthreads();
     const int r = threadIdx.x % kMB, g = threadIdx.x / kMB;
-    const int h = blockIdx.x * 8 + g;
-    float dh = 0.f;
-    for (int o = 0; o < d_out; ++o) dh = fmaf(sdl[r][o], bf16_to_f(w2b[(size_t)h * d_out + o]), dh);
-    const float dz = zt[(size_t)h * kMB + r] > 0.f ? dh : 0.f;
-    dzt[(size_t)h * kMB + r] = __float2bfloat16_rn(dz);
-    const float hf = bf16_to_f(hbt[(size_t)h * kMB + r]);
-    // reductions over the 64 samples: values [0, d_out) are dW2[h][o], value d_out is db1[h]
-    float vals[kOutPad + 1];
+    float hv[8];
 #pragma unroll
-    for (int o = 0; o < kOutPad; ++o) vals[o] = o < d_out ? hf * sdl[r][o] : 0.f;
-    vals[kOutPad] = dz;
-#pragma unroll
-    for (int o = 0; o <= kOutPad; ++o) {
-        float v = vals[o];
-#pragma unroll
-        for (int off = 16; off > 0; off >>= 1) v += __shfl_xor_sync(0xffffffffu, v, off);
-        vals[o] = v;
-    }
-    const int half = (threadIdx.x % kMB) / 32;
-    if (threadIdx.x % 32 == 0)
-#pragma unroll
-        for (int o = 0; o <= kOutPad; ++o) red[g][half][o] = vals[o];
+    for (int j = 0; j < 8; ++j) hv[j] = bf16_to_f(hbt[(size_t)(h_beg + g * 8 + j) * kMB + r]);
     __syncthreads();
-    if (r <= kOutPad) {
-        const float s = red[g][0][r] + red[g][1][r];
-        if (r < d_out) acc_w2[(size_t)h * d_out + r] += s;
-        else if (r == kOutPad) acc_b1[h] += s;
+    {
+        float dl[kOutPad];
+#pragma unroll
+        for (int o = 0; o < kOutPad; ++o) dl[o] = sdl[r][o];
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+            const int hl = g * 8 + j;
+            float dh = 0.f;
+#pragma unroll
+            for (int o = 0; o < kOutPad; ++o) dh = fmaf(dl[o], sw2[hl][o], dh);
+            const float dz = hv[j] > 0.f ? dh : 0.f;
+            dzt[(size_t)(h_beg + hl) * kMB + r] = __float2bfloat16_rn(dz);
+            sh[hl][r] = hv[j];
+            sdz[hl][r] = dz;
+        }
+    }
+    __syncthreads();
+    {
+        const int hl = threadIdx.x / 8, slot = threadIdx.x % 8;   // dW2 outputs `slot` and `slot + 8`; slot 0 also db1
+        float a = 0.f, b = 0.f, c = 0.f;
+#pragma unroll 8
+        for (int rr = 0; rr < kMB; ++rr) {
+            const float h = sh[hl][rr];
+            a = fmaf(h, sdl[rr][slot], a);
+            b = fmaf(h, sdl[rr][slot + 8], b);
+            if (slot == 0) c += sdz[hl][rr];
+        }
+        const int h = h_beg + hl;
+        if (slot < d_out) acc_w2[(size_t)h * d_out + slot] += a;
+        if (slot + 8 < d_out) acc_w2[(size_t)h * d_out + slot + 8] += b;
+        if (slot == 0) acc_b1[h] += c;
     }
     if (blockIdx.x == 0 && threadIdx.x == 0) cnt[0] += 1;   // M_t^i += M_r
 }
 
 // ============================================================================================
-// dW1 = X^T dZ on tcgen05.  One CTA per 128 x 128 output tile; K = 64 = four UMMA steps.
+// tcgen05 / TMA / mbarrier helpers
 // ============================================================================================
-constexpr int kTileM = 128, kTileN = 128;
 constexpr uint32_t kSpinLimit = 1u << 22;
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -234,6 +319,9 @@ __device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
 }
 __device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, uint32_t bytes) {
     asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
 }
 // Bounded wait: gives up after kSpinLimit polls and reports failure instead of hanging.
 __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity) {
@@ -272,15 +360,71 @@ __device__ __forceinline__ uint64_t umma_desc_k_sw128(uint32_t smem_addr) {
     d |= (uint64_t)2 << 61;                               // 128-byte swizzle
     return d;
 }
-// Instruction descriptor: D = f32, A = B = bf16, both K-major, M x N tile.
+// Same for an MN-major tile: a TMA box of 64 MN-elements x 64 k (128-byte rows, 128-byte swizzle).
+// Groups of 8 k-rows are 1024 bytes apart (stride offset); the next 64-wide MN block is `lbo_bytes` away.
+__device__ __forceinline__ uint64_t umma_desc_mn_sw128(uint32_t smem_addr, uint32_t lbo_bytes) {
+    uint64_t d = 0;
+    d |= (uint64_t)((smem_addr & 0x3FFFF) >> 4);
+    d |= (uint64_t)(lbo_bytes >> 4) << 16;
+    d |= (uint64_t)(1024 >> 4) << 32;
+    d |= (uint64_t)1 << 46;
+    d |= (uint64_t)2 << 61;
+    return d;
+}
+// Instruction descriptor: D = f32, A = B = bf16, both K-major (set bit 15 for an MN-major A), M x N tile.
 __host__ __device__ constexpr uint32_t umma_idesc_bf16(int M, int N) {
     return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(N >> 3) << 17) | ((uint32_t)(M >> 4) << 24);
 }
+__device__ __forceinline__ void umma_bf16(uint32_t tmem_d, uint64_t da, uint64_t db, uint32_t idesc, uint32_t accumulate) {
+    asm volatile(
+        "{\n .reg .pred p;\n setp.ne.b32 p, %4, 0;\n"
+        " tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n}\n"
+        ::"r"(tmem_d), "l"(da), "l"(db), "r"(idesc), "r"(accumulate) : "memory");
+}
+__device__ __forceinline__ void umma_commit(uint64_t* bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+// 32 consecutive fp32 columns of this thread's TMEM lane.
+__device__ __forceinline__ void tmem_ld_32(uint32_t taddr, uint32_t (&v)[32]) {
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+        "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];"
+        : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]), "=r"(v[8]),
+          "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15]), "=r"(v[16]),
+          "=r"(v[17]), "=r"(v[18]), "=r"(v[19]), "=r"(v[20]), "=r"(v[21]), "=r"(v[22]), "=r"(v[23]), "=r"(v[24]),
+          "=r"(v[25]), "=r"(v[26]), "=r"(v[27]), "=r"(v[28]), "=r"(v[29]), "=r"(v[30]), "=r"(v[31])
+        : "r"(taddr) : "memory");
+    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+}
+// Adds the 32 TMEM values of one row into that row of a swizzled [128][32] fp32 panel in shared
+// memory (row = 128 bytes; 16-byte chunk j sits at position j ^ (row % 8), as the TMA box wrote it).
+template <bool kAdd>
+__device__ __forceinline__ void panel_row_update(float* panel, int row, const uint32_t (&v)[32]) {
+    float4* prow = reinterpret_cast<float4*>(panel + row * 32);
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+        float4* q = prow + (j ^ (row & 7));
+        float4 d = make_float4(__uint_as_float(v[4 * j]), __uint_as_float(v[4 * j + 1]), __uint_as_float(v[4 * j + 2]),
+                               __uint_as_float(v[4 * j + 3]));
+        if (kAdd) {
+            const float4 c = *q;
+            d.x += c.x; d.y += c.y; d.z += c.z; d.w += c.w;
+        }
+        *q = d;
+    }
+}
+
+// ============================================================================================
+// dW1 = X^T dZ on tcgen05.  One CTA per 128 x kDwN output tile; K = 64 = four UMMA steps.
+// ============================================================================================
+constexpr int kTileM = 128;
+constexpr int kDwN = 64;
+constexpr int kPanels = kDwN / 32;
 
 struct DwSmem {
-    alignas(1024) uint8_t a[kTileM * 128];        // A tile  [128 m][64 k] bf16, swizzled rows
-    alignas(1024) uint8_t b[kTileN * 128];        // B tile  [128 n][64 k] bf16
-    alignas(1024) float c[4][kTileM * 32];        // accumulator tile as 4 column panels [128][32] fp32, swizzled rows
+    alignas(1024) uint8_t a[kTileM * 128];            // A tile  [128 m][64 k] bf16, swizzled rows
+    alignas(1024) uint8_t b[kDwN * 128];              // B tile  [kDwN n][64 k] bf16
+    alignas(1024) float c[kPanels][kTileM * 32];      // accumulator tile as column panels [128][32] fp32, swizzled rows
     alignas(8) uint64_t bar_ab;
     uint64_t bar_c;
     uint64_t bar_mma;
@@ -294,12 +438,12 @@ __global__ void __launch_bounds__(128) k_dw1_tcgen05(const __grid_constant__ CUt
                                                      const __grid_constant__ CUtensorMap tm_acc, int* status) {
     extern __shared__ uint8_t smem_raw[];
     DwSmem& s = *reinterpret_cast<DwSmem*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
-    const int warp = threadIdx.x / 32, lane = threadIdx.x % 32;
-    const int n0 = blockIdx.x * kTileN;   // hidden offset
+    const int warp = threadIdx.x / 32;
+    const int n0 = blockIdx.x * kDwN;     // hidden offset
     const int m0 = blockIdx.y * kTileM;   // input-feature offset
 
     if (warp == 0) {
-        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&s.tmem_base)), "r"(kTileN) : "memory");
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&s.tmem_base)), "r"(kDwN) : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
     }
     if (threadIdx.x == 0) {
@@ -315,29 +459,23 @@ __global__ void __launch_bounds__(128) k_dw1_tcgen05(const __grid_constant__ CUt
     const uint32_t tmem = s.tmem_base;
 
     if (threadIdx.x == 0) {
-        mbar_expect_tx(&s.bar_ab, kTileM * 128 + kTileN * 128);
+        mbar_expect_tx(&s.bar_ab, kTileM * 128 + kDwN * 128);
         tma_load_2d(s.a, &tm_xt, 0, m0, &s.bar_ab);
         tma_load_2d(s.b, &tm_dzt, 0, n0, &s.bar_ab);
         if (!kReduce) {   // the accumulator tile streams in while the MMA runs
-            mbar_expect_tx(&s.bar_c, kTileM * kTileN * 4);
+            mbar_expect_tx(&s.bar_c, kTileM * kDwN * 4);
 #pragma unroll
-            for (int p = 0; p < 4; ++p) tma_load_2d(s.c[p], &tm_acc, n0 + p * 32, m0, &s.bar_c);
+            for (int p = 0; p < kPanels; ++p) tma_load_2d(s.c[p], &tm_acc, n0 + p * 32, m0, &s.bar_c);
         }
         if (mbar_wait(&s.bar_ab, 0)) {
             asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
             const uint64_t da = umma_desc_k_sw128(smem_u32(s.a));
             const uint64_t db = umma_desc_k_sw128(smem_u32(s.b));
-            constexpr uint32_t idesc = umma_idesc_bf16(kTileM, kTileN);
+            constexpr uint32_t idesc = umma_idesc_bf16(kTileM, kDwN);
 #pragma unroll
-            for (int k = 0; k < kMB / 16; ++k) {
-                const uint32_t accumulate = k > 0;
-                // advancing K by 16 bf16 = 32 bytes inside the swizzled row: +2 in the address field
-                asm volatile(
-                    "{\n .reg .pred p;\n setp.ne.b32 p, %4, 0;\n"
-                    " tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n}\n"
-                    ::"r"(tmem), "l"(da + 2 * k), "l"(db + 2 * k), "r"(idesc), "r"(accumulate) : "memory");
-            }
-            asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(&s.bar_mma)) : "memory");
+            for (int k = 0; k < kMB / 16; ++k)   // K advances by 16 bf16 = 32 bytes: +2 in the address field
+                umma_bf16(tmem, da + 2 * k, db + 2 * k, idesc, k > 0);
+            umma_commit(&s.bar_mma);
         } else {
             s.failed = 1;
         }
@@ -346,35 +484,15 @@ __global__ void __launch_bounds__(128) k_dw1_tcgen05(const __grid_constant__ CUt
 
     bool ok = mbar_wait(&s.bar_mma, 0);
     if (!kReduce) ok = mbar_wait(&s.bar_c, 0) && ok;
+    ok = __all_sync(0xffffffffu, ok);
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
     if (ok) {
         const int row = threadIdx.x;                    // TMEM lane = output row
 #pragma unroll 1
-        for (int p = 0; p < 4; ++p) {
+        for (int p = 0; p < kPanels; ++p) {
             uint32_t v[32];
-            const uint32_t taddr = tmem + ((uint32_t)(warp * 32) << 16) + (uint32_t)(p * 32);
-            asm volatile(
-                "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
-                "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];"
-                : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]), "=r"(v[8]),
-                  "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15]), "=r"(v[16]),
-                  "=r"(v[17]), "=r"(v[18]), "=r"(v[19]), "=r"(v[20]), "=r"(v[21]), "=r"(v[22]), "=r"(v[23]), "=r"(v[24]),
-                  "=r"(v[25]), "=r"(v[26]), "=r"(v[27]), "=r"(v[28]), "=r"(v[29]), "=r"(v[30]), "=r"(v[31])
-                : "r"(taddr) : "memory");
-            asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-            // panel p: row `row` is 128 bytes; 16-byte chunk j sits at position j ^ (row % 8)
-            float4* prow = reinterpret_cast<float4*>(s.c[p] + row * 32);
-#pragma unroll
-            for (int j = 0; j < 8; ++j) {
-                float4* q = prow + (j ^ (row & 7));
-                float4 d = make_float4(__uint_as_float(v[4 * j]), __uint_as_float(v[4 * j + 1]),
-                                       __uint_as_float(v[4 * j + 2]), __uint_as_float(v[4 * j + 3]));
-                if (!kReduce) {
-                    const float4 c = *q;
-                    d.x += c.x; d.y += c.y; d.z += c.z; d.w += c.w;
-                }
-                *q = d;
-            }
+            tmem_ld_32(tmem + ((uint32_t)(warp * 32) << 16) + (uint32_t)(p * 32), v);
+            panel_row_update<!kReduce>(s.c[p], row, v);
         }
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // smem writes -> visible to the TMA engine
     } else {
@@ -385,12 +503,13 @@ __global__ void __launch_bounds__(128) k_dw1_tcgen05(const __grid_constant__ CUt
     if (threadIdx.x == 0) {
         if (!s.failed) {
 #pragma unroll
-            for (int p = 0; p < 4; ++p) {
+            for (int p = 0; p < kPanels; ++p) {
                 if (kReduce) tma_reduce_add_2d(&tm_acc, s.c[p], n0 + p * 32, m0);
                 else tma_store_2d(&tm_acc, s.c[p], n0 + p * 32, m0);
             }
             asm volatile("cp.async.bulk.commit_group;" ::: "memory");
-            asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
+            // shared memory may be released once the engine has read it; the global writes complete on their own
+            asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
         } else {
             atomicExch(status, ABS_ETIMEOUT);
             // give copies that may still be in flight a bounded chance to land before smem is released
@@ -400,7 +519,151 @@ __global__ void __launch_bounds__(128) k_dw1_tcgen05(const __grid_constant__ CUt
     }
     __syncthreads();
     if (warp == 0) {
-        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(kTileN) : "memory");
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(kDwN) : "memory");
+    }
+}
+
+// ============================================================================================
+// dW1, persistent warp-specialised version.  One CTA per SM walks over its share of the
+// 128 x 64 output tiles (hidden index fastest, so neighbouring CTAs share the X^T tile in L2).
+// A kDwStages-deep shared-memory ring holds {A, B, accumulator tile} per tile, so that the
+// loads of the next tiles are always in flight while the current one is added and stored:
+//   warp 0 (one lane)   TMA producer: waits for a free ring slot, loads A, B and the fp32 tile
+//   warp 1 (one lane)   MMA issuer: 4 x tcgen05.mma into one of two TMEM accumulators
+//   warps 2..5          epilogue: tcgen05.ld, add into the swizzled fp32 tile in shared memory,
+//                       TMA store; a ring slot is released once its store has read it
+// The kernel is bound by the read-modify-write of the accumulator (8 bytes per output element).
+// ============================================================================================
+constexpr int kDwStages = 4;
+constexpr int kDwStageBytes = kTileM * 128 + kDwN * 128 + kTileM * kDwN * 4;   // 16 KB + 8 KB + 32 KB
+
+struct DwPersistSmem {
+    alignas(1024) uint8_t stage[kDwStages][kDwStageBytes];   // [A | B | C panel 0 | C panel 1]
+    alignas(8) uint64_t full[kDwStages];
+    uint64_t empty[kDwStages];
+    uint64_t acc_full[2];
+    uint64_t acc_empty[2];
+    uint32_t tmem_base;
+    uint32_t failed;
+    uint32_t stop[2];
+};
+
+__global__ void __launch_bounds__(192) k_dw1_persistent(const __grid_constant__ CUtensorMap tm_xt,
+                                                        const __grid_constant__ CUtensorMap tm_dzt,
+                                                        const __grid_constant__ CUtensorMap tm_acc, int n_tiles_n,
+                                                        int n_tiles, int* status) {
+    extern __shared__ uint8_t smem_raw[];
+    DwPersistSmem& s = *reinterpret_cast<DwPersistSmem*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+    const int warp = threadIdx.x / 32, lane = threadIdx.x % 32;
+    constexpr int kOffB = kTileM * 128, kOffC = kOffB + kDwN * 128;
+    const int my_tiles = (n_tiles - (int)blockIdx.x + (int)gridDim.x - 1) / (int)gridDim.x;
+
+    if (warp == 1) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&s.tmem_base)), "r"(2 * kDwN) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    if (threadIdx.x == 0) {
+        for (int i = 0; i < kDwStages; ++i) {
+            mbar_init(&s.full[i], 1);
+            mbar_init(&s.empty[i], 1);
+        }
+        for (int i = 0; i < 2; ++i) {
+            mbar_init(&s.acc_full[i], 1);
+            mbar_init(&s.acc_empty[i], 128);
+        }
+        s.failed = 0;
+        s.stop[0] = s.stop[1] = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    const uint32_t tmem = s.tmem_base;
+
+    if (warp == 0) {
+        if (lane == 0) {                             // ---- TMA producer
+            for (int i = 0; i < my_tiles; ++i) {
+                const int st = i % kDwStages;
+                if (i >= kDwStages && !mbar_wait(&s.empty[st], ((i / kDwStages) - 1) & 1)) { s.failed = 1; break; }
+                const int t = (int)blockIdx.x + i * (int)gridDim.x;
+                const int n0 = (t % n_tiles_n) * kDwN, m0 = (t / n_tiles_n) * kTileM;
+                uint8_t* base = s.stage[st];
+                mbar_expect_tx(&s.full[st], kDwStageBytes);
+                tma_load_2d(base, &tm_xt, 0, m0, &s.full[st]);
+                tma_load_2d(base + kOffB, &tm_dzt, 0, n0, &s.full[st]);
+#pragma unroll
+                for (int p = 0; p < kPanels; ++p)
+                    tma_load_2d(base + kOffC + p * (kTileM * 128), &tm_acc, n0 + p * 32, m0, &s.full[st]);
+            }
+        }
+    } else if (warp == 1) {
+        if (lane == 0) {                             // ---- MMA issuer
+            constexpr uint32_t idesc = umma_idesc_bf16(kTileM, kDwN);
+            for (int i = 0; i < my_tiles; ++i) {
+                const int st = i % kDwStages, ab = i & 1;
+                if (!mbar_wait(&s.full[st], (i / kDwStages) & 1)) { s.failed = 1; break; }
+                if (i >= 2 && !mbar_wait(&s.acc_empty[ab], ((i / 2) - 1) & 1)) { s.failed = 1; break; }
+                asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                const uint32_t a0 = smem_u32(s.stage[st]);
+                const uint64_t da = umma_desc_k_sw128(a0), db = umma_desc_k_sw128(a0 + kOffB);
+#pragma unroll
+                for (int k = 0; k < kMB / 16; ++k) umma_bf16(tmem + ab * kDwN, da + 2 * k, db + 2 * k, idesc, k > 0);
+                umma_commit(&s.acc_full[ab]);
+            }
+        }
+    } else {                                         // ---- epilogue warps 2..5
+        const int q = warp % 4;                      // TMEM lane quarter this warp may access
+        const int row = q * 32 + lane;
+        const bool leader = (threadIdx.x == 64);
+        for (int i = 0; i < my_tiles; ++i) {
+            const int st = i % kDwStages, ab = i & 1;
+            bool ok = mbar_wait(&s.full[st], (i / kDwStages) & 1);
+            ok = mbar_wait(&s.acc_full[ab], (i / 2) & 1) && ok;
+            ok = __all_sync(0xffffffffu, ok);
+            if (!ok) s.failed = 1;
+            float* cbase = reinterpret_cast<float*>(s.stage[st] + kOffC);
+            if (ok) {
+                asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+#pragma unroll 1
+                for (int p = 0; p < kPanels; ++p) {
+                    uint32_t v[32];
+                    tmem_ld_32(tmem + ((uint32_t)(q * 32) << 16) + (uint32_t)(ab * kDwN + p * 32), v);
+                    panel_row_update<true>(cbase + p * (kTileM * 32), row, v);
+                }
+                asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+                mbar_arrive(&s.acc_empty[ab]);
+                asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+            }
+            // Every epilogue warp reaches this barrier in every iteration (also after a failed wait); the
+            // leader samples the failure flag before it and all four warps act on that one sample after it,
+            // so they leave the loop together.
+            if (leader) s.stop[i & 1] = *reinterpret_cast<volatile uint32_t*>(&s.failed);
+            asm volatile("bar.sync 1, 128;" ::: "memory");
+            if (*reinterpret_cast<volatile uint32_t*>(&s.stop[i & 1])) break;
+            if (leader) {
+                const int t = (int)blockIdx.x + i * (int)gridDim.x;
+                const int n0 = (t % n_tiles_n) * kDwN, m0 = (t / n_tiles_n) * kTileM;
+#pragma unroll
+                for (int p = 0; p < kPanels; ++p) tma_store_2d(&tm_acc, cbase + p * (kTileM * 32), n0 + p * 32, m0);
+                asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+                if (i >= 1) {                        // the previous tile's store has read its slot: release it
+                    asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory");
+                    mbar_arrive(&s.empty[(i - 1) % kDwStages]);
+                }
+            }
+        }
+        if (leader) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
+    }
+    __syncwarp();
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    if (threadIdx.x == 0 && s.failed) {
+        atomicExch(status, ABS_ETIMEOUT);
+        for (int i = 0; i < kDwStages; ++i) mbar_wait(&s.full[i], 0);   // bounded chance for copies in flight to land
+    }
+    __syncthreads();
+    if (warp == 1) {
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(2 * kDwN) : "memory");
     }
 }
 
@@ -417,16 +680,6 @@ __global__ void __launch_bounds__(128) k_dw1_tcgen05(const __grid_constant__ CUt
 // ============================================================================================
 constexpr int kFwdStages = 6;
 constexpr int kFwdStageBytes = 2 * 8192 + 8192;   // two A boxes + one B box
-
-__device__ __forceinline__ uint64_t umma_desc_mn_sw128(uint32_t smem_addr, uint32_t lbo_bytes) {
-    uint64_t d = 0;
-    d |= (uint64_t)((smem_addr & 0x3FFFF) >> 4);
-    d |= (uint64_t)(lbo_bytes >> 4) << 16;                // leading-dim byte offset: next 64-wide MN block
-    d |= (uint64_t)(1024 >> 4) << 32;                     // stride-dim byte offset: next group of 8 k-rows
-    d |= (uint64_t)1 << 46;
-    d |= (uint64_t)2 << 61;
-    return d;
-}
 
 struct FwdSmem {
     alignas(1024) uint8_t stage[kFwdStages][kFwdStageBytes];   // [A h0..63 | A h64..127 | B]
@@ -488,18 +741,11 @@ __global__ void __launch_bounds__(128) k_fwd1_tcgen05(const __grid_constant__ CU
             const uint32_t a0 = smem_u32(s.stage[st]);
             const uint64_t db = umma_desc_k_sw128(a0 + 16384);
 #pragma unroll
-            for (int k = 0; k < 4; ++k) {
-                const uint64_t da = umma_desc_mn_sw128(a0 + k * 2048, 8192);
-                const uint32_t accumulate = (kb > 0 || k > 0);
-                asm volatile(
-                    "{\n .reg .pred p;\n setp.ne.b32 p, %4, 0;\n"
-                    " tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n}\n"
-                    ::"r"(tmem), "l"(da), "l"(db + 2 * k), "r"(idesc), "r"(accumulate) : "memory");
-            }
-            // frees the stage for the producer once these MMAs have read it
-            asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(&s.empty[st])) : "memory");
+            for (int k = 0; k < 4; ++k)
+                umma_bf16(tmem, umma_desc_mn_sw128(a0 + k * 2048, 8192), db + 2 * k, idesc, (kb > 0 || k > 0));
+            umma_commit(&s.empty[st]);               // frees the stage once these MMAs have read it
         }
-        if (ok) asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(&s.done)) : "memory");
+        if (ok) umma_commit(&s.done);
         else s.failed = 1;
     }
     __syncwarp();
@@ -513,16 +759,7 @@ __global__ void __launch_bounds__(128) k_fwd1_tcgen05(const __grid_constant__ CU
 #pragma unroll 1
         for (int p = 0; p < 2; ++p) {
             uint32_t v[32];
-            const uint32_t taddr = tmem + ((uint32_t)(warp * 32) << 16) + (uint32_t)(p * 32);
-            asm volatile(
-                "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
-                "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];"
-                : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]), "=r"(v[8]),
-                  "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15]), "=r"(v[16]),
-                  "=r"(v[17]), "=r"(v[18]), "=r"(v[19]), "=r"(v[20]), "=r"(v[21]), "=r"(v[22]), "=r"(v[23]), "=r"(v[24]),
-                  "=r"(v[25]), "=r"(v[26]), "=r"(v[27]), "=r"(v[28]), "=r"(v[29]), "=r"(v[30]), "=r"(v[31])
-                : "r"(taddr) : "memory");
-            asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+            tmem_ld_32(tmem + ((uint32_t)(warp * 32) << 16) + (uint32_t)(p * 32), v);
 #pragma unroll
             for (int j = 0; j < 8; ++j)
                 *reinterpret_cast<float4*>(out + p * 32 + 4 * j) =
@@ -573,44 +810,51 @@ bool encode_2d(CUtensorMap* tm, CUtensorMapDataType dt, int esize, void* base, u
 
 size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 
-}  // namespace
-
-size_t mlp_scratch_bytes(const MlpDims& d) {
+// One description of the scratch layout, used for sizing (base == nullptr) and for carving.
+size_t layout_scratch(MlpScratch* s, const MlpDims& d, char* base) {
     size_t o = 0;
-    auto take = [&](size_t b) { o = align_up(o + b, 1024); };
-    take((size_t)kMB * d.d_in * 2);                 // xb
-    take((size_t)d.d_in * kMB * 2);                 // xtb
-    take((size_t)kSplitK * d.d_hidden * kMB * 4);   // zpart
-    take((size_t)d.d_hidden * kMB * 4);             // zt
-    take((size_t)d.d_hidden * kMB * 2);             // hbt
-    take((size_t)d.d_hidden * kMB * 2);             // dzt
-    take((size_t)(d.d_hidden / kChunkH) * kMB * kOutPad * 4);   // lpart
-    take((size_t)kMB * kOutPad * 4);                // dl
-    take((size_t)kMB * kOutPad * 2);                // dlb
-    take(256);                                      // status word
+    auto take = [&](size_t b) { char* at = base ? base + o : nullptr; o = align_up(o + b, 1024); return at; };
+    const int n_cta = d.d_hidden / kHB;
+    const int n_groups = (n_cta + kGroup - 1) / kGroup;
+    char* xb = take((size_t)kMB * d.d_in * 2);
+    char* xtb = take((size_t)d.d_in * kMB * 2);
+    char* zpart = take((size_t)kSplitK * d.d_hidden * kMB * 4);
+    char* hbt = take((size_t)d.d_hidden * kMB * 2);
+    char* dzt = take((size_t)d.d_hidden * kMB * 2);
+    char* lpart = take((size_t)n_cta * kMB * kOutPad * 4);
+    char* gpart = take((size_t)n_groups * kMB * kOutPad * 4);
+    char* dlb = take((size_t)kMB * kOutPad * 2);
+    char* tickets = take((size_t)(n_groups + 1) * 4);
+    char* status = take(256);
+    if (s) {
+        s->xb = reinterpret_cast<__nv_bfloat16*>(xb);
+        s->xtb = reinterpret_cast<__nv_bfloat16*>(xtb);
+        s->zpart = reinterpret_cast<float*>(zpart);
+        s->hbt = reinterpret_cast<__nv_bfloat16*>(hbt);
+        s->dzt = reinterpret_cast<__nv_bfloat16*>(dzt);
+        s->lpart = reinterpret_cast<float*>(lpart);
+        s->gpart = reinterpret_cast<float*>(gpart);
+        s->dlb = reinterpret_cast<__nv_bfloat16*>(dlb);
+        s->tickets = reinterpret_cast<unsigned int*>(tickets);
+        s->status = reinterpret_cast<int*>(status);
+        s->zero_from = tickets;
+        s->zero_bytes = (size_t)(status + 256 - tickets);
+    }
     return o;
 }
 
+}  // namespace
+
+size_t mlp_scratch_bytes(const MlpDims& d) { return layout_scratch(nullptr, d, nullptr); }
+
 cudaError_t mlp_scratch_init(MlpScratch* s, const MlpDims& d, void* base, __nv_bfloat16* shadow0,
                              __nv_bfloat16* shadow1, const char** err) {
-    char* p = static_cast<char*>(base);
-    size_t o = 0;
-    auto take = [&](size_t b) { char* at = p + o; o = align_up(o + b, 1024); return at; };
-    s->xb = reinterpret_cast<__nv_bfloat16*>(take((size_t)kMB * d.d_in * 2));
-    s->xtb = reinterpret_cast<__nv_bfloat16*>(take((size_t)d.d_in * kMB * 2));
-    s->zpart = reinterpret_cast<float*>(take((size_t)kSplitK * d.d_hidden * kMB * 4));
-    s->zt = reinterpret_cast<float*>(take((size_t)d.d_hidden * kMB * 4));
-    s->hbt = reinterpret_cast<__nv_bfloat16*>(take((size_t)d.d_hidden * kMB * 2));
-    s->dzt = reinterpret_cast<__nv_bfloat16*>(take((size_t)d.d_hidden * kMB * 2));
-    s->lpart = reinterpret_cast<float*>(take((size_t)(d.d_hidden / kChunkH) * kMB * kOutPad * 4));
-    s->dl = reinterpret_cast<float*>(take((size_t)kMB * kOutPad * 4));
-    s->dlb = reinterpret_cast<__nv_bfloat16*>(take((size_t)kMB * kOutPad * 2));
-    s->status = reinterpret_cast<int*>(take(256));
+    layout_scratch(s, d, static_cast<char*>(base));
     static_assert(sizeof(CUtensorMap) == sizeof(TmapBytes), "tensor map size");
     if (!encode_2d(reinterpret_cast<CUtensorMap*>(&s->tmap_xt), CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, s->xtb, d.d_in, kMB,
                    kTileM, kMB) ||
         !encode_2d(reinterpret_cast<CUtensorMap*>(&s->tmap_dzt), CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, s->dzt, d.d_hidden,
-                   kMB, kTileN, kMB)) {
+                   kMB, kDwN, kMB)) {
         *err = "cuTensorMapEncodeTiled failed for the dW1 operands";
         return cudaErrorInvalidValue;
     }
@@ -624,17 +868,18 @@ cudaError_t mlp_scratch_init(MlpScratch* s, const MlpDims& d, void* base, __nv_b
         *err = "cuTensorMapEncodeTiled failed for the forward GEMM operands";
         return cudaErrorInvalidValue;
     }
-    cudaError_t e0 = cudaFuncSetAttribute(k_fwd1_tcgen05, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                          (int)sizeof(FwdSmem) + 1024);
-    if (e0 != cudaSuccess) {
-        *err = "cudaFuncSetAttribute(forward kernel)";
-        return e0;
-    }
-    cudaError_t e = cudaFuncSetAttribute(k_dw1_tcgen05<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                         (int)sizeof(DwSmem) + 1024);
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e == cudaSuccess) e = cudaDeviceGetAttribute(&s->num_sms, cudaDevAttrMultiProcessorCount, dev);
+    if (e == cudaSuccess)
+        e = cudaFuncSetAttribute(k_dw1_persistent, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(DwPersistSmem) + 1024);
+    if (e == cudaSuccess)
+        e = cudaFuncSetAttribute(k_fwd1_tcgen05, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(FwdSmem) + 1024);
+    if (e == cudaSuccess)
+        e = cudaFuncSetAttribute(k_dw1_tcgen05<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(DwSmem) + 1024);
     if (e == cudaSuccess)
         e = cudaFuncSetAttribute(k_dw1_tcgen05<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(DwSmem) + 1024);
-    if (e != cudaSuccess) *err = "cudaFuncSetAttribute(dW1 kernel)";
+    if (e != cudaSuccess) *err = "cudaFuncSetAttribute(tcgen05 kernels)";
     return e;
 }
 
@@ -646,15 +891,14 @@ cudaError_t mlp_make_acc_tmap(void* tmap_out, const MlpDims& d, float* acc_row) 
                : cudaErrorInvalidValue;
 }
 
-cudaError_t launch_mlp_grad(const MlpDims& d, const MlpScratch& s, const float* x_pub, const __nv_bfloat16* shadow,
-                            int shadow_idx, const float* x_dev, const int32_t* y_dev, float* acc_row, const void* acc_tmap,
-                            int32_t* cnt, int variant, cudaStream_t stream, void (*mark)(void*, int, int), void* user) {
+cudaError_t launch_mlp_front(const MlpDims& d, const MlpScratch& s, const float* x_pub, const __nv_bfloat16* shadow,
+                             int shadow_idx, const float* x_dev, const int32_t* y_dev, float* acc_row, int32_t* cnt,
+                             int variant, cudaStream_t stream, MlpMark mark, void* user) {
     const size_t o_b1 = (size_t)d.d_in * d.d_hidden, o_w2 = o_b1 + d.d_hidden, o_b2 = o_w2 + (size_t)d.d_hidden * d.d_out;
-    const int n_chunks = d.d_hidden / kChunkH;
     cudaError_t e;
 
-    mark(user, ABS_K_MLP_FWD, 0);
-    k_cast_x<<<d.d_in / 64, 256, 0, stream>>>(x_dev, s.xb, s.xtb, d.d_in);
+    mark(user, ABS_K_MLP_FWD, 0, stream);
+    k_cast_x<<<d.d_in / 16, 256, 0, stream>>>(x_dev, s.xb, s.xtb, d.d_in);
     // every K split must be a whole number of 64-wide pipeline steps (d_in is a multiple of 128)
     const int nsplit = (d.d_in % (64 * kSplitK) == 0) ? kSplitK : 2;
     if (variant & 2) {
@@ -665,28 +909,35 @@ cudaError_t launch_mlp_grad(const MlpDims& d, const MlpScratch& s, const float* 
         k_fwd1_tcgen05<<<dim3(d.d_hidden / 128, nsplit), 128, sizeof(FwdSmem) + 1024, stream>>>(*tw, *tx, s.zpart, d.d_in,
                                                                                            d.d_hidden, s.status);
     }
-    k_fwd2<<<n_chunks, 256, 0, stream>>>(s.zpart, x_pub + o_b1, shadow + o_w2, s.zt, s.hbt, s.lpart, d.d_hidden, d.d_out,
-                                         nsplit);
-    k_loss<<<1, kMB, 0, stream>>>(s.lpart, n_chunks, x_pub + o_b2, y_dev, s.dl, s.dlb, acc_row + o_b2, d.d_out);
-    mark(user, ABS_K_MLP_FWD, 4);
+    k_fwd2<<<d.d_hidden / kHB, 256, 0, stream>>>(s.zpart, nsplit, x_pub + o_b1, shadow + o_w2, x_pub + o_b2, y_dev, s.hbt,
+                                                 s.lpart, s.gpart, s.tickets, s.dlb, acc_row + o_b2, d.d_hidden, d.d_out);
+    mark(user, ABS_K_MLP_FWD, 3, stream);
     if ((e = cudaGetLastError()) != cudaSuccess) return e;
 
-    mark(user, ABS_K_MLP_BWD, 0);
-    k_bwd<<<d.d_hidden / 8, 512, 0, stream>>>(s.zt, s.hbt, s.dlb, shadow + o_w2, s.dzt, acc_row + o_b1, acc_row + o_w2, cnt,
-                                              d.d_out);
-    mark(user, ABS_K_MLP_BWD, 1);
-    if ((e = cudaGetLastError()) != cudaSuccess) return e;
+    mark(user, ABS_K_MLP_BWD, 0, stream);
+    k_bwd<<<d.d_hidden / kHB, 256, 0, stream>>>(s.hbt, s.dlb, shadow + o_w2, s.dzt, acc_row + o_b1, acc_row + o_w2, cnt,
+                                                d.d_out);
+    mark(user, ABS_K_MLP_BWD, 1, stream);
+    return cudaGetLastError();
+}
 
-    mark(user, ABS_K_MLP_DW1, 0);
-    const dim3 grid(d.d_hidden / kTileN, d.d_in / kTileM);
+cudaError_t launch_mlp_dw1(const MlpDims& d, const MlpScratch& s, const void* acc_tmap, int variant, cudaStream_t stream,
+                           MlpMark mark, void* user) {
+    mark(user, ABS_K_MLP_DW1, 0, stream);
+    const dim3 grid(d.d_hidden / kDwN, d.d_in / kTileM);
     const CUtensorMap* ta = reinterpret_cast<const CUtensorMap*>(&s.tmap_xt);
     const CUtensorMap* tb = reinterpret_cast<const CUtensorMap*>(&s.tmap_dzt);
     const CUtensorMap* tc = reinterpret_cast<const CUtensorMap*>(acc_tmap);
-    if (variant & 1)
+    if (variant & 4) {
+        const int n_tiles_n = d.d_hidden / kDwN, n_tiles = n_tiles_n * (d.d_in / kTileM);
+        const int ctas = n_tiles < s.num_sms ? n_tiles : s.num_sms;
+        k_dw1_persistent<<<ctas, 192, sizeof(DwPersistSmem) + 1024, stream>>>(*ta, *tb, *tc, n_tiles_n, n_tiles, s.status);
+    } else if (variant & 1) {
         k_dw1_tcgen05<true><<<grid, 128, sizeof(DwSmem) + 1024, stream>>>(*ta, *tb, *tc, s.status);
-    else
+    } else {
         k_dw1_tcgen05<false><<<grid, 128, sizeof(DwSmem) + 1024, stream>>>(*ta, *tb, *tc, s.status);
-    mark(user, ABS_K_MLP_DW1, 1);
+    }
+    mark(user, ABS_K_MLP_DW1, 1, stream);
     return cudaGetLastError();
 }
 
