@@ -59,6 +59,7 @@ class ClockSampler:
         self.gpu = gpu_index
         self.proc = None
         self.path = None
+        self.skip = 0
 
     def start(self):
         try:
@@ -66,7 +67,13 @@ class ClockSampler:
             os.close(fd)
             self.proc = subprocess.Popen(
                 ["nvidia-smi", f"--id={self.gpu}", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits",
-                 "-lms", "100"], stdout=open(self.path, "w"), stderr=subprocess.DEVNULL)
+                 "-lms", "50"], stdout=open(self.path, "w"), stderr=subprocess.DEVNULL)
+            # nvidia-smi takes a few hundred ms to start: wait for its first (idle) sample so that the
+            # samples that follow fall inside the timed region
+            t0 = time.time()
+            while time.time() - t0 < 5.0 and os.path.getsize(self.path) == 0:
+                time.sleep(0.02)
+            self.skip = sum(1 for _ in open(self.path))
         except Exception:
             self.proc = None
 
@@ -81,7 +88,9 @@ class ClockSampler:
             self.proc.kill()
         sm, mx, reasons = [], [], set()
         try:
-            for line in open(self.path):
+            for n, line in enumerate(open(self.path)):
+                if n < self.skip:
+                    continue
                 f = [s.strip() for s in line.split(",")]
                 if len(f) < 9:
                     continue
@@ -215,8 +224,9 @@ def run_ours(args):
     eng = make(pipelined=True)
     sampler = ClockSampler(local_rank if "CUDA_VISIBLE_DEVICES" not in os.environ else
                            int(os.environ["CUDA_VISIBLE_DEVICES"].split(",")[local_rank]))
+    timed(eng, 2, args.warmup)              # warm-up (also outside the clock samples)
     sampler.start()
-    secs, launches = timed(eng, args.steps, args.warmup)
+    secs, launches = timed(eng, args.steps, 0)
     clocks = sampler.stop()
     value, worst = D.aggregate_throughput(step_bytes * args.steps / 1e9, secs, dev)
 
@@ -280,9 +290,10 @@ def run_ours(args):
 
 
 def run_mlp(B, wlm, dev, peaks, iters=12):
-    """Secondary measurement on the MLP workload (3072-4096-10, W=4, b_i ~ U{1..8}): per-kernel-class
-    durations of the micro-batch gradient, and the dW1 = X^T dZ GEMM (M=3072, N=4096, K=64) as TFLOP/s
-    and as HBM GB/s -- with K = 64 it is bound by the read-modify-write of the fp32 accumulator slice."""
+    """Secondary measurement on the MLP workload (3072-4096-10, W=4, b_i ~ U{1..8}): time per micro-batch
+    of the whole gradient (dW1 overlapping the next micro-batch's front part), and -- in serial mode, every
+    kernel alone on the GPU -- per-kernel-class durations, with the dW1 = X^T dZ GEMM (M=3072, N=4096, K=64)
+    as TFLOP/s and as HBM GB/s: with K = 64 it is bound by the read-modify-write of the fp32 accumulator."""
     import torch
 
     wl = wlm.config(4, T=iters)
@@ -293,45 +304,53 @@ def run_mlp(B, wlm, dev, peaks, iters=12):
     xp = [xs_d[b].data_ptr() for b in range(wl.mlp_pool)]      # raw device addresses of the micro-batches
     yp = [ys_d[b].data_ptr() for b in range(wl.mlp_pool)]
     torch.cuda.synchronize()
-    out = {"workload": "cfg4 mlp 3072-4096-10, mb=64, W=4, b_i~U{1..8}, pipelined", "iterations": iters}
-    for name, epi in (("tma_load_add_store", 0), ("tma_reduce_add", 1), ("persistent", 4)):
-        eng = B.AbsSgd(x0_d, wl.W, wl.lr, wl.momentum, wl.weight_decay, pipelined=True, mlp=(d.d_in, d.d_hidden, d.d_out, d.mb))
-        eng.set_launch(B.K_MLP_DW1, epi)
-        calls = list(wlm.iter_calls(wl))
+    calls = list(wlm.iter_calls(wl))
+    flop = 2.0 * d.d_in * d.d_hidden * d.mb
+    rmw_bytes = 8.0 * d.d_in * d.d_hidden + 2.0 * d.mb * (d.d_in + d.d_hidden)
+    out = {"workload": "cfg4 mlp 3072-4096-10, mb=64, W=4, b_i~U{1..8}, pipelined", "iterations": iters,
+           "dw1_flop": flop, "dw1_algorithmic_bytes": rmw_bytes}
+    for name, variant in (("tma_load_add_store", 0), ("tma_reduce_add", 1), ("persistent", 4), ("register_prefetch", 8)):
+        res = {}
+        for serial in (0, 1):
+            eng = B.AbsSgd(x0_d, wl.W, wl.lr, wl.momentum, wl.weight_decay, pipelined=True,
+                           mlp=(d.d_in, d.d_hidden, d.d_out, d.mb))
+            eng.set_launch(B.K_MLP_DW1, variant)
+            eng.set_launch(B.K_MLP_FWD, serial)
 
-        def run(profile):
-            eng.profile(profile)
-            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-            n = 0
-            with torch.cuda.stream(eng.stream_acc):
-                e0.record()
-                for it in calls:
-                    for (i, k, c) in it:
-                        eng.accumulate_mlp(i, xp[c % wl.mlp_pool], yp[c % wl.mlp_pool]); n += 1
-                    eng.sync_step()
-                eng.wait()
-                e1.record()
-            torch.cuda.synchronize()
-            return e0.elapsed_time(e1), n
+            def run(profile):
+                eng.profile(profile)
+                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                n = 0
+                with torch.cuda.stream(eng.stream_acc):
+                    e0.record()
+                    for it in calls:
+                        for (i, k, c) in it:
+                            eng.accumulate_mlp(i, xp[c % wl.mlp_pool], yp[c % wl.mlp_pool]); n += 1
+                        eng.sync_step()
+                    eng.wait()
+                    e1.record()
+                torch.cuda.synchronize()
+                return e0.elapsed_time(e1), n
 
-        run(False)                                  # warm-up
-        ms_total, n_mb = run(False)
-        run(True)
-        stats = {nm: eng.kernel_stats(k) for nm, k in (("fwd", B.K_MLP_FWD), ("bwd", B.K_MLP_BWD), ("dw1", B.K_MLP_DW1), ("sync", B.K_SYNC))}
-        eng.check()
-        eng.destroy()
-        n_dw, ms_dw = stats["dw1"]
-        us_dw = ms_dw / n_dw * 1e3
-        flop = 2.0 * d.d_in * d.d_hidden * d.mb
-        rmw_bytes = 8.0 * d.d_in * d.d_hidden + 2.0 * d.mb * (d.d_in + d.d_hidden)
-        out[name] = {
-            "us_per_microbatch_all_kernels": ms_total / n_mb * 1e3,
-            "us_fwd": stats["fwd"][1] / max(stats["fwd"][0], 1) * 1e3, "us_bwd": stats["bwd"][1] / max(stats["bwd"][0], 1) * 1e3,
-            "us_dw1": us_dw, "us_sync": stats["sync"][1] / max(stats["sync"][0], 1) * 1e3,
-            "dw1_tflops": flop / us_dw / 1e6, "dw1_frac_of_bf16_peak_sustained": flop / us_dw / 1e6 / peaks["bf16_tflops_sustained"],
-            "dw1_hbm_gbs": rmw_bytes / us_dw / 1e3, "dw1_frac_of_hbm": rmw_bytes / us_dw / 1e3 / peaks["hbm_gbs"],
-            "microbatches": n_mb,
-        }
+            run(False)                                  # warm-up
+            ms_total, n_mb = run(False)
+            if not serial:
+                res["us_per_microbatch_overlapped"] = ms_total / n_mb * 1e3
+                res["microbatches"] = n_mb
+            else:
+                res["us_per_microbatch_serial"] = ms_total / n_mb * 1e3
+                run(True)
+                st = {nm: eng.kernel_stats(k) for nm, k in (("fwd", B.K_MLP_FWD), ("bwd", B.K_MLP_BWD),
+                                                            ("dw1", B.K_MLP_DW1), ("sync", B.K_SYNC))}
+                us = {nm: v[1] / max(v[0], 1) * 1e3 for nm, v in st.items()}
+                res.update({"us_fwd_3_kernels": us["fwd"], "us_bwd": us["bwd"], "us_dw1": us["dw1"], "us_sync": us["sync"],
+                            "dw1_tflops": flop / us["dw1"] / 1e6,
+                            "dw1_frac_of_bf16_peak_sustained": flop / us["dw1"] / 1e6 / peaks["bf16_tflops_sustained"],
+                            "dw1_hbm_gbs": rmw_bytes / us["dw1"] / 1e3,
+                            "dw1_frac_of_hbm": rmw_bytes / us["dw1"] / 1e3 / peaks["hbm_gbs"]})
+            eng.check()
+            eng.destroy()
+        out[name] = res
     return out
 
 

@@ -175,9 +175,13 @@ int abs_wait(abs_ctx *ctx);
 int abs_check(abs_ctx *ctx);
 
 /* Launch shape of a kernel class: CTAs per SM for the persistent grid (0 = default, -1 = one
- * tile per CTA).  For ABS_K_MLP_DW1 the value is a bit mask of MLP kernel variants instead:
- * bit 0 = dW1 epilogue by TMA reduce-add (default: TMA load + add + TMA store of the accumulator
- * tile); bit 1 = forward GEMM on CUDA cores (default: tcgen05).  Results agree within rounding. */
+ * tile per CTA) for ABS_K_ACCUMULATE and ABS_K_SYNC.  For the MLP classes the value selects
+ * kernel variants instead (results agree within rounding):
+ *   ABS_K_MLP_DW1  bit mask: 1 = dW1 epilogue by TMA reduce-add (default: TMA load + add + TMA store);
+ *                  2 = forward GEMM on CUDA cores (default: tcgen05); 4 = persistent warp-specialised
+ *                  dW1 kernel; 8 = dW1 with the accumulator tile prefetched into registers.
+ *   ABS_K_MLP_FWD  1 = serial mode: the dW1 GEMM runs on stream_acc instead of overlapping the next
+ *                  micro-batch on the internal stream (for per-kernel timing). */
 int abs_set_launch(abs_ctx *ctx, int kernel_class, int ctas_per_sm);
 
 /* Per-kernel timing with CUDA events on the launching stream.  abs_profile(ctx, 1) starts

@@ -332,7 +332,11 @@ int abs_init(abs_ctx** out, const abs_config* cfg, void* workspace_dev, size_t w
             if ((e = cudaEventCreateWithFlags(&c->ev_front_done[k], cudaEventDisableTiming)) != cudaSuccess) return bail(e, "cudaEventCreate");
             if ((e = cudaEventCreateWithFlags(&c->ev_dw_done[k], cudaEventDisableTiming)) != cudaSuccess) return bail(e, "cudaEventCreate");
         }
-        if ((e = cudaStreamCreateWithFlags(&c->s_dw, cudaStreamNonBlocking)) != cudaSuccess) return bail(e, "cudaStreamCreate");
+        // Lowest priority: when CTA slots free up, the short front kernels of the next micro-batch (on
+        // stream_acc) are placed before the remaining CTAs of the long, bandwidth-bound dW1 kernel.
+        int prio_lo = 0, prio_hi = 0;
+        if ((e = cudaDeviceGetStreamPriorityRange(&prio_lo, &prio_hi)) != cudaSuccess) return bail(e, "cudaDeviceGetStreamPriorityRange");
+        if ((e = cudaStreamCreateWithPriority(&c->s_dw, cudaStreamNonBlocking, prio_lo)) != cudaSuccess) return bail(e, "cudaStreamCreate");
         c->acc_tmaps.resize((size_t)2 * cfg->W);
         for (uint32_t set = 0; set < 2; ++set)
             for (uint32_t i = 0; i < cfg->W; ++i)
@@ -408,17 +412,27 @@ int abs_accumulate_mlp(abs_ctx* c, uint32_t worker, const float* x_dev, const in
     const int k = c->mlp_slot;
     c->mlp_slot ^= 1;
     const int variant = c->ctas_per_sm[ABS_K_MLP_DW1];
-    if (c->slot_used[k]) CK(cudaStreamWaitEvent(c->s_acc, c->ev_dw_done[k], 0));   // scratch set k is free again
-    CK(launch_mlp_front(c->mlp_dims, c->mlp_scratch[k], c->x(c->pub), c->shadow(c->pub), c->pub, x_dev, y_dev,
-                        c->acc(c->cur, worker), c->cnt(c->cur, worker), variant, c->s_acc, mlp_mark, c));
-    CK(cudaEventRecord(c->ev_front_done[k], c->s_acc));
-    CK(cudaStreamWaitEvent(c->s_dw, c->ev_front_done[k], 0));
-    CK(launch_mlp_dw1(c->mlp_dims, c->mlp_scratch[k], &c->acc_tmaps[(size_t)c->cur * c->cfg.W + worker], variant, c->s_dw,
-                      mlp_mark, c));
-    CK(cudaEventRecord(c->ev_dw_done[k], c->s_dw));
-    c->slot_used[k] = true;
-    c->dw_outstanding = true;
-    c->dw_last_slot = k;
+    if (c->ctas_per_sm[ABS_K_MLP_FWD] == 1) {
+        // serial mode (measurement aid): everything on stream_acc, no overlap between micro-batches
+        if (int rc = join_dw(c)) return rc;
+        CK(launch_mlp_front(c->mlp_dims, c->mlp_scratch[k], c->x(c->pub), c->shadow(c->pub), c->pub, x_dev, y_dev,
+                            c->acc(c->cur, worker), c->cnt(c->cur, worker), variant, c->s_acc, mlp_mark, c));
+        CK(launch_mlp_dw1(c->mlp_dims, c->mlp_scratch[k], c->acc(c->cur, worker),
+                          &c->acc_tmaps[(size_t)c->cur * c->cfg.W + worker], variant, c->s_acc, mlp_mark, c));
+        c->slot_used[0] = c->slot_used[1] = false;
+    } else {
+        if (c->slot_used[k]) CK(cudaStreamWaitEvent(c->s_acc, c->ev_dw_done[k], 0));   // scratch set k is free again
+        CK(launch_mlp_front(c->mlp_dims, c->mlp_scratch[k], c->x(c->pub), c->shadow(c->pub), c->pub, x_dev, y_dev,
+                            c->acc(c->cur, worker), c->cnt(c->cur, worker), variant, c->s_acc, mlp_mark, c));
+        CK(cudaEventRecord(c->ev_front_done[k], c->s_acc));
+        CK(cudaStreamWaitEvent(c->s_dw, c->ev_front_done[k], 0));
+        CK(launch_mlp_dw1(c->mlp_dims, c->mlp_scratch[k], c->acc(c->cur, worker),
+                          &c->acc_tmaps[(size_t)c->cur * c->cfg.W + worker], variant, c->s_dw, mlp_mark, c));
+        CK(cudaEventRecord(c->ev_dw_done[k], c->s_dw));
+        c->slot_used[k] = true;
+        c->dw_outstanding = true;
+        c->dw_last_slot = k;
+    }
     c->h_cnt[(size_t)c->cur * c->cfg.W + worker] += 1;
     return ABS_OK;
 }

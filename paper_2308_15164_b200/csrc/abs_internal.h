@@ -75,14 +75,15 @@ cudaError_t mlp_make_acc_tmap(void* tmap_out, const MlpDims& d, float* acc_row);
 //          into acc_row; bumps cnt);   dw1: the dW1 GEMM, which reads xtb/dzt and adds into the W1 slice.
 // shadow: bf16 copy of the published parameters (same flat layout), shadow_idx: which of the two copies it is.
 // x_pub: the fp32 parameters.  variant: bit 0 = dW1 epilogue by TMA reduce-add (else TMA load + add + TMA
-// store); bit 1 = forward GEMM on CUDA cores (cross-check of the tcgen05 one); bit 2 = persistent dW1 kernel.
+// store); bit 1 = forward GEMM on CUDA cores (cross-check of the tcgen05 one); bit 2 = persistent dW1 kernel;
+// bit 3 = dW1 with the accumulator tile prefetched into registers by plain coalesced loads.
 // mark(user, kernel_class, 0, stream) is called before a kernel group, mark(user, kernel_class, n, stream) after
 // its n launches.
 typedef void (*MlpMark)(void* user, int kernel_class, int n, cudaStream_t stream);
 cudaError_t launch_mlp_front(const MlpDims& d, const MlpScratch& s, const float* x_pub, const __nv_bfloat16* shadow,
                              int shadow_idx, const float* x_dev, const int32_t* y_dev, float* acc_row, int32_t* cnt,
                              int variant, cudaStream_t stream, MlpMark mark, void* user);
-cudaError_t launch_mlp_dw1(const MlpDims& d, const MlpScratch& s, const void* acc_tmap, int variant, cudaStream_t stream,
-                           MlpMark mark, void* user);
+cudaError_t launch_mlp_dw1(const MlpDims& d, const MlpScratch& s, float* acc_row, const void* acc_tmap, int variant,
+                           cudaStream_t stream, MlpMark mark, void* user);
 
 }  // namespace abs_sgd

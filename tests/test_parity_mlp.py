@@ -75,7 +75,8 @@ def _check_gradient(got_flat, params, X, y, dims):
     return len(amb)
 
 
-@pytest.mark.parametrize("epilogue", [0, 1, 2, 4], ids=["tma-load-add-store", "tma-reduce", "cuda-core-forward", "persistent-dw1"])
+@pytest.mark.parametrize("epilogue", [0, 1, 2, 4, 8],
+                         ids=["tma-load-add-store", "tma-reduce", "cuda-core-forward", "persistent-dw1", "register-prefetch-dw1"])
 @pytest.mark.parametrize("small", [True, False], ids=["384x512", "3072x4096"])
 def test_single_microbatch_gradient(small, epilogue):
     wl = wlm.config(4, small=small)
