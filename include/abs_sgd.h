@@ -158,6 +158,13 @@ int abs_counters(abs_ctx *ctx, int32_t *cnt_host, uint32_t *cur, uint64_t *t);
  * cleared them.  b_host[W].  Blocks until the logging kernel has finished. */
 int abs_consumed(abs_ctx *ctx, uint64_t step, int32_t *b_host);
 
+/* Algorithm 1, Step 2 loop condition "while Step 1 not finished": *done = 0 while the fused kernel
+ * launched by the last abs_sync_step (pipelined mode) is still running, 1 once it has completed
+ * (always 1 in eager mode or when nothing is in flight).  Never blocks.  A driver that keeps
+ * calling abs_accumulate* until *done becomes 1 gets the paper's adaptive batch size: b_i is
+ * whatever the workers managed to compute while the synchronisation ran. */
+int abs_step1_finished(abs_ctx *ctx, int *done);
+
 /* gamma may change between iterations (Theorem 1 allows gamma_t).  The rate travels with the
  * gradients: the value in effect when abs_sync_step ends iteration t is the one used to apply
  * that iteration's gradients, i.e. it is the paper's gamma_{t+1} (x_{t+2} = x_{t+1} - gamma_{t+1} *

@@ -58,6 +58,7 @@ _sig = {
     "abs_counters": (ctypes.c_int, [_vp, _vp, ctypes.POINTER(_u32), ctypes.POINTER(_u64)]),
     "abs_consumed": (ctypes.c_int, [_vp, _u64, _vp]),
     "abs_set_lr": (ctypes.c_int, [_vp, ctypes.c_float]),
+    "abs_step1_finished": (ctypes.c_int, [_vp, ctypes.POINTER(ctypes.c_int)]),
     "abs_wait": (ctypes.c_int, [_vp]),
     "abs_check": (ctypes.c_int, [_vp]),
     "abs_set_launch": (ctypes.c_int, [_vp, ctypes.c_int, ctypes.c_int]),
@@ -182,6 +183,11 @@ class AbsSgd:
         b = np.zeros(self.W, dtype=np.int32)
         self._ck(lib.abs_consumed(self._h, step, b.ctypes.data))
         return b
+
+    def step1_finished(self) -> bool:
+        done = ctypes.c_int(1)
+        self._ck(lib.abs_step1_finished(self._h, ctypes.byref(done)))
+        return bool(done.value)
 
     def set_lr(self, lr: float):
         self._ck(lib.abs_set_lr(self._h, lr))

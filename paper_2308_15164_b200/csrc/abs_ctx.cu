@@ -542,6 +542,18 @@ int abs_consumed(abs_ctx* c, uint64_t step, int32_t* b_host) {
     return ABS_OK;
 }
 
+int abs_step1_finished(abs_ctx* c, int* done) {
+    if (!live(c)) return ABS_ESTATE;
+    if (!done) return invalid(c, "output pointer is NULL");
+    *done = 1;
+    if (c->pipelined && c->pending) {
+        const cudaError_t e = cudaEventQuery(c->ev_sync_done);
+        if (e == cudaErrorNotReady) *done = 0;
+        else if (e != cudaSuccess) return cuda_fail(c, e, "cudaEventQuery");
+    }
+    return ABS_OK;
+}
+
 int abs_set_lr(abs_ctx* c, float lr) {
     if (!live(c)) return ABS_ESTATE;
     if (!std::isfinite(lr)) return invalid(c, "lr must be finite");

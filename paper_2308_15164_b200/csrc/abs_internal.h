@@ -55,8 +55,7 @@ struct MlpScratch {      // device pointers carved from the workspace (all hidde
     __nv_bfloat16* dzt;  // [d_hidden][mb]        bf16(dZ)^T: K-major B operand of dW1
     float* lpart;        // [d_hidden/32][mb][16] partial logits per CTA of k_fwd2
     float* gpart;        // [groups][mb][16]      partial logits per group of 8 CTAs
-    __nv_bfloat16* dlb;  // [mb][16]              bf16(dL)
-    unsigned int* tickets;  // [groups + 1]       "last CTA done" tickets of the logit reduction (zero between launches)
+    unsigned int* tickets;  // [groups]           "last CTA done" tickets of the logit reduction (zero between launches)
     int* status;         // device status word: ABS_ETIMEOUT if a bounded wait ran out
     void* zero_from;     // region that must be zero before first use (tickets + status) ...
     size_t zero_bytes;   // ... and its size

@@ -18,10 +18,10 @@
 //   k_cast_x        X fp32 -> bf16 in both orientations
 //   k_fwd1_tcgen05  Z^T partials = W1^T X^T, split over d_in, on tcgen05 (W1 as an MN-major operand)
 //   (k_fwd1         the same on CUDA cores, kept as a cross-check selectable through abs_set_launch)
-//   k_fwd2          Z = sum of partials + b1, bf16(H), partial logits per 32 hidden units; the last CTAs
-//                   to finish (two-level ticket) reduce the partial logits in a fixed order and compute
-//                   softmax, dL and db2
-//   k_bwd           dH, dZ, bf16(dZ)^T, db1 += ..., dW2 += ..., b_i += 1
+//   k_fwd2          Z = sum of partials + b1, bf16(H), partial logits per 32 hidden units; the last CTA of
+//                   each group of 8 ("last CTA done" ticket) sums the group's partial logits in a fixed order
+//   k_bwd           every CTA: logits = sum of group partials + b2, softmax, dL (CTA 0: db2 += ...); then
+//                   dH, dZ, bf16(dZ)^T, db1 += ..., dW2 += ..., b_i += 1
 //   k_dw1_tcgen05   dW1 tile = A B^T on the 5th-gen tensor cores (TMEM accumulator); epilogue adds the
 //                   tile into the worker's accumulator slice via TMA load / TMA store (or TMA reduce-add)
 //   (k_dw1_persistent  the same as a persistent, warp-specialised kernel with a shared-memory ring)
@@ -125,24 +125,18 @@ __global__ void __launch_bounds__(256) k_fwd1(const __nv_bfloat16* __restrict__ 
 // k_fwd2: per CTA 32 hidden units x 64 samples.
 //   phase 1 (thread = sample r, 8 hidden units): Z = sum_s zpart + b1 ; hb = bf16(relu(Z)) -> hbt
 //   phase 2 (thread = sample r, 4 logits):        partial logits of these 32 hidden units -> lpart[cta]
-//   tail: the last CTA of each group of 8 sums the group's partials (fixed order) -> gpart[group];
-//         the last group to finish sums the group partials, adds b2, and computes
-//         dL = (softmax - onehot)/mb, bf16(dL), db2 += sum_r dL.
-// tickets[0 .. n_groups) are the group tickets, tickets[n_groups] the global one; all zero on entry
-// and reset before exit.
+//   tail: the last CTA of each group of 8 sums the group's partials (fixed order) -> gpart[group].
+//         The remaining sum over the groups is cheap (n_groups x 4 KB) and is done by every CTA of k_bwd.
+// tickets[0 .. n_groups) are the group tickets: all zero on entry and reset before exit.
 // --------------------------------------------------------------------------------------------
 __global__ void __launch_bounds__(256) k_fwd2(const float* __restrict__ zpart, int nsplit, const float* __restrict__ b1,
-                                              const __nv_bfloat16* __restrict__ w2b, const float* __restrict__ b2,
-                                              const int32_t* __restrict__ y, __nv_bfloat16* __restrict__ hbt,
-                                              float* lpart, float* gpart, unsigned int* tickets,
-                                              __nv_bfloat16* __restrict__ dlb, float* acc_b2, int d_h, int d_out) {
+                                              const __nv_bfloat16* __restrict__ w2b, __nv_bfloat16* __restrict__ hbt,
+                                              float* lpart, float* gpart, unsigned int* tickets, int d_h, int d_out) {
     __shared__ float sh[kHB][kMB + 1];
     __shared__ float sw2[kHB][kOutPad];
-    __shared__ float sl[kMB][kOutPad + 1];
     __shared__ unsigned int s_last;
     const int h_beg = blockIdx.x * kHB;
     const int n_cta = gridDim.x;
-    const int n_groups = (n_cta + kGroup - 1) / kGroup;
 
     for (int e = threadIdx.x; e < kHB * kOutPad; e += 256) {
         const int hl = e / kOutPad, o = e % kOutPad;
@@ -195,74 +189,37 @@ __global__ void __launch_bounds__(256) k_fwd2(const float* __restrict__ zpart, i
         }
         reinterpret_cast<float4*>(gpart)[(size_t)group * (kMB * kOutPad / 4) + threadIdx.x] = acc;
     }
-    // ---- second level: the last group sums all group partials and finishes the loss
-    __threadfence();
-    __syncthreads();
-    if (threadIdx.x == 0) {
-        tickets[group] = 0u;
-        s_last = (atomicAdd(&tickets[n_groups], 1u) == (unsigned)(n_groups - 1));
-    }
-    __syncthreads();
-    if (!s_last) return;
-    __threadfence();
-    {
-        float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-        for (int c = 0; c < n_groups; ++c) {
-            const float4 v = __ldcg(reinterpret_cast<const float4*>(gpart) + (size_t)c * (kMB * kOutPad / 4) + threadIdx.x);
-            acc.x += v.x; acc.y += v.y; acc.z += v.z; acc.w += v.w;
-        }
-        const int r = threadIdx.x / 4, og = threadIdx.x % 4;
-        sl[r][4 * og + 0] = acc.x; sl[r][4 * og + 1] = acc.y; sl[r][4 * og + 2] = acc.z; sl[r][4 * og + 3] = acc.w;
-    }
-    __syncthreads();
-    if (threadIdx.x < kMB) {
-        const int r = threadIdx.x;
-        float l[kOutPad];
-        float mx = -INFINITY;
-#pragma unroll
-        for (int o = 0; o < kOutPad; ++o) {
-            l[o] = o < d_out ? sl[r][o] + b2[o] : -INFINITY;
-            mx = fmaxf(mx, l[o]);
-        }
-        float den = 0.f;
-#pragma unroll
-        for (int o = 0; o < kOutPad; ++o) {
-            l[o] = o < d_out ? expf(l[o] - mx) : 0.f;
-            den += l[o];
-        }
-        const int yr = y[r];
-#pragma unroll
-        for (int o = 0; o < kOutPad; ++o) {
-            const float g = o < d_out ? (l[o] / den - (o == yr ? 1.f : 0.f)) * (1.0f / kMB) : 0.f;
-            dlb[r * kOutPad + o] = __float2bfloat16_rn(g);
-            sl[r][o] = g;
-        }
-    }
-    __syncthreads();
-    if (threadIdx.x < d_out) {
-        float s = 0.f;
-        for (int rr = 0; rr < kMB; ++rr) s += sl[rr][threadIdx.x];
-        acc_b2[threadIdx.x] += s;
-    }
-    if (threadIdx.x == 0) tickets[n_groups] = 0u;
+    if (threadIdx.x == 0) tickets[group] = 0u;   // ready for the next launch
 }
 
 // --------------------------------------------------------------------------------------------
 // k_bwd: per CTA 32 hidden units x 64 samples.
+//   prologue (every CTA, identical result): logits = sum over groups of gpart + b2 (fixed order);
+//            dL = (softmax - onehot)/mb; CTA 0 also adds db2 = sum_r dL
 //   phase 1 (thread = sample r, 8 hidden units): dH = sum_o bf16(dL)[r][o] W2b[h][o]; dZ = dH * [H > 0]
 //            (H > 0 exactly when Z > 0); dzt[h][r] = bf16(dZ)
 //   phase 2 (thread = hidden unit, 2 outputs): dW2[h][o] += sum_r bf16(H)[h][r] bf16(dL)[r][o],
 //            db1[h] += sum_r dZ[h][r]   (fixed summation order over r)
 // --------------------------------------------------------------------------------------------
-__global__ void __launch_bounds__(256) k_bwd(const __nv_bfloat16* __restrict__ hbt, const __nv_bfloat16* __restrict__ dlb,
+__global__ void __launch_bounds__(256) k_bwd(const __nv_bfloat16* __restrict__ hbt, const float* __restrict__ gpart,
+                                             int n_groups, const float* __restrict__ b2, const int32_t* __restrict__ y,
                                              const __nv_bfloat16* __restrict__ w2b, __nv_bfloat16* __restrict__ dzt,
-                                             float* acc_b1, float* acc_w2, int32_t* cnt, int d_out) {
-    __shared__ float sdl[kMB][kOutPad + 1];
+                                             float* acc_b1, float* acc_w2, float* acc_b2, int32_t* cnt, int d_out) {
+    __shared__ float sdl[kMB][kOutPad + 1];     // bf16(dL) as float (first: the logits)
+    __shared__ float sdl32[kMB][kOutPad + 1];   // dL unrounded (CTA 0: db2)
     __shared__ float sw2[kHB][kOutPad];
     __shared__ float sh[kHB][kMB + 1];
     __shared__ float sdz[kHB][kMB + 1];
     const int h_beg = blockIdx.x * kHB;
-    for (int e = threadIdx.x; e < kMB * kOutPad; e += 256) sdl[e / kOutPad][e % kOutPad] = bf16_to_f(dlb[e]);
+    {
+        float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+        for (int c = 0; c < n_groups; ++c) {
+            const float4 v = reinterpret_cast<const float4*>(gpart)[(size_t)c * (kMB * kOutPad / 4) + threadIdx.x];
+            acc.x += v.x; acc.y += v.y; acc.z += v.z; acc.w += v.w;
+        }
+        const int rr = threadIdx.x / 4, og = threadIdx.x % 4;
+        sdl[rr][4 * og + 0] = acc.x; sdl[rr][4 * og + 1] = acc.y; sdl[rr][4 * og + 2] = acc.z; sdl[rr][4 * og + 3] = acc.w;
+    }
     for (int e = threadIdx.x; e < kHB * kOutPad; e += 256) {
         const int hl = e / kOutPad, o = e % kOutPad;
         sw2[hl][o] = o < d_out ? bf16_to_f(w2b[(size_t)(h_beg + hl) * d_out + o]) : 0.f;
@@ -272,6 +229,35 @@ __global__ void __launch_bounds__(256) k_bwd(const __nv_bfloat16* __restrict__ h
 #pragma unroll
     for (int j = 0; j < 8; ++j) hv[j] = bf16_to_f(hbt[(size_t)(h_beg + g * 8 + j) * kMB + r]);
     __syncthreads();
+    if (threadIdx.x < kMB) {
+        const int rr = threadIdx.x;
+        float l[kOutPad];
+        float mx = -INFINITY;
+#pragma unroll
+        for (int o = 0; o < kOutPad; ++o) {
+            l[o] = o < d_out ? sdl[rr][o] + b2[o] : -INFINITY;
+            mx = fmaxf(mx, l[o]);
+        }
+        float den = 0.f;
+#pragma unroll
+        for (int o = 0; o < kOutPad; ++o) {
+            l[o] = o < d_out ? expf(l[o] - mx) : 0.f;
+            den += l[o];
+        }
+        const int yr = y[rr];
+#pragma unroll
+        for (int o = 0; o < kOutPad; ++o) {
+            const float gl = o < d_out ? (l[o] / den - (o == yr ? 1.f : 0.f)) * (1.0f / kMB) : 0.f;
+            sdl32[rr][o] = gl;
+            sdl[rr][o] = bf16_to_f(__float2bfloat16_rn(gl));
+        }
+    }
+    __syncthreads();
+    if (blockIdx.x == 0 && threadIdx.x < d_out) {
+        float sum = 0.f;
+        for (int rr = 0; rr < kMB; ++rr) sum += sdl32[rr][threadIdx.x];
+        acc_b2[threadIdx.x] += sum;
+    }
     {
         float dl[kOutPad];
 #pragma unroll
@@ -935,8 +921,7 @@ size_t layout_scratch(MlpScratch* s, const MlpDims& d, char* base) {
     char* dzt = take((size_t)d.d_hidden * kMB * 2);
     char* lpart = take((size_t)n_cta * kMB * kOutPad * 4);
     char* gpart = take((size_t)n_groups * kMB * kOutPad * 4);
-    char* dlb = take((size_t)kMB * kOutPad * 2);
-    char* tickets = take((size_t)(n_groups + 1) * 4);
+    char* tickets = take((size_t)n_groups * 4);
     char* status = take(256);
     if (s) {
         s->xb = reinterpret_cast<__nv_bfloat16*>(xb);
@@ -946,7 +931,6 @@ size_t layout_scratch(MlpScratch* s, const MlpDims& d, char* base) {
         s->dzt = reinterpret_cast<__nv_bfloat16*>(dzt);
         s->lpart = reinterpret_cast<float*>(lpart);
         s->gpart = reinterpret_cast<float*>(gpart);
-        s->dlb = reinterpret_cast<__nv_bfloat16*>(dlb);
         s->tickets = reinterpret_cast<unsigned int*>(tickets);
         s->status = reinterpret_cast<int*>(status);
         s->zero_from = tickets;
@@ -1023,14 +1007,15 @@ cudaError_t launch_mlp_front(const MlpDims& d, const MlpScratch& s, const float*
         k_fwd1_tcgen05<<<dim3(d.d_hidden / 128, nsplit), 128, sizeof(FwdSmem) + 1024, stream>>>(*tw, *tx, s.zpart, d.d_in,
                                                                                            d.d_hidden, s.status);
     }
-    k_fwd2<<<d.d_hidden / kHB, 256, 0, stream>>>(s.zpart, nsplit, x_pub + o_b1, shadow + o_w2, x_pub + o_b2, y_dev, s.hbt,
-                                                 s.lpart, s.gpart, s.tickets, s.dlb, acc_row + o_b2, d.d_hidden, d.d_out);
+    k_fwd2<<<d.d_hidden / kHB, 256, 0, stream>>>(s.zpart, nsplit, x_pub + o_b1, shadow + o_w2, s.hbt, s.lpart, s.gpart,
+                                                 s.tickets, d.d_hidden, d.d_out);
     mark(user, ABS_K_MLP_FWD, 3, stream);
     if ((e = cudaGetLastError()) != cudaSuccess) return e;
 
     mark(user, ABS_K_MLP_BWD, 0, stream);
-    k_bwd<<<d.d_hidden / kHB, 256, 0, stream>>>(s.hbt, s.dlb, shadow + o_w2, s.dzt, acc_row + o_b1, acc_row + o_w2, cnt,
-                                                d.d_out);
+    const int n_groups = (d.d_hidden / kHB + kGroup - 1) / kGroup;
+    k_bwd<<<d.d_hidden / kHB, 256, 0, stream>>>(s.hbt, s.gpart, n_groups, x_pub + o_b2, y_dev, shadow + o_w2, s.dzt,
+                                                acc_row + o_b1, acc_row + o_w2, acc_row + o_b2, cnt, d.d_out);
     mark(user, ABS_K_MLP_BWD, 1, stream);
     return cudaGetLastError();
 }

@@ -1,0 +1,46 @@
+"""GPU: the paper's adaptive batch size -- micro-batch counts that emerge from polling "is Step 1
+finished?" instead of a preset schedule -- still matches the oracle replaying the realised schedule."""
+
+import numpy as np
+import pytest
+
+pytestmark = pytest.mark.gpu
+
+
+def test_adaptive_schedule_matches_oracle():
+    import torch
+
+    from oracle.abs_oracle import AbsSgdOracle
+    from paper_2308_15164_b200 import binding as B
+    from paper_2308_15164_b200.adaptive import run_adaptive
+
+    rng = np.random.default_rng(3)
+    P, W, T = 3_000_001, 4, 8
+    x0 = (rng.standard_normal(P) * 0.02).astype(np.float32)
+    pool = (rng.standard_normal((6, P)) * 0.1).astype(np.float32)
+    pool_d = torch.zeros((6, (P + 7) // 8 * 8), dtype=torch.float32, device="cuda")
+    pool_d[:, :P] = torch.from_numpy(pool).cuda()
+    torch.cuda.synchronize()
+    eng = B.AbsSgd(torch.from_numpy(x0).cuda(), W, 0.05, 0.9, 1e-4, pipelined=True)
+    pick = lambda t, i, k: (7 * t + 3 * i + k) % 6            # which pool row a micro-batch uses
+    sched = run_adaptive(eng, lambda t, i, k: pool_d[pick(t, i, k)], T, period=(1, 1, 2, 4), max_batches=16)
+    got = eng.params_host()
+    cnt, cur, t = eng.counters()
+    eng.destroy()
+
+    assert len(sched) == T and all(min(c) >= 1 for c in sched)
+    assert all(c[0] >= c[2] >= c[3] for c in sched)            # faster workers contribute more
+    ref = AbsSgdOracle(x0, W, 0.05, 0.9, 1e-4)
+    for t_, counts in enumerate(sched):
+        rounds = 0
+        done = [0] * W
+        while any(done[i] < counts[i] for i in range(W)):       # same arrival order as the driver
+            rounds += 1
+            for i, p in enumerate((1, 1, 2, 4)):
+                if rounds % p == 0 and done[i] < counts[i]:
+                    ref.accumulate(i, pool[pick(t_, i, done[i])]); done[i] += 1
+        ref.sync_step()
+    want = ref.params()
+    assert np.abs(got - want).max() <= 1e-5 * np.abs(want).max()
+    rc, rcur, rt = ref.counters()
+    assert np.array_equal(cnt, rc) and (cur, t) == (rcur, rt)
