@@ -62,6 +62,12 @@ extern "C" {
 #define ABS_FLAG_PIPELINED  1u  /* Step 1 of iteration t runs on stream_sync, concurrently with Step 2 of t+1 */
 #define ABS_FLAG_MLP        2u  /* the flat vector is a 2-layer MLP; enables abs_accumulate_mlp               */
 #define ABS_FLAG_HOST_INPUT 4u  /* reserve staging so abs_accumulate_host may be used                         */
+#define ABS_FLAG_OVERWRITE_FIRST 8u /* byte-saving variant: the fused step does not write zeros over the set it
+                                       consumed; instead a worker's first micro-batch of an iteration stores
+                                       (acc = g) rather than adds.  Same results; the fused step moves
+                                       4*W_act + 16 instead of 8*W_act + 16 bytes per parameter and those first
+                                       accumulates 8 (6 for bf16) instead of 12 (10).  Rows of workers that were
+                                       idle keep stale values (never read).  Not available with ABS_FLAG_MLP. */
 
 #define ABS_MAX_WORKERS 64u
 

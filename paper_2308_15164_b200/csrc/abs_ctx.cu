@@ -36,12 +36,14 @@ bool config_ok(const abs_config* c, std::string* why) {
     if (c->P == 0) return fail("P must be > 0");
     if (c->W == 0 || c->W > ABS_MAX_WORKERS) return fail("W must be in 1..64");
     if (c->grad_dtype != ABS_GRAD_F32 && c->grad_dtype != ABS_GRAD_BF16) return fail("unknown grad_dtype");
-    if (c->flags & ~(ABS_FLAG_PIPELINED | ABS_FLAG_MLP | ABS_FLAG_HOST_INPUT)) return fail("unknown flag bits");
+    if (c->flags & ~(ABS_FLAG_PIPELINED | ABS_FLAG_MLP | ABS_FLAG_HOST_INPUT | ABS_FLAG_OVERWRITE_FIRST)) return fail("unknown flag bits");
     if (!std::isfinite(c->lr) || !std::isfinite(c->momentum) || !std::isfinite(c->weight_decay) ||
         !std::isfinite(c->lambda_dc))
         return fail("lr, momentum, weight_decay and lambda_dc must be finite");
     if ((c->flags & ABS_FLAG_PIPELINED) && c->stream_acc == c->stream_sync)
         return fail("pipelined mode needs two different streams");
+    if ((c->flags & ABS_FLAG_MLP) && (c->flags & ABS_FLAG_OVERWRITE_FIRST))
+        return fail("ABS_FLAG_OVERWRITE_FIRST is not available with ABS_FLAG_MLP");
     if (c->flags & ABS_FLAG_MLP) {
         if (c->mlp_in == 0 || c->mlp_in % 128 || c->mlp_hidden == 0 || c->mlp_hidden % 128)
             return fail("mlp_in and mlp_hidden must be positive multiples of 128");
@@ -243,6 +245,7 @@ int launch_fused(abs_ctx* c, uint32_t set, int in, int out, uint64_t log_step, c
     a.lambda_dc = c->cfg.lambda_dc;
     a.disp_scale = c->disp_scale;
     a.shadow = c->mlp ? c->shadow(out) : nullptr;
+    a.zero_acc = (c->cfg.flags & ABS_FLAG_OVERWRITE_FIRST) ? 0 : 1;
     {
         Timed tm(c, ABS_K_SYNC, stream);
         CK(launch_sync(a, c->ctas_per_sm[ABS_K_SYNC], c->num_sms, stream));
@@ -363,9 +366,11 @@ int abs_accumulate(abs_ctx* c, uint32_t worker, const void* grad_dev) {
     if (worker >= c->cfg.W) return invalid(c, "worker index out of range");
     if (!grad_dev || (reinterpret_cast<uintptr_t>(grad_dev) & 15)) return invalid(c, "gradient pointer must be non-NULL and 16-byte aligned");
     if (int rc = join_dw(c)) return rc;
+    // overwrite-first mode: the row is not kept zeroed, so a worker's first micro-batch of an iteration stores
+    const bool first = (c->cfg.flags & ABS_FLAG_OVERWRITE_FIRST) && c->h_cnt[(size_t)c->cur * c->cfg.W + worker] == 0;
     {
         Timed tm(c, ABS_K_ACCUMULATE, c->s_acc);
-        CK(launch_accumulate(c->acc(c->cur, worker), grad_dev, c->cfg.grad_dtype, c->cfg.P, c->cnt(c->cur, worker),
+        CK(launch_accumulate(c->acc(c->cur, worker), grad_dev, c->cfg.grad_dtype, c->cfg.P, c->cnt(c->cur, worker), first,
                              c->ctas_per_sm[ABS_K_ACCUMULATE], c->num_sms, c->s_acc));
     }
     c->launches += 1;
@@ -379,6 +384,7 @@ int abs_accumulate_host(abs_ctx* c, uint32_t worker, const void* grad_host) {
     if (worker >= c->cfg.W) return invalid(c, "worker index out of range");
     if (!grad_host) return invalid(c, "gradient pointer is NULL");
     if (int rc = join_dw(c)) return rc;
+    const bool first = (c->cfg.flags & ABS_FLAG_OVERWRITE_FIRST) && c->h_cnt[(size_t)c->cur * c->cfg.W + worker] == 0;
     const int k = c->stage_next;
     c->stage_next ^= 1;
     const size_t es = c->cfg.grad_dtype == ABS_GRAD_BF16 ? 2 : 4;
@@ -390,7 +396,7 @@ int abs_accumulate_host(abs_ctx* c, uint32_t worker, const void* grad_host) {
     CK(cudaStreamWaitEvent(c->s_acc, c->ev_stage_full[k], 0));
     {
         Timed tm(c, ABS_K_ACCUMULATE, c->s_acc);
-        CK(launch_accumulate(c->acc(c->cur, worker), stage, c->cfg.grad_dtype, c->cfg.P, c->cnt(c->cur, worker),
+        CK(launch_accumulate(c->acc(c->cur, worker), stage, c->cfg.grad_dtype, c->cfg.P, c->cnt(c->cur, worker), first,
                              c->ctas_per_sm[ABS_K_ACCUMULATE], c->num_sms, c->s_acc));
     }
     CK(cudaEventRecord(c->ev_stage_free[k], c->s_acc));

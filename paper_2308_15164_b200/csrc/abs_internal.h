@@ -15,7 +15,8 @@ constexpr size_t kPadElems = 256; // accumulator row stride is P rounded up to t
 
 // ---- Step 2: acc_row[j] += g[j], cnt[0] += 1 (Algorithm 1, Step 2) ------------------------
 // grad_dtype: ABS_GRAD_F32 / ABS_GRAD_BF16.  P = number of valid elements in g.
-cudaError_t launch_accumulate(float* acc_row, const void* g, uint32_t grad_dtype, size_t P, int32_t* cnt,
+// overwrite: acc_row[j] = g[j] instead (first micro-batch of a worker when the row is not kept zeroed).
+cudaError_t launch_accumulate(float* acc_row, const void* g, uint32_t grad_dtype, size_t P, int32_t* cnt, bool overwrite,
                               int ctas_per_sm, int num_sms, cudaStream_t stream);
 
 // ---- Step 1 + update (Algorithm 1, Step 1, Eq. 6, "Update parameters") --------------------
@@ -34,6 +35,7 @@ struct SyncArgs {
     float lambda_dc;          // Eq. 6 coefficient
     float disp_scale;         // x_t - x_{t-1} = -disp_scale * v   (0 when the previous step was a no-op)
     __nv_bfloat16* shadow;    // optional bf16 copy of x_{t+1} [P_pad], or nullptr
+    int zero_acc;             // 1: overwrite the consumed rows with zeros; 0: leave them (overwrite-first mode)
 };
 cudaError_t launch_sync(const SyncArgs& a, int ctas_per_sm, int num_sms, cudaStream_t stream);
 

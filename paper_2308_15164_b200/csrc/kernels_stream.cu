@@ -40,7 +40,7 @@ __device__ __forceinline__ float bf16_hi(uint32_t w) { return __uint_as_float(w 
 // ------------------------------------------------------------------------------------------
 // Step 2, fp32 gradient: 12 bytes per parameter (read g, read acc, write acc).
 // ------------------------------------------------------------------------------------------
-template <int U>
+template <int U, bool kOverwrite>
 __global__ void __launch_bounds__(kBlock) k_accumulate_f32(float* acc, const float* __restrict__ g,
                                                            unsigned long long n_vec, unsigned long long P,
                                                            int32_t* cnt) {
@@ -54,21 +54,25 @@ __global__ void __launch_bounds__(kBlock) k_accumulate_f32(float* acc, const flo
             const unsigned long long idx = base + (unsigned long long)u * kBlock + threadIdx.x;
             if (idx < n_vec) {
                 b[u] = ld_stream(g4 + idx);
-                a[u] = acc4[idx];
+                if (!kOverwrite) a[u] = acc4[idx];
             }
         }
 #pragma unroll
         for (int u = 0; u < U; ++u) {
             const unsigned long long idx = base + (unsigned long long)u * kBlock + threadIdx.x;
             if (idx < n_vec) {
-                a[u].x += b[u].x; a[u].y += b[u].y; a[u].z += b[u].z; a[u].w += b[u].w;
+                if (kOverwrite) {
+                    a[u] = b[u];
+                } else {
+                    a[u].x += b[u].x; a[u].y += b[u].y; a[u].z += b[u].z; a[u].w += b[u].w;
+                }
                 st_stream(acc4 + idx, a[u]);
             }
         }
     }
     if (blockIdx.x == 0) {
         const unsigned long long j = n_vec * 4 + threadIdx.x;   // ragged tail (P % 4 elements)
-        if (j < P) acc[j] += g[j];
+        if (j < P) acc[j] = kOverwrite ? g[j] : acc[j] + g[j];
         if (threadIdx.x == 0) cnt[0] += 1;                      // M_t^i += M_r
     }
 }
@@ -76,7 +80,7 @@ __global__ void __launch_bounds__(kBlock) k_accumulate_f32(float* acc, const flo
 // ------------------------------------------------------------------------------------------
 // Step 2, bf16 gradient: 10 bytes per parameter.  One 128-bit load carries 8 gradients.
 // ------------------------------------------------------------------------------------------
-template <int U>
+template <int U, bool kOverwrite>
 __global__ void __launch_bounds__(kBlock) k_accumulate_bf16(float* acc, const uint16_t* __restrict__ g,
                                                             unsigned long long n_vec8, unsigned long long P,
                                                             int32_t* cnt) {
@@ -91,8 +95,13 @@ __global__ void __launch_bounds__(kBlock) k_accumulate_bf16(float* acc, const ui
             const unsigned long long idx = base + (unsigned long long)u * kBlock + threadIdx.x;
             if (idx < n_vec8) {
                 b[u] = ld_stream(g8 + idx);
-                a0[u] = acc4[2 * idx];
-                a1[u] = acc4[2 * idx + 1];
+                if (!kOverwrite) {
+                    a0[u] = acc4[2 * idx];
+                    a1[u] = acc4[2 * idx + 1];
+                } else {
+                    a0[u] = make_float4(0.f, 0.f, 0.f, 0.f);
+                    a1[u] = a0[u];
+                }
             }
         }
 #pragma unroll
@@ -110,7 +119,7 @@ __global__ void __launch_bounds__(kBlock) k_accumulate_bf16(float* acc, const ui
     }
     if (blockIdx.x == 0) {
         const unsigned long long j = n_vec8 * 8 + threadIdx.x;  // ragged tail (P % 8 elements)
-        if (j < P) acc[j] += __uint_as_float((uint32_t)g[j] << 16);
+        if (j < P) acc[j] = (kOverwrite ? 0.f : acc[j]) + __uint_as_float((uint32_t)g[j] << 16);
         if (threadIdx.x == 0) cnt[0] += 1;
     }
 }
@@ -195,7 +204,7 @@ __global__ void __launch_bounds__(kBlock) k_sync(const SyncArgs a) {
                         if (a.shadow) store_shadow(a.shadow, idx, x[u]);
 #pragma unroll
                         for (int i = 0; i < WT; ++i)
-                            if ((active >> i) & 1) st_stream(acc4 + i * rs + idx, zero);
+                            if (a.zero_acc && ((active >> i) & 1)) st_stream(acc4 + i * rs + idx, zero);
                     }
                 }
             } else {
@@ -212,7 +221,7 @@ __global__ void __launch_bounds__(kBlock) k_sync(const SyncArgs a) {
                         for (int c = 0; c < 8; ++c)
                             if (i0 + c < W && ((active >> (i0 + c)) & 1)) {
                                 s.x += r[c].x; s.y += r[c].y; s.z += r[c].z; s.w += r[c].w;
-                                st_stream(acc4 + (i0 + c) * rs + idx, zero);
+                                if (a.zero_acc) st_stream(acc4 + (i0 + c) * rs + idx, zero);
                             }
                     }
                     update_vec(x, v, s, Bf, a);
@@ -276,18 +285,24 @@ cudaError_t launch_sync_t(const SyncArgs& a, int ctas_per_sm, int num_sms, cudaS
 
 }  // namespace
 
-cudaError_t launch_accumulate(float* acc_row, const void* g, uint32_t grad_dtype, size_t P, int32_t* cnt,
+cudaError_t launch_accumulate(float* acc_row, const void* g, uint32_t grad_dtype, size_t P, int32_t* cnt, bool overwrite,
                               int ctas_per_sm, int num_sms, cudaStream_t stream) {
     constexpr int U = 4;
     if (ctas_per_sm == 0) ctas_per_sm = -1;   // measured: one tile per CTA beats a persistent grid
     if (grad_dtype == ABS_GRAD_F32) {
         const unsigned long long n_vec = P / 4;
         const unsigned grid = grid_for(n_vec, kBlock * U, ctas_per_sm, num_sms);
-        k_accumulate_f32<U><<<grid, kBlock, 0, stream>>>(acc_row, static_cast<const float*>(g), n_vec, P, cnt);
+        if (overwrite)
+            k_accumulate_f32<U, true><<<grid, kBlock, 0, stream>>>(acc_row, static_cast<const float*>(g), n_vec, P, cnt);
+        else
+            k_accumulate_f32<U, false><<<grid, kBlock, 0, stream>>>(acc_row, static_cast<const float*>(g), n_vec, P, cnt);
     } else {
         const unsigned long long n_vec8 = P / 8;
         const unsigned grid = grid_for(n_vec8, kBlock * U, ctas_per_sm, num_sms);
-        k_accumulate_bf16<U><<<grid, kBlock, 0, stream>>>(acc_row, static_cast<const uint16_t*>(g), n_vec8, P, cnt);
+        if (overwrite)
+            k_accumulate_bf16<U, true><<<grid, kBlock, 0, stream>>>(acc_row, static_cast<const uint16_t*>(g), n_vec8, P, cnt);
+        else
+            k_accumulate_bf16<U, false><<<grid, kBlock, 0, stream>>>(acc_row, static_cast<const uint16_t*>(g), n_vec8, P, cnt);
     }
     return cudaGetLastError();
 }

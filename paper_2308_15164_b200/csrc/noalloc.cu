@@ -86,5 +86,6 @@ extern "C" int abs_sync_step_noalloc(float* x_dev, float* v_dev, float* acc_dev,
     a.lambda_dc = 0.0f;
     a.disp_scale = 0.0f;
     a.shadow = nullptr;
+    a.zero_acc = 1;
     return abs_sgd::launch_sync(a, 0, num_sms, s) == cudaSuccess ? ABS_OK : ABS_ECUDA;
 }

@@ -42,7 +42,7 @@ def oracle_run(wl, x0, pool, columns=None, lambda_dc=0.0, oracle_cls=None, lr_sc
 
 
 def gpu_run(wl, x0, pool, pipelined, columns=None, lambda_dc=0.0, every_iteration=True, lr_schedule=None,
-            host_input=False):
+            host_input=False, overwrite_first=False):
     """Run the CUDA path over the workload.  Returns the same dict as oracle_run (xs restricted to
     `columns` when given).  With every_iteration=False only the final parameters are read back."""
     import torch
@@ -53,7 +53,7 @@ def gpu_run(wl, x0, pool, pipelined, columns=None, lambda_dc=0.0, every_iteratio
     x0_d = torch.from_numpy(x0).to(dev)
     gd = B.GRAD_BF16 if wl.grad_dtype == "bf16" else B.GRAD_F32
     eng = B.AbsSgd(x0_d, wl.W, wl.lr, wl.momentum, wl.weight_decay, lambda_dc, grad_dtype=gd,
-                   pipelined=pipelined, host_input=host_input)
+                   pipelined=pipelined, host_input=host_input, overwrite_first=overwrite_first)
     pool_d = None
     pool_h = None
     if wl.pool_size:

@@ -153,6 +153,22 @@ def test_eager_and_pipelined_are_bit_identical():
         assert np.array_equal(b1, b2)
 
 
+@pytest.mark.parametrize("cfg,T", [(2, 12), (3, 40), (5, 6)])
+@pytest.mark.parametrize("pipelined", [False, True], ids=["eager", "pipelined"])
+def test_overwrite_first_mode_gives_the_same_results(cfg, T, pipelined):
+    """Byte-saving variant (no zero writes in the fused step, first micro-batch of a worker stores instead of
+    adds): same parameters bit for bit as the default mode, idle workers included, and oracle parity."""
+    wl = wlm.config(cfg, small=True, T=T)
+    x0 = wlm.params0(wl); pool = wlm.grad_pool(wl)
+    a = H.gpu_run(wl, x0, pool, pipelined=pipelined)
+    b = H.gpu_run(wl, x0, pool, pipelined=pipelined, overwrite_first=True)
+    for s, (xa, xb) in enumerate(zip(a["xs"], b["xs"])):
+        assert np.array_equal(xa, xb), f"x_{s + 1} differs in overwrite-first mode"
+    ref = H.oracle_run(wl, x0, pool)
+    H.assert_states_equal(b, ref)
+    H.assert_params_close(b["xs"][-1], ref["xs"][-1], what="overwrite-first x_T")
+
+
 def test_accumulator_matches_oracle_bitwise():
     """fp32 adds of the same operands in the same order: the accumulators agree bit for bit."""
     import torch
