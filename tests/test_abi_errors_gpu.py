@@ -1,0 +1,61 @@
+"""GPU: argument errors on a live context are reported as status codes before anything is enqueued, and a
+destroyed context is rejected."""
+
+import ctypes
+
+import numpy as np
+import pytest
+
+pytestmark = pytest.mark.gpu
+
+
+def test_runtime_argument_errors_and_use_after_destroy():
+    import torch
+
+    from paper_2308_15164_b200 import binding as B
+
+    P, W = 10_000, 3
+    x0 = torch.zeros(P, device="cuda")
+    eng = B.AbsSgd(x0, W, 0.1, 0.9)
+    g = torch.ones(P + 8, device="cuda")
+    h = eng._h
+    n0 = eng.launch_count()
+    assert B.lib.abs_accumulate(h, W, g.data_ptr()) == B.EINVAL                 # worker out of range
+    assert B.lib.abs_accumulate(h, 0, None) == B.EINVAL                         # null gradient
+    assert B.lib.abs_accumulate(h, 0, g.data_ptr() + 4) == B.EINVAL             # misaligned gradient
+    assert B.lib.abs_accumulate_mlp(h, 0, g.data_ptr(), g.data_ptr()) == B.EINVAL   # not an MLP context
+    assert B.lib.abs_accumulate_host(h, 0, g.data_ptr()) == B.EINVAL            # no host-input staging reserved
+    assert B.lib.abs_params(h, None) == B.EINVAL
+    assert B.lib.abs_consumed(h, 0, None) == B.EINVAL
+    b = np.zeros(W, dtype=np.int32)
+    assert B.lib.abs_consumed(h, 5, b.ctypes.data) == B.EINVAL                  # step not reached yet
+    assert B.lib.abs_set_lr(h, float("inf")) == B.EINVAL
+    assert B.lib.abs_set_launch(h, 99, 1) == B.EINVAL
+    assert B.lib.abs_last_error(h) != b""
+    assert eng.launch_count() == n0                                             # nothing was launched
+    eng.accumulate(1, g)                                                        # the context is still usable
+    eng.sync_step(); eng.sync_step()
+    assert np.allclose(eng.params_host(), -0.1)
+    assert eng.consumed(1).tolist() == [0, 1, 0]
+    eng.check()
+    raw = ctypes.c_void_p(h.value)
+    eng.destroy()
+    assert B.lib.abs_sync_step(raw) == B.ESTATE                                 # use after destroy
+    assert B.lib.abs_accumulate(raw, 0, g.data_ptr()) == B.ESTATE
+    assert B.lib.abs_destroy(raw) == B.ESTATE
+
+
+def test_workspace_too_small_and_overwrite_first_with_mlp_rejected():
+    import torch
+
+    from paper_2308_15164_b200 import binding as B
+
+    cfg = B.make_config(P=4096, W=2, lr=0.1)
+    need = B.abs_workspace_bytes(cfg)
+    ws = torch.empty(need, dtype=torch.uint8, device="cuda")
+    x0 = torch.zeros(4096, device="cuda")
+    h = ctypes.c_void_p()
+    assert B.lib.abs_init(ctypes.byref(h), ctypes.byref(cfg), ws.data_ptr(), need - 1, x0.data_ptr()) == B.ENOMEM
+    assert not h.value
+    bad = B.make_config(P=128 * 128 + 128 + 1280 + 10, W=2, lr=0.1, flags=B.FLAG_MLP | B.FLAG_OVERWRITE_FIRST, mlp=(128, 128, 10, 64))
+    assert B.abs_workspace_bytes(bad) == 0
