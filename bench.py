@@ -365,6 +365,50 @@ def run_mlp(B, wlm, dev, peaks, iters=12):
             eng.check()
             eng.destroy()
         out[name] = res
+
+    # K-batched variant: up to 4 consecutive reference batches of a worker per call, one K = 64 n dW1 GEMM
+    res = {}
+    for serial in (0, 1):
+        eng = B.AbsSgd(x0_d, wl.W, wl.lr, wl.momentum, wl.weight_decay, pipelined=True, mlp=(d.d_in, d.d_hidden, d.d_out, d.mb))
+        eng.set_launch(B.K_MLP_FWD, serial)
+        sched = wlm.schedule(wl)
+
+        def run_b(profile):
+            eng.profile(profile)
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            n_mb = n_calls = 0
+            with torch.cuda.stream(eng.stream_acc):
+                e0.record()
+                for b_row in sched:
+                    for i, b in enumerate(b_row):
+                        left = int(b)
+                        while left > 0:
+                            n = min(4, left)
+                            p0 = (n_mb * 7) % (wl.mlp_pool - 4)
+                            eng.accumulate_mlp_batch(i, n, xp[p0], yp[p0]); left -= n; n_mb += n; n_calls += 1
+                    eng.sync_step()
+                eng.wait()
+                e1.record()
+            torch.cuda.synchronize()
+            return e0.elapsed_time(e1), n_mb, n_calls
+
+        run_b(False)
+        ms_total, n_mb, n_calls = run_b(False)
+        if not serial:
+            res.update({"us_per_microbatch_overlapped": ms_total / n_mb * 1e3, "microbatches": n_mb, "calls": n_calls})
+        else:
+            res["us_per_microbatch_serial"] = ms_total / n_mb * 1e3
+            run_b(True)
+            n_dw, ms_dw = eng.kernel_stats(B.K_MLP_DW1)
+            us_dw = ms_dw / n_dw * 1e3
+            mean_n = n_mb / n_calls
+            res.update({"us_dw1_per_call": us_dw, "mean_microbatches_per_call": mean_n,
+                        "dw1_tflops": flop * mean_n / us_dw / 1e6,
+                        "dw1_frac_of_bf16_peak_sustained": flop * mean_n / us_dw / 1e6 / peaks["bf16_tflops_sustained"],
+                        "dw1_hbm_gbs": rmw_bytes / us_dw / 1e3, "dw1_frac_of_hbm": rmw_bytes / us_dw / 1e3 / peaks["hbm_gbs"]})
+        eng.check()
+        eng.destroy()
+    out["k_batched_up_to_4"] = res
     return out
 
 

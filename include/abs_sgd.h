@@ -132,6 +132,14 @@ int abs_accumulate_host(abs_ctx *ctx, uint32_t worker, const void *grad_host);
  * Needs ABS_FLAG_MLP.  Enqueued on stream_acc. */
 int abs_accumulate_mlp(abs_ctx *ctx, uint32_t worker, const float *x_dev, const int32_t *y_dev);
 
+/* n (1..4) consecutive reference batches of one worker in one call: the same computation as n calls of
+ * abs_accumulate_mlp (forward, loss and backward of every micro-batch at x_t; b_i += n), but the n dW1
+ * products are contracted by ONE tcgen05 GEMM with K = 64 n, so the worker's fp32 accumulator slice is
+ * read and written once instead of n times -- that traffic, not the MMAs, bounds the kernel.  The sum
+ * over the n micro-batches is formed in the fp32 TMEM accumulator, so results agree with n single
+ * calls to fp32 rounding, not bit for bit.  x_dev: [n][mlp_mb][mlp_in] fp32; y_dev: [n][mlp_mb] int32. */
+int abs_accumulate_mlp_batch(abs_ctx *ctx, uint32_t worker, uint32_t n, const float *x_dev, const int32_t *y_dev);
+
 /* Algorithm 1, Step 1 + compensation + "Update parameters" + t = t + 1 (see the file header).
  * Without ABS_FLAG_PIPELINED the fused kernel runs on stream_acc.  With it, the call makes
  * x_{t+1} (computed by the kernel launched one call earlier on stream_sync) visible to

@@ -50,6 +50,7 @@ _sig = {
     "abs_accumulate": (ctypes.c_int, [_vp, _u32, _vp]),
     "abs_accumulate_host": (ctypes.c_int, [_vp, _u32, _vp]),
     "abs_accumulate_mlp": (ctypes.c_int, [_vp, _u32, _vp, _vp]),
+    "abs_accumulate_mlp_batch": (ctypes.c_int, [_vp, _u32, _u32, _vp, _vp]),
     "abs_sync_step": (ctypes.c_int, [_vp]),
     "abs_params": (ctypes.c_int, [_vp, ctypes.POINTER(_vp)]),
     "abs_params_host": (ctypes.c_int, [_vp, _vp]),
@@ -147,6 +148,9 @@ class AbsSgd:
 
     def accumulate_mlp(self, worker: int, x, y):
         self._ck(lib.abs_accumulate_mlp(self._h, worker, _ptr(x), _ptr(y)))
+
+    def accumulate_mlp_batch(self, worker: int, n: int, x, y):
+        self._ck(lib.abs_accumulate_mlp_batch(self._h, worker, n, _ptr(x), _ptr(y)))
 
     def sync_step(self):
         self._ck(lib.abs_sync_step(self._h))

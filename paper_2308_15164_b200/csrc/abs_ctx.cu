@@ -406,41 +406,51 @@ int abs_accumulate_host(abs_ctx* c, uint32_t worker, const void* grad_host) {
     return ABS_OK;
 }
 
-int abs_accumulate_mlp(abs_ctx* c, uint32_t worker, const float* x_dev, const int32_t* y_dev) {
+int abs_accumulate_mlp_batch(abs_ctx* c, uint32_t worker, uint32_t n, const float* x_dev, const int32_t* y_dev) {
     if (!live(c)) return ABS_ESTATE;
     if (!c->mlp) return invalid(c, "context was created without ABS_FLAG_MLP");
     if (worker >= c->cfg.W) return invalid(c, "worker index out of range");
+    if (n == 0 || n > (uint32_t)kMlpMaxBatch) return invalid(c, "n must be in 1..4");
     if (!x_dev || (reinterpret_cast<uintptr_t>(x_dev) & 15)) return invalid(c, "x pointer must be non-NULL and 16-byte aligned");
     if (!y_dev || (reinterpret_cast<uintptr_t>(y_dev) & 3)) return invalid(c, "y pointer must be non-NULL and 4-byte aligned");
     // Two scratch sets and a second stream: the latency-bound front part (cast, forward, loss,
-    // layer-2 backward) of micro-batch n+1 runs on stream_acc while the HBM-bound dW1 GEMM of
-    // micro-batch n runs on the internal stream.  dW1 kernels stay in call order on that stream.
+    // layer-2 backward) of the next call runs on stream_acc while the HBM-bound dW1 GEMM of
+    // this one runs on the internal stream.  dW1 kernels stay in call order on that stream.
     const int k = c->mlp_slot;
     c->mlp_slot ^= 1;
     const int variant = c->ctas_per_sm[ABS_K_MLP_DW1];
-    if (c->ctas_per_sm[ABS_K_MLP_FWD] == 1) {
-        // serial mode (measurement aid): everything on stream_acc, no overlap between micro-batches
+    const bool serial = c->ctas_per_sm[ABS_K_MLP_FWD] == 1;   // measurement aid: everything on stream_acc
+    const size_t x_stride = (size_t)c->mlp_dims.mb * c->mlp_dims.d_in, y_stride = (size_t)c->mlp_dims.mb;
+    if (serial) {
         if (int rc = join_dw(c)) return rc;
-        CK(launch_mlp_front(c->mlp_dims, c->mlp_scratch[k], c->x(c->pub), c->shadow(c->pub), c->pub, x_dev, y_dev,
-                            c->acc(c->cur, worker), c->cnt(c->cur, worker), variant, c->s_acc, mlp_mark, c));
-        CK(launch_mlp_dw1(c->mlp_dims, c->mlp_scratch[k], c->acc(c->cur, worker),
-                          &c->acc_tmaps[(size_t)c->cur * c->cfg.W + worker], variant, c->s_acc, mlp_mark, c));
-        c->slot_used[0] = c->slot_used[1] = false;
-    } else {
-        if (c->slot_used[k]) CK(cudaStreamWaitEvent(c->s_acc, c->ev_dw_done[k], 0));   // scratch set k is free again
-        CK(launch_mlp_front(c->mlp_dims, c->mlp_scratch[k], c->x(c->pub), c->shadow(c->pub), c->pub, x_dev, y_dev,
-                            c->acc(c->cur, worker), c->cnt(c->cur, worker), variant, c->s_acc, mlp_mark, c));
+    } else if (c->slot_used[k]) {
+        CK(cudaStreamWaitEvent(c->s_acc, c->ev_dw_done[k], 0));   // scratch set k is free again
+    }
+    for (uint32_t j = 0; j < n; ++j)   // each micro-batch: forward, loss, layer-2 backward; operands into slot j
+        CK(launch_mlp_front(c->mlp_dims, c->mlp_scratch[k], c->x(c->pub), c->shadow(c->pub), c->pub, (int)j,
+                            x_dev + j * x_stride, y_dev + j * y_stride, c->acc(c->cur, worker), c->cnt(c->cur, worker),
+                            variant, c->s_acc, mlp_mark, c));
+    cudaStream_t s_gemm = serial ? c->s_acc : c->s_dw;
+    if (!serial) {
         CK(cudaEventRecord(c->ev_front_done[k], c->s_acc));
         CK(cudaStreamWaitEvent(c->s_dw, c->ev_front_done[k], 0));
-        CK(launch_mlp_dw1(c->mlp_dims, c->mlp_scratch[k], c->acc(c->cur, worker),
-                          &c->acc_tmaps[(size_t)c->cur * c->cfg.W + worker], variant, c->s_dw, mlp_mark, c));
+    }
+    CK(launch_mlp_dw1(c->mlp_dims, c->mlp_scratch[k], c->acc(c->cur, worker),
+                      &c->acc_tmaps[(size_t)c->cur * c->cfg.W + worker], (int)n, variant, s_gemm, mlp_mark, c));
+    if (serial) {
+        c->slot_used[0] = c->slot_used[1] = false;
+    } else {
         CK(cudaEventRecord(c->ev_dw_done[k], c->s_dw));
         c->slot_used[k] = true;
         c->dw_outstanding = true;
         c->dw_last_slot = k;
     }
-    c->h_cnt[(size_t)c->cur * c->cfg.W + worker] += 1;
+    c->h_cnt[(size_t)c->cur * c->cfg.W + worker] += (int32_t)n;
     return ABS_OK;
+}
+
+int abs_accumulate_mlp(abs_ctx* c, uint32_t worker, const float* x_dev, const int32_t* y_dev) {
+    return abs_accumulate_mlp_batch(c, worker, 1, x_dev, y_dev);
 }
 
 int abs_sync_step(abs_ctx* c) {

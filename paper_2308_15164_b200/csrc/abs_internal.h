@@ -51,10 +51,10 @@ struct alignas(64) TmapBytes {   // storage for one CUtensorMap (encoded on the 
 };
 struct MlpScratch {      // device pointers carved from the workspace (all hidden-major, see mlp.cu)
     __nv_bfloat16* xb;   // [mb][d_in]            bf16(X)
-    __nv_bfloat16* xtb;  // [d_in][mb]            bf16(X)^T: K-major A operand of dW1
+    __nv_bfloat16* xtb;  // [4][d_in][mb]         bf16(X)^T of up to 4 stacked micro-batches: K-major A operand of dW1
     float* zpart;        // [split][d_hidden][mb] split-K partial sums of the forward GEMM
     __nv_bfloat16* hbt;  // [d_hidden][mb]        bf16(relu(Z))^T
-    __nv_bfloat16* dzt;  // [d_hidden][mb]        bf16(dZ)^T: K-major B operand of dW1
+    __nv_bfloat16* dzt;  // [4][d_hidden][mb]     bf16(dZ)^T of up to 4 stacked micro-batches: K-major B operand of dW1
     float* lpart;        // [d_hidden/32][mb][16] partial logits per CTA of k_fwd2
     float* gpart;        // [groups][mb][16]      partial logits per group of 8 CTAs
     unsigned int* tickets;  // [groups]           "last CTA done" tickets of the logit reduction (zero between launches)
@@ -82,9 +82,12 @@ cudaError_t mlp_make_acc_tmap(void* tmap_out, const MlpDims& d, float* acc_row);
 // its n launches.
 typedef void (*MlpMark)(void* user, int kernel_class, int n, cudaStream_t stream);
 cudaError_t launch_mlp_front(const MlpDims& d, const MlpScratch& s, const float* x_pub, const __nv_bfloat16* shadow,
-                             int shadow_idx, const float* x_dev, const int32_t* y_dev, float* acc_row, int32_t* cnt,
+                             int shadow_idx, int slot, const float* x_dev, const int32_t* y_dev, float* acc_row, int32_t* cnt,
                              int variant, cudaStream_t stream, MlpMark mark, void* user);
-cudaError_t launch_mlp_dw1(const MlpDims& d, const MlpScratch& s, float* acc_row, const void* acc_tmap, int variant,
+// slot (front) / nb (dw1): up to kMlpMaxBatch micro-batches may be run through the front part into slots
+// 0..nb-1 and then contracted by ONE dW1 launch with K = 64 nb (the accumulator slice is read and written once).
+constexpr int kMlpMaxBatch = 4;
+cudaError_t launch_mlp_dw1(const MlpDims& d, const MlpScratch& s, float* acc_row, const void* acc_tmap, int nb, int variant,
                            cudaStream_t stream, MlpMark mark, void* user);
 
 }  // namespace abs_sgd

@@ -510,33 +510,40 @@ __global__ void __launch_bounds__(128) k_dw1_tcgen05(const __grid_constant__ CUt
 }
 
 // ============================================================================================
-// dW1 with a register-prefetched accumulator tile.  Same tile and MMA as k_dw1_tcgen05, but the
-// fp32 accumulator tile never goes through TMA: every thread loads its 8 float4 of the tile with
-// plain coalesced loads at kernel entry (all in flight while the operands arrive and the MMA
-// runs), the TMEM result is transposed through a padded shared-memory tile, and the sums go back
-// with coalesced stores.  A plain read-modify-write of the 50 MB slice with this many loads in
-// flight measures 18.5 us on B200 for any tile shape; the TMA-staged epilogues need 22-25 us.
+// dW1 with a register-prefetched accumulator tile, optionally K-batched.  Same tile as
+// k_dw1_tcgen05, but the fp32 accumulator tile never goes through TMA: every thread loads its
+// 8 float4 of the tile with plain coalesced loads at kernel entry (all in flight while the
+// operands arrive and the MMAs run), the TMEM result is transposed through a padded shared-memory
+// tile, and the sums go back with coalesced stores.
+// K batching: the operands of nb (1..kMaxBatch) micro-batches are stacked along K, so one launch
+// computes  acc += sum_j X_j^T dZ_j  (K = 64 nb) and the accumulator slice is read and written once
+// for nb micro-batches instead of nb times -- the kernel is bound by that traffic, not by the MMAs.
+// Operand j lives at row offset j*d_in (X^T) / j*d_h (dZ^T) of the stacked operand tensors.
 // 256 threads: warps 0-3 read TMEM columns 0..31 of their lane quarter, warps 4-7 columns 32..63.
 // ============================================================================================
+constexpr int kMaxBatch = 4;
 constexpr int kDwPitch = kDwN + 4;   // floats per row of the staging tile (pitch 272 B: conflict-free float4 rows)
+constexpr int kDwOperandBytes = kTileM * 128 + kDwN * 128;   // A tile 16 KB + B tile 8 KB per micro-batch
+constexpr int kDwStagingBytes = kTileM * kDwPitch * 4;       // 34 KB
 
-struct DwRegSmem {
-    // A tile [128][64] bf16 (16 KB) and B tile [kDwN][64] bf16 (8 KB); once the MMAs have completed the same
-    // bytes are reused as the fp32 staging tile d[128][kDwPitch] (34 KB), which keeps a CTA under 36 KB of
-    // shared memory so that four CTAs (with their 32 KB of accumulator loads each) are resident per SM.
-    alignas(1024) uint8_t buf[kTileM * kDwPitch * 4];
+// Dynamic shared memory: [operands of nb micro-batches | reused as the staging tile once the MMAs are done]
+// followed by this control block.
+struct DwRegCtl {
     alignas(8) uint64_t bar_ab;
     uint64_t bar_mma;
     uint32_t tmem_base;
     uint32_t failed;
 };
-static_assert(kTileM * kDwPitch * 4 >= kTileM * 128 + kDwN * 128, "staging tile must cover both operand tiles");
+__host__ __device__ constexpr int dw_regs_buf_bytes(int nb) {
+    return (nb * kDwOperandBytes > kDwStagingBytes ? nb * kDwOperandBytes : kDwStagingBytes + 1023) / 1024 * 1024;
+}
 
 __global__ void __launch_bounds__(256) k_dw1_regs(const __grid_constant__ CUtensorMap tm_xt,
-                                                  const __grid_constant__ CUtensorMap tm_dzt, float* acc_w1, int ld,
-                                                  int* status) {
+                                                  const __grid_constant__ CUtensorMap tm_dzt, float* acc_w1, int d_in,
+                                                  int ld, int nb, int* status) {
     extern __shared__ uint8_t smem_raw[];
-    DwRegSmem& s = *reinterpret_cast<DwRegSmem*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+    uint8_t* buf = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+    DwRegCtl& s = *reinterpret_cast<DwRegCtl*>(buf + dw_regs_buf_bytes(nb));
     const int warp = threadIdx.x / 32, lane = threadIdx.x % 32;
     const int n0 = blockIdx.x * kDwN, m0 = blockIdx.y * kTileM;
     constexpr int kC4 = kDwN / 4;                   // float4 per tile row
@@ -568,15 +575,20 @@ __global__ void __launch_bounds__(256) k_dw1_regs(const __grid_constant__ CUtens
     const uint32_t tmem = s.tmem_base;
 
     if (threadIdx.x == 0) {
-        mbar_expect_tx(&s.bar_ab, kTileM * 128 + kDwN * 128);
-        tma_load_2d(s.buf, &tm_xt, 0, m0, &s.bar_ab);
-        tma_load_2d(s.buf + kTileM * 128, &tm_dzt, 0, n0, &s.bar_ab);
+        mbar_expect_tx(&s.bar_ab, nb * kDwOperandBytes);
+        for (int j = 0; j < nb; ++j) {
+            tma_load_2d(buf + j * kDwOperandBytes, &tm_xt, 0, j * d_in + m0, &s.bar_ab);
+            tma_load_2d(buf + j * kDwOperandBytes + kTileM * 128, &tm_dzt, 0, j * ld + n0, &s.bar_ab);
+        }
         if (mbar_wait(&s.bar_ab, 0)) {
             asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-            const uint64_t da = umma_desc_k_sw128(smem_u32(s.buf)), db = umma_desc_k_sw128(smem_u32(s.buf) + kTileM * 128);
             constexpr uint32_t idesc = umma_idesc_bf16(kTileM, kDwN);
+            for (int j = 0; j < nb; ++j) {
+                const uint32_t a0 = smem_u32(buf + j * kDwOperandBytes);
+                const uint64_t da = umma_desc_k_sw128(a0), db = umma_desc_k_sw128(a0 + kTileM * 128);
 #pragma unroll
-            for (int k = 0; k < kMB / 16; ++k) umma_bf16(tmem, da + 2 * k, db + 2 * k, idesc, k > 0);
+                for (int k = 0; k < kMB / 16; ++k) umma_bf16(tmem, da + 2 * k, db + 2 * k, idesc, (j > 0 || k > 0));
+            }
             umma_commit(&s.bar_mma);
         } else {
             s.failed = 1;
@@ -592,7 +604,7 @@ __global__ void __launch_bounds__(256) k_dw1_regs(const __grid_constant__ CUtens
         const int row = q * 32 + lane;
         uint32_t v[32];
         tmem_ld_32(tmem + ((uint32_t)(q * 32) << 16) + (uint32_t)(half * 32), v);
-        float4* drow = reinterpret_cast<float4*>(reinterpret_cast<float*>(s.buf) + row * kDwPitch + half * 32);
+        float4* drow = reinterpret_cast<float4*>(reinterpret_cast<float*>(buf) + row * kDwPitch + half * 32);
 #pragma unroll
         for (int j = 0; j < 8; ++j)
             drow[j] = make_float4(__uint_as_float(v[4 * j]), __uint_as_float(v[4 * j + 1]), __uint_as_float(v[4 * j + 2]),
@@ -606,7 +618,7 @@ __global__ void __launch_bounds__(256) k_dw1_regs(const __grid_constant__ CUtens
 #pragma unroll
         for (int k = 0; k < kPer; ++k) {
             const int e = threadIdx.x + 256 * k;
-            const float4 d = *reinterpret_cast<const float4*>(reinterpret_cast<const float*>(s.buf) + (e / kC4) * kDwPitch + (e % kC4) * 4);
+            const float4 d = *reinterpret_cast<const float4*>(reinterpret_cast<const float*>(buf) + (e / kC4) * kDwPitch + (e % kC4) * 4);
             float4 o = c[k];
             o.x += d.x; o.y += d.y; o.z += d.z; o.w += d.w;
             gbase[(size_t)(e / kC4) * ld4 + (e % kC4)] = o;
@@ -915,10 +927,10 @@ size_t layout_scratch(MlpScratch* s, const MlpDims& d, char* base) {
     const int n_cta = d.d_hidden / kHB;
     const int n_groups = (n_cta + kGroup - 1) / kGroup;
     char* xb = take((size_t)kMB * d.d_in * 2);
-    char* xtb = take((size_t)d.d_in * kMB * 2);
+    char* xtb = take((size_t)kMaxBatch * d.d_in * kMB * 2);
     char* zpart = take((size_t)kSplitK * d.d_hidden * kMB * 4);
     char* hbt = take((size_t)d.d_hidden * kMB * 2);
-    char* dzt = take((size_t)d.d_hidden * kMB * 2);
+    char* dzt = take((size_t)kMaxBatch * d.d_hidden * kMB * 2);
     char* lpart = take((size_t)n_cta * kMB * kOutPad * 4);
     char* gpart = take((size_t)n_groups * kMB * kOutPad * 4);
     char* tickets = take((size_t)n_groups * 4);
@@ -947,10 +959,12 @@ cudaError_t mlp_scratch_init(MlpScratch* s, const MlpDims& d, void* base, __nv_b
                              __nv_bfloat16* shadow1, const char** err) {
     layout_scratch(s, d, static_cast<char*>(base));
     static_assert(sizeof(CUtensorMap) == sizeof(TmapBytes), "tensor map size");
-    if (!encode_2d(reinterpret_cast<CUtensorMap*>(&s->tmap_xt), CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, s->xtb, d.d_in, kMB,
-                   kTileM, kMB) ||
-        !encode_2d(reinterpret_cast<CUtensorMap*>(&s->tmap_dzt), CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, s->dzt, d.d_hidden,
-                   kMB, kDwN, kMB)) {
+    // the operands of up to kMaxBatch micro-batches are stacked: micro-batch j at rows [j*d_in, (j+1)*d_in) of X^T
+    // and [j*d_h, (j+1)*d_h) of dZ^T
+    if (!encode_2d(reinterpret_cast<CUtensorMap*>(&s->tmap_xt), CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, s->xtb,
+                   (uint64_t)kMaxBatch * d.d_in, kMB, kTileM, kMB) ||
+        !encode_2d(reinterpret_cast<CUtensorMap*>(&s->tmap_dzt), CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, s->dzt,
+                   (uint64_t)kMaxBatch * d.d_hidden, kMB, kDwN, kMB)) {
         *err = "cuTensorMapEncodeTiled failed for the dW1 operands";
         return cudaErrorInvalidValue;
     }
@@ -970,7 +984,8 @@ cudaError_t mlp_scratch_init(MlpScratch* s, const MlpDims& d, void* base, __nv_b
     if (e == cudaSuccess)
         e = cudaFuncSetAttribute(k_dw1_persistent, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(DwPersistSmem) + 1024);
     if (e == cudaSuccess)
-        e = cudaFuncSetAttribute(k_dw1_regs, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(DwRegSmem) + 1024);
+        e = cudaFuncSetAttribute(k_dw1_regs, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 dw_regs_buf_bytes(kMaxBatch) + (int)sizeof(DwRegCtl) + 1024);
     if (e == cudaSuccess)
         e = cudaFuncSetAttribute(k_fwd1_tcgen05, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(FwdSmem) + 1024);
     if (e == cudaSuccess)
@@ -990,13 +1005,15 @@ cudaError_t mlp_make_acc_tmap(void* tmap_out, const MlpDims& d, float* acc_row) 
 }
 
 cudaError_t launch_mlp_front(const MlpDims& d, const MlpScratch& s, const float* x_pub, const __nv_bfloat16* shadow,
-                             int shadow_idx, const float* x_dev, const int32_t* y_dev, float* acc_row, int32_t* cnt,
+                             int shadow_idx, int slot, const float* x_dev, const int32_t* y_dev, float* acc_row, int32_t* cnt,
                              int variant, cudaStream_t stream, MlpMark mark, void* user) {
+    __nv_bfloat16* xtb = s.xtb + (size_t)slot * d.d_in * kMB;      // this micro-batch's place in the stacked operands
+    __nv_bfloat16* dzt = s.dzt + (size_t)slot * d.d_hidden * kMB;
     const size_t o_b1 = (size_t)d.d_in * d.d_hidden, o_w2 = o_b1 + d.d_hidden, o_b2 = o_w2 + (size_t)d.d_hidden * d.d_out;
     cudaError_t e;
 
     mark(user, ABS_K_MLP_FWD, 0, stream);
-    k_cast_x<<<d.d_in / 16, 256, 0, stream>>>(x_dev, s.xb, s.xtb, d.d_in);
+    k_cast_x<<<d.d_in / 16, 256, 0, stream>>>(x_dev, s.xb, xtb, d.d_in);
     // every K split must be a whole number of 64-wide pipeline steps (d_in is a multiple of 128)
     const int nsplit = (d.d_in % (64 * kSplitK) == 0) ? kSplitK : 2;
     if (variant & 2) {
@@ -1014,21 +1031,22 @@ cudaError_t launch_mlp_front(const MlpDims& d, const MlpScratch& s, const float*
 
     mark(user, ABS_K_MLP_BWD, 0, stream);
     const int n_groups = (d.d_hidden / kHB + kGroup - 1) / kGroup;
-    k_bwd<<<d.d_hidden / kHB, 256, 0, stream>>>(s.hbt, s.gpart, n_groups, x_pub + o_b2, y_dev, shadow + o_w2, s.dzt,
+    k_bwd<<<d.d_hidden / kHB, 256, 0, stream>>>(s.hbt, s.gpart, n_groups, x_pub + o_b2, y_dev, shadow + o_w2, dzt,
                                                 acc_row + o_b1, acc_row + o_w2, acc_row + o_b2, cnt, d.d_out);
     mark(user, ABS_K_MLP_BWD, 1, stream);
     return cudaGetLastError();
 }
 
-cudaError_t launch_mlp_dw1(const MlpDims& d, const MlpScratch& s, float* acc_row, const void* acc_tmap, int variant,
+cudaError_t launch_mlp_dw1(const MlpDims& d, const MlpScratch& s, float* acc_row, const void* acc_tmap, int nb, int variant,
                            cudaStream_t stream, MlpMark mark, void* user) {
     mark(user, ABS_K_MLP_DW1, 0, stream);
     const dim3 grid(d.d_hidden / kDwN, d.d_in / kTileM);
     const CUtensorMap* ta = reinterpret_cast<const CUtensorMap*>(&s.tmap_xt);
     const CUtensorMap* tb = reinterpret_cast<const CUtensorMap*>(&s.tmap_dzt);
     const CUtensorMap* tc = reinterpret_cast<const CUtensorMap*>(acc_tmap);
-    if (variant & 8) {
-        k_dw1_regs<<<grid, 256, sizeof(DwRegSmem) + 1024, stream>>>(*ta, *tb, acc_row, d.d_hidden, s.status);
+    if ((variant & 8) || nb > 1) {   // the K-batched form exists only for the register-prefetch kernel
+        const size_t smem = dw_regs_buf_bytes(nb) + sizeof(DwRegCtl) + 1024;
+        k_dw1_regs<<<grid, 256, smem, stream>>>(*ta, *tb, acc_row, d.d_in, d.d_hidden, nb, s.status);
     } else if (variant & 4) {
         const int n_tiles_n = d.d_hidden / kDwN, n_tiles = n_tiles_n * (d.d_in / kTileM);
         const int ctas = n_tiles < s.num_sms ? n_tiles : s.num_sms;

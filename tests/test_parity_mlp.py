@@ -183,3 +183,48 @@ def test_training_run_matches_oracle(small, T):
             assert np.array_equal(a, b)
         outs.append(got)
     assert np.array_equal(outs[0], outs[1]), "eager and pipelined runs must be bit-identical"
+
+
+@pytest.mark.parametrize("n", [2, 4])
+@pytest.mark.parametrize("small", [True, False], ids=["384x512", "3072x4096"])
+def test_batched_microbatches_match_the_sum_of_gradients(small, n):
+    """abs_accumulate_mlp_batch: n reference batches of one worker contracted by one K = 64 n GEMM give the sum
+    of the n micro-batch gradients (b_i += n)."""
+    import torch
+
+    wl = wlm.config(4, small=small)
+    d = wl.mlp
+    dims = (d.d_in, d.d_hidden, d.d_out)
+    x0 = wlm.params0(wl)
+    xs, ys = wlm.mlp_batches(wl)
+    eng = _engine(wl, x0)
+    b0 = 8
+    xd, yd = torch.from_numpy(xs[b0:b0 + n]).cuda().contiguous(), torch.from_numpy(ys[b0:b0 + n]).cuda().contiguous()
+    torch.cuda.synchronize()
+    eng.accumulate_mlp_batch(3, n, xd, yd)
+    eng.check()
+    got = eng.accumulator(0, 3).cpu().numpy().astype(np.float64)
+    assert eng.counters()[0][0].tolist() == [0, 0, 0, n]
+    want = np.zeros(wl.P)
+    undecided = set()
+    for j in range(n):
+        _, g, aux = mlp_loss_and_grad(x0, xs[b0 + j], ys[b0 + j], *dims, mode="bf16")
+        want += g
+        undecided |= set(int(h) for _, h in np.argwhere(np.abs(aux["Z"]) < TAU))
+    clear = np.setdiff1d(np.arange(d.d_hidden), sorted(undecided))
+    gW1, gb1, gW2, gb2 = mlp_split(got, *dims)
+    wW1, wb1, wW2, wb2 = mlp_split(want, *dims)
+    _close(gW2, wW2, "dW2"); _close(gb2, wb2, "db2")
+    _close(gW1[:, clear], wW1[:, clear], "dW1"); _close(gb1[clear], wb1[clear], "db1")
+    # hidden units with an undecided ReLU gate: bounded by the contribution of those few gates
+    if undecided:
+        u = sorted(undecided)
+        assert np.abs(gW1[:, u] - wW1[:, u]).max() <= 0.2 * np.abs(wW1).max()
+    # and the same data through n single calls agrees to fp32 rounding of the sums
+    eng2 = _engine(wl, x0)
+    for j in range(n):
+        eng2.accumulate_mlp(3, xd[j], yd[j])
+    eng2.check()
+    single = eng2.accumulator(0, 3).cpu().numpy().astype(np.float64)
+    assert np.abs(got - single).max() <= 1e-5 * np.abs(single).max()
+    eng.destroy(); eng2.destroy()
