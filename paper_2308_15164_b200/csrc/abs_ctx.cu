@@ -420,16 +420,13 @@ int abs_accumulate_mlp_batch(abs_ctx* c, uint32_t worker, uint32_t n, const floa
     c->mlp_slot ^= 1;
     const int variant = c->ctas_per_sm[ABS_K_MLP_DW1];
     const bool serial = c->ctas_per_sm[ABS_K_MLP_FWD] == 1;   // measurement aid: everything on stream_acc
-    const size_t x_stride = (size_t)c->mlp_dims.mb * c->mlp_dims.d_in, y_stride = (size_t)c->mlp_dims.mb;
     if (serial) {
         if (int rc = join_dw(c)) return rc;
     } else if (c->slot_used[k]) {
         CK(cudaStreamWaitEvent(c->s_acc, c->ev_dw_done[k], 0));   // scratch set k is free again
     }
-    for (uint32_t j = 0; j < n; ++j)   // each micro-batch: forward, loss, layer-2 backward; operands into slot j
-        CK(launch_mlp_front(c->mlp_dims, c->mlp_scratch[k], c->x(c->pub), c->shadow(c->pub), c->pub, (int)j,
-                            x_dev + j * x_stride, y_dev + j * y_stride, c->acc(c->cur, worker), c->cnt(c->cur, worker),
-                            variant, c->s_acc, mlp_mark, c));
+    CK(launch_mlp_front(c->mlp_dims, c->mlp_scratch[k], c->x(c->pub), c->shadow(c->pub), c->pub, (int)n, x_dev, y_dev,
+                        c->acc(c->cur, worker), c->cnt(c->cur, worker), variant, c->s_acc, mlp_mark, c));
     cudaStream_t s_gemm = serial ? c->s_acc : c->s_dw;
     if (!serial) {
         CK(cudaEventRecord(c->ev_front_done[k], c->s_acc));

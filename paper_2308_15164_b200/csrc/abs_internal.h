@@ -43,6 +43,7 @@ cudaError_t launch_sync(const SyncArgs& a, int ctas_per_sm, int num_sms, cudaStr
 cudaError_t launch_cast_bf16(const float* src, __nv_bfloat16* dst, size_t n, int num_sms, cudaStream_t stream);
 
 // ---- MLP micro-batch gradient (Step 2 with the gradient computed on the device) ----------
+constexpr int kMlpMaxBatch = 4;
 struct MlpDims {
     int d_in, d_hidden, d_out, mb;
 };
@@ -57,6 +58,8 @@ struct MlpScratch {      // device pointers carved from the workspace (all hidde
     __nv_bfloat16* dzt;  // [4][d_hidden][mb]     bf16(dZ)^T of up to 4 stacked micro-batches: K-major B operand of dW1
     float* lpart;        // [d_hidden/32][mb][16] partial logits per CTA of k_fwd2
     float* gpart;        // [groups][mb][16]      partial logits per group of 8 CTAs
+    float* bpart;        // [4][d_hidden/32][4][256] partial dW2 / db1 / db2 sums of k_bwd, per micro-batch of a call
+    unsigned int* tickets_b;  // [d_hidden/32]     "last CTA done" tickets of k_bwd (zero between launches)
     unsigned int* tickets;  // [groups]           "last CTA done" tickets of the logit reduction (zero between launches)
     int* status;         // device status word: ABS_ETIMEOUT if a bounded wait ran out
     void* zero_from;     // region that must be zero before first use (tickets + status) ...
@@ -82,11 +85,11 @@ cudaError_t mlp_make_acc_tmap(void* tmap_out, const MlpDims& d, float* acc_row);
 // its n launches.
 typedef void (*MlpMark)(void* user, int kernel_class, int n, cudaStream_t stream);
 cudaError_t launch_mlp_front(const MlpDims& d, const MlpScratch& s, const float* x_pub, const __nv_bfloat16* shadow,
-                             int shadow_idx, int slot, const float* x_dev, const int32_t* y_dev, float* acc_row, int32_t* cnt,
+                             int shadow_idx, int nb, const float* x_dev, const int32_t* y_dev, float* acc_row, int32_t* cnt,
                              int variant, cudaStream_t stream, MlpMark mark, void* user);
-// slot (front) / nb (dw1): up to kMlpMaxBatch micro-batches may be run through the front part into slots
-// 0..nb-1 and then contracted by ONE dW1 launch with K = 64 nb (the accumulator slice is read and written once).
-constexpr int kMlpMaxBatch = 4;
+// nb: a call may carry up to kMlpMaxBatch micro-batches (x_dev [nb][mb][d_in], y_dev [nb][mb]): the front kernels
+// take them as an extra grid dimension, and ONE dW1 launch contracts them with K = 64 nb (the accumulator slice is
+// read and written once).
 cudaError_t launch_mlp_dw1(const MlpDims& d, const MlpScratch& s, float* acc_row, const void* acc_tmap, int nb, int variant,
                            cudaStream_t stream, MlpMark mark, void* user);
 

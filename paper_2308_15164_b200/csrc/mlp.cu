@@ -40,6 +40,7 @@ constexpr int kOutPad = 16;      // logits / dL rows are padded to 16 columns
 constexpr int kSplitK = 4;       // forward GEMM: d_in is split into at most this many partial sums
 constexpr int kHB = 32;          // hidden units per CTA in k_fwd2 / k_bwd
 constexpr int kGroup = 8;        // CTAs per first-level group of the logit reduction
+constexpr int kMaxBatch = kMlpMaxBatch;   // micro-batches one call may carry (grid dimension of the front kernels)
 
 __device__ __forceinline__ float bf16_to_f(__nv_bfloat16 v) { return __bfloat162float(v); }
 __device__ __forceinline__ uint32_t pack_bf16x2(float a, float b) {
@@ -54,6 +55,9 @@ __global__ void __launch_bounds__(256) k_cast_x(const float* __restrict__ x, __n
                                                 __nv_bfloat16* __restrict__ xtb, int d_in) {
     __shared__ __nv_bfloat16 tile[16][kMB + 8];
     const int c0 = blockIdx.x * 16;
+    x += (size_t)blockIdx.y * kMB * d_in;      // micro-batch blockIdx.y of the call
+    xb += (size_t)blockIdx.y * kMB * d_in;
+    xtb += (size_t)blockIdx.y * d_in * kMB;
     {
         const int r = threadIdx.x / 4, q = threadIdx.x % 4;
         const float4 v = *reinterpret_cast<const float4*>(x + (size_t)r * d_in + c0 + 4 * q);
@@ -85,6 +89,8 @@ __global__ void __launch_bounds__(256) k_fwd1(const __nv_bfloat16* __restrict__ 
     __shared__ float sx[KT][64 + 4];   // [k][r]
     const int h0 = blockIdx.x * 64;
     const int s = blockIdx.y;
+    xb += (size_t)blockIdx.z * kMB * d_in;                   // micro-batch blockIdx.z of the call
+    zpart += (size_t)blockIdx.z * kSplitK * d_h * kMB;
     const int k_per = d_in / (int)gridDim.y;
     const int kbeg = s * k_per, kend = kbeg + k_per;
     const int th = threadIdx.x / 16, tr = threadIdx.x % 16;   // 16 x 16 threads, 4 h x 4 r each
@@ -129,14 +135,22 @@ __global__ void __launch_bounds__(256) k_fwd1(const __nv_bfloat16* __restrict__ 
 //         The remaining sum over the groups is cheap (n_groups x 4 KB) and is done by every CTA of k_bwd.
 // tickets[0 .. n_groups) are the group tickets: all zero on entry and reset before exit.
 // --------------------------------------------------------------------------------------------
-__global__ void __launch_bounds__(256) k_fwd2(const float* __restrict__ zpart, int nsplit, const float* __restrict__ b1,
-                                              const __nv_bfloat16* __restrict__ w2b, __nv_bfloat16* __restrict__ hbt,
+__global__ void __launch_bounds__(256) k_fwd2(const float* zpart, int nsplit, const float* __restrict__ b1,
+                                              const __nv_bfloat16* __restrict__ w2b, __nv_bfloat16* hbt,
                                               float* lpart, float* gpart, unsigned int* tickets, int d_h, int d_out) {
     __shared__ float sh[kHB][kMB + 1];
     __shared__ float sw2[kHB][kOutPad];
     __shared__ unsigned int s_last;
     const int h_beg = blockIdx.x * kHB;
     const int n_cta = gridDim.x;
+    {   // micro-batch blockIdx.y of the call: its own slices of every scratch array
+        const int j = blockIdx.y, n_groups = (n_cta + kGroup - 1) / kGroup;
+        zpart += (size_t)j * kSplitK * d_h * kMB;
+        hbt += (size_t)j * d_h * kMB;
+        lpart += (size_t)j * n_cta * kMB * kOutPad;
+        gpart += (size_t)j * n_groups * kMB * kOutPad;
+        tickets += (size_t)j * n_groups;
+    }
 
     for (int e = threadIdx.x; e < kHB * kOutPad; e += 256) {
         const int hl = e / kOutPad, o = e % kOutPad;
@@ -201,16 +215,23 @@ __global__ void __launch_bounds__(256) k_fwd2(const float* __restrict__ zpart, i
 //   phase 2 (thread = hidden unit, 2 outputs): dW2[h][o] += sum_r bf16(H)[h][r] bf16(dL)[r][o],
 //            db1[h] += sum_r dZ[h][r]   (fixed summation order over r)
 // --------------------------------------------------------------------------------------------
-__global__ void __launch_bounds__(256) k_bwd(const __nv_bfloat16* __restrict__ hbt, const float* __restrict__ gpart,
-                                             int n_groups, const float* __restrict__ b2, const int32_t* __restrict__ y,
-                                             const __nv_bfloat16* __restrict__ w2b, __nv_bfloat16* __restrict__ dzt,
-                                             float* acc_b1, float* acc_w2, float* acc_b2, int32_t* cnt, int d_out) {
+__global__ void __launch_bounds__(256) k_bwd(const __nv_bfloat16* hbt, const float* gpart, int n_groups,
+                                             const float* __restrict__ b2, const int32_t* y,
+                                             const __nv_bfloat16* __restrict__ w2b, __nv_bfloat16* dzt, float* bpart,
+                                             unsigned int* tickets_b, float* acc_b1, float* acc_w2, float* acc_b2,
+                                             int32_t* cnt, int d_h, int d_out) {
     __shared__ float sdl[kMB][kOutPad + 1];     // bf16(dL) as float (first: the logits)
     __shared__ float sdl32[kMB][kOutPad + 1];   // dL unrounded (CTA 0: db2)
     __shared__ float sw2[kHB][kOutPad];
     __shared__ float sh[kHB][kMB + 1];
     __shared__ float sdz[kHB][kMB + 1];
+    __shared__ unsigned int s_last;
     const int h_beg = blockIdx.x * kHB;
+    const int jb = blockIdx.y, nb = gridDim.y;       // micro-batch of this CTA, micro-batches in the call
+    hbt += (size_t)jb * d_h * kMB;
+    dzt += (size_t)jb * d_h * kMB;
+    gpart += (size_t)jb * n_groups * kMB * kOutPad;
+    y += (size_t)jb * kMB;
     {
         float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
         for (int c = 0; c < n_groups; ++c) {
@@ -253,11 +274,9 @@ __global__ void __launch_bounds__(256) k_bwd(const __nv_bfloat16* __restrict__ h
         }
     }
     __syncthreads();
-    if (blockIdx.x == 0 && threadIdx.x < d_out) {
-        float sum = 0.f;
-        for (int rr = 0; rr < kMB; ++rr) sum += sdl32[rr][threadIdx.x];
-        acc_b2[threadIdx.x] += sum;
-    }
+    float db2 = 0.f;                                 // CTA column 0, thread o < d_out: sum_r dL[r][o]
+    if (blockIdx.x == 0 && threadIdx.x < d_out)
+        for (int rr = 0; rr < kMB; ++rr) db2 += sdl32[rr][threadIdx.x];
     {
         float dl[kOutPad];
 #pragma unroll
@@ -286,11 +305,32 @@ __global__ void __launch_bounds__(256) k_bwd(const __nv_bfloat16* __restrict__ h
             if (slot == 0) c += sdz[hl][rr];
         }
         const int h = h_beg + hl;
+        if (nb > 1) {
+            // Several micro-batches add into the same accumulator entries: every CTA parks its partial sums, and
+            // the last of the nb CTAs of this hidden chunk ("last CTA done" ticket) adds them up in micro-batch
+            // order and does the one read-modify-write -- a fixed summation order, no atomics on the data.
+            float* mine = bpart + ((size_t)(jb * gridDim.x + blockIdx.x) * 4) * 256;
+            mine[threadIdx.x] = a; mine[256 + threadIdx.x] = b; mine[512 + threadIdx.x] = c; mine[768 + threadIdx.x] = db2;
+            __threadfence();
+            __syncthreads();
+            if (threadIdx.x == 0) s_last = (atomicAdd(&tickets_b[blockIdx.x], 1u) == (unsigned)(nb - 1));
+            __syncthreads();
+            if (!s_last) return;
+            __threadfence();
+            a = b = c = db2 = 0.f;
+            for (int q = 0; q < nb; ++q) {
+                const float* p = bpart + ((size_t)(q * gridDim.x + blockIdx.x) * 4) * 256;
+                a += __ldcg(p + threadIdx.x); b += __ldcg(p + 256 + threadIdx.x);
+                c += __ldcg(p + 512 + threadIdx.x); db2 += __ldcg(p + 768 + threadIdx.x);
+            }
+            if (threadIdx.x == 0) tickets_b[blockIdx.x] = 0u;
+        }
         if (slot < d_out) acc_w2[(size_t)h * d_out + slot] += a;
         if (slot + 8 < d_out) acc_w2[(size_t)h * d_out + slot + 8] += b;
         if (slot == 0) acc_b1[h] += c;
+        if (blockIdx.x == 0 && threadIdx.x < d_out) acc_b2[threadIdx.x] += db2;
+        if (blockIdx.x == 0 && threadIdx.x == 0) cnt[0] += nb;   // M_t^i += nb * M_r
     }
-    if (blockIdx.x == 0 && threadIdx.x == 0) cnt[0] += 1;   // M_t^i += M_r
 }
 
 // ============================================================================================
@@ -521,7 +561,6 @@ __global__ void __launch_bounds__(128) k_dw1_tcgen05(const __grid_constant__ CUt
 // Operand j lives at row offset j*d_in (X^T) / j*d_h (dZ^T) of the stacked operand tensors.
 // 256 threads: warps 0-3 read TMEM columns 0..31 of their lane quarter, warps 4-7 columns 32..63.
 // ============================================================================================
-constexpr int kMaxBatch = 4;
 constexpr int kDwPitch = kDwN + 4;   // floats per row of the staging tile (pitch 272 B: conflict-free float4 rows)
 constexpr int kDwOperandBytes = kTileM * 128 + kDwN * 128;   // A tile 16 KB + B tile 8 KB per micro-batch
 constexpr int kDwStagingBytes = kTileM * kDwPitch * 4;       // 34 KB
@@ -811,6 +850,8 @@ __global__ void __launch_bounds__(128) k_fwd1_tcgen05(const __grid_constant__ CU
     const int k_per = d_in / (int)gridDim.y;
     const int kbeg = split * k_per;
     const int nk = k_per / 64;                       // pipeline steps of 64 k
+    const int jb = blockIdx.z;                       // micro-batch of the call: rows jb*64.. of the stacked xb
+    zpart += (size_t)jb * kSplitK * d_h * kMB;
 
     if (warp == 0) {
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&s.tmem_base)), "r"(64) : "memory");
@@ -838,7 +879,7 @@ __global__ void __launch_bounds__(128) k_fwd1_tcgen05(const __grid_constant__ CU
             const int k0 = kbeg + kb * 64;
             tma_load_2d(s.stage[st], &tm_w1, h0, k0, &s.full[st]);
             tma_load_2d(s.stage[st] + 8192, &tm_w1, h0 + 64, k0, &s.full[st]);
-            tma_load_2d(s.stage[st] + 16384, &tm_xb, k0, 0, &s.full[st]);
+            tma_load_2d(s.stage[st] + 16384, &tm_xb, k0, jb * kMB, &s.full[st]);
         }
     } else if (warp == 1 && lane == 0) {             // ---- MMA issuer
         constexpr uint32_t idesc = umma_idesc_bf16(128, 64) | (1u << 15);   // A is MN-major
@@ -926,14 +967,15 @@ size_t layout_scratch(MlpScratch* s, const MlpDims& d, char* base) {
     auto take = [&](size_t b) { char* at = base ? base + o : nullptr; o = align_up(o + b, 1024); return at; };
     const int n_cta = d.d_hidden / kHB;
     const int n_groups = (n_cta + kGroup - 1) / kGroup;
-    char* xb = take((size_t)kMB * d.d_in * 2);
+    char* xb = take((size_t)kMaxBatch * kMB * d.d_in * 2);
     char* xtb = take((size_t)kMaxBatch * d.d_in * kMB * 2);
-    char* zpart = take((size_t)kSplitK * d.d_hidden * kMB * 4);
-    char* hbt = take((size_t)d.d_hidden * kMB * 2);
+    char* zpart = take((size_t)kMaxBatch * kSplitK * d.d_hidden * kMB * 4);
+    char* hbt = take((size_t)kMaxBatch * d.d_hidden * kMB * 2);
     char* dzt = take((size_t)kMaxBatch * d.d_hidden * kMB * 2);
-    char* lpart = take((size_t)n_cta * kMB * kOutPad * 4);
-    char* gpart = take((size_t)n_groups * kMB * kOutPad * 4);
-    char* tickets = take((size_t)n_groups * 4);
+    char* lpart = take((size_t)kMaxBatch * n_cta * kMB * kOutPad * 4);
+    char* gpart = take((size_t)kMaxBatch * n_groups * kMB * kOutPad * 4);
+    char* bpart = take((size_t)kMaxBatch * n_cta * 4 * 256 * 4);
+    char* tickets = take((size_t)(kMaxBatch * n_groups + n_cta) * 4);   // k_fwd2 group tickets, then k_bwd chunk tickets
     char* status = take(256);
     if (s) {
         s->xb = reinterpret_cast<__nv_bfloat16*>(xb);
@@ -944,6 +986,8 @@ size_t layout_scratch(MlpScratch* s, const MlpDims& d, char* base) {
         s->lpart = reinterpret_cast<float*>(lpart);
         s->gpart = reinterpret_cast<float*>(gpart);
         s->tickets = reinterpret_cast<unsigned int*>(tickets);
+        s->tickets_b = reinterpret_cast<unsigned int*>(tickets) + kMaxBatch * n_groups;
+        s->bpart = reinterpret_cast<float*>(bpart);
         s->status = reinterpret_cast<int*>(status);
         s->zero_from = tickets;
         s->zero_bytes = (size_t)(status + 256 - tickets);
@@ -973,8 +1017,8 @@ cudaError_t mlp_scratch_init(MlpScratch* s, const MlpDims& d, void* base, __nv_b
                    d.d_hidden, 64, 64) ||
         !encode_2d(reinterpret_cast<CUtensorMap*>(&s->tmap_w1[1]), CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, shadow1, d.d_in,
                    d.d_hidden, 64, 64) ||
-        !encode_2d(reinterpret_cast<CUtensorMap*>(&s->tmap_xb), CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, s->xb, kMB, d.d_in, kMB,
-                   64)) {
+        !encode_2d(reinterpret_cast<CUtensorMap*>(&s->tmap_xb), CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, s->xb,
+                   (uint64_t)kMaxBatch * kMB, d.d_in, kMB, 64)) {
         *err = "cuTensorMapEncodeTiled failed for the forward GEMM operands";
         return cudaErrorInvalidValue;
     }
@@ -1005,34 +1049,35 @@ cudaError_t mlp_make_acc_tmap(void* tmap_out, const MlpDims& d, float* acc_row) 
 }
 
 cudaError_t launch_mlp_front(const MlpDims& d, const MlpScratch& s, const float* x_pub, const __nv_bfloat16* shadow,
-                             int shadow_idx, int slot, const float* x_dev, const int32_t* y_dev, float* acc_row, int32_t* cnt,
+                             int shadow_idx, int nb, const float* x_dev, const int32_t* y_dev, float* acc_row, int32_t* cnt,
                              int variant, cudaStream_t stream, MlpMark mark, void* user) {
-    __nv_bfloat16* xtb = s.xtb + (size_t)slot * d.d_in * kMB;      // this micro-batch's place in the stacked operands
-    __nv_bfloat16* dzt = s.dzt + (size_t)slot * d.d_hidden * kMB;
     const size_t o_b1 = (size_t)d.d_in * d.d_hidden, o_w2 = o_b1 + d.d_hidden, o_b2 = o_w2 + (size_t)d.d_hidden * d.d_out;
     cudaError_t e;
+    const unsigned n_cta = d.d_hidden / kHB;
 
+    // every kernel carries the nb micro-batches of the call as an extra grid dimension
     mark(user, ABS_K_MLP_FWD, 0, stream);
-    k_cast_x<<<d.d_in / 16, 256, 0, stream>>>(x_dev, s.xb, xtb, d.d_in);
+    k_cast_x<<<dim3(d.d_in / 16, nb), 256, 0, stream>>>(x_dev, s.xb, s.xtb, d.d_in);
     // every K split must be a whole number of 64-wide pipeline steps (d_in is a multiple of 128)
     const int nsplit = (d.d_in % (64 * kSplitK) == 0) ? kSplitK : 2;
     if (variant & 2) {
-        k_fwd1<<<dim3(d.d_hidden / 64, nsplit), 256, 0, stream>>>(shadow, s.xb, s.zpart, d.d_in, d.d_hidden);
+        k_fwd1<<<dim3(d.d_hidden / 64, nsplit, nb), 256, 0, stream>>>(shadow, s.xb, s.zpart, d.d_in, d.d_hidden);
     } else {
         const CUtensorMap* tw = reinterpret_cast<const CUtensorMap*>(&s.tmap_w1[shadow_idx]);
         const CUtensorMap* tx = reinterpret_cast<const CUtensorMap*>(&s.tmap_xb);
-        k_fwd1_tcgen05<<<dim3(d.d_hidden / 128, nsplit), 128, sizeof(FwdSmem) + 1024, stream>>>(*tw, *tx, s.zpart, d.d_in,
-                                                                                           d.d_hidden, s.status);
+        k_fwd1_tcgen05<<<dim3(d.d_hidden / 128, nsplit, nb), 128, sizeof(FwdSmem) + 1024, stream>>>(*tw, *tx, s.zpart, d.d_in,
+                                                                                               d.d_hidden, s.status);
     }
-    k_fwd2<<<d.d_hidden / kHB, 256, 0, stream>>>(s.zpart, nsplit, x_pub + o_b1, shadow + o_w2, s.hbt, s.lpart, s.gpart,
-                                                 s.tickets, d.d_hidden, d.d_out);
+    k_fwd2<<<dim3(n_cta, nb), 256, 0, stream>>>(s.zpart, nsplit, x_pub + o_b1, shadow + o_w2, s.hbt, s.lpart, s.gpart,
+                                                s.tickets, d.d_hidden, d.d_out);
     mark(user, ABS_K_MLP_FWD, 3, stream);
     if ((e = cudaGetLastError()) != cudaSuccess) return e;
 
     mark(user, ABS_K_MLP_BWD, 0, stream);
-    const int n_groups = (d.d_hidden / kHB + kGroup - 1) / kGroup;
-    k_bwd<<<d.d_hidden / kHB, 256, 0, stream>>>(s.hbt, s.gpart, n_groups, x_pub + o_b2, y_dev, shadow + o_w2, dzt,
-                                                acc_row + o_b1, acc_row + o_w2, acc_row + o_b2, cnt, d.d_out);
+    const int n_groups = (n_cta + kGroup - 1) / kGroup;
+    k_bwd<<<dim3(n_cta, nb), 256, 0, stream>>>(s.hbt, s.gpart, n_groups, x_pub + o_b2, y_dev, shadow + o_w2, s.dzt, s.bpart,
+                                               s.tickets_b, acc_row + o_b1, acc_row + o_w2, acc_row + o_b2, cnt, d.d_hidden,
+                                               d.d_out);
     mark(user, ABS_K_MLP_BWD, 1, stream);
     return cudaGetLastError();
 }
