@@ -824,37 +824,46 @@ __global__ void __launch_bounds__(192) k_dw1_persistent(const __grid_constant__ 
 //       8-k-row groups 1024 B apart (stride offset), the two 64-wide h blocks of the tile one box
 //       (8192 B) apart (leading offset).  One UMMA step (K = 16) consumes two 8-k groups: +2048 B.
 //   B = xb tile [64 samples][64 k], K-major as in the dW1 kernel.
-// One CTA per (128-hidden tile, K split); a kFwdStages-deep TMA -> MMA pipeline streams the
-// weights once.  Warp 0 lane 0 issues TMA, warp 1 lane 0 issues MMAs, all four warps store D.
+//       The NB micro-batches of a call are stacked along N (N = 64 NB <= 256): one 64 x 64 box
+//       each, 8192 B apart -- the same 8-row groups 1024 B apart, so one descriptor covers them
+//       and the weights are streamed once per call, not once per micro-batch.
+// One CTA per (128-hidden tile, K split); a ring of TMA -> MMA stages streams the weights
+// once.  Warp 0 lane 0 issues TMA, warp 1 lane 0 issues MMAs, all four warps store D.
 // ============================================================================================
-constexpr int kFwdStages = 6;
-constexpr int kFwdStageBytes = 2 * 8192 + 8192;   // two A boxes + one B box
+template <int NB>
+struct FwdCfg {
+    static constexpr int kStages = NB <= 2 ? 6 : (NB == 3 ? 5 : 4);       // <= 200 KB of stages
+    static constexpr int kStageBytes = 2 * 8192 + NB * 8192;              // two A boxes + NB B boxes
+    static constexpr int kTmemCols = NB == 1 ? 64 : (NB == 2 ? 128 : 256);   // power of two >= 64 NB
+};
 
+template <int NB>
 struct FwdSmem {
-    alignas(1024) uint8_t stage[kFwdStages][kFwdStageBytes];   // [A h0..63 | A h64..127 | B]
-    alignas(8) uint64_t full[kFwdStages];
-    uint64_t empty[kFwdStages];
+    alignas(1024) uint8_t stage[FwdCfg<NB>::kStages][FwdCfg<NB>::kStageBytes];   // [A h0..63 | A h64..127 | B x NB]
+    alignas(8) uint64_t full[FwdCfg<NB>::kStages];
+    uint64_t empty[FwdCfg<NB>::kStages];
     uint64_t done;
     uint32_t tmem_base;
     uint32_t failed;
 };
 
+template <int NB>
 __global__ void __launch_bounds__(128) k_fwd1_tcgen05(const __grid_constant__ CUtensorMap tm_w1,
                                                       const __grid_constant__ CUtensorMap tm_xb, float* __restrict__ zpart,
                                                       int d_in, int d_h, int* status) {
+    constexpr int kFwdStages = FwdCfg<NB>::kStages, kFwdStageBytes = FwdCfg<NB>::kStageBytes;
+    constexpr int kTmemCols = FwdCfg<NB>::kTmemCols;
     extern __shared__ uint8_t smem_raw[];
-    FwdSmem& s = *reinterpret_cast<FwdSmem*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+    FwdSmem<NB>& s = *reinterpret_cast<FwdSmem<NB>*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
     const int warp = threadIdx.x / 32, lane = threadIdx.x % 32;
     const int h0 = blockIdx.x * 128;
     const int split = blockIdx.y;
     const int k_per = d_in / (int)gridDim.y;
     const int kbeg = split * k_per;
     const int nk = k_per / 64;                       // pipeline steps of 64 k
-    const int jb = blockIdx.z;                       // micro-batch of the call: rows jb*64.. of the stacked xb
-    zpart += (size_t)jb * kSplitK * d_h * kMB;
 
     if (warp == 0) {
-        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&s.tmem_base)), "r"(64) : "memory");
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&s.tmem_base)), "r"(kTmemCols) : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
     }
     if (threadIdx.x == 0) {
@@ -879,10 +888,12 @@ __global__ void __launch_bounds__(128) k_fwd1_tcgen05(const __grid_constant__ CU
             const int k0 = kbeg + kb * 64;
             tma_load_2d(s.stage[st], &tm_w1, h0, k0, &s.full[st]);
             tma_load_2d(s.stage[st] + 8192, &tm_w1, h0 + 64, k0, &s.full[st]);
-            tma_load_2d(s.stage[st] + 16384, &tm_xb, k0, jb * kMB, &s.full[st]);
+#pragma unroll
+            for (int jb = 0; jb < NB; ++jb)          // rows jb*64.. of the stacked xb
+                tma_load_2d(s.stage[st] + 16384 + jb * 8192, &tm_xb, k0, jb * kMB, &s.full[st]);
         }
     } else if (warp == 1 && lane == 0) {             // ---- MMA issuer
-        constexpr uint32_t idesc = umma_idesc_bf16(128, 64) | (1u << 15);   // A is MN-major
+        constexpr uint32_t idesc = umma_idesc_bf16(128, 64 * NB) | (1u << 15);   // A is MN-major
         bool ok = true;
         for (int kb = 0; kb < nk && ok; ++kb) {
             const int st = kb % kFwdStages;
@@ -906,14 +917,14 @@ __global__ void __launch_bounds__(128) k_fwd1_tcgen05(const __grid_constant__ CU
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
     if (ok) {
         const int h = h0 + threadIdx.x;               // TMEM lane = hidden unit
-        float* out = zpart + ((size_t)split * d_h + h) * kMB;
 #pragma unroll 1
-        for (int p = 0; p < 2; ++p) {
+        for (int p = 0; p < 2 * NB; ++p) {           // 32 accumulator columns = half a micro-batch per step
+            float* out = zpart + (((size_t)(p >> 1) * kSplitK + split) * d_h + h) * kMB + (p & 1) * 32;
             uint32_t v[32];
             tmem_ld_32(tmem + ((uint32_t)(warp * 32) << 16) + (uint32_t)(p * 32), v);
 #pragma unroll
             for (int j = 0; j < 8; ++j)
-                *reinterpret_cast<float4*>(out + p * 32 + 4 * j) =
+                *reinterpret_cast<float4*>(out + 4 * j) =
                     make_float4(__uint_as_float(v[4 * j]), __uint_as_float(v[4 * j + 1]), __uint_as_float(v[4 * j + 2]),
                                 __uint_as_float(v[4 * j + 3]));
         }
@@ -925,8 +936,19 @@ __global__ void __launch_bounds__(128) k_fwd1_tcgen05(const __grid_constant__ CU
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
     __syncthreads();
     if (warp == 0) {
-        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(64) : "memory");
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(kTmemCols) : "memory");
     }
+}
+
+template <int NB>
+cudaError_t fwd1_set_attr() {
+    return cudaFuncSetAttribute(k_fwd1_tcgen05<NB>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                (int)sizeof(FwdSmem<NB>) + 1024);
+}
+template <int NB>
+void fwd1_launch(dim3 grid, cudaStream_t stream, const CUtensorMap& tw, const CUtensorMap& tx, float* zpart, int d_in,
+                 int d_h, int* status) {
+    k_fwd1_tcgen05<NB><<<grid, 128, sizeof(FwdSmem<NB>) + 1024, stream>>>(tw, tx, zpart, d_in, d_h, status);
 }
 
 // ---- host helpers --------------------------------------------------------------------------
@@ -1031,7 +1053,10 @@ cudaError_t mlp_scratch_init(MlpScratch* s, const MlpDims& d, void* base, __nv_b
         e = cudaFuncSetAttribute(k_dw1_regs, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                  dw_regs_buf_bytes(kMaxBatch) + (int)sizeof(DwRegCtl) + 1024);
     if (e == cudaSuccess)
-        e = cudaFuncSetAttribute(k_fwd1_tcgen05, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(FwdSmem) + 1024);
+        e = fwd1_set_attr<1>();
+        if (e == cudaSuccess) e = fwd1_set_attr<2>();
+        if (e == cudaSuccess) e = fwd1_set_attr<3>();
+        if (e == cudaSuccess) e = fwd1_set_attr<4>();
     if (e == cudaSuccess)
         e = cudaFuncSetAttribute(k_dw1_tcgen05<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(DwSmem) + 1024);
     if (e == cudaSuccess)
@@ -1065,8 +1090,13 @@ cudaError_t launch_mlp_front(const MlpDims& d, const MlpScratch& s, const float*
     } else {
         const CUtensorMap* tw = reinterpret_cast<const CUtensorMap*>(&s.tmap_w1[shadow_idx]);
         const CUtensorMap* tx = reinterpret_cast<const CUtensorMap*>(&s.tmap_xb);
-        k_fwd1_tcgen05<<<dim3(d.d_hidden / 128, nsplit, nb), 128, sizeof(FwdSmem) + 1024, stream>>>(*tw, *tx, s.zpart, d.d_in,
-                                                                                               d.d_hidden, s.status);
+        const dim3 grid(d.d_hidden / 128, nsplit);
+        switch (nb) {                                // the nb micro-batches are stacked along N of one GEMM
+            case 1: fwd1_launch<1>(grid, stream, *tw, *tx, s.zpart, d.d_in, d.d_hidden, s.status); break;
+            case 2: fwd1_launch<2>(grid, stream, *tw, *tx, s.zpart, d.d_in, d.d_hidden, s.status); break;
+            case 3: fwd1_launch<3>(grid, stream, *tw, *tx, s.zpart, d.d_in, d.d_hidden, s.status); break;
+            default: fwd1_launch<4>(grid, stream, *tw, *tx, s.zpart, d.d_in, d.d_hidden, s.status); break;
+        }
     }
     k_fwd2<<<dim3(n_cta, nb), 256, 0, stream>>>(s.zpart, nsplit, x_pub + o_b1, shadow + o_w2, s.hbt, s.lpart, s.gpart,
                                                 s.tickets, d.d_hidden, d.d_out);

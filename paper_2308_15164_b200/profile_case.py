@@ -2,7 +2,7 @@
 
     python -m paper_2308_15164_b200.profile_case sync       [--P 11689512] [--W 4] [--iters 3]
     python -m paper_2308_15164_b200.profile_case accumulate [--P 11689512] [--W 4] [--iters 3] [--bf16]
-    python -m paper_2308_15164_b200.profile_case mlp        [--iters 2]
+    python -m paper_2308_15164_b200.profile_case mlp        [--iters 2] [--batch 4]
 
 Each case keeps its working set larger than the 126 MB L2 but to a few hundred MB, launches the
 kernel of interest a handful of times and exits, so that a multi-pass capture ends by itself.
@@ -27,6 +27,7 @@ def main(argv=None):
     ap.add_argument("--bf16", action="store_true")
     ap.add_argument("--pipelined", action="store_true")
     ap.add_argument("--epilogue", type=int, default=0)
+    ap.add_argument("--batch", type=int, default=1, help="mlp: reference batches per call (1..4)")
     args = ap.parse_args(argv)
 
     from . import binding as B
@@ -61,7 +62,12 @@ def main(argv=None):
         c = 0
         for _ in range(args.iters + 1):
             for i in range(wl.W):
-                eng.accumulate_mlp(i, xs_d[c % 8], ys_d[c % 8]); c += 1
+                if args.batch > 1:
+                    lo = (c * args.batch) % 8 if 8 % args.batch == 0 else 0
+                    eng.accumulate_mlp_batch(i, args.batch, xs_d[lo:lo + args.batch], ys_d[lo:lo + args.batch])
+                else:
+                    eng.accumulate_mlp(i, xs_d[c % 8], ys_d[c % 8])
+                c += 1
             eng.sync_step()
         eng.check()
         eng.destroy()
