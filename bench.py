@@ -402,6 +402,9 @@ def run_mlp(B, wlm, dev, peaks, iters=12):
             n_dw, ms_dw = eng.kernel_stats(B.K_MLP_DW1)
             us_dw = ms_dw / n_dw * 1e3
             mean_n = n_mb / n_calls
+            for nm, k in (("us_fwd_3_kernels_per_call", B.K_MLP_FWD), ("us_bwd_per_call", B.K_MLP_BWD)):
+                n_k, ms_k = eng.kernel_stats(k)
+                res[nm] = ms_k / max(n_k, 1) * 1e3
             res.update({"us_dw1_per_call": us_dw, "mean_microbatches_per_call": mean_n,
                         "dw1_tflops": flop * mean_n / us_dw / 1e6,
                         "dw1_frac_of_bf16_peak_sustained": flop * mean_n / us_dw / 1e6 / peaks["bf16_tflops_sustained"],

@@ -73,7 +73,7 @@ Layout make_layout(const abs_config& c) {
         L.off_shadow[0] = take(L.P_pad * 2);
         L.off_shadow[1] = pipe ? take(L.P_pad * 2) : L.off_shadow[0];
         MlpDims d{(int)c.mlp_in, (int)c.mlp_hidden, (int)c.mlp_out, (int)c.mlp_mb};
-        L.off_mlp = take(2 * mlp_scratch_bytes(d));
+        L.off_mlp = take((size_t)kMlpSets * mlp_scratch_bytes(d));
     }
     if (c.flags & ABS_FLAG_HOST_INPUT) {
         const size_t es = c.grad_dtype == ABS_GRAD_BF16 ? 2 : 4;
@@ -117,12 +117,18 @@ struct abs_ctx {
     int stage_next = 0;
     int ctas_per_sm[ABS_K_COUNT] = {0, 0, 0, 0, 0};
     MlpDims mlp_dims{0, 0, 0, 0};
-    MlpScratch mlp_scratch[2]{};         // two sets: front part of micro-batch n+1 overlaps dW1 of micro-batch n
-    cudaStream_t s_dw = nullptr;         // internal stream of the dW1 GEMMs
-    cudaEvent_t ev_front_done[2] = {nullptr, nullptr}, ev_dw_done[2] = {nullptr, nullptr};
-    bool slot_used[2] = {false, false};
-    int mlp_slot = 0, dw_last_slot = 0;
-    bool dw_outstanding = false;         // a dW1 kernel was enqueued since stream_acc last waited for that stream
+    // The paper's workers compute concurrently: the gradient kernels of worker i run on internal stream
+    // i % n_wstreams (calls of one worker stay in order: its accumulator is added to in call order), each call
+    // in its own scratch set, taken round-robin.
+    MlpScratch mlp_scratch[kMlpSets]{};
+    cudaStream_t s_w[kMlpStreams] = {};
+    int n_wstreams = 0;
+    cudaEvent_t ev_fork = nullptr;                 // stream_acc -> worker stream (re-recorded per call)
+    cudaEvent_t ev_set_done[kMlpSets] = {};        // last use of a scratch set has finished
+    cudaEvent_t ev_w_done[kMlpStreams] = {};       // newest call enqueued on a worker stream has finished
+    bool set_used[kMlpSets] = {};
+    bool w_outstanding[kMlpStreams] = {};          // enqueued since stream_acc last waited for that stream
+    int mlp_set_next = 0;
     std::vector<TmapBytes> acc_tmaps;   // [2][W]: TMA descriptor of each accumulator row's W1 slice
 
     // bookkeeping
@@ -217,12 +223,13 @@ int collect_timings(abs_ctx* c) {
 
 void mlp_mark(void* user, int kernel_class, int n, cudaStream_t stream);
 
-// stream_acc waits (on the device) for every dW1 GEMM enqueued so far on the internal stream.
+// stream_acc waits (on the device) for every gradient kernel enqueued so far on the worker streams.
 int join_dw(abs_ctx* c) {
-    if (c->dw_outstanding) {
-        CK(cudaStreamWaitEvent(c->s_acc, c->ev_dw_done[c->dw_last_slot], 0));
-        c->dw_outstanding = false;
-    }
+    for (int k = 0; k < c->n_wstreams; ++k)
+        if (c->w_outstanding[k]) {
+            CK(cudaStreamWaitEvent(c->s_acc, c->ev_w_done[k], 0));
+            c->w_outstanding[k] = false;
+        }
     return ABS_OK;
 }
 
@@ -326,20 +333,20 @@ int abs_init(abs_ctx** out, const abs_config* cfg, void* workspace_dev, size_t w
         if (c->pipelined && (e = cudaMemsetAsync(c->ws + L.off_shadow[1], 0, L.P_pad * 2, c->s_acc)) != cudaSuccess)
             return bail(e, "cudaMemsetAsync");
         const size_t one = mlp_scratch_bytes(c->mlp_dims);
-        for (int k = 0; k < 2; ++k) {
+        for (int k = 0; k < kMlpSets; ++k) {
             if ((e = mlp_scratch_init(&c->mlp_scratch[k], c->mlp_dims, c->ws + L.off_mlp + k * one, c->shadow(0), c->shadow(1),
                                       &msg)) != cudaSuccess)
                 return bail(e, msg ? msg : "mlp_scratch_init");
             if ((e = cudaMemsetAsync(c->mlp_scratch[k].zero_from, 0, c->mlp_scratch[k].zero_bytes, c->s_acc)) != cudaSuccess)
                 return bail(e, "cudaMemsetAsync");
-            if ((e = cudaEventCreateWithFlags(&c->ev_front_done[k], cudaEventDisableTiming)) != cudaSuccess) return bail(e, "cudaEventCreate");
-            if ((e = cudaEventCreateWithFlags(&c->ev_dw_done[k], cudaEventDisableTiming)) != cudaSuccess) return bail(e, "cudaEventCreate");
+            if ((e = cudaEventCreateWithFlags(&c->ev_set_done[k], cudaEventDisableTiming)) != cudaSuccess) return bail(e, "cudaEventCreate");
         }
-        // Lowest priority: when CTA slots free up, the short front kernels of the next micro-batch (on
-        // stream_acc) are placed before the remaining CTAs of the long, bandwidth-bound dW1 kernel.
-        int prio_lo = 0, prio_hi = 0;
-        if ((e = cudaDeviceGetStreamPriorityRange(&prio_lo, &prio_hi)) != cudaSuccess) return bail(e, "cudaDeviceGetStreamPriorityRange");
-        if ((e = cudaStreamCreateWithPriority(&c->s_dw, cudaStreamNonBlocking, prio_lo)) != cudaSuccess) return bail(e, "cudaStreamCreate");
+        if ((e = cudaEventCreateWithFlags(&c->ev_fork, cudaEventDisableTiming)) != cudaSuccess) return bail(e, "cudaEventCreate");
+        c->n_wstreams = (int)std::min<uint32_t>(cfg->W, kMlpStreams);
+        for (int k = 0; k < c->n_wstreams; ++k) {
+            if ((e = cudaStreamCreateWithFlags(&c->s_w[k], cudaStreamNonBlocking)) != cudaSuccess) return bail(e, "cudaStreamCreate");
+            if ((e = cudaEventCreateWithFlags(&c->ev_w_done[k], cudaEventDisableTiming)) != cudaSuccess) return bail(e, "cudaEventCreate");
+        }
         c->acc_tmaps.resize((size_t)2 * cfg->W);
         for (uint32_t set = 0; set < 2; ++set)
             for (uint32_t i = 0; i < cfg->W; ++i)
@@ -413,34 +420,37 @@ int abs_accumulate_mlp_batch(abs_ctx* c, uint32_t worker, uint32_t n, const floa
     if (n == 0 || n > (uint32_t)kMlpMaxBatch) return invalid(c, "n must be in 1..4");
     if (!x_dev || (reinterpret_cast<uintptr_t>(x_dev) & 15)) return invalid(c, "x pointer must be non-NULL and 16-byte aligned");
     if (!y_dev || (reinterpret_cast<uintptr_t>(y_dev) & 3)) return invalid(c, "y pointer must be non-NULL and 4-byte aligned");
-    // Two scratch sets and a second stream: the latency-bound front part (cast, forward, loss,
-    // layer-2 backward) of the next call runs on stream_acc while the HBM-bound dW1 GEMM of
-    // this one runs on the internal stream.  dW1 kernels stay in call order on that stream.
-    const int k = c->mlp_slot;
-    c->mlp_slot ^= 1;
+    // Only the cast kernel reads the caller's buffers; it runs on stream_acc, in call order.  The rest of the
+    // call (forward, loss, backward, dW1) runs on the worker's internal stream, so that the latency chains of
+    // different workers overlap and the HBM-bound dW1 GEMMs fill the gaps of the small kernels.
+    const int set = c->mlp_set_next;
+    c->mlp_set_next = (set + 1) % kMlpSets;
+    const int k = (int)(worker % (uint32_t)c->n_wstreams);
     const int variant = c->ctas_per_sm[ABS_K_MLP_DW1];
     const bool serial = c->ctas_per_sm[ABS_K_MLP_FWD] == 1;   // measurement aid: everything on stream_acc
     if (serial) {
         if (int rc = join_dw(c)) return rc;
-    } else if (c->slot_used[k]) {
-        CK(cudaStreamWaitEvent(c->s_acc, c->ev_dw_done[k], 0));   // scratch set k is free again
+    } else if (c->set_used[set]) {
+        CK(cudaStreamWaitEvent(c->s_acc, c->ev_set_done[set], 0));   // the scratch set is free again
     }
-    CK(launch_mlp_front(c->mlp_dims, c->mlp_scratch[k], c->x(c->pub), c->shadow(c->pub), c->pub, (int)n, x_dev, y_dev,
-                        c->acc(c->cur, worker), c->cnt(c->cur, worker), variant, c->s_acc, mlp_mark, c));
-    cudaStream_t s_gemm = serial ? c->s_acc : c->s_dw;
+    const MlpScratch& sc = c->mlp_scratch[set];
+    CK(launch_mlp_cast(c->mlp_dims, sc, (int)n, x_dev, y_dev, c->s_acc, mlp_mark, c));
+    cudaStream_t s_run = serial ? c->s_acc : c->s_w[k];
     if (!serial) {
-        CK(cudaEventRecord(c->ev_front_done[k], c->s_acc));
-        CK(cudaStreamWaitEvent(c->s_dw, c->ev_front_done[k], 0));
+        CK(cudaEventRecord(c->ev_fork, c->s_acc));
+        CK(cudaStreamWaitEvent(s_run, c->ev_fork, 0));
     }
-    CK(launch_mlp_dw1(c->mlp_dims, c->mlp_scratch[k], c->acc(c->cur, worker),
-                      &c->acc_tmaps[(size_t)c->cur * c->cfg.W + worker], (int)n, variant, s_gemm, mlp_mark, c));
+    CK(launch_mlp_front(c->mlp_dims, sc, c->x(c->pub), c->shadow(c->pub), c->pub, (int)n, c->acc(c->cur, worker),
+                        c->cnt(c->cur, worker), variant, s_run, mlp_mark, c));
+    CK(launch_mlp_dw1(c->mlp_dims, sc, c->acc(c->cur, worker), &c->acc_tmaps[(size_t)c->cur * c->cfg.W + worker], (int)n,
+                      variant, s_run, mlp_mark, c));
     if (serial) {
-        c->slot_used[0] = c->slot_used[1] = false;
+        for (bool& u : c->set_used) u = false;
     } else {
-        CK(cudaEventRecord(c->ev_dw_done[k], c->s_dw));
-        c->slot_used[k] = true;
-        c->dw_outstanding = true;
-        c->dw_last_slot = k;
+        CK(cudaEventRecord(c->ev_set_done[set], s_run));
+        CK(cudaEventRecord(c->ev_w_done[k], s_run));
+        c->set_used[set] = true;
+        c->w_outstanding[k] = true;
     }
     c->h_cnt[(size_t)c->cur * c->cfg.W + worker] += (int32_t)n;
     return ABS_OK;
@@ -587,13 +597,16 @@ int abs_wait(abs_ctx* c) {
 int abs_check(abs_ctx* c) {
     if (!live(c)) return ABS_ESTATE;
     if (c->pipelined) CK(cudaStreamSynchronize(c->s_sync));
-    if (c->s_dw) CK(cudaStreamSynchronize(c->s_dw));
+    for (int k = 0; k < c->n_wstreams; ++k) CK(cudaStreamSynchronize(c->s_w[k]));
     CK(cudaStreamSynchronize(c->s_acc));
     if (c->mlp) {
-        int st = 0, st1 = 0;
-        CK(cudaMemcpy(&st, c->mlp_scratch[0].status, sizeof(int), cudaMemcpyDeviceToHost));
-        CK(cudaMemcpy(&st1, c->mlp_scratch[1].status, sizeof(int), cudaMemcpyDeviceToHost));
-        if (st != 0 || st1 != 0) {
+        int bad = 0;
+        for (int k = 0; k < kMlpSets; ++k) {
+            int st = 0;
+            CK(cudaMemcpy(&st, c->mlp_scratch[k].status, sizeof(int), cudaMemcpyDeviceToHost));
+            bad |= st;
+        }
+        if (bad != 0) {
             c->err = "a bounded device-side wait ran out (MLP dW1 kernel)";
             return ABS_ETIMEOUT;
         }
@@ -647,9 +660,11 @@ int abs_destroy(abs_ctx* c) {
     cudaStreamSynchronize(c->s_acc);
     if (c->pipelined) cudaStreamSynchronize(c->s_sync);
     if (c->s_copy) { cudaStreamSynchronize(c->s_copy); cudaStreamDestroy(c->s_copy); }
-    if (c->s_dw) { cudaStreamSynchronize(c->s_dw); cudaStreamDestroy(c->s_dw); }
-    for (cudaEvent_t e : {c->ev_front_done[0], c->ev_front_done[1], c->ev_dw_done[0], c->ev_dw_done[1]})
-        if (e) cudaEventDestroy(e);
+    for (int k = 0; k < c->n_wstreams; ++k)
+        if (c->s_w[k]) { cudaStreamSynchronize(c->s_w[k]); cudaStreamDestroy(c->s_w[k]); }
+    for (cudaEvent_t e : c->ev_set_done) if (e) cudaEventDestroy(e);
+    for (cudaEvent_t e : c->ev_w_done) if (e) cudaEventDestroy(e);
+    if (c->ev_fork) cudaEventDestroy(c->ev_fork);
     for (auto& tl : c->timed) { cudaEventDestroy(tl.start); cudaEventDestroy(tl.stop); }
     for (auto e : c->ev_pool) cudaEventDestroy(e);
     for (cudaEvent_t e : {c->ev_acc_done, c->ev_sync_done, c->ev_aux, c->ev_stage_free[0], c->ev_stage_free[1],

@@ -44,6 +44,8 @@ cudaError_t launch_cast_bf16(const float* src, __nv_bfloat16* dst, size_t n, int
 
 // ---- MLP micro-batch gradient (Step 2 with the gradient computed on the device) ----------
 constexpr int kMlpMaxBatch = 4;
+constexpr int kMlpStreams = 4;   // internal worker streams (worker i runs on stream i % kMlpStreams)
+constexpr int kMlpSets = 8;      // scratch sets, one per call in flight, taken round-robin
 struct MlpDims {
     int d_in, d_hidden, d_out, mb;
 };
@@ -58,6 +60,7 @@ struct MlpScratch {      // device pointers carved from the workspace (all hidde
     __nv_bfloat16* dzt;  // [4][d_hidden][mb]     bf16(dZ)^T of up to 4 stacked micro-batches: K-major B operand of dW1
     float* lpart;        // [d_hidden/32][mb][16] partial logits per CTA of k_fwd2
     float* gpart;        // [groups][mb][16]      partial logits per group of 8 CTAs
+    int32_t* ycopy;      // [4][mb]               labels of the call's micro-batches (copied by k_cast_x)
     float* bpart;        // [4][d_hidden/32][4][256] partial dW2 / db1 / db2 sums of k_bwd, per micro-batch of a call
     unsigned int* tickets_b;  // [d_hidden/32]     "last CTA done" tickets of k_bwd (zero between launches)
     unsigned int* tickets;  // [groups]           "last CTA done" tickets of the logit reduction (zero between launches)
@@ -74,9 +77,10 @@ cudaError_t mlp_scratch_init(MlpScratch* s, const MlpDims& d, void* base, __nv_b
                              __nv_bfloat16* shadow1, const char** err);
 // TMA descriptor of the W1 slice of one worker's accumulator row (fp32 [d_in][d_hidden]).
 cudaError_t mlp_make_acc_tmap(void* tmap_out, const MlpDims& d, float* acc_row);
-// The micro-batch gradient is enqueued in two parts so that the caller can put them on different streams:
-//   front: cast, forward GEMM, loss, layer-2 backward (writes dzt/xtb of this scratch set; adds db2, db1, dW2
-//          into acc_row; bumps cnt);   dw1: the dW1 GEMM, which reads xtb/dzt and adds into the W1 slice.
+// The gradient of a call is enqueued in three parts so that the caller can put them on different streams:
+//   cast:  the only part that reads the caller's x_dev / y_dev (bf16 copies and labels into this scratch set);
+//   front: forward GEMM, loss, layer-2 backward (writes dzt of this scratch set; adds db2, db1, dW2 into
+//          acc_row; bumps cnt);   dw1: the dW1 GEMM, which reads xtb/dzt and adds into the W1 slice.
 // shadow: bf16 copy of the published parameters (same flat layout), shadow_idx: which of the two copies it is.
 // x_pub: the fp32 parameters.  variant: bit 0 = dW1 epilogue by TMA reduce-add (else TMA load + add + TMA
 // store); bit 1 = forward GEMM on CUDA cores (cross-check of the tcgen05 one); bit 2 = persistent dW1 kernel;
@@ -84,9 +88,11 @@ cudaError_t mlp_make_acc_tmap(void* tmap_out, const MlpDims& d, float* acc_row);
 // mark(user, kernel_class, 0, stream) is called before a kernel group, mark(user, kernel_class, n, stream) after
 // its n launches.
 typedef void (*MlpMark)(void* user, int kernel_class, int n, cudaStream_t stream);
+cudaError_t launch_mlp_cast(const MlpDims& d, const MlpScratch& s, int nb, const float* x_dev, const int32_t* y_dev,
+                            cudaStream_t stream, MlpMark mark, void* user);
 cudaError_t launch_mlp_front(const MlpDims& d, const MlpScratch& s, const float* x_pub, const __nv_bfloat16* shadow,
-                             int shadow_idx, int nb, const float* x_dev, const int32_t* y_dev, float* acc_row, int32_t* cnt,
-                             int variant, cudaStream_t stream, MlpMark mark, void* user);
+                             int shadow_idx, int nb, float* acc_row, int32_t* cnt, int variant, cudaStream_t stream,
+                             MlpMark mark, void* user);
 // nb: a call may carry up to kMlpMaxBatch micro-batches (x_dev [nb][mb][d_in], y_dev [nb][mb]): the front kernels
 // take them as an extra grid dimension, and ONE dW1 launch contracts them with K = 64 nb (the accumulator slice is
 // read and written once).

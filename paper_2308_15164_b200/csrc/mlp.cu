@@ -13,8 +13,8 @@
 // K = mb = 64), K-major: A = X^T stored [d_in][64], B = dZ^T stored [d_h][64].  A 64-element
 // bf16 row is exactly one 128-byte swizzle row, so each operand tile is one TMA box.
 //
-// Kernels (five launches per micro-batch; the first four form the "front" part, the last one
-// may run on another stream):
+// Kernels (five launches per call of 1..4 micro-batches; only the first reads the caller's buffers, the
+// others may run on another stream):
 //   k_cast_x        X fp32 -> bf16 in both orientations
 //   k_fwd1_tcgen05  Z^T partials = W1^T X^T, split over d_in, on tcgen05 (W1 as an MN-major operand)
 //   (k_fwd1         the same on CUDA cores, kept as a cross-check selectable through abs_set_launch)
@@ -50,11 +50,15 @@ __device__ __forceinline__ uint32_t pack_bf16x2(float a, float b) {
 
 // --------------------------------------------------------------------------------------------
 // X [64][d_in] fp32  ->  xb [64][d_in] bf16  and  xtb [d_in][64] bf16.   CTA: 16 columns.
+// Also copies the labels, so that the caller's buffers are read by this kernel only (the rest of
+// the gradient may run on another stream after the caller's stream has moved on).
 // --------------------------------------------------------------------------------------------
-__global__ void __launch_bounds__(256) k_cast_x(const float* __restrict__ x, __nv_bfloat16* __restrict__ xb,
-                                                __nv_bfloat16* __restrict__ xtb, int d_in) {
+__global__ void __launch_bounds__(256) k_cast_x(const float* __restrict__ x, const int32_t* __restrict__ y,
+                                                __nv_bfloat16* __restrict__ xb, __nv_bfloat16* __restrict__ xtb,
+                                                int32_t* __restrict__ ycopy, int d_in) {
     __shared__ __nv_bfloat16 tile[16][kMB + 8];
     const int c0 = blockIdx.x * 16;
+    if (blockIdx.x == 0 && threadIdx.x < kMB) ycopy[blockIdx.y * kMB + threadIdx.x] = y[blockIdx.y * kMB + threadIdx.x];
     x += (size_t)blockIdx.y * kMB * d_in;      // micro-batch blockIdx.y of the call
     xb += (size_t)blockIdx.y * kMB * d_in;
     xtb += (size_t)blockIdx.y * d_in * kMB;
@@ -997,6 +1001,7 @@ size_t layout_scratch(MlpScratch* s, const MlpDims& d, char* base) {
     char* lpart = take((size_t)kMaxBatch * n_cta * kMB * kOutPad * 4);
     char* gpart = take((size_t)kMaxBatch * n_groups * kMB * kOutPad * 4);
     char* bpart = take((size_t)kMaxBatch * n_cta * 4 * 256 * 4);
+    char* ycopy = take((size_t)kMaxBatch * kMB * 4);
     char* tickets = take((size_t)(kMaxBatch * n_groups + n_cta) * 4);   // k_fwd2 group tickets, then k_bwd chunk tickets
     char* status = take(256);
     if (s) {
@@ -1010,6 +1015,7 @@ size_t layout_scratch(MlpScratch* s, const MlpDims& d, char* base) {
         s->tickets = reinterpret_cast<unsigned int*>(tickets);
         s->tickets_b = reinterpret_cast<unsigned int*>(tickets) + kMaxBatch * n_groups;
         s->bpart = reinterpret_cast<float*>(bpart);
+        s->ycopy = reinterpret_cast<int32_t*>(ycopy);
         s->status = reinterpret_cast<int*>(status);
         s->zero_from = tickets;
         s->zero_bytes = (size_t)(status + 256 - tickets);
@@ -1073,16 +1079,21 @@ cudaError_t mlp_make_acc_tmap(void* tmap_out, const MlpDims& d, float* acc_row) 
                : cudaErrorInvalidValue;
 }
 
+cudaError_t launch_mlp_cast(const MlpDims& d, const MlpScratch& s, int nb, const float* x_dev, const int32_t* y_dev,
+                            cudaStream_t stream, MlpMark mark, void* user) {
+    mark(user, ABS_K_MLP_FWD, 0, stream);
+    k_cast_x<<<dim3(d.d_in / 16, nb), 256, 0, stream>>>(x_dev, y_dev, s.xb, s.xtb, s.ycopy, d.d_in);
+    return cudaGetLastError();
+}
+
 cudaError_t launch_mlp_front(const MlpDims& d, const MlpScratch& s, const float* x_pub, const __nv_bfloat16* shadow,
-                             int shadow_idx, int nb, const float* x_dev, const int32_t* y_dev, float* acc_row, int32_t* cnt,
-                             int variant, cudaStream_t stream, MlpMark mark, void* user) {
+                             int shadow_idx, int nb, float* acc_row, int32_t* cnt, int variant, cudaStream_t stream,
+                             MlpMark mark, void* user) {
     const size_t o_b1 = (size_t)d.d_in * d.d_hidden, o_w2 = o_b1 + d.d_hidden, o_b2 = o_w2 + (size_t)d.d_hidden * d.d_out;
     cudaError_t e;
     const unsigned n_cta = d.d_hidden / kHB;
 
     // every kernel carries the nb micro-batches of the call as an extra grid dimension
-    mark(user, ABS_K_MLP_FWD, 0, stream);
-    k_cast_x<<<dim3(d.d_in / 16, nb), 256, 0, stream>>>(x_dev, s.xb, s.xtb, d.d_in);
     // every K split must be a whole number of 64-wide pipeline steps (d_in is a multiple of 128)
     const int nsplit = (d.d_in % (64 * kSplitK) == 0) ? kSplitK : 2;
     if (variant & 2) {
@@ -1105,7 +1116,7 @@ cudaError_t launch_mlp_front(const MlpDims& d, const MlpScratch& s, const float*
 
     mark(user, ABS_K_MLP_BWD, 0, stream);
     const int n_groups = (n_cta + kGroup - 1) / kGroup;
-    k_bwd<<<dim3(n_cta, nb), 256, 0, stream>>>(s.hbt, s.gpart, n_groups, x_pub + o_b2, y_dev, shadow + o_w2, s.dzt, s.bpart,
+    k_bwd<<<dim3(n_cta, nb), 256, 0, stream>>>(s.hbt, s.gpart, n_groups, x_pub + o_b2, s.ycopy, shadow + o_w2, s.dzt, s.bpart,
                                                s.tickets_b, acc_row + o_b1, acc_row + o_w2, acc_row + o_b2, cnt, d.d_hidden,
                                                d.d_out);
     mark(user, ABS_K_MLP_BWD, 1, stream);
