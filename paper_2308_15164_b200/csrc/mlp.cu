@@ -920,17 +920,29 @@ __global__ void __launch_bounds__(128) k_fwd1_tcgen05(const __grid_constant__ CU
     ok = __all_sync(0xffffffffu, ok);
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
     if (ok) {
-        const int h = h0 + threadIdx.x;               // TMEM lane = hidden unit
+        // A thread holds one hidden unit's row (TMEM lane), 32 columns per load; stored directly, a warp
+        // would write 32 rows x 16 bytes per instruction.  Each warp turns its 32 x 32 block round through
+        // shared memory (stage 0 is free: every load has landed and every MMA has completed; pitch 36
+        // floats: conflict-free both ways) and stores 4 rows x 128 contiguous bytes per instruction.
+        constexpr int kPitch = 36;
+        float* tr = reinterpret_cast<float*>(s.stage[0]) + warp * 32 * kPitch;
 #pragma unroll 1
         for (int p = 0; p < 2 * NB; ++p) {           // 32 accumulator columns = half a micro-batch per step
-            float* out = zpart + (((size_t)(p >> 1) * kSplitK + split) * d_h + h) * kMB + (p & 1) * 32;
             uint32_t v[32];
             tmem_ld_32(tmem + ((uint32_t)(warp * 32) << 16) + (uint32_t)(p * 32), v);
 #pragma unroll
             for (int j = 0; j < 8; ++j)
-                *reinterpret_cast<float4*>(out + 4 * j) =
+                *reinterpret_cast<float4*>(tr + lane * kPitch + 4 * j) =
                     make_float4(__uint_as_float(v[4 * j]), __uint_as_float(v[4 * j + 1]), __uint_as_float(v[4 * j + 2]),
                                 __uint_as_float(v[4 * j + 3]));
+            __syncwarp();
+            float* out = zpart + (((size_t)(p >> 1) * kSplitK + split) * d_h + h0 + warp * 32) * kMB + (p & 1) * 32;
+#pragma unroll
+            for (int it = 0; it < 8; ++it) {
+                const int row = it * 4 + lane / 8, c4 = (lane % 8) * 4;
+                *reinterpret_cast<float4*>(out + (size_t)row * kMB + c4) = *reinterpret_cast<const float4*>(tr + row * kPitch + c4);
+            }
+            __syncwarp();
         }
     } else if (threadIdx.x == 0) {
         atomicExch(status, ABS_ETIMEOUT);
