@@ -67,7 +67,9 @@ extern "C" {
                                        (acc = g) rather than adds.  Same results; the fused step moves
                                        4*W_act + 16 instead of 8*W_act + 16 bytes per parameter and those first
                                        accumulates 8 (6 for bf16) instead of 12 (10).  Rows of workers that were
-                                       idle keep stale values (never read).  Not available with ABS_FLAG_MLP. */
+                                       idle keep stale values (never read).  abs_accumulate_mlp* store a worker's
+                                       first gradient of an iteration in either mode (the row is then known
+                                       to be empty), which saves the read of the W1 slice.                    */
 
 #define ABS_MAX_WORKERS 64u
 

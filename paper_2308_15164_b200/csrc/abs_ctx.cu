@@ -42,8 +42,6 @@ bool config_ok(const abs_config* c, std::string* why) {
         return fail("lr, momentum, weight_decay and lambda_dc must be finite");
     if ((c->flags & ABS_FLAG_PIPELINED) && c->stream_acc == c->stream_sync)
         return fail("pipelined mode needs two different streams");
-    if ((c->flags & ABS_FLAG_MLP) && (c->flags & ABS_FLAG_OVERWRITE_FIRST))
-        return fail("ABS_FLAG_OVERWRITE_FIRST is not available with ABS_FLAG_MLP");
     if (c->flags & ABS_FLAG_MLP) {
         if (c->mlp_in == 0 || c->mlp_in % 128 || c->mlp_hidden == 0 || c->mlp_hidden % 128)
             return fail("mlp_in and mlp_hidden must be positive multiples of 128");
@@ -434,16 +432,20 @@ int abs_accumulate_mlp_batch(abs_ctx* c, uint32_t worker, uint32_t n, const floa
         CK(cudaStreamWaitEvent(c->s_acc, c->ev_set_done[set], 0));   // the scratch set is free again
     }
     const MlpScratch& sc = c->mlp_scratch[set];
+    // A worker's first gradient of an iteration finds its accumulator row empty (all zero, or -- with
+    // ABS_FLAG_OVERWRITE_FIRST -- stale): it is stored, not added, and dW1 skips reading the 4 d_in d_hidden
+    // bytes of the slice.  0 + g = g, so the default mode's results do not change.
+    const bool first = c->h_cnt[(size_t)c->cur * c->cfg.W + worker] == 0;
     CK(launch_mlp_cast(c->mlp_dims, sc, (int)n, x_dev, y_dev, c->s_acc, mlp_mark, c));
     cudaStream_t s_run = serial ? c->s_acc : c->s_w[k];
     if (!serial) {
         CK(cudaEventRecord(c->ev_fork, c->s_acc));
         CK(cudaStreamWaitEvent(s_run, c->ev_fork, 0));
     }
-    CK(launch_mlp_front(c->mlp_dims, sc, c->x(c->pub), c->shadow(c->pub), c->pub, (int)n, c->acc(c->cur, worker),
+    CK(launch_mlp_front(c->mlp_dims, sc, c->x(c->pub), c->shadow(c->pub), c->pub, (int)n, first, c->acc(c->cur, worker),
                         c->cnt(c->cur, worker), variant, s_run, mlp_mark, c));
     CK(launch_mlp_dw1(c->mlp_dims, sc, c->acc(c->cur, worker), &c->acc_tmaps[(size_t)c->cur * c->cfg.W + worker], (int)n,
-                      variant, s_run, mlp_mark, c));
+                      first, variant, s_run, mlp_mark, c));
     if (serial) {
         for (bool& u : c->set_used) u = false;
     } else {

@@ -91,12 +91,14 @@ typedef void (*MlpMark)(void* user, int kernel_class, int n, cudaStream_t stream
 cudaError_t launch_mlp_cast(const MlpDims& d, const MlpScratch& s, int nb, const float* x_dev, const int32_t* y_dev,
                             cudaStream_t stream, MlpMark mark, void* user);
 cudaError_t launch_mlp_front(const MlpDims& d, const MlpScratch& s, const float* x_pub, const __nv_bfloat16* shadow,
-                             int shadow_idx, int nb, float* acc_row, int32_t* cnt, int variant, cudaStream_t stream,
-                             MlpMark mark, void* user);
+                             int shadow_idx, int nb, bool store, float* acc_row, int32_t* cnt, int variant,
+                             cudaStream_t stream, MlpMark mark, void* user);
 // nb: a call may carry up to kMlpMaxBatch micro-batches (x_dev [nb][mb][d_in], y_dev [nb][mb]): the front kernels
 // take them as an extra grid dimension, and ONE dW1 launch contracts them with K = 64 nb (the accumulator slice is
 // read and written once).
-cudaError_t launch_mlp_dw1(const MlpDims& d, const MlpScratch& s, float* acc_row, const void* acc_tmap, int nb, int variant,
-                           cudaStream_t stream, MlpMark mark, void* user);
+// store: the accumulator row holds nothing yet (the worker's first gradient of the iteration): front and dw1
+// store their results instead of adding them, and dw1 does not read the accumulator slice at all.
+cudaError_t launch_mlp_dw1(const MlpDims& d, const MlpScratch& s, float* acc_row, const void* acc_tmap, int nb, bool store,
+                           int variant, cudaStream_t stream, MlpMark mark, void* user);
 
 }  // namespace abs_sgd

@@ -223,7 +223,7 @@ __global__ void __launch_bounds__(256) k_bwd(const __nv_bfloat16* hbt, const flo
                                              const float* __restrict__ b2, const int32_t* y,
                                              const __nv_bfloat16* __restrict__ w2b, __nv_bfloat16* dzt, float* bpart,
                                              unsigned int* tickets_b, float* acc_b1, float* acc_w2, float* acc_b2,
-                                             int32_t* cnt, int d_h, int d_out) {
+                                             int32_t* cnt, int d_h, int d_out, int store) {
     __shared__ float sdl[kMB][kOutPad + 1];     // bf16(dL) as float (first: the logits)
     __shared__ float sdl32[kMB][kOutPad + 1];   // dL unrounded (CTA 0: db2)
     __shared__ float sw2[kHB][kOutPad];
@@ -329,10 +329,17 @@ __global__ void __launch_bounds__(256) k_bwd(const __nv_bfloat16* hbt, const flo
             }
             if (threadIdx.x == 0) tickets_b[blockIdx.x] = 0u;
         }
-        if (slot < d_out) acc_w2[(size_t)h * d_out + slot] += a;
-        if (slot + 8 < d_out) acc_w2[(size_t)h * d_out + slot + 8] += b;
-        if (slot == 0) acc_b1[h] += c;
-        if (blockIdx.x == 0 && threadIdx.x < d_out) acc_b2[threadIdx.x] += db2;
+        if (store) {   // a worker's first gradient of the iteration: the slices hold nothing yet
+            if (slot < d_out) acc_w2[(size_t)h * d_out + slot] = a;
+            if (slot + 8 < d_out) acc_w2[(size_t)h * d_out + slot + 8] = b;
+            if (slot == 0) acc_b1[h] = c;
+            if (blockIdx.x == 0 && threadIdx.x < d_out) acc_b2[threadIdx.x] = db2;
+        } else {
+            if (slot < d_out) acc_w2[(size_t)h * d_out + slot] += a;
+            if (slot + 8 < d_out) acc_w2[(size_t)h * d_out + slot + 8] += b;
+            if (slot == 0) acc_b1[h] += c;
+            if (blockIdx.x == 0 && threadIdx.x < d_out) acc_b2[threadIdx.x] += db2;
+        }
         if (blockIdx.x == 0 && threadIdx.x == 0) cnt[0] += nb;   // M_t^i += nb * M_r
     }
 }
@@ -465,10 +472,14 @@ struct DwSmem {
 template <bool kReduce>
 __global__ void __launch_bounds__(128) k_dw1_tcgen05(const __grid_constant__ CUtensorMap tm_xt,
                                                      const __grid_constant__ CUtensorMap tm_dzt,
-                                                     const __grid_constant__ CUtensorMap tm_acc, int* status) {
+                                                     const __grid_constant__ CUtensorMap tm_acc, int store,
+                                                     int* status) {
+    // store != 0: the accumulator slice is known to hold nothing yet (a worker's first gradient of the
+    // iteration): the tile is not read, the product is stored instead of added.
     extern __shared__ uint8_t smem_raw[];
     DwSmem& s = *reinterpret_cast<DwSmem*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
     const int warp = threadIdx.x / 32;
+    const bool load_c = !kReduce && !store;
     const int n0 = blockIdx.x * kDwN;     // hidden offset
     const int m0 = blockIdx.y * kTileM;   // input-feature offset
 
@@ -492,7 +503,7 @@ __global__ void __launch_bounds__(128) k_dw1_tcgen05(const __grid_constant__ CUt
         mbar_expect_tx(&s.bar_ab, kTileM * 128 + kDwN * 128);
         tma_load_2d(s.a, &tm_xt, 0, m0, &s.bar_ab);
         tma_load_2d(s.b, &tm_dzt, 0, n0, &s.bar_ab);
-        if (!kReduce) {   // the accumulator tile streams in while the MMA runs
+        if (load_c) {   // the accumulator tile streams in while the MMA runs
             mbar_expect_tx(&s.bar_c, kTileM * kDwN * 4);
 #pragma unroll
             for (int p = 0; p < kPanels; ++p) tma_load_2d(s.c[p], &tm_acc, n0 + p * 32, m0, &s.bar_c);
@@ -513,7 +524,7 @@ __global__ void __launch_bounds__(128) k_dw1_tcgen05(const __grid_constant__ CUt
     __syncwarp();
 
     bool ok = mbar_wait(&s.bar_mma, 0);
-    if (!kReduce) ok = mbar_wait(&s.bar_c, 0) && ok;
+    if (load_c) ok = mbar_wait(&s.bar_c, 0) && ok;
     ok = __all_sync(0xffffffffu, ok);
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
     if (ok) {
@@ -522,7 +533,8 @@ __global__ void __launch_bounds__(128) k_dw1_tcgen05(const __grid_constant__ CUt
         for (int p = 0; p < kPanels; ++p) {
             uint32_t v[32];
             tmem_ld_32(tmem + ((uint32_t)(warp * 32) << 16) + (uint32_t)(p * 32), v);
-            panel_row_update<!kReduce>(s.c[p], row, v);
+            if (load_c) panel_row_update<true>(s.c[p], row, v);
+            else panel_row_update<false>(s.c[p], row, v);
         }
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // smem writes -> visible to the TMA engine
     } else {
@@ -534,7 +546,7 @@ __global__ void __launch_bounds__(128) k_dw1_tcgen05(const __grid_constant__ CUt
         if (!s.failed) {
 #pragma unroll
             for (int p = 0; p < kPanels; ++p) {
-                if (kReduce) tma_reduce_add_2d(&tm_acc, s.c[p], n0 + p * 32, m0);
+                if (kReduce && !store) tma_reduce_add_2d(&tm_acc, s.c[p], n0 + p * 32, m0);
                 else tma_store_2d(&tm_acc, s.c[p], n0 + p * 32, m0);
             }
             asm volatile("cp.async.bulk.commit_group;" ::: "memory");
@@ -544,7 +556,7 @@ __global__ void __launch_bounds__(128) k_dw1_tcgen05(const __grid_constant__ CUt
             atomicExch(status, ABS_ETIMEOUT);
             // give copies that may still be in flight a bounded chance to land before smem is released
             mbar_wait(&s.bar_ab, 0);
-            if (!kReduce) mbar_wait(&s.bar_c, 0);
+            if (load_c) mbar_wait(&s.bar_c, 0);
         }
     }
     __syncthreads();
@@ -583,7 +595,7 @@ __host__ __device__ constexpr int dw_regs_buf_bytes(int nb) {
 
 __global__ void __launch_bounds__(256) k_dw1_regs(const __grid_constant__ CUtensorMap tm_xt,
                                                   const __grid_constant__ CUtensorMap tm_dzt, float* acc_w1, int d_in,
-                                                  int ld, int nb, int* status) {
+                                                  int ld, int nb, int store, int* status) {
     extern __shared__ uint8_t smem_raw[];
     uint8_t* buf = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
     DwRegCtl& s = *reinterpret_cast<DwRegCtl*>(buf + dw_regs_buf_bytes(nb));
@@ -599,7 +611,7 @@ __global__ void __launch_bounds__(256) k_dw1_regs(const __grid_constant__ CUtens
 #pragma unroll
     for (int k = 0; k < kPer; ++k) {
         const int e = threadIdx.x + 256 * k;
-        c[k] = gbase[(size_t)(e / kC4) * ld4 + (e % kC4)];
+        c[k] = store ? make_float4(0.f, 0.f, 0.f, 0.f) : gbase[(size_t)(e / kC4) * ld4 + (e % kC4)];   // store: see k_dw1_tcgen05
     }
 
     if (warp == 0) {
@@ -704,7 +716,7 @@ struct DwPersistSmem {
 __global__ void __launch_bounds__(192) k_dw1_persistent(const __grid_constant__ CUtensorMap tm_xt,
                                                         const __grid_constant__ CUtensorMap tm_dzt,
                                                         const __grid_constant__ CUtensorMap tm_acc, int n_tiles_n,
-                                                        int n_tiles, int* status) {
+                                                        int n_tiles, int store, int* status) {
     extern __shared__ uint8_t smem_raw[];
     DwPersistSmem& s = *reinterpret_cast<DwPersistSmem*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
     const int warp = threadIdx.x / 32, lane = threadIdx.x % 32;
@@ -741,12 +753,14 @@ __global__ void __launch_bounds__(192) k_dw1_persistent(const __grid_constant__ 
                 const int t = (int)blockIdx.x + i * (int)gridDim.x;
                 const int n0 = (t % n_tiles_n) * kDwN, m0 = (t / n_tiles_n) * kTileM;
                 uint8_t* base = s.stage[st];
-                mbar_expect_tx(&s.full[st], kDwStageBytes);
+                mbar_expect_tx(&s.full[st], store ? kOffC : kDwStageBytes);   // store: see k_dw1_tcgen05
                 tma_load_2d(base, &tm_xt, 0, m0, &s.full[st]);
                 tma_load_2d(base + kOffB, &tm_dzt, 0, n0, &s.full[st]);
+                if (!store) {
 #pragma unroll
-                for (int p = 0; p < kPanels; ++p)
-                    tma_load_2d(base + kOffC + p * (kTileM * 128), &tm_acc, n0 + p * 32, m0, &s.full[st]);
+                    for (int p = 0; p < kPanels; ++p)
+                        tma_load_2d(base + kOffC + p * (kTileM * 128), &tm_acc, n0 + p * 32, m0, &s.full[st]);
+                }
             }
         }
     } else if (warp == 1) {
@@ -781,7 +795,8 @@ __global__ void __launch_bounds__(192) k_dw1_persistent(const __grid_constant__ 
                 for (int p = 0; p < kPanels; ++p) {
                     uint32_t v[32];
                     tmem_ld_32(tmem + ((uint32_t)(q * 32) << 16) + (uint32_t)(ab * kDwN + p * 32), v);
-                    panel_row_update<true>(cbase + p * (kTileM * 32), row, v);
+                    if (store) panel_row_update<false>(cbase + p * (kTileM * 32), row, v);
+                    else panel_row_update<true>(cbase + p * (kTileM * 32), row, v);
                 }
                 asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
                 mbar_arrive(&s.acc_empty[ab]);
@@ -1099,8 +1114,8 @@ cudaError_t launch_mlp_cast(const MlpDims& d, const MlpScratch& s, int nb, const
 }
 
 cudaError_t launch_mlp_front(const MlpDims& d, const MlpScratch& s, const float* x_pub, const __nv_bfloat16* shadow,
-                             int shadow_idx, int nb, float* acc_row, int32_t* cnt, int variant, cudaStream_t stream,
-                             MlpMark mark, void* user) {
+                             int shadow_idx, int nb, bool store, float* acc_row, int32_t* cnt, int variant,
+                             cudaStream_t stream, MlpMark mark, void* user) {
     const size_t o_b1 = (size_t)d.d_in * d.d_hidden, o_w2 = o_b1 + d.d_hidden, o_b2 = o_w2 + (size_t)d.d_hidden * d.d_out;
     cudaError_t e;
     const unsigned n_cta = d.d_hidden / kHB;
@@ -1130,13 +1145,14 @@ cudaError_t launch_mlp_front(const MlpDims& d, const MlpScratch& s, const float*
     const int n_groups = (n_cta + kGroup - 1) / kGroup;
     k_bwd<<<dim3(n_cta, nb), 256, 0, stream>>>(s.hbt, s.gpart, n_groups, x_pub + o_b2, s.ycopy, shadow + o_w2, s.dzt, s.bpart,
                                                s.tickets_b, acc_row + o_b1, acc_row + o_w2, acc_row + o_b2, cnt, d.d_hidden,
-                                               d.d_out);
+                                               d.d_out, store ? 1 : 0);
     mark(user, ABS_K_MLP_BWD, 1, stream);
     return cudaGetLastError();
 }
 
-cudaError_t launch_mlp_dw1(const MlpDims& d, const MlpScratch& s, float* acc_row, const void* acc_tmap, int nb, int variant,
-                           cudaStream_t stream, MlpMark mark, void* user) {
+cudaError_t launch_mlp_dw1(const MlpDims& d, const MlpScratch& s, float* acc_row, const void* acc_tmap, int nb, bool store,
+                           int variant, cudaStream_t stream, MlpMark mark, void* user) {
+    const int st = store ? 1 : 0;
     mark(user, ABS_K_MLP_DW1, 0, stream);
     const dim3 grid(d.d_hidden / kDwN, d.d_in / kTileM);
     const CUtensorMap* ta = reinterpret_cast<const CUtensorMap*>(&s.tmap_xt);
@@ -1144,15 +1160,15 @@ cudaError_t launch_mlp_dw1(const MlpDims& d, const MlpScratch& s, float* acc_row
     const CUtensorMap* tc = reinterpret_cast<const CUtensorMap*>(acc_tmap);
     if ((variant & 8) || nb > 1) {   // the K-batched form exists only for the register-prefetch kernel
         const size_t smem = dw_regs_buf_bytes(nb) + sizeof(DwRegCtl) + 1024;
-        k_dw1_regs<<<grid, 256, smem, stream>>>(*ta, *tb, acc_row, d.d_in, d.d_hidden, nb, s.status);
+        k_dw1_regs<<<grid, 256, smem, stream>>>(*ta, *tb, acc_row, d.d_in, d.d_hidden, nb, st, s.status);
     } else if (variant & 4) {
         const int n_tiles_n = d.d_hidden / kDwN, n_tiles = n_tiles_n * (d.d_in / kTileM);
         const int ctas = n_tiles < s.num_sms ? n_tiles : s.num_sms;
-        k_dw1_persistent<<<ctas, 192, sizeof(DwPersistSmem) + 1024, stream>>>(*ta, *tb, *tc, n_tiles_n, n_tiles, s.status);
+        k_dw1_persistent<<<ctas, 192, sizeof(DwPersistSmem) + 1024, stream>>>(*ta, *tb, *tc, n_tiles_n, n_tiles, st, s.status);
     } else if (variant & 1) {
-        k_dw1_tcgen05<true><<<grid, 128, sizeof(DwSmem) + 1024, stream>>>(*ta, *tb, *tc, s.status);
+        k_dw1_tcgen05<true><<<grid, 128, sizeof(DwSmem) + 1024, stream>>>(*ta, *tb, *tc, st, s.status);
     } else {
-        k_dw1_tcgen05<false><<<grid, 128, sizeof(DwSmem) + 1024, stream>>>(*ta, *tb, *tc, s.status);
+        k_dw1_tcgen05<false><<<grid, 128, sizeof(DwSmem) + 1024, stream>>>(*ta, *tb, *tc, st, s.status);
     }
     mark(user, ABS_K_MLP_DW1, 1, stream);
     return cudaGetLastError();

@@ -45,7 +45,7 @@ def test_runtime_argument_errors_and_use_after_destroy():
     assert B.lib.abs_destroy(raw) == B.ESTATE
 
 
-def test_workspace_too_small_and_overwrite_first_with_mlp_rejected():
+def test_workspace_too_small_and_inconsistent_mlp_shape_rejected():
     import torch
 
     from paper_2308_15164_b200 import binding as B
@@ -57,5 +57,5 @@ def test_workspace_too_small_and_overwrite_first_with_mlp_rejected():
     h = ctypes.c_void_p()
     assert B.lib.abs_init(ctypes.byref(h), ctypes.byref(cfg), ws.data_ptr(), need - 1, x0.data_ptr()) == B.ENOMEM
     assert not h.value
-    bad = B.make_config(P=128 * 128 + 128 + 1280 + 10, W=2, lr=0.1, flags=B.FLAG_MLP | B.FLAG_OVERWRITE_FIRST, mlp=(128, 128, 10, 64))
-    assert B.abs_workspace_bytes(bad) == 0
+    bad = B.make_config(P=128 * 128 + 128 + 1280 + 10 + 1, W=2, lr=0.1, flags=B.FLAG_MLP, mlp=(128, 128, 10, 64))
+    assert B.abs_workspace_bytes(bad) == 0                     # P does not match the MLP shape

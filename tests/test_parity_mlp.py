@@ -24,14 +24,14 @@ TOL = 2e-3
 TAU = 1e-4
 
 
-def _engine(wl, x0, pipelined=False, epilogue=0):
+def _engine(wl, x0, pipelined=False, epilogue=0, overwrite_first=False):
     import torch
 
     from paper_2308_15164_b200 import binding as B
 
     d = wl.mlp
     eng = B.AbsSgd(torch.from_numpy(x0).cuda(), wl.W, wl.lr, wl.momentum, wl.weight_decay,
-                   pipelined=pipelined, mlp=(d.d_in, d.d_hidden, d.d_out, d.mb))
+                   pipelined=pipelined, mlp=(d.d_in, d.d_hidden, d.d_out, d.mb), overwrite_first=overwrite_first)
     eng.set_launch(B.K_MLP_DW1, epilogue)
     return eng
 
@@ -101,6 +101,16 @@ def test_single_microbatch_gradient(small, epilogue):
         _check_gradient(got, x0, xs[b], ys[b], dims)
     cnt, cur, t = eng.counters()
     assert cnt[0].tolist() == [1, 1, 0, 0] and cur == 0 and t == 0
+    # A worker's first gradient of an iteration is stored, later ones are added: the second call on worker 0
+    # takes the read-modify-write path; what it added must be the gradient of its micro-batch.
+    before = eng.accumulator(0, 0).cpu().numpy().astype(np.float64)
+    xd, yd = torch.from_numpy(xs[3]).cuda(), torch.from_numpy(ys[3]).cuda()
+    torch.cuda.synchronize()
+    eng.accumulate_mlp(0, xd, yd)
+    eng.check()
+    after = eng.accumulator(0, 0).cpu().numpy().astype(np.float64)
+    _check_gradient(after - before, x0, xs[3], ys[3], dims)
+    assert eng.counters()[0][0].tolist() == [2, 1, 0, 0]
     eng.destroy()
 
 
@@ -129,13 +139,13 @@ def test_two_microbatches_add_up():
     eng.destroy()
 
 
-def _run_training(wl, pipelined, x0, xs, ys, eng=None):
+def _run_training(wl, pipelined, x0, xs, ys, eng=None, overwrite_first=False):
     import torch
 
     d = wl.mlp
     own = eng is None
     if own:
-        eng = _engine(wl, x0, pipelined=pipelined)
+        eng = _engine(wl, x0, pipelined=pipelined, overwrite_first=overwrite_first)
     xs_d, ys_d = torch.from_numpy(xs).cuda(), torch.from_numpy(ys).cuda()
     torch.cuda.synchronize()
     states = []
@@ -183,6 +193,11 @@ def test_training_run_matches_oracle(small, T):
             assert np.array_equal(a, b)
         outs.append(got)
     assert np.array_equal(outs[0], outs[1]), "eager and pipelined runs must be bit-identical"
+    # byte-saving mode (accumulator rows are not cleared; every worker's first gradient overwrites its row)
+    got, states, consumed = _run_training(wl, True, x0, xs, ys, overwrite_first=True)
+    assert np.array_equal(got, outs[0]), "overwrite-first mode must give the same parameters"
+    for a, b in zip(consumed, ref_consumed):
+        assert np.array_equal(a, b)
 
 
 @pytest.mark.parametrize("n", [2, 4])
