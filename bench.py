@@ -367,10 +367,19 @@ def run_mlp(B, wlm, dev, peaks, iters=12):
         out[name] = res
 
     # K-batched variant: up to 4 consecutive reference batches of a worker per call, one K = 64 n dW1 GEMM
+    for bname, bvariant in (("k_batched_up_to_4", 0), ("k_batched_up_to_4_ring", 4)):
+        out[bname] = run_mlp_batched(B, wlm, wl, d, x0_d, xp, yp, flop, rmw_bytes, peaks, bvariant)
+    return out
+
+
+def run_mlp_batched(B, wlm, wl, d, x0_d, xp, yp, flop, rmw_bytes, peaks, variant):
+    import torch
+
     res = {}
     for serial in (0, 1):
         eng = B.AbsSgd(x0_d, wl.W, wl.lr, wl.momentum, wl.weight_decay, pipelined=True, mlp=(d.d_in, d.d_hidden, d.d_out, d.mb))
         eng.set_launch(B.K_MLP_FWD, serial)
+        eng.set_launch(B.K_MLP_DW1, variant)
         sched = wlm.schedule(wl)
 
         def run_b(profile):
@@ -411,8 +420,7 @@ def run_mlp(B, wlm, dev, peaks, iters=12):
                         "dw1_hbm_gbs": rmw_bytes / us_dw / 1e3, "dw1_frac_of_hbm": rmw_bytes / us_dw / 1e3 / peaks["hbm_gbs"]})
         eng.check()
         eng.destroy()
-    out["k_batched_up_to_4"] = res
-    return out
+    return res
 
 
 def run_e2e(B, wlm, wl, x0_d, pool, order, step_bytes, steps):

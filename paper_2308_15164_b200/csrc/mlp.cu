@@ -24,7 +24,8 @@
 //                   dH, dZ, bf16(dZ)^T, db1 += ..., dW2 += ..., b_i += 1
 //   k_dw1_tcgen05   dW1 tile = A B^T on the 5th-gen tensor cores (TMEM accumulator); epilogue adds the
 //                   tile into the worker's accumulator slice via TMA load / TMA store (or TMA reduce-add)
-//   (k_dw1_persistent  the same as a persistent, warp-specialised kernel with a shared-memory ring)
+//   (k_dw1_ring     persistent, warp-specialised, K-batched: operand ring in shared memory, two TMEM
+//                   accumulators, TMA store / reduce-add of the finished tiles)
 #include <cuda.h>
 
 #include <cstdio>
@@ -689,23 +690,26 @@ __global__ void __launch_bounds__(256) k_dw1_regs(const __grid_constant__ CUtens
 }
 
 // ============================================================================================
-// dW1, persistent warp-specialised version.  One CTA per SM walks over its share of the
-// 128 x 64 output tiles (hidden index fastest, so neighbouring CTAs share the X^T tile in L2).
-// A kDwStages-deep shared-memory ring holds {A, B, accumulator tile} per tile, so that the
-// loads of the next tiles are always in flight while the current one is added and stored:
-//   warp 0 (one lane)   TMA producer: waits for a free ring slot, loads A, B and the fp32 tile
-//   warp 1 (one lane)   MMA issuer: 4 x tcgen05.mma into one of two TMEM accumulators
-//   warps 2..5          epilogue: tcgen05.ld, add into the swizzled fp32 tile in shared memory,
-//                       TMA store; a ring slot is released once its store has read it
-// The kernel is bound by the read-modify-write of the accumulator (8 bytes per output element).
+// dW1, persistent warp-specialised version, K-batched.  One CTA per SM walks over its share of
+// the 128 x 64 output tiles (hidden index fastest, so neighbouring CTAs share the X^T tile in L2):
+//   warp 0 (one lane)   TMA producer: one ring slot = the operands {A, B} of one micro-batch of one
+//                       tile; the slots of the next tiles fill while the current one is computed
+//   warp 1 (one lane)   MMA issuer: 4 nb x tcgen05.mma per tile into one of two TMEM accumulators;
+//                       each slot is handed back by a tcgen05.commit on its `empty` barrier
+//   warps 2..5          epilogue: tcgen05.ld -> registers (the accumulator is free again), write the
+//                       tile into one of kRingC swizzled staging tiles, then ONE thread issues the TMA
+//                       store (store mode) or TMA reduce-add (fp32 add done by the memory system)
+// The accumulator slice never passes through the SM on its way in: no CTA ever waits for DRAM, the
+// only loads are the (L2-resident) bf16 operands.
 // ============================================================================================
-constexpr int kDwStages = 4;
-constexpr int kDwStageBytes = kTileM * 128 + kDwN * 128 + kTileM * kDwN * 4;   // 16 KB + 8 KB + 32 KB
+constexpr int kRingOps = 6;                       // operand slots of 24 KB
+constexpr int kRingC = 2;                         // outgoing staging tiles of 32 KB
 
-struct DwPersistSmem {
-    alignas(1024) uint8_t stage[kDwStages][kDwStageBytes];   // [A | B | C panel 0 | C panel 1]
-    alignas(8) uint64_t full[kDwStages];
-    uint64_t empty[kDwStages];
+struct DwRingSmem {
+    alignas(1024) uint8_t op[kRingOps][kDwOperandBytes];   // [A 128 x 64 | B 64 x 64] bf16, swizzled rows
+    alignas(1024) float c[kRingC][kTileM * kDwN];          // two [128][32] fp32 column panels, swizzled rows
+    alignas(8) uint64_t op_full[kRingOps];
+    uint64_t op_empty[kRingOps];
     uint64_t acc_full[2];
     uint64_t acc_empty[2];
     uint32_t tmem_base;
@@ -713,14 +717,13 @@ struct DwPersistSmem {
     uint32_t stop[2];
 };
 
-__global__ void __launch_bounds__(192) k_dw1_persistent(const __grid_constant__ CUtensorMap tm_xt,
-                                                        const __grid_constant__ CUtensorMap tm_dzt,
-                                                        const __grid_constant__ CUtensorMap tm_acc, int n_tiles_n,
-                                                        int n_tiles, int store, int* status) {
+__global__ void __launch_bounds__(192) k_dw1_ring(const __grid_constant__ CUtensorMap tm_xt,
+                                                  const __grid_constant__ CUtensorMap tm_dzt,
+                                                  const __grid_constant__ CUtensorMap tm_acc, int n_tiles_n, int n_tiles,
+                                                  int d_in, int ld, int nb, int store, int* status) {
     extern __shared__ uint8_t smem_raw[];
-    DwPersistSmem& s = *reinterpret_cast<DwPersistSmem*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+    DwRingSmem& s = *reinterpret_cast<DwRingSmem*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
     const int warp = threadIdx.x / 32, lane = threadIdx.x % 32;
-    constexpr int kOffB = kTileM * 128, kOffC = kOffB + kDwN * 128;
     const int my_tiles = (n_tiles - (int)blockIdx.x + (int)gridDim.x - 1) / (int)gridDim.x;
 
     if (warp == 1) {
@@ -728,9 +731,9 @@ __global__ void __launch_bounds__(192) k_dw1_persistent(const __grid_constant__ 
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
     }
     if (threadIdx.x == 0) {
-        for (int i = 0; i < kDwStages; ++i) {
-            mbar_init(&s.full[i], 1);
-            mbar_init(&s.empty[i], 1);
+        for (int i = 0; i < kRingOps; ++i) {
+            mbar_init(&s.op_full[i], 1);
+            mbar_init(&s.op_empty[i], 1);
         }
         for (int i = 0; i < 2; ++i) {
             mbar_init(&s.acc_full[i], 1);
@@ -747,77 +750,81 @@ __global__ void __launch_bounds__(192) k_dw1_persistent(const __grid_constant__ 
 
     if (warp == 0) {
         if (lane == 0) {                             // ---- TMA producer
-            for (int i = 0; i < my_tiles; ++i) {
-                const int st = i % kDwStages;
-                if (i >= kDwStages && !mbar_wait(&s.empty[st], ((i / kDwStages) - 1) & 1)) { s.failed = 1; break; }
+            int q = 0;                               // running slot count
+            for (int i = 0; i < my_tiles && !s.failed; ++i) {
                 const int t = (int)blockIdx.x + i * (int)gridDim.x;
                 const int n0 = (t % n_tiles_n) * kDwN, m0 = (t / n_tiles_n) * kTileM;
-                uint8_t* base = s.stage[st];
-                mbar_expect_tx(&s.full[st], store ? kOffC : kDwStageBytes);   // store: see k_dw1_tcgen05
-                tma_load_2d(base, &tm_xt, 0, m0, &s.full[st]);
-                tma_load_2d(base + kOffB, &tm_dzt, 0, n0, &s.full[st]);
-                if (!store) {
-#pragma unroll
-                    for (int p = 0; p < kPanels; ++p)
-                        tma_load_2d(base + kOffC + p * (kTileM * 128), &tm_acc, n0 + p * 32, m0, &s.full[st]);
+                for (int j = 0; j < nb; ++j, ++q) {
+                    const int st = q % kRingOps;
+                    if (q >= kRingOps && !mbar_wait(&s.op_empty[st], ((q / kRingOps) - 1) & 1)) { s.failed = 1; break; }
+                    mbar_expect_tx(&s.op_full[st], kDwOperandBytes);
+                    tma_load_2d(s.op[st], &tm_xt, 0, j * d_in + m0, &s.op_full[st]);
+                    tma_load_2d(s.op[st] + kTileM * 128, &tm_dzt, 0, j * ld + n0, &s.op_full[st]);
                 }
             }
         }
     } else if (warp == 1) {
         if (lane == 0) {                             // ---- MMA issuer
             constexpr uint32_t idesc = umma_idesc_bf16(kTileM, kDwN);
-            for (int i = 0; i < my_tiles; ++i) {
-                const int st = i % kDwStages, ab = i & 1;
-                if (!mbar_wait(&s.full[st], (i / kDwStages) & 1)) { s.failed = 1; break; }
-                if (i >= 2 && !mbar_wait(&s.acc_empty[ab], ((i / 2) - 1) & 1)) { s.failed = 1; break; }
-                asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-                const uint32_t a0 = smem_u32(s.stage[st]);
-                const uint64_t da = umma_desc_k_sw128(a0), db = umma_desc_k_sw128(a0 + kOffB);
+            int q = 0;
+            bool ok = true;
+            for (int i = 0; i < my_tiles && ok; ++i) {
+                const int ab = i & 1;
+                if (i >= 2 && !mbar_wait(&s.acc_empty[ab], ((i / 2) - 1) & 1)) { ok = false; break; }
+                for (int j = 0; j < nb; ++j, ++q) {
+                    const int st = q % kRingOps;
+                    if (!mbar_wait(&s.op_full[st], (q / kRingOps) & 1)) { ok = false; break; }
+                    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                    const uint32_t a0 = smem_u32(s.op[st]);
+                    const uint64_t da = umma_desc_k_sw128(a0), db = umma_desc_k_sw128(a0 + kTileM * 128);
 #pragma unroll
-                for (int k = 0; k < kMB / 16; ++k) umma_bf16(tmem + ab * kDwN, da + 2 * k, db + 2 * k, idesc, k > 0);
-                umma_commit(&s.acc_full[ab]);
+                    for (int k = 0; k < kMB / 16; ++k) umma_bf16(tmem + ab * kDwN, da + 2 * k, db + 2 * k, idesc, (j > 0 || k > 0));
+                    umma_commit(&s.op_empty[st]);    // the slot is free once these MMAs have read it
+                }
+                if (ok) umma_commit(&s.acc_full[ab]);
             }
+            if (!ok) s.failed = 1;
         }
     } else {                                         // ---- epilogue warps 2..5
-        const int q = warp % 4;                      // TMEM lane quarter this warp may access
-        const int row = q * 32 + lane;
+        const int qd = warp % 4;                     // TMEM lane quarter this warp may access
+        const int row = qd * 32 + lane;
         const bool leader = (threadIdx.x == 64);
         for (int i = 0; i < my_tiles; ++i) {
-            const int st = i % kDwStages, ab = i & 1;
-            bool ok = mbar_wait(&s.full[st], (i / kDwStages) & 1);
-            ok = mbar_wait(&s.acc_full[ab], (i / 2) & 1) && ok;
+            const int ab = i & 1, ci = i % kRingC;
+            bool ok = mbar_wait(&s.acc_full[ab], (i / 2) & 1);
             ok = __all_sync(0xffffffffu, ok);
             if (!ok) s.failed = 1;
-            float* cbase = reinterpret_cast<float*>(s.stage[st] + kOffC);
+            uint32_t v0[32], v1[32];
             if (ok) {
                 asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-#pragma unroll 1
-                for (int p = 0; p < kPanels; ++p) {
-                    uint32_t v[32];
-                    tmem_ld_32(tmem + ((uint32_t)(q * 32) << 16) + (uint32_t)(ab * kDwN + p * 32), v);
-                    if (store) panel_row_update<false>(cbase + p * (kTileM * 32), row, v);
-                    else panel_row_update<true>(cbase + p * (kTileM * 32), row, v);
-                }
+                tmem_ld_32(tmem + ((uint32_t)(qd * 32) << 16) + (uint32_t)(ab * kDwN), v0);
+                tmem_ld_32(tmem + ((uint32_t)(qd * 32) << 16) + (uint32_t)(ab * kDwN + 32), v1);
                 asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
-                mbar_arrive(&s.acc_empty[ab]);
-                asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+                mbar_arrive(&s.acc_empty[ab]);       // the accumulator is in registers: the next tile may use it
             }
-            // Every epilogue warp reaches this barrier in every iteration (also after a failed wait); the
-            // leader samples the failure flag before it and all four warps act on that one sample after it,
-            // so they leave the loop together.
-            if (leader) s.stop[i & 1] = *reinterpret_cast<volatile uint32_t*>(&s.failed);
+            // Every epilogue warp reaches both barriers of an iteration (also after a failed wait); the leader
+            // samples the failure flag before the first one and all four warps act on that one sample after
+            // it, so they leave the loop together.  Before it, the leader also makes sure that the TMA
+            // operation which last read staging tile ci has finished reading.
+            if (leader) {
+                asm volatile("cp.async.bulk.wait_group.read %0;" ::"n"(kRingC - 1) : "memory");
+                s.stop[i & 1] = *reinterpret_cast<volatile uint32_t*>(&s.failed);
+            }
             asm volatile("bar.sync 1, 128;" ::: "memory");
             if (*reinterpret_cast<volatile uint32_t*>(&s.stop[i & 1])) break;
+            panel_row_update<false>(s.c[ci], row, v0);
+            panel_row_update<false>(s.c[ci] + kTileM * 32, row, v1);
+            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // smem writes -> visible to the TMA engine
+            asm volatile("bar.sync 1, 128;" ::: "memory");
             if (leader) {
                 const int t = (int)blockIdx.x + i * (int)gridDim.x;
                 const int n0 = (t % n_tiles_n) * kDwN, m0 = (t / n_tiles_n) * kTileM;
 #pragma unroll
-                for (int p = 0; p < kPanels; ++p) tma_store_2d(&tm_acc, cbase + p * (kTileM * 32), n0 + p * 32, m0);
-                asm volatile("cp.async.bulk.commit_group;" ::: "memory");
-                if (i >= 1) {                        // the previous tile's store has read its slot: release it
-                    asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory");
-                    mbar_arrive(&s.empty[(i - 1) % kDwStages]);
+                for (int p = 0; p < kPanels; ++p) {
+                    if (store) tma_store_2d(&tm_acc, s.c[ci] + p * (kTileM * 32), n0 + p * 32, m0);
+                    else tma_reduce_add_2d(&tm_acc, s.c[ci] + p * (kTileM * 32), n0 + p * 32, m0);
                 }
+                asm volatile("cp.async.bulk.commit_group;" ::: "memory");
             }
         }
         if (leader) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
@@ -827,7 +834,7 @@ __global__ void __launch_bounds__(192) k_dw1_persistent(const __grid_constant__ 
     __syncthreads();
     if (threadIdx.x == 0 && s.failed) {
         atomicExch(status, ABS_ETIMEOUT);
-        for (int i = 0; i < kDwStages; ++i) mbar_wait(&s.full[i], 0);   // bounded chance for copies in flight to land
+        for (int i = 0; i < kRingOps; ++i) mbar_wait(&s.op_full[i], 0);   // bounded chance for copies in flight to land
     }
     __syncthreads();
     if (warp == 1) {
@@ -1081,7 +1088,7 @@ cudaError_t mlp_scratch_init(MlpScratch* s, const MlpDims& d, void* base, __nv_b
     cudaError_t e = cudaGetDevice(&dev);
     if (e == cudaSuccess) e = cudaDeviceGetAttribute(&s->num_sms, cudaDevAttrMultiProcessorCount, dev);
     if (e == cudaSuccess)
-        e = cudaFuncSetAttribute(k_dw1_persistent, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(DwPersistSmem) + 1024);
+        e = cudaFuncSetAttribute(k_dw1_ring, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(DwRingSmem) + 1024);
     if (e == cudaSuccess)
         e = cudaFuncSetAttribute(k_dw1_regs, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                  dw_regs_buf_bytes(kMaxBatch) + (int)sizeof(DwRegCtl) + 1024);
@@ -1158,13 +1165,14 @@ cudaError_t launch_mlp_dw1(const MlpDims& d, const MlpScratch& s, float* acc_row
     const CUtensorMap* ta = reinterpret_cast<const CUtensorMap*>(&s.tmap_xt);
     const CUtensorMap* tb = reinterpret_cast<const CUtensorMap*>(&s.tmap_dzt);
     const CUtensorMap* tc = reinterpret_cast<const CUtensorMap*>(acc_tmap);
-    if ((variant & 8) || nb > 1) {   // the K-batched form exists only for the register-prefetch kernel
-        const size_t smem = dw_regs_buf_bytes(nb) + sizeof(DwRegCtl) + 1024;
-        k_dw1_regs<<<grid, 256, smem, stream>>>(*ta, *tb, acc_row, d.d_in, d.d_hidden, nb, st, s.status);
-    } else if (variant & 4) {
+    if (variant & 4) {               // persistent ring kernel (any nb)
         const int n_tiles_n = d.d_hidden / kDwN, n_tiles = n_tiles_n * (d.d_in / kTileM);
         const int ctas = n_tiles < s.num_sms ? n_tiles : s.num_sms;
-        k_dw1_persistent<<<ctas, 192, sizeof(DwPersistSmem) + 1024, stream>>>(*ta, *tb, *tc, n_tiles_n, n_tiles, st, s.status);
+        k_dw1_ring<<<ctas, 192, sizeof(DwRingSmem) + 1024, stream>>>(*ta, *tb, *tc, n_tiles_n, n_tiles, d.d_in, d.d_hidden, nb,
+                                                                     st, s.status);
+    } else if ((variant & 8) || nb > 1) {   // one CTA per tile, accumulator tile prefetched into registers (any nb)
+        const size_t smem = dw_regs_buf_bytes(nb) + sizeof(DwRegCtl) + 1024;
+        k_dw1_regs<<<grid, 256, smem, stream>>>(*ta, *tb, acc_row, d.d_in, d.d_hidden, nb, st, s.status);
     } else if (variant & 1) {
         k_dw1_tcgen05<true><<<grid, 128, sizeof(DwSmem) + 1024, stream>>>(*ta, *tb, *tc, st, s.status);
     } else {

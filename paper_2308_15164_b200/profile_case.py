@@ -2,7 +2,7 @@
 
     python -m paper_2308_15164_b200.profile_case sync       [--P 11689512] [--W 4] [--iters 3]
     python -m paper_2308_15164_b200.profile_case accumulate [--P 11689512] [--W 4] [--iters 3] [--bf16]
-    python -m paper_2308_15164_b200.profile_case mlp        [--iters 2] [--batch 4]
+    python -m paper_2308_15164_b200.profile_case mlp        [--iters 2] [--batch 4] [--calls 2]
 
 Each case keeps its working set larger than the 126 MB L2 but to a few hundred MB, launches the
 kernel of interest a handful of times and exits, so that a multi-pass capture ends by itself.
@@ -28,6 +28,7 @@ def main(argv=None):
     ap.add_argument("--pipelined", action="store_true")
     ap.add_argument("--epilogue", type=int, default=0)
     ap.add_argument("--batch", type=int, default=1, help="mlp: reference batches per call (1..4)")
+    ap.add_argument("--calls", type=int, default=1, help="mlp: calls per worker and iteration (the first one stores)")
     args = ap.parse_args(argv)
 
     from . import binding as B
@@ -61,7 +62,7 @@ def main(argv=None):
         torch.cuda.synchronize()
         c = 0
         for _ in range(args.iters + 1):
-            for i in range(wl.W):
+            for i in [w for _ in range(args.calls) for w in range(wl.W)]:
                 if args.batch > 1:
                     lo = (c * args.batch) % 8 if 8 % args.batch == 0 else 0
                     eng.accumulate_mlp_batch(i, args.batch, xs_d[lo:lo + args.batch], ys_d[lo:lo + args.batch])

@@ -200,9 +200,10 @@ def test_training_run_matches_oracle(small, T):
         assert np.array_equal(a, b)
 
 
-@pytest.mark.parametrize("n", [2, 4])
+@pytest.mark.parametrize("epilogue", [0, 4], ids=["tile-per-cta", "persistent-ring"])
+@pytest.mark.parametrize("n", [2, 3, 4])
 @pytest.mark.parametrize("small", [True, False], ids=["384x512", "3072x4096"])
-def test_batched_microbatches_match_the_sum_of_gradients(small, n):
+def test_batched_microbatches_match_the_sum_of_gradients(small, n, epilogue):
     """abs_accumulate_mlp_batch: n reference batches of one worker contracted by one K = 64 n GEMM give the sum
     of the n micro-batch gradients (b_i += n)."""
     import torch
@@ -212,7 +213,7 @@ def test_batched_microbatches_match_the_sum_of_gradients(small, n):
     dims = (d.d_in, d.d_hidden, d.d_out)
     x0 = wlm.params0(wl)
     xs, ys = wlm.mlp_batches(wl)
-    eng = _engine(wl, x0)
+    eng = _engine(wl, x0, epilogue=epilogue)
     b0 = 8
     xd, yd = torch.from_numpy(xs[b0:b0 + n]).cuda().contiguous(), torch.from_numpy(ys[b0:b0 + n]).cuda().contiguous()
     torch.cuda.synchronize()
@@ -236,10 +237,16 @@ def test_batched_microbatches_match_the_sum_of_gradients(small, n):
         u = sorted(undecided)
         assert np.abs(gW1[:, u] - wW1[:, u]).max() <= 0.2 * np.abs(wW1).max()
     # and the same data through n single calls agrees to fp32 rounding of the sums
-    eng2 = _engine(wl, x0)
+    eng2 = _engine(wl, x0, epilogue=epilogue)
     for j in range(n):
         eng2.accumulate_mlp(3, xd[j], yd[j])
     eng2.check()
     single = eng2.accumulator(0, 3).cpu().numpy().astype(np.float64)
     assert np.abs(got - single).max() <= 1e-5 * np.abs(single).max()
+    # a second call on the same worker takes the adding path: the row doubles
+    eng.accumulate_mlp_batch(3, n, xd, yd)
+    eng.check()
+    twice = eng.accumulator(0, 3).cpu().numpy().astype(np.float64)
+    assert np.abs(twice - 2.0 * got).max() <= 1e-5 * np.abs(got).max()
+    assert eng.counters()[0][0].tolist() == [0, 0, 0, 2 * n]
     eng.destroy(); eng2.destroy()
