@@ -323,7 +323,7 @@ def run_mlp(B, wlm, dev, peaks, iters=12):
     rmw_bytes = 8.0 * d.d_in * d.d_hidden + 2.0 * d.mb * (d.d_in + d.d_hidden)
     out = {"workload": "cfg4 mlp 3072-4096-10, mb=64, W=4, b_i~U{1..8}, pipelined", "iterations": iters,
            "dw1_flop": flop, "dw1_algorithmic_bytes": rmw_bytes}
-    for name, variant in (("tma_load_add_store", 0), ("tma_reduce_add", 1), ("persistent", 4), ("register_prefetch", 8)):
+    for name, variant in (("auto", 0), ("tma_load_add_store", 16), ("tma_reduce_add", 1), ("persistent_ring", 4), ("register_prefetch", 8)):
         res = {}
         for serial in (0, 1):
             eng = B.AbsSgd(x0_d, wl.W, wl.lr, wl.momentum, wl.weight_decay, pipelined=True,
@@ -367,7 +367,7 @@ def run_mlp(B, wlm, dev, peaks, iters=12):
         out[name] = res
 
     # K-batched variant: up to 4 consecutive reference batches of a worker per call, one K = 64 n dW1 GEMM
-    for bname, bvariant in (("k_batched_up_to_4", 0), ("k_batched_up_to_4_ring", 4)):
+    for bname, bvariant in (("k_batched_up_to_4", 0), ("k_batched_up_to_4_ring", 4), ("k_batched_up_to_4_tile_per_cta", 8)):
         out[bname] = run_mlp_batched(B, wlm, wl, d, x0_d, xp, yp, flop, rmw_bytes, peaks, bvariant)
     return out
 

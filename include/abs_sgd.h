@@ -204,11 +204,14 @@ int abs_check(abs_ctx *ctx);
 /* Launch shape of a kernel class: CTAs per SM for the persistent grid (0 = default, -1 = one
  * tile per CTA) for ABS_K_ACCUMULATE and ABS_K_SYNC.  For the MLP classes the value selects
  * kernel variants instead (results agree within rounding):
- *   ABS_K_MLP_DW1  bit mask: 1 = dW1 epilogue by TMA reduce-add (default: TMA load + add + TMA store);
- *                  2 = forward GEMM on CUDA cores (default: tcgen05); 4 = persistent warp-specialised
- *                  dW1 kernel; 8 = dW1 with the accumulator tile prefetched into registers.
- *   ABS_K_MLP_FWD  1 = serial mode: the dW1 GEMM runs on stream_acc instead of overlapping the next
- *                  micro-batch on the internal stream (for per-kernel timing). */
+ *   ABS_K_MLP_DW1  bit mask.  dW1 kernel: 0 = chosen per call (the persistent ring kernel when the tile is
+ *                  stored or the call is K-batched, the register-prefetch kernel for single adds);
+ *                  1 = one tile per CTA, TMA reduce-add epilogue; 16 = one tile per CTA, TMA load + add +
+ *                  TMA store; 4 = persistent warp-specialised ring kernel (TMA store / reduce-add);
+ *                  8 = one tile per CTA, accumulator tile prefetched into registers.
+ *                  2 = forward GEMM on CUDA cores (default: tcgen05).
+ *   ABS_K_MLP_FWD  1 = serial mode: every kernel of a gradient call runs on stream_acc instead of the
+ *                  worker's internal stream (for per-kernel timing). */
 int abs_set_launch(abs_ctx *ctx, int kernel_class, int ctas_per_sm);
 
 /* Per-kernel timing with CUDA events on the launching stream.  abs_profile(ctx, 1) starts

@@ -82,9 +82,8 @@ cudaError_t mlp_make_acc_tmap(void* tmap_out, const MlpDims& d, float* acc_row);
 //   front: forward GEMM, loss, layer-2 backward (writes dzt of this scratch set; adds db2, db1, dW2 into
 //          acc_row; bumps cnt);   dw1: the dW1 GEMM, which reads xtb/dzt and adds into the W1 slice.
 // shadow: bf16 copy of the published parameters (same flat layout), shadow_idx: which of the two copies it is.
-// x_pub: the fp32 parameters.  variant: bit 0 = dW1 epilogue by TMA reduce-add (else TMA load + add + TMA
-// store); bit 1 = forward GEMM on CUDA cores (cross-check of the tcgen05 one); bit 2 = persistent dW1 kernel;
-// bit 3 = dW1 with the accumulator tile prefetched into registers by plain coalesced loads.
+// x_pub: the fp32 parameters.  variant: the ABS_K_MLP_DW1 bit mask of abs_set_launch (0 = dW1 kernel chosen per
+// call; 1, 4, 8, 16 force one; 2 = forward GEMM on CUDA cores, a cross-check of the tcgen05 one).
 // mark(user, kernel_class, 0, stream) is called before a kernel group, mark(user, kernel_class, n, stream) after
 // its n launches.
 typedef void (*MlpMark)(void* user, int kernel_class, int n, cudaStream_t stream);

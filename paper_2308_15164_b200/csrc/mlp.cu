@@ -1165,15 +1165,21 @@ cudaError_t launch_mlp_dw1(const MlpDims& d, const MlpScratch& s, float* acc_row
     const CUtensorMap* ta = reinterpret_cast<const CUtensorMap*>(&s.tmap_xt);
     const CUtensorMap* tb = reinterpret_cast<const CUtensorMap*>(&s.tmap_dzt);
     const CUtensorMap* tc = reinterpret_cast<const CUtensorMap*>(acc_tmap);
-    if (variant & 4) {               // persistent ring kernel (any nb)
+    // Which kernel: bits 4 (ring), 8 (register prefetch), 16 (TMA load + add + store), 1 (TMA reduce-add) force
+    // one; otherwise the measured best for the case: the persistent ring kernel when the tile is stored (it
+    // never reads the accumulator) and for K-batched adds, the register-prefetch kernel for single adds.
+    int kind = (variant & 4) ? 4 : (variant & 8) ? 8 : (variant & 16) ? 16 : (variant & 1) ? 1 : 0;
+    if (kind == 0) kind = (store || nb > 1) ? 4 : 8;
+    if ((kind == 16 || kind == 1) && nb > 1) kind = 8;   // the one-tile-per-CTA TMA kernels are not K-batched
+    if (kind == 4) {
         const int n_tiles_n = d.d_hidden / kDwN, n_tiles = n_tiles_n * (d.d_in / kTileM);
         const int ctas = n_tiles < s.num_sms ? n_tiles : s.num_sms;
         k_dw1_ring<<<ctas, 192, sizeof(DwRingSmem) + 1024, stream>>>(*ta, *tb, *tc, n_tiles_n, n_tiles, d.d_in, d.d_hidden, nb,
                                                                      st, s.status);
-    } else if ((variant & 8) || nb > 1) {   // one CTA per tile, accumulator tile prefetched into registers (any nb)
+    } else if (kind == 8) {
         const size_t smem = dw_regs_buf_bytes(nb) + sizeof(DwRegCtl) + 1024;
         k_dw1_regs<<<grid, 256, smem, stream>>>(*ta, *tb, acc_row, d.d_in, d.d_hidden, nb, st, s.status);
-    } else if (variant & 1) {
+    } else if (kind == 1) {
         k_dw1_tcgen05<true><<<grid, 128, sizeof(DwSmem) + 1024, stream>>>(*ta, *tb, *tc, st, s.status);
     } else {
         k_dw1_tcgen05<false><<<grid, 128, sizeof(DwSmem) + 1024, stream>>>(*ta, *tb, *tc, st, s.status);

@@ -75,8 +75,9 @@ def _check_gradient(got_flat, params, X, y, dims):
     return len(amb)
 
 
-@pytest.mark.parametrize("epilogue", [0, 1, 2, 4, 8],
-                         ids=["tma-load-add-store", "tma-reduce", "cuda-core-forward", "persistent-dw1", "register-prefetch-dw1"])
+@pytest.mark.parametrize("epilogue", [0, 16, 1, 2, 4, 8],
+                         ids=["auto", "tma-load-add-store", "tma-reduce", "cuda-core-forward", "persistent-ring-dw1",
+                              "register-prefetch-dw1"])
 @pytest.mark.parametrize("small", [True, False], ids=["384x512", "3072x4096"])
 def test_single_microbatch_gradient(small, epilogue):
     wl = wlm.config(4, small=small)
@@ -200,7 +201,7 @@ def test_training_run_matches_oracle(small, T):
         assert np.array_equal(a, b)
 
 
-@pytest.mark.parametrize("epilogue", [0, 4], ids=["tile-per-cta", "persistent-ring"])
+@pytest.mark.parametrize("epilogue", [0, 8, 4], ids=["auto", "tile-per-cta", "persistent-ring"])
 @pytest.mark.parametrize("n", [2, 3, 4])
 @pytest.mark.parametrize("small", [True, False], ids=["384x512", "3072x4096"])
 def test_batched_microbatches_match_the_sum_of_gradients(small, n, epilogue):
