@@ -254,12 +254,18 @@ def run_ours(args):
     w_act = int(sum(1 for b in b_row if b > 0))
     ow_bytes = (int(sum(b_row)) - w_act) * 12 * wl.P + w_act * 8 * wl.P + (4 * w_act + 16) * wl.P
 
+    # DRAM bytes (read + write) of ONE launch of each kernel at this workload's size, from an ncu capture of the
+    # current kernels (profiles/k_accumulate_resnet18_and_bf16.md, profiles/k_sync_w4_resnet18.md): a lone launch
+    # under the profiler, whose reads equal the algorithmic reads and whose writes partly stay in the 126 MB L2.
+    NCU_TRAFFIC = {"k_accumulate_f32": 93_521_408 + 2_586_112, "k_sync<4>": 280_564_224 + 217_552_896}
+
     def roof(alg_bytes, n, ms, name, note):
         ach = alg_bytes / (ms / n / 1e3) / 1e9 if n and ms > 0 else None
         return {"kernel": name, "bound": "hbm", "achieved": ach, "peak": peaks["hbm_gbs"], "unit": "GB/s",
                 "frac": (ach / peaks["hbm_gbs"]) if ach else None, "peak_source": "of " + peaks["source"],
                 "frac_of_nominal_8TBs": (ach / HBM_NOMINAL_GBS) if ach else None,
-                "avg_us": ms / n * 1e3 if n else None, "launches": n, "traffic": None, "how": note}
+                "avg_us": ms / n * 1e3 if n else None, "launches": n, "algorithmic_bytes": alg_bytes,
+                "traffic": NCU_TRAFFIC.get(name) if wl.P == 11_689_512 else None, "how": note}
 
     per_acc = 12 * wl.P
     roofline = roof(per_acc, n_acc, ms_acc, "k_accumulate_f32",
