@@ -251,3 +251,73 @@ def test_batched_microbatches_match_the_sum_of_gradients(small, n, epilogue):
     assert np.abs(twice - 2.0 * got).max() <= 1e-5 * np.abs(got).max()
     assert eng.counters()[0][0].tolist() == [0, 0, 0, 2 * n]
     eng.destroy(); eng2.destroy()
+
+
+# Hand-made schedule for the small network: idle workers (rows of zeros stay stale in overwrite-first mode), all
+# workers idle, batch calls of every size, and precomputed gradients (abs_accumulate) mixed into the same rows
+# before and after a device-computed one -- the first call of a worker in an iteration stores, whatever its kind.
+# Entry: (worker, kind, n) with kind "mlp" (n micro-batches in one call) or "vec" (one precomputed gradient).
+_MIXED = [
+    [(0, "mlp", 1), (2, "mlp", 3), (0, "mlp", 2), (3, "vec", 1), (3, "mlp", 1)],
+    [(1, "mlp", 4), (1, "vec", 1), (0, "mlp", 1)],
+    [],
+    [(3, "mlp", 2), (3, "mlp", 2), (2, "vec", 1), (2, "vec", 1), (2, "mlp", 1)],
+    [(0, "vec", 1)],
+    [(1, "mlp", 1), (2, "mlp", 4), (3, "mlp", 3), (0, "mlp", 2)],
+    [(2, "mlp", 1)],
+]
+
+
+@pytest.mark.parametrize("overwrite_first", [False, True], ids=["clear-in-sync", "overwrite-first"])
+@pytest.mark.parametrize("pipelined", [False, True], ids=["eager", "pipelined"])
+def test_mixed_calls_idle_workers_and_batches(pipelined, overwrite_first):
+    import torch
+
+    wl = wlm.config(4, small=True, T=len(_MIXED))
+    d = wl.mlp
+    dims = (d.d_in, d.d_hidden, d.d_out)
+    x0 = wlm.params0(wl)
+    xs, ys = wlm.mlp_batches(wl)
+    vec = np.random.default_rng(11).standard_normal((3, wl.P)).astype(np.float32) * 1e-3
+    # oracle
+    o = AbsSgdOracle(x0, wl.W, wl.lr, wl.momentum, wl.weight_decay)
+    ref_states, c = [], 0
+    for calls in _MIXED:
+        p = o.params()
+        for (i, kind, n) in calls:
+            for _ in range(n):
+                if kind == "mlp":
+                    g = mlp_loss_and_grad(p, xs[c % wl.mlp_pool], ys[c % wl.mlp_pool], *dims, mode="bf16")[1].astype(np.float32)
+                else:
+                    g = vec[c % 3]
+                o.accumulate(i, g)
+                c += 1
+        o.sync_step()
+        ref_states.append(o.counters())
+    ref = o.params()
+    assert np.abs(ref - x0).max() > 1e-5
+    # library
+    eng = _engine(wl, x0, pipelined=pipelined, overwrite_first=overwrite_first)
+    xs_d, ys_d = torch.from_numpy(xs).cuda(), torch.from_numpy(ys).cuda()
+    vec_d = [torch.from_numpy(vec[j]).cuda() for j in range(3)]   # one allocation each: 16-byte aligned
+    torch.cuda.synchronize()
+    c = 0
+    for t, calls in enumerate(_MIXED):
+        for (i, kind, n) in calls:
+            if kind == "mlp":
+                lo = c % wl.mlp_pool
+                assert lo + n <= wl.mlp_pool
+                eng.accumulate_mlp_batch(i, n, xs_d[lo:lo + n], ys_d[lo:lo + n])
+            else:
+                eng.accumulate(i, vec_d[c % 3])
+            c += n
+        eng.sync_step()
+        cnt, cur, tt = eng.counters()
+        assert np.array_equal(cnt, ref_states[t][0]) and (cur, tt) == ref_states[t][1:]
+    eng.check()
+    got = eng.params_host()
+    consumed = [eng.consumed(s) for s in range(len(_MIXED))]
+    eng.destroy()
+    assert np.abs(got.astype(np.float64) - ref).max() <= TOL * np.abs(ref).max()
+    for a, b in zip(consumed, o.consumed):
+        assert np.array_equal(a, b)
