@@ -466,9 +466,10 @@ int abs_sync_step(abs_ctx* c) {
     if (!live(c)) return ABS_ESTATE;
     const uint32_t W = c->cfg.W;
     const uint32_t d = c->cur ^ 1;   // the delayed set (filled during iteration t-1)
-    if (int rc = join_dw(c)) return rc;
     if (!c->pipelined) {
-        // Step 1 on the delayed set, in place, on stream_acc.
+        // Step 1 on the delayed set, in place, on stream_acc: the gradient kernels still running on the
+        // worker streams read the parameters it overwrites.
+        if (int rc = join_dw(c)) return rc;
         int64_t B = 0;
         for (uint32_t i = 0; i < W; ++i) B += c->h_cnt[(size_t)d * W + i];
         if (B > 0) {
@@ -497,6 +498,10 @@ int abs_sync_step(abs_ctx* c) {
         for (uint32_t i = 0; i < W; ++i) B += c->h_cnt[(size_t)c->cur * W + i];
         CK(cudaEventRecord(c->ev_acc_done, c->s_acc));
         CK(cudaStreamWaitEvent(c->s_sync, c->ev_acc_done, 0));
+        // Step 1 needs every gradient of iteration t; stream_acc does not: the workers go straight on with
+        // iteration t+1 (other accumulator set, other parameter buffer), each behind its own previous call only.
+        for (int k = 0; k < c->n_wstreams; ++k)
+            if (c->w_outstanding[k]) CK(cudaStreamWaitEvent(c->s_sync, c->ev_w_done[k], 0));
         if (B > 0) {
             const int out = c->pub ^ 1;
             int rc = launch_fused(c, c->cur, c->pub, out, c->t + 1, c->s_sync);
