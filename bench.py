@@ -373,17 +373,19 @@ def run_mlp(B, wlm, dev, peaks, iters=12):
         out[name] = res
 
     # K-batched variant: up to 4 consecutive reference batches of a worker per call, one K = 64 n dW1 GEMM
-    for bname, bvariant in (("k_batched_up_to_4", 0), ("k_batched_up_to_4_ring", 4), ("k_batched_up_to_4_tile_per_cta", 8)):
-        out[bname] = run_mlp_batched(B, wlm, wl, d, x0_d, xp, yp, flop, rmw_bytes, peaks, bvariant)
+    for bname, bvariant, ow in (("k_batched_up_to_4", 0, False), ("k_batched_up_to_4_ring", 4, False),
+                                ("k_batched_up_to_4_tile_per_cta", 8, False), ("k_batched_up_to_4_overwrite_first", 0, True)):
+        out[bname] = run_mlp_batched(B, wlm, wl, d, x0_d, xp, yp, flop, rmw_bytes, peaks, bvariant, ow)
     return out
 
 
-def run_mlp_batched(B, wlm, wl, d, x0_d, xp, yp, flop, rmw_bytes, peaks, variant):
+def run_mlp_batched(B, wlm, wl, d, x0_d, xp, yp, flop, rmw_bytes, peaks, variant, overwrite_first):
     import torch
 
     res = {}
     for serial in (0, 1):
-        eng = B.AbsSgd(x0_d, wl.W, wl.lr, wl.momentum, wl.weight_decay, pipelined=True, mlp=(d.d_in, d.d_hidden, d.d_out, d.mb))
+        eng = B.AbsSgd(x0_d, wl.W, wl.lr, wl.momentum, wl.weight_decay, pipelined=True, mlp=(d.d_in, d.d_hidden, d.d_out, d.mb),
+                       overwrite_first=overwrite_first)
         eng.set_launch(B.K_MLP_FWD, serial)
         eng.set_launch(B.K_MLP_DW1, variant)
         sched = wlm.schedule(wl)
@@ -420,6 +422,8 @@ def run_mlp_batched(B, wlm, wl, d, x0_d, xp, yp, flop, rmw_bytes, peaks, variant
             for nm, k in (("us_fwd_3_kernels_per_call", B.K_MLP_FWD), ("us_bwd_per_call", B.K_MLP_BWD)):
                 n_k, ms_k = eng.kernel_stats(k)
                 res[nm] = ms_k / max(n_k, 1) * 1e3
+            n_sy, ms_sy = eng.kernel_stats(B.K_SYNC)
+            res["us_sync"] = ms_sy / max(n_sy, 1) * 1e3
             res.update({"us_dw1_per_call": us_dw, "mean_microbatches_per_call": mean_n,
                         "dw1_tflops": flop * mean_n / us_dw / 1e6,
                         "dw1_frac_of_bf16_peak_sustained": flop * mean_n / us_dw / 1e6 / peaks["bf16_tflops_sustained"],
