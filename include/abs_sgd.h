@@ -119,6 +119,14 @@ int abs_init(abs_ctx **out, const abs_config *cfg, void *workspace_dev, size_t w
  * gradient of a micro-batch is the MEAN over its M_r samples.  Enqueued on stream_acc. */
 int abs_accumulate(abs_ctx *ctx, uint32_t worker, const void *grad_dev);
 
+/* Algorithm 1, Step 2 for n (1..8) reference batches of one worker whose gradients are all at hand:
+ * G_t^i += g_0, += g_1, ... (added one after the other in list order, so the result equals n calls of
+ * abs_accumulate bit for bit); b_i += n.  One pass over the accumulator row: (4 n + 8) bytes per parameter
+ * for fp32 gradients (2 n + 8 for bf16) instead of 12 n (10 n).  grads_dev: HOST array of n device
+ * pointers, each as for abs_accumulate; the array itself is read before the call returns.
+ * Enqueued on stream_acc. */
+int abs_accumulate_batch(abs_ctx *ctx, uint32_t worker, uint32_t n, const void *const *grads_dev);
+
 /* Same as abs_accumulate for a gradient in (preferably pinned) HOST memory: copies it to
  * the device through an internal double-buffered staging area, then accumulates.  Needs
  * ABS_FLAG_HOST_INPUT.  grad_host must stay valid until the copy has completed (the call

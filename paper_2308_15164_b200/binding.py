@@ -48,6 +48,7 @@ _sig = {
     "abs_workspace_bytes": (ctypes.c_size_t, [ctypes.POINTER(AbsConfig)]),
     "abs_init": (ctypes.c_int, [ctypes.POINTER(_vp), ctypes.POINTER(AbsConfig), _vp, ctypes.c_size_t, _vp]),
     "abs_accumulate": (ctypes.c_int, [_vp, _u32, _vp]),
+    "abs_accumulate_batch": (ctypes.c_int, [_vp, _u32, _u32, ctypes.POINTER(ctypes.c_void_p)]),
     "abs_accumulate_host": (ctypes.c_int, [_vp, _u32, _vp]),
     "abs_accumulate_mlp": (ctypes.c_int, [_vp, _u32, _vp, _vp]),
     "abs_accumulate_mlp_batch": (ctypes.c_int, [_vp, _u32, _u32, _vp, _vp]),
@@ -142,6 +143,11 @@ class AbsSgd:
 
     def accumulate(self, worker: int, grad):
         self._ck(lib.abs_accumulate(self._h, worker, _ptr(grad)))
+
+    def accumulate_batch(self, worker: int, grads):
+        """grads: sequence of 1..8 device tensors (or raw device addresses), added in this order."""
+        arr = (ctypes.c_void_p * len(grads))(*[_ptr(g) for g in grads])
+        self._ck(lib.abs_accumulate_batch(self._h, worker, len(grads), arr))
 
     def accumulate_host(self, worker: int, grad_host):
         self._ck(lib.abs_accumulate_host(self._h, worker, _ptr(grad_host)))

@@ -383,6 +383,29 @@ int abs_accumulate(abs_ctx* c, uint32_t worker, const void* grad_dev) {
     return ABS_OK;
 }
 
+int abs_accumulate_batch(abs_ctx* c, uint32_t worker, uint32_t n, const void* const* grads_dev) {
+    if (!live(c)) return ABS_ESTATE;
+    if (worker >= c->cfg.W) return invalid(c, "worker index out of range");
+    if (n == 0 || n > (uint32_t)kMaxAccBatch) return invalid(c, "n must be in 1..8");
+    if (!grads_dev) return invalid(c, "gradient pointer list is NULL");
+    GradList gl{};
+    for (uint32_t k = 0; k < n; ++k) {
+        if (!grads_dev[k] || (reinterpret_cast<uintptr_t>(grads_dev[k]) & 15))
+            return invalid(c, "every gradient pointer must be non-NULL and 16-byte aligned");
+        gl.p[k] = grads_dev[k];
+    }
+    if (int rc = join_dw(c)) return rc;
+    const bool first = (c->cfg.flags & ABS_FLAG_OVERWRITE_FIRST) && c->h_cnt[(size_t)c->cur * c->cfg.W + worker] == 0;
+    {
+        Timed tm(c, ABS_K_ACCUMULATE, c->s_acc);
+        CK(launch_accumulate_multi(c->acc(c->cur, worker), gl, (int)n, c->cfg.grad_dtype, c->cfg.P, c->cnt(c->cur, worker),
+                                   first, c->ctas_per_sm[ABS_K_ACCUMULATE], c->num_sms, c->s_acc));
+    }
+    c->launches += 1;
+    c->h_cnt[(size_t)c->cur * c->cfg.W + worker] += (int32_t)n;
+    return ABS_OK;
+}
+
 int abs_accumulate_host(abs_ctx* c, uint32_t worker, const void* grad_host) {
     if (!live(c)) return ABS_ESTATE;
     if (!(c->cfg.flags & ABS_FLAG_HOST_INPUT)) return invalid(c, "context was created without ABS_FLAG_HOST_INPUT");

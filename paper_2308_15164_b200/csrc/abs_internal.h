@@ -37,6 +37,13 @@ struct SyncArgs {
     __nv_bfloat16* shadow;    // optional bf16 copy of x_{t+1} [P_pad], or nullptr
     int zero_acc;             // 1: overwrite the consumed rows with zeros; 0: leave them (overwrite-first mode)
 };
+// n (1..kMaxAccBatch) gradients of one worker added in one pass over its accumulator row, in list order.
+constexpr int kMaxAccBatch = 8;
+struct GradList {
+    const void* p[kMaxAccBatch];
+};
+cudaError_t launch_accumulate_multi(float* acc_row, const GradList& gl, int n, uint32_t grad_dtype, size_t P, int32_t* cnt,
+                                    bool overwrite, int ctas_per_sm, int num_sms, cudaStream_t stream);
 cudaError_t launch_sync(const SyncArgs& a, int ctas_per_sm, int num_sms, cudaStream_t stream);
 
 // bf16 copy of an fp32 vector (n multiple of 4): used once at init for the MLP weight shadow.

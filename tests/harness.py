@@ -42,9 +42,11 @@ def oracle_run(wl, x0, pool, columns=None, lambda_dc=0.0, oracle_cls=None, lr_sc
 
 
 def gpu_run(wl, x0, pool, pipelined, columns=None, lambda_dc=0.0, every_iteration=True, lr_schedule=None,
-            host_input=False, overwrite_first=False):
+            host_input=False, overwrite_first=False, batch=0):
     """Run the CUDA path over the workload.  Returns the same dict as oracle_run (xs restricted to
-    `columns` when given).  With every_iteration=False only the final parameters are read back."""
+    `columns` when given).  With every_iteration=False only the final parameters are read back.
+    batch > 0 (pool workloads): each worker's gradients of an iteration go through abs_accumulate_batch in
+    chunks of up to `batch`, in the worker's own arrival order (rows of different workers are independent)."""
     import torch
 
     from paper_2308_15164_b200 import binding as B
@@ -71,6 +73,14 @@ def gpu_run(wl, x0, pool, pipelined, columns=None, lambda_dc=0.0, every_iteratio
     for t, calls in enumerate(wlm.iter_calls(wl)):
         if lr_schedule is not None and t + 1 < len(lr_schedule):
             eng.set_lr(float(lr_schedule[t + 1]))     # gamma_{t+1}: supplied one iteration ahead
+        if batch and wl.pool_size and not host_input:
+            per_worker = {}
+            for (i, k, c) in calls:
+                per_worker.setdefault(i, []).append(pool_d[c % wl.pool_size])
+            for i, gs in per_worker.items():
+                for lo in range(0, len(gs), batch):
+                    eng.accumulate_batch(i, gs[lo:lo + batch])
+            calls = []
         for (i, k, c) in calls:
             if wl.pool_size:
                 if host_input:

@@ -169,6 +169,61 @@ def test_overwrite_first_mode_gives_the_same_results(cfg, T, pipelined):
     H.assert_params_close(b["xs"][-1], ref["xs"][-1], what="overwrite-first x_T")
 
 
+@pytest.mark.parametrize("batch", [2, 3, 8])
+@pytest.mark.parametrize("overwrite_first", [False, True], ids=["clear-in-sync", "overwrite-first"])
+@pytest.mark.parametrize("cfg,T", [(2, 12), (3, 30), (5, 6)])
+def test_accumulate_batch_equals_single_calls(cfg, T, overwrite_first, batch):
+    """abs_accumulate_batch adds a worker's gradients one after the other in list order, in one pass over its
+    row: bit-identical parameters to single abs_accumulate calls (fp32 and bf16 gradients, ragged P, idle
+    workers), same counters, oracle parity."""
+    wl = wlm.config(cfg, small=True, T=T)
+    x0 = wlm.params0(wl); pool = wlm.grad_pool(wl)
+    a = H.gpu_run(wl, x0, pool, pipelined=True, overwrite_first=overwrite_first)
+    b = H.gpu_run(wl, x0, pool, pipelined=True, overwrite_first=overwrite_first, batch=batch)
+    assert b["launches"] < a["launches"]
+    for s, (xa, xb) in enumerate(zip(a["xs"], b["xs"])):
+        assert np.array_equal(xa, xb), f"x_{s + 1} differs with batched accumulation"
+    ref = H.oracle_run(wl, x0, pool)
+    H.assert_states_equal(b, ref)
+    H.assert_params_close(b["xs"][-1], ref["xs"][-1], what="batched accumulate x_T")
+
+
+@pytest.mark.parametrize("P", [5, 257, 4099])
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_accumulate_batch_ragged_and_argument_errors(P, dtype):
+    import torch
+
+    from paper_2308_15164_b200 import binding as B
+
+    rng = np.random.default_rng(P)
+    n = 5
+    g = rng.standard_normal((n, P)).astype(np.float32)
+    if dtype == "bf16":
+        bits = wlm.f32_to_bf16_bits(g)
+        g = (bits.astype(np.uint32) << 16).view(np.float32)
+        g_d = [torch.from_numpy(bits[k].view(np.int16)).cuda() for k in range(n)]
+    else:
+        g_d = [torch.from_numpy(g[k]).cuda() for k in range(n)]
+    eng = B.AbsSgd(torch.zeros(P, device="cuda"), 2, 0.1, grad_dtype=B.GRAD_BF16 if dtype == "bf16" else B.GRAD_F32)
+    eng.accumulate_batch(1, g_d[:2])
+    eng.accumulate_batch(1, g_d[2:])
+    want = np.zeros(P, dtype=np.float32)
+    for k in range(n):
+        want = want + g[k]                       # fp32 adds, same order
+    got = eng.accumulator(0, 1)[:P].cpu().numpy()
+    assert np.array_equal(got, want)
+    assert eng.counters()[0][0].tolist() == [0, n]
+    import ctypes
+    arr = (ctypes.c_void_p * 9)(*[g_d[0].data_ptr()] * 9)
+    assert B.lib.abs_accumulate_batch(eng._h, 0, 9, arr) == B.EINVAL           # more than 8
+    assert B.lib.abs_accumulate_batch(eng._h, 0, 0, arr) == B.EINVAL
+    assert B.lib.abs_accumulate_batch(eng._h, 2, 1, arr) == B.EINVAL           # worker out of range
+    arr[1] = None
+    assert B.lib.abs_accumulate_batch(eng._h, 0, 2, arr) == B.EINVAL           # NULL entry
+    assert eng.counters()[0][0].tolist() == [0, n]                              # nothing was enqueued
+    eng.destroy()
+
+
 def test_accumulator_matches_oracle_bitwise():
     """fp32 adds of the same operands in the same order: the accumulators agree bit for bit."""
     import torch
