@@ -203,7 +203,18 @@ def run_ours(args):
         call_idx[0] = c
         eng.sync_step()
 
-    def timed(eng, steps, warmup):
+    def one_step_batched(eng):
+        # every worker hands over its b_i gradients of the iteration in one call (one pass over its row)
+        c = call_idx[0]
+        per_worker = {}
+        for (i, k) in order:
+            per_worker.setdefault(i, []).append(rows[c % wl.pool_size]); c += 1
+        call_idx[0] = c
+        for i, gs in per_worker.items():
+            eng.accumulate_batch(i, gs)
+        eng.sync_step()
+
+    def timed(eng, steps, warmup, one_step=one_step):
         for _ in range(warmup):
             one_step(eng)
         eng.wait(); eng.synchronize()
@@ -254,6 +265,18 @@ def run_ours(args):
     w_act = int(sum(1 for b in b_row if b > 0))
     ow_bytes = (int(sum(b_row)) - w_act) * 12 * wl.P + w_act * 8 * wl.P + (4 * w_act + 16) * wl.P
 
+    # ---- pass 5: batched accumulation (abs_accumulate_batch): each row read and written once per iteration ----
+    batched = {}
+    for name, ow in (("default_mode", False), ("overwrite_first", True)):
+        eng = make(pipelined=True, overwrite_first=ow)
+        secs_b, launches_b = timed(eng, args.steps, args.warmup, one_step_batched)
+        eng.destroy()
+        acc_bytes = sum((4 * int(b) + (4 if ow else 8)) * wl.P for b in b_row if b > 0)
+        syn_bytes = ((4 if ow else 8) * w_act + 16) * wl.P
+        batched[name] = {"ms_per_step": secs_b / args.steps * 1e3, "bytes_per_step": acc_bytes + syn_bytes,
+                         "hbm_gbs_on_its_own_bytes": (acc_bytes + syn_bytes) * args.steps / secs_b / 1e9,
+                         "step_time_vs_default": secs_b / secs, "launches_per_step": launches_b / args.steps}
+
     # DRAM bytes (read + write) of ONE launch of each kernel at this workload's size, from an ncu capture of the
     # current kernels (profiles/k_accumulate_resnet18_and_bf16.md, profiles/k_sync_w4_resnet18.md): a lone launch
     # under the profiler, whose reads equal the algorithmic reads and whose writes partly stay in the 126 MB L2.
@@ -285,6 +308,9 @@ def run_ours(args):
                    "accumulators 374 MB", "parallelism": f"replicas x{world}", "bytes_per_step": step_bytes},
         "frac_of_measured_hbm": value / world / peaks["hbm_gbs"],
         "roofline": roofline, "roofline_sync": roofline_sync, "isolated": isolated,
+        "batched_accumulate_variant": dict(batched, what="abs_accumulate_batch: the b_i gradients of a worker in one "
+                                           "pass over its accumulator row, (4 b_i + 8) instead of 12 b_i bytes per "
+                                           "parameter; bit-identical results"),
         "gpu_launches": launches, "clocks": clocks,
         "overwrite_first_variant": {
             "what": "ABS_FLAG_OVERWRITE_FIRST: no zero writes in the fused step, a worker's first micro-batch stores "
