@@ -217,6 +217,7 @@ int abs_check(abs_ctx *ctx);
  *                  1 = one tile per CTA, TMA reduce-add epilogue; 16 = one tile per CTA, TMA load + add +
  *                  TMA store; 4 = persistent warp-specialised ring kernel (TMA store / reduce-add);
  *                  8 = one tile per CTA, accumulator tile prefetched into registers.
+ *                  32 = the ring kernel keeps 128 x 64 tiles for K-batched calls (default there: 128 x 128).
  *                  2 = forward GEMM on CUDA cores (default: tcgen05).
  *   ABS_K_MLP_FWD  1 = serial mode: every kernel of a gradient call runs on stream_acc instead of the
  *                  worker's internal stream (for per-kernel timing). */

@@ -702,14 +702,22 @@ __global__ void __launch_bounds__(256) k_dw1_regs(const __grid_constant__ CUtens
 // The accumulator slice never passes through the SM on its way in: no CTA ever waits for DRAM, the
 // only loads are the (L2-resident) bf16 operands.
 // ============================================================================================
-constexpr int kRingOps = 6;                       // operand slots of 24 KB
-constexpr int kRingC = 2;                         // outgoing staging tiles of 32 KB
+constexpr int kRingC = 2;                         // outgoing staging tiles of 32 KB (128 x 64 fp32)
 
+// kN = 64: 128 x 64 tiles (1536 of them at 3072 x 4096: even shares for 148 CTAs); kN = 128: 128 x 128 tiles, a
+// third less operand traffic per output element -- the choice for K-batched calls, which are bound by it.
+template <int kN>
+struct DwRingCfg {
+    static constexpr int kSlotBytes = kTileM * 128 + kN * 128;   // [A 128 x 64 | B kN x 64] bf16
+    static constexpr int kOps = kN == 64 ? 6 : 5;                 // operand slots
+};
+
+template <int kN>
 struct DwRingSmem {
-    alignas(1024) uint8_t op[kRingOps][kDwOperandBytes];   // [A 128 x 64 | B 64 x 64] bf16, swizzled rows
-    alignas(1024) float c[kRingC][kTileM * kDwN];          // two [128][32] fp32 column panels, swizzled rows
-    alignas(8) uint64_t op_full[kRingOps];
-    uint64_t op_empty[kRingOps];
+    alignas(1024) uint8_t op[DwRingCfg<kN>::kOps][DwRingCfg<kN>::kSlotBytes];   // swizzled 128-byte rows
+    alignas(1024) float c[kRingC][kTileM * kDwN];          // two [128][32] fp32 column panels each, swizzled rows
+    alignas(8) uint64_t op_full[DwRingCfg<kN>::kOps];
+    uint64_t op_empty[DwRingCfg<kN>::kOps];
     uint64_t acc_full[2];
     uint64_t acc_empty[2];
     uint32_t tmem_base;
@@ -717,17 +725,20 @@ struct DwRingSmem {
     uint32_t stop[2];
 };
 
+template <int kN>
 __global__ void __launch_bounds__(192) k_dw1_ring(const __grid_constant__ CUtensorMap tm_xt,
                                                   const __grid_constant__ CUtensorMap tm_dzt,
                                                   const __grid_constant__ CUtensorMap tm_acc, int n_tiles_n, int n_tiles,
                                                   int d_in, int ld, int nb, int store, int* status) {
+    constexpr int kRingOps = DwRingCfg<kN>::kOps, kSlotBytes = DwRingCfg<kN>::kSlotBytes;
+    constexpr int kHalves = kN / kDwN;               // the epilogue works on 64-column pieces of the tile
     extern __shared__ uint8_t smem_raw[];
-    DwRingSmem& s = *reinterpret_cast<DwRingSmem*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+    DwRingSmem<kN>& s = *reinterpret_cast<DwRingSmem<kN>*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
     const int warp = threadIdx.x / 32, lane = threadIdx.x % 32;
     const int my_tiles = (n_tiles - (int)blockIdx.x + (int)gridDim.x - 1) / (int)gridDim.x;
 
     if (warp == 1) {
-        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&s.tmem_base)), "r"(2 * kDwN) : "memory");
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&s.tmem_base)), "r"(2 * kN) : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
     }
     if (threadIdx.x == 0) {
@@ -753,19 +764,21 @@ __global__ void __launch_bounds__(192) k_dw1_ring(const __grid_constant__ CUtens
             int q = 0;                               // running slot count
             for (int i = 0; i < my_tiles && !s.failed; ++i) {
                 const int t = (int)blockIdx.x + i * (int)gridDim.x;
-                const int n0 = (t % n_tiles_n) * kDwN, m0 = (t / n_tiles_n) * kTileM;
+                const int n0 = (t % n_tiles_n) * kN, m0 = (t / n_tiles_n) * kTileM;
                 for (int j = 0; j < nb; ++j, ++q) {
                     const int st = q % kRingOps;
                     if (q >= kRingOps && !mbar_wait(&s.op_empty[st], ((q / kRingOps) - 1) & 1)) { s.failed = 1; break; }
-                    mbar_expect_tx(&s.op_full[st], kDwOperandBytes);
+                    mbar_expect_tx(&s.op_full[st], kSlotBytes);
                     tma_load_2d(s.op[st], &tm_xt, 0, j * d_in + m0, &s.op_full[st]);
-                    tma_load_2d(s.op[st] + kTileM * 128, &tm_dzt, 0, j * ld + n0, &s.op_full[st]);
+#pragma unroll
+                    for (int b = 0; b < kHalves; ++b)   // 64-row boxes, 8 KB apart: one K-major B operand of kN rows
+                        tma_load_2d(s.op[st] + kTileM * 128 + b * (kDwN * 128), &tm_dzt, 0, j * ld + n0 + b * kDwN, &s.op_full[st]);
                 }
             }
         }
     } else if (warp == 1) {
         if (lane == 0) {                             // ---- MMA issuer
-            constexpr uint32_t idesc = umma_idesc_bf16(kTileM, kDwN);
+            constexpr uint32_t idesc = umma_idesc_bf16(kTileM, kN);
             int q = 0;
             bool ok = true;
             for (int i = 0; i < my_tiles && ok; ++i) {
@@ -778,7 +791,7 @@ __global__ void __launch_bounds__(192) k_dw1_ring(const __grid_constant__ CUtens
                     const uint32_t a0 = smem_u32(s.op[st]);
                     const uint64_t da = umma_desc_k_sw128(a0), db = umma_desc_k_sw128(a0 + kTileM * 128);
 #pragma unroll
-                    for (int k = 0; k < kMB / 16; ++k) umma_bf16(tmem + ab * kDwN, da + 2 * k, db + 2 * k, idesc, (j > 0 || k > 0));
+                    for (int k = 0; k < kMB / 16; ++k) umma_bf16(tmem + ab * kN, da + 2 * k, db + 2 * k, idesc, (j > 0 || k > 0));
                     umma_commit(&s.op_empty[st]);    // the slot is free once these MMAs have read it
                 }
                 if (ok) umma_commit(&s.acc_full[ab]);
@@ -789,42 +802,49 @@ __global__ void __launch_bounds__(192) k_dw1_ring(const __grid_constant__ CUtens
         const int qd = warp % 4;                     // TMEM lane quarter this warp may access
         const int row = qd * 32 + lane;
         const bool leader = (threadIdx.x == 64);
-        for (int i = 0; i < my_tiles; ++i) {
-            const int ab = i & 1, ci = i % kRingC;
+        bool stopped = false;
+        for (int i = 0; i < my_tiles && !stopped; ++i) {
+            const int ab = i & 1;
             bool ok = mbar_wait(&s.acc_full[ab], (i / 2) & 1);
             ok = __all_sync(0xffffffffu, ok);
             if (!ok) s.failed = 1;
-            uint32_t v0[32], v1[32];
-            if (ok) {
-                asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-                tmem_ld_32(tmem + ((uint32_t)(qd * 32) << 16) + (uint32_t)(ab * kDwN), v0);
-                tmem_ld_32(tmem + ((uint32_t)(qd * 32) << 16) + (uint32_t)(ab * kDwN + 32), v1);
-                asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
-                mbar_arrive(&s.acc_empty[ab]);       // the accumulator is in registers: the next tile may use it
-            }
-            // Every epilogue warp reaches both barriers of an iteration (also after a failed wait); the leader
-            // samples the failure flag before the first one and all four warps act on that one sample after
-            // it, so they leave the loop together.  Before it, the leader also makes sure that the TMA
-            // operation which last read staging tile ci has finished reading.
-            if (leader) {
-                asm volatile("cp.async.bulk.wait_group.read %0;" ::"n"(kRingC - 1) : "memory");
-                s.stop[i & 1] = *reinterpret_cast<volatile uint32_t*>(&s.failed);
-            }
-            asm volatile("bar.sync 1, 128;" ::: "memory");
-            if (*reinterpret_cast<volatile uint32_t*>(&s.stop[i & 1])) break;
-            panel_row_update<false>(s.c[ci], row, v0);
-            panel_row_update<false>(s.c[ci] + kTileM * 32, row, v1);
-            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // smem writes -> visible to the TMA engine
-            asm volatile("bar.sync 1, 128;" ::: "memory");
-            if (leader) {
-                const int t = (int)blockIdx.x + i * (int)gridDim.x;
-                const int n0 = (t % n_tiles_n) * kDwN, m0 = (t / n_tiles_n) * kTileM;
-#pragma unroll
-                for (int p = 0; p < kPanels; ++p) {
-                    if (store) tma_store_2d(&tm_acc, s.c[ci] + p * (kTileM * 32), n0 + p * 32, m0);
-                    else tma_reduce_add_2d(&tm_acc, s.c[ci] + p * (kTileM * 32), n0 + p * 32, m0);
+            const int t = (int)blockIdx.x + i * (int)gridDim.x;
+            const int n0 = (t % n_tiles_n) * kN, m0 = (t / n_tiles_n) * kTileM;
+#pragma unroll 1
+            for (int hh = 0; hh < kHalves; ++hh) {
+                const int e = i * kHalves + hh, ci = e % kRingC;
+                uint32_t v0[32], v1[32];
+                if (ok) {
+                    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                    tmem_ld_32(tmem + ((uint32_t)(qd * 32) << 16) + (uint32_t)(ab * kN + hh * kDwN), v0);
+                    tmem_ld_32(tmem + ((uint32_t)(qd * 32) << 16) + (uint32_t)(ab * kN + hh * kDwN + 32), v1);
+                    if (hh == kHalves - 1) {         // the accumulator is in registers: the next tile may use it
+                        asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+                        mbar_arrive(&s.acc_empty[ab]);
+                    }
                 }
-                asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+                // Every epilogue warp reaches both barriers of a step (also after a failed wait); the leader
+                // samples the failure flag before the first one and all four warps act on that one sample after
+                // it, so they leave the loop together.  Before it, the leader also makes sure that the TMA
+                // operation which last read staging tile ci has finished reading.
+                if (leader) {
+                    asm volatile("cp.async.bulk.wait_group.read %0;" ::"n"(kRingC - 1) : "memory");
+                    s.stop[e & 1] = *reinterpret_cast<volatile uint32_t*>(&s.failed);
+                }
+                asm volatile("bar.sync 1, 128;" ::: "memory");
+                if (*reinterpret_cast<volatile uint32_t*>(&s.stop[e & 1])) { stopped = true; break; }
+                panel_row_update<false>(s.c[ci], row, v0);
+                panel_row_update<false>(s.c[ci] + kTileM * 32, row, v1);
+                asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // smem writes -> visible to the TMA engine
+                asm volatile("bar.sync 1, 128;" ::: "memory");
+                if (leader) {
+#pragma unroll
+                    for (int p = 0; p < kPanels; ++p) {
+                        if (store) tma_store_2d(&tm_acc, s.c[ci] + p * (kTileM * 32), n0 + hh * kDwN + p * 32, m0);
+                        else tma_reduce_add_2d(&tm_acc, s.c[ci] + p * (kTileM * 32), n0 + hh * kDwN + p * 32, m0);
+                    }
+                    asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+                }
             }
         }
         if (leader) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
@@ -838,7 +858,7 @@ __global__ void __launch_bounds__(192) k_dw1_ring(const __grid_constant__ CUtens
     }
     __syncthreads();
     if (warp == 1) {
-        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(2 * kDwN) : "memory");
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(2 * kN) : "memory");
     }
 }
 
@@ -1088,7 +1108,9 @@ cudaError_t mlp_scratch_init(MlpScratch* s, const MlpDims& d, void* base, __nv_b
     cudaError_t e = cudaGetDevice(&dev);
     if (e == cudaSuccess) e = cudaDeviceGetAttribute(&s->num_sms, cudaDevAttrMultiProcessorCount, dev);
     if (e == cudaSuccess)
-        e = cudaFuncSetAttribute(k_dw1_ring, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(DwRingSmem) + 1024);
+        e = cudaFuncSetAttribute(k_dw1_ring<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(DwRingSmem<64>) + 1024);
+    if (e == cudaSuccess)
+        e = cudaFuncSetAttribute(k_dw1_ring<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(DwRingSmem<128>) + 1024);
     if (e == cudaSuccess)
         e = cudaFuncSetAttribute(k_dw1_regs, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                  dw_regs_buf_bytes(kMaxBatch) + (int)sizeof(DwRegCtl) + 1024);
@@ -1172,10 +1194,17 @@ cudaError_t launch_mlp_dw1(const MlpDims& d, const MlpScratch& s, float* acc_row
     if (kind == 0) kind = (store || nb > 1) ? 4 : 8;
     if ((kind == 16 || kind == 1) && nb > 1) kind = 8;   // the one-tile-per-CTA TMA kernels are not K-batched
     if (kind == 4) {
-        const int n_tiles_n = d.d_hidden / kDwN, n_tiles = n_tiles_n * (d.d_in / kTileM);
-        const int ctas = n_tiles < s.num_sms ? n_tiles : s.num_sms;
-        k_dw1_ring<<<ctas, 192, sizeof(DwRingSmem) + 1024, stream>>>(*ta, *tb, *tc, n_tiles_n, n_tiles, d.d_in, d.d_hidden, nb,
-                                                                     st, s.status);
+        if (nb > 1 && !(variant & 32)) {   // K-batched: 128 x 128 tiles (bit 5 keeps 128 x 64)
+            const int n_tiles_n = d.d_hidden / 128, n_tiles = n_tiles_n * (d.d_in / kTileM);
+            const int ctas = n_tiles < s.num_sms ? n_tiles : s.num_sms;
+            k_dw1_ring<128><<<ctas, 192, sizeof(DwRingSmem<128>) + 1024, stream>>>(*ta, *tb, *tc, n_tiles_n, n_tiles, d.d_in,
+                                                                                   d.d_hidden, nb, st, s.status);
+        } else {
+            const int n_tiles_n = d.d_hidden / kDwN, n_tiles = n_tiles_n * (d.d_in / kTileM);
+            const int ctas = n_tiles < s.num_sms ? n_tiles : s.num_sms;
+            k_dw1_ring<64><<<ctas, 192, sizeof(DwRingSmem<64>) + 1024, stream>>>(*ta, *tb, *tc, n_tiles_n, n_tiles, d.d_in,
+                                                                                 d.d_hidden, nb, st, s.status);
+        }
     } else if (kind == 8) {
         const size_t smem = dw_regs_buf_bytes(nb) + sizeof(DwRegCtl) + 1024;
         k_dw1_regs<<<grid, 256, smem, stream>>>(*ta, *tb, acc_row, d.d_in, d.d_hidden, nb, st, s.status);

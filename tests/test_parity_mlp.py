@@ -201,7 +201,7 @@ def test_training_run_matches_oracle(small, T):
         assert np.array_equal(a, b)
 
 
-@pytest.mark.parametrize("epilogue", [0, 8, 4], ids=["auto", "tile-per-cta", "persistent-ring"])
+@pytest.mark.parametrize("epilogue", [0, 8, 4, 36], ids=["auto", "tile-per-cta", "persistent-ring-128x128", "persistent-ring-128x64"])
 @pytest.mark.parametrize("n", [2, 3, 4])
 @pytest.mark.parametrize("small", [True, False], ids=["384x512", "3072x4096"])
 def test_batched_microbatches_match_the_sum_of_gradients(small, n, epilogue):
