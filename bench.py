@@ -355,7 +355,7 @@ def run_mlp(B, wlm, dev, peaks, iters=12):
     rmw_bytes = 8.0 * d.d_in * d.d_hidden + 2.0 * d.mb * (d.d_in + d.d_hidden)
     out = {"workload": "cfg4 mlp 3072-4096-10, mb=64, W=4, b_i~U{1..8}, pipelined", "iterations": iters,
            "dw1_flop": flop, "dw1_algorithmic_bytes": rmw_bytes}
-    for name, variant in (("auto", 0), ("tma_load_add_store", 16), ("tma_reduce_add", 1), ("persistent_ring", 4), ("register_prefetch", 8)):
+    for name, variant in (("auto", 0), ("tma_load_add_store", 16), ("tma_reduce_add", 1), ("persistent_ring", 4), ("register_prefetch", 8), ("cluster_fused_forward", 64)):
         res = {}
         for serial in (0, 1):
             eng = B.AbsSgd(x0_d, wl.W, wl.lr, wl.momentum, wl.weight_decay, pipelined=True,
@@ -400,7 +400,7 @@ def run_mlp(B, wlm, dev, peaks, iters=12):
 
     # K-batched variant: up to 4 consecutive reference batches of a worker per call, one K = 64 n dW1 GEMM
     for bname, bvariant, ow in (("k_batched_up_to_4", 0, False), ("k_batched_up_to_4_ring", 4, False), ("k_batched_up_to_4_ring_128x64", 36, False),
-                                ("k_batched_up_to_4_tile_per_cta", 8, False), ("k_batched_up_to_4_overwrite_first", 0, True)):
+                                ("k_batched_up_to_4_tile_per_cta", 8, False), ("k_batched_up_to_4_overwrite_first", 0, True), ("k_batched_up_to_4_cluster_fused_forward", 64, False)):
         out[bname] = run_mlp_batched(B, wlm, wl, d, x0_d, xp, yp, flop, rmw_bytes, peaks, bvariant, ow)
     return out
 

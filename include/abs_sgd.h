@@ -218,7 +218,9 @@ int abs_check(abs_ctx *ctx);
  *                  TMA store; 4 = persistent warp-specialised ring kernel (TMA store / reduce-add);
  *                  8 = one tile per CTA, accumulator tile prefetched into registers.
  *                  32 = the ring kernel keeps 128 x 64 tiles for K-batched calls (default there: 128 x 128).
- *                  2 = forward GEMM on CUDA cores (default: tcgen05).
+ *                  2 = forward GEMM on CUDA cores; 64 = forward GEMM on tcgen05 and its epilogue as ONE
+ *                  kernel, split-K sums through a thread-block cluster's shared memory (default: two
+ *                  kernels; the results are bit-identical).
  *   ABS_K_MLP_FWD  1 = serial mode: every kernel of a gradient call runs on stream_acc instead of the
  *                  worker's internal stream (for per-kernel timing). */
 int abs_set_launch(abs_ctx *ctx, int kernel_class, int ctas_per_sm);

@@ -16,6 +16,8 @@
 // Kernels (five launches per call of 1..4 micro-batches; only the first reads the caller's buffers, the
 // others may run on another stream):
 //   k_cast_x        X fp32 -> bf16 in both orientations
+//   (k_fwd_fused    k_fwd1_tcgen05 + k_fwd2 in one kernel: the K splits of a hidden tile form a thread-block cluster
+//                   and are added up through distributed shared memory; same bits, selectable)
 //   k_fwd1_tcgen05  Z^T partials = W1^T X^T, split over d_in, on tcgen05 (W1 as an MN-major operand)
 //   (k_fwd1         the same on CUDA cores, kept as a cross-check selectable through abs_set_launch)
 //   k_fwd2          Z = sum of partials + b1, bf16(H), partial logits per 32 hidden units; the last CTA of
@@ -998,6 +1000,248 @@ __global__ void __launch_bounds__(128) k_fwd1_tcgen05(const __grid_constant__ CU
     }
 }
 
+// ============================================================================================
+// Forward, fused:  k_fwd1_tcgen05 + k_fwd2 in one kernel.  The CTAs that hold the K splits of one
+// 128-hidden tile form a thread-block cluster (1 x nsplit x 1).  Each runs the same TMA -> MMA
+// pipeline as k_fwd1_tcgen05, then parks its partial accumulator [128][64 NB] in its own shared
+// memory (the pipeline stages are free by then); after a cluster barrier, CTA rank q adds up rows
+// [q 128/nsplit, (q+1) 128/nsplit) of all nsplit partials through distributed shared memory, in
+// rank order (fixed summation order), and does k_fwd2's work for those hidden units: bias, ReLU,
+// bf16 H -> hbt, partial logits -> lpart, group ticket -> gpart.  The split-K partials never
+// leave the SMs (k_fwd1_tcgen05 writes and k_fwd2 re-reads 4 bytes x nsplit per element of Z).
+// ============================================================================================
+__device__ __forceinline__ float4 ld_dsmem_f4(uint32_t local_addr, uint32_t rank) {
+    uint32_t remote;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(remote) : "r"(local_addr), "r"(rank));
+    float4 v;
+    asm volatile("ld.shared::cluster.v4.f32 {%0,%1,%2,%3}, [%4];" : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "r"(remote));
+    return v;
+}
+__device__ __forceinline__ void cluster_sync_all() {
+    asm volatile("barrier.cluster.arrive.release.aligned;\n barrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+
+template <int NB>
+__global__ void __launch_bounds__(128) k_fwd_fused(const __grid_constant__ CUtensorMap tm_w1,
+                                                   const __grid_constant__ CUtensorMap tm_xb, const float* __restrict__ b1,
+                                                   const __nv_bfloat16* __restrict__ w2b, __nv_bfloat16* hbt, float* lpart,
+                                                   float* gpart, unsigned int* tickets, int d_in, int d_h, int d_out,
+                                                   int* status) {
+    constexpr int kFwdStages = FwdCfg<NB>::kStages, kFwdStageBytes = FwdCfg<NB>::kStageBytes;
+    constexpr int kTmemCols = FwdCfg<NB>::kTmemCols;
+    constexpr int kPitch = 64 * NB + 4;              // floats per row of the parked partial (conflict-free float4 rows)
+    static_assert(128 * kPitch * 4 <= kFwdStages * kFwdStageBytes, "the parked partial must fit into the stages");
+    extern __shared__ uint8_t smem_raw[];
+    FwdSmem<NB>& s = *reinterpret_cast<FwdSmem<NB>*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+    __shared__ float sh[kHB][kMB + 1];
+    __shared__ float sw2[kHB][kOutPad];
+    __shared__ unsigned int s_last[2 * kMaxBatch];
+    const int warp = threadIdx.x / 32, lane = threadIdx.x % 32;
+    const int h0 = blockIdx.x * 128;
+    const int nsplit = gridDim.y;                    // = cluster size
+    const int split = blockIdx.y;
+    const int k_per = d_in / nsplit;
+    const int kbeg = split * k_per;
+    const int nk = k_per / 64;                       // pipeline steps of 64 k
+    uint32_t rank;
+    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(rank));
+
+    if (warp == 0) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&s.tmem_base)), "r"(kTmemCols) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    if (threadIdx.x == 0) {
+        for (int i = 0; i < kFwdStages; ++i) {
+            mbar_init(&s.full[i], 1);
+            mbar_init(&s.empty[i], 1);
+        }
+        mbar_init(&s.done, 1);
+        s.failed = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    const uint32_t tmem = s.tmem_base;
+
+    if (warp == 0 && lane == 0) {                    // ---- TMA producer
+        for (int kb = 0; kb < nk; ++kb) {
+            const int st = kb % kFwdStages;
+            if (kb >= kFwdStages && !mbar_wait(&s.empty[st], ((kb / kFwdStages) - 1) & 1)) { s.failed = 1; break; }
+            mbar_expect_tx(&s.full[st], kFwdStageBytes);
+            const int k0 = kbeg + kb * 64;
+            tma_load_2d(s.stage[st], &tm_w1, h0, k0, &s.full[st]);
+            tma_load_2d(s.stage[st] + 8192, &tm_w1, h0 + 64, k0, &s.full[st]);
+#pragma unroll
+            for (int jb = 0; jb < NB; ++jb)
+                tma_load_2d(s.stage[st] + 16384 + jb * 8192, &tm_xb, k0, jb * kMB, &s.full[st]);
+        }
+    } else if (warp == 1 && lane == 0) {             // ---- MMA issuer
+        constexpr uint32_t idesc = umma_idesc_bf16(128, 64 * NB) | (1u << 15);   // A is MN-major
+        bool ok = true;
+        for (int kb = 0; kb < nk && ok; ++kb) {
+            const int st = kb % kFwdStages;
+            ok = mbar_wait(&s.full[st], (kb / kFwdStages) & 1);
+            if (!ok) break;
+            asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+            const uint32_t a0 = smem_u32(s.stage[st]);
+            const uint64_t db = umma_desc_k_sw128(a0 + 16384);
+#pragma unroll
+            for (int k = 0; k < 4; ++k)
+                umma_bf16(tmem, umma_desc_mn_sw128(a0 + k * 2048, 8192), db + 2 * k, idesc, (kb > 0 || k > 0));
+            umma_commit(&s.empty[st]);
+        }
+        if (ok) umma_commit(&s.done);
+        else s.failed = 1;
+    }
+    __syncwarp();
+
+    bool ok = mbar_wait(&s.done, 0);
+    ok = __all_sync(0xffffffffu, ok);
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    float* red = reinterpret_cast<float*>(s.stage[0]);   // every load has landed, every MMA has completed
+    if (ok) {
+        const int row = warp * 32 + lane;            // TMEM lane = hidden unit within the tile
+#pragma unroll 1
+        for (int p = 0; p < 2 * NB; ++p) {
+            uint32_t v[32];
+            tmem_ld_32(tmem + ((uint32_t)(warp * 32) << 16) + (uint32_t)(p * 32), v);
+#pragma unroll
+            for (int j = 0; j < 8; ++j)
+                *reinterpret_cast<float4*>(red + row * kPitch + p * 32 + 4 * j) =
+                    make_float4(__uint_as_float(v[4 * j]), __uint_as_float(v[4 * j + 1]), __uint_as_float(v[4 * j + 2]),
+                                __uint_as_float(v[4 * j + 3]));
+        }
+    } else if (threadIdx.x == 0) {
+        atomicExch(status, ABS_ETIMEOUT);
+        for (int i = 0; i < kFwdStages; ++i) mbar_wait(&s.full[i], 0);   // bounded chance for copies in flight to land
+    }
+    __syncwarp();
+    // From here on every CTA of the cluster takes the same path (also after a failed wait: its numbers are
+    // then meaningless and the status word says so), so that both cluster barriers and every ticket are met.
+    cluster_sync_all();
+    {
+        const int rows_per_rank = 128 / nsplit, n_chunk = rows_per_rank / kHB;   // 32 (64) rows = 1 (2) chunks of 32
+        const int n_cta2 = d_h / kHB, n_groups = (n_cta2 + kGroup - 1) / kGroup; // chunk = what one k_fwd2 CTA handles
+        const uint32_t red_addr = smem_u32(red);
+        for (int ch = 0; ch < n_chunk; ++ch) {
+            const int hl0 = (int)rank * rows_per_rank + ch * kHB;                 // first tile row of the chunk
+            const int cta2 = (h0 + hl0) / kHB;
+            for (int e = threadIdx.x; e < kHB * kOutPad; e += 128) {
+                const int hl = e / kOutPad, o = e % kOutPad;
+                sw2[hl][o] = o < d_out ? bf16_to_f(w2b[(size_t)(h0 + hl0 + hl) * d_out + o]) : 0.f;
+            }
+#pragma unroll 1
+            for (int jb = 0; jb < NB; ++jb) {
+                // Z = sum over the K splits (rank order) + b1 ; H = bf16(relu(Z)) -> hbt and sh.
+                // All 4 x nsplit remote loads of a thread are issued before the first add.
+                float4 part[4][kSplitK];
+#pragma unroll
+                for (int k = 0; k < 4; ++k) {
+                    const int hl = threadIdx.x / 16 + 8 * k, r4 = (threadIdx.x % 16) * 4;
+                    const uint32_t off = red_addr + (uint32_t)(((hl0 + hl) * kPitch + jb * kMB + r4) * 4);
+#pragma unroll
+                    for (int sp = 0; sp < kSplitK; ++sp)
+                        if (sp < nsplit) part[k][sp] = ld_dsmem_f4(off, (uint32_t)sp);
+                }
+#pragma unroll
+                for (int k = 0; k < 4; ++k) {
+                    const int hl = threadIdx.x / 16 + 8 * k, r4 = (threadIdx.x % 16) * 4;
+                    const int h = h0 + hl0 + hl;
+                    const float bias = b1[h];
+                    float4 z = make_float4(bias, bias, bias, bias);
+#pragma unroll
+                    for (int sp = 0; sp < kSplitK; ++sp)
+                        if (sp < nsplit) { z.x += part[k][sp].x; z.y += part[k][sp].y; z.z += part[k][sp].z; z.w += part[k][sp].w; }
+                    const __nv_bfloat16 q0 = __float2bfloat16_rn(z.x > 0.f ? z.x : 0.f), q1 = __float2bfloat16_rn(z.y > 0.f ? z.y : 0.f);
+                    const __nv_bfloat16 q2 = __float2bfloat16_rn(z.z > 0.f ? z.z : 0.f), q3 = __float2bfloat16_rn(z.w > 0.f ? z.w : 0.f);
+                    uint2 pk;
+                    pk.x = (uint32_t)__bfloat16_as_ushort(q0) | ((uint32_t)__bfloat16_as_ushort(q1) << 16);
+                    pk.y = (uint32_t)__bfloat16_as_ushort(q2) | ((uint32_t)__bfloat16_as_ushort(q3) << 16);
+                    *reinterpret_cast<uint2*>(hbt + ((size_t)jb * d_h + h) * kMB + r4) = pk;
+                    sh[hl][r4 + 0] = bf16_to_f(q0); sh[hl][r4 + 1] = bf16_to_f(q1);
+                    sh[hl][r4 + 2] = bf16_to_f(q2); sh[hl][r4 + 3] = bf16_to_f(q3);
+                }
+                __syncthreads();
+                {   // partial logits of these 32 hidden units: thread = (sample r, 8 of the 16 padded outputs)
+                    const int r = threadIdx.x / 2, og = threadIdx.x % 2;
+                    float a[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+#pragma unroll 8
+                    for (int hl = 0; hl < kHB; ++hl) {
+                        const float hv = sh[hl][r];
+#pragma unroll
+                        for (int j = 0; j < 8; ++j) a[j] = fmaf(hv, sw2[hl][8 * og + j], a[j]);
+                    }
+                    float4* dst = reinterpret_cast<float4*>(lpart + ((size_t)jb * n_cta2 + cta2) * (kMB * kOutPad)) + r * 4 + og * 2;
+                    dst[0] = make_float4(a[0], a[1], a[2], a[3]);
+                    dst[1] = make_float4(a[4], a[5], a[6], a[7]);
+                }
+                __syncthreads();                     // sh is rewritten by the next micro-batch
+            }
+            __syncthreads();                         // sw2 is rewritten by the next chunk
+        }
+        // ---- group tickets (one per chunk and micro-batch), as in k_fwd2
+        __threadfence();
+        __syncthreads();
+        const int n_units = n_chunk * NB;
+        if ((int)threadIdx.x < n_units) {
+            const int ch = threadIdx.x / NB, jb = threadIdx.x % NB;
+            const int cta2 = (h0 + (int)rank * rows_per_rank + ch * kHB) / kHB;
+            const int group = cta2 / kGroup, g_count = min(kGroup, n_cta2 - group * kGroup);
+            s_last[threadIdx.x] = (atomicAdd(&tickets[(size_t)jb * n_groups + group], 1u) == (unsigned)(g_count - 1));
+        }
+        __syncthreads();
+        for (int u = 0; u < n_units; ++u) {
+            if (!s_last[u]) continue;
+            __threadfence();
+            const int ch = u / NB, jb = u % NB;
+            const int cta2 = (h0 + (int)rank * rows_per_rank + ch * kHB) / kHB;
+            const int group = cta2 / kGroup, g_first = group * kGroup, g_count = min(kGroup, n_cta2 - g_first);
+            const float4* lp = reinterpret_cast<const float4*>(lpart + (size_t)jb * n_cta2 * (kMB * kOutPad));
+            float4* gp = reinterpret_cast<float4*>(gpart + ((size_t)jb * n_groups + group) * (kMB * kOutPad));
+            for (int i = threadIdx.x; i < kMB * kOutPad / 4; i += 128) {
+                float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+                for (int c = 0; c < g_count; ++c) {
+                    const float4 v = __ldcg(lp + (size_t)(g_first + c) * (kMB * kOutPad / 4) + i);
+                    acc.x += v.x; acc.y += v.y; acc.z += v.z; acc.w += v.w;
+                }
+                gp[i] = acc;
+            }
+            if (threadIdx.x == 0) tickets[(size_t)jb * n_groups + group] = 0u;   // ready for the next launch
+        }
+    }
+    cluster_sync_all();                              // nobody leaves while its shared memory may still be read
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    if (warp == 0) {
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(kTmemCols) : "memory");
+    }
+}
+
+template <int NB>
+cudaError_t fwd_fused_set_attr() {
+    return cudaFuncSetAttribute(k_fwd_fused<NB>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(FwdSmem<NB>) + 1024);
+}
+// Launch with the nsplit CTAs of a hidden tile as one thread-block cluster.
+template <int NB>
+cudaError_t fwd_fused_launch(int n_tiles, int nsplit, cudaStream_t stream, const CUtensorMap& tw, const CUtensorMap& tx,
+                             const float* b1, const __nv_bfloat16* w2b, __nv_bfloat16* hbt, float* lpart, float* gpart,
+                             unsigned int* tickets, int d_in, int d_h, int d_out, int* status) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(n_tiles, nsplit, 1);
+    cfg.blockDim = dim3(128, 1, 1);
+    cfg.dynamicSmemBytes = sizeof(FwdSmem<NB>) + 1024;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = 1;
+    attr[0].val.clusterDim.y = nsplit;
+    attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, k_fwd_fused<NB>, tw, tx, b1, w2b, hbt, lpart, gpart, tickets, d_in, d_h, d_out, status);
+}
+
 template <int NB>
 cudaError_t fwd1_set_attr() {
     return cudaFuncSetAttribute(k_fwd1_tcgen05<NB>, cudaFuncAttributeMaxDynamicSharedMemorySize,
@@ -1119,6 +1363,10 @@ cudaError_t mlp_scratch_init(MlpScratch* s, const MlpDims& d, void* base, __nv_b
         if (e == cudaSuccess) e = fwd1_set_attr<2>();
         if (e == cudaSuccess) e = fwd1_set_attr<3>();
         if (e == cudaSuccess) e = fwd1_set_attr<4>();
+        if (e == cudaSuccess) e = fwd_fused_set_attr<1>();
+        if (e == cudaSuccess) e = fwd_fused_set_attr<2>();
+        if (e == cudaSuccess) e = fwd_fused_set_attr<3>();
+        if (e == cudaSuccess) e = fwd_fused_set_attr<4>();
     if (e == cudaSuccess)
         e = cudaFuncSetAttribute(k_dw1_tcgen05<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(DwSmem) + 1024);
     if (e == cudaSuccess)
@@ -1149,25 +1397,40 @@ cudaError_t launch_mlp_front(const MlpDims& d, const MlpScratch& s, const float*
     cudaError_t e;
     const unsigned n_cta = d.d_hidden / kHB;
 
-    // every kernel carries the nb micro-batches of the call as an extra grid dimension
     // every K split must be a whole number of 64-wide pipeline steps (d_in is a multiple of 128)
     const int nsplit = (d.d_in % (64 * kSplitK) == 0) ? kSplitK : 2;
-    if (variant & 2) {
-        k_fwd1<<<dim3(d.d_hidden / 64, nsplit, nb), 256, 0, stream>>>(shadow, s.xb, s.zpart, d.d_in, d.d_hidden);
-    } else {
-        const CUtensorMap* tw = reinterpret_cast<const CUtensorMap*>(&s.tmap_w1[shadow_idx]);
-        const CUtensorMap* tx = reinterpret_cast<const CUtensorMap*>(&s.tmap_xb);
-        const dim3 grid(d.d_hidden / 128, nsplit);
-        switch (nb) {                                // the nb micro-batches are stacked along N of one GEMM
-            case 1: fwd1_launch<1>(grid, stream, *tw, *tx, s.zpart, d.d_in, d.d_hidden, s.status); break;
-            case 2: fwd1_launch<2>(grid, stream, *tw, *tx, s.zpart, d.d_in, d.d_hidden, s.status); break;
-            case 3: fwd1_launch<3>(grid, stream, *tw, *tx, s.zpart, d.d_in, d.d_hidden, s.status); break;
-            default: fwd1_launch<4>(grid, stream, *tw, *tx, s.zpart, d.d_in, d.d_hidden, s.status); break;
+    const CUtensorMap* tw = reinterpret_cast<const CUtensorMap*>(&s.tmap_w1[shadow_idx]);
+    const CUtensorMap* tx = reinterpret_cast<const CUtensorMap*>(&s.tmap_xb);
+    if ((variant & 64) && !(variant & 2)) {
+        // one kernel: forward GEMM, split-K sum through the cluster's shared memory, bias / ReLU / logits.  Same
+        // bits as the two-kernel path; measured slower when several workers' calls overlap (its 128 CTAs keep a
+        // whole SM's shared memory each while 128 threads do the epilogue work), so it is not the default.
+        const int n_tiles = d.d_hidden / 128;
+        const float* b1 = x_pub + o_b1;
+        const __nv_bfloat16* w2b = shadow + o_w2;
+        switch (nb) {
+            case 1: e = fwd_fused_launch<1>(n_tiles, nsplit, stream, *tw, *tx, b1, w2b, s.hbt, s.lpart, s.gpart, s.tickets, d.d_in, d.d_hidden, d.d_out, s.status); break;
+            case 2: e = fwd_fused_launch<2>(n_tiles, nsplit, stream, *tw, *tx, b1, w2b, s.hbt, s.lpart, s.gpart, s.tickets, d.d_in, d.d_hidden, d.d_out, s.status); break;
+            case 3: e = fwd_fused_launch<3>(n_tiles, nsplit, stream, *tw, *tx, b1, w2b, s.hbt, s.lpart, s.gpart, s.tickets, d.d_in, d.d_hidden, d.d_out, s.status); break;
+            default: e = fwd_fused_launch<4>(n_tiles, nsplit, stream, *tw, *tx, b1, w2b, s.hbt, s.lpart, s.gpart, s.tickets, d.d_in, d.d_hidden, d.d_out, s.status); break;
         }
+        if (e != cudaSuccess) return e;
+    } else {
+        if (variant & 2) {
+            k_fwd1<<<dim3(d.d_hidden / 64, nsplit, nb), 256, 0, stream>>>(shadow, s.xb, s.zpart, d.d_in, d.d_hidden);
+        } else {
+            const dim3 grid(d.d_hidden / 128, nsplit);
+            switch (nb) {                                // the nb micro-batches are stacked along N of one GEMM
+                case 1: fwd1_launch<1>(grid, stream, *tw, *tx, s.zpart, d.d_in, d.d_hidden, s.status); break;
+                case 2: fwd1_launch<2>(grid, stream, *tw, *tx, s.zpart, d.d_in, d.d_hidden, s.status); break;
+                case 3: fwd1_launch<3>(grid, stream, *tw, *tx, s.zpart, d.d_in, d.d_hidden, s.status); break;
+                default: fwd1_launch<4>(grid, stream, *tw, *tx, s.zpart, d.d_in, d.d_hidden, s.status); break;
+            }
+        }
+        k_fwd2<<<dim3(n_cta, nb), 256, 0, stream>>>(s.zpart, nsplit, x_pub + o_b1, shadow + o_w2, s.hbt, s.lpart, s.gpart,
+                                                    s.tickets, d.d_hidden, d.d_out);
     }
-    k_fwd2<<<dim3(n_cta, nb), 256, 0, stream>>>(s.zpart, nsplit, x_pub + o_b1, shadow + o_w2, s.hbt, s.lpart, s.gpart,
-                                                s.tickets, d.d_hidden, d.d_out);
-    mark(user, ABS_K_MLP_FWD, 3, stream);
+    mark(user, ABS_K_MLP_FWD, ((variant & 64) && !(variant & 2)) ? 2 : 3, stream);   // launches of the group, the cast included
     if ((e = cudaGetLastError()) != cudaSuccess) return e;
 
     mark(user, ABS_K_MLP_BWD, 0, stream);

@@ -75,9 +75,9 @@ def _check_gradient(got_flat, params, X, y, dims):
     return len(amb)
 
 
-@pytest.mark.parametrize("epilogue", [0, 16, 1, 2, 4, 8],
-                         ids=["auto", "tma-load-add-store", "tma-reduce", "cuda-core-forward", "persistent-ring-dw1",
-                              "register-prefetch-dw1"])
+@pytest.mark.parametrize("epilogue", [0, 16, 1, 2, 64, 4, 8],
+                         ids=["auto", "tma-load-add-store", "tma-reduce", "cuda-core-forward", "cluster-fused-forward",
+                              "persistent-ring-dw1", "register-prefetch-dw1"])
 @pytest.mark.parametrize("small", [True, False], ids=["384x512", "3072x4096"])
 def test_single_microbatch_gradient(small, epilogue):
     wl = wlm.config(4, small=small)
@@ -321,3 +321,30 @@ def test_mixed_calls_idle_workers_and_batches(pipelined, overwrite_first):
     assert np.abs(got.astype(np.float64) - ref).max() <= TOL * np.abs(ref).max()
     for a, b in zip(consumed, o.consumed):
         assert np.array_equal(a, b)
+
+
+@pytest.mark.parametrize("n", [1, 2, 3, 4])
+@pytest.mark.parametrize("small", [True, False], ids=["384x512", "3072x4096"])
+def test_cluster_fused_forward_is_bit_identical_to_the_two_kernel_forward(small, n):
+    """The cluster kernel adds the K-split partial sums in the same order as k_fwd2 does: same H, same logits,
+    hence the same accumulator bits."""
+    import torch
+
+    wl = wlm.config(4, small=small)
+    x0 = wlm.params0(wl)
+    rng = np.random.default_rng(3)
+    d = wl.mlp
+    o_w1, o_b1, o_w2, o_b2 = d.offsets
+    x0[o_b1:o_w2] = rng.standard_normal(d.d_hidden).astype(np.float32) * 0.1
+    xs, ys = wlm.mlp_batches(wl)
+    xd, yd = torch.from_numpy(xs[20:20 + n]).cuda().contiguous(), torch.from_numpy(ys[20:20 + n]).cuda().contiguous()
+    torch.cuda.synchronize()
+    outs = []
+    for variant in (0, 64):
+        eng = _engine(wl, x0, epilogue=variant)
+        eng.accumulate_mlp_batch(1, n, xd, yd)
+        eng.accumulate_mlp_batch(1, n, xd, yd)
+        eng.check()
+        outs.append(eng.accumulator(0, 1).cpu().numpy())
+        eng.destroy()
+    assert np.array_equal(outs[0], outs[1])
