@@ -341,8 +341,12 @@ int abs_init(abs_ctx** out, const abs_config* cfg, void* workspace_dev, size_t w
         }
         if ((e = cudaEventCreateWithFlags(&c->ev_fork, cudaEventDisableTiming)) != cudaSuccess) return bail(e, "cudaEventCreate");
         c->n_wstreams = (int)std::min<uint32_t>(cfg->W, kMlpStreams);
+        // Highest priority: the short, dependent gradient kernels get free CTA slots before the long HBM-bound
+        // fused step that runs beside them on stream_sync and would otherwise fill every slot with its own CTAs.
+        int prio_lo = 0, prio_hi = 0;
+        if ((e = cudaDeviceGetStreamPriorityRange(&prio_lo, &prio_hi)) != cudaSuccess) return bail(e, "cudaDeviceGetStreamPriorityRange");
         for (int k = 0; k < c->n_wstreams; ++k) {
-            if ((e = cudaStreamCreateWithFlags(&c->s_w[k], cudaStreamNonBlocking)) != cudaSuccess) return bail(e, "cudaStreamCreate");
+            if ((e = cudaStreamCreateWithPriority(&c->s_w[k], cudaStreamNonBlocking, prio_hi)) != cudaSuccess) return bail(e, "cudaStreamCreate");
             if ((e = cudaEventCreateWithFlags(&c->ev_w_done[k], cudaEventDisableTiming)) != cudaSuccess) return bail(e, "cudaEventCreate");
         }
         c->acc_tmaps.resize((size_t)2 * cfg->W);
