@@ -216,7 +216,8 @@ __global__ void __launch_bounds__(256) k_fwd2(const float* zpart, int nsplit, co
 // --------------------------------------------------------------------------------------------
 // k_bwd: per CTA 32 hidden units x 64 samples.
 //   prologue (every CTA, identical result): logits = sum over groups of gpart + b2 (fixed order);
-//            dL = (softmax - onehot)/mb; CTA 0 also adds db2 = sum_r dL
+//            dL = (softmax - onehot)/mb, 4 lanes per sample row (max and sum by shuffles); CTA 0 also adds
+//            db2 = sum_r dL
 //   phase 1 (thread = sample r, 8 hidden units): dH = sum_o bf16(dL)[r][o] W2b[h][o]; dZ = dH * [H > 0]
 //            (H > 0 exactly when Z > 0); dzt[h][r] = bf16(dZ)
 //   phase 2 (thread = hidden unit, 2 outputs): dW2[h][o] += sum_r bf16(H)[h][r] bf16(dL)[r][o],
@@ -227,7 +228,7 @@ __global__ void __launch_bounds__(256) k_bwd(const __nv_bfloat16* hbt, const flo
                                              const __nv_bfloat16* __restrict__ w2b, __nv_bfloat16* dzt, float* bpart,
                                              unsigned int* tickets_b, float* acc_b1, float* acc_w2, float* acc_b2,
                                              int32_t* cnt, int d_h, int d_out, int store) {
-    __shared__ float sdl[kMB][kOutPad + 1];     // bf16(dL) as float (first: the logits)
+    __shared__ float sdl[kMB][kOutPad + 1];     // bf16(dL) as float
     __shared__ float sdl32[kMB][kOutPad + 1];   // dL unrounded (CTA 0: db2)
     __shared__ float sw2[kHB][kOutPad];
     __shared__ float sh[kHB][kMB + 1];
@@ -239,46 +240,48 @@ __global__ void __launch_bounds__(256) k_bwd(const __nv_bfloat16* hbt, const flo
     dzt += (size_t)jb * d_h * kMB;
     gpart += (size_t)jb * n_groups * kMB * kOutPad;
     y += (size_t)jb * kMB;
+    const int r = threadIdx.x % kMB, g = threadIdx.x / kMB;
+    float hv[8];                                     // issued first: independent of the logit sums below
+#pragma unroll
+    for (int j = 0; j < 8; ++j) hv[j] = bf16_to_f(hbt[(size_t)(h_beg + g * 8 + j) * kMB + r]);
     {
         float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
         for (int c = 0; c < n_groups; ++c) {
             const float4 v = reinterpret_cast<const float4*>(gpart)[(size_t)c * (kMB * kOutPad / 4) + threadIdx.x];
             acc.x += v.x; acc.y += v.y; acc.z += v.z; acc.w += v.w;
         }
+        // softmax and dL on the registers that hold the sums: 4 adjacent lanes share a sample row
         const int rr = threadIdx.x / 4, og = threadIdx.x % 4;
-        sdl[rr][4 * og + 0] = acc.x; sdl[rr][4 * og + 1] = acc.y; sdl[rr][4 * og + 2] = acc.z; sdl[rr][4 * og + 3] = acc.w;
+        float l[4] = {acc.x, acc.y, acc.z, acc.w};
+        float mx = -INFINITY;
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            const int o = 4 * og + j;
+            l[j] = o < d_out ? l[j] + b2[o] : -INFINITY;
+            mx = fmaxf(mx, l[j]);
+        }
+        mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 1));
+        mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 2));
+        float den = 0.f;
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            l[j] = (4 * og + j) < d_out ? expf(l[j] - mx) : 0.f;
+            den += l[j];
+        }
+        den += __shfl_xor_sync(0xffffffffu, den, 1);
+        den += __shfl_xor_sync(0xffffffffu, den, 2);
+        const int yr = y[rr];
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            const int o = 4 * og + j;
+            const float gl = o < d_out ? (l[j] / den - (o == yr ? 1.f : 0.f)) * (1.0f / kMB) : 0.f;
+            sdl32[rr][o] = gl;
+            sdl[rr][o] = bf16_to_f(__float2bfloat16_rn(gl));
+        }
     }
     for (int e = threadIdx.x; e < kHB * kOutPad; e += 256) {
         const int hl = e / kOutPad, o = e % kOutPad;
         sw2[hl][o] = o < d_out ? bf16_to_f(w2b[(size_t)(h_beg + hl) * d_out + o]) : 0.f;
-    }
-    const int r = threadIdx.x % kMB, g = threadIdx.x / kMB;
-    float hv[8];
-#pragma unroll
-    for (int j = 0; j < 8; ++j) hv[j] = bf16_to_f(hbt[(size_t)(h_beg + g * 8 + j) * kMB + r]);
-    __syncthreads();
-    if (threadIdx.x < kMB) {
-        const int rr = threadIdx.x;
-        float l[kOutPad];
-        float mx = -INFINITY;
-#pragma unroll
-        for (int o = 0; o < kOutPad; ++o) {
-            l[o] = o < d_out ? sdl[rr][o] + b2[o] : -INFINITY;
-            mx = fmaxf(mx, l[o]);
-        }
-        float den = 0.f;
-#pragma unroll
-        for (int o = 0; o < kOutPad; ++o) {
-            l[o] = o < d_out ? expf(l[o] - mx) : 0.f;
-            den += l[o];
-        }
-        const int yr = y[rr];
-#pragma unroll
-        for (int o = 0; o < kOutPad; ++o) {
-            const float gl = o < d_out ? (l[o] / den - (o == yr ? 1.f : 0.f)) * (1.0f / kMB) : 0.f;
-            sdl32[rr][o] = gl;
-            sdl[rr][o] = bf16_to_f(__float2bfloat16_rn(gl));
-        }
     }
     __syncthreads();
     float db2 = 0.f;                                 // CTA column 0, thread o < d_out: sum_r dL[r][o]
