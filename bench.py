@@ -330,9 +330,87 @@ def run_ours(args):
         torch.cuda.empty_cache()
         if "mlp" in sections:
             line["mlp"] = run_mlp(B, wlm, dev, peaks)
+        if "tiny" in sections:
+            line["tiny"] = run_tiny(B, wlm, dev)
         print(json.dumps(line), flush=True)
     D.barrier(dev)
     D.shutdown()
+
+
+def run_tiny(B, wlm, dev, iters=2000):
+    """Workload 1 (P = 4096, W = 2, b = (3, 1)) moves 131 KB per iteration: it is bound by launches, not bytes,
+    so it is reported as microseconds per iteration (4 accumulate + 1 fused step): plain calls in eager and in
+    pipelined mode, two iterations captured into a CUDA graph and replayed (eager mode enqueues on stream_acc
+    only; the accumulator sets alternate with period 2), and the C oracle on the host."""
+    import time
+
+    import torch
+
+    from oracle.c_oracle import AbsSgdOracleC
+
+    wl = wlm.config(1)
+    order = wlm.call_order(wlm.schedule(wl)[0])
+    x0 = wlm.params0(wl)
+    pool = [wlm.fresh_grad(wl, 0, 0, k) for k in range(8)]
+    pool_d = [torch.from_numpy(g).to(dev) for g in pool]
+    x0_d = torch.from_numpy(x0).to(dev)
+    out = {"workload": "cfg1 tiny: P=4096, W=2, b=(3,1); 5 launches per iteration", "iterations": iters}
+
+    def iterate(eng, n, c0=0, batched=False):
+        c = c0
+        for _ in range(n):
+            if batched:                                   # one abs_accumulate_batch per worker: 3 launches per iteration
+                per_worker = {}
+                for (i, k) in order:
+                    per_worker.setdefault(i, []).append(pool_d[c % 8]); c += 1
+                for i, gs in per_worker.items():
+                    eng.accumulate_batch(i, gs)
+            else:
+                for (i, k) in order:
+                    eng.accumulate(i, pool_d[c % 8]); c += 1
+            eng.sync_step()
+
+    for name, pipelined in (("eager", False), ("pipelined", True)):
+        eng = B.AbsSgd(x0_d, wl.W, wl.lr, wl.momentum, wl.weight_decay, pipelined=pipelined)
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        with torch.cuda.stream(eng.stream_acc):
+            iterate(eng, 20)
+            eng.wait(); e0.record()
+            iterate(eng, iters)
+            eng.wait(); e1.record()
+        torch.cuda.synchronize()
+        out["us_per_iteration_" + name] = e0.elapsed_time(e1) / iters * 1e3
+        eng.check(); eng.destroy()
+
+    for name, batched in (("cuda_graph", False), ("cuda_graph_batched_accumulate", True)):
+        eng = B.AbsSgd(x0_d, wl.W, wl.lr, wl.momentum, wl.weight_decay)
+        with torch.cuda.stream(eng.stream_acc):
+            iterate(eng, 2, batched=batched)
+        eng.synchronize()
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g, stream=eng.stream_acc):
+            iterate(eng, 2, batched=batched)              # recorded, not run: two iterations
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        with torch.cuda.stream(eng.stream_acc):
+            for _ in range(10):
+                g.replay()
+            e0.record()
+            for _ in range(iters // 2):
+                g.replay()
+            e1.record()
+        torch.cuda.synchronize()
+        out["us_per_iteration_" + name] = e0.elapsed_time(e1) / (iters // 2 * 2) * 1e3
+        eng.check(); eng.destroy()
+
+    o = AbsSgdOracleC(x0, wl.W, wl.lr, wl.momentum, wl.weight_decay)
+    c = 0
+    t0 = time.perf_counter()
+    for _ in range(iters):
+        for (i, k) in order:
+            o.accumulate(i, pool[c % 8]); c += 1
+        o.sync_step()
+    out["us_per_iteration_cpu_oracle"] = (time.perf_counter() - t0) / iters * 1e6
+    return out
 
 
 def run_mlp(B, wlm, dev, peaks, iters=12):
@@ -520,7 +598,7 @@ def main():
     ap.add_argument("--steps", type=int, default=1000)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--sections", default="e2e,cpu,mlp",
+    ap.add_argument("--sections", default="e2e,cpu,mlp,tiny",
                     help="extra measurements after the timed region (drop them for a profiler's launch list)")
     args = ap.parse_args()
     if args.warmup < 3:

@@ -243,3 +243,51 @@ def test_accumulator_matches_oracle_bitwise():
     for i in range(wl.W):
         assert np.array_equal(e.accumulator(0, i).cpu().numpy(), o.acc[0, i])
     e.destroy()
+
+
+def test_cuda_graph_replay_of_the_tiny_workload():
+    """Workload 1 is launch-bound (5 launches of a few microseconds per iteration).  In eager mode every call
+    enqueues on stream_acc only, so two iterations (the accumulator sets alternate with period 2) can be captured
+    into a CUDA graph and replayed; the parameters after R replays match the oracle after 2 + 2 R iterations."""
+    import torch
+
+    from oracle.abs_oracle import AbsSgdOracle
+    from paper_2308_15164_b200 import binding as B
+
+    wl = wlm.config(1)
+    order = wlm.call_order(wlm.schedule(wl)[0])                 # b = (3, 1): 4 calls per iteration
+    rng = np.random.default_rng(21)
+    x0 = wlm.params0(wl)
+    pool = (rng.standard_normal((8, wl.P)) * 0.5).astype(np.float32)
+    pool_d = [torch.from_numpy(pool[j]).cuda() for j in range(8)]
+    eng = B.AbsSgd(torch.from_numpy(x0).cuda(), wl.W, wl.lr, wl.momentum, wl.weight_decay)   # eager
+    c = [0]
+
+    def two_iterations():
+        for _ in range(2):
+            for (i, k) in order:
+                eng.accumulate(i, pool_d[c[0] % 8]); c[0] += 1
+            eng.sync_step()
+
+    with torch.cuda.stream(eng.stream_acc):
+        two_iterations()                                        # iterations 0, 1 (the first step applies nothing)
+    eng.synchronize()
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(g, stream=eng.stream_acc):
+        two_iterations()                                        # recorded, not run
+    R = 25
+    for _ in range(R):
+        g.replay()
+    torch.cuda.synchronize()
+    got = eng.params_host()
+    eng.destroy()
+
+    o = AbsSgdOracle(x0, wl.W, wl.lr, wl.momentum, wl.weight_decay)
+    cc = 0
+    for _ in range(2 + 2 * R):
+        for (i, k) in order:
+            o.accumulate(i, pool[cc % 8]); cc += 1
+        o.sync_step()
+    want = o.params()
+    assert np.abs(want - x0).max() > 1e-3
+    assert np.abs(got - want).max() <= H.TOL_F32 * np.abs(want).max()
