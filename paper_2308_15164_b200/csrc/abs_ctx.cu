@@ -222,7 +222,7 @@ int collect_timings(abs_ctx* c) {
 void mlp_mark(void* user, int kernel_class, int n, cudaStream_t stream);
 
 // stream_acc waits (on the device) for every gradient kernel enqueued so far on the worker streams.
-int join_dw(abs_ctx* c) {
+int join_workers(abs_ctx* c) {
     for (int k = 0; k < c->n_wstreams; ++k)
         if (c->w_outstanding[k]) {
             CK(cudaStreamWaitEvent(c->s_acc, c->ev_w_done[k], 0));
@@ -374,7 +374,7 @@ int abs_accumulate(abs_ctx* c, uint32_t worker, const void* grad_dev) {
     if (!live(c)) return ABS_ESTATE;
     if (worker >= c->cfg.W) return invalid(c, "worker index out of range");
     if (!grad_dev || (reinterpret_cast<uintptr_t>(grad_dev) & 15)) return invalid(c, "gradient pointer must be non-NULL and 16-byte aligned");
-    if (int rc = join_dw(c)) return rc;
+    if (int rc = join_workers(c)) return rc;
     // overwrite-first mode: the row is not kept zeroed, so a worker's first micro-batch of an iteration stores
     const bool first = (c->cfg.flags & ABS_FLAG_OVERWRITE_FIRST) && c->h_cnt[(size_t)c->cur * c->cfg.W + worker] == 0;
     {
@@ -398,7 +398,7 @@ int abs_accumulate_batch(abs_ctx* c, uint32_t worker, uint32_t n, const void* co
             return invalid(c, "every gradient pointer must be non-NULL and 16-byte aligned");
         gl.p[k] = grads_dev[k];
     }
-    if (int rc = join_dw(c)) return rc;
+    if (int rc = join_workers(c)) return rc;
     const bool first = (c->cfg.flags & ABS_FLAG_OVERWRITE_FIRST) && c->h_cnt[(size_t)c->cur * c->cfg.W + worker] == 0;
     {
         Timed tm(c, ABS_K_ACCUMULATE, c->s_acc);
@@ -415,7 +415,7 @@ int abs_accumulate_host(abs_ctx* c, uint32_t worker, const void* grad_host) {
     if (!(c->cfg.flags & ABS_FLAG_HOST_INPUT)) return invalid(c, "context was created without ABS_FLAG_HOST_INPUT");
     if (worker >= c->cfg.W) return invalid(c, "worker index out of range");
     if (!grad_host) return invalid(c, "gradient pointer is NULL");
-    if (int rc = join_dw(c)) return rc;
+    if (int rc = join_workers(c)) return rc;
     const bool first = (c->cfg.flags & ABS_FLAG_OVERWRITE_FIRST) && c->h_cnt[(size_t)c->cur * c->cfg.W + worker] == 0;
     const int k = c->stage_next;
     c->stage_next ^= 1;
@@ -454,7 +454,7 @@ int abs_accumulate_mlp_batch(abs_ctx* c, uint32_t worker, uint32_t n, const floa
     const int variant = c->ctas_per_sm[ABS_K_MLP_DW1];
     const bool serial = c->ctas_per_sm[ABS_K_MLP_FWD] == 1;   // measurement aid: everything on stream_acc
     if (serial) {
-        if (int rc = join_dw(c)) return rc;
+        if (int rc = join_workers(c)) return rc;
     } else if (c->set_used[set]) {
         CK(cudaStreamWaitEvent(c->s_acc, c->ev_set_done[set], 0));   // the scratch set is free again
     }
@@ -496,7 +496,7 @@ int abs_sync_step(abs_ctx* c) {
     if (!c->pipelined) {
         // Step 1 on the delayed set, in place, on stream_acc: the gradient kernels still running on the
         // worker streams read the parameters it overwrites.
-        if (int rc = join_dw(c)) return rc;
+        if (int rc = join_workers(c)) return rc;
         int64_t B = 0;
         for (uint32_t i = 0; i < W; ++i) B += c->h_cnt[(size_t)d * W + i];
         if (B > 0) {
@@ -576,7 +576,7 @@ int abs_momentum(abs_ctx* c, const float** v_dev_out) {
 int abs_accumulator(abs_ctx* c, uint32_t set, uint32_t worker, const float** acc_dev_out) {
     if (!live(c)) return ABS_ESTATE;
     if (set > 1 || worker >= c->cfg.W || !acc_dev_out) return invalid(c, "bad set / worker / output pointer");
-    if (int rc = join_dw(c)) return rc;
+    if (int rc = join_workers(c)) return rc;
     *acc_dev_out = c->acc(set, worker);
     return ABS_OK;
 }
@@ -620,7 +620,7 @@ int abs_set_lr(abs_ctx* c, float lr) {
 
 int abs_wait(abs_ctx* c) {
     if (!live(c)) return ABS_ESTATE;
-    if (int rc = join_dw(c)) return rc;
+    if (int rc = join_workers(c)) return rc;
     if (c->pipelined) {
         CK(cudaEventRecord(c->ev_aux, c->s_sync));
         CK(cudaStreamWaitEvent(c->s_acc, c->ev_aux, 0));
