@@ -332,9 +332,42 @@ def run_ours(args):
             line["mlp"] = run_mlp(B, wlm, dev, peaks)
         if "tiny" in sections:
             line["tiny"] = run_tiny(B, wlm, dev)
+        if "batch_curve" in sections:
+            line["accumulate_batch_curve"] = run_batch_curve(B, dev, peaks)
         print(json.dumps(line), flush=True)
     D.barrier(dev)
     D.shutdown()
+
+
+def run_batch_curve(B, dev, peaks, P=40_000_000):
+    """abs_accumulate_batch alone on the GPU (eager mode, an event pair around every launch) for n = 1..8
+    gradients per call, fp32 and bf16: GB/s on the call's own algorithmic bytes, (g n + 8) P with g = 4 or 2."""
+    import torch
+
+    out = {"P": P, "unit": "GB/s on (g*n + 8) * P bytes", "peak": peaks["hbm_gbs"]}
+    for dtype, gd, gb in (("f32", B.GRAD_F32, 4), ("bf16", B.GRAD_BF16, 2)):
+        gen = torch.Generator(device=dev).manual_seed(1)
+        pool = [torch.randn(P, device=dev, generator=gen).to(torch.float32 if gb == 4 else torch.bfloat16) for _ in range(12)]
+        eng = B.AbsSgd(torch.zeros(P, device=dev), 4, 0.1, grad_dtype=gd)
+        res = {}
+        for n in range(1, 9):
+            for rep_ in range(2):                      # the first round warms up
+                eng.profile(True)
+                with torch.cuda.stream(eng.stream_acc):
+                    for it in range(24):
+                        gs = [pool[(it * 5 + k) % 12] for k in range(n)]
+                        if n == 1:
+                            eng.accumulate(it % 4, gs[0])
+                        else:
+                            eng.accumulate_batch(it % 4, gs)
+                cnt, ms = eng.kernel_stats(B.K_ACCUMULATE)
+                eng.profile(False)
+            res[str(n)] = {"us": ms / cnt * 1e3, "gbs": (gb * n + 8) * P / (ms / cnt) / 1e6}
+        out[dtype] = res
+        eng.check(); eng.destroy()
+        del pool
+        torch.cuda.empty_cache()
+    return out
 
 
 def run_tiny(B, wlm, dev, iters=2000):
@@ -598,7 +631,7 @@ def main():
     ap.add_argument("--steps", type=int, default=1000)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--sections", default="e2e,cpu,mlp,tiny",
+    ap.add_argument("--sections", default="e2e,cpu,mlp,tiny,batch_curve",
                     help="extra measurements after the timed region (drop them for a profiler's launch list)")
     args = ap.parse_args()
     if args.warmup < 3:

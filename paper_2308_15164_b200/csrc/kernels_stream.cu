@@ -170,29 +170,45 @@ __global__ void __launch_bounds__(kBlock) k_accumulate_multi_f32(float* acc, Gra
     }
 }
 
-template <bool kOverwrite>
+template <int U, int MAXN, bool kOverwrite>   // n <= MAXN
 __global__ void __launch_bounds__(kBlock) k_accumulate_multi_bf16(float* acc, GradList gl, int n, unsigned long long n_vec8,
                                                                   unsigned long long P, int32_t* cnt) {
     float4* acc4 = reinterpret_cast<float4*>(acc);
-    for (unsigned long long idx = blockIdx.x * (unsigned long long)kBlock + threadIdx.x; idx < n_vec8;
-         idx += (unsigned long long)gridDim.x * kBlock) {
-        uint4 b[kMaxAccBatch];
+    const unsigned long long tile = (unsigned long long)kBlock * U;
+    for (unsigned long long base = blockIdx.x * tile; base < n_vec8; base += gridDim.x * tile) {
+        uint4 b[U][MAXN];
+        float4 a0[U], a1[U];
 #pragma unroll
-        for (int k = 0; k < kMaxAccBatch; ++k)
-            if (k < n) b[k] = ld_stream(static_cast<const uint4*>(gl.p[k]) + idx);
-        float4 a0 = make_float4(0.f, 0.f, 0.f, 0.f), a1 = a0;   // 0 + g = g: storing is adding to zero
-        if (!kOverwrite) {
-            a0 = acc4[2 * idx];
-            a1 = acc4[2 * idx + 1];
+        for (int u = 0; u < U; ++u) {
+            const unsigned long long idx = base + (unsigned long long)u * kBlock + threadIdx.x;
+            if (idx < n_vec8) {
+#pragma unroll
+                for (int k = 0; k < MAXN; ++k)
+                    if (k < n) b[u][k] = ld_stream(static_cast<const uint4*>(gl.p[k]) + idx);
+                a0[u] = make_float4(0.f, 0.f, 0.f, 0.f);   // 0 + g = g: storing is adding to zero
+                a1[u] = a0[u];
+                if (!kOverwrite) {
+                    a0[u] = acc4[2 * idx];
+                    a1[u] = acc4[2 * idx + 1];
+                }
+            }
         }
 #pragma unroll
-        for (int k = 0; k < kMaxAccBatch; ++k)
-            if (k < n) {
-                a0.x += bf16_lo(b[k].x); a0.y += bf16_hi(b[k].x); a0.z += bf16_lo(b[k].y); a0.w += bf16_hi(b[k].y);
-                a1.x += bf16_lo(b[k].z); a1.y += bf16_hi(b[k].z); a1.z += bf16_lo(b[k].w); a1.w += bf16_hi(b[k].w);
+        for (int u = 0; u < U; ++u) {
+            const unsigned long long idx = base + (unsigned long long)u * kBlock + threadIdx.x;
+            if (idx < n_vec8) {
+#pragma unroll
+                for (int k = 0; k < MAXN; ++k)
+                    if (k < n) {
+                        a0[u].x += bf16_lo(b[u][k].x); a0[u].y += bf16_hi(b[u][k].x);
+                        a0[u].z += bf16_lo(b[u][k].y); a0[u].w += bf16_hi(b[u][k].y);
+                        a1[u].x += bf16_lo(b[u][k].z); a1[u].y += bf16_hi(b[u][k].z);
+                        a1[u].z += bf16_lo(b[u][k].w); a1[u].w += bf16_hi(b[u][k].w);
+                    }
+                st_stream(acc4 + 2 * idx, a0[u]);
+                st_stream(acc4 + 2 * idx + 1, a1[u]);
             }
-        st_stream(acc4 + 2 * idx, a0);
-        st_stream(acc4 + 2 * idx + 1, a1);
+        }
     }
     if (blockIdx.x == 0) {
         const unsigned long long j = n_vec8 * 8 + threadIdx.x;  // ragged tail (P % 8 elements)
@@ -397,6 +413,10 @@ cudaError_t launch_accumulate_multi(float* acc_row, const GradList& gl, int n, u
             const unsigned grid = grid_for(n_vec, kBlock * 2, ctas_per_sm, num_sms);
             if (overwrite) k_accumulate_multi_f32<2, 4, true><<<grid, kBlock, 0, stream>>>(acc_row, gl, n, n_vec, P, cnt);
             else k_accumulate_multi_f32<2, 4, false><<<grid, kBlock, 0, stream>>>(acc_row, gl, n, n_vec, P, cnt);
+        } else if (n <= 6) {
+            const unsigned grid = grid_for(n_vec, kBlock * 2, ctas_per_sm, num_sms);
+            if (overwrite) k_accumulate_multi_f32<2, 6, true><<<grid, kBlock, 0, stream>>>(acc_row, gl, n, n_vec, P, cnt);
+            else k_accumulate_multi_f32<2, 6, false><<<grid, kBlock, 0, stream>>>(acc_row, gl, n, n_vec, P, cnt);
         } else {
             const unsigned grid = grid_for(n_vec, kBlock, ctas_per_sm, num_sms);
             if (overwrite) k_accumulate_multi_f32<1, 8, true><<<grid, kBlock, 0, stream>>>(acc_row, gl, n, n_vec, P, cnt);
@@ -404,9 +424,15 @@ cudaError_t launch_accumulate_multi(float* acc_row, const GradList& gl, int n, u
         }
     } else {
         const unsigned long long n_vec8 = P / 8;
-        const unsigned grid = grid_for(n_vec8, kBlock, ctas_per_sm, num_sms);
-        if (overwrite) k_accumulate_multi_bf16<true><<<grid, kBlock, 0, stream>>>(acc_row, gl, n, n_vec8, P, cnt);
-        else k_accumulate_multi_bf16<false><<<grid, kBlock, 0, stream>>>(acc_row, gl, n, n_vec8, P, cnt);
+        if (n <= 4) {
+            const unsigned grid = grid_for(n_vec8, kBlock * 2, ctas_per_sm, num_sms);
+            if (overwrite) k_accumulate_multi_bf16<2, 4, true><<<grid, kBlock, 0, stream>>>(acc_row, gl, n, n_vec8, P, cnt);
+            else k_accumulate_multi_bf16<2, 4, false><<<grid, kBlock, 0, stream>>>(acc_row, gl, n, n_vec8, P, cnt);
+        } else {
+            const unsigned grid = grid_for(n_vec8, kBlock, ctas_per_sm, num_sms);
+            if (overwrite) k_accumulate_multi_bf16<1, 8, true><<<grid, kBlock, 0, stream>>>(acc_row, gl, n, n_vec8, P, cnt);
+            else k_accumulate_multi_bf16<1, 8, false><<<grid, kBlock, 0, stream>>>(acc_row, gl, n, n_vec8, P, cnt);
+        }
     }
     return cudaGetLastError();
 }
