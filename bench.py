@@ -332,11 +332,71 @@ def run_ours(args):
             line["mlp"] = run_mlp(B, wlm, dev, peaks)
         if "tiny" in sections:
             line["tiny"] = run_tiny(B, wlm, dev)
+        if "workloads35" in sections:                 # opt-in: generating workload 5's gradient pool takes a while
+            line["workloads_3_and_5"] = run_other_workloads(B, wlm, dev)
         if "batch_curve" in sections:
             line["accumulate_batch_curve"] = run_batch_curve(B, dev, peaks)
         print(json.dumps(line), flush=True)
     D.barrier(dev)
     D.shutdown()
+
+
+def run_other_workloads(B, wlm, dev):
+    """Whole iterations of workloads 3 (W = 8, idle workers) and 5 (W = 16, bf16 gradients) at full size,
+    pipelined, with single and with batched accumulate calls: time per iteration and GB/s on the run's own
+    algorithmic bytes ((g + 8) P per single call, (g n + 8) P per batch call, (8 W_act + 16) P per fused step)."""
+    import numpy as np
+    import torch
+
+    out = {}
+    for cfg, T in ((3, 60), (5, 20)):
+        wl = wlm.config(cfg, T=T)
+        x0 = wlm.params0(wl)
+        pool = wlm.grad_pool(wl)
+        src = torch.from_numpy(pool.view(np.int16) if pool.dtype == np.uint16 else pool)
+        pool_d = torch.zeros((pool.shape[0], (pool.shape[1] + 7) // 8 * 8), dtype=src.dtype, device=dev)
+        pool_d[:, :pool.shape[1]] = src.to(dev)
+        rows = [pool_d[r].data_ptr() for r in range(wl.pool_size)]
+        bf16 = wl.grad_dtype == "bf16"
+        gb = 2 if bf16 else 4
+        sched = wlm.schedule(wl)
+        res = {"P": wl.P, "W": wl.W, "iterations": T, "grad_dtype": wl.grad_dtype}
+        for name, batched in (("single_calls", False), ("batch_calls", True)):
+            eng = B.AbsSgd(torch.from_numpy(x0).to(dev), wl.W, wl.lr, wl.momentum, wl.weight_decay,
+                           grad_dtype=B.GRAD_BF16 if bf16 else B.GRAD_F32, pipelined=True)
+            for rep_ in range(2):                      # the first round warms up
+                torch.cuda.synchronize()
+                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                nbytes, prev_active = 0, 0
+                with torch.cuda.stream(eng.stream_acc):
+                    e0.record()
+                    for t, calls in enumerate(wlm.iter_calls(wl)):
+                        if batched:
+                            per = {}
+                            for (i, k, c) in calls:
+                                per.setdefault(i, []).append(rows[c % wl.pool_size])
+                            for i, gs in per.items():
+                                for lo in range(0, len(gs), 8):
+                                    eng.accumulate_batch(i, gs[lo:lo + 8])
+                                    nbytes += (gb * len(gs[lo:lo + 8]) + 8) * wl.P
+                        else:
+                            for (i, k, c) in calls:
+                                eng.accumulate(i, rows[c % wl.pool_size])
+                                nbytes += (gb + 8) * wl.P
+                        eng.sync_step()                # applies the previous iteration's set
+                        if prev_active:
+                            nbytes += (8 * prev_active + 16) * wl.P
+                        prev_active = int((sched[t] > 0).sum())
+                    eng.wait()
+                    e1.record()
+                torch.cuda.synchronize()
+            ms = e0.elapsed_time(e1)
+            res[name] = {"us_per_iteration": ms / T * 1e3, "gbs_on_its_own_bytes": nbytes / ms / 1e6}
+            eng.check(); eng.destroy()
+        out[f"workload_{cfg}"] = res
+        del pool_d
+        torch.cuda.empty_cache()
+    return out
 
 
 def run_batch_curve(B, dev, peaks, P=40_000_000):
