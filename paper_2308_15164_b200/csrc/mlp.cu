@@ -24,10 +24,13 @@
 //                   each group of 8 ("last CTA done" ticket) sums the group's partial logits in a fixed order
 //   k_bwd           every CTA: logits = sum of group partials + b2, softmax, dL (CTA 0: db2 += ...); then
 //                   dH, dZ, bf16(dZ)^T, db1 += ..., dW2 += ..., b_i += 1
-//   k_dw1_tcgen05   dW1 tile = A B^T on the 5th-gen tensor cores (TMEM accumulator); epilogue adds the
-//                   tile into the worker's accumulator slice via TMA load / TMA store (or TMA reduce-add)
-//   (k_dw1_ring     persistent, warp-specialised, K-batched: operand ring in shared memory, two TMEM
-//                   accumulators, TMA store / reduce-add of the finished tiles)
+//   dW1 = X^T dZ on the 5th-gen tensor cores (TMEM accumulator), one of (chosen per call, see launch_mlp_dw1):
+//   k_dw1_ring      persistent, warp-specialised, K-batched: operand ring in shared memory, two TMEM
+//                   accumulators, finished tiles leave by TMA store (a worker's first gradient of an iteration)
+//                   or TMA reduce-add; 128 x 64 or 128 x 128 tiles
+//   k_dw1_regs      one 128 x 64 tile per CTA, the accumulator tile prefetched into registers, K-batched
+//   k_dw1_tcgen05   one tile per CTA, the accumulator tile by TMA load / add in shared memory / TMA store
+//                   (or TMA reduce-add); the first version, kept selectable
 #include <cuda.h>
 
 #include <cstdio>
