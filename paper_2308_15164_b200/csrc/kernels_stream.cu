@@ -224,8 +224,8 @@ __global__ void __launch_bounds__(kBlock) k_accumulate_multi_bf16(float* acc, Gr
 // ------------------------------------------------------------------------------------------
 // Step 1 + update, fused.  (8*W_act + 16) bytes per parameter, W_act = #{i : b_i > 0}:
 // read W_act accumulators + x + v, write x' + v + W_act zeros.  Rows of idle workers
-// (b_i = 0) are neither read nor rewritten.  WT > 0: W known at compile time (all loads of a
-// vector are issued before the first add); WT == 0: any W, in chunks of 8 rows.
+// (b_i = 0) are neither read nor rewritten.  WT > 0 (used for W <= 4): W known at compile time, all
+// loads of a vector are issued before the first add; WT == 0: any W, in chunks of 8 rows.
 // ------------------------------------------------------------------------------------------
 __device__ __forceinline__ void update_vec(float4& x, float4& v, const float4 s, const float Bf,
                                            const SyncArgs& a) {
@@ -438,26 +438,24 @@ cudaError_t launch_accumulate_multi(float* acc_row, const GradList& gl, int n, u
 }
 
 cudaError_t launch_sync(const SyncArgs& a, int ctas_per_sm, int num_sms, cudaStream_t stream) {
-    if (ctas_per_sm == 0) ctas_per_sm = -1;   // measured: one tile per CTA beats a persistent grid
+    // Measured on B200 (kernel alone, accumulators far larger than L2, GB/s on (8 W + 16) P bytes):
+    //   W <= 4   compile-time W, every load of a vector in flight at once, one tile per CTA: 6.2 - 6.5 TB/s
+    //            (W = 1: two vectors per thread);
+    //   W >= 5   rows in chunks of 8 (at most 10 loads in flight per thread, 2 CTAs resident per SM).  With
+    //            compile-time W the same kernels fell to 4.4 - 4.9 TB/s (W = 5..12) and 2.9 TB/s (W = 16: 142
+    //            registers, one CTA per SM).  Up to W = 24 a persistent grid of exactly the resident CTAs is
+    //            best (5.4 - 6.25 TB/s against 4.3 - 6.0 with one tile per CTA); beyond, a tile already takes
+    //            long enough and one tile per CTA wins again (6.2 - 6.4 TB/s).
+    if (a.W > 4) {
+        if (ctas_per_sm == 0) ctas_per_sm = a.W <= 24 ? 2 : -1;
+        return launch_sync_t<0, 1>(a, ctas_per_sm, num_sms, stream);
+    }
+    if (ctas_per_sm == 0) ctas_per_sm = -1;
     switch (a.W) {
-        // One vector per thread measured best for every W (W = 2..16: 6.5-6.8 TB/s); W = 1 likes two.
         case 1: return launch_sync_t<1, 2>(a, ctas_per_sm, num_sms, stream);
         case 2: return launch_sync_t<2, 1>(a, ctas_per_sm, num_sms, stream);
         case 3: return launch_sync_t<3, 1>(a, ctas_per_sm, num_sms, stream);
-        case 4: return launch_sync_t<4, 1>(a, ctas_per_sm, num_sms, stream);
-        case 5: return launch_sync_t<5, 1>(a, ctas_per_sm, num_sms, stream);
-        case 6: return launch_sync_t<6, 1>(a, ctas_per_sm, num_sms, stream);
-        case 7: return launch_sync_t<7, 1>(a, ctas_per_sm, num_sms, stream);
-        case 8: return launch_sync_t<8, 1>(a, ctas_per_sm, num_sms, stream);
-        case 9: return launch_sync_t<9, 1>(a, ctas_per_sm, num_sms, stream);
-        case 10: return launch_sync_t<10, 1>(a, ctas_per_sm, num_sms, stream);
-        case 11: return launch_sync_t<11, 1>(a, ctas_per_sm, num_sms, stream);
-        case 12: return launch_sync_t<12, 1>(a, ctas_per_sm, num_sms, stream);
-        case 13: return launch_sync_t<13, 1>(a, ctas_per_sm, num_sms, stream);
-        case 14: return launch_sync_t<14, 1>(a, ctas_per_sm, num_sms, stream);
-        case 15: return launch_sync_t<15, 1>(a, ctas_per_sm, num_sms, stream);
-        case 16: return launch_sync_t<16, 1>(a, ctas_per_sm, num_sms, stream);
-        default: return launch_sync_t<0, 1>(a, ctas_per_sm, num_sms, stream);
+        default: return launch_sync_t<4, 1>(a, ctas_per_sm, num_sms, stream);
     }
 }
 
