@@ -334,6 +334,8 @@ def run_ours(args):
             line["tiny"] = run_tiny(B, wlm, dev)
         if "workloads35" in sections:                 # opt-in: generating workload 5's gradient pool takes a while
             line["workloads_3_and_5"] = run_other_workloads(B, wlm, dev)
+        if "sync_curve" in sections:
+            line["sync_curve"] = run_sync_curve(B, dev, peaks)
         if "batch_curve" in sections:
             line["accumulate_batch_curve"] = run_batch_curve(B, dev, peaks)
         print(json.dumps(line), flush=True)
@@ -396,6 +398,31 @@ def run_other_workloads(B, wlm, dev):
         out[f"workload_{cfg}"] = res
         del pool_d
         torch.cuda.empty_cache()
+    return out
+
+
+def run_sync_curve(B, dev, peaks, P=11_689_512):
+    """The fused step alone on the GPU (eager mode, an event pair around every launch) for several worker
+    counts W, every worker active: GB/s on its algorithmic bytes (8 W + 16) P.  For W <= 2 the accumulators
+    written just before partly sit in the 126 MB L2, so those two points are optimistic."""
+    import torch
+
+    out = {"P": P, "unit": "GB/s on (8*W + 16) * P bytes", "peak": peaks["hbm_gbs"]}
+    gen = torch.Generator(device=dev).manual_seed(2)
+    g = torch.randn(P + 8, device=dev, generator=gen)
+    for W in (1, 2, 4, 5, 6, 8, 12, 16, 17, 24, 32, 64):
+        eng = B.AbsSgd(torch.zeros(P, device=dev), W, 0.1, 0.9, 5e-4)
+        for rep_ in range(2):                          # the first round warms up
+            eng.profile(True)
+            with torch.cuda.stream(eng.stream_acc):
+                for it in range(5):
+                    for i in range(W):
+                        eng.accumulate(i, g)
+                    eng.sync_step()
+            n, ms = eng.kernel_stats(B.K_SYNC)
+            eng.profile(False)
+        out[str(W)] = {"us": ms / n * 1e3, "gbs": (8 * W + 16) * P / (ms / n) / 1e6}
+        eng.check(); eng.destroy()
     return out
 
 
@@ -691,7 +718,7 @@ def main():
     ap.add_argument("--steps", type=int, default=1000)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--sections", default="e2e,cpu,mlp,tiny,batch_curve",
+    ap.add_argument("--sections", default="e2e,cpu,mlp,tiny,batch_curve,sync_curve",
                     help="extra measurements after the timed region (drop them for a profiler's launch list)")
     args = ap.parse_args()
     if args.warmup < 3:
