@@ -10,8 +10,9 @@
 // 128-bit accesses, all independent loads of a thread issued before the first use, and one pass
 // over every byte (each accumulator element is read once and overwritten with zero by the same
 // thread that read it).  Launch shape: measured on B200, one tile per CTA (a grid of thousands
-// of 256-thread CTAs) beats a persistent grid of 148 x k CTAs by 5-10 % for these kernels, so
-// that is the default; abs_set_launch can still select a persistent grid.
+// of 256-thread CTAs) beats a persistent grid of 148 x k CTAs by 5-10 % for the accumulate kernels
+// and for the fused step with up to 4 workers, so that is their default; the fused step with more
+// workers runs its chunked form on a persistent grid (see launch_sync).  abs_set_launch overrides.
 #include "abs_internal.h"
 
 namespace abs_sgd {
