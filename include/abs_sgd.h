@@ -72,6 +72,8 @@ extern "C" {
                                        to be empty), which saves the read of the W1 slice.                    */
 
 #define ABS_MAX_WORKERS 64u
+#define ABS_MAX_RANKS   16u   /* GPUs taking part in abs_global_* (n_ranks * W <= ABS_MAX_WORKERS)        */
+#define ABS_IPC_HANDLE_BYTES 64
 
 /* Kernel classes, for abs_kernel_stats() and abs_set_launch(). */
 #define ABS_K_ACCUMULATE 0   /* Step 2: acc += g                                        */
@@ -242,6 +244,75 @@ const char *abs_last_error(abs_ctx *ctx);
 /* Waits for the context's enqueued work, releases events and host state.  The workspace
  * is the caller's to free afterwards.  Using ctx after this returns ABS_ESTATE. */
 int abs_destroy(abs_ctx *ctx);
+
+/* ---------------------------------------------------------------------------------------------------
+ * Step 1 across GPUs: the paper's own setting (Section 5.1-5.2: the workers are different GPUs and Step 1 is
+ * the "global synchronization" of G_{t-1}^i and of the batch sizes M_{t-1}^i between them).
+ *
+ * One process and one context per GPU ("rank"); a context's W workers are that GPU's local workers, and the
+ * global worker index of local worker i on rank q is q*W + i.  All ranks use the same abs_config (so their
+ * workspaces have the same layout), ABS_FLAG_PIPELINED, and make the same sequence of abs_global_* calls.
+ * abs_accumulate* are used as before; ONE iteration ends with, on every rank,
+ *
+ *     abs_global_begin(ctx, &counts, &n);     // x_{t+1} becomes visible to stream_acc; this rank's b_i go
+ *                                             // into its slots of counts[0..n), zeros elsewhere
+ *     <sum counts[0..n) (int32) over all ranks, in place, ordered on stream_sync>    -- exchange A
+ *     abs_global_step(ctx);                   // the fused kernel, on stream_sync
+ *     <any collective over all ranks ordered on stream_sync>                          -- exchange B
+ *     abs_global_end(ctx);
+ *
+ * instead of abs_sync_step.  The two exchanges are the caller's (ncclAllReduce on stream_sync, or any
+ * equivalent that is ordered with the work on that stream); they carry n <= 64 integers, not gradients.
+ * Exchange A is the paper's batch-size synchronisation and also guarantees that every rank has finished
+ * the iteration's accumulation before any kernel reads its rows; exchange B guarantees that every rank's
+ * kernel has finished before anyone uses x_{t+1} or accumulates into the cleared set again.
+ *
+ * The gradients themselves are moved by the kernel of abs_global_step, not by a collective library: rank r
+ * owns a contiguous slice of the flat vector (abs_global_slice); for its slice it reads every worker row
+ * of every rank through the peer mappings given to abs_global_attach, forms
+ * Gbar = sum_{q,i} G^{q,i} / sum_{q,i} b_{q,i} in global worker order, applies Eq. 6 / weight decay /
+ * momentum exactly as abs_sync_step does, writes x_{t+1} into EVERY rank's parameter buffer (and bf16
+ * copy), and writes zeros over what it read (not with ABS_FLAG_OVERWRITE_FIRST).  Per iteration a rank
+ * receives (G-1)/G * W * 4 bytes per parameter and sends (G-1)/G * (W + 1) * 4: the volume of a
+ * reduce-scatter plus an all-gather, in one pass.  Results equal a one-GPU context with G*W workers fed the
+ * same gradients, bit for bit.  The momentum vector is sharded: a rank keeps only its slice of v current.
+ * If all b are 0 the kernel copies x_t to x_{t+1} everywhere and leaves v alone.
+ * --------------------------------------------------------------------------------------------------- */
+typedef struct abs_peer_table {
+    uint32_t n_ranks;                        /* G, 1..ABS_MAX_RANKS                                          */
+    uint32_t rank;                           /* this context's rank                                          */
+    void *workspace_dev[ABS_MAX_RANKS];      /* every rank's workspace (the pointer it gave abs_init) AS MAPPED
+                                                IN THIS PROCESS: [rank] is the own workspace, the others come
+                                                from abs_ipc_open (other processes) or are plain pointers
+                                                (same process, peer access enabled)                          */
+} abs_peer_table;
+
+/* Once, after abs_init and before the first iteration ends; every rank's abs_init must have completed
+ * (synchronise the streams and the processes first).  Errors: ABS_EINVAL (not pipelined, bad table,
+ * n_ranks * W > 64, called twice).  After it, abs_sync_step returns ABS_EINVAL on this context. */
+int abs_global_attach(abs_ctx *ctx, const abs_peer_table *peers);
+/* See above.  *counts_dev: device pointer (inside the workspace) to n = n_ranks * W int32; valid until
+ * abs_destroy.  Never block the host.  Calls out of order return ABS_EINVAL. */
+int abs_global_begin(abs_ctx *ctx, int32_t **counts_dev, uint32_t *n_counts);
+int abs_global_step(abs_ctx *ctx);
+int abs_global_end(abs_ctx *ctx);
+/* The slice of the flat vector this rank reduces and whose momentum it holds: elements [first, first+count). */
+int abs_global_slice(abs_ctx *ctx, uint64_t *first, uint64_t *count);
+/* The same partition without a context (host arithmetic only): the slices of ranks 0..n_ranks-1 are
+ * consecutive, disjoint and cover [0, P); each starts on a multiple of 1024 elements; trailing ranks may
+ * get an empty slice when P is small. */
+int abs_global_partition(uint64_t P, uint32_t n_ranks, uint32_t rank, uint64_t *first, uint64_t *count);
+/* abs_consumed for a context in multi-GPU mode: b_host[n_ranks * W], global worker order. */
+int abs_global_consumed(abs_ctx *ctx, uint64_t step, int32_t *b_host);
+
+/* CUDA IPC plumbing for ranks in separate processes.  abs_ipc_export: handle_out receives
+ * ABS_IPC_HANDLE_BYTES bytes naming the device allocation that contains dev_ptr, *offset_out the offset of
+ * dev_ptr inside it; send both to the peers.  abs_ipc_open (in a peer process, its GPU current): maps the
+ * allocation and returns the address that corresponds to dev_ptr.  abs_ipc_close undoes abs_ipc_open.
+ * The memory must come from cudaMalloc (not from a virtual-memory pool).  Status codes as everywhere. */
+int abs_ipc_export(const void *dev_ptr, void *handle_out, uint64_t *offset_out);
+int abs_ipc_open(const void *handle, uint64_t offset, void **dev_ptr_out);
+int abs_ipc_close(void *dev_ptr, uint64_t offset);
 
 /* One fused sync step on buffers the CALLER owns, for callers that cannot allocate device
  * memory.  (No counterpart in the paper: this is a packaging variant of the kernel behind

@@ -28,6 +28,7 @@ OK, EINVAL, ESTATE, ECUDA, ENOMEM, ETIMEOUT, ELIMIT = 0, -1, -2, -3, -4, -5, -6
 GRAD_F32, GRAD_BF16 = 0, 1
 FLAG_PIPELINED, FLAG_MLP, FLAG_HOST_INPUT, FLAG_OVERWRITE_FIRST = 1, 2, 4, 8
 K_ACCUMULATE, K_SYNC, K_MLP_FWD, K_MLP_BWD, K_MLP_DW1 = range(5)
+MAX_WORKERS, MAX_RANKS, IPC_HANDLE_BYTES = 64, 16, 64
 KERNEL_NAMES = ["accumulate", "sync", "mlp_fwd", "mlp_bwd", "mlp_dw1"]
 
 
@@ -41,6 +42,10 @@ class AbsConfig(ctypes.Structure):
         ("mlp_mb", ctypes.c_uint32),
         ("stream_acc", ctypes.c_void_p), ("stream_sync", ctypes.c_void_p),
     ]
+
+
+class AbsPeerTable(ctypes.Structure):
+    _fields_ = [("n_ranks", ctypes.c_uint32), ("rank", ctypes.c_uint32), ("workspace_dev", ctypes.c_void_p * MAX_RANKS)]
 
 
 _vp, _u32, _u64 = ctypes.c_void_p, ctypes.c_uint32, ctypes.c_uint64
@@ -69,6 +74,16 @@ _sig = {
     "abs_launch_count": (ctypes.c_uint64, [_vp]),
     "abs_last_error": (ctypes.c_char_p, [_vp]),
     "abs_destroy": (ctypes.c_int, [_vp]),
+    "abs_global_attach": (ctypes.c_int, [_vp, ctypes.POINTER(AbsPeerTable)]),
+    "abs_global_begin": (ctypes.c_int, [_vp, ctypes.POINTER(_vp), ctypes.POINTER(_u32)]),
+    "abs_global_step": (ctypes.c_int, [_vp]),
+    "abs_global_end": (ctypes.c_int, [_vp]),
+    "abs_global_slice": (ctypes.c_int, [_vp, ctypes.POINTER(_u64), ctypes.POINTER(_u64)]),
+    "abs_global_consumed": (ctypes.c_int, [_vp, _u64, _vp]),
+    "abs_global_partition": (ctypes.c_int, [_u64, _u32, _u32, ctypes.POINTER(_u64), ctypes.POINTER(_u64)]),
+    "abs_ipc_export": (ctypes.c_int, [_vp, _vp, ctypes.POINTER(_u64)]),
+    "abs_ipc_open": (ctypes.c_int, [_vp, _u64, ctypes.POINTER(_vp)]),
+    "abs_ipc_close": (ctypes.c_int, [_vp, _u64]),
     "abs_sync_step_noalloc": (ctypes.c_int, [_vp, _vp, _vp, _u64, _u64, _u32, _vp, ctypes.c_float, ctypes.c_float,
                                              ctypes.c_float, _vp]),
 }
@@ -194,6 +209,38 @@ class AbsSgd:
         self._ck(lib.abs_consumed(self._h, step, b.ctypes.data))
         return b
 
+    # ---- Step 1 across GPUs (one context per rank) ----
+    def global_attach(self, rank: int, workspaces):
+        """workspaces: device address of every rank's workspace as mapped in this process (own one at [rank])."""
+        tab = AbsPeerTable()
+        tab.n_ranks, tab.rank = len(workspaces), rank
+        for q, w in enumerate(workspaces):
+            tab.workspace_dev[q] = _ptr(w)
+        self._ck(lib.abs_global_attach(self._h, ctypes.byref(tab)))
+        self.n_ranks = len(workspaces)
+
+    def global_begin(self) -> torch.Tensor:
+        """Returns the int32 exchange vector (aliasing library memory) that the caller sums over all ranks."""
+        p, n = _vp(), _u32(0)
+        self._ck(lib.abs_global_begin(self._h, ctypes.byref(p), ctypes.byref(n)))
+        return _alias(p.value, int(n.value), torch.int32, self.device)
+
+    def global_step(self):
+        self._ck(lib.abs_global_step(self._h))
+
+    def global_end(self):
+        self._ck(lib.abs_global_end(self._h))
+
+    def global_slice(self):
+        first, count = _u64(0), _u64(0)
+        self._ck(lib.abs_global_slice(self._h, ctypes.byref(first), ctypes.byref(count)))
+        return int(first.value), int(count.value)
+
+    def global_consumed(self, step: int) -> np.ndarray:
+        b = np.zeros(self.n_ranks * self.W, dtype=np.int32)
+        self._ck(lib.abs_global_consumed(self._h, step, b.ctypes.data))
+        return b
+
     def step1_finished(self) -> bool:
         done = ctypes.c_int(1)
         self._ck(lib.abs_step1_finished(self._h, ctypes.byref(done)))
@@ -248,13 +295,45 @@ def sync_step_noalloc(x: torch.Tensor, v: torch.Tensor, acc: torch.Tensor, cnt: 
                                          acc.shape[0], cnt.data_ptr(), lr, momentum, weight_decay, s))
 
 
+def global_partition(P: int, n_ranks: int, rank: int) -> tuple:
+    """(first, count): the slice of the flat vector that `rank` of `n_ranks` reduces in multi-GPU mode."""
+    first, count = _u64(0), _u64(0)
+    rc = lib.abs_global_partition(P, n_ranks, rank, ctypes.byref(first), ctypes.byref(count))
+    if rc != OK:
+        raise AbsError(rc, "abs_global_partition: bad arguments")
+    return int(first.value), int(count.value)
+
+
+def ipc_export(dev_ptr) -> tuple:
+    """(handle bytes, offset) naming the device allocation that holds ``dev_ptr``, for abs_ipc_open in another process."""
+    buf = ctypes.create_string_buffer(IPC_HANDLE_BYTES)
+    off = _u64(0)
+    rc = lib.abs_ipc_export(_ptr(dev_ptr), buf, ctypes.byref(off))
+    if rc != OK:
+        raise AbsError(rc, "abs_ipc_export failed (memory not from cudaMalloc?)")
+    return bytes(buf.raw), int(off.value)
+
+
+def ipc_open(handle: bytes, offset: int) -> int:
+    p = _vp()
+    rc = lib.abs_ipc_open(ctypes.c_char_p(handle), offset, ctypes.byref(p))
+    if rc != OK:
+        raise AbsError(rc, "abs_ipc_open failed")
+    return int(p.value)
+
+
+def ipc_close(dev_ptr: int, offset: int):
+    lib.abs_ipc_close(dev_ptr, offset)
+
+
 def _alias(addr: int, n: int, dtype, device) -> torch.Tensor:
     """A tensor viewing ``n`` elements of library-owned device memory at ``addr`` (no copy)."""
     itemsize = torch.empty(0, dtype=dtype).element_size()
 
     class _Mem:
         __cuda_array_interface__ = {
-            "shape": (n,), "typestr": {4: "<f4", 2: "<u2"}[itemsize], "data": (addr, False), "version": 2,
+            "shape": (n,), "typestr": {torch.float32: "<f4", torch.int32: "<i4"}.get(dtype, "<u2"), "data": (addr, False),
+            "version": 2,
         }
 
     return torch.as_tensor(_Mem(), device=device)

@@ -1,5 +1,8 @@
 // Host side of the C ABI: state machine of Algorithm 1 (arXiv 2308.15164), workspace carving,
 // argument checks, stream ordering of Step 1 against Step 2, kernel launches.
+#include <cuda.h>
+
+#include <algorithm>
 #include <cmath>
 #include <cstdio>
 #include <cstring>
@@ -25,7 +28,7 @@ size_t round_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 
 struct Layout {
     size_t P_pad = 0;
-    size_t off_x[2] = {0, 0}, off_v = 0, off_acc = 0, off_cnt = 0, off_ticket = 0, off_log = 0;
+    size_t off_x[2] = {0, 0}, off_v = 0, off_acc = 0, off_cnt = 0, off_ticket = 0, off_log = 0, off_gcnt = 0;
     size_t off_shadow[2] = {0, 0}, off_mlp = 0, off_stage[2] = {0, 0};
     size_t total = 0;
 };
@@ -67,6 +70,7 @@ Layout make_layout(const abs_config& c) {
     L.off_cnt = take((size_t)2 * kMaxW * 4);
     L.off_ticket = take(256);
     L.off_log = take((size_t)kLogDepth * kMaxW * 4);
+    L.off_gcnt = take((size_t)(kMaxW + 64) * 4);   // multi-GPU mode: exchanged b_i of all ranks + "previous step applied" word
     if (c.flags & ABS_FLAG_MLP) {
         L.off_shadow[0] = take(L.P_pad * 2);
         L.off_shadow[1] = pipe ? take(L.P_pad * 2) : L.off_shadow[0];
@@ -80,6 +84,15 @@ Layout make_layout(const abs_config& c) {
     }
     L.total = o;
     return L;
+}
+
+// Multi-GPU mode: rank r owns the float4 vectors [lo, hi) of the padded flat vector -- equal runs of whole
+// 256-vector tiles, the last rank(s) take what is left (possibly nothing).
+void slice_vectors(size_t P_pad, uint32_t G, uint32_t r, unsigned long long* lo, unsigned long long* hi) {
+    const unsigned long long n_vec = P_pad / 4;
+    const unsigned long long per = ((n_vec + G - 1) / G + 255) / 256 * 256;
+    *lo = std::min(n_vec, per * r);
+    *hi = std::min(n_vec, *lo + per);
 }
 
 std::mutex g_live_mu;
@@ -129,6 +142,12 @@ struct abs_ctx {
     int mlp_set_next = 0;
     std::vector<TmapBytes> acc_tmaps;   // [2][W]: TMA descriptor of each accumulator row's W1 slice
 
+    // multi-GPU mode (abs_global_*): every rank's workspace as mapped in this process
+    uint32_t n_ranks = 0, rank = 0;
+    char* peer_ws[kMaxRanks] = {};
+    int global_phase = 0;         // 0 = idle, 1 = after abs_global_begin, 2 = after abs_global_step
+    float global_prev_lr = 0.f;   // rate of the previous abs_global_step
+
     // bookkeeping
     uint64_t launches = 0;
     bool profiling = false;
@@ -149,6 +168,8 @@ struct abs_ctx {
         return reinterpret_cast<int32_t*>(ws + L.off_log) + (step % kLogDepth) * kMaxW;
     }
     __nv_bfloat16* shadow(int k) const { return reinterpret_cast<__nv_bfloat16*>(ws + L.off_shadow[k]); }
+    int32_t* gcnt() const { return reinterpret_cast<int32_t*>(ws + L.off_gcnt); }
+    int* applied_word() const { return reinterpret_cast<int*>(ws + L.off_gcnt) + kMaxW; }
 };
 
 namespace {
@@ -320,7 +341,7 @@ int abs_init(abs_ctx** out, const abs_config* cfg, void* workspace_dev, size_t w
     }
 
     // Algorithm 1, Initialization: G_{-1}^i = 0, counters 0, v = 0, x_0 = params0.
-    const size_t state_bytes = L.off_log + (size_t)kLogDepth * kMaxW * 4;
+    const size_t state_bytes = L.off_gcnt + (size_t)(kMaxW + 64) * 4;
     if ((e = cudaMemsetAsync(c->ws, 0, state_bytes, c->s_acc)) != cudaSuccess) return bail(e, "cudaMemsetAsync");
     if ((e = cudaMemcpyAsync(c->x(0), params0_dev, cfg->P * 4, cudaMemcpyDeviceToDevice, c->s_acc)) != cudaSuccess)
         return bail(e, "cudaMemcpyAsync(params0)");
@@ -491,6 +512,7 @@ int abs_accumulate_mlp(abs_ctx* c, uint32_t worker, const float* x_dev, const in
 
 int abs_sync_step(abs_ctx* c) {
     if (!live(c)) return ABS_ESTATE;
+    if (c->n_ranks != 0) return invalid(c, "context is in multi-GPU mode: end iterations with abs_global_begin / _step / _end");
     const uint32_t W = c->cfg.W;
     const uint32_t d = c->cur ^ 1;   // the delayed set (filled during iteration t-1)
     if (!c->pipelined) {
@@ -551,6 +573,160 @@ int abs_sync_step(abs_ctx* c) {
     return ABS_OK;
 }
 
+// ---- Step 1 across GPUs: one rank per GPU, this context holds the rank's W local workers ---------------
+int abs_global_attach(abs_ctx* c, const abs_peer_table* peers) {
+    if (!live(c)) return ABS_ESTATE;
+    if (!peers) return invalid(c, "peer table is NULL");
+    if (!c->pipelined) return invalid(c, "multi-GPU mode needs ABS_FLAG_PIPELINED (two parameter buffers)");
+    if (peers->n_ranks == 0 || peers->n_ranks > ABS_MAX_RANKS) return invalid(c, "n_ranks must be in 1..16");
+    if (peers->rank >= peers->n_ranks) return invalid(c, "rank out of range");
+    if ((uint64_t)peers->n_ranks * c->cfg.W > ABS_MAX_WORKERS) return invalid(c, "n_ranks * W must not exceed 64");
+    if (c->t != 0 || c->n_ranks != 0) return invalid(c, "attach once, before the first step");
+    for (uint32_t q = 0; q < peers->n_ranks; ++q) {
+        void* p = peers->workspace_dev[q];
+        if (!p || (reinterpret_cast<uintptr_t>(p) & 255)) return invalid(c, "peer workspace must be non-NULL and 256-byte aligned");
+    }
+    if (peers->workspace_dev[peers->rank] != c->ws) return invalid(c, "workspace_dev[rank] must be this context's own workspace");
+    c->n_ranks = peers->n_ranks;
+    c->rank = peers->rank;
+    for (uint32_t q = 0; q < peers->n_ranks; ++q) c->peer_ws[q] = static_cast<char*>(peers->workspace_dev[q]);
+    c->global_phase = 0;
+    return ABS_OK;
+}
+
+int abs_global_begin(abs_ctx* c, int32_t** counts_dev, uint32_t* n_counts) {
+    if (!live(c)) return ABS_ESTATE;
+    if (c->n_ranks == 0) return invalid(c, "abs_global_attach has not been called");
+    if (c->global_phase != 0) return invalid(c, "abs_global_begin / _step / _end must be called in that order");
+    if (!counts_dev || !n_counts) return invalid(c, "output pointer is NULL");
+    const uint32_t W = c->cfg.W;
+    // Publish x_{t+1}: the kernels launched one call ago, on every rank, have all finished (ev_sync_done was
+    // recorded behind the caller's closing barrier).
+    if (c->pending) {
+        CK(cudaStreamWaitEvent(c->s_acc, c->ev_sync_done, 0));
+        c->pub = c->pending_out;
+        c->pending = false;
+    }
+    CK(cudaEventRecord(c->ev_acc_done, c->s_acc));
+    CK(cudaStreamWaitEvent(c->s_sync, c->ev_acc_done, 0));
+    for (int k = 0; k < c->n_wstreams; ++k)
+        if (c->w_outstanding[k]) CK(cudaStreamWaitEvent(c->s_sync, c->ev_w_done[k], 0));
+    // This rank's b_i into its slots of the exchange vector (zeros elsewhere: the caller's sum over ranks then
+    // is a gather); the device counters of the set are cleared here, the kernel reads the exchanged copy.
+    CK(launch_global_counts(c->gcnt(), c->cnt(c->cur, 0), (int)(c->rank * W), (int)W, (int)(c->n_ranks * W), c->s_sync));
+    c->launches += 1;
+    *counts_dev = c->gcnt();
+    *n_counts = c->n_ranks * W;
+    c->global_phase = 1;
+    return ABS_OK;
+}
+
+int abs_global_step(abs_ctx* c) {
+    if (!live(c)) return ABS_ESTATE;
+    if (c->n_ranks == 0) return invalid(c, "abs_global_attach has not been called");
+    if (c->global_phase != 1) return invalid(c, "abs_global_begin / _step / _end must be called in that order");
+    const uint32_t W = c->cfg.W, G = c->n_ranks;
+    const int out = c->pub ^ 1;
+    GlobalSyncArgs a{};
+    a.x_in = c->x(c->pub);
+    a.v = c->v();
+    for (uint32_t q = 0; q < G; ++q) {
+        char* ws = c->peer_ws[q];   // identical configuration on every rank: identical layout
+        a.acc[q] = reinterpret_cast<float*>(ws + c->L.off_acc) + (size_t)c->cur * W * c->L.P_pad;
+        a.x_out[q] = reinterpret_cast<float*>(ws + c->L.off_x[out]);
+        a.shadow[q] = c->mlp ? reinterpret_cast<__nv_bfloat16*>(ws + c->L.off_shadow[out]) : nullptr;
+    }
+    a.row_stride = c->L.P_pad;
+    slice_vectors(c->L.P_pad, G, c->rank, &a.vec_lo, &a.vec_hi);
+    a.G = (int)G;
+    a.W_local = (int)W;
+    a.cnt_all = c->gcnt();
+    a.log_row = c->log_row(c->t + 1);
+    a.ticket = c->ticket();
+    a.applied = c->applied_word();
+    a.lr = c->lr_now;
+    a.mu = c->cfg.momentum;
+    a.wd = c->cfg.weight_decay;
+    a.lambda_dc = c->cfg.lambda_dc;
+    a.disp_scale = c->global_prev_lr;
+    a.zero_acc = (c->cfg.flags & ABS_FLAG_OVERWRITE_FIRST) ? 0 : 1;
+    {
+        Timed tm(c, ABS_K_SYNC, c->s_sync);
+        CK(launch_sync_global(a, c->num_sms, c->s_sync));
+    }
+    c->launches += 1;
+    c->global_prev_lr = c->lr_now;
+    c->pending_out = out;
+    // Logical state (Algorithm 1: clear the consumed set, swap roles, t = t + 1).
+    const uint32_t d = c->cur ^ 1;
+    for (uint32_t i = 0; i < W; ++i) c->h_cnt[(size_t)d * W + i] = 0;
+    c->lr_prev_call = c->lr_now;
+    c->cur = d;
+    c->t += 1;
+    c->global_phase = 2;
+    return ABS_OK;
+}
+
+int abs_global_end(abs_ctx* c) {
+    if (!live(c)) return ABS_ESTATE;
+    if (c->n_ranks == 0) return invalid(c, "abs_global_attach has not been called");
+    if (c->global_phase != 2) return invalid(c, "abs_global_begin / _step / _end must be called in that order");
+    CK(cudaEventRecord(c->ev_sync_done, c->s_sync));
+    c->pending = true;
+    c->global_phase = 0;
+    return ABS_OK;
+}
+
+int abs_global_slice(abs_ctx* c, uint64_t* first, uint64_t* count) {
+    if (!live(c)) return ABS_ESTATE;
+    if (c->n_ranks == 0) return invalid(c, "abs_global_attach has not been called");
+    return abs_global_partition(c->cfg.P, c->n_ranks, c->rank, first, count);
+}
+
+int abs_global_partition(uint64_t P, uint32_t n_ranks, uint32_t rank, uint64_t* first, uint64_t* count) {
+    if (P == 0 || n_ranks == 0 || n_ranks > ABS_MAX_RANKS || rank >= n_ranks) return ABS_EINVAL;
+    unsigned long long lo = 0, hi = 0;
+    slice_vectors(round_up(P, kPadElems), n_ranks, rank, &lo, &hi);
+    const uint64_t e_lo = std::min<uint64_t>(lo * 4, P), e_hi = std::min<uint64_t>(hi * 4, P);
+    if (first) *first = e_lo;
+    if (count) *count = e_hi - e_lo;
+    return ABS_OK;
+}
+
+// CUDA IPC plumbing for abs_global_attach when the ranks are separate processes.
+int abs_ipc_export(const void* dev_ptr, void* handle_out, uint64_t* offset_out) {
+    if (!dev_ptr || !handle_out || !offset_out) return ABS_EINVAL;
+    static_assert(sizeof(cudaIpcMemHandle_t) == ABS_IPC_HANDLE_BYTES, "handle size");
+    typedef CUresult (*GetRange)(CUdeviceptr*, size_t*, CUdeviceptr);
+    void* fn = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuMemGetAddressRange", &fn, cudaEnableDefault, &q) != cudaSuccess || !fn) return ABS_ECUDA;
+    CUdeviceptr base = 0;
+    size_t size = 0;
+    if (reinterpret_cast<GetRange>(fn)(&base, &size, reinterpret_cast<CUdeviceptr>(dev_ptr)) != CUDA_SUCCESS) return ABS_ECUDA;
+    cudaIpcMemHandle_t h;
+    if (cudaIpcGetMemHandle(&h, reinterpret_cast<void*>(base)) != cudaSuccess) { cudaGetLastError(); return ABS_ECUDA; }
+    memcpy(handle_out, &h, sizeof h);
+    *offset_out = reinterpret_cast<CUdeviceptr>(dev_ptr) - base;
+    return ABS_OK;
+}
+
+int abs_ipc_open(const void* handle, uint64_t offset, void** dev_ptr_out) {
+    if (!handle || !dev_ptr_out) return ABS_EINVAL;
+    cudaIpcMemHandle_t h;
+    memcpy(&h, handle, sizeof h);
+    void* base = nullptr;
+    if (cudaIpcOpenMemHandle(&base, h, cudaIpcMemLazyEnablePeerAccess) != cudaSuccess) { cudaGetLastError(); return ABS_ECUDA; }
+    *dev_ptr_out = static_cast<char*>(base) + offset;
+    return ABS_OK;
+}
+
+int abs_ipc_close(void* dev_ptr, uint64_t offset) {
+    if (!dev_ptr) return ABS_EINVAL;
+    if (cudaIpcCloseMemHandle(static_cast<char*>(dev_ptr) - offset) != cudaSuccess) { cudaGetLastError(); return ABS_ECUDA; }
+    return ABS_OK;
+}
+
 int abs_params(abs_ctx* c, const float** x_dev_out) {
     if (!live(c)) return ABS_ESTATE;
     if (!x_dev_out) return invalid(c, "output pointer is NULL");
@@ -596,6 +772,17 @@ int abs_consumed(abs_ctx* c, uint64_t step, int32_t* b_host) {
     if (c->pipelined) CK(cudaStreamSynchronize(c->s_sync));
     CK(cudaStreamSynchronize(c->s_acc));
     CK(cudaMemcpy(b_host, c->log_row(step), c->cfg.W * sizeof(int32_t), cudaMemcpyDeviceToHost));
+    return ABS_OK;
+}
+
+int abs_global_consumed(abs_ctx* c, uint64_t step, int32_t* b_host) {
+    if (!live(c)) return ABS_ESTATE;
+    if (c->n_ranks == 0) return invalid(c, "abs_global_attach has not been called");
+    if (!b_host) return invalid(c, "output pointer is NULL");
+    if (step >= c->t || c->t - step >= (uint64_t)kLogDepth) return invalid(c, "step is not in the logged window");
+    CK(cudaStreamSynchronize(c->s_sync));
+    CK(cudaStreamSynchronize(c->s_acc));
+    CK(cudaMemcpy(b_host, c->log_row(step), (size_t)c->n_ranks * c->cfg.W * sizeof(int32_t), cudaMemcpyDeviceToHost));
     return ABS_OK;
 }
 

@@ -46,6 +46,32 @@ cudaError_t launch_accumulate_multi(float* acc_row, const GradList& gl, int n, u
                                     bool overwrite, int ctas_per_sm, int num_sms, cudaStream_t stream);
 cudaError_t launch_sync(const SyncArgs& a, int ctas_per_sm, int num_sms, cudaStream_t stream);
 
+// ---- Step 1 across GPUs (Algorithm 1, Step 1 as the paper runs it: workers on different GPUs) -----
+// Rank r reduces, updates and redistributes the vectors [vec_lo, vec_hi) of the flat parameter: it reads that
+// slice of every worker row of every rank (its own rows and the peers' rows through peer mappings), applies the
+// same update as k_sync, stores x_{t+1} into every rank's output buffer and clears the slice of every row it read.
+constexpr int kMaxRanks = ABS_MAX_RANKS;
+struct GlobalSyncArgs {
+    const float* x_in;                    // this rank's x_t [P_pad]
+    float* v;                             // this rank's momentum; only [vec_lo, vec_hi) is kept up to date
+    float* acc[kMaxRanks];                // rank q's set being applied, [W_local][row_stride], as mapped here
+    float* x_out[kMaxRanks];              // rank q's buffer for x_{t+1}
+    __nv_bfloat16* shadow[kMaxRanks];     // rank q's bf16 copy of x_{t+1}, or nullptr
+    unsigned long long row_stride;        // elements between worker rows
+    unsigned long long vec_lo, vec_hi;    // this rank's slice, in float4 vectors
+    int G, W_local;
+    const int32_t* cnt_all;               // [G * W_local] b_i of every worker of every rank (exchanged beforehand)
+    int32_t* log_row;                     // [G * W_local] receives the consumed b_i
+    unsigned int* ticket;                 // last-CTA-done ticket, zero on entry and on exit
+    int* applied;                         // in: 1 if the previous step changed x; out: whether this one did
+    float lr, mu, wd, lambda_dc;
+    float disp_scale;                     // rate of the previous step (x_t - x_{t-1} = -disp_scale * v if it applied)
+    int zero_acc;
+};
+cudaError_t launch_sync_global(const GlobalSyncArgs& a, int num_sms, cudaStream_t stream);
+// gcnt[j] = (own_lo <= j < own_lo + W_local) ? cnt[j - own_lo] : 0 for j < n_total;  cnt[0..W_local) = 0.
+cudaError_t launch_global_counts(int32_t* gcnt, int32_t* cnt, int own_lo, int W_local, int n_total, cudaStream_t stream);
+
 // bf16 copy of an fp32 vector (n multiple of 4): used once at init for the MLP weight shadow.
 cudaError_t launch_cast_bf16(const float* src, __nv_bfloat16* dst, size_t n, int num_sms, cudaStream_t stream);
 

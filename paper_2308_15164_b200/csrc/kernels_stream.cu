@@ -228,8 +228,12 @@ __global__ void __launch_bounds__(kBlock) k_accumulate_multi_bf16(float* acc, Gr
 // (b_i = 0) are neither read nor rewritten.  WT > 0 (used for W <= 4): W known at compile time, all
 // loads of a vector are issued before the first add; WT == 0: any W, in chunks of 8 rows.
 // ------------------------------------------------------------------------------------------
+struct UpdateCoef {
+    float lr, mu, wd, lambda_dc;
+    float disp_scale;   // x_t - x_{t-1} = -disp_scale * v   (0 when the previous step was a no-op)
+};
 __device__ __forceinline__ void update_vec(float4& x, float4& v, const float4 s, const float Bf,
-                                           const SyncArgs& a) {
+                                           const UpdateCoef& a) {
     float gx = __fdiv_rn(s.x, Bf), gy = __fdiv_rn(s.y, Bf), gz = __fdiv_rn(s.z, Bf), gw = __fdiv_rn(s.w, Bf);
     if (a.lambda_dc != 0.0f) {   // Eq. 6 with x_t - x_{t-1} = -disp_scale * v
         const float c = -a.lambda_dc * a.disp_scale;
@@ -262,6 +266,7 @@ __global__ void __launch_bounds__(kBlock) k_sync(const SyncArgs a) {
         if (s_cnt[i] > 0) active |= 1ull << i;
     }
     const float Bf = (float)B;
+    const UpdateCoef uc{a.lr, a.mu, a.wd, a.lambda_dc, a.disp_scale};
 
     const float4* xin = reinterpret_cast<const float4*>(a.x_in);
     float4* xout = reinterpret_cast<float4*>(a.x_out);
@@ -296,7 +301,7 @@ __global__ void __launch_bounds__(kBlock) k_sync(const SyncArgs a) {
                             if ((active >> i) & 1) {
                                 s.x += r[u][i].x; s.y += r[u][i].y; s.z += r[u][i].z; s.w += r[u][i].w;
                             }
-                        update_vec(x[u], v[u], s, Bf, a);
+                        update_vec(x[u], v[u], s, Bf, uc);
                         st_stream(xout + idx, x[u]);
                         st_stream(v4 + idx, v[u]);
                         if (a.shadow) store_shadow(a.shadow, idx, x[u]);
@@ -322,7 +327,7 @@ __global__ void __launch_bounds__(kBlock) k_sync(const SyncArgs a) {
                                 if (a.zero_acc) st_stream(acc4 + (i0 + c) * rs + idx, zero);
                             }
                     }
-                    update_vec(x, v, s, Bf, a);
+                    update_vec(x, v, s, Bf, uc);
                     st_stream(xout + idx, x);
                     st_stream(v4 + idx, v);
                     if (a.shadow) store_shadow(a.shadow, idx, x);
@@ -354,6 +359,88 @@ __global__ void __launch_bounds__(kBlock) k_sync(const SyncArgs a) {
             *a.ticket = 0u;
         }
     }
+}
+
+// ------------------------------------------------------------------------------------------
+// Step 1 when the workers live on G GPUs (the paper's setting: "global synchronization" of G_{t-1}^i and
+// M_{t-1}^i between workers).  One kernel per rank does what a reduce-scatter, the update and an all-gather
+// would do as three passes: rank r owns the vectors [vec_lo, vec_hi); for each of them it loads the element of
+// every worker row of every rank (local rows from HBM, the peers' rows through NVLink peer mappings), sums them
+// in global worker order (rank-major, so the result equals the one-GPU kernel on G * W_local rows bit for bit),
+// updates x and its slice of v, stores x_{t+1} into every rank's output buffer and writes zeros over the
+// elements it consumed.  Every accumulator byte crosses HBM once and NVLink at most once; x_{t+1} crosses
+// NVLink once per peer.  No CTA waits for another rank: the caller orders the launches with two stream-ordered
+// collectives (all b_i exchanged before, a barrier after).
+// ------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(kBlock) k_sync_global(const GlobalSyncArgs a) {
+    __shared__ int s_cnt[kMaxW];
+    __shared__ float4* s_row[kMaxW];
+    const int R = a.G * a.W_local;                    // rows in global worker order: j = q * W_local + i
+    if (threadIdx.x < R) {
+        const int q = threadIdx.x / a.W_local, i = threadIdx.x - q * a.W_local;
+        s_cnt[threadIdx.x] = a.cnt_all[threadIdx.x];
+        s_row[threadIdx.x] = reinterpret_cast<float4*>(a.acc[q] + (unsigned long long)i * a.row_stride);
+    }
+    const int applied_before = *a.applied;
+    __syncthreads();
+    long long B = 0;
+    unsigned long long active = 0;
+    for (int j = 0; j < R; ++j) {
+        B += s_cnt[j];
+        if (s_cnt[j] > 0) active |= 1ull << j;
+    }
+    const float Bf = (float)B;
+    const UpdateCoef uc{a.lr, a.mu, a.wd, a.lambda_dc, applied_before ? a.disp_scale : 0.0f};
+    const float4* xin = reinterpret_cast<const float4*>(a.x_in);
+    float4* v4 = reinterpret_cast<float4*>(a.v);
+    const float4 zero = make_float4(0.f, 0.f, 0.f, 0.f);
+
+    for (unsigned long long idx = a.vec_lo + blockIdx.x * (unsigned long long)kBlock + threadIdx.x; idx < a.vec_hi;
+         idx += (unsigned long long)gridDim.x * kBlock) {
+        float4 x = ld_stream(xin + idx);
+        if (B > 0) {
+            float4 v = ld_stream(v4 + idx);
+            float4 s = zero;
+            for (int j0 = 0; j0 < R; j0 += 8) {
+                float4 r[8];
+#pragma unroll
+                for (int c = 0; c < 8; ++c)
+                    if (j0 + c < R && ((active >> (j0 + c)) & 1)) r[c] = ld_stream(s_row[j0 + c] + idx);
+#pragma unroll
+                for (int c = 0; c < 8; ++c)
+                    if (j0 + c < R && ((active >> (j0 + c)) & 1)) {
+                        s.x += r[c].x; s.y += r[c].y; s.z += r[c].z; s.w += r[c].w;
+                        if (a.zero_acc) st_stream(s_row[j0 + c] + idx, zero);
+                    }
+            }
+            update_vec(x, v, s, Bf, uc);
+            st_stream(v4 + idx, v);
+        }
+        // sum_i b_i = 0: x_{t+1} = x_t on every rank, v untouched
+        for (int q = 0; q < a.G; ++q) {
+            st_stream(reinterpret_cast<float4*>(a.x_out[q]) + idx, x);
+            if (a.shadow[q]) store_shadow(a.shadow[q], idx, x);
+        }
+    }
+    __threadfence_system();   // the peers' copies of this slice are complete before the kernel counts as done
+
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        const unsigned int t = atomicAdd(a.ticket, 1u);
+        if (t == gridDim.x - 1) {
+            for (int j = 0; j < R; ++j) a.log_row[j] = s_cnt[j];
+            *a.applied = B > 0 ? 1 : 0;
+            *a.ticket = 0u;
+        }
+    }
+}
+
+__global__ void k_global_counts(int32_t* gcnt, int32_t* cnt, int own_lo, int W_local, int n_total) {
+    const int j = threadIdx.x;
+    if (j >= n_total) return;
+    const bool own = j >= own_lo && j < own_lo + W_local;
+    gcnt[j] = own ? cnt[j - own_lo] : 0;
+    if (own) cnt[j - own_lo] = 0;
 }
 
 __global__ void __launch_bounds__(kBlock) k_cast_bf16(const float4* __restrict__ src, __nv_bfloat16* dst,
@@ -458,6 +545,20 @@ cudaError_t launch_sync(const SyncArgs& a, int ctas_per_sm, int num_sms, cudaStr
         case 3: return launch_sync_t<3, 1>(a, ctas_per_sm, num_sms, stream);
         default: return launch_sync_t<4, 1>(a, ctas_per_sm, num_sms, stream);
     }
+}
+
+cudaError_t launch_sync_global(const GlobalSyncArgs& a, int num_sms, cudaStream_t stream) {
+    // Chunked rows like the one-GPU kernel for W > 4: two CTAs resident per SM, persistent grid of exactly those
+    // (never more CTAs than the slice has tiles).
+    const unsigned long long n = a.vec_hi > a.vec_lo ? a.vec_hi - a.vec_lo : 0;
+    const unsigned grid = grid_for(n, kBlock, 2, num_sms);
+    k_sync_global<<<grid, kBlock, 0, stream>>>(a);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_global_counts(int32_t* gcnt, int32_t* cnt, int own_lo, int W_local, int n_total, cudaStream_t stream) {
+    k_global_counts<<<1, kMaxW, 0, stream>>>(gcnt, cnt, own_lo, W_local, n_total);
+    return cudaGetLastError();
 }
 
 cudaError_t launch_cast_bf16(const float* src, __nv_bfloat16* dst, size_t n, int num_sms, cudaStream_t stream) {

@@ -89,3 +89,36 @@ def test_dead_context_is_rejected(B):
     bogus = ctypes.create_string_buffer(4096)        # not a context the library created
     assert B.lib.abs_sync_step(ctypes.addressof(bogus)) == B.ESTATE
     assert B.lib.abs_launch_count(None) == 0
+
+
+@pytest.mark.parametrize("P", [1, 1023, 1024, 1025, 4096, 11_689_512, 25_557_032, 124_439_808])
+@pytest.mark.parametrize("G", [1, 2, 3, 4, 7, 8, 16])
+def test_multi_gpu_partition_covers_the_vector_once(B, P, G):
+    """Slices of ranks 0..G-1 are consecutive, disjoint, cover [0, P), start on 1024-element boundaries
+    (whole 256-vector tiles) and differ in length by at most one tile, except that trailing ranks take
+    what is left."""
+    at = 0
+    sizes = []
+    for r in range(G):
+        first, count = B.global_partition(P, G, r)
+        assert first == min(at, P) and first % 1024 == 0 or count == 0
+        at = first + count
+        sizes.append(count)
+    assert at == P and sum(sizes) == P
+    full = [s for s in sizes if s and s % 1024 == 0]
+    assert len(set(full)) <= 1 or max(full) == sizes[0]
+    assert sizes == sorted(sizes, reverse=True)
+
+
+def test_multi_gpu_entry_points_reject_bad_arguments_on_the_host(B):
+    assert B.lib.abs_global_partition(0, 2, 0, None, None) == B.EINVAL
+    assert B.lib.abs_global_partition(16, 0, 0, None, None) == B.EINVAL
+    assert B.lib.abs_global_partition(16, 17, 0, None, None) == B.EINVAL
+    assert B.lib.abs_global_partition(16, 2, 2, None, None) == B.EINVAL
+    for name in ("abs_global_step", "abs_global_end"):
+        assert getattr(B.lib, name)(None) == B.ESTATE
+    assert B.lib.abs_global_attach(None, None) == B.ESTATE
+    assert B.lib.abs_global_begin(None, None, None) == B.ESTATE
+    assert B.lib.abs_ipc_export(None, None, None) == B.EINVAL
+    assert B.lib.abs_ipc_open(None, 0, None) == B.EINVAL
+    assert B.lib.abs_ipc_close(None, 0) == B.EINVAL
