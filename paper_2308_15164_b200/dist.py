@@ -24,12 +24,17 @@ def rank_info() -> Tuple[int, int, int]:
             int(os.environ.get("WORLD_SIZE", "1")))
 
 
-def init(backend: str) -> Tuple[int, int, int]:
+def init(backend: str, timeout_s: float = 0.0) -> Tuple[int, int, int]:
+    """Joins the process group named by the torchrun environment.  timeout_s > 0 bounds every collective of a
+    host-side backend (a rank that never arrives then ends the others with an error instead of a hang)."""
     rank, local_rank, world = rank_info()
     if world > 1 and not dist.is_initialized():
+        import datetime
+
         os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
         os.environ.setdefault("MASTER_PORT", "29511")
-        dist.init_process_group(backend=backend, rank=rank, world_size=world)
+        kw = dict(timeout=datetime.timedelta(seconds=timeout_s)) if timeout_s > 0 else {}
+        dist.init_process_group(backend=backend, rank=rank, world_size=world, **kw)
     return rank, local_rank, world
 
 
