@@ -336,6 +336,8 @@ def run_ours(args):
             line["workloads_3_and_5"] = run_other_workloads(B, wlm, dev)
         if "sync_curve" in sections:
             line["sync_curve"] = run_sync_curve(B, dev, peaks)
+        if "global" in sections:
+            line["global_sync_emulated_ranks"] = run_global_sync(B, dev, peaks)
         if "batch_curve" in sections:
             line["accumulate_batch_curve"] = run_batch_curve(B, dev, peaks)
         print(json.dumps(line), flush=True)
@@ -423,6 +425,47 @@ def run_sync_curve(B, dev, peaks, P=11_689_512):
             eng.profile(False)
         out[str(W)] = {"us": ms / n * 1e3, "gbs": (8 * W + 16) * P / (ms / n) / 1e6}
         eng.check(); eng.destroy()
+    return out
+
+
+def run_global_sync(B, dev, peaks):
+    """Step 1 across GPUs (abs_global_*), G ranks emulated in one process on this one GPU (dist.LocalRanks).  The
+    G fused kernels of an iteration run side by side (as they would on G GPUs) but here share one HBM, so the
+    figure is all ranks' bytes over the time from the first kernel's start to the last one's end (an event pair
+    on the control stream).  Bytes per parameter, R = G * W_local rows: read R rows + x + v, write R zero rows +
+    v + x into G buffers = 8 R + 12 + 4 G.  Every one of them is local HBM traffic here; between real GPUs
+    (G - 1) / G of the row and x traffic crosses NVLink instead, so this is the kernel's streaming rate on one
+    GPU, not a multi-GPU measurement."""
+    import torch
+
+    from paper_2308_15164_b200 import dist as D
+
+    out = {"unit": "GB/s on (8*R + 12 + 4*G) * P bytes per iteration, all ranks on one GPU", "peak": peaks["hbm_gbs"]}
+    gen = torch.Generator(device=dev).manual_seed(3)
+    for name, P, G, Wl in (("resnet18_4_ranks_x_1_worker", 11_689_512, 4, 1), ("resnet50_4_ranks_x_2_workers", 25_557_032, 4, 2),
+                           ("resnet50_8_ranks_x_1_worker", 25_557_032, 8, 1)):
+        g = torch.randn(P + 8, device=dev, generator=gen)
+        x0 = torch.zeros(P, device=dev)
+        ranks = [B.AbsSgd(x0, Wl, 0.1, 0.9, 5e-4, pipelined=True) for _ in range(G)]
+        grp = D.LocalRanks(ranks)
+        evs = []
+        for it in range(13):
+            for e in ranks:
+                for i in range(Wl):
+                    e.accumulate(i, g)
+            ev = grp.sync_step(timed=True)
+            if it >= 3:                                 # the first rounds warm up
+                evs.append(ev)
+        torch.cuda.synchronize()
+        ms = sum(a.elapsed_time(b) for a, b in evs) / len(evs)
+        R = G * Wl
+        nbytes = (8 * R + 12 + 4 * G) * P
+        out[name] = {"P": P, "ranks": G, "workers_per_rank": Wl, "us_all_ranks": ms * 1e3,
+                     "gbs": nbytes / ms / 1e6, "frac_of_measured_hbm": nbytes / ms / 1e6 / peaks["hbm_gbs"]}
+        for e in ranks:
+            e.check(); e.destroy()
+        del ranks, grp, g, x0
+        torch.cuda.empty_cache()
     return out
 
 
@@ -718,7 +761,7 @@ def main():
     ap.add_argument("--steps", type=int, default=1000)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--sections", default="e2e,cpu,mlp,tiny,batch_curve,sync_curve",
+    ap.add_argument("--sections", default="e2e,cpu,mlp,tiny,batch_curve,sync_curve,global",
                     help="extra measurements after the timed region (drop them for a profiler's launch list)")
     args = ap.parse_args()
     if args.warmup < 3:

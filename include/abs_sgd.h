@@ -9,6 +9,7 @@
  *     learning rate gamma  = lr         compensation lambda = lambda_dc
  * The W workers of the paper are W gradient buffers in this GPU's memory, so the "global
  * synchronization" of Step 1 is an in-device weighted reduction; no collective is involved.
+ * (Workers spread over several GPUs: the abs_global_* calls further down.)
  *
  * One iteration t (Algorithm 1, body of the while loop):
  *     abs_accumulate*(worker i, ...)   any number of times per worker, in any order

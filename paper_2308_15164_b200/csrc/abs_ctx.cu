@@ -652,7 +652,7 @@ int abs_global_step(abs_ctx* c) {
     a.zero_acc = (c->cfg.flags & ABS_FLAG_OVERWRITE_FIRST) ? 0 : 1;
     {
         Timed tm(c, ABS_K_SYNC, c->s_sync);
-        CK(launch_sync_global(a, c->num_sms, c->s_sync));
+        CK(launch_sync_global(a, c->ctas_per_sm[ABS_K_SYNC], c->num_sms, c->s_sync));
     }
     c->launches += 1;
     c->global_prev_lr = c->lr_now;

@@ -68,7 +68,7 @@ struct GlobalSyncArgs {
     float disp_scale;                     // rate of the previous step (x_t - x_{t-1} = -disp_scale * v if it applied)
     int zero_acc;
 };
-cudaError_t launch_sync_global(const GlobalSyncArgs& a, int num_sms, cudaStream_t stream);
+cudaError_t launch_sync_global(const GlobalSyncArgs& a, int ctas_per_sm, int num_sms, cudaStream_t stream);
 // gcnt[j] = (own_lo <= j < own_lo + W_local) ? cnt[j - own_lo] : 0 for j < n_total;  cnt[0..W_local) = 0.
 cudaError_t launch_global_counts(int32_t* gcnt, int32_t* cnt, int own_lo, int W_local, int n_total, cudaStream_t stream);
 

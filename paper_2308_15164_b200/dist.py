@@ -177,17 +177,26 @@ class LocalRanks:
         for e in self.engines:
             e.stream_sync.wait_stream(self.ctrl)
 
-    def sync_step(self):
+    def sync_step(self, timed: bool = False):
+        """One end of iteration on all ranks.  timed=True returns a CUDA event pair on the control stream that
+        brackets the G fused kernels (which run side by side on this one GPU)."""
         counts = [e.global_begin() for e in self.engines]
         self._join()
         with torch.cuda.stream(self.ctrl):                    # exchange A
             total = torch.stack(counts).sum(dim=0, dtype=torch.int32)
             for c in counts:
                 c.copy_(total)
+        ev = None
+        if timed:
+            ev = (torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True))
+            ev[0].record(self.ctrl)
         self._fork()
         for e in self.engines:
             e.global_step()
         self._join()                                          # exchange B
+        if timed:
+            ev[1].record(self.ctrl)
         self._fork()
         for e in self.engines:
             e.global_end()
+        return ev
