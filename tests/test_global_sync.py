@@ -225,3 +225,63 @@ def test_call_order_and_mode_errors():
     for e in [a, b] + big:
         e.check()
         e.destroy()
+
+
+def test_mlp_gradients_computed_on_two_ranks_match_one_context_and_oracle():
+    """Workload 4 (small layer sizes): every rank computes its workers' MLP gradients at x_t (single and batch
+    calls) -- the fused kernel must also refresh every rank's bf16 copy of the weights, which the next forward
+    pass reads."""
+    import torch
+
+    from oracle.abs_oracle import AbsSgdOracle, mlp_loss_and_grad
+    from paper_2308_15164_b200 import binding as B
+    from paper_2308_15164_b200 import dist as D
+
+    G, T = 2, 8
+    wl = wlm.config(4, small=True, T=T)
+    d = wl.mlp
+    Wl = wl.W // G
+    x0 = wlm.params0(wl)
+    xs, ys = wlm.mlp_batches(wl)
+    sched = wlm.schedule(wl).copy()
+    sched[2, 1] = 0                                   # an idle worker
+    dev = torch.device("cuda:0")
+    xs_d, ys_d = torch.from_numpy(xs).to(dev), torch.from_numpy(ys).to(dev)
+    x0_d = torch.from_numpy(x0).to(dev)
+    torch.cuda.synchronize()
+    mlp = (d.d_in, d.d_hidden, d.d_out, d.mb)
+    one = B.AbsSgd(x0_d, wl.W, wl.lr, wl.momentum, wl.weight_decay, pipelined=True, mlp=mlp)
+    ranks = [B.AbsSgd(x0_d, Wl, wl.lr, wl.momentum, wl.weight_decay, pipelined=True, mlp=mlp) for _ in range(G)]
+    grp = D.LocalRanks(ranks)
+    ref = AbsSgdOracle(x0, wl.W, wl.lr, wl.momentum, wl.weight_decay)
+    for t, b_row in enumerate(sched):
+        p = ref.params()
+        for i, b in enumerate(b_row):                 # worker by worker: up to 2 reference batches per call
+            lo = (7 * t + 3 * i) % (wl.mlp_pool - 8)
+            k = 0
+            while k < int(b):
+                n = min(2, int(b) - k)
+                for j in range(n):
+                    _, g, _ = mlp_loss_and_grad(p, xs[lo + k + j], ys[lo + k + j], d.d_in, d.d_hidden, d.d_out, mode="bf16")
+                    ref.accumulate(i, g.astype(np.float32))
+                for eng, w in ((one, i), (ranks[i // Wl], i % Wl)):
+                    if n == 1:
+                        eng.accumulate_mlp(w, xs_d[lo + k], ys_d[lo + k])
+                    else:
+                        eng.accumulate_mlp_batch(w, n, xs_d[lo + k:lo + k + n], ys_d[lo + k:lo + k + n])
+                k += n
+        ref.sync_step()
+        one.sync_step()
+        grp.sync_step()
+        got_one = one.params_host()
+        for r, e in enumerate(ranks):
+            assert np.array_equal(e.params_host(), got_one), f"x_{t + 1} on rank {r}"
+    want = ref.params()
+    assert np.abs(want - x0).max() > 1e-4
+    assert np.abs(got_one.astype(np.float64) - want).max() <= H.TOL_BF16 * np.abs(want).max()
+    for r, e in enumerate(ranks):
+        for s in range(T):
+            assert np.array_equal(e.global_consumed(s), np.asarray(ref.consumed[s]))
+    for e in [one] + ranks:
+        e.check()
+        e.destroy()
