@@ -3,6 +3,7 @@
     python -m paper_2308_15164_b200.profile_case sync       [--P 11689512] [--W 4] [--iters 3]
     python -m paper_2308_15164_b200.profile_case accumulate [--P 11689512] [--W 4] [--iters 3] [--bf16]
     python -m paper_2308_15164_b200.profile_case mlp        [--iters 2] [--batch 4] [--calls 2]
+    python -m paper_2308_15164_b200.profile_case global     [--P 25557032] [--ranks 4] [--W 2] [--iters 2]
 
 Each case keeps its working set larger than the 126 MB L2 but to a few hundred MB, launches the
 kernel of interest a handful of times and exits, so that a multi-pass capture ends by itself.
@@ -20,7 +21,7 @@ import torch
 
 def main(argv=None):
     ap = argparse.ArgumentParser()
-    ap.add_argument("case", choices=["sync", "accumulate", "mlp"])
+    ap.add_argument("case", choices=["sync", "accumulate", "mlp", "global"])
     ap.add_argument("--P", type=int, default=11_689_512)
     ap.add_argument("--W", type=int, default=4)
     ap.add_argument("--iters", type=int, default=3)
@@ -28,6 +29,7 @@ def main(argv=None):
     ap.add_argument("--pipelined", action="store_true")
     ap.add_argument("--epilogue", type=int, default=0)
     ap.add_argument("--batch", type=int, default=1, help="mlp: reference batches per call (1..4)")
+    ap.add_argument("--ranks", type=int, default=4, help="global: ranks emulated in this process (W = workers per rank)")
     ap.add_argument("--calls", type=int, default=1, help="mlp: calls per worker and iteration (the first one stores)")
     args = ap.parse_args(argv)
 
@@ -36,7 +38,23 @@ def main(argv=None):
 
     dev = torch.device("cuda:0")
     torch.cuda.set_device(dev)
-    if args.case in ("sync", "accumulate"):
+    if args.case == "global":
+        from . import dist as D
+
+        g = torch.Generator(device="cpu").manual_seed(0)
+        x0 = (torch.randn(args.P, generator=g) * 0.02).to(dev)
+        grad = torch.randn((args.P + 7) // 8 * 8, generator=g).to(dev)
+        ranks = [B.AbsSgd(x0, args.W, 0.1, 0.9, 5e-4, pipelined=True) for _ in range(args.ranks)]
+        grp = D.LocalRanks(ranks)
+        for _ in range(args.iters):
+            for e in ranks:
+                for i in range(args.W):
+                    e.accumulate(i, grad)
+            grp.sync_step()
+        for e in ranks:
+            e.check()
+            e.destroy()
+    elif args.case in ("sync", "accumulate"):
         g = torch.Generator(device="cpu").manual_seed(0)
         x0 = (torch.randn(args.P, generator=g) * 0.02).to(dev)
         pool = torch.randn((4, (args.P + 7) // 8 * 8), generator=g)
