@@ -596,11 +596,13 @@ def run_mlp(B, wlm, dev, peaks, iters=12):
     rmw_bytes = 8.0 * d.d_in * d.d_hidden + 2.0 * d.mb * (d.d_in + d.d_hidden)
     out = {"workload": "cfg4 mlp 3072-4096-10, mb=64, W=4, b_i~U{1..8}, pipelined", "iterations": iters,
            "dw1_flop": flop, "dw1_algorithmic_bytes": rmw_bytes}
-    for name, variant in (("auto", 0), ("tma_load_add_store", 16), ("tma_reduce_add", 1), ("persistent_ring", 4), ("register_prefetch", 8), ("cluster_fused_forward", 64)):
+    for name, variant, coalesce in (("auto", 0, False), ("single_calls_gathered_by_the_library", 0, True), ("tma_load_add_store", 16, False),
+                                    ("tma_reduce_add", 1, False), ("persistent_ring", 4, False), ("register_prefetch", 8, False),
+                                    ("cluster_fused_forward", 64, False)):
         res = {}
-        for serial in (0, 1):
+        for serial in ((0,) if coalesce else (0, 1)):      # (serial mode runs every call at once: nothing to gather)
             eng = B.AbsSgd(x0_d, wl.W, wl.lr, wl.momentum, wl.weight_decay, pipelined=True,
-                           mlp=(d.d_in, d.d_hidden, d.d_out, d.mb))
+                           mlp=(d.d_in, d.d_hidden, d.d_out, d.mb), mlp_coalesce=coalesce)
             eng.set_launch(B.K_MLP_DW1, variant)
             eng.set_launch(B.K_MLP_FWD, serial)
 

@@ -72,6 +72,21 @@ extern "C" {
                                        first gradient of an iteration in either mode (the row is then known
                                        to be empty), which saves the read of the W1 slice.                    */
 
+#define ABS_FLAG_MLP_COALESCE 16u /* with ABS_FLAG_MLP: single abs_accumulate_mlp calls of a worker are gathered, up to
+                                       four, and run as ONE batch (exactly what abs_accumulate_mlp_batch does with
+                                       the same micro-batches: one forward GEMM over the stacked samples, one dW1
+                                       GEMM with K = 64 n whose epilogue touches the accumulator slice once).  The
+                                       call still reads x_dev / y_dev right away (its cast kernel is enqueued on
+                                       stream_acc before it returns) and counts b_i right away; the rest of the
+                                       gradient is enqueued when the group is full or when anything needs it:
+                                       abs_sync_step / abs_global_begin (every micro-batch of iteration t is
+                                       evaluated at x_t and lands in iteration t's accumulator), another kind of
+                                       accumulate call for that worker, abs_wait, abs_check, abs_accumulator,
+                                       abs_set_launch.  Results equal those of explicit batch calls over the same
+                                       groups bit for bit, and those of ungrouped single calls to fp32 rounding.
+                                       At most four groups wait at a time (the oldest is started when a fifth
+                                       worker opens one).                                                       */
+
 #define ABS_MAX_WORKERS 64u
 #define ABS_MAX_RANKS   16u   /* GPUs taking part in abs_global_* (n_ranks * W <= ABS_MAX_WORKERS)        */
 #define ABS_IPC_HANDLE_BYTES 64

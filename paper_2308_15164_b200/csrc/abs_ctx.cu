@@ -39,7 +39,9 @@ bool config_ok(const abs_config* c, std::string* why) {
     if (c->P == 0) return fail("P must be > 0");
     if (c->W == 0 || c->W > ABS_MAX_WORKERS) return fail("W must be in 1..64");
     if (c->grad_dtype != ABS_GRAD_F32 && c->grad_dtype != ABS_GRAD_BF16) return fail("unknown grad_dtype");
-    if (c->flags & ~(ABS_FLAG_PIPELINED | ABS_FLAG_MLP | ABS_FLAG_HOST_INPUT | ABS_FLAG_OVERWRITE_FIRST)) return fail("unknown flag bits");
+    if (c->flags & ~(ABS_FLAG_PIPELINED | ABS_FLAG_MLP | ABS_FLAG_HOST_INPUT | ABS_FLAG_OVERWRITE_FIRST | ABS_FLAG_MLP_COALESCE))
+        return fail("unknown flag bits");
+    if ((c->flags & ABS_FLAG_MLP_COALESCE) && !(c->flags & ABS_FLAG_MLP)) return fail("ABS_FLAG_MLP_COALESCE needs ABS_FLAG_MLP");
     if (!std::isfinite(c->lr) || !std::isfinite(c->momentum) || !std::isfinite(c->weight_decay) ||
         !std::isfinite(c->lambda_dc))
         return fail("lr, momentum, weight_decay and lambda_dc must be finite");
@@ -140,6 +142,16 @@ struct abs_ctx {
     bool set_used[kMlpSets] = {};
     bool w_outstanding[kMlpStreams] = {};          // enqueued since stream_acc last waited for that stream
     int mlp_set_next = 0;
+    // ABS_FLAG_MLP_COALESCE: single calls of a worker wait, already cast into consecutive slots of one scratch
+    // set, until four have gathered (or something needs the accumulator), then run as one batch call.
+    bool coalesce = false;
+    int pend_n[kMaxW] = {};        // micro-batches of worker i waiting (0..kMlpMaxBatch)
+    int pend_set[kMaxW] = {};      // scratch set that holds them
+    bool pend_first[kMaxW] = {};   // they open the worker's iteration (the row holds nothing yet)
+    bool set_reserved[kMlpSets] = {};
+    int n_reserved = 0;
+    uint64_t pend_age[kMaxW] = {}; // order in which the pending groups were opened
+    uint64_t pend_clock = 0;
     std::vector<TmapBytes> acc_tmaps;   // [2][W]: TMA descriptor of each accumulator row's W1 slice
 
     // multi-GPU mode (abs_global_*): every rank's workspace as mapped in this process
@@ -242,8 +254,13 @@ int collect_timings(abs_ctx* c) {
 
 void mlp_mark(void* user, int kernel_class, int n, cudaStream_t stream);
 
-// stream_acc waits (on the device) for every gradient kernel enqueued so far on the worker streams.
+int flush_all(abs_ctx* c);
+int flush_worker(abs_ctx* c, uint32_t worker);
+
+// stream_acc waits (on the device) for every gradient kernel enqueued so far on the worker streams (waiting
+// micro-batch groups are started first).
 int join_workers(abs_ctx* c) {
+    if (int rc = flush_all(c)) return rc;
     for (int k = 0; k < c->n_wstreams; ++k)
         if (c->w_outstanding[k]) {
             CK(cudaStreamWaitEvent(c->s_acc, c->ev_w_done[k], 0));
@@ -277,6 +294,95 @@ int launch_fused(abs_ctx* c, uint32_t set, int in, int out, uint64_t log_step, c
         CK(launch_sync(a, c->ctas_per_sm[ABS_K_SYNC], c->num_sms, stream));
     }
     c->launches += 1;
+    return ABS_OK;
+}
+
+// Next scratch set that no pending group holds; stream_acc waits (on the device) for its previous user.
+int take_scratch_set(abs_ctx* c, bool serial, int* out) {
+    int set = c->mlp_set_next;
+    for (int tries = 0; tries < kMlpSets && c->set_reserved[set]; ++tries) set = (set + 1) % kMlpSets;
+    c->mlp_set_next = (set + 1) % kMlpSets;
+    if (!serial && c->set_used[set]) CK(cudaStreamWaitEvent(c->s_acc, c->ev_set_done[set], 0));
+    *out = set;
+    return ABS_OK;
+}
+
+// Forward, loss, backward and dW1 of the n micro-batches that sit, cast, in slots 0..n-1 of scratch set `set`,
+// on the worker's internal stream (which first waits for everything enqueued on stream_acc so far, the casts
+// included).  deferred: the casts were launched, and counted, by earlier calls.
+int run_mlp_group(abs_ctx* c, uint32_t worker, int set, int n, bool first, bool deferred) {
+    const int k = (int)(worker % (uint32_t)c->n_wstreams);
+    const int variant = c->ctas_per_sm[ABS_K_MLP_DW1];
+    const bool serial = c->ctas_per_sm[ABS_K_MLP_FWD] == 1;
+    const MlpScratch& sc = c->mlp_scratch[set];
+    cudaStream_t s_run = serial ? c->s_acc : c->s_w[k];
+    if (!serial) {
+        CK(cudaEventRecord(c->ev_fork, c->s_acc));
+        CK(cudaStreamWaitEvent(s_run, c->ev_fork, 0));
+    }
+    if (deferred) mlp_mark(c, ABS_K_MLP_FWD, 0, s_run);
+    CK(launch_mlp_front(c->mlp_dims, sc, c->x(c->pub), c->shadow(c->pub), c->pub, n, first, c->acc(c->cur, worker),
+                        c->cnt(c->cur, worker), variant, s_run, mlp_mark, c));
+    if (deferred) c->launches -= 1;   // launch_mlp_front counts one cast with its group
+    CK(launch_mlp_dw1(c->mlp_dims, sc, c->acc(c->cur, worker), &c->acc_tmaps[(size_t)c->cur * c->cfg.W + worker], n,
+                      first, variant, s_run, mlp_mark, c));
+    if (serial) {
+        for (bool& u : c->set_used) u = false;
+    } else {
+        CK(cudaEventRecord(c->ev_set_done[set], s_run));
+        CK(cudaEventRecord(c->ev_w_done[k], s_run));
+        c->set_used[set] = true;
+        c->w_outstanding[k] = true;
+    }
+    return ABS_OK;
+}
+
+// Runs the worker's waiting micro-batches (ABS_FLAG_MLP_COALESCE) as one group.
+int flush_worker(abs_ctx* c, uint32_t worker) {
+    const int n = c->pend_n[worker];
+    if (n == 0) return ABS_OK;
+    const int set = c->pend_set[worker];
+    c->pend_n[worker] = 0;
+    c->set_reserved[set] = false;
+    c->n_reserved -= 1;
+    return run_mlp_group(c, worker, set, n, c->pend_first[worker], true);
+}
+
+int flush_all(abs_ctx* c) {
+    if (c->n_reserved == 0) return ABS_OK;
+    for (;;) {   // oldest group first: the order does not change results (rows are independent), only timing
+        int best = -1;
+        for (uint32_t i = 0; i < c->cfg.W; ++i)
+            if (c->pend_n[i] && (best < 0 || c->pend_age[i] < c->pend_age[best])) best = (int)i;
+        if (best < 0) return ABS_OK;
+        if (int rc = flush_worker(c, (uint32_t)best)) return rc;
+    }
+}
+
+// One micro-batch of `worker` joins its waiting group: cast now (the caller's buffers are free again once
+// stream_acc has passed this point), everything else when the group runs.
+int coalesce_one(abs_ctx* c, uint32_t worker, const float* x_dev, const int32_t* y_dev) {
+    if (c->pend_n[worker] == 0) {
+        if (c->n_reserved >= kMlpSets / 2) {   // keep half of the scratch sets for groups that are running
+            int oldest = -1;
+            for (uint32_t i = 0; i < c->cfg.W; ++i)
+                if (c->pend_n[i] && (oldest < 0 || c->pend_age[i] < c->pend_age[oldest])) oldest = (int)i;
+            if (int rc = flush_worker(c, (uint32_t)oldest)) return rc;
+        }
+        int set = 0;
+        if (int rc = take_scratch_set(c, false, &set)) return rc;
+        c->set_reserved[set] = true;
+        c->n_reserved += 1;
+        c->pend_set[worker] = set;
+        c->pend_first[worker] = c->h_cnt[(size_t)c->cur * c->cfg.W + worker] == 0;
+        c->pend_age[worker] = ++c->pend_clock;
+    }
+    const int slot = c->pend_n[worker];
+    CK(launch_mlp_cast(c->mlp_dims, c->mlp_scratch[c->pend_set[worker]], slot, 1, x_dev, y_dev, c->s_acc, mlp_mark, c));
+    mlp_mark(c, ABS_K_MLP_FWD, 1, c->s_acc);
+    c->pend_n[worker] = slot + 1;
+    c->h_cnt[(size_t)c->cur * c->cfg.W + worker] += 1;
+    if (c->pend_n[worker] == kMlpMaxBatch) return flush_worker(c, worker);
     return ABS_OK;
 }
 
@@ -315,6 +421,7 @@ int abs_init(abs_ctx** out, const abs_config* cfg, void* workspace_dev, size_t w
     c->s_sync = static_cast<cudaStream_t>(cfg->stream_sync);
     c->pipelined = cfg->flags & ABS_FLAG_PIPELINED;
     c->mlp = cfg->flags & ABS_FLAG_MLP;
+    c->coalesce = cfg->flags & ABS_FLAG_MLP_COALESCE;
     c->h_cnt.assign((size_t)2 * cfg->W, 0);
     c->lr_now = cfg->lr;
     c->lr_prev_call = cfg->lr;
@@ -466,42 +573,23 @@ int abs_accumulate_mlp_batch(abs_ctx* c, uint32_t worker, uint32_t n, const floa
     if (n == 0 || n > (uint32_t)kMlpMaxBatch) return invalid(c, "n must be in 1..4");
     if (!x_dev || (reinterpret_cast<uintptr_t>(x_dev) & 15)) return invalid(c, "x pointer must be non-NULL and 16-byte aligned");
     if (!y_dev || (reinterpret_cast<uintptr_t>(y_dev) & 3)) return invalid(c, "y pointer must be non-NULL and 4-byte aligned");
+    const bool serial = c->ctas_per_sm[ABS_K_MLP_FWD] == 1;   // measurement aid: everything on stream_acc
+    if (c->coalesce && n == 1 && !serial) return coalesce_one(c, worker, x_dev, y_dev);
+    if (int rc = flush_worker(c, worker)) return rc;           // the worker's row is added to in call order
     // Only the cast kernel reads the caller's buffers; it runs on stream_acc, in call order.  The rest of the
     // call (forward, loss, backward, dW1) runs on the worker's internal stream, so that the latency chains of
     // different workers overlap and the HBM-bound dW1 GEMMs fill the gaps of the small kernels.
-    const int set = c->mlp_set_next;
-    c->mlp_set_next = (set + 1) % kMlpSets;
-    const int k = (int)(worker % (uint32_t)c->n_wstreams);
-    const int variant = c->ctas_per_sm[ABS_K_MLP_DW1];
-    const bool serial = c->ctas_per_sm[ABS_K_MLP_FWD] == 1;   // measurement aid: everything on stream_acc
     if (serial) {
         if (int rc = join_workers(c)) return rc;
-    } else if (c->set_used[set]) {
-        CK(cudaStreamWaitEvent(c->s_acc, c->ev_set_done[set], 0));   // the scratch set is free again
     }
-    const MlpScratch& sc = c->mlp_scratch[set];
+    int set = 0;
+    if (int rc = take_scratch_set(c, serial, &set)) return rc;
     // A worker's first gradient of an iteration finds its accumulator row empty (all zero, or -- with
     // ABS_FLAG_OVERWRITE_FIRST -- stale): it is stored, not added, and dW1 skips reading the 4 d_in d_hidden
     // bytes of the slice.  0 + g = g, so the default mode's results do not change.
     const bool first = c->h_cnt[(size_t)c->cur * c->cfg.W + worker] == 0;
-    CK(launch_mlp_cast(c->mlp_dims, sc, (int)n, x_dev, y_dev, c->s_acc, mlp_mark, c));
-    cudaStream_t s_run = serial ? c->s_acc : c->s_w[k];
-    if (!serial) {
-        CK(cudaEventRecord(c->ev_fork, c->s_acc));
-        CK(cudaStreamWaitEvent(s_run, c->ev_fork, 0));
-    }
-    CK(launch_mlp_front(c->mlp_dims, sc, c->x(c->pub), c->shadow(c->pub), c->pub, (int)n, first, c->acc(c->cur, worker),
-                        c->cnt(c->cur, worker), variant, s_run, mlp_mark, c));
-    CK(launch_mlp_dw1(c->mlp_dims, sc, c->acc(c->cur, worker), &c->acc_tmaps[(size_t)c->cur * c->cfg.W + worker], (int)n,
-                      first, variant, s_run, mlp_mark, c));
-    if (serial) {
-        for (bool& u : c->set_used) u = false;
-    } else {
-        CK(cudaEventRecord(c->ev_set_done[set], s_run));
-        CK(cudaEventRecord(c->ev_w_done[k], s_run));
-        c->set_used[set] = true;
-        c->w_outstanding[k] = true;
-    }
+    CK(launch_mlp_cast(c->mlp_dims, c->mlp_scratch[set], 0, (int)n, x_dev, y_dev, c->s_acc, mlp_mark, c));
+    if (int rc = run_mlp_group(c, worker, set, (int)n, first, false)) return rc;
     c->h_cnt[(size_t)c->cur * c->cfg.W + worker] += (int32_t)n;
     return ABS_OK;
 }
@@ -513,6 +601,7 @@ int abs_accumulate_mlp(abs_ctx* c, uint32_t worker, const float* x_dev, const in
 int abs_sync_step(abs_ctx* c) {
     if (!live(c)) return ABS_ESTATE;
     if (c->n_ranks != 0) return invalid(c, "context is in multi-GPU mode: end iterations with abs_global_begin / _step / _end");
+    if (int rc = flush_all(c)) return rc;   // every gradient of iteration t is under way before the iteration ends
     const uint32_t W = c->cfg.W;
     const uint32_t d = c->cur ^ 1;   // the delayed set (filled during iteration t-1)
     if (!c->pipelined) {
@@ -599,6 +688,7 @@ int abs_global_begin(abs_ctx* c, int32_t** counts_dev, uint32_t* n_counts) {
     if (c->n_ranks == 0) return invalid(c, "abs_global_attach has not been called");
     if (c->global_phase != 0) return invalid(c, "abs_global_begin / _step / _end must be called in that order");
     if (!counts_dev || !n_counts) return invalid(c, "output pointer is NULL");
+    if (int rc = flush_all(c)) return rc;
     const uint32_t W = c->cfg.W;
     // Publish x_{t+1}: the kernels launched one call ago, on every rank, have all finished (ev_sync_done was
     // recorded behind the caller's closing barrier).
@@ -817,6 +907,7 @@ int abs_wait(abs_ctx* c) {
 
 int abs_check(abs_ctx* c) {
     if (!live(c)) return ABS_ESTATE;
+    if (int rc = flush_all(c)) return rc;
     if (c->pipelined) CK(cudaStreamSynchronize(c->s_sync));
     for (int k = 0; k < c->n_wstreams; ++k) CK(cudaStreamSynchronize(c->s_w[k]));
     CK(cudaStreamSynchronize(c->s_acc));
@@ -839,6 +930,7 @@ int abs_set_launch(abs_ctx* c, int kernel_class, int ctas_per_sm) {
     if (!live(c)) return ABS_ESTATE;
     if (kernel_class < 0 || kernel_class >= ABS_K_COUNT || ctas_per_sm < -1 || ctas_per_sm > 64)
         return invalid(c, "bad kernel class or CTA count");
+    if (int rc = flush_all(c)) return rc;
     c->ctas_per_sm[kernel_class] = ctas_per_sm;
     return ABS_OK;
 }

@@ -120,7 +120,7 @@ cudaError_t mlp_make_acc_tmap(void* tmap_out, const MlpDims& d, float* acc_row);
 // mark(user, kernel_class, 0, stream) is called before a kernel group, mark(user, kernel_class, n, stream) after
 // its n launches.
 typedef void (*MlpMark)(void* user, int kernel_class, int n, cudaStream_t stream);
-cudaError_t launch_mlp_cast(const MlpDims& d, const MlpScratch& s, int nb, const float* x_dev, const int32_t* y_dev,
+cudaError_t launch_mlp_cast(const MlpDims& d, const MlpScratch& s, int slot0, int nb, const float* x_dev, const int32_t* y_dev,
                             cudaStream_t stream, MlpMark mark, void* user);
 cudaError_t launch_mlp_front(const MlpDims& d, const MlpScratch& s, const float* x_pub, const __nv_bfloat16* shadow,
                              int shadow_idx, int nb, bool store, float* acc_row, int32_t* cnt, int variant,

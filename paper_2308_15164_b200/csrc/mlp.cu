@@ -1389,10 +1389,12 @@ cudaError_t mlp_make_acc_tmap(void* tmap_out, const MlpDims& d, float* acc_row) 
                : cudaErrorInvalidValue;
 }
 
-cudaError_t launch_mlp_cast(const MlpDims& d, const MlpScratch& s, int nb, const float* x_dev, const int32_t* y_dev,
+cudaError_t launch_mlp_cast(const MlpDims& d, const MlpScratch& s, int slot0, int nb, const float* x_dev, const int32_t* y_dev,
                             cudaStream_t stream, MlpMark mark, void* user) {
     mark(user, ABS_K_MLP_FWD, 0, stream);
-    k_cast_x<<<dim3(d.d_in / 16, nb), 256, 0, stream>>>(x_dev, y_dev, s.xb, s.xtb, s.ycopy, d.d_in);
+    // micro-batch j of the call goes to slot slot0 + j of the scratch set
+    k_cast_x<<<dim3(d.d_in / 16, nb), 256, 0, stream>>>(x_dev, y_dev, s.xb + (size_t)slot0 * kMB * d.d_in,
+                                                        s.xtb + (size_t)slot0 * d.d_in * kMB, s.ycopy + slot0 * kMB, d.d_in);
     return cudaGetLastError();
 }
 
