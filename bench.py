@@ -280,7 +280,7 @@ def run_ours(args):
     # DRAM bytes (read + write) of ONE launch of each kernel at this workload's size, from an ncu capture of the
     # current kernels (profiles/k_accumulate_resnet18_and_bf16.md, profiles/k_sync_w4_resnet18.md): a lone launch
     # under the profiler, whose reads equal the algorithmic reads and whose writes partly stay in the 126 MB L2.
-    NCU_TRAFFIC = {"k_accumulate_f32": 93_521_408 + 2_586_112, "k_sync<4>": 280_564_224 + 217_552_896}
+    NCU_TRAFFIC = {"k_accumulate_f32": 93_522_432 + 2_617_088, "k_sync<4>": 280_577_024 + 217_864_192}
 
     def roof(alg_bytes, n, ms, name, note):
         ach = alg_bytes / (ms / n / 1e3) / 1e9 if n and ms > 0 else None
