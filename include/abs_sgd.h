@@ -330,6 +330,19 @@ int abs_ipc_export(const void *dev_ptr, void *handle_out, uint64_t *offset_out);
 int abs_ipc_open(const void *handle, uint64_t offset, void **dev_ptr_out);
 int abs_ipc_close(void *dev_ptr, uint64_t offset);
 
+/* Checkpoint and resume (the paper has no counterpart).  abs_state_export writes everything a later
+ * abs_state_import needs to continue the run bit for bit: parameters (both buffers), momentum, both
+ * accumulator sets, counters and logs, iteration counter, set index, rates in effect -- abs_state_bytes()
+ * bytes of HOST memory, dominated by the accumulators (8 * W * P bytes).  Both calls block: they start any
+ * waiting micro-batch groups and wait for everything enqueued on the context's streams.  Import needs a
+ * context created with the same abs_config (streams and initial lr may differ; the saved rate wins) and, in
+ * multi-GPU mode, attached with the same rank layout; it replaces the context's whole state.  Errors:
+ * ABS_EINVAL (NULL / short buffer, foreign or mismatching state, called between abs_global_begin and
+ * abs_global_end), ABS_ECUDA. */
+size_t abs_state_bytes(abs_ctx *ctx);
+int abs_state_export(abs_ctx *ctx, void *dst_host, size_t bytes);
+int abs_state_import(abs_ctx *ctx, const void *src_host, size_t bytes);
+
 /* One fused sync step on buffers the CALLER owns, for callers that cannot allocate device
  * memory.  (No counterpart in the paper: this is a packaging variant of the kernel behind
  * abs_sync_step, not another algorithm step.)

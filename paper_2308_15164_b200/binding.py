@@ -84,6 +84,9 @@ _sig = {
     "abs_ipc_export": (ctypes.c_int, [_vp, _vp, ctypes.POINTER(_u64)]),
     "abs_ipc_open": (ctypes.c_int, [_vp, _u64, ctypes.POINTER(_vp)]),
     "abs_ipc_close": (ctypes.c_int, [_vp, _u64]),
+    "abs_state_bytes": (ctypes.c_size_t, [_vp]),
+    "abs_state_export": (ctypes.c_int, [_vp, _vp, ctypes.c_size_t]),
+    "abs_state_import": (ctypes.c_int, [_vp, _vp, ctypes.c_size_t]),
     "abs_sync_step_noalloc": (ctypes.c_int, [_vp, _vp, _vp, _u64, _u64, _u32, _vp, ctypes.c_float, ctypes.c_float,
                                              ctypes.c_float, _vp]),
 }
@@ -240,6 +243,16 @@ class AbsSgd:
         b = np.zeros(self.n_ranks * self.W, dtype=np.int32)
         self._ck(lib.abs_global_consumed(self._h, step, b.ctypes.data))
         return b
+
+    # ---- checkpoint / resume ----
+    def state_export(self) -> np.ndarray:
+        buf = np.empty(int(lib.abs_state_bytes(self._h)), dtype=np.uint8)
+        self._ck(lib.abs_state_export(self._h, buf.ctypes.data, buf.nbytes))
+        return buf
+
+    def state_import(self, buf: np.ndarray):
+        buf = np.ascontiguousarray(buf, dtype=np.uint8)
+        self._ck(lib.abs_state_import(self._h, buf.ctypes.data, buf.nbytes))
 
     def step1_finished(self) -> bool:
         done = ctypes.c_int(1)

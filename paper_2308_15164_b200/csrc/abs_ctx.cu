@@ -926,6 +926,113 @@ int abs_check(abs_ctx* c) {
     return ABS_OK;
 }
 
+// ---- checkpoint / resume ----------------------------------------------------------------------------
+namespace {
+struct StateHeader {
+    uint32_t magic, version;
+    abs_config cfg;            // stream fields zeroed
+    uint64_t payload_bytes;    // workspace prefix that holds x, v, accumulators, counters, logs
+    uint64_t t;
+    uint32_t cur, n_ranks, rank;
+    int32_t pub, pending, pending_out;
+    float lr_now, lr_prev_call, disp_scale, global_prev_lr;
+    int32_t h_cnt[2 * kMaxW];
+};
+constexpr uint32_t kStateMagic = 0x53534241u;   // "ABSS"
+
+size_t state_payload_bytes(const abs_ctx* c) { return c->L.off_gcnt + (size_t)(kMaxW + 64) * 4; }
+
+bool same_config(const abs_config& a, const abs_config& b) {
+    return a.P == b.P && a.W == b.W && a.grad_dtype == b.grad_dtype && a.flags == b.flags && a.mlp_in == b.mlp_in &&
+           a.mlp_hidden == b.mlp_hidden && a.mlp_out == b.mlp_out && a.mlp_mb == b.mlp_mb && a.momentum == b.momentum &&
+           a.weight_decay == b.weight_decay && a.lambda_dc == b.lambda_dc;
+}
+
+// Everything enqueued so far has finished (waiting micro-batch groups are started first).
+int drain(abs_ctx* c) {
+    if (int rc = flush_all(c)) return rc;
+    if (c->pipelined) CK(cudaStreamSynchronize(c->s_sync));
+    for (int k = 0; k < c->n_wstreams; ++k) CK(cudaStreamSynchronize(c->s_w[k]));
+    if (c->s_copy) CK(cudaStreamSynchronize(c->s_copy));
+    CK(cudaStreamSynchronize(c->s_acc));
+    if (c->pipelined) CK(cudaStreamSynchronize(c->s_sync));
+    for (int k = 0; k < c->n_wstreams; ++k) c->w_outstanding[k] = false;
+    return ABS_OK;
+}
+}  // namespace
+
+size_t abs_state_bytes(abs_ctx* c) {
+    if (!live(c)) return 0;
+    return sizeof(StateHeader) + state_payload_bytes(c);
+}
+
+int abs_state_export(abs_ctx* c, void* dst_host, size_t bytes) {
+    if (!live(c)) return ABS_ESTATE;
+    if (!dst_host) return invalid(c, "destination pointer is NULL");
+    if (bytes < sizeof(StateHeader) + state_payload_bytes(c)) return invalid(c, "buffer smaller than abs_state_bytes()");
+    if (c->global_phase != 0) return invalid(c, "between abs_global_begin and abs_global_end");
+    if (int rc = drain(c)) return rc;
+    StateHeader h{};
+    h.magic = kStateMagic;
+    h.version = 1;
+    h.cfg = c->cfg;
+    h.cfg.stream_acc = h.cfg.stream_sync = nullptr;
+    h.cfg.lr = 0.f;   // the rate in effect is saved below
+    h.payload_bytes = state_payload_bytes(c);
+    h.t = c->t;
+    h.cur = c->cur;
+    h.n_ranks = c->n_ranks;
+    h.rank = c->rank;
+    h.pub = c->pub;
+    h.pending = c->pending ? 1 : 0;
+    h.pending_out = c->pending_out;
+    h.lr_now = c->lr_now;
+    h.lr_prev_call = c->lr_prev_call;
+    h.disp_scale = c->disp_scale;
+    h.global_prev_lr = c->global_prev_lr;
+    for (size_t k = 0; k < c->h_cnt.size(); ++k) h.h_cnt[k] = c->h_cnt[k];
+    memcpy(dst_host, &h, sizeof h);
+    CK(cudaMemcpy(static_cast<char*>(dst_host) + sizeof h, c->ws, h.payload_bytes, cudaMemcpyDeviceToHost));
+    return ABS_OK;
+}
+
+int abs_state_import(abs_ctx* c, const void* src_host, size_t bytes) {
+    if (!live(c)) return ABS_ESTATE;
+    if (!src_host) return invalid(c, "source pointer is NULL");
+    if (bytes < sizeof(StateHeader)) return invalid(c, "buffer smaller than a state header");
+    StateHeader h;
+    memcpy(&h, src_host, sizeof h);
+    if (h.magic != kStateMagic || h.version != 1) return invalid(c, "not a state written by abs_state_export");
+    if (!same_config(h.cfg, c->cfg)) return invalid(c, "the state was exported from a context with another configuration");
+    if (h.payload_bytes != state_payload_bytes(c) || bytes < sizeof h + h.payload_bytes) return invalid(c, "state is truncated");
+    if (h.n_ranks != c->n_ranks || h.rank != c->rank) return invalid(c, "the state belongs to another rank layout (abs_global_attach first)");
+    if (c->global_phase != 0) return invalid(c, "between abs_global_begin and abs_global_end");
+    if (h.cur > 1 || h.pub < 0 || h.pub > 1 || h.pending_out < 0 || h.pending_out > 1) return invalid(c, "state header is corrupt");
+    if (int rc = drain(c)) return rc;
+    CK(cudaMemcpy(c->ws, static_cast<const char*>(src_host) + sizeof h, h.payload_bytes, cudaMemcpyHostToDevice));
+    c->t = h.t;
+    c->cur = h.cur;
+    c->pub = h.pub;
+    c->pending = h.pending != 0;
+    c->pending_out = h.pending_out;
+    c->lr_now = h.lr_now;
+    c->lr_prev_call = h.lr_prev_call;
+    c->disp_scale = h.disp_scale;
+    c->global_prev_lr = h.global_prev_lr;
+    for (size_t k = 0; k < c->h_cnt.size(); ++k) c->h_cnt[k] = h.h_cnt[k];
+    if (c->mlp) {   // the bf16 copies are a function of the parameters: rebuild them
+        CK(launch_cast_bf16(c->x(0), c->shadow(0), c->L.P_pad, c->num_sms, c->s_acc));
+        c->launches += 1;
+        if (c->pipelined) {
+            CK(launch_cast_bf16(c->x(1), c->shadow(1), c->L.P_pad, c->num_sms, c->s_acc));
+            c->launches += 1;
+        }
+        CK(cudaStreamSynchronize(c->s_acc));
+    }
+    if (c->pipelined) CK(cudaEventRecord(c->ev_sync_done, c->s_sync));   // what "pending" waits for has happened
+    return ABS_OK;
+}
+
 int abs_set_launch(abs_ctx* c, int kernel_class, int ctas_per_sm) {
     if (!live(c)) return ABS_ESTATE;
     if (kernel_class < 0 || kernel_class >= ABS_K_COUNT || ctas_per_sm < -1 || ctas_per_sm > 64)
