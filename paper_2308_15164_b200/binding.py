@@ -132,7 +132,8 @@ class AbsSgd:
 
     def __init__(self, params0: torch.Tensor, W: int, lr: float, momentum=0.0, weight_decay=0.0, lambda_dc=0.0,
                  grad_dtype=GRAD_F32, pipelined=False, mlp=None, host_input=False, overwrite_first=False,
-                 mlp_coalesce=False, stream_acc: Optional[torch.cuda.Stream] = None, stream_sync: Optional[torch.cuda.Stream] = None):
+                 mlp_coalesce=False, stream_acc: Optional[torch.cuda.Stream] = None, stream_sync: Optional[torch.cuda.Stream] = None,
+                 workspace: Optional[torch.Tensor] = None):
         assert params0.is_cuda and params0.dtype == torch.float32 and params0.is_contiguous()
         self.device = params0.device
         self.P, self.W = params0.numel(), W
@@ -144,7 +145,10 @@ class AbsSgd:
         nbytes = abs_workspace_bytes(self.cfg)
         if nbytes == 0:
             raise AbsError(EINVAL, "invalid configuration")
-        self.workspace = torch.empty(nbytes, dtype=torch.uint8, device=self.device)
+        if workspace is None:
+            workspace = torch.empty(nbytes, dtype=torch.uint8, device=self.device)
+        assert workspace.dtype == torch.uint8 and workspace.is_cuda and workspace.numel() >= nbytes
+        self.workspace = workspace            # caller-provided memory is used as it is (abs_init checks the alignment)
         self._h = _vp()
         # params0 may have been produced on another stream: make it visible to stream_acc.
         self.stream_acc.wait_stream(torch.cuda.current_stream(self.device))
