@@ -87,6 +87,12 @@ extern "C" {
                                        At most four groups wait at a time (the oldest is started when a fifth
                                        worker opens one).                                                       */
 
+#define ABS_FLAG_GRAD_NORM 32u   /* the fused step also forms |Gbar|^2, the squared norm of the weighted average it
+                                     applies (before Eq. 6 and weight decay): per-thread fp32 squares, summed in fp64
+                                     by warp shuffles, one partial per CTA, added in a fixed order by the last CTA
+                                     (reproducible run to run).  No extra memory traffic beyond 8 bytes per CTA.
+                                     Read it with abs_grad_norm2.  Not with abs_global_*.                        */
+
 #define ABS_MAX_WORKERS 64u
 #define ABS_MAX_RANKS   16u   /* GPUs taking part in abs_global_* (n_ranks * W <= ABS_MAX_WORKERS)        */
 #define ABS_IPC_HANDLE_BYTES 64
@@ -203,6 +209,11 @@ int abs_counters(abs_ctx *ctx, int32_t *cnt_host, uint32_t *cur, uint64_t *t);
  * counted ON THE DEVICE by the accumulate kernels and logged by the fused kernel before it
  * cleared them.  b_host[W].  Blocks until the logging kernel has finished. */
 int abs_consumed(abs_ctx *ctx, uint64_t step, int32_t *b_host);
+
+/* |Gbar|^2 of the weighted average that sync step `step` applied (0 if it applied nothing); same window
+ * and blocking behaviour as abs_consumed.  Needs ABS_FLAG_GRAD_NORM.  (A run-time metric; the paper's
+ * experiments log accuracy over time only.) */
+int abs_grad_norm2(abs_ctx *ctx, uint64_t step, double *out);
 
 /* Algorithm 1, Step 2 loop condition "while Step 1 not finished": *done = 0 while the fused kernel
  * launched by the last abs_sync_step (pipelined mode) is still running, 1 once it has completed
@@ -338,7 +349,7 @@ int abs_ipc_close(void *dev_ptr, uint64_t offset);
  * context created with the same abs_config (streams and initial lr may differ; the saved rate wins) and, in
  * multi-GPU mode, attached with the same rank layout; it replaces the context's whole state.  Errors:
  * ABS_EINVAL (NULL / short buffer, foreign or mismatching state, called between abs_global_begin and
- * abs_global_end), ABS_ECUDA. */
+ * abs_global_end), ABS_ECUDA.  The log behind abs_grad_norm2 is not part of the state. */
 size_t abs_state_bytes(abs_ctx *ctx);
 int abs_state_export(abs_ctx *ctx, void *dst_host, size_t bytes);
 int abs_state_import(abs_ctx *ctx, const void *src_host, size_t bytes);

@@ -58,6 +58,7 @@ class AbsSgdOracle:
         self.cur = 0
         self.t = 0
         self.consumed = []                                # b_i used by each sync step
+        self.gnorm2 = []                                  # |Gbar|^2 applied by each sync step (0: nothing applied)
 
     # Step 2 of Algorithm 1: G_t^i = G_t^i + g ; M_t^i = M_t^i + M_r
     def accumulate(self, i, g):
@@ -82,11 +83,14 @@ class AbsSgdOracle:
             for i in range(self.W):                       # sum_i G_{t-1}^i, worker order
                 G += self.acc[d, i].astype(np.float64)
             Gbar = G / B                                  # weighted average (Algorithm 1, Step 1)
+            self.gnorm2.append(float(np.dot(Gbar, Gbar)))  # a logged metric; takes no part in the update
             if self.lambda_dc != 0.0:                     # Eq. 6, delayed-gradient compensation
                 Gbar = Gbar + self.lambda_dc * Gbar * Gbar * (self.x - self.x_prev)
             g = Gbar + self.weight_decay * self.x
             self.v = self.momentum * self.v + g
             self.x = self.x - self.lr * self.v            # x_{t+1} = x_t - gamma * Gtilde_t
+        else:
+            self.gnorm2.append(0.0)
         self.x_prev = x_old
         self.acc[d].fill(0.0)                             # Step 2 "Initialization" of the next
         self.cnt[d].fill(0)                               # iteration's G and M

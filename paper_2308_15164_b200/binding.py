@@ -26,7 +26,7 @@ lib = ctypes.CDLL(LIB_PATH)
 
 OK, EINVAL, ESTATE, ECUDA, ENOMEM, ETIMEOUT, ELIMIT = 0, -1, -2, -3, -4, -5, -6
 GRAD_F32, GRAD_BF16 = 0, 1
-FLAG_PIPELINED, FLAG_MLP, FLAG_HOST_INPUT, FLAG_OVERWRITE_FIRST, FLAG_MLP_COALESCE = 1, 2, 4, 8, 16
+FLAG_PIPELINED, FLAG_MLP, FLAG_HOST_INPUT, FLAG_OVERWRITE_FIRST, FLAG_MLP_COALESCE, FLAG_GRAD_NORM = 1, 2, 4, 8, 16, 32
 K_ACCUMULATE, K_SYNC, K_MLP_FWD, K_MLP_BWD, K_MLP_DW1 = range(5)
 MAX_WORKERS, MAX_RANKS, IPC_HANDLE_BYTES = 64, 16, 64
 KERNEL_NAMES = ["accumulate", "sync", "mlp_fwd", "mlp_bwd", "mlp_dw1"]
@@ -64,6 +64,7 @@ _sig = {
     "abs_accumulator": (ctypes.c_int, [_vp, _u32, _u32, ctypes.POINTER(_vp)]),
     "abs_counters": (ctypes.c_int, [_vp, _vp, ctypes.POINTER(_u32), ctypes.POINTER(_u64)]),
     "abs_consumed": (ctypes.c_int, [_vp, _u64, _vp]),
+    "abs_grad_norm2": (ctypes.c_int, [_vp, _u64, ctypes.POINTER(ctypes.c_double)]),
     "abs_set_lr": (ctypes.c_int, [_vp, ctypes.c_float]),
     "abs_step1_finished": (ctypes.c_int, [_vp, ctypes.POINTER(ctypes.c_int)]),
     "abs_wait": (ctypes.c_int, [_vp]),
@@ -132,14 +133,14 @@ class AbsSgd:
 
     def __init__(self, params0: torch.Tensor, W: int, lr: float, momentum=0.0, weight_decay=0.0, lambda_dc=0.0,
                  grad_dtype=GRAD_F32, pipelined=False, mlp=None, host_input=False, overwrite_first=False,
-                 mlp_coalesce=False, stream_acc: Optional[torch.cuda.Stream] = None, stream_sync: Optional[torch.cuda.Stream] = None,
+                 mlp_coalesce=False, grad_norm=False, stream_acc: Optional[torch.cuda.Stream] = None, stream_sync: Optional[torch.cuda.Stream] = None,
                  workspace: Optional[torch.Tensor] = None):
         assert params0.is_cuda and params0.dtype == torch.float32 and params0.is_contiguous()
         self.device = params0.device
         self.P, self.W = params0.numel(), W
         self.stream_acc = stream_acc or torch.cuda.Stream(device=self.device)
         self.stream_sync = stream_sync or (torch.cuda.Stream(device=self.device) if pipelined else None)
-        flags = (FLAG_PIPELINED if pipelined else 0) | (FLAG_MLP if mlp else 0) | (FLAG_HOST_INPUT if host_input else 0) | (FLAG_OVERWRITE_FIRST if overwrite_first else 0) | (FLAG_MLP_COALESCE if mlp_coalesce else 0)
+        flags = (FLAG_PIPELINED if pipelined else 0) | (FLAG_MLP if mlp else 0) | (FLAG_HOST_INPUT if host_input else 0) | (FLAG_OVERWRITE_FIRST if overwrite_first else 0) | (FLAG_MLP_COALESCE if mlp_coalesce else 0) | (FLAG_GRAD_NORM if grad_norm else 0)
         self.cfg = make_config(self.P, W, lr, momentum, weight_decay, lambda_dc, grad_dtype, flags, mlp,
                                self.stream_acc.cuda_stream, self.stream_sync.cuda_stream if self.stream_sync else 0)
         nbytes = abs_workspace_bytes(self.cfg)
@@ -257,6 +258,11 @@ class AbsSgd:
     def state_import(self, buf: np.ndarray):
         buf = np.ascontiguousarray(buf, dtype=np.uint8)
         self._ck(lib.abs_state_import(self._h, buf.ctypes.data, buf.nbytes))
+
+    def grad_norm2(self, step: int) -> float:
+        out = ctypes.c_double(0.0)
+        self._ck(lib.abs_grad_norm2(self._h, step, ctypes.byref(out)))
+        return float(out.value)
 
     def step1_finished(self) -> bool:
         done = ctypes.c_int(1)

@@ -29,7 +29,8 @@ size_t round_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 struct Layout {
     size_t P_pad = 0;
     size_t off_x[2] = {0, 0}, off_v = 0, off_acc = 0, off_cnt = 0, off_ticket = 0, off_log = 0, off_gcnt = 0;
-    size_t off_shadow[2] = {0, 0}, off_mlp = 0, off_stage[2] = {0, 0};
+    size_t off_shadow[2] = {0, 0}, off_mlp = 0, off_stage[2] = {0, 0}, off_norm_part = 0, off_norm_log = 0;
+    size_t norm_slots = 0;
     size_t total = 0;
 };
 
@@ -39,7 +40,8 @@ bool config_ok(const abs_config* c, std::string* why) {
     if (c->P == 0) return fail("P must be > 0");
     if (c->W == 0 || c->W > ABS_MAX_WORKERS) return fail("W must be in 1..64");
     if (c->grad_dtype != ABS_GRAD_F32 && c->grad_dtype != ABS_GRAD_BF16) return fail("unknown grad_dtype");
-    if (c->flags & ~(ABS_FLAG_PIPELINED | ABS_FLAG_MLP | ABS_FLAG_HOST_INPUT | ABS_FLAG_OVERWRITE_FIRST | ABS_FLAG_MLP_COALESCE))
+    if (c->flags & ~(ABS_FLAG_PIPELINED | ABS_FLAG_MLP | ABS_FLAG_HOST_INPUT | ABS_FLAG_OVERWRITE_FIRST | ABS_FLAG_MLP_COALESCE |
+                     ABS_FLAG_GRAD_NORM))
         return fail("unknown flag bits");
     if ((c->flags & ABS_FLAG_MLP_COALESCE) && !(c->flags & ABS_FLAG_MLP)) return fail("ABS_FLAG_MLP_COALESCE needs ABS_FLAG_MLP");
     if (!std::isfinite(c->lr) || !std::isfinite(c->momentum) || !std::isfinite(c->weight_decay) ||
@@ -83,6 +85,11 @@ Layout make_layout(const abs_config& c) {
         const size_t es = c.grad_dtype == ABS_GRAD_BF16 ? 2 : 4;
         L.off_stage[0] = take(L.P_pad * es);
         L.off_stage[1] = take(L.P_pad * es);
+    }
+    if (c.flags & ABS_FLAG_GRAD_NORM) {
+        L.norm_slots = L.P_pad / 1024 + 1;            // one per CTA of the fused step's largest grid
+        L.off_norm_part = take(L.norm_slots * 8);
+        L.off_norm_log = take((size_t)kLogDepth * 8);
     }
     L.total = o;
     return L;
@@ -180,6 +187,9 @@ struct abs_ctx {
         return reinterpret_cast<int32_t*>(ws + L.off_log) + (step % kLogDepth) * kMaxW;
     }
     __nv_bfloat16* shadow(int k) const { return reinterpret_cast<__nv_bfloat16*>(ws + L.off_shadow[k]); }
+    double* norm_part() const { return reinterpret_cast<double*>(ws + L.off_norm_part); }
+    double* norm_log(uint64_t step) const { return reinterpret_cast<double*>(ws + L.off_norm_log) + step % kLogDepth; }
+    bool grad_norm() const { return (cfg.flags & ABS_FLAG_GRAD_NORM) != 0; }
     int32_t* gcnt() const { return reinterpret_cast<int32_t*>(ws + L.off_gcnt); }
     int* applied_word() const { return reinterpret_cast<int*>(ws + L.off_gcnt) + kMaxW; }
 };
@@ -289,6 +299,11 @@ int launch_fused(abs_ctx* c, uint32_t set, int in, int out, uint64_t log_step, c
     a.disp_scale = c->disp_scale;
     a.shadow = c->mlp ? c->shadow(out) : nullptr;
     a.zero_acc = (c->cfg.flags & ABS_FLAG_OVERWRITE_FIRST) ? 0 : 1;
+    if (c->grad_norm()) {
+        a.norm_part = c->norm_part();
+        a.norm_out = c->norm_log(log_step);
+        a.norm_slots = (unsigned int)c->L.norm_slots;
+    }
     {
         Timed tm(c, ABS_K_SYNC, stream);
         CK(launch_sync(a, c->ctas_per_sm[ABS_K_SYNC], c->num_sms, stream));
@@ -452,6 +467,9 @@ int abs_init(abs_ctx** out, const abs_config* cfg, void* workspace_dev, size_t w
     if ((e = cudaMemsetAsync(c->ws, 0, state_bytes, c->s_acc)) != cudaSuccess) return bail(e, "cudaMemsetAsync");
     if ((e = cudaMemcpyAsync(c->x(0), params0_dev, cfg->P * 4, cudaMemcpyDeviceToDevice, c->s_acc)) != cudaSuccess)
         return bail(e, "cudaMemcpyAsync(params0)");
+    if ((cfg->flags & ABS_FLAG_GRAD_NORM) &&
+        (e = cudaMemsetAsync(c->ws + L.off_norm_log, 0, (size_t)kLogDepth * 8, c->s_acc)) != cudaSuccess)
+        return bail(e, "cudaMemsetAsync");
     if (c->mlp) {
         c->mlp_dims = MlpDims{(int)cfg->mlp_in, (int)cfg->mlp_hidden, (int)cfg->mlp_out, (int)cfg->mlp_mb};
         const char* msg = nullptr;
@@ -622,6 +640,7 @@ int abs_sync_step(abs_ctx* c) {
             c->disp_scale = c->lr_prev_call;
         } else {
             CK(cudaMemsetAsync(c->log_row(c->t), 0, kMaxW * 4, c->s_acc));
+            if (c->grad_norm()) CK(cudaMemsetAsync(c->norm_log(c->t), 0, 8, c->s_acc));
             c->disp_scale = 0.f;
         }
     } else {
@@ -648,6 +667,7 @@ int abs_sync_step(abs_ctx* c) {
             c->pending_out = out;
         } else {
             CK(cudaMemsetAsync(c->log_row(c->t + 1), 0, kMaxW * 4, c->s_sync));
+            if (c->grad_norm()) CK(cudaMemsetAsync(c->norm_log(c->t + 1), 0, 8, c->s_sync));
             c->disp_scale = 0.f;
             c->pending_out = c->pub;
         }
@@ -670,6 +690,7 @@ int abs_global_attach(abs_ctx* c, const abs_peer_table* peers) {
     if (peers->n_ranks == 0 || peers->n_ranks > ABS_MAX_RANKS) return invalid(c, "n_ranks must be in 1..16");
     if (peers->rank >= peers->n_ranks) return invalid(c, "rank out of range");
     if ((uint64_t)peers->n_ranks * c->cfg.W > ABS_MAX_WORKERS) return invalid(c, "n_ranks * W must not exceed 64");
+    if (c->grad_norm()) return invalid(c, "ABS_FLAG_GRAD_NORM is not available in multi-GPU mode");
     if (c->t != 0 || c->n_ranks != 0) return invalid(c, "attach once, before the first step");
     for (uint32_t q = 0; q < peers->n_ranks; ++q) {
         void* p = peers->workspace_dev[q];
@@ -873,6 +894,18 @@ int abs_global_consumed(abs_ctx* c, uint64_t step, int32_t* b_host) {
     CK(cudaStreamSynchronize(c->s_sync));
     CK(cudaStreamSynchronize(c->s_acc));
     CK(cudaMemcpy(b_host, c->log_row(step), (size_t)c->n_ranks * c->cfg.W * sizeof(int32_t), cudaMemcpyDeviceToHost));
+    return ABS_OK;
+}
+
+int abs_grad_norm2(abs_ctx* c, uint64_t step, double* out) {
+    if (!live(c)) return ABS_ESTATE;
+    if (!c->grad_norm()) return invalid(c, "context was created without ABS_FLAG_GRAD_NORM");
+    if (c->n_ranks != 0) return invalid(c, "not available in multi-GPU mode");
+    if (!out) return invalid(c, "output pointer is NULL");
+    if (step >= c->t || c->t - step >= (uint64_t)kLogDepth) return invalid(c, "step is not in the logged window");
+    if (c->pipelined) CK(cudaStreamSynchronize(c->s_sync));
+    CK(cudaStreamSynchronize(c->s_acc));
+    CK(cudaMemcpy(out, c->norm_log(step), sizeof(double), cudaMemcpyDeviceToHost));
     return ABS_OK;
 }
 

@@ -36,6 +36,9 @@ struct SyncArgs {
     float disp_scale;         // x_t - x_{t-1} = -disp_scale * v   (0 when the previous step was a no-op)
     __nv_bfloat16* shadow;    // optional bf16 copy of x_{t+1} [P_pad], or nullptr
     int zero_acc;             // 1: overwrite the consumed rows with zeros; 0: leave them (overwrite-first mode)
+    double* norm_part;        // optional: one slot per CTA for the partial sums of |Gbar|^2 ...
+    double* norm_out;         // ... and where the last CTA puts the total (nullptr: the norm is not computed)
+    unsigned int norm_slots;  // slots in norm_part
 };
 // n (1..kMaxAccBatch) gradients of one worker added in one pass over its accumulator row, in list order.
 constexpr int kMaxAccBatch = 8;

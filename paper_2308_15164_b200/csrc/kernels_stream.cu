@@ -234,9 +234,11 @@ struct UpdateCoef {
     float lr, mu, wd, lambda_dc;
     float disp_scale;   // x_t - x_{t-1} = -disp_scale * v   (0 when the previous step was a no-op)
 };
-__device__ __forceinline__ void update_vec(float4& x, float4& v, const float4 s, const float Bf,
-                                           const UpdateCoef& a) {
+// Returns the squared norm of the four averaged-gradient components (before Eq. 6 and weight decay).
+__device__ __forceinline__ float update_vec(float4& x, float4& v, const float4 s, const float Bf,
+                                            const UpdateCoef& a) {
     float gx = __fdiv_rn(s.x, Bf), gy = __fdiv_rn(s.y, Bf), gz = __fdiv_rn(s.z, Bf), gw = __fdiv_rn(s.w, Bf);
+    const float n2 = gx * gx + gy * gy + gz * gz + gw * gw;
     if (a.lambda_dc != 0.0f) {   // Eq. 6 with x_t - x_{t-1} = -disp_scale * v
         const float c = -a.lambda_dc * a.disp_scale;
         gx += c * gx * gx * v.x; gy += c * gy * gy * v.y; gz += c * gz * gz * v.z; gw += c * gw * gw * v.w;
@@ -244,6 +246,7 @@ __device__ __forceinline__ void update_vec(float4& x, float4& v, const float4 s,
     gx += a.wd * x.x; gy += a.wd * x.y; gz += a.wd * x.z; gw += a.wd * x.w;
     v.x = a.mu * v.x + gx; v.y = a.mu * v.y + gy; v.z = a.mu * v.z + gz; v.w = a.mu * v.w + gw;
     x.x -= a.lr * v.x; x.y -= a.lr * v.y; x.z -= a.lr * v.z; x.w -= a.lr * v.w;
+    return n2;
 }
 
 __device__ __forceinline__ void store_shadow(__nv_bfloat16* shadow, unsigned long long idx, const float4 x) {
@@ -255,9 +258,11 @@ __device__ __forceinline__ void store_shadow(__nv_bfloat16* shadow, unsigned lon
     reinterpret_cast<uint2*>(shadow)[idx] = pk;
 }
 
-template <int WT, int U>
+template <int WT, int U, bool kNorm>
 __global__ void __launch_bounds__(kBlock) k_sync(const SyncArgs a) {
     __shared__ int s_cnt[kMaxW];
+    __shared__ double s_norm[kBlock / 32];
+    float norm_acc = 0.f;   // kNorm: this thread's share of |Gbar|^2 (a handful of vectors)
     const int W = WT > 0 ? WT : a.W;
     if (threadIdx.x < W) s_cnt[threadIdx.x] = a.cnt[threadIdx.x];
     __syncthreads();
@@ -303,7 +308,7 @@ __global__ void __launch_bounds__(kBlock) k_sync(const SyncArgs a) {
                             if ((active >> i) & 1) {
                                 s.x += r[u][i].x; s.y += r[u][i].y; s.z += r[u][i].z; s.w += r[u][i].w;
                             }
-                        update_vec(x[u], v[u], s, Bf, uc);
+                        norm_acc += update_vec(x[u], v[u], s, Bf, uc);
                         st_stream(xout + idx, x[u]);
                         st_stream(v4 + idx, v[u]);
                         if (a.shadow) store_shadow(a.shadow, idx, x[u]);
@@ -329,7 +334,7 @@ __global__ void __launch_bounds__(kBlock) k_sync(const SyncArgs a) {
                                 if (a.zero_acc) st_stream(acc4 + (i0 + c) * rs + idx, zero);
                             }
                     }
-                    update_vec(x, v, s, Bf, uc);
+                    norm_acc += update_vec(x, v, s, Bf, uc);
                     st_stream(xout + idx, x);
                     st_stream(v4 + idx, v);
                     if (a.shadow) store_shadow(a.shadow, idx, x);
@@ -347,18 +352,51 @@ __global__ void __launch_bounds__(kBlock) k_sync(const SyncArgs a) {
         }
     }
 
+    if constexpr (kNorm) {
+        // |Gbar|^2: per-thread fp32 share -> warp sum in fp64 by shuffles -> one fp64 partial per CTA, in a slot
+        // of its own; the last CTA adds the slots in a fixed order, so the figure is reproducible run to run.
+        double w = (double)norm_acc;
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) w += __shfl_xor_sync(0xFFFFFFFFu, w, o);
+        if ((threadIdx.x & 31) == 0) s_norm[threadIdx.x >> 5] = w;
+        __syncthreads();
+        if (threadIdx.x == 0) {
+            double c = 0.0;
+            for (int k = 0; k < kBlock / 32; ++k) c += s_norm[k];
+            a.norm_part[blockIdx.x] = c;
+        }
+    }
+
     // The last CTA to finish logs the consumed b_i and clears the device counters (every CTA
     // read them before taking its ticket).
+    __shared__ unsigned int s_last;
     __syncthreads();
     if (threadIdx.x == 0) {
         __threadfence();
         const unsigned int t = atomicAdd(a.ticket, 1u);
+        s_last = (t == gridDim.x - 1) ? 1u : 0u;
         if (t == gridDim.x - 1) {
             for (int i = 0; i < W; ++i) {
                 a.log_row[i] = s_cnt[i];
                 a.cnt[i] = 0;
             }
             *a.ticket = 0u;
+        }
+    }
+    if constexpr (kNorm) {
+        __syncthreads();
+        if (s_last) {   // every other CTA's partial was written (and fenced) before it took its ticket
+            __threadfence();
+            double c = 0.0;
+            for (unsigned k = threadIdx.x; k < gridDim.x; k += kBlock) c += __ldcg(a.norm_part + k);
+            __shared__ double s_all[kBlock];
+            s_all[threadIdx.x] = c;
+            __syncthreads();
+            if (threadIdx.x == 0) {
+                double tot = 0.0;
+                for (int k = 0; k < kBlock; ++k) tot += s_all[k];
+                *a.norm_out = B > 0 ? tot : 0.0;
+            }
         }
     }
 }
@@ -466,7 +504,12 @@ inline unsigned grid_for(unsigned long long n_items, int per_cta, int ctas_per_s
 template <int WT, int U>
 cudaError_t launch_sync_t(const SyncArgs& a, int ctas_per_sm, int num_sms, cudaStream_t stream) {
     const unsigned grid = grid_for(a.n_vec, kBlock * U, ctas_per_sm, num_sms);
-    k_sync<WT, U><<<grid, kBlock, 0, stream>>>(a);
+    if (a.norm_out) {
+        if (grid > a.norm_slots) return cudaErrorInvalidValue;
+        k_sync<WT, U, true><<<grid, kBlock, 0, stream>>>(a);
+    } else {
+        k_sync<WT, U, false><<<grid, kBlock, 0, stream>>>(a);
+    }
     return cudaGetLastError();
 }
 

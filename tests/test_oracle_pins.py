@@ -159,3 +159,20 @@ def test_unbroken_mutant_passes():
 
     for pin in ALL_PINS:
         pin(make)
+
+
+def test_logged_gradient_norm_closed_form():
+    """|Gbar|^2 for constant-per-worker gradients c_i: P * (sum_i b_i c_i / sum_i b_i)^2, logged one step late
+    (the delayed gradients), 0 for steps that applied nothing; Eq. 6 and weight decay do not enter it."""
+    P, W = 37, 3
+    o = AbsSgdOracle(np.ones(P, dtype=np.float32), W, 0.1, 0.9, 0.01, 0.5)
+    b, c = (3, 0, 2), (2.0, 100.0, -1.0)
+    for i in range(W):
+        for _ in range(b[i]):
+            o.accumulate(i, np.full(P, c[i], dtype=np.float32))
+    o.sync_step()                                      # applies G_{-1} = 0: nothing
+    o.sync_step()                                      # applies the set above
+    o.sync_step()                                      # nothing again
+    want = P * ((3 * 2.0 + 2 * -1.0) / 5.0) ** 2
+    assert o.gnorm2[0] == 0.0 and o.gnorm2[2] == 0.0
+    assert abs(o.gnorm2[1] - want) <= 1e-12 * want
