@@ -239,7 +239,9 @@ int abs_wait(abs_ctx *ctx);
 int abs_check(abs_ctx *ctx);
 
 /* Launch shape of a kernel class: CTAs per SM for the persistent grid (0 = default, -1 = one
- * tile per CTA) for ABS_K_ACCUMULATE and ABS_K_SYNC.  For the MLP classes the value selects
+ * tile per CTA) for ABS_K_ACCUMULATE and ABS_K_SYNC.  ABS_K_SYNC also takes -2: the fused step with its rows
+ * staged through shared memory by the bulk-copy engine (cp.async.bulk loads and stores, mbarrier pipeline;
+ * W <= 24 and no ABS_FLAG_GRAD_NORM, else the default kernel runs); same results bit for bit.  For the MLP classes the value selects
  * kernel variants instead (results agree within rounding):
  *   ABS_K_MLP_DW1  bit mask.  dW1 kernel: 0 = chosen per call (the persistent ring kernel when the tile is
  *                  stored or the call is K-batched, the register-prefetch kernel for single adds);

@@ -299,6 +299,7 @@ int launch_fused(abs_ctx* c, uint32_t set, int in, int out, uint64_t log_step, c
     a.disp_scale = c->disp_scale;
     a.shadow = c->mlp ? c->shadow(out) : nullptr;
     a.zero_acc = (c->cfg.flags & ABS_FLAG_OVERWRITE_FIRST) ? 0 : 1;
+    a.status = reinterpret_cast<int*>(c->ticket() + 2);
     if (c->grad_norm()) {
         a.norm_part = c->norm_part();
         a.norm_out = c->norm_log(log_step);
@@ -944,6 +945,14 @@ int abs_check(abs_ctx* c) {
     if (c->pipelined) CK(cudaStreamSynchronize(c->s_sync));
     for (int k = 0; k < c->n_wstreams; ++k) CK(cudaStreamSynchronize(c->s_w[k]));
     CK(cudaStreamSynchronize(c->s_acc));
+    {
+        int st = 0;
+        CK(cudaMemcpy(&st, c->ticket() + 2, sizeof(int), cudaMemcpyDeviceToHost));
+        if (st != 0) {
+            c->err = "a bounded device-side wait ran out (fused step, bulk-copy kernel)";
+            return ABS_ETIMEOUT;
+        }
+    }
     if (c->mlp) {
         int bad = 0;
         for (int k = 0; k < kMlpSets; ++k) {
@@ -1068,7 +1077,7 @@ int abs_state_import(abs_ctx* c, const void* src_host, size_t bytes) {
 
 int abs_set_launch(abs_ctx* c, int kernel_class, int ctas_per_sm) {
     if (!live(c)) return ABS_ESTATE;
-    if (kernel_class < 0 || kernel_class >= ABS_K_COUNT || ctas_per_sm < -1 || ctas_per_sm > 64)
+    if (kernel_class < 0 || kernel_class >= ABS_K_COUNT || ctas_per_sm < (kernel_class == ABS_K_SYNC ? -2 : -1) || ctas_per_sm > 64)
         return invalid(c, "bad kernel class or CTA count");
     if (int rc = flush_all(c)) return rc;
     c->ctas_per_sm[kernel_class] = ctas_per_sm;

@@ -39,6 +39,7 @@ struct SyncArgs {
     double* norm_part;        // optional: one slot per CTA for the partial sums of |Gbar|^2 ...
     double* norm_out;         // ... and where the last CTA puts the total (nullptr: the norm is not computed)
     unsigned int norm_slots;  // slots in norm_part
+    int* status;              // optional device status word (ABS_ETIMEOUT if a bounded wait of the bulk-copy kernel ran out)
 };
 // n (1..kMaxAccBatch) gradients of one worker added in one pass over its accumulator row, in list order.
 constexpr int kMaxAccBatch = 8;
@@ -47,7 +48,13 @@ struct GradList {
 };
 cudaError_t launch_accumulate_multi(float* acc_row, const GradList& gl, int n, uint32_t grad_dtype, size_t P, int32_t* cnt,
                                     bool overwrite, int ctas_per_sm, int num_sms, cudaStream_t stream);
+// ctas_per_sm: 0 = default shape, -1 = one tile per CTA, > 0 = persistent grid, -2 = the bulk-copy kernel below
+// where it applies (else the default).
 cudaError_t launch_sync(const SyncArgs& a, int ctas_per_sm, int num_sms, cudaStream_t stream);
+// Same step with the rows staged through shared memory by cp.async.bulk (sync_tma.cu).  cudaErrorNotSupported for
+// W > kSyncTmaMaxW or when the gradient norm is wanted: the caller then uses launch_sync.
+constexpr int kSyncTmaMaxW = 24;
+cudaError_t launch_sync_tma(const SyncArgs& a, int num_sms, cudaStream_t stream);
 
 // ---- Step 1 across GPUs (Algorithm 1, Step 1 as the paper runs it: workers on different GPUs) -----
 // Rank r reduces, updates and redistributes the vectors [vec_lo, vec_hi) of the flat parameter: it reads that

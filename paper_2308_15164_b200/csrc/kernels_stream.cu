@@ -571,6 +571,16 @@ cudaError_t launch_accumulate_multi(float* acc_row, const GradList& gl, int n, u
 }
 
 cudaError_t launch_sync(const SyncArgs& a, int ctas_per_sm, int num_sms, cudaStream_t stream) {
+    // The bulk-copy kernel (sync_tma.cu) gives the same bits.  Measured against the kernels below (alone on a
+    // B200, P = 11.7 M and 40 M): ahead by 3 - 11 % for W = 5, 6, 9, 12, by 1 - 2 % for W = 7, 10, 13, level for
+    // W = 14 - 17 (ahead by 2 % at 40 M parameters and W = 16), behind for W <= 4 (6.0 against 6.7 TB/s), W = 8,
+    // 11 and W >= 18.  It is the default where it is ahead or level; -2 asks for it wherever it can run.
+    const bool bulk_default = (a.W >= 5 && a.W <= 7) || a.W == 9 || a.W == 10 || (a.W >= 12 && a.W <= 17);
+    if (ctas_per_sm == -2 || (ctas_per_sm == 0 && bulk_default && !a.norm_out)) {
+        const cudaError_t e = launch_sync_tma(a, num_sms, stream);
+        if (e != cudaErrorNotSupported) return e;
+        ctas_per_sm = 0;
+    }
     // Measured on B200 (kernel alone, accumulators far larger than L2, GB/s on (8 W + 16) P bytes):
     //   W <= 4   compile-time W, every load of a vector in flight at once, one tile per CTA: 6.2 - 6.5 TB/s
     //            (W = 1: two vectors per thread);
