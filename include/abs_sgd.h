@@ -238,6 +238,12 @@ int abs_wait(abs_ctx *ctx);
  * wait on an mbarrier; its output tile was not written). */
 int abs_check(abs_ctx *ctx);
 
+/* Failure-reporting self-test: enqueues (on stream_acc) one tiny kernel that waits, with the library's bounded
+ * polling loop, for a barrier that nothing completes; it gives up within a fraction of a millisecond and records
+ * the time-out exactly as a stuck copy pipeline of the fused step would.  The next abs_check then returns
+ * ABS_ETIMEOUT once (and clears the record); the context and the GPU stay fully usable.  Nothing faults or hangs. */
+int abs_selftest_timeout(abs_ctx *ctx);
+
 /* Launch shape of a kernel class: CTAs per SM for the persistent grid (0 = default, -1 = one
  * tile per CTA) for ABS_K_ACCUMULATE and ABS_K_SYNC.  ABS_K_SYNC also takes -2: the fused step with its rows
  * staged through shared memory by the bulk-copy engine (cp.async.bulk loads and stores, mbarrier pipeline;

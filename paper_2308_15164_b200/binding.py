@@ -69,6 +69,7 @@ _sig = {
     "abs_step1_finished": (ctypes.c_int, [_vp, ctypes.POINTER(ctypes.c_int)]),
     "abs_wait": (ctypes.c_int, [_vp]),
     "abs_check": (ctypes.c_int, [_vp]),
+    "abs_selftest_timeout": (ctypes.c_int, [_vp]),
     "abs_set_launch": (ctypes.c_int, [_vp, ctypes.c_int, ctypes.c_int]),
     "abs_profile": (ctypes.c_int, [_vp, ctypes.c_int]),
     "abs_kernel_stats": (ctypes.c_int, [_vp, ctypes.c_int, ctypes.POINTER(_u64), ctypes.POINTER(ctypes.c_double)]),
@@ -277,6 +278,9 @@ class AbsSgd:
 
     def check(self):
         self._ck(lib.abs_check(self._h))
+
+    def selftest_timeout(self):
+        self._ck(lib.abs_selftest_timeout(self._h))
 
     def set_launch(self, kernel_class: int, ctas_per_sm: int):
         self._ck(lib.abs_set_launch(self._h, kernel_class, ctas_per_sm))

@@ -949,6 +949,7 @@ int abs_check(abs_ctx* c) {
         int st = 0;
         CK(cudaMemcpy(&st, c->ticket() + 2, sizeof(int), cudaMemcpyDeviceToHost));
         if (st != 0) {
+            CK(cudaMemset(c->ticket() + 2, 0, sizeof(int)));   // reported once; the context stays usable
             c->err = "a bounded device-side wait ran out (fused step, bulk-copy kernel)";
             return ABS_ETIMEOUT;
         }
@@ -1072,6 +1073,13 @@ int abs_state_import(abs_ctx* c, const void* src_host, size_t bytes) {
         CK(cudaStreamSynchronize(c->s_acc));
     }
     if (c->pipelined) CK(cudaEventRecord(c->ev_sync_done, c->s_sync));   // what "pending" waits for has happened
+    return ABS_OK;
+}
+
+int abs_selftest_timeout(abs_ctx* c) {
+    if (!live(c)) return ABS_ESTATE;
+    CK(launch_bounded_wait_selftest(reinterpret_cast<int*>(c->ticket() + 2), c->s_acc));
+    c->launches += 1;
     return ABS_OK;
 }
 

@@ -55,6 +55,9 @@ cudaError_t launch_sync(const SyncArgs& a, int ctas_per_sm, int num_sms, cudaStr
 // W > kSyncTmaMaxW or when the gradient norm is wanted: the caller then uses launch_sync.
 constexpr int kSyncTmaMaxW = 24;
 cudaError_t launch_sync_tma(const SyncArgs& a, int num_sms, cudaStream_t stream);
+// One small launch whose only wait can never be satisfied: it gives up after a few thousand polls and writes
+// ABS_ETIMEOUT to *status (the path a stuck pipeline takes), leaving the context usable.
+cudaError_t launch_bounded_wait_selftest(int* status, cudaStream_t stream);
 
 // ---- Step 1 across GPUs (Algorithm 1, Step 1 as the paper runs it: workers on different GPUs) -----
 // Rank r reduces, updates and redistributes the vectors [vec_lo, vec_hi) of the flat parameter: it reads that

@@ -246,7 +246,32 @@ __global__ void __launch_bounds__(kThreads) k_sync_tma(const SyncArgs a, const i
     }
 }
 
+// Waits, with the same bounded polling loop, for an mbarrier that nothing ever completes, and reports the
+// time-out the way the pipeline above does.  `polls` keeps the whole kernel to well under a second.
+__global__ void k_bounded_wait_selftest(int* status, uint32_t polls) {
+    __shared__ uint64_t bar;
+    if (threadIdx.x == 0) {
+        mbar_init(&bar, 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        const uint32_t addr = smem_u32(&bar);
+        bool done = false;
+        for (uint32_t it = 0; it < polls && !done; ++it) {
+            uint32_t ok;
+            asm volatile(
+                "{\n .reg .pred p;\n mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n selp.u32 %0, 1, 0, p;\n}\n"
+                : "=r"(ok) : "r"(addr), "r"(0u) : "memory");
+            done = ok != 0;
+        }
+        if (!done) *status = ABS_ETIMEOUT;
+    }
+}
+
 }  // namespace
+
+cudaError_t launch_bounded_wait_selftest(int* status, cudaStream_t stream) {
+    k_bounded_wait_selftest<<<1, 32, 0, stream>>>(status, 1u << 12);
+    return cudaGetLastError();
+}
 
 cudaError_t launch_sync_tma(const SyncArgs& a, int num_sms, cudaStream_t stream) {
     if (a.W < 1 || a.W > kSyncTmaMaxW || a.norm_out) return cudaErrorNotSupported;

@@ -59,3 +59,31 @@ def test_workspace_too_small_and_inconsistent_mlp_shape_rejected():
     assert not h.value
     bad = B.make_config(P=128 * 128 + 128 + 1280 + 10 + 1, W=2, lr=0.1, flags=B.FLAG_MLP, mlp=(128, 128, 10, 64))
     assert B.abs_workspace_bytes(bad) == 0                     # P does not match the MLP shape
+
+
+def test_a_wait_that_runs_out_is_reported_and_leaves_the_context_usable():
+    """The bounded device-side wait: a barrier that nothing completes makes the polling loop give up; the host
+    reads ABS_ETIMEOUT from abs_check once, and the same context then runs a normal step with correct results."""
+    import numpy as np
+    import torch
+
+    from paper_2308_15164_b200 import binding as B
+
+    dev = torch.device("cuda:0")
+    P = 5000
+    x0 = torch.ones(P, device=dev)
+    g = torch.full((P + 8,), 2.0, device=dev)
+    eng = B.AbsSgd(x0, 5, 0.1, pipelined=True)          # W = 5: the fused step is the bulk-copy pipeline
+    eng.check()
+    eng.selftest_timeout()
+    with pytest.raises(B.AbsError) as e:
+        eng.check()
+    assert e.value.code == B.ETIMEOUT
+    eng.check()                                          # reported once
+    for i in range(5):
+        eng.accumulate(i, g)
+    eng.sync_step(); eng.sync_step()
+    eng.check()
+    got = eng.params_host()
+    assert np.allclose(got, 1.0 - 0.1 * 2.0, rtol=0, atol=1e-6)
+    eng.destroy()
