@@ -576,7 +576,8 @@ cudaError_t launch_sync(const SyncArgs& a, int ctas_per_sm, int num_sms, cudaStr
     // W = 14 - 17 (ahead by 2 % at 40 M parameters and W = 16), behind for W <= 4 (6.0 against 6.7 TB/s), W = 8,
     // 11 and W >= 18.  It is the default where it is ahead or level; -2 asks for it wherever it can run.
     const bool bulk_default = (a.W >= 5 && a.W <= 7) || a.W == 9 || a.W == 10 || (a.W >= 12 && a.W <= 17);
-    if (ctas_per_sm == -2 || (ctas_per_sm == 0 && bulk_default && !a.norm_out)) {
+    const bool long_enough = a.n_vec >= (1ull << 18);   // short vectors are launch-bound: keep the lighter kernel
+    if (ctas_per_sm == -2 || (ctas_per_sm == 0 && bulk_default && long_enough && !a.norm_out)) {
         const cudaError_t e = launch_sync_tma(a, num_sms, stream);
         if (e != cudaErrorNotSupported) return e;
         ctas_per_sm = 0;

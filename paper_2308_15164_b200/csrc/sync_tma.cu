@@ -288,8 +288,16 @@ cudaError_t launch_sync_tma(const SyncArgs& a, int num_sms, cudaStream_t stream)
     if (stages < 2) return cudaErrorNotSupported;
     const int lazy = stages >= 3 ? 1 : 0;
     const size_t smem = fixed + (size_t)stages * stage_bytes;
-    cudaError_t e = cudaFuncSetAttribute(k_sync_tma, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)whole);
+    // the opt-in to large dynamic shared memory is per device: once each
+    static bool opted_in[64] = {};
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
     if (e != cudaSuccess) return e;
+    if (dev < 0 || dev >= 64 || !opted_in[dev]) {
+        e = cudaFuncSetAttribute(k_sync_tma, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)whole);
+        if (e != cudaSuccess) return e;
+        if (dev >= 0 && dev < 64) opted_in[dev] = true;
+    }
     const unsigned long long n_tiles = (a.n_vec * 4 + kTileElems - 1) / kTileElems;
     unsigned long long grid = (unsigned long long)num_sms * ctas;
     if (grid > n_tiles) grid = n_tiles;

@@ -73,7 +73,8 @@ def test_a_wait_that_runs_out_is_reported_and_leaves_the_context_usable():
     P = 5000
     x0 = torch.ones(P, device=dev)
     g = torch.full((P + 8,), 2.0, device=dev)
-    eng = B.AbsSgd(x0, 5, 0.1, pipelined=True)          # W = 5: the fused step is the bulk-copy pipeline
+    eng = B.AbsSgd(x0, 5, 0.1, pipelined=True)
+    eng.set_launch(B.K_SYNC, -2)                         # the fused step as the bulk-copy pipeline
     eng.check()
     eng.selftest_timeout()
     with pytest.raises(B.AbsError) as e:
