@@ -305,9 +305,14 @@ int launch_fused(abs_ctx* c, uint32_t set, int in, int out, uint64_t log_step, c
         a.norm_out = c->norm_log(log_step);
         a.norm_slots = (unsigned int)c->L.norm_slots;
     }
+    // Beside the MLP's gradient kernels (pipelined mode) the bulk-copy form is the better neighbour: it holds six
+    // warps per SM instead of every thread slot.  Measured on the 3072-4096-10 workload with batch calls: 16.9
+    // against 17.5 us per micro-batch, although alone on the GPU it is the slower one at W = 4.
+    int shape = c->ctas_per_sm[ABS_K_SYNC];
+    if (shape == 0 && c->mlp && c->pipelined) shape = -2;
     {
         Timed tm(c, ABS_K_SYNC, stream);
-        CK(launch_sync(a, c->ctas_per_sm[ABS_K_SYNC], c->num_sms, stream));
+        CK(launch_sync(a, shape, c->num_sms, stream));
     }
     c->launches += 1;
     return ABS_OK;
