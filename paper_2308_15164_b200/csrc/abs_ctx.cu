@@ -300,6 +300,7 @@ int launch_fused(abs_ctx* c, uint32_t set, int in, int out, uint64_t log_step, c
     a.shadow = c->mlp ? c->shadow(out) : nullptr;
     a.zero_acc = (c->cfg.flags & ABS_FLAG_OVERWRITE_FIRST) ? 0 : 1;
     a.status = reinterpret_cast<int*>(c->ticket() + 2);
+    a.overlapped = c->pipelined ? 1 : 0;
     if (c->grad_norm()) {
         a.norm_part = c->norm_part();
         a.norm_out = c->norm_log(log_step);

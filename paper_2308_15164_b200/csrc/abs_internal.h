@@ -39,6 +39,7 @@ struct SyncArgs {
     double* norm_part;        // optional: one slot per CTA for the partial sums of |Gbar|^2 ...
     double* norm_out;         // ... and where the last CTA puts the total (nullptr: the norm is not computed)
     unsigned int norm_slots;  // slots in norm_part
+    int overlapped;           // the launch runs beside the next iteration's accumulate kernels (pipelined mode)
     int* status;              // optional device status word (ABS_ETIMEOUT if a bounded wait of the bulk-copy kernel ran out)
 };
 // n (1..kMaxAccBatch) gradients of one worker added in one pass over its accumulator row, in list order.
