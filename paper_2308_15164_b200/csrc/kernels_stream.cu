@@ -572,14 +572,15 @@ cudaError_t launch_accumulate_multi(float* acc_row, const GradList& gl, int n, u
 
 cudaError_t launch_sync(const SyncArgs& a, int ctas_per_sm, int num_sms, cudaStream_t stream) {
     // The bulk-copy kernel (sync_tma.cu) gives the same bits; which form is faster depends on W and on whether
-    // the step runs alone or beside the next iteration's accumulate kernels (pipelined mode).  Measured on a B200:
-    //   alone (P = 11.7 M and 40 M): bulk copy ahead by 3 - 11 % for W = 5, 6, 9, 12, by 1 - 2 % for W = 7, 10, 13,
-    //     level for W = 14 - 17, behind for W <= 4 (6.0 against 6.7 TB/s), W = 8, 11 and W >= 18;
-    //   overlapped (whole pipelined iterations, P = 25.6 M, two micro-batches per worker): bulk copy ahead by 2 - 6 %
-    //     for W = 5, 7, 8, 9, 12, 13, 16 - 21, behind by 1 - 9 % for W <= 4, 6, 10, 11, 14, 15 and W >= 22.
+    // the step runs alone or beside the next iteration's accumulate kernels (pipelined mode).  Measured on a B200
+    // (P = 25.6 M, every W from 2 to 24):
+    //   alone: bulk copy ahead by 1 - 8 % for W = 5 - 7 and 9 - 17, behind by 3 - 10 % for W <= 4, by 3 % for W = 8
+    //     and W >= 18;
+    //   overlapped (whole pipelined iterations, two micro-batches per worker): bulk copy ahead by 2 - 6 % for
+    //     W = 5 - 21, level for W = 3, 4, behind for W = 2 and for W >= 22 (two stages of 100 KiB are too few).
     // Each table lists the W where the bulk-copy form is the default; -2 asks for it wherever it can run.
-    constexpr unsigned kBulkAlone = (1u << 5) | (1u << 6) | (1u << 7) | (1u << 9) | (1u << 10) | (0x3Fu << 12);
-    constexpr unsigned kBulkOverlapped = (1u << 5) | (1u << 7) | (1u << 8) | (1u << 9) | (1u << 12) | (1u << 13) | (0x3Fu << 16);
+    constexpr unsigned kBulkAlone = (0x7u << 5) | (0x1FFu << 9);          // 5 - 7, 9 - 17
+    constexpr unsigned kBulkOverlapped = 0x1FFFFu << 5;                   // 5 - 21
     const bool bulk_default = a.W < 32 && (((a.overlapped ? kBulkOverlapped : kBulkAlone) >> a.W) & 1u);
     const bool long_enough = a.n_vec >= (1ull << 18);   // short vectors are launch-bound: keep the lighter kernel
     if (ctas_per_sm == -2 || (ctas_per_sm == 0 && bulk_default && long_enough && !a.norm_out)) {

@@ -277,15 +277,18 @@ cudaError_t launch_sync_tma(const SyncArgs& a, int num_sms, cudaStream_t stream)
     if (a.W < 1 || a.W > kSyncTmaMaxW || a.norm_out) return cudaErrorNotSupported;
     const size_t stage_bytes = (size_t)(a.W + 2) * kTileBytes + kTileBytes / 2;
     const size_t fixed = kCtlBytes + kTileBytes;
-    // Three stages or more let a stage be released lazily (see the kernel).  Two CTAs per SM when three stages
-    // fit into half an SM's shared memory, else one CTA with as many stages as fit (at least two).
-    const size_t half = 112 * 1024, whole = 224 * 1024;
+    // Three stages or more let a stage be released lazily (see the kernel).  The stages of all CTAs of an SM
+    // together stay below 200 KiB: configurations that take (nearly) all of an SM's shared memory measured 5 - 12 %
+    // slower beside other kernels (W = 10, 11: four stages against three; W = 14, 15: three against two; W = 6: two
+    // CTAs of three against one of four) and no faster alone.  Two CTAs per SM when three stages each fit into that
+    // budget, else one CTA with up to four stages.
+    const size_t budget_sm = 200 * 1024, whole = 224 * 1024;
     int ctas = 2;
-    size_t budget = half;
-    if (fixed + 3 * stage_bytes > half) { ctas = 1; budget = whole; }
-    int stages = (int)((budget - fixed) / stage_bytes);
+    if (2 * (fixed + 3 * stage_bytes) > budget_sm) ctas = 1;
+    int stages = (int)((budget_sm / ctas - fixed) / stage_bytes);
     if (stages > kMaxStages) stages = kMaxStages;
-    if (stages < 2) return cudaErrorNotSupported;
+    if (stages < 2) stages = 2;
+    if (fixed + (size_t)stages * stage_bytes > whole) return cudaErrorNotSupported;
     const int lazy = stages >= 3 ? 1 : 0;
     const size_t smem = fixed + (size_t)stages * stage_bytes;
     // the opt-in to large dynamic shared memory is per device: once each
