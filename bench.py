@@ -642,7 +642,7 @@ def run_mlp(B, wlm, dev, peaks, iters=12):
         out[name] = res
 
     # K-batched variant: up to 4 consecutive reference batches of a worker per call, one K = 64 n dW1 GEMM
-    for bname, bvariant, ow in (("k_batched_up_to_4", 0, False), ("k_batched_up_to_4_ring", 4, False), ("k_batched_up_to_4_ring_128x64", 36, False),
+    for bname, bvariant, ow in (("k_batched_up_to_4", 0, False), ("k_batched_up_to_4_deep_pipelines", 128, False), ("k_batched_up_to_4_ring", 4, False), ("k_batched_up_to_4_ring_128x64", 36, False),
                                 ("k_batched_up_to_4_tile_per_cta", 8, False), ("k_batched_up_to_4_overwrite_first", 0, True), ("k_batched_up_to_4_cluster_fused_forward", 64, False)):
         out[bname] = run_mlp_batched(B, wlm, wl, d, x0_d, xp, yp, flop, rmw_bytes, peaks, bvariant, ow)
     return out

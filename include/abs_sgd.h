@@ -258,6 +258,9 @@ int abs_selftest_timeout(abs_ctx *ctx);
  *                  2 = forward GEMM on CUDA cores; 64 = forward GEMM on tcgen05 and its epilogue as ONE
  *                  kernel, split-K sums through a thread-block cluster's shared memory (default: two
  *                  kernels; the results are bit-identical).
+ *                  128 = forward GEMM and ring dW1 kernel always with their deep pipelines, which take a whole
+ *                  SM's shared memory (default: with W > 1, outside serial mode, their light forms of about
+ *                  100 KB, so that CTAs of different workers' calls share an SM; same results bit for bit).
  *   ABS_K_MLP_FWD  1 = serial mode: every kernel of a gradient call runs on stream_acc instead of the
  *                  worker's internal stream (for per-kernel timing). */
 int abs_set_launch(abs_ctx *ctx, int kernel_class, int ctas_per_sm);

@@ -334,8 +334,11 @@ int take_scratch_set(abs_ctx* c, bool serial, int* out) {
 // included).  deferred: the casts were launched, and counted, by earlier calls.
 int run_mlp_group(abs_ctx* c, uint32_t worker, int set, int n, bool first, bool deferred) {
     const int k = (int)(worker % (uint32_t)c->n_wstreams);
-    const int variant = c->ctas_per_sm[ABS_K_MLP_DW1];
+    int variant = c->ctas_per_sm[ABS_K_MLP_DW1];
     const bool serial = c->ctas_per_sm[ABS_K_MLP_FWD] == 1;
+    // With several workers' calls in flight the forward GEMM and the ring dW1 kernel run in their light
+    // shared-memory configurations (a CTA of each fits on one SM); alone, the deep pipelines are faster.
+    if (!serial && c->cfg.W > 1 && !(variant & 128)) variant |= kMlpLightBit;
     const MlpScratch& sc = c->mlp_scratch[set];
     cudaStream_t s_run = serial ? c->s_acc : c->s_w[k];
     if (!serial) {
@@ -1091,7 +1094,8 @@ int abs_selftest_timeout(abs_ctx* c) {
 
 int abs_set_launch(abs_ctx* c, int kernel_class, int ctas_per_sm) {
     if (!live(c)) return ABS_ESTATE;
-    if (kernel_class < 0 || kernel_class >= ABS_K_COUNT || ctas_per_sm < (kernel_class == ABS_K_SYNC ? -2 : -1) || ctas_per_sm > 64)
+    if (kernel_class < 0 || kernel_class >= ABS_K_COUNT || ctas_per_sm < (kernel_class == ABS_K_SYNC ? -2 : -1) ||
+        ctas_per_sm > (kernel_class == ABS_K_MLP_DW1 ? 255 : 64))
         return invalid(c, "bad kernel class or CTA count");
     if (int rc = flush_all(c)) return rc;
     c->ctas_per_sm[kernel_class] = ctas_per_sm;

@@ -710,22 +710,25 @@ __global__ void __launch_bounds__(256) k_dw1_regs(const __grid_constant__ CUtens
 // The accumulator slice never passes through the SM on its way in: no CTA ever waits for DRAM, the
 // only loads are the (L2-resident) bf16 operands.
 // ============================================================================================
-constexpr int kRingC = 2;                         // outgoing staging tiles of 32 KB (128 x 64 fp32)
-
 // kN = 64: 128 x 64 tiles (1536 of them at 3072 x 4096: even shares for 148 CTAs); kN = 128: 128 x 128 tiles, a
 // third less operand traffic per output element -- the choice for K-batched calls, which are bound by it.
-template <int kN>
+// kLight: half the operand slots and one outgoing staging tile (104 / 96 KB instead of 208 / 224 KB), so that a
+// forward-GEMM CTA of another worker's call fits on the same SM.  Alone on the GPU the deep form is faster
+// (K = 256: 20.5 against 24.7 us); with several workers' calls in flight the light forms are (16.5 -> 15.6 us per
+// micro-batch with batch calls), because forward and dW1 CTAs then run side by side instead of taking turns.
+template <int kN, bool kLight = false>
 struct DwRingCfg {
     static constexpr int kSlotBytes = kTileM * 128 + kN * 128;   // [A 128 x 64 | B kN x 64] bf16
-    static constexpr int kOps = kN == 64 ? 6 : 5;                 // operand slots
+    static constexpr int kOps = kLight ? (kN == 64 ? 3 : 2) : (kN == 64 ? 6 : 5);   // operand slots
+    static constexpr int kC = kLight ? 1 : 2;                    // outgoing staging tiles of 32 KB (128 x 64 fp32)
 };
 
-template <int kN>
+template <int kN, bool kLight = false>
 struct DwRingSmem {
-    alignas(1024) uint8_t op[DwRingCfg<kN>::kOps][DwRingCfg<kN>::kSlotBytes];   // swizzled 128-byte rows
-    alignas(1024) float c[kRingC][kTileM * kDwN];          // two [128][32] fp32 column panels each, swizzled rows
-    alignas(8) uint64_t op_full[DwRingCfg<kN>::kOps];
-    uint64_t op_empty[DwRingCfg<kN>::kOps];
+    alignas(1024) uint8_t op[DwRingCfg<kN, kLight>::kOps][DwRingCfg<kN, kLight>::kSlotBytes];   // swizzled 128-byte rows
+    alignas(1024) float c[DwRingCfg<kN, kLight>::kC][kTileM * kDwN];   // two [128][32] fp32 column panels each, swizzled rows
+    alignas(8) uint64_t op_full[DwRingCfg<kN, kLight>::kOps];
+    uint64_t op_empty[DwRingCfg<kN, kLight>::kOps];
     uint64_t acc_full[2];
     uint64_t acc_empty[2];
     uint32_t tmem_base;
@@ -733,15 +736,16 @@ struct DwRingSmem {
     uint32_t stop[2];
 };
 
-template <int kN>
+template <int kN, bool kLight = false>
 __global__ void __launch_bounds__(192) k_dw1_ring(const __grid_constant__ CUtensorMap tm_xt,
                                                   const __grid_constant__ CUtensorMap tm_dzt,
                                                   const __grid_constant__ CUtensorMap tm_acc, int n_tiles_n, int n_tiles,
                                                   int d_in, int ld, int nb, int store, int* status) {
-    constexpr int kRingOps = DwRingCfg<kN>::kOps, kSlotBytes = DwRingCfg<kN>::kSlotBytes;
+    constexpr int kRingOps = DwRingCfg<kN, kLight>::kOps, kSlotBytes = DwRingCfg<kN, kLight>::kSlotBytes;
+    constexpr int kRingC = DwRingCfg<kN, kLight>::kC;
     constexpr int kHalves = kN / kDwN;               // the epilogue works on 64-column pieces of the tile
     extern __shared__ uint8_t smem_raw[];
-    DwRingSmem<kN>& s = *reinterpret_cast<DwRingSmem<kN>*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+    DwRingSmem<kN, kLight>& s = *reinterpret_cast<DwRingSmem<kN, kLight>*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
     const int warp = threadIdx.x / 32, lane = threadIdx.x % 32;
     const int my_tiles = (n_tiles - (int)blockIdx.x + (int)gridDim.x - 1) / (int)gridDim.x;
 
@@ -884,31 +888,32 @@ __global__ void __launch_bounds__(192) k_dw1_ring(const __grid_constant__ CUtens
 // One CTA per (128-hidden tile, K split); a ring of TMA -> MMA stages streams the weights
 // once.  Warp 0 lane 0 issues TMA, warp 1 lane 0 issues MMAs, all four warps store D.
 // ============================================================================================
-template <int NB>
+// kLight: 2 - 3 stages (72 - 96 KB) instead of 4 - 6, so that a dW1 CTA of another worker's call fits beside it.
+template <int NB, bool kLight = false>
 struct FwdCfg {
-    static constexpr int kStages = NB <= 2 ? 6 : (NB == 3 ? 5 : 4);       // <= 200 KB of stages
+    static constexpr int kStages = kLight ? (NB <= 2 ? 3 : 2) : (NB <= 2 ? 6 : (NB == 3 ? 5 : 4));   // <= 200 KB of stages
     static constexpr int kStageBytes = 2 * 8192 + NB * 8192;              // two A boxes + NB B boxes
     static constexpr int kTmemCols = NB == 1 ? 64 : (NB == 2 ? 128 : 256);   // power of two >= 64 NB
 };
 
-template <int NB>
+template <int NB, bool kLight = false>
 struct FwdSmem {
-    alignas(1024) uint8_t stage[FwdCfg<NB>::kStages][FwdCfg<NB>::kStageBytes];   // [A h0..63 | A h64..127 | B x NB]
-    alignas(8) uint64_t full[FwdCfg<NB>::kStages];
-    uint64_t empty[FwdCfg<NB>::kStages];
+    alignas(1024) uint8_t stage[FwdCfg<NB, kLight>::kStages][FwdCfg<NB, kLight>::kStageBytes];   // [A h0..63 | A h64..127 | B x NB]
+    alignas(8) uint64_t full[FwdCfg<NB, kLight>::kStages];
+    uint64_t empty[FwdCfg<NB, kLight>::kStages];
     uint64_t done;
     uint32_t tmem_base;
     uint32_t failed;
 };
 
-template <int NB>
+template <int NB, bool kLight = false>
 __global__ void __launch_bounds__(128) k_fwd1_tcgen05(const __grid_constant__ CUtensorMap tm_w1,
                                                       const __grid_constant__ CUtensorMap tm_xb, float* __restrict__ zpart,
                                                       int d_in, int d_h, int* status) {
-    constexpr int kFwdStages = FwdCfg<NB>::kStages, kFwdStageBytes = FwdCfg<NB>::kStageBytes;
-    constexpr int kTmemCols = FwdCfg<NB>::kTmemCols;
+    constexpr int kFwdStages = FwdCfg<NB, kLight>::kStages, kFwdStageBytes = FwdCfg<NB, kLight>::kStageBytes;
+    constexpr int kTmemCols = FwdCfg<NB, kLight>::kTmemCols;
     extern __shared__ uint8_t smem_raw[];
-    FwdSmem<NB>& s = *reinterpret_cast<FwdSmem<NB>*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+    FwdSmem<NB, kLight>& s = *reinterpret_cast<FwdSmem<NB, kLight>*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
     const int warp = threadIdx.x / 32, lane = threadIdx.x % 32;
     const int h0 = blockIdx.x * 128;
     const int split = blockIdx.y;
@@ -1250,13 +1255,19 @@ cudaError_t fwd_fused_launch(int n_tiles, int nsplit, cudaStream_t stream, const
 
 template <int NB>
 cudaError_t fwd1_set_attr() {
-    return cudaFuncSetAttribute(k_fwd1_tcgen05<NB>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                (int)sizeof(FwdSmem<NB>) + 1024);
+    cudaError_t e = cudaFuncSetAttribute(k_fwd1_tcgen05<NB, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                         (int)sizeof(FwdSmem<NB, false>) + 1024);
+    if (e != cudaSuccess) return e;
+    return cudaFuncSetAttribute(k_fwd1_tcgen05<NB, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                (int)sizeof(FwdSmem<NB, true>) + 1024);
 }
 template <int NB>
-void fwd1_launch(dim3 grid, cudaStream_t stream, const CUtensorMap& tw, const CUtensorMap& tx, float* zpart, int d_in,
-                 int d_h, int* status) {
-    k_fwd1_tcgen05<NB><<<grid, 128, sizeof(FwdSmem<NB>) + 1024, stream>>>(tw, tx, zpart, d_in, d_h, status);
+void fwd1_launch(dim3 grid, cudaStream_t stream, bool light, const CUtensorMap& tw, const CUtensorMap& tx, float* zpart,
+                 int d_in, int d_h, int* status) {
+    if (light)
+        k_fwd1_tcgen05<NB, true><<<grid, 128, sizeof(FwdSmem<NB, true>) + 1024, stream>>>(tw, tx, zpart, d_in, d_h, status);
+    else
+        k_fwd1_tcgen05<NB, false><<<grid, 128, sizeof(FwdSmem<NB, false>) + 1024, stream>>>(tw, tx, zpart, d_in, d_h, status);
 }
 
 // ---- host helpers --------------------------------------------------------------------------
@@ -1358,9 +1369,13 @@ cudaError_t mlp_scratch_init(MlpScratch* s, const MlpDims& d, void* base, __nv_b
     cudaError_t e = cudaGetDevice(&dev);
     if (e == cudaSuccess) e = cudaDeviceGetAttribute(&s->num_sms, cudaDevAttrMultiProcessorCount, dev);
     if (e == cudaSuccess)
-        e = cudaFuncSetAttribute(k_dw1_ring<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(DwRingSmem<64>) + 1024);
+        e = cudaFuncSetAttribute(k_dw1_ring<64, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(DwRingSmem<64, false>) + 1024);
     if (e == cudaSuccess)
-        e = cudaFuncSetAttribute(k_dw1_ring<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(DwRingSmem<128>) + 1024);
+        e = cudaFuncSetAttribute(k_dw1_ring<128, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(DwRingSmem<128, false>) + 1024);
+    if (e == cudaSuccess)
+        e = cudaFuncSetAttribute(k_dw1_ring<64, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(DwRingSmem<64, true>) + 1024);
+    if (e == cudaSuccess)
+        e = cudaFuncSetAttribute(k_dw1_ring<128, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(DwRingSmem<128, true>) + 1024);
     if (e == cudaSuccess)
         e = cudaFuncSetAttribute(k_dw1_regs, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                  dw_regs_buf_bytes(kMaxBatch) + (int)sizeof(DwRegCtl) + 1024);
@@ -1404,6 +1419,7 @@ cudaError_t launch_mlp_front(const MlpDims& d, const MlpScratch& s, const float*
     const size_t o_b1 = (size_t)d.d_in * d.d_hidden, o_w2 = o_b1 + d.d_hidden, o_b2 = o_w2 + (size_t)d.d_hidden * d.d_out;
     cudaError_t e;
     const unsigned n_cta = d.d_hidden / kHB;
+    const bool light = (variant & kMlpLightBit) != 0;
 
     // every K split must be a whole number of 64-wide pipeline steps (d_in is a multiple of 128)
     const int nsplit = (d.d_in % (64 * kSplitK) == 0) ? kSplitK : 2;
@@ -1429,10 +1445,10 @@ cudaError_t launch_mlp_front(const MlpDims& d, const MlpScratch& s, const float*
         } else {
             const dim3 grid(d.d_hidden / 128, nsplit);
             switch (nb) {                                // the nb micro-batches are stacked along N of one GEMM
-                case 1: fwd1_launch<1>(grid, stream, *tw, *tx, s.zpart, d.d_in, d.d_hidden, s.status); break;
-                case 2: fwd1_launch<2>(grid, stream, *tw, *tx, s.zpart, d.d_in, d.d_hidden, s.status); break;
-                case 3: fwd1_launch<3>(grid, stream, *tw, *tx, s.zpart, d.d_in, d.d_hidden, s.status); break;
-                default: fwd1_launch<4>(grid, stream, *tw, *tx, s.zpart, d.d_in, d.d_hidden, s.status); break;
+                case 1: fwd1_launch<1>(grid, stream, light, *tw, *tx, s.zpart, d.d_in, d.d_hidden, s.status); break;
+                case 2: fwd1_launch<2>(grid, stream, light, *tw, *tx, s.zpart, d.d_in, d.d_hidden, s.status); break;
+                case 3: fwd1_launch<3>(grid, stream, light, *tw, *tx, s.zpart, d.d_in, d.d_hidden, s.status); break;
+                default: fwd1_launch<4>(grid, stream, light, *tw, *tx, s.zpart, d.d_in, d.d_hidden, s.status); break;
             }
         }
         k_fwd2<<<dim3(n_cta, nb), 256, 0, stream>>>(s.zpart, nsplit, x_pub + o_b1, shadow + o_w2, s.hbt, s.lpart, s.gpart,
@@ -1453,6 +1469,7 @@ cudaError_t launch_mlp_front(const MlpDims& d, const MlpScratch& s, const float*
 cudaError_t launch_mlp_dw1(const MlpDims& d, const MlpScratch& s, float* acc_row, const void* acc_tmap, int nb, bool store,
                            int variant, cudaStream_t stream, MlpMark mark, void* user) {
     const int st = store ? 1 : 0;
+    const bool light = (variant & kMlpLightBit) != 0;
     mark(user, ABS_K_MLP_DW1, 0, stream);
     const dim3 grid(d.d_hidden / kDwN, d.d_in / kTileM);
     const CUtensorMap* ta = reinterpret_cast<const CUtensorMap*>(&s.tmap_xt);
@@ -1468,13 +1485,21 @@ cudaError_t launch_mlp_dw1(const MlpDims& d, const MlpScratch& s, float* acc_row
         if (nb > 1 && !(variant & 32)) {   // K-batched: 128 x 128 tiles (bit 5 keeps 128 x 64)
             const int n_tiles_n = d.d_hidden / 128, n_tiles = n_tiles_n * (d.d_in / kTileM);
             const int ctas = n_tiles < s.num_sms ? n_tiles : s.num_sms;
-            k_dw1_ring<128><<<ctas, 192, sizeof(DwRingSmem<128>) + 1024, stream>>>(*ta, *tb, *tc, n_tiles_n, n_tiles, d.d_in,
-                                                                                   d.d_hidden, nb, st, s.status);
+            if (light)
+                k_dw1_ring<128, true><<<ctas, 192, sizeof(DwRingSmem<128, true>) + 1024, stream>>>(*ta, *tb, *tc, n_tiles_n, n_tiles,
+                                                                                                 d.d_in, d.d_hidden, nb, st, s.status);
+            else
+                k_dw1_ring<128, false><<<ctas, 192, sizeof(DwRingSmem<128, false>) + 1024, stream>>>(*ta, *tb, *tc, n_tiles_n, n_tiles,
+                                                                                                   d.d_in, d.d_hidden, nb, st, s.status);
         } else {
             const int n_tiles_n = d.d_hidden / kDwN, n_tiles = n_tiles_n * (d.d_in / kTileM);
             const int ctas = n_tiles < s.num_sms ? n_tiles : s.num_sms;
-            k_dw1_ring<64><<<ctas, 192, sizeof(DwRingSmem<64>) + 1024, stream>>>(*ta, *tb, *tc, n_tiles_n, n_tiles, d.d_in,
-                                                                                 d.d_hidden, nb, st, s.status);
+            if (light)
+                k_dw1_ring<64, true><<<ctas, 192, sizeof(DwRingSmem<64, true>) + 1024, stream>>>(*ta, *tb, *tc, n_tiles_n, n_tiles,
+                                                                                               d.d_in, d.d_hidden, nb, st, s.status);
+            else
+                k_dw1_ring<64, false><<<ctas, 192, sizeof(DwRingSmem<64, false>) + 1024, stream>>>(*ta, *tb, *tc, n_tiles_n, n_tiles,
+                                                                                                 d.d_in, d.d_hidden, nb, st, s.status);
         }
     } else if (kind == 8) {
         const size_t smem = dw_regs_buf_bytes(nb) + sizeof(DwRegCtl) + 1024;
