@@ -94,7 +94,7 @@ constexpr int kMlpMaxBatch = 4;
 // Internal bit of the `variant` argument below (set by the context, never by abs_set_launch): forward GEMM and ring
 // dW1 kernel in their light shared-memory configurations, so that CTAs of different workers' calls share an SM.
 constexpr int kMlpLightBit = 256;
-constexpr int kMlpStreams = 4;   // internal worker streams (worker i runs on stream i % kMlpStreams)
+constexpr int kMlpStreams = 8;   // internal worker streams (worker i runs on stream i % kMlpStreams)
 constexpr int kMlpSets = 8;      // scratch sets, one per call in flight, taken round-robin
 struct MlpDims {
     int d_in, d_hidden, d_out, mb;
