@@ -36,6 +36,11 @@ METRIC = "delayed-sync iteration HBM throughput (16 accumulate + 1 fused sync st
 UNIT = "GB/s"
 HBM_NOMINAL_GBS = 8000.0
 HBM_FALLBACK_GBS = 6650.0
+NVLINK_MEASURED_GBS = 770.0        # peer copy, per direction and GPU, measured on this machine
+# the same string in both arms: the workload the benchmark's metric is quoted on
+WORKLOAD = ("cfg2 resnet18-sized static heterogeneity: P=11689512 fp32 (62 tensors), W=4, b=(2,2,4,8), lr=0.1 mu=0.9 "
+            "wd=5e-4; one step = one iteration = 16 accumulate + 1 fused sync step")
+MIN_TIMED_SECONDS = 1.0            # the --steps-long region is repeated until this much time has been measured
 
 
 def measured_peaks():
@@ -55,8 +60,15 @@ class ClockSampler:
               "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
               "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
 
-    def __init__(self, gpu_index: int):
-        self.gpu = gpu_index
+    def __init__(self, local_rank: int):
+        # nvidia-smi takes an index or a UUID: with CUDA_VISIBLE_DEVICES set, the local rank's entry as it stands
+        self.gpu = str(local_rank)
+        try:
+            vis = [t.strip() for t in os.environ.get("CUDA_VISIBLE_DEVICES", "").split(",") if t.strip()]
+            if vis:
+                self.gpu = vis[local_rank]
+        except Exception:
+            pass
         self.proc = None
         self.path = None
         self.skip = 0
@@ -67,7 +79,7 @@ class ClockSampler:
             os.close(fd)
             self.proc = subprocess.Popen(
                 ["nvidia-smi", f"--id={self.gpu}", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits",
-                 "-lms", "50"], stdout=open(self.path, "w"), stderr=subprocess.DEVNULL)
+                 "-lms", "20"], stdout=open(self.path, "w"), stderr=subprocess.DEVNULL)
             # nvidia-smi takes a few hundred ms to start: wait for its first (idle) sample so that the
             # samples that follow fall inside the timed region
             t0 = time.time()
@@ -156,7 +168,7 @@ def run_reference(args):
         "impl": "reference", "metric": METRIC, "value": val, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": dt / args.steps * 1e3, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "f32", "data": "synthetic",
-        "config": {"workload": "cfg2 resnet18-sized: P=11689512, W=4, b=(2,2,4,8), full size, every step on the host"},
+        "config": {"workload": WORKLOAD, "where": "every step in full on the host cores (C oracle, OpenMP)"},
         "cpu_baseline": {"value": val, "unit": UNIT, "cores": cores, "kind": "oracle",
                          "sample": f"{args.steps} full iterations of the workload (C oracle, OpenMP)"},
         "e2e": {"value": val, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
@@ -183,8 +195,10 @@ def run_ours(args):
     pool = wlm.grad_pool(wl)                      # 16 x P fp32 = 748 MB (larger than the 126 MB L2)
     b_row = wlm.schedule(wl)[0]
     order = wlm.call_order(b_row)
+    n_acc_step = len(order)
     acc_b, sync_b = bytes_per_step(wl, b_row)
     step_bytes = acc_b + sync_b
+    per_acc = acc_b // n_acc_step
     pool_d = torch.from_numpy(pool).to(dev)
     x0_d = torch.from_numpy(x0).to(dev)
     torch.cuda.synchronize()
@@ -196,11 +210,14 @@ def run_ours(args):
     call_idx = [0]
     rows = [pool_d[r].data_ptr() for r in range(wl.pool_size)]      # raw device addresses of the pool rows
 
-    def one_step(eng):
+    def accumulates(eng):
         c = call_idx[0]
         for (i, k) in order:
             eng.accumulate(i, rows[c % wl.pool_size]); c += 1
         call_idx[0] = c
+
+    def one_step(eng):
+        accumulates(eng)
         eng.sync_step()
 
     def one_step_batched(eng):
@@ -215,36 +232,47 @@ def run_ours(args):
         eng.sync_step()
 
     def timed(eng, steps, warmup, one_step=one_step):
+        """`steps` steps between a barrier + synchronize on both sides, timed by CUDA events on stream_acc (the
+        stream every accumulate kernel is launched on).  Returns (seconds of the region, seconds from its start
+        to the end of the LAST ACCUMULATE kernel, launches)."""
         for _ in range(warmup):
             one_step(eng)
         eng.wait(); eng.synchronize()
         D.barrier(dev)
         torch.cuda.synchronize()
         n0 = eng.launch_count()
-        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0, e1, e2 = (torch.cuda.Event(enable_timing=True) for _ in range(3))
         with torch.cuda.stream(eng.stream_acc):
             e0.record()
             for _ in range(steps):
                 one_step(eng)
+            e1.record()                     # behind the last accumulate kernel; the last fused step may still run
             eng.wait()                      # stream_acc waits for the last fused kernel on stream_sync
-            e1.record()
+            e2.record()
         torch.cuda.synchronize()
         D.barrier(dev)
-        return e0.elapsed_time(e1) / 1e3, eng.launch_count() - n0
+        return e0.elapsed_time(e2) / 1e3, e0.elapsed_time(e1) / 1e3, eng.launch_count() - n0
 
-    # ---- pass 1: the timed region (pipelined, nothing instrumented) -------------------------
+    # ---- pass 1: the timed region (pipelined, nothing instrumented), repeated until >= MIN_TIMED_SECONDS ----
     eng = make(pipelined=True)
-    sampler = ClockSampler(local_rank if "CUDA_VISIBLE_DEVICES" not in os.environ else
-                           int(os.environ["CUDA_VISIBLE_DEVICES"].split(",")[local_rank]))
-    timed(eng, 2, args.warmup)              # warm-up (also outside the clock samples)
+    sampler = ClockSampler(local_rank)
+    secs_w, _, _ = timed(eng, max(args.steps // 10, 2), args.warmup)      # warm-up (outside the clock samples)
+    est = secs_w / max(args.steps // 10, 2)
+    repeats = int(min(max(1, np.ceil(MIN_TIMED_SECONDS / max(est * args.steps, 1e-9))), 200))
+    repeats = int(D.reduce_max(float(repeats), dev))                      # the same count on every rank
     sampler.start()
-    secs, launches = timed(eng, args.steps, 0)
+    regions = [timed(eng, args.steps, 0) for _ in range(repeats)]
     clocks = sampler.stop()
+    secs_all = sorted(r[0] for r in regions)
+    secs = float(np.median(secs_all))
+    acc_chain_secs = float(np.median([r[1] for r in regions]))
+    launches = regions[0][2]
     value, worst = D.aggregate_throughput(step_bytes * args.steps / 1e9, secs, dev)
 
-    # ---- pass 2: same region with an event pair around every launch -> per-kernel durations --
+    # ---- pass 2: same region with an event pair around every launch -> per-kernel durations (the events keep
+    # consecutive kernels from being chained, so this pass is slower than pass 1) --
     eng.profile(True)
-    timed(eng, args.steps, 1)
+    secs_p2, _, _ = timed(eng, args.steps, 1)
     n_acc, ms_acc = eng.kernel_stats(B.K_ACCUMULATE)
     n_syn, ms_syn = eng.kernel_stats(B.K_SYNC)
     eng.profile(False)
@@ -252,15 +280,29 @@ def run_ours(args):
 
     # ---- pass 3: eager mode (no overlap): each kernel class alone on the GPU ------------------
     eng = make(pipelined=False)
+    secs_eager, _, _ = timed(eng, args.steps, args.warmup)
+    # the accumulate kernel alone, back to back on its stream (64 launches over the workers' rows, pool cycled)
+    for rep_ in range(2):
+        eng.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        with torch.cuda.stream(eng.stream_acc):
+            e0.record()
+            for _ in range(4):
+                accumulates(eng)
+            e1.record()
+        torch.cuda.synchronize()
+    ms_chain, n_chain = e0.elapsed_time(e1), 4 * n_acc_step
+    eng.sync_step()
     eng.profile(True)
-    timed(eng, args.steps, args.warmup)
+    timed(eng, min(args.steps, 100), 2)
     n_acc_e, ms_acc_e = eng.kernel_stats(B.K_ACCUMULATE)
     n_syn_e, ms_syn_e = eng.kernel_stats(B.K_SYNC)
+    eng.profile(False)
     eng.destroy()
 
     # ---- pass 4: byte-saving variant (ABS_FLAG_OVERWRITE_FIRST): fewer bytes per step, same results -----
     eng = make(pipelined=True, overwrite_first=True)
-    secs_ow, _ = timed(eng, args.steps, args.warmup)
+    secs_ow, _, _ = timed(eng, args.steps, args.warmup)
     eng.destroy()
     w_act = int(sum(1 for b in b_row if b > 0))
     ow_bytes = (int(sum(b_row)) - w_act) * 12 * wl.P + w_act * 8 * wl.P + (4 * w_act + 16) * wl.P
@@ -269,7 +311,7 @@ def run_ours(args):
     batched = {}
     for name, ow in (("default_mode", False), ("overwrite_first", True)):
         eng = make(pipelined=True, overwrite_first=ow)
-        secs_b, launches_b = timed(eng, args.steps, args.warmup, one_step_batched)
+        secs_b, _, launches_b = timed(eng, args.steps, args.warmup, one_step_batched)
         eng.destroy()
         acc_bytes = sum((4 * int(b) + (4 if ow else 8)) * wl.P for b in b_row if b > 0)
         syn_bytes = ((4 if ow else 8) * w_act + 16) * wl.P
@@ -277,10 +319,9 @@ def run_ours(args):
                          "hbm_gbs_on_its_own_bytes": (acc_bytes + syn_bytes) * args.steps / secs_b / 1e9,
                          "step_time_vs_default": secs_b / secs, "launches_per_step": launches_b / args.steps}
 
-    # DRAM bytes (read + write) of ONE launch of each kernel at this workload's size, from an ncu capture of the
-    # current kernels (profiles/k_accumulate_resnet18_and_bf16.md, profiles/k_sync_w4_resnet18.md): a lone launch
-    # under the profiler, whose reads equal the algorithmic reads and whose writes partly stay in the 126 MB L2.
-    NCU_TRAFFIC = {"k_accumulate_f32": 93_522_432 + 2_617_088, "k_sync<4>": 280_577_024 + 217_864_192}
+    # DRAM bytes (read + write) of ONE launch of each kernel at this workload's size, from an ncu capture of a lone
+    # launch of the current kernels: reads equal the algorithmic reads, the writes partly stay in the 126 MB L2.
+    NCU_TRAFFIC = {"k_accumulate_f32": None, "k_sync<4>": None}
 
     def roof(alg_bytes, n, ms, name, note):
         ach = alg_bytes / (ms / n / 1e3) / 1e9 if n and ms > 0 else None
@@ -290,24 +331,51 @@ def run_ours(args):
                 "avg_us": ms / n * 1e3 if n else None, "launches": n, "algorithmic_bytes": alg_bytes,
                 "traffic": NCU_TRAFFIC.get(name) if wl.P == 11_689_512 else None, "how": note}
 
-    per_acc = 12 * wl.P
-    roofline = roof(per_acc, n_acc, ms_acc, "k_accumulate_f32",
-                    "CUDA events around every launch on stream_acc inside the pipelined timed region")
-    roofline_sync = roof(sync_b, n_syn, ms_syn, "k_sync<4>",
-                         "CUDA events around every launch on stream_sync inside the pipelined timed region "
-                         "(shares HBM with concurrent accumulate kernels)")
-    isolated = {"accumulate": roof(per_acc, n_acc_e, ms_acc_e, "k_accumulate_f32", "eager mode, kernel alone on the GPU"),
-                "sync": roof(sync_b, n_syn_e, ms_syn_e, "k_sync<4>", "eager mode, kernel alone on the GPU")}
+    # The dominant kernel inside the timed region: the 16 * steps accumulate launches are back to back on stream_acc
+    # (each waits for the one ahead; the fused step runs beside them on stream_sync), so their average duration is
+    # the event-timed span from the start of the region to the end of its last accumulate, divided by their number.
+    n_acc_region = n_acc_step * args.steps
+    roofline = roof(per_acc, n_acc_region, acc_chain_secs * 1e3, "k_accumulate_f32",
+                    "CUDA events on stream_acc around the timed region's accumulate launches (back to back on that stream, "
+                    "median over the repetitions); the fused step of the previous iteration runs concurrently on "
+                    "stream_sync and takes its share of the HBM bandwidth")
+    roofline["concurrent_kernel"] = {"kernel": "k_sync<4>", "algorithmic_bytes_per_step": sync_b,
+                                     "frac_of_both_kernels_together": value / world / peaks["hbm_gbs"]}
+    # 16 accumulate launches, one after the other, fit into a step of the same pass
+    assert n_acc_step * roofline["avg_us"] <= secs / args.steps * 1e6 * (1 + 1e-6), "per-kernel time does not reconcile with the step time"
+    in_step_pairs = {
+        "what": "the same pipelined region once more with an event pair around EVERY launch: the pairs keep consecutive "
+                "kernels from being chained, so this pass is slower than the timed one and is no part of the headline",
+        "ms_per_step": secs_p2 / args.steps * 1e3,
+        "accumulate": roof(per_acc, n_acc, ms_acc, "k_accumulate_f32", "event pair per launch on stream_acc, fused step concurrent"),
+        "sync": roof(sync_b, n_syn, ms_syn, "k_sync<4>", "event pair per launch on stream_sync, accumulate kernels concurrent")}
+    isolated = {
+        "accumulate": roof(per_acc, n_chain, ms_chain, "k_accumulate_f32",
+                           "eager mode, 64 launches back to back with nothing else on the GPU, one event pair around all of them"),
+        "accumulate_event_pair_per_launch": roof(per_acc, n_acc_e, ms_acc_e, "k_accumulate_f32",
+                                                 "eager mode, kernel alone on the GPU, event pair around each launch"),
+        "sync": roof(sync_b, n_syn_e, ms_syn_e, "k_sync<4>", "eager mode, kernel alone on the GPU, event pair around each launch"),
+        "eager_ms_per_step": secs_eager / args.steps * 1e3,
+        "eager_gbs": step_bytes * args.steps / secs_eager / 1e9}
+    sync_alone = isolated["sync"]
 
+    ms_step = worst / args.steps * 1e3
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
-        "ms_per_step": worst / args.steps * 1e3, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "f32", "data": "synthetic",
-        "config": {"workload": "cfg2 resnet18-sized: P=11689512 (62 tensors), W=4, b=(2,2,4,8), lr=0.1 mu=0.9 wd=5e-4",
-                   "mode": "pipelined (two streams)", "l2": "inputs larger than L2: gradient pool 748 MB cycled, "
-                   "accumulators 374 MB", "parallelism": f"replicas x{world}", "bytes_per_step": step_bytes},
+        "config": {"workload": WORKLOAD, "mode": "pipelined (two streams)", "l2": "inputs larger than L2: gradient pool "
+                   "748 MB cycled, accumulators 374 MB", "parallelism": f"replicas x{world}", "bytes_per_step": step_bytes},
+        "timing": {"repeats": repeats, "what": f"the {args.steps}-step region repeated {repeats} times (at least "
+                   f"{MIN_TIMED_SECONDS} s in all); ms_per_step and value are the median repetition",
+                   "ms_per_step_min": secs_all[0] / args.steps * 1e3, "ms_per_step_max": secs_all[-1] / args.steps * 1e3,
+                   "us_per_step_x_sm_mhz": (ms_step * 1e3 * clocks["sm_mhz"]) if clocks["sm_mhz"] else None},
         "frac_of_measured_hbm": value / world / peaks["hbm_gbs"],
-        "roofline": roofline, "roofline_sync": roofline_sync, "isolated": isolated,
+        "frac_of_nominal_8TBs": value / world / HBM_NOMINAL_GBS,
+        "sync_step_gbs": sync_alone["achieved"], "sync_step_us": sync_alone["avg_us"],
+        "sync_step_frac_of_measured_hbm": sync_alone["frac"], "sync_step_frac_of_nominal_8TBs": sync_alone["frac_of_nominal_8TBs"],
+        "sync_step_how": "the fused step alone on the GPU (eager mode), event pair around each launch, (8*4+16)*P bytes",
+        "roofline": roofline, "in_step_event_pairs": in_step_pairs, "isolated": isolated,
         "batched_accumulate_variant": dict(batched, what="abs_accumulate_batch: the b_i gradients of a worker in one "
                                            "pass over its accumulator row, (4 b_i + 8) instead of 12 b_i bytes per "
                                            "parameter; bit-identical results"),
@@ -320,8 +388,14 @@ def run_ours(args):
             "step_time_vs_default": secs_ow / secs},
     }
 
+    sections = args.sections.split(",")
+    if world > 1 or "global_step" in sections:
+        # Step 1 across the GPUs of this job (every rank takes part; rank 0 reports)
+        try:
+            line["global_step"] = run_global_step(B, D, wlm, wl, dev, rank, world, rows, min(args.steps, 50), peaks)
+        except Exception as exc:                       # the replica figure above stands on its own
+            line["global_step"] = {"error": f"{type(exc).__name__}: {exc}"}
     if rank == 0:
-        sections = args.sections.split(",")
         if "e2e" in sections:
             line["e2e"] = run_e2e(B, wlm, wl, x0_d, pool, order, step_bytes, min(args.steps, 10))
         if "cpu" in sections:
@@ -332,6 +406,8 @@ def run_ours(args):
             line["mlp"] = run_mlp(B, wlm, dev, peaks)
         if "tiny" in sections:
             line["tiny"] = run_tiny(B, wlm, dev)
+        if "schedules" in sections:
+            line["other_schedules"] = run_schedules(B, wlm, dev, peaks)
         if "workloads35" in sections:                 # opt-in: generating workload 5's gradient pool takes a while
             line["workloads_3_and_5"] = run_other_workloads(B, wlm, dev)
         if "sync_curve" in sections:
@@ -343,6 +419,68 @@ def run_ours(args):
         print(json.dumps(line), flush=True)
     D.barrier(dev)
     D.shutdown()
+
+
+def run_global_step(B, D, wlm, wl, dev, rank, world, rows, steps, peaks):
+    """Step 1 across the job's GPUs (the paper's own setting: Algorithm 1, Step 1 between workers on different
+    GPUs; dist.GlobalStep): the workload's W workers are spread over the G = world ranks (W / G local workers each when G
+    divides W, else one worker per rank with the b_i pattern repeated); per iteration a rank accumulates its own
+    workers' micro-batches and then takes part in the global step, whose kernel reads the peers' rows and writes the
+    peers' parameters through NVLink peer mappings.  Reported per rank: time per iteration (max over ranks), time of
+    the fused kernel alone (event pair on stream_sync), and its NVLink bytes in / out over that time against the
+    measured 770 GB/s per direction."""
+    import torch
+
+    G = world
+    Wl = wl.W // G if wl.W % G == 0 else 1
+    base = wlm.schedule(wl)[0]
+    b_all = [int(base[j % len(base)]) for j in range(G * Wl)]          # b_i of the global workers
+    mine = [(i, b_all[rank * Wl + i]) for i in range(Wl)]
+    x0_d = torch.from_numpy(wlm.params0(wl)).to(dev)
+    eng = B.AbsSgd(x0_d, Wl, wl.lr, wl.momentum, wl.weight_decay, pipelined=True)
+    step = D.GlobalStep(eng)
+    c = [rank * 5]
+
+    def one():
+        for (i, k) in wlm.call_order([b for _, b in mine]):
+            eng.accumulate(i, rows[c[0] % len(rows)]); c[0] += 1
+        return step.sync_step(timed=True)
+
+    for _ in range(3):
+        one()
+    eng.wait(); eng.synchronize()
+    D.barrier(dev)
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    pairs = []
+    with torch.cuda.stream(eng.stream_acc):
+        e0.record()
+        for _ in range(steps):
+            pairs.append(one())
+        eng.wait()
+        e1.record()
+    torch.cuda.synchronize()
+    D.barrier(dev)
+    secs = D.reduce_max(e0.elapsed_time(e1) / 1e3, dev)
+    k_us = D.reduce_max(float(np.median([a.elapsed_time(b) for a, b in pairs])) * 1e3, dev)
+    eng.check()
+    step.close()
+    eng.destroy()
+    P, R = wl.P, G * Wl
+    first, count = B.global_partition(P, G, rank)
+    nv_in = (G - 1) * Wl * 4 * count                   # the peers' rows of this rank's slice
+    nv_out = (G - 1) * (Wl + 1) * 4 * count            # zeros over them, and x' to every peer
+    hbm = (8 * R + 12 + 4 * G) * count                 # this GPU's kernel: local and remote bytes together
+    acc_bytes = sum(b for _, b in mine) * 12 * P
+    out = {"ranks": G, "workers_per_rank": Wl, "b_of_the_global_workers": b_all, "iterations": steps,
+           "us_per_iteration_max_over_ranks": secs / steps * 1e6,
+           "us_fused_kernel_max_over_ranks": k_us,
+           "nvlink_bytes_in_per_rank": nv_in, "nvlink_bytes_out_per_rank": nv_out,
+           "nvlink_gbs_in": nv_in / k_us / 1e3 if k_us > 0 else None, "nvlink_gbs_out": nv_out / k_us / 1e3 if k_us > 0 else None,
+           "nvlink_frac_of_770_out": (nv_out / k_us / 1e3 / NVLINK_MEASURED_GBS) if k_us > 0 and G > 1 else None,
+           "kernel_bytes_per_rank": hbm, "accumulate_bytes_per_rank_and_iteration": acc_bytes,
+           "whole_job_gbs": D.reduce_sum(float(acc_bytes + hbm), dev) * steps / secs / 1e9}
+    return out
 
 
 def run_other_workloads(B, wlm, dev):
@@ -576,11 +714,38 @@ def run_tiny(B, wlm, dev, iters=2000):
     return out
 
 
+def mlp_run_bytes(sched, d, P, max_batch, overwrite_first):
+    """Algorithmic HBM bytes of an MLP run over the schedule `sched` [T, W] when every worker hands over its b_i
+    micro-batches in calls of up to `max_batch`: per call the bf16 weights are streamed once (2 bytes per W1
+    element) and the W1 slice of the accumulator is written (4 bytes per element: the worker's first call of the
+    iteration stores) or read and written (8: later calls add); per micro-batch the bf16 operands of dW1; per
+    iteration the fused step, (8 W_act + 16 + 2) bytes per parameter (the 2: the bf16 copy of the new weights;
+    4 W_act + 18 when the step does not write zeros).  Returns (bytes, calls, stored calls, micro-batches)."""
+    w1 = d.d_in * d.d_hidden
+    total = calls = stored = mbs = 0
+    prev_active = 0
+    for b_row in sched:
+        if prev_active:
+            total += ((4 if overwrite_first else 8) * prev_active + 18) * P
+        for b in b_row:
+            left, first = int(b), True
+            while left > 0:
+                n = min(max_batch, left)
+                total += 2 * w1 + (4 if first else 8) * w1 + n * 2 * d.mb * (d.d_in + d.d_hidden)
+                calls += 1; stored += 1 if first else 0; mbs += n
+                left -= n; first = False
+        prev_active = int(sum(1 for b in b_row if b > 0))
+    return total, calls, stored, mbs
+
+
 def run_mlp(B, wlm, dev, peaks, iters=12):
-    """Secondary measurement on the MLP workload (3072-4096-10, W=4, b_i ~ U{1..8}): time per micro-batch
-    of the whole gradient (dW1 overlapping the next micro-batch's front part), and -- in serial mode, every
-    kernel alone on the GPU -- per-kernel-class durations, with the dW1 = X^T dZ GEMM (M=3072, N=4096, K=64)
-    as TFLOP/s and as HBM GB/s: with K = 64 it is bound by the read-modify-write of the fp32 accumulator."""
+    """The MLP workload (3072-4096-10, W=4, b_i ~ U{1..8}), pipelined: time per micro-batch of the whole run (all
+    workers' gradient calls overlapping on their streams, the fused step included) with single calls, with single
+    calls gathered by the library, and with batch calls of up to 4; each against the run's HBM floor (its
+    algorithmic bytes, see mlp_run_bytes, over the measured copy bandwidth).  In serial mode (every kernel alone on
+    the GPU, an event pair around each kernel group) also the per-kernel durations, with the dW1 = X^T dZ GEMM
+    (M=3072, N=4096, K=64 n) as TFLOP/s and as GB/s on the bytes its launches moved (4 bytes per W1 element when
+    the tile is stored, 8 when it is added to): at K = 64 n it is bound by that traffic, not by the tensor pipe."""
     import torch
 
     wl = wlm.config(4, T=iters)
@@ -592,114 +757,117 @@ def run_mlp(B, wlm, dev, peaks, iters=12):
     yp = [ys_d[b].data_ptr() for b in range(wl.mlp_pool)]
     torch.cuda.synchronize()
     calls = list(wlm.iter_calls(wl))
-    flop = 2.0 * d.d_in * d.d_hidden * d.mb
-    rmw_bytes = 8.0 * d.d_in * d.d_hidden + 2.0 * d.mb * (d.d_in + d.d_hidden)
+    sched = wlm.schedule(wl)
+    w1 = d.d_in * d.d_hidden
+    flop = 2.0 * w1 * d.mb
     out = {"workload": "cfg4 mlp 3072-4096-10, mb=64, W=4, b_i~U{1..8}, pipelined", "iterations": iters,
-           "dw1_flop": flop, "dw1_algorithmic_bytes": rmw_bytes}
-    for name, variant, coalesce in (("auto", 0, False), ("single_calls_gathered_by_the_library", 0, True), ("tma_load_add_store", 16, False),
-                                    ("tma_reduce_add", 1, False), ("persistent_ring", 4, False), ("register_prefetch", 8, False),
-                                    ("cluster_fused_forward", 64, False)):
-        res = {}
-        for serial in ((0,) if coalesce else (0, 1)):      # (serial mode runs every call at once: nothing to gather)
-            eng = B.AbsSgd(x0_d, wl.W, wl.lr, wl.momentum, wl.weight_decay, pipelined=True,
-                           mlp=(d.d_in, d.d_hidden, d.d_out, d.mb), mlp_coalesce=coalesce)
-            eng.set_launch(B.K_MLP_DW1, variant)
-            eng.set_launch(B.K_MLP_FWD, serial)
+           "dw1_flop_per_microbatch": flop}
 
-            def run(profile):
-                eng.profile(profile)
-                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-                n = 0
-                with torch.cuda.stream(eng.stream_acc):
-                    e0.record()
-                    for it in calls:
+    def run_case(max_batch, variant=0, coalesce=False, overwrite_first=False, serial=0):
+        eng = B.AbsSgd(x0_d, wl.W, wl.lr, wl.momentum, wl.weight_decay, pipelined=True, mlp=(d.d_in, d.d_hidden, d.d_out, d.mb),
+                       mlp_coalesce=coalesce, overwrite_first=overwrite_first)
+        eng.set_launch(B.K_MLP_DW1, variant)
+        eng.set_launch(B.K_MLP_FWD, serial)
+
+        def run(profile):
+            eng.profile(profile)
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            n_mb = 0
+            with torch.cuda.stream(eng.stream_acc):
+                e0.record()
+                if max_batch == 1:
+                    for it in calls:                     # the workload's interleaved arrival order
                         for (i, k, c) in it:
-                            eng.accumulate_mlp(i, xp[c % wl.mlp_pool], yp[c % wl.mlp_pool]); n += 1
+                            eng.accumulate_mlp(i, xp[c % wl.mlp_pool], yp[c % wl.mlp_pool]); n_mb += 1
                         eng.sync_step()
-                    eng.wait()
-                    e1.record()
-                torch.cuda.synchronize()
-                return e0.elapsed_time(e1), n
+                else:
+                    for b_row in sched:
+                        for i, b in enumerate(b_row):
+                            left = int(b)
+                            while left > 0:
+                                n = min(max_batch, left)
+                                p0 = (n_mb * 7) % (wl.mlp_pool - max_batch)
+                                eng.accumulate_mlp_batch(i, n, xp[p0], yp[p0]); left -= n; n_mb += n
+                        eng.sync_step()
+                eng.wait()
+                e1.record()
+            torch.cuda.synchronize()
+            return e0.elapsed_time(e1), n_mb
 
-            run(False)                                  # warm-up
-            ms_total, n_mb = run(False)
-            if not serial:
-                res["us_per_microbatch_overlapped"] = ms_total / n_mb * 1e3
-                res["microbatches"] = n_mb
-            else:
-                res["us_per_microbatch_serial"] = ms_total / n_mb * 1e3
-                run(True)
-                st = {nm: eng.kernel_stats(k) for nm, k in (("fwd", B.K_MLP_FWD), ("bwd", B.K_MLP_BWD),
-                                                            ("dw1", B.K_MLP_DW1), ("sync", B.K_SYNC))}
-                us = {nm: v[1] / max(v[0], 1) * 1e3 for nm, v in st.items()}
-                res.update({"us_fwd_3_kernels": us["fwd"], "us_bwd": us["bwd"], "us_dw1": us["dw1"], "us_sync": us["sync"],
-                            "dw1_tflops": flop / us["dw1"] / 1e6,
-                            "dw1_frac_of_bf16_peak_sustained": flop / us["dw1"] / 1e6 / peaks["bf16_tflops_sustained"],
-                            "dw1_hbm_gbs": rmw_bytes / us["dw1"] / 1e3,
-                            "dw1_frac_of_hbm": rmw_bytes / us["dw1"] / 1e3 / peaks["hbm_gbs"]})
-            eng.check()
-            eng.destroy()
-        out[name] = res
+        run(False)                                       # warm-up
+        ms = min(run(False)[0] for _ in range(3))
+        n_mb = run(False)[1]
+        res = {"us_per_microbatch": ms / n_mb * 1e3, "microbatches": n_mb}
+        if serial:
+            run(True)
+            st = {nm: eng.kernel_stats(k) for nm, k in (("fwd", B.K_MLP_FWD), ("bwd", B.K_MLP_BWD), ("dw1", B.K_MLP_DW1),
+                                                        ("sync", B.K_SYNC))}
+            us = {nm: v[1] / max(v[0], 1) * 1e3 for nm, v in st.items()}
+            _, n_calls, n_stored, _ = mlp_run_bytes(sched, d, wl.P, max_batch, overwrite_first)
+            dw1_bytes = ((4 * n_stored + 8 * (n_calls - n_stored)) * w1 + n_mb * 2 * d.mb * (d.d_in + d.d_hidden)) / n_calls
+            res.update({"us_cast_fwd1_fwd2_per_call": us["fwd"], "us_bwd_per_call": us["bwd"], "us_dw1_per_call": us["dw1"],
+                        "us_sync": us["sync"], "calls": n_calls, "calls_that_store": n_stored,
+                        "dw1_tflops": flop * n_mb / n_calls / us["dw1"] / 1e6,
+                        "dw1_frac_of_bf16_peak_sustained": flop * n_mb / n_calls / us["dw1"] / 1e6 / peaks["bf16_tflops_sustained"],
+                        "dw1_bytes_per_call": dw1_bytes, "dw1_hbm_gbs": dw1_bytes / us["dw1"] / 1e3,
+                        "dw1_frac_of_hbm": dw1_bytes / us["dw1"] / 1e3 / peaks["hbm_gbs"]})
+        else:
+            nbytes, n_calls, n_stored, _ = mlp_run_bytes(sched, d, wl.P, 4 if coalesce else max_batch, overwrite_first)
+            floor_us = nbytes / peaks["hbm_gbs"] / 1e3 / n_mb
+            res.update({"algorithmic_bytes_per_microbatch": nbytes / n_mb, "hbm_floor_us_per_microbatch": floor_us,
+                        "frac_of_hbm_floor": floor_us / res["us_per_microbatch"]})
+        eng.check()
+        eng.destroy()
+        return res
 
-    # K-batched variant: up to 4 consecutive reference batches of a worker per call, one K = 64 n dW1 GEMM
-    for bname, bvariant, ow in (("k_batched_up_to_4", 0, False), ("k_batched_up_to_4_deep_pipelines", 128, False), ("k_batched_up_to_4_ring", 4, False), ("k_batched_up_to_4_ring_128x64", 36, False),
-                                ("k_batched_up_to_4_tile_per_cta", 8, False), ("k_batched_up_to_4_overwrite_first", 0, True), ("k_batched_up_to_4_cluster_fused_forward", 64, False)):
-        out[bname] = run_mlp_batched(B, wlm, wl, d, x0_d, xp, yp, flop, rmw_bytes, peaks, bvariant, ow)
+    for name, kw in (("single_calls", dict(max_batch=1)),
+                     ("single_calls_gathered_by_the_library", dict(max_batch=1, coalesce=True)),
+                     ("batch_calls_up_to_4", dict(max_batch=4)),
+                     ("batch_calls_up_to_4_overwrite_first", dict(max_batch=4, overwrite_first=True)),
+                     ("batch_calls_up_to_4_deep_pipelines", dict(max_batch=4, variant=128))):
+        out[name] = run_case(**kw)
+    for name, kw in (("single_calls", dict(max_batch=1)), ("single_calls_ring_dw1", dict(max_batch=1, variant=4)),
+                     ("batch_calls_up_to_4", dict(max_batch=4)), ("batch_calls_up_to_4_tile_per_cta_dw1", dict(max_batch=4, variant=8))):
+        out["serial_" + name] = run_case(serial=1, **kw)
     return out
 
 
-def run_mlp_batched(B, wlm, wl, d, x0_d, xp, yp, flop, rmw_bytes, peaks, variant, overwrite_first):
+def run_schedules(B, wlm, dev, peaks, steps=200):
+    """Workload 2's vector with the paper's own static cluster (Section 6.1-6.2: iteration times in the ratio
+    1 : 2 : 3 : 4, so the workers finish 12, 6, 4 and 3 reference batches in the same span) beside the benchmark's
+    b = (2, 2, 4, 8): whole pipelined iterations, GB/s on each schedule's own algorithmic bytes."""
+    import dataclasses
+
     import torch
 
-    res = {}
-    for serial in (0, 1):
-        eng = B.AbsSgd(x0_d, wl.W, wl.lr, wl.momentum, wl.weight_decay, pipelined=True, mlp=(d.d_in, d.d_hidden, d.d_out, d.mb),
-                       overwrite_first=overwrite_first)
-        eng.set_launch(B.K_MLP_FWD, serial)
-        eng.set_launch(B.K_MLP_DW1, variant)
-        sched = wlm.schedule(wl)
-
-        def run_b(profile):
-            eng.profile(profile)
+    wl0 = wlm.config(2)
+    x0_d = torch.from_numpy(wlm.params0(wl0)).to(dev)
+    gen = torch.Generator(device=dev).manual_seed(7)
+    pool_d = torch.randn((16, wl0.P), device=dev, generator=gen)
+    rows = [pool_d[r].data_ptr() for r in range(16)]
+    out = {}
+    for name, b_row in (("b_2_2_4_8", (2, 2, 4, 8)), ("paper_static_cluster_b_12_6_4_3", (12, 6, 4, 3))):
+        wl = dataclasses.replace(wl0, sched_arg=tuple(b_row))
+        order = wlm.call_order(b_row)
+        acc_b, sync_b = bytes_per_step(wl, b_row)
+        eng = B.AbsSgd(x0_d, wl.W, wl.lr, wl.momentum, wl.weight_decay, pipelined=True)
+        c = 0
+        for rep_ in range(2):                              # the first round warms up
             e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-            n_mb = n_calls = 0
             with torch.cuda.stream(eng.stream_acc):
                 e0.record()
-                for b_row in sched:
-                    for i, b in enumerate(b_row):
-                        left = int(b)
-                        while left > 0:
-                            n = min(4, left)
-                            p0 = (n_mb * 7) % (wl.mlp_pool - 4)
-                            eng.accumulate_mlp_batch(i, n, xp[p0], yp[p0]); left -= n; n_mb += n; n_calls += 1
+                for _ in range(steps):
+                    for (i, k) in order:
+                        eng.accumulate(i, rows[c % 16]); c += 1
                     eng.sync_step()
                 eng.wait()
                 e1.record()
             torch.cuda.synchronize()
-            return e0.elapsed_time(e1), n_mb, n_calls
-
-        run_b(False)
-        ms_total, n_mb, n_calls = run_b(False)
-        if not serial:
-            res.update({"us_per_microbatch_overlapped": ms_total / n_mb * 1e3, "microbatches": n_mb, "calls": n_calls})
-        else:
-            res["us_per_microbatch_serial"] = ms_total / n_mb * 1e3
-            run_b(True)
-            n_dw, ms_dw = eng.kernel_stats(B.K_MLP_DW1)
-            us_dw = ms_dw / n_dw * 1e3
-            mean_n = n_mb / n_calls
-            for nm, k in (("us_fwd_3_kernels_per_call", B.K_MLP_FWD), ("us_bwd_per_call", B.K_MLP_BWD)):
-                n_k, ms_k = eng.kernel_stats(k)
-                res[nm] = ms_k / max(n_k, 1) * 1e3
-            n_sy, ms_sy = eng.kernel_stats(B.K_SYNC)
-            res["us_sync"] = ms_sy / max(n_sy, 1) * 1e3
-            res.update({"us_dw1_per_call": us_dw, "mean_microbatches_per_call": mean_n,
-                        "dw1_tflops": flop * mean_n / us_dw / 1e6,
-                        "dw1_frac_of_bf16_peak_sustained": flop * mean_n / us_dw / 1e6 / peaks["bf16_tflops_sustained"],
-                        "dw1_hbm_gbs": rmw_bytes / us_dw / 1e3, "dw1_frac_of_hbm": rmw_bytes / us_dw / 1e3 / peaks["hbm_gbs"]})
-        eng.check()
-        eng.destroy()
-    return res
+        ms = e0.elapsed_time(e1) / steps
+        out[name] = {"b": list(b_row), "us_per_iteration": ms * 1e3, "bytes_per_iteration": acc_b + sync_b,
+                     "gbs": (acc_b + sync_b) / ms / 1e6, "frac_of_measured_hbm": (acc_b + sync_b) / ms / 1e6 / peaks["hbm_gbs"]}
+        eng.check(); eng.destroy()
+    return out
 
 
 def run_e2e(B, wlm, wl, x0_d, pool, order, step_bytes, steps):
@@ -763,7 +931,7 @@ def main():
     ap.add_argument("--steps", type=int, default=1000)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--sections", default="e2e,cpu,mlp,tiny,batch_curve,sync_curve,global",
+    ap.add_argument("--sections", default="e2e,cpu,mlp,tiny,schedules,batch_curve,sync_curve,global",
                     help="extra measurements after the timed region (drop them for a profiler's launch list)")
     args = ap.parse_args()
     if args.warmup < 3:

@@ -93,6 +93,9 @@ extern "C" {
                                      (reproducible run to run).  No extra memory traffic beyond 8 bytes per CTA.
                                      Read it with abs_grad_norm2.  Not with abs_global_*.                        */
 
+#define ABS_FLAG_MLP_X_BF16 64u   /* with ABS_FLAG_MLP: abs_accumulate_mlp* take x_dev as bf16 values ([mlp_mb, mlp_in] row-major,
+                                     2 bytes each) instead of fp32; they enter the GEMMs as they are (no rounding step) */
+
 #define ABS_MAX_WORKERS 64u
 #define ABS_MAX_RANKS   16u   /* GPUs taking part in abs_global_* (n_ranks * W <= ABS_MAX_WORKERS)        */
 #define ABS_IPC_HANDLE_BYTES 64
@@ -103,7 +106,8 @@ extern "C" {
 #define ABS_K_MLP_FWD    2   /* MLP: operand cast, forward GEMM, loss gradient          */
 #define ABS_K_MLP_BWD    3   /* MLP: layer-2 backward, dZ, bias gradients               */
 #define ABS_K_MLP_DW1    4   /* MLP: dW1 = X^T dZ on tcgen05, accumulated into acc      */
-#define ABS_K_COUNT      5
+#define ABS_K_CHAIN      5   /* not a kernel: how consecutive kernels of a stream follow one another  */
+#define ABS_K_COUNT      6
 
 typedef struct abs_ctx abs_ctx;   /* opaque; host memory owned by the library */
 
@@ -160,23 +164,24 @@ int abs_accumulate_host(abs_ctx *ctx, uint32_t worker, const void *grad_host);
 /* Algorithm 1, Step 2 with the gradient computed here: forward and backward pass of the
  * 2-layer ReLU MLP with mean softmax cross-entropy on one micro-batch, evaluated at the
  * current parameters x_t, and accumulated into worker `worker`'s buffer; b_i += 1.
- * x_dev: [mlp_mb, mlp_in] fp32 row-major; y_dev: [mlp_mb] int32 class indices in
- * [0, mlp_out).  GEMM operands are rounded to bf16 (nearest even) with fp32 accumulation;
+ * x_dev: [mlp_mb, mlp_in] row-major, fp32 (bf16 with ABS_FLAG_MLP_X_BF16), 16-byte aligned; y_dev: [mlp_mb]
+ * int32 class indices in [0, mlp_out).  GEMM operands are rounded to bf16 (nearest even) with fp32 accumulation;
  * dW1 = X^T dZ runs on the tcgen05 tensor cores and its epilogue adds into the accumulator.
  * Needs ABS_FLAG_MLP.  x_dev and y_dev are read by the first kernel only, which is enqueued on stream_acc
  * (they may be reused by later work on that stream).  The remaining kernels run on an internal stream of
  * the worker (workers compute concurrently, as in the paper; calls of one worker stay in call order), which
  * starts after everything enqueued on stream_acc so far; abs_sync_step, abs_wait, abs_check, abs_accumulate,
  * abs_accumulate_host and abs_accumulator make stream_acc wait for all of them. */
-int abs_accumulate_mlp(abs_ctx *ctx, uint32_t worker, const float *x_dev, const int32_t *y_dev);
+int abs_accumulate_mlp(abs_ctx *ctx, uint32_t worker, const void *x_dev, const int32_t *y_dev);
 
 /* n (1..4) consecutive reference batches of one worker in one call: the same computation as n calls of
  * abs_accumulate_mlp (forward, loss and backward of every micro-batch at x_t; b_i += n), but the n dW1
  * products are contracted by ONE tcgen05 GEMM with K = 64 n, so the worker's fp32 accumulator slice is
  * read and written once instead of n times -- that traffic, not the MMAs, bounds the kernel.  The sum
  * over the n micro-batches is formed in the fp32 TMEM accumulator, so results agree with n single
- * calls to fp32 rounding, not bit for bit.  x_dev: [n][mlp_mb][mlp_in] fp32; y_dev: [n][mlp_mb] int32. */
-int abs_accumulate_mlp_batch(abs_ctx *ctx, uint32_t worker, uint32_t n, const float *x_dev, const int32_t *y_dev);
+ * calls to fp32 rounding, not bit for bit.  x_dev: [n][mlp_mb][mlp_in] fp32 (bf16 with ABS_FLAG_MLP_X_BF16);
+ * y_dev: [n][mlp_mb] int32. */
+int abs_accumulate_mlp_batch(abs_ctx *ctx, uint32_t worker, uint32_t n, const void *x_dev, const int32_t *y_dev);
 
 /* Algorithm 1, Step 1 + compensation + "Update parameters" + t = t + 1 (see the file header).
  * Without ABS_FLAG_PIPELINED the fused kernel runs on stream_acc.  With it, the call makes
@@ -251,18 +256,18 @@ int abs_selftest_timeout(abs_ctx *ctx);
  * kernel variants instead (results agree within rounding):
  *   ABS_K_MLP_DW1  bit mask.  dW1 kernel: 0 = chosen per call (the persistent ring kernel when the tile is
  *                  stored or the call is K-batched, the register-prefetch kernel for single adds);
- *                  1 = one tile per CTA, TMA reduce-add epilogue; 16 = one tile per CTA, TMA load + add +
- *                  TMA store; 4 = persistent warp-specialised ring kernel (TMA store / reduce-add);
+ *                  4 = persistent warp-specialised ring kernel (TMA store / reduce-add);
  *                  8 = one tile per CTA, accumulator tile prefetched into registers.
  *                  32 = the ring kernel keeps 128 x 64 tiles for K-batched calls (default there: 128 x 128).
- *                  2 = forward GEMM on CUDA cores; 64 = forward GEMM on tcgen05 and its epilogue as ONE
- *                  kernel, split-K sums through a thread-block cluster's shared memory (default: two
- *                  kernels; the results are bit-identical).
  *                  128 = forward GEMM and ring dW1 kernel always with their deep pipelines, which take a whole
  *                  SM's shared memory (default: with W > 1, outside serial mode, their light forms of about
  *                  100 KB, so that CTAs of different workers' calls share an SM; same results bit for bit).
  *   ABS_K_MLP_FWD  1 = serial mode: every kernel of a gradient call runs on stream_acc instead of the
- *                  worker's internal stream (for per-kernel timing). */
+ *                  worker's internal stream (for per-kernel timing).
+ *   ABS_K_CHAIN    0 = consecutive kernels of a stream are chained by programmatic dependent launch: the next
+ *                  kernel is made resident and does its set-up while the one ahead drains, and waits on the
+ *                  device for that one's completion before it reads anything it wrote (default; same results);
+ *                  1 = plain stream order. */
 int abs_set_launch(abs_ctx *ctx, int kernel_class, int ctas_per_sm);
 
 /* Per-kernel timing with CUDA events on the launching stream.  abs_profile(ctx, 1) starts
@@ -271,6 +276,22 @@ int abs_set_launch(abs_ctx *ctx, int kernel_class, int ctas_per_sm);
  * profiling was switched on (or last reset by abs_profile(ctx, 1)). */
 int abs_profile(abs_ctx *ctx, int enable);
 int abs_kernel_stats(abs_ctx *ctx, int kernel_class, uint64_t *launches, double *total_ms);
+
+/* Timeline of the timed launches.  abs_profile(ctx, 2) records, besides the totals, when each timed kernel (or
+ * kernel group of a gradient call) started and stopped, in microseconds since the moment stream_acc reached the
+ * abs_profile call.  stream: 0 = stream_acc, 1 = stream_sync, 2 + k = internal worker stream k.  A span starts
+ * when its stream reaches the kernel (the kernel may still queue for SM resources behind other streams' kernels)
+ * and ends when the kernel has finished, so overlapping spans of different streams show which kernels really ran
+ * side by side.  abs_profile_timeline blocks until the recorded work has finished, writes up to `capacity` spans
+ * to `out` (may be NULL) in launch order and the number recorded so far to *n. */
+typedef struct abs_span {
+    int32_t kernel_class;   /* ABS_K_* */
+    int32_t stream;
+    int32_t part;           /* ordinal of the kernel within its class for one gradient call (ABS_K_MLP_FWD: 0 = operand
+                               cast, 1 = forward GEMM, 2 = bias / ReLU / partial logits); 0 otherwise */
+    float start_us, stop_us;
+} abs_span;
+int abs_profile_timeline(abs_ctx *ctx, abs_span *out, size_t capacity, size_t *n);
 
 /* Number of kernels this context has launched since abs_init. */
 uint64_t abs_launch_count(abs_ctx *ctx);
@@ -386,8 +407,14 @@ int abs_state_import(abs_ctx *ctx, const void *src_host, size_t bytes);
  *   row_stride, P  in elements; both multiples of 4, row_stride >= P
  *   cnt_dev        W int32 device counters b_i (input, cleared on output)
  *   stream         cudaStream_t (NULL = default stream)
+ * All four buffers and the stream must belong to the CURRENT device (the built-in array used is the current
+ * device's copy); buffers of another device, or host pointers, return ABS_EINVAL.
  * Limit: W <= 64 (what the built-in working memory can log); larger W returns ABS_ELIMIT and
  * nothing is launched.  Other bad arguments return ABS_EINVAL, CUDA failures ABS_ECUDA.
+ * The step always runs the load/store form of the fused kernel (never the bulk-copy form abs_sync_step picks
+ * for some worker counts): that form has no device-side wait that could run out, so a call that returned
+ * ABS_OK either completes in full or shows up as a CUDA error on the stream.  Results equal abs_sync_step's
+ * bit for bit (both forms compute the same bits).
  *
  * The first call on each device looks up the device address of the built-in array (one
  * cudaGetSymbolAddress, no allocation); make that first call outside any stream capture.

@@ -142,7 +142,8 @@ def mlp_loss_and_grad(flat_params, X, y, d_in, d_hidden, d_out, mode="exact", re
     relu_flip:    (row, hidden) entries whose ReLU gate is inverted.  Tests use it to
                   enumerate the valid outcomes when a pre-activation is so close to zero
                   that fp32 and fp64 accumulation may disagree about its sign.
-    Returns (loss, grad_flat fp64, aux) with aux = {"Z": pre-activations}.
+    Returns (loss, grad_flat fp64, aux); aux holds intermediates (Z: pre-activations, dL: gradient of the loss
+    w.r.t. the logits, dH: gradient w.r.t. the hidden activations, X: the first-layer operand as used).
     """
     p = np.asarray(flat_params, dtype=np.float32).astype(np.float64)   # fp32 master weights
     W1, b1, W2, b2 = mlp_split(p, d_in, d_hidden, d_out)
@@ -175,4 +176,4 @@ def mlp_loss_and_grad(flat_params, X, y, d_in, d_hidden, d_out, mode="exact", re
     dZo = rnd(dZ)
     dW1 = Xo.T @ dZo
     grad = np.concatenate([dW1.ravel(), db1, dW2.ravel(), db2])
-    return loss, grad, {"Z": Z, "dH": dH, "X": Xo}
+    return loss, grad, {"Z": Z, "dH": dH, "X": Xo, "dL": dL}

@@ -26,8 +26,8 @@ lib = ctypes.CDLL(LIB_PATH)
 
 OK, EINVAL, ESTATE, ECUDA, ENOMEM, ETIMEOUT, ELIMIT = 0, -1, -2, -3, -4, -5, -6
 GRAD_F32, GRAD_BF16 = 0, 1
-FLAG_PIPELINED, FLAG_MLP, FLAG_HOST_INPUT, FLAG_OVERWRITE_FIRST, FLAG_MLP_COALESCE, FLAG_GRAD_NORM = 1, 2, 4, 8, 16, 32
-K_ACCUMULATE, K_SYNC, K_MLP_FWD, K_MLP_BWD, K_MLP_DW1 = range(5)
+FLAG_PIPELINED, FLAG_MLP, FLAG_HOST_INPUT, FLAG_OVERWRITE_FIRST, FLAG_MLP_COALESCE, FLAG_GRAD_NORM, FLAG_MLP_X_BF16 = 1, 2, 4, 8, 16, 32, 64
+K_ACCUMULATE, K_SYNC, K_MLP_FWD, K_MLP_BWD, K_MLP_DW1, K_CHAIN = range(6)
 MAX_WORKERS, MAX_RANKS, IPC_HANDLE_BYTES = 64, 16, 64
 KERNEL_NAMES = ["accumulate", "sync", "mlp_fwd", "mlp_bwd", "mlp_dw1"]
 
@@ -42,6 +42,11 @@ class AbsConfig(ctypes.Structure):
         ("mlp_mb", ctypes.c_uint32),
         ("stream_acc", ctypes.c_void_p), ("stream_sync", ctypes.c_void_p),
     ]
+
+
+class AbsSpan(ctypes.Structure):
+    _fields_ = [("kernel_class", ctypes.c_int32), ("stream", ctypes.c_int32), ("part", ctypes.c_int32),
+                ("start_us", ctypes.c_float), ("stop_us", ctypes.c_float)]
 
 
 class AbsPeerTable(ctypes.Structure):
@@ -73,6 +78,7 @@ _sig = {
     "abs_set_launch": (ctypes.c_int, [_vp, ctypes.c_int, ctypes.c_int]),
     "abs_profile": (ctypes.c_int, [_vp, ctypes.c_int]),
     "abs_kernel_stats": (ctypes.c_int, [_vp, ctypes.c_int, ctypes.POINTER(_u64), ctypes.POINTER(ctypes.c_double)]),
+    "abs_profile_timeline": (ctypes.c_int, [_vp, ctypes.POINTER(AbsSpan), ctypes.c_size_t, ctypes.POINTER(ctypes.c_size_t)]),
     "abs_launch_count": (ctypes.c_uint64, [_vp]),
     "abs_last_error": (ctypes.c_char_p, [_vp]),
     "abs_destroy": (ctypes.c_int, [_vp]),
@@ -134,14 +140,14 @@ class AbsSgd:
 
     def __init__(self, params0: torch.Tensor, W: int, lr: float, momentum=0.0, weight_decay=0.0, lambda_dc=0.0,
                  grad_dtype=GRAD_F32, pipelined=False, mlp=None, host_input=False, overwrite_first=False,
-                 mlp_coalesce=False, grad_norm=False, stream_acc: Optional[torch.cuda.Stream] = None, stream_sync: Optional[torch.cuda.Stream] = None,
+                 mlp_coalesce=False, grad_norm=False, mlp_x_bf16=False, stream_acc: Optional[torch.cuda.Stream] = None, stream_sync: Optional[torch.cuda.Stream] = None,
                  workspace: Optional[torch.Tensor] = None):
         assert params0.is_cuda and params0.dtype == torch.float32 and params0.is_contiguous()
         self.device = params0.device
         self.P, self.W = params0.numel(), W
         self.stream_acc = stream_acc or torch.cuda.Stream(device=self.device)
         self.stream_sync = stream_sync or (torch.cuda.Stream(device=self.device) if pipelined else None)
-        flags = (FLAG_PIPELINED if pipelined else 0) | (FLAG_MLP if mlp else 0) | (FLAG_HOST_INPUT if host_input else 0) | (FLAG_OVERWRITE_FIRST if overwrite_first else 0) | (FLAG_MLP_COALESCE if mlp_coalesce else 0) | (FLAG_GRAD_NORM if grad_norm else 0)
+        flags = (FLAG_PIPELINED if pipelined else 0) | (FLAG_MLP if mlp else 0) | (FLAG_HOST_INPUT if host_input else 0) | (FLAG_OVERWRITE_FIRST if overwrite_first else 0) | (FLAG_MLP_COALESCE if mlp_coalesce else 0) | (FLAG_GRAD_NORM if grad_norm else 0) | (FLAG_MLP_X_BF16 if mlp_x_bf16 else 0)
         self.cfg = make_config(self.P, W, lr, momentum, weight_decay, lambda_dc, grad_dtype, flags, mlp,
                                self.stream_acc.cuda_stream, self.stream_sync.cuda_stream if self.stream_sync else 0)
         nbytes = abs_workspace_bytes(self.cfg)
@@ -285,8 +291,17 @@ class AbsSgd:
     def set_launch(self, kernel_class: int, ctas_per_sm: int):
         self._ck(lib.abs_set_launch(self._h, kernel_class, ctas_per_sm))
 
-    def profile(self, enable: bool):
+    def profile(self, enable):
+        """False / True: per-kernel totals; 2: the timeline of the timed launches as well (profile_timeline)."""
         self._ck(lib.abs_profile(self._h, int(enable)))
+
+    def profile_timeline(self):
+        """[(kernel class name, part, stream, start_us, stop_us), ...] of the launches timed since profile(2)."""
+        n = ctypes.c_size_t(0)
+        self._ck(lib.abs_profile_timeline(self._h, None, 0, ctypes.byref(n)))
+        buf = (AbsSpan * max(n.value, 1))()
+        self._ck(lib.abs_profile_timeline(self._h, buf, n.value, ctypes.byref(n)))
+        return [(KERNEL_NAMES[b.kernel_class], b.part, b.stream, b.start_us, b.stop_us) for b in buf[:n.value]]
 
     def kernel_stats(self, kernel_class: int):
         n, ms = _u64(0), ctypes.c_double(0.0)
@@ -318,8 +333,9 @@ def sync_step_noalloc(x: torch.Tensor, v: torch.Tensor, acc: torch.Tensor, cnt: 
     """abs_sync_step_noalloc on caller-owned tensors: x, v fp32 [P]; acc fp32 [W, row_stride]; cnt int32 [W].
     Returns the status code (no exception), so callers can test for ELIMIT / EINVAL."""
     s = stream.cuda_stream if stream is not None else torch.cuda.current_stream(x.device).cuda_stream
-    return int(lib.abs_sync_step_noalloc(x.data_ptr(), v.data_ptr(), acc.data_ptr(), acc.stride(0), x.numel(),
-                                         acc.shape[0], cnt.data_ptr(), lr, momentum, weight_decay, s))
+    with torch.cuda.device(x.device):             # the entry point works on the current device
+        return int(lib.abs_sync_step_noalloc(x.data_ptr(), v.data_ptr(), acc.data_ptr(), acc.stride(0), x.numel(),
+                                             acc.shape[0], cnt.data_ptr(), lr, momentum, weight_decay, s))
 
 
 def global_partition(P: int, n_ranks: int, rank: int) -> tuple:

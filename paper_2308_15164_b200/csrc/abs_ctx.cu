@@ -18,10 +18,13 @@ using namespace abs_sgd;
 namespace {
 
 constexpr uint32_t kMagic = 0xAB55D6D0u;
+constexpr size_t kMaxSpans = 1u << 20;
 
 struct TimedLaunch {
     int kernel_class;
     cudaEvent_t start, stop;
+    cudaStream_t stream;
+    int part;
 };
 
 size_t round_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
@@ -41,9 +44,10 @@ bool config_ok(const abs_config* c, std::string* why) {
     if (c->W == 0 || c->W > ABS_MAX_WORKERS) return fail("W must be in 1..64");
     if (c->grad_dtype != ABS_GRAD_F32 && c->grad_dtype != ABS_GRAD_BF16) return fail("unknown grad_dtype");
     if (c->flags & ~(ABS_FLAG_PIPELINED | ABS_FLAG_MLP | ABS_FLAG_HOST_INPUT | ABS_FLAG_OVERWRITE_FIRST | ABS_FLAG_MLP_COALESCE |
-                     ABS_FLAG_GRAD_NORM))
+                     ABS_FLAG_GRAD_NORM | ABS_FLAG_MLP_X_BF16))
         return fail("unknown flag bits");
     if ((c->flags & ABS_FLAG_MLP_COALESCE) && !(c->flags & ABS_FLAG_MLP)) return fail("ABS_FLAG_MLP_COALESCE needs ABS_FLAG_MLP");
+    if ((c->flags & ABS_FLAG_MLP_X_BF16) && !(c->flags & ABS_FLAG_MLP)) return fail("ABS_FLAG_MLP_X_BF16 needs ABS_FLAG_MLP");
     if (!std::isfinite(c->lr) || !std::isfinite(c->momentum) || !std::isfinite(c->weight_decay) ||
         !std::isfinite(c->lambda_dc))
         return fail("lr, momentum, weight_decay and lambda_dc must be finite");
@@ -135,13 +139,33 @@ struct abs_ctx {
     cudaEvent_t ev_stage_free[2] = {nullptr, nullptr}, ev_stage_full[2] = {nullptr, nullptr};
     bool stage_used[2] = {false, false};
     int stage_next = 0;
-    int ctas_per_sm[ABS_K_COUNT] = {0, 0, 0, 0, 0};
+    int ctas_per_sm[ABS_K_COUNT] = {0, 0, 0, 0, 0, 0};
+    // consecutive kernels of a stream are chained by programmatic dependent launch (abs_set_launch(ABS_K_CHAIN, 1): off)
+    bool chained() const { return ctas_per_sm[ABS_K_CHAIN] == 0; }
+    // the gradient kernels of the MLP: which of them are chained (kChain* bits); nb = micro-batches of the call
+    int mlp_chain(bool serial, int nb) const {
+        if (!chained()) return 0;
+        // Measured (3072-4096-10, W = 4): with every kernel of a call alone on the GPU the whole chain gains (55 -> 50 us
+        // per single call, 73 -> 69 per batch call).  With several workers' calls in flight the gaps are filled by the
+        // other workers' kernels anyway, and a forward or dW1 CTA that is resident early only holds shared memory and
+        // TMEM another worker's kernel could use: there only the two small kernels of single calls are chained
+        // (33.4 -> 32.2 us per micro-batch; K-batched calls measured best with none: 15.5 against 15.7 - 16.1).
+        if (serial || cfg.W == 1) return kChainCast | kChainFwd1 | kChainFwd2 | kChainBwd | kChainDw1;
+        return nb == 1 ? (kChainFwd2 | kChainBwd) : 0;
+    }
+    bool x_bf16() const { return (cfg.flags & ABS_FLAG_MLP_X_BF16) != 0; }
     MlpDims mlp_dims{0, 0, 0, 0};
     // The paper's workers compute concurrently: the gradient kernels of worker i run on internal stream
     // i % n_wstreams (calls of one worker stay in order: its accumulator is added to in call order), each call
     // in its own scratch set, taken round-robin.
     MlpScratch mlp_scratch[kMlpSets]{};
     cudaStream_t s_w[kMlpStreams] = {};
+    // The dW1 GEMM of a call runs on a second stream of the worker, one priority level below: the worker's next
+    // call (forward, loss, backward: short, latency-bound kernels that only touch the bias / W2 slices of the row)
+    // overlaps it, and the short kernels of every worker get free CTA slots before the HBM-bound GEMMs.
+    cudaStream_t s_d[kMlpStreams] = {};
+    cudaEvent_t ev_front[kMlpStreams] = {};        // front kernels of the newest call on s_w[k] have finished
+    bool gemm_on_d[kMlpStreams] = {};              // where the newest dW1 of worker stream k was enqueued
     int n_wstreams = 0;
     cudaEvent_t ev_fork = nullptr;                 // stream_acc -> worker stream (re-recorded per call)
     cudaEvent_t ev_set_done[kMlpSets] = {};        // last use of a scratch set has finished
@@ -172,6 +196,9 @@ struct abs_ctx {
     bool profiling = false;
     std::vector<TimedLaunch> timed;
     std::vector<cudaEvent_t> ev_pool;
+    bool timeline_on = false;         // abs_profile(ctx, 2): the spans of the timed launches are kept as well
+    cudaEvent_t ev_origin = nullptr;  // time zero of the timeline (recorded on stream_acc when it was switched on)
+    std::vector<abs_span> spans;
     uint64_t stat_n[ABS_K_COUNT] = {0};
     double stat_ms[ABS_K_COUNT] = {0};
     std::string err;
@@ -241,12 +268,22 @@ struct Timed {
         stop = take_event(c);
         if (!start || !stop) { stop = nullptr; return; }
         cudaEventRecord(start, s);
-        c->timed.push_back({kernel_class, start, stop});
+        c->timed.push_back({kernel_class, start, stop, s, 0});
     }
     ~Timed() {
         if (stop) cudaEventRecord(stop, s);
     }
 };
+
+int stream_index(const abs_ctx* c, cudaStream_t s) {
+    if (s == c->s_acc) return 0;
+    if (s == c->s_sync) return 1;
+    for (int k = 0; k < c->n_wstreams; ++k) {
+        if (s == c->s_w[k]) return 2 + k;
+        if (s == c->s_d[k]) return 2 + kMlpStreams + k;
+    }
+    return -1;
+}
 
 int collect_timings(abs_ctx* c) {
     for (auto& tl : c->timed) {
@@ -255,6 +292,11 @@ int collect_timings(abs_ctx* c) {
         CK(cudaEventElapsedTime(&ms, tl.start, tl.stop));
         c->stat_n[tl.kernel_class] += 1;
         c->stat_ms[tl.kernel_class] += ms;
+        if (c->timeline_on && c->ev_origin && c->spans.size() < kMaxSpans) {
+            float t0 = 0.f;
+            CK(cudaEventElapsedTime(&t0, c->ev_origin, tl.start));
+            c->spans.push_back({tl.kernel_class, stream_index(c, tl.stream), tl.part, t0 * 1e3f, (t0 + ms) * 1e3f});
+        }
         c->ev_pool.push_back(tl.start);
         c->ev_pool.push_back(tl.stop);
     }
@@ -313,7 +355,7 @@ int launch_fused(abs_ctx* c, uint32_t set, int in, int out, uint64_t log_step, c
     if (shape == 0 && c->mlp && c->pipelined) shape = -2;
     {
         Timed tm(c, ABS_K_SYNC, stream);
-        CK(launch_sync(a, shape, c->num_sms, stream));
+        CK(launch_sync(a, shape, c->num_sms, stream, c->chained()));
     }
     c->launches += 1;
     return ABS_OK;
@@ -345,17 +387,30 @@ int run_mlp_group(abs_ctx* c, uint32_t worker, int set, int n, bool first, bool 
         CK(cudaEventRecord(c->ev_fork, c->s_acc));
         CK(cudaStreamWaitEvent(s_run, c->ev_fork, 0));
     }
-    if (deferred) mlp_mark(c, ABS_K_MLP_FWD, 0, s_run);
+    (void)deferred;
     CK(launch_mlp_front(c->mlp_dims, sc, c->x(c->pub), c->shadow(c->pub), c->pub, n, first, c->acc(c->cur, worker),
-                        c->cnt(c->cur, worker), variant, s_run, mlp_mark, c));
-    if (deferred) c->launches -= 1;   // launch_mlp_front counts one cast with its group
+                        c->cnt(c->cur, worker), variant, s_run, c->mlp_chain(serial, n), mlp_mark, c));
+    cudaStream_t s_gemm = s_run;
+    // Single calls: dW1 on the worker's second stream (measured on 3072-4096-10, W = 4: 32.2 -> 31.3 us per
+    // micro-batch); K-batched calls keep it behind their front kernels (15.6 against 16.0 us).
+    const bool split = !serial && n == 1;
+    if (split) s_gemm = c->s_d[k];
+    if (!serial && c->w_outstanding[k] && c->gemm_on_d[k] != split)   // the worker's previous dW1 ran on the other stream
+        CK(cudaStreamWaitEvent(s_gemm, c->ev_w_done[k], 0));
+    if (split) {
+        CK(cudaEventRecord(c->ev_front[k], s_run));
+        CK(cudaStreamWaitEvent(s_gemm, c->ev_front[k], 0));
+    }
+    if (!serial) c->gemm_on_d[k] = split;
+    // On its own stream the kernel ahead of this dW1 is the worker's previous dW1, which writes the same slice:
+    // never chained there (the register-prefetch kernel reads the slice in front of its wait).
     CK(launch_mlp_dw1(c->mlp_dims, sc, c->acc(c->cur, worker), &c->acc_tmaps[(size_t)c->cur * c->cfg.W + worker], n,
-                      first, variant, s_run, mlp_mark, c));
+                      first, variant, s_gemm, serial && (c->mlp_chain(serial, n) & kChainDw1) != 0, mlp_mark, c));
     if (serial) {
         for (bool& u : c->set_used) u = false;
     } else {
-        CK(cudaEventRecord(c->ev_set_done[set], s_run));
-        CK(cudaEventRecord(c->ev_w_done[k], s_run));
+        CK(cudaEventRecord(c->ev_set_done[set], s_gemm));
+        CK(cudaEventRecord(c->ev_w_done[k], s_gemm));
         c->set_used[set] = true;
         c->w_outstanding[k] = true;
     }
@@ -386,7 +441,7 @@ int flush_all(abs_ctx* c) {
 
 // One micro-batch of `worker` joins its waiting group: cast now (the caller's buffers are free again once
 // stream_acc has passed this point), everything else when the group runs.
-int coalesce_one(abs_ctx* c, uint32_t worker, const float* x_dev, const int32_t* y_dev) {
+int coalesce_one(abs_ctx* c, uint32_t worker, const void* x_dev, const int32_t* y_dev) {
     if (c->pend_n[worker] == 0) {
         if (c->n_reserved >= kMlpSets / 2) {   // keep half of the scratch sets for groups that are running
             int oldest = -1;
@@ -403,8 +458,8 @@ int coalesce_one(abs_ctx* c, uint32_t worker, const float* x_dev, const int32_t*
         c->pend_age[worker] = ++c->pend_clock;
     }
     const int slot = c->pend_n[worker];
-    CK(launch_mlp_cast(c->mlp_dims, c->mlp_scratch[c->pend_set[worker]], slot, 1, x_dev, y_dev, c->s_acc, mlp_mark, c));
-    mlp_mark(c, ABS_K_MLP_FWD, 1, c->s_acc);
+    CK(launch_mlp_cast(c->mlp_dims, c->mlp_scratch[c->pend_set[worker]], slot, 1, x_dev, c->x_bf16(), y_dev, c->s_acc,
+                       (c->mlp_chain(false, 1) & kChainCast) != 0, mlp_mark, c));
     c->pend_n[worker] = slot + 1;
     c->h_cnt[(size_t)c->cur * c->cfg.W + worker] += 1;
     if (c->pend_n[worker] == kMlpMaxBatch) return flush_worker(c, worker);
@@ -503,7 +558,10 @@ int abs_init(abs_ctx** out, const abs_config* cfg, void* workspace_dev, size_t w
         if ((e = cudaDeviceGetStreamPriorityRange(&prio_lo, &prio_hi)) != cudaSuccess) return bail(e, "cudaDeviceGetStreamPriorityRange");
         for (int k = 0; k < c->n_wstreams; ++k) {
             if ((e = cudaStreamCreateWithPriority(&c->s_w[k], cudaStreamNonBlocking, prio_hi)) != cudaSuccess) return bail(e, "cudaStreamCreate");
+            const int prio_gemm = prio_hi < prio_lo ? prio_hi + 1 : prio_hi;   // (numerically lower = higher priority)
+            if ((e = cudaStreamCreateWithPriority(&c->s_d[k], cudaStreamNonBlocking, prio_gemm)) != cudaSuccess) return bail(e, "cudaStreamCreate");
             if ((e = cudaEventCreateWithFlags(&c->ev_w_done[k], cudaEventDisableTiming)) != cudaSuccess) return bail(e, "cudaEventCreate");
+            if ((e = cudaEventCreateWithFlags(&c->ev_front[k], cudaEventDisableTiming)) != cudaSuccess) return bail(e, "cudaEventCreate");
         }
         c->acc_tmaps.resize((size_t)2 * cfg->W);
         for (uint32_t set = 0; set < 2; ++set)
@@ -536,7 +594,7 @@ int abs_accumulate(abs_ctx* c, uint32_t worker, const void* grad_dev) {
     {
         Timed tm(c, ABS_K_ACCUMULATE, c->s_acc);
         CK(launch_accumulate(c->acc(c->cur, worker), grad_dev, c->cfg.grad_dtype, c->cfg.P, c->cnt(c->cur, worker), first,
-                             c->ctas_per_sm[ABS_K_ACCUMULATE], c->num_sms, c->s_acc));
+                             c->ctas_per_sm[ABS_K_ACCUMULATE], c->num_sms, c->s_acc, c->chained()));
     }
     c->launches += 1;
     c->h_cnt[(size_t)c->cur * c->cfg.W + worker] += 1;
@@ -559,7 +617,7 @@ int abs_accumulate_batch(abs_ctx* c, uint32_t worker, uint32_t n, const void* co
     {
         Timed tm(c, ABS_K_ACCUMULATE, c->s_acc);
         CK(launch_accumulate_multi(c->acc(c->cur, worker), gl, (int)n, c->cfg.grad_dtype, c->cfg.P, c->cnt(c->cur, worker),
-                                   first, c->ctas_per_sm[ABS_K_ACCUMULATE], c->num_sms, c->s_acc));
+                                   first, c->ctas_per_sm[ABS_K_ACCUMULATE], c->num_sms, c->s_acc, c->chained()));
     }
     c->launches += 1;
     c->h_cnt[(size_t)c->cur * c->cfg.W + worker] += (int32_t)n;
@@ -585,7 +643,7 @@ int abs_accumulate_host(abs_ctx* c, uint32_t worker, const void* grad_host) {
     {
         Timed tm(c, ABS_K_ACCUMULATE, c->s_acc);
         CK(launch_accumulate(c->acc(c->cur, worker), stage, c->cfg.grad_dtype, c->cfg.P, c->cnt(c->cur, worker), first,
-                             c->ctas_per_sm[ABS_K_ACCUMULATE], c->num_sms, c->s_acc));
+                             c->ctas_per_sm[ABS_K_ACCUMULATE], c->num_sms, c->s_acc, c->chained()));
     }
     CK(cudaEventRecord(c->ev_stage_free[k], c->s_acc));
     c->stage_used[k] = true;
@@ -594,7 +652,7 @@ int abs_accumulate_host(abs_ctx* c, uint32_t worker, const void* grad_host) {
     return ABS_OK;
 }
 
-int abs_accumulate_mlp_batch(abs_ctx* c, uint32_t worker, uint32_t n, const float* x_dev, const int32_t* y_dev) {
+int abs_accumulate_mlp_batch(abs_ctx* c, uint32_t worker, uint32_t n, const void* x_dev, const int32_t* y_dev) {
     if (!live(c)) return ABS_ESTATE;
     if (!c->mlp) return invalid(c, "context was created without ABS_FLAG_MLP");
     if (worker >= c->cfg.W) return invalid(c, "worker index out of range");
@@ -616,13 +674,14 @@ int abs_accumulate_mlp_batch(abs_ctx* c, uint32_t worker, uint32_t n, const floa
     // ABS_FLAG_OVERWRITE_FIRST -- stale): it is stored, not added, and dW1 skips reading the 4 d_in d_hidden
     // bytes of the slice.  0 + g = g, so the default mode's results do not change.
     const bool first = c->h_cnt[(size_t)c->cur * c->cfg.W + worker] == 0;
-    CK(launch_mlp_cast(c->mlp_dims, c->mlp_scratch[set], 0, (int)n, x_dev, y_dev, c->s_acc, mlp_mark, c));
+    CK(launch_mlp_cast(c->mlp_dims, c->mlp_scratch[set], 0, (int)n, x_dev, c->x_bf16(), y_dev, c->s_acc,
+                       (c->mlp_chain(serial, (int)n) & kChainCast) != 0, mlp_mark, c));
     if (int rc = run_mlp_group(c, worker, set, (int)n, first, false)) return rc;
     c->h_cnt[(size_t)c->cur * c->cfg.W + worker] += (int32_t)n;
     return ABS_OK;
 }
 
-int abs_accumulate_mlp(abs_ctx* c, uint32_t worker, const float* x_dev, const int32_t* y_dev) {
+int abs_accumulate_mlp(abs_ctx* c, uint32_t worker, const void* x_dev, const int32_t* y_dev) {
     return abs_accumulate_mlp_batch(c, worker, 1, x_dev, y_dev);
 }
 
@@ -707,6 +766,26 @@ int abs_global_attach(abs_ctx* c, const abs_peer_table* peers) {
         if (!p || (reinterpret_cast<uintptr_t>(p) & 255)) return invalid(c, "peer workspace must be non-NULL and 256-byte aligned");
     }
     if (peers->workspace_dev[peers->rank] != c->ws) return invalid(c, "workspace_dev[rank] must be this context's own workspace");
+    // A peer's workspace on another GPU is read and written by this GPU's kernel with plain loads and stores: that
+    // needs peer access from this device to the peer's.  Mappings opened with abs_ipc_open have it already (the IPC
+    // open enables it); plain pointers of another device of the same process get it here.
+    for (uint32_t q = 0; q < peers->n_ranks; ++q) {
+        if (q == peers->rank) continue;
+        cudaPointerAttributes at{};
+        if (cudaPointerGetAttributes(&at, peers->workspace_dev[q]) != cudaSuccess) { cudaGetLastError(); return invalid(c, "a peer workspace is not a device pointer known to this process"); }
+        if (at.type != cudaMemoryTypeDevice) return invalid(c, "a peer workspace is not device memory");
+        if (at.device == c->device) continue;
+        int can = 0;
+        CK(cudaDeviceCanAccessPeer(&can, c->device, at.device));
+        if (!can) return invalid(c, "this GPU has no peer access to a peer workspace's GPU");
+        int cur_dev = c->device;
+        CK(cudaGetDevice(&cur_dev));
+        if (cur_dev != c->device) CK(cudaSetDevice(c->device));   // peer access is granted to the current device
+        const cudaError_t e = cudaDeviceEnablePeerAccess(at.device, 0);
+        if (cur_dev != c->device) cudaSetDevice(cur_dev);
+        if (e == cudaErrorPeerAccessAlreadyEnabled) cudaGetLastError();
+        else if (e != cudaSuccess) return cuda_fail(c, e, "cudaDeviceEnablePeerAccess");
+    }
     c->n_ranks = peers->n_ranks;
     c->rank = peers->rank;
     for (uint32_t q = 0; q < peers->n_ranks; ++q) c->peer_ws[q] = static_cast<char*>(peers->workspace_dev[q]);
@@ -773,7 +852,7 @@ int abs_global_step(abs_ctx* c) {
     a.zero_acc = (c->cfg.flags & ABS_FLAG_OVERWRITE_FIRST) ? 0 : 1;
     {
         Timed tm(c, ABS_K_SYNC, c->s_sync);
-        CK(launch_sync_global(a, c->ctas_per_sm[ABS_K_SYNC], c->num_sms, c->s_sync));
+        CK(launch_sync_global(a, c->ctas_per_sm[ABS_K_SYNC], c->num_sms, c->s_sync, c->chained()));
     }
     c->launches += 1;
     c->global_prev_lr = c->lr_now;
@@ -952,7 +1031,10 @@ int abs_check(abs_ctx* c) {
     if (!live(c)) return ABS_ESTATE;
     if (int rc = flush_all(c)) return rc;
     if (c->pipelined) CK(cudaStreamSynchronize(c->s_sync));
-    for (int k = 0; k < c->n_wstreams; ++k) CK(cudaStreamSynchronize(c->s_w[k]));
+    for (int k = 0; k < c->n_wstreams; ++k) {
+        CK(cudaStreamSynchronize(c->s_w[k]));
+        CK(cudaStreamSynchronize(c->s_d[k]));
+    }
     CK(cudaStreamSynchronize(c->s_acc));
     {
         int st = 0;
@@ -1004,7 +1086,10 @@ bool same_config(const abs_config& a, const abs_config& b) {
 int drain(abs_ctx* c) {
     if (int rc = flush_all(c)) return rc;
     if (c->pipelined) CK(cudaStreamSynchronize(c->s_sync));
-    for (int k = 0; k < c->n_wstreams; ++k) CK(cudaStreamSynchronize(c->s_w[k]));
+    for (int k = 0; k < c->n_wstreams; ++k) {
+        CK(cudaStreamSynchronize(c->s_w[k]));
+        CK(cudaStreamSynchronize(c->s_d[k]));
+    }
     if (c->s_copy) CK(cudaStreamSynchronize(c->s_copy));
     CK(cudaStreamSynchronize(c->s_acc));
     if (c->pipelined) CK(cudaStreamSynchronize(c->s_sync));
@@ -1097,6 +1182,10 @@ int abs_set_launch(abs_ctx* c, int kernel_class, int ctas_per_sm) {
     if (kernel_class < 0 || kernel_class >= ABS_K_COUNT || ctas_per_sm < (kernel_class == ABS_K_SYNC ? -2 : -1) ||
         ctas_per_sm > (kernel_class == ABS_K_MLP_DW1 ? 255 : 64))
         return invalid(c, "bad kernel class or CTA count");
+    if (kernel_class == ABS_K_MLP_DW1 && ctas_per_sm > 0 && (ctas_per_sm & ~(4 | 8 | 32 | 128)))
+        return invalid(c, "unknown bits in the ABS_K_MLP_DW1 mask");
+    if (kernel_class == ABS_K_CHAIN && (ctas_per_sm < 0 || ctas_per_sm > 1)) return invalid(c, "ABS_K_CHAIN takes 0 or 1");
+    if (kernel_class == ABS_K_MLP_FWD && (ctas_per_sm < 0 || ctas_per_sm > 1)) return invalid(c, "ABS_K_MLP_FWD takes 0 or 1");
     if (int rc = flush_all(c)) return rc;
     c->ctas_per_sm[kernel_class] = ctas_per_sm;
     return ABS_OK;
@@ -1108,8 +1197,27 @@ int abs_profile(abs_ctx* c, int enable) {
     if (rc != ABS_OK) return rc;
     if (enable) {
         for (int k = 0; k < ABS_K_COUNT; ++k) { c->stat_n[k] = 0; c->stat_ms[k] = 0.0; }
+        c->spans.clear();
     }
     c->profiling = enable != 0;
+    c->timeline_on = enable == 2;
+    if (c->timeline_on) {
+        if (!c->ev_origin) CK(cudaEventCreate(&c->ev_origin));
+        CK(cudaEventRecord(c->ev_origin, c->s_acc));
+    }
+    return ABS_OK;
+}
+
+int abs_profile_timeline(abs_ctx* c, abs_span* out, size_t capacity, size_t* n) {
+    if (!live(c)) return ABS_ESTATE;
+    if (!n) return invalid(c, "output pointer is NULL");
+    int rc = collect_timings(c);
+    if (rc != ABS_OK) return rc;
+    *n = c->spans.size();
+    if (out) {
+        const size_t m = std::min(capacity, c->spans.size());
+        for (size_t k = 0; k < m; ++k) out[k] = c->spans[k];
+    }
     return ABS_OK;
 }
 
@@ -1142,9 +1250,13 @@ int abs_destroy(abs_ctx* c) {
     if (c->s_copy) { cudaStreamSynchronize(c->s_copy); cudaStreamDestroy(c->s_copy); }
     for (int k = 0; k < c->n_wstreams; ++k)
         if (c->s_w[k]) { cudaStreamSynchronize(c->s_w[k]); cudaStreamDestroy(c->s_w[k]); }
+    for (int k = 0; k < c->n_wstreams; ++k)
+        if (c->s_d[k]) { cudaStreamSynchronize(c->s_d[k]); cudaStreamDestroy(c->s_d[k]); }
+    for (cudaEvent_t e : c->ev_front) if (e) cudaEventDestroy(e);
     for (cudaEvent_t e : c->ev_set_done) if (e) cudaEventDestroy(e);
     for (cudaEvent_t e : c->ev_w_done) if (e) cudaEventDestroy(e);
     if (c->ev_fork) cudaEventDestroy(c->ev_fork);
+    if (c->ev_origin) cudaEventDestroy(c->ev_origin);
     for (auto& tl : c->timed) { cudaEventDestroy(tl.start); cudaEventDestroy(tl.stop); }
     for (auto e : c->ev_pool) cudaEventDestroy(e);
     for (cudaEvent_t e : {c->ev_acc_done, c->ev_sync_done, c->ev_aux, c->ev_stage_free[0], c->ev_stage_free[1],
@@ -1158,16 +1270,16 @@ int abs_destroy(abs_ctx* c) {
 }  // extern "C"
 
 namespace {
-// Called by the MLP launcher around each group of its kernels: n = 0 before, n = launches made after.
+// Called by the MLP launcher around each of its kernels: n = -1 - part before, n = launches made after.
 void mlp_mark(void* user, int kernel_class, int n, cudaStream_t stream) {
     abs_ctx* c = static_cast<abs_ctx*>(user);
-    c->launches += (uint64_t)n;
+    if (n > 0) c->launches += (uint64_t)n;
     if (!c->profiling) return;
-    if (n == 0) {
+    if (n < 0) {
         cudaEvent_t start = take_event(c), stop = take_event(c);
         if (!start || !stop) return;
         cudaEventRecord(start, stream);
-        c->timed.push_back({kernel_class, start, stop});
+        c->timed.push_back({kernel_class, start, stop, stream, -1 - n});
     } else if (!c->timed.empty() && c->timed.back().kernel_class == kernel_class) {
         cudaEventRecord(c->timed.back().stop, stream);
     }

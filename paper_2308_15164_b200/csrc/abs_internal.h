@@ -13,11 +13,42 @@ constexpr int kMaxW = ABS_MAX_WORKERS;
 constexpr int kLogDepth = 64;     // sync steps kept in the device-side consumed-count log
 constexpr size_t kPadElems = 256; // accumulator row stride is P rounded up to this many elements
 
+// ---- programmatic dependent launch ----------------------------------------------------------
+// Consecutive kernels of a stream are chained so that kernel n+1 is made resident (CTAs scheduled, shared
+// memory carved, barriers initialised, TMEM allocated) while kernel n is still draining.  Every kernel of this
+// library executes pdl_wait() in every CTA before it touches anything an earlier kernel of its stream wrote --
+// the wait returns once the predecessor grid has completed and its writes are visible -- and only THEN lets its
+// own successor start (pdl_trigger()).  By induction, when a kernel starts, every kernel two or more places ahead
+// of it in the stream has completed, so code in front of pdl_wait() may read what those wrote, but nothing
+// the immediate predecessor writes.  Both instructions do nothing in a launch without the attribute.
+#ifdef __CUDACC__
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void pdl_trigger() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+#endif
+// kernel<<<grid, block, smem, stream>>>(args...), with the programmatic-stream-serialization attribute when
+// `chained` is set.
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_kernel(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t stream,
+                                 bool chained, Args&&... args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = chained ? 1 : 0;
+    return cudaLaunchKernelEx(&cfg, kernel, static_cast<Args&&>(args)...);
+}
+
 // ---- Step 2: acc_row[j] += g[j], cnt[0] += 1 (Algorithm 1, Step 2) ------------------------
 // grad_dtype: ABS_GRAD_F32 / ABS_GRAD_BF16.  P = number of valid elements in g.
 // overwrite: acc_row[j] = g[j] instead (first micro-batch of a worker when the row is not kept zeroed).
+// chained (here and below): launch with programmatic dependent launch on the kernel ahead on `stream`.
 cudaError_t launch_accumulate(float* acc_row, const void* g, uint32_t grad_dtype, size_t P, int32_t* cnt, bool overwrite,
-                              int ctas_per_sm, int num_sms, cudaStream_t stream);
+                              int ctas_per_sm, int num_sms, cudaStream_t stream, bool chained);
 
 // ---- Step 1 + update (Algorithm 1, Step 1, Eq. 6, "Update parameters") --------------------
 struct SyncArgs {
@@ -41,6 +72,7 @@ struct SyncArgs {
     unsigned int norm_slots;  // slots in norm_part
     int overlapped;           // the launch runs beside the next iteration's accumulate kernels (pipelined mode)
     int* status;              // optional device status word (ABS_ETIMEOUT if a bounded wait of the bulk-copy kernel ran out)
+    int plain_only;           // 1: never the bulk-copy form (a caller without a status word to report its time-outs through)
 };
 // n (1..kMaxAccBatch) gradients of one worker added in one pass over its accumulator row, in list order.
 constexpr int kMaxAccBatch = 8;
@@ -48,14 +80,14 @@ struct GradList {
     const void* p[kMaxAccBatch];
 };
 cudaError_t launch_accumulate_multi(float* acc_row, const GradList& gl, int n, uint32_t grad_dtype, size_t P, int32_t* cnt,
-                                    bool overwrite, int ctas_per_sm, int num_sms, cudaStream_t stream);
+                                    bool overwrite, int ctas_per_sm, int num_sms, cudaStream_t stream, bool chained);
 // ctas_per_sm: 0 = default shape, -1 = one tile per CTA, > 0 = persistent grid, -2 = the bulk-copy kernel below
 // where it applies (else the default).
-cudaError_t launch_sync(const SyncArgs& a, int ctas_per_sm, int num_sms, cudaStream_t stream);
+cudaError_t launch_sync(const SyncArgs& a, int ctas_per_sm, int num_sms, cudaStream_t stream, bool chained);
 // Same step with the rows staged through shared memory by cp.async.bulk (sync_tma.cu).  cudaErrorNotSupported for
 // W > kSyncTmaMaxW or when the gradient norm is wanted: the caller then uses launch_sync.
 constexpr int kSyncTmaMaxW = 24;
-cudaError_t launch_sync_tma(const SyncArgs& a, int num_sms, cudaStream_t stream);
+cudaError_t launch_sync_tma(const SyncArgs& a, int num_sms, cudaStream_t stream, bool chained);
 // One small launch whose only wait can never be satisfied: it gives up after a few thousand polls and writes
 // ABS_ETIMEOUT to *status (the path a stuck pipeline takes), leaving the context usable.
 cudaError_t launch_bounded_wait_selftest(int* status, cudaStream_t stream);
@@ -82,7 +114,7 @@ struct GlobalSyncArgs {
     float disp_scale;                     // rate of the previous step (x_t - x_{t-1} = -disp_scale * v if it applied)
     int zero_acc;
 };
-cudaError_t launch_sync_global(const GlobalSyncArgs& a, int ctas_per_sm, int num_sms, cudaStream_t stream);
+cudaError_t launch_sync_global(const GlobalSyncArgs& a, int ctas_per_sm, int num_sms, cudaStream_t stream, bool chained);
 // gcnt[j] = (own_lo <= j < own_lo + W_local) ? cnt[j - own_lo] : 0 for j < n_total;  cnt[0..W_local) = 0.
 cudaError_t launch_global_counts(int32_t* gcnt, int32_t* cnt, int own_lo, int W_local, int n_total, cudaStream_t stream);
 
@@ -94,6 +126,9 @@ constexpr int kMlpMaxBatch = 4;
 // Internal bit of the `variant` argument below (set by the context, never by abs_set_launch): forward GEMM and ring
 // dW1 kernel in their light shared-memory configurations, so that CTAs of different workers' calls share an SM.
 constexpr int kMlpLightBit = 256;
+// Which kernels of a gradient call are launched chained to the kernel ahead (bits of the `chain` argument of
+// launch_mlp_front; the cast and the dW1 kernel take a bool).
+constexpr int kChainCast = 1, kChainFwd1 = 2, kChainFwd2 = 4, kChainBwd = 8, kChainDw1 = 16;
 constexpr int kMlpStreams = 8;   // internal worker streams (worker i runs on stream i % kMlpStreams)
 constexpr int kMlpSets = 8;      // scratch sets, one per call in flight, taken round-robin
 struct MlpDims {
@@ -133,21 +168,22 @@ cudaError_t mlp_make_acc_tmap(void* tmap_out, const MlpDims& d, float* acc_row);
 //          acc_row; bumps cnt);   dw1: the dW1 GEMM, which reads xtb/dzt and adds into the W1 slice.
 // shadow: bf16 copy of the published parameters (same flat layout), shadow_idx: which of the two copies it is.
 // x_pub: the fp32 parameters.  variant: the ABS_K_MLP_DW1 bit mask of abs_set_launch (0 = dW1 kernel chosen per
-// call; 1, 4, 8, 16 force one; 2 = forward GEMM on CUDA cores, a cross-check of the tcgen05 one).
-// mark(user, kernel_class, 0, stream) is called before a kernel group, mark(user, kernel_class, n, stream) after
-// its n launches.
+// call; 4, 8 force one).  x_is_bf16: the caller's X holds bf16 values (copied as they are) instead of fp32.
+// mark(user, kernel_class, -1 - part, stream) is called before a kernel (part: its ordinal within the class for
+// one call -- forward class: 0 cast, 1 forward GEMM, 2 bias / ReLU / logits), mark(user, kernel_class, n, stream)
+// after its n launches.
 typedef void (*MlpMark)(void* user, int kernel_class, int n, cudaStream_t stream);
-cudaError_t launch_mlp_cast(const MlpDims& d, const MlpScratch& s, int slot0, int nb, const float* x_dev, const int32_t* y_dev,
-                            cudaStream_t stream, MlpMark mark, void* user);
+cudaError_t launch_mlp_cast(const MlpDims& d, const MlpScratch& s, int slot0, int nb, const void* x_dev, bool x_is_bf16,
+                            const int32_t* y_dev, cudaStream_t stream, bool chained, MlpMark mark, void* user);
 cudaError_t launch_mlp_front(const MlpDims& d, const MlpScratch& s, const float* x_pub, const __nv_bfloat16* shadow,
                              int shadow_idx, int nb, bool store, float* acc_row, int32_t* cnt, int variant,
-                             cudaStream_t stream, MlpMark mark, void* user);
+                             cudaStream_t stream, int chain, MlpMark mark, void* user);
 // nb: a call may carry up to kMlpMaxBatch micro-batches (x_dev [nb][mb][d_in], y_dev [nb][mb]): the front kernels
 // take them as an extra grid dimension, and ONE dW1 launch contracts them with K = 64 nb (the accumulator slice is
 // read and written once).
 // store: the accumulator row holds nothing yet (the worker's first gradient of the iteration): front and dw1
 // store their results instead of adding them, and dw1 does not read the accumulator slice at all.
 cudaError_t launch_mlp_dw1(const MlpDims& d, const MlpScratch& s, float* acc_row, const void* acc_tmap, int nb, bool store,
-                           int variant, cudaStream_t stream, MlpMark mark, void* user);
+                           int variant, cudaStream_t stream, bool chained, MlpMark mark, void* user);
 
 }  // namespace abs_sgd

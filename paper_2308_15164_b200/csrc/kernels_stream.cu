@@ -50,6 +50,8 @@ __global__ void __launch_bounds__(kBlock) k_accumulate_f32(float* acc, const flo
     float4* acc4 = reinterpret_cast<float4*>(acc);
     const float4* g4 = reinterpret_cast<const float4*>(g);
     const unsigned long long tile = (unsigned long long)kBlock * U;
+    pdl_wait();      // the row may have been written by the kernel just ahead on the stream
+    pdl_trigger();
     for (unsigned long long base = blockIdx.x * tile; base < n_vec; base += gridDim.x * tile) {
         float4 a[U], b[U];
 #pragma unroll
@@ -90,6 +92,8 @@ __global__ void __launch_bounds__(kBlock) k_accumulate_bf16(float* acc, const ui
     float4* acc4 = reinterpret_cast<float4*>(acc);
     const uint4* g8 = reinterpret_cast<const uint4*>(g);
     const unsigned long long tile = (unsigned long long)kBlock * U;
+    pdl_wait();
+    pdl_trigger();
     for (unsigned long long base = blockIdx.x * tile; base < n_vec8; base += gridDim.x * tile) {
         float4 a0[U], a1[U];
         uint4 b[U];
@@ -138,6 +142,8 @@ __global__ void __launch_bounds__(kBlock) k_accumulate_multi_f32(float* acc, Gra
                                                                  unsigned long long P, int32_t* cnt) {
     float4* acc4 = reinterpret_cast<float4*>(acc);
     const unsigned long long tile = (unsigned long long)kBlock * U;
+    pdl_wait();
+    pdl_trigger();
     for (unsigned long long base = blockIdx.x * tile; base < n_vec; base += gridDim.x * tile) {
         float4 a[U], b[U][MAXN];
 #pragma unroll
@@ -178,6 +184,8 @@ __global__ void __launch_bounds__(kBlock) k_accumulate_multi_bf16(float* acc, Gr
                                                                   unsigned long long P, int32_t* cnt) {
     float4* acc4 = reinterpret_cast<float4*>(acc);
     const unsigned long long tile = (unsigned long long)kBlock * U;
+    pdl_wait();
+    pdl_trigger();
     for (unsigned long long base = blockIdx.x * tile; base < n_vec8; base += gridDim.x * tile) {
         uint4 b[U][MAXN];
         float4 a0[U], a1[U];
@@ -264,6 +272,8 @@ __global__ void __launch_bounds__(kBlock) k_sync(const SyncArgs a) {
     __shared__ double s_norm[kBlock / 32];
     float norm_acc = 0.f;   // kNorm: this thread's share of |Gbar|^2 (a handful of vectors)
     const int W = WT > 0 ? WT : a.W;
+    pdl_wait();      // counters and rows come from the accumulate kernels ahead on the stream
+    pdl_trigger();
     if (threadIdx.x < W) s_cnt[threadIdx.x] = a.cnt[threadIdx.x];
     __syncthreads();
     long long B = 0;
@@ -416,6 +426,8 @@ __global__ void __launch_bounds__(kBlock) k_sync_global(const GlobalSyncArgs a) 
     __shared__ int s_cnt[kMaxW];
     __shared__ float4* s_row[kMaxW];
     const int R = a.G * a.W_local;                    // rows in global worker order: j = q * W_local + i
+    pdl_wait();
+    pdl_trigger();
     if (threadIdx.x < R) {
         const int q = threadIdx.x / a.W_local, i = threadIdx.x - q * a.W_local;
         s_cnt[threadIdx.x] = a.cnt_all[threadIdx.x];
@@ -476,6 +488,8 @@ __global__ void __launch_bounds__(kBlock) k_sync_global(const GlobalSyncArgs a) 
 }
 
 __global__ void k_global_counts(int32_t* gcnt, int32_t* cnt, int own_lo, int W_local, int n_total) {
+    pdl_wait();
+    pdl_trigger();
     const int j = threadIdx.x;
     if (j >= n_total) return;
     const bool own = j >= own_lo && j < own_lo + W_local;
@@ -485,6 +499,8 @@ __global__ void k_global_counts(int32_t* gcnt, int32_t* cnt, int own_lo, int W_l
 
 __global__ void __launch_bounds__(kBlock) k_cast_bf16(const float4* __restrict__ src, __nv_bfloat16* dst,
                                                       unsigned long long n_vec) {
+    pdl_wait();
+    pdl_trigger();
     for (unsigned long long idx = blockIdx.x * (unsigned long long)kBlock + threadIdx.x; idx < n_vec;
          idx += (unsigned long long)gridDim.x * kBlock)
         store_shadow(dst, idx, src[idx]);
@@ -502,75 +518,68 @@ inline unsigned grid_for(unsigned long long n_items, int per_cta, int ctas_per_s
 }
 
 template <int WT, int U>
-cudaError_t launch_sync_t(const SyncArgs& a, int ctas_per_sm, int num_sms, cudaStream_t stream) {
+cudaError_t launch_sync_t(const SyncArgs& a, int ctas_per_sm, int num_sms, cudaStream_t stream, bool chained) {
     const unsigned grid = grid_for(a.n_vec, kBlock * U, ctas_per_sm, num_sms);
     if (a.norm_out) {
         if (grid > a.norm_slots) return cudaErrorInvalidValue;
-        k_sync<WT, U, true><<<grid, kBlock, 0, stream>>>(a);
-    } else {
-        k_sync<WT, U, false><<<grid, kBlock, 0, stream>>>(a);
+        return launch_kernel(k_sync<WT, U, true>, grid, kBlock, 0, stream, chained, a);
     }
-    return cudaGetLastError();
+    return launch_kernel(k_sync<WT, U, false>, grid, kBlock, 0, stream, chained, a);
 }
 
 }  // namespace
 
 cudaError_t launch_accumulate(float* acc_row, const void* g, uint32_t grad_dtype, size_t P, int32_t* cnt, bool overwrite,
-                              int ctas_per_sm, int num_sms, cudaStream_t stream) {
+                              int ctas_per_sm, int num_sms, cudaStream_t stream, bool chained) {
     constexpr int U = 4;
     if (ctas_per_sm == 0) ctas_per_sm = -1;   // measured: one tile per CTA beats a persistent grid
+    const unsigned long long P_ = P;
     if (grad_dtype == ABS_GRAD_F32) {
         const unsigned long long n_vec = P / 4;
         const unsigned grid = grid_for(n_vec, kBlock * U, ctas_per_sm, num_sms);
-        if (overwrite)
-            k_accumulate_f32<U, true><<<grid, kBlock, 0, stream>>>(acc_row, static_cast<const float*>(g), n_vec, P, cnt);
-        else
-            k_accumulate_f32<U, false><<<grid, kBlock, 0, stream>>>(acc_row, static_cast<const float*>(g), n_vec, P, cnt);
-    } else {
-        const unsigned long long n_vec8 = P / 8;
-        const unsigned grid = grid_for(n_vec8, kBlock * U, ctas_per_sm, num_sms);
-        if (overwrite)
-            k_accumulate_bf16<U, true><<<grid, kBlock, 0, stream>>>(acc_row, static_cast<const uint16_t*>(g), n_vec8, P, cnt);
-        else
-            k_accumulate_bf16<U, false><<<grid, kBlock, 0, stream>>>(acc_row, static_cast<const uint16_t*>(g), n_vec8, P, cnt);
+        const float* gf = static_cast<const float*>(g);
+        return launch_kernel(overwrite ? k_accumulate_f32<U, true> : k_accumulate_f32<U, false>, grid, kBlock, 0, stream,
+                             chained, acc_row, gf, n_vec, P_, cnt);
     }
-    return cudaGetLastError();
+    const unsigned long long n_vec8 = P / 8;
+    const unsigned grid = grid_for(n_vec8, kBlock * U, ctas_per_sm, num_sms);
+    const uint16_t* gb = static_cast<const uint16_t*>(g);
+    return launch_kernel(overwrite ? k_accumulate_bf16<U, true> : k_accumulate_bf16<U, false>, grid, kBlock, 0, stream,
+                         chained, acc_row, gb, n_vec8, P_, cnt);
 }
 
 cudaError_t launch_accumulate_multi(float* acc_row, const GradList& gl, int n, uint32_t grad_dtype, size_t P, int32_t* cnt,
-                                    bool overwrite, int ctas_per_sm, int num_sms, cudaStream_t stream) {
+                                    bool overwrite, int ctas_per_sm, int num_sms, cudaStream_t stream, bool chained) {
     if (ctas_per_sm == 0) ctas_per_sm = -1;
+    const unsigned long long P_ = P;
     if (grad_dtype == ABS_GRAD_F32) {
         const unsigned long long n_vec = P / 4;
         if (n <= 4) {   // few gradients: two vectors per thread keep enough loads in flight
             const unsigned grid = grid_for(n_vec, kBlock * 2, ctas_per_sm, num_sms);
-            if (overwrite) k_accumulate_multi_f32<2, 4, true><<<grid, kBlock, 0, stream>>>(acc_row, gl, n, n_vec, P, cnt);
-            else k_accumulate_multi_f32<2, 4, false><<<grid, kBlock, 0, stream>>>(acc_row, gl, n, n_vec, P, cnt);
-        } else if (n <= 6) {
+            return launch_kernel(overwrite ? k_accumulate_multi_f32<2, 4, true> : k_accumulate_multi_f32<2, 4, false>, grid, kBlock,
+                                 0, stream, chained, acc_row, gl, n, n_vec, P_, cnt);
+        }
+        if (n <= 6) {
             const unsigned grid = grid_for(n_vec, kBlock * 2, ctas_per_sm, num_sms);
-            if (overwrite) k_accumulate_multi_f32<2, 6, true><<<grid, kBlock, 0, stream>>>(acc_row, gl, n, n_vec, P, cnt);
-            else k_accumulate_multi_f32<2, 6, false><<<grid, kBlock, 0, stream>>>(acc_row, gl, n, n_vec, P, cnt);
-        } else {
-            const unsigned grid = grid_for(n_vec, kBlock, ctas_per_sm, num_sms);
-            if (overwrite) k_accumulate_multi_f32<1, 8, true><<<grid, kBlock, 0, stream>>>(acc_row, gl, n, n_vec, P, cnt);
-            else k_accumulate_multi_f32<1, 8, false><<<grid, kBlock, 0, stream>>>(acc_row, gl, n, n_vec, P, cnt);
+            return launch_kernel(overwrite ? k_accumulate_multi_f32<2, 6, true> : k_accumulate_multi_f32<2, 6, false>, grid, kBlock,
+                                 0, stream, chained, acc_row, gl, n, n_vec, P_, cnt);
         }
-    } else {
-        const unsigned long long n_vec8 = P / 8;
-        if (n <= 4) {
-            const unsigned grid = grid_for(n_vec8, kBlock * 2, ctas_per_sm, num_sms);
-            if (overwrite) k_accumulate_multi_bf16<2, 4, true><<<grid, kBlock, 0, stream>>>(acc_row, gl, n, n_vec8, P, cnt);
-            else k_accumulate_multi_bf16<2, 4, false><<<grid, kBlock, 0, stream>>>(acc_row, gl, n, n_vec8, P, cnt);
-        } else {
-            const unsigned grid = grid_for(n_vec8, kBlock, ctas_per_sm, num_sms);
-            if (overwrite) k_accumulate_multi_bf16<1, 8, true><<<grid, kBlock, 0, stream>>>(acc_row, gl, n, n_vec8, P, cnt);
-            else k_accumulate_multi_bf16<1, 8, false><<<grid, kBlock, 0, stream>>>(acc_row, gl, n, n_vec8, P, cnt);
-        }
+        const unsigned grid = grid_for(n_vec, kBlock, ctas_per_sm, num_sms);
+        return launch_kernel(overwrite ? k_accumulate_multi_f32<1, 8, true> : k_accumulate_multi_f32<1, 8, false>, grid, kBlock, 0,
+                             stream, chained, acc_row, gl, n, n_vec, P_, cnt);
     }
-    return cudaGetLastError();
+    const unsigned long long n_vec8 = P / 8;
+    if (n <= 4) {
+        const unsigned grid = grid_for(n_vec8, kBlock * 2, ctas_per_sm, num_sms);
+        return launch_kernel(overwrite ? k_accumulate_multi_bf16<2, 4, true> : k_accumulate_multi_bf16<2, 4, false>, grid, kBlock, 0,
+                             stream, chained, acc_row, gl, n, n_vec8, P_, cnt);
+    }
+    const unsigned grid = grid_for(n_vec8, kBlock, ctas_per_sm, num_sms);
+    return launch_kernel(overwrite ? k_accumulate_multi_bf16<1, 8, true> : k_accumulate_multi_bf16<1, 8, false>, grid, kBlock, 0,
+                         stream, chained, acc_row, gl, n, n_vec8, P_, cnt);
 }
 
-cudaError_t launch_sync(const SyncArgs& a, int ctas_per_sm, int num_sms, cudaStream_t stream) {
+cudaError_t launch_sync(const SyncArgs& a, int ctas_per_sm, int num_sms, cudaStream_t stream, bool chained) {
     // The bulk-copy kernel (sync_tma.cu) gives the same bits; which form is faster depends on W and on whether
     // the step runs alone or beside the next iteration's accumulate kernels (pipelined mode).  Measured on a B200
     // (P = 25.6 M, every W from 2 to 24):
@@ -583,8 +592,8 @@ cudaError_t launch_sync(const SyncArgs& a, int ctas_per_sm, int num_sms, cudaStr
     constexpr unsigned kBulkOverlapped = 0x1FFFFu << 5;                   // 5 - 21
     const bool bulk_default = a.W < 32 && (((a.overlapped ? kBulkOverlapped : kBulkAlone) >> a.W) & 1u);
     const bool long_enough = a.n_vec >= (1ull << 18);   // short vectors are launch-bound: keep the lighter kernel
-    if (ctas_per_sm == -2 || (ctas_per_sm == 0 && bulk_default && long_enough && !a.norm_out)) {
-        const cudaError_t e = launch_sync_tma(a, num_sms, stream);
+    if (!a.plain_only && (ctas_per_sm == -2 || (ctas_per_sm == 0 && bulk_default && long_enough && !a.norm_out))) {
+        const cudaError_t e = launch_sync_tma(a, num_sms, stream, chained);
         if (e != cudaErrorNotSupported) return e;
         ctas_per_sm = 0;
     }
@@ -598,26 +607,25 @@ cudaError_t launch_sync(const SyncArgs& a, int ctas_per_sm, int num_sms, cudaStr
     //            long enough and one tile per CTA wins again (6.2 - 6.4 TB/s).
     if (a.W > 4) {
         if (ctas_per_sm == 0) ctas_per_sm = a.W <= 24 ? 2 : -1;
-        return launch_sync_t<0, 1>(a, ctas_per_sm, num_sms, stream);
+        return launch_sync_t<0, 1>(a, ctas_per_sm, num_sms, stream, chained);
     }
     if (ctas_per_sm == 0) ctas_per_sm = -1;
     switch (a.W) {
-        case 1: return launch_sync_t<1, 2>(a, ctas_per_sm, num_sms, stream);
-        case 2: return launch_sync_t<2, 1>(a, ctas_per_sm, num_sms, stream);
-        case 3: return launch_sync_t<3, 1>(a, ctas_per_sm, num_sms, stream);
-        default: return launch_sync_t<4, 1>(a, ctas_per_sm, num_sms, stream);
+        case 1: return launch_sync_t<1, 2>(a, ctas_per_sm, num_sms, stream, chained);
+        case 2: return launch_sync_t<2, 1>(a, ctas_per_sm, num_sms, stream, chained);
+        case 3: return launch_sync_t<3, 1>(a, ctas_per_sm, num_sms, stream, chained);
+        default: return launch_sync_t<4, 1>(a, ctas_per_sm, num_sms, stream, chained);
     }
 }
 
-cudaError_t launch_sync_global(const GlobalSyncArgs& a, int ctas_per_sm, int num_sms, cudaStream_t stream) {
+cudaError_t launch_sync_global(const GlobalSyncArgs& a, int ctas_per_sm, int num_sms, cudaStream_t stream, bool chained) {
     // Chunked rows like the one-GPU kernel for W > 4.  Default grid: 6 CTAs per SM (3 are resident at 74
     // registers), never more CTAs than the slice has tiles.  Measured with all ranks on one B200: 2 to 8 per SM
     // differ by a few per cent, one tile per CTA is 25 - 40 % slower.
     const unsigned long long n = a.vec_hi > a.vec_lo ? a.vec_hi - a.vec_lo : 0;
     if (ctas_per_sm == 0) ctas_per_sm = 6;
     const unsigned grid = grid_for(n, kBlock, ctas_per_sm, num_sms);
-    k_sync_global<<<grid, kBlock, 0, stream>>>(a);
-    return cudaGetLastError();
+    return launch_kernel(k_sync_global, grid, kBlock, 0, stream, chained, a);
 }
 
 cudaError_t launch_global_counts(int32_t* gcnt, int32_t* cnt, int own_lo, int W_local, int n_total, cudaStream_t stream) {

@@ -13,13 +13,10 @@
 // K = mb = 64), K-major: A = X^T stored [d_in][64], B = dZ^T stored [d_h][64].  A 64-element
 // bf16 row is exactly one 128-byte swizzle row, so each operand tile is one TMA box.
 //
-// Kernels (five launches per call of 1..4 micro-batches; only the first reads the caller's buffers, the
-// others may run on another stream):
-//   k_cast_x        X fp32 -> bf16 in both orientations
-//   (k_fwd_fused    k_fwd1_tcgen05 + k_fwd2 in one kernel: the K splits of a hidden tile form a thread-block cluster
-//                   and are added up through distributed shared memory; same bits, selectable)
+// Kernels (five launches per call of 1..4 micro-batches, chained by programmatic dependent launch; only the
+// first reads the caller's buffers, the others may run on another stream):
+//   k_cast_x        X (fp32 or bf16) -> bf16 in both orientations, labels copied
 //   k_fwd1_tcgen05  Z^T partials = W1^T X^T, split over d_in, on tcgen05 (W1 as an MN-major operand)
-//   (k_fwd1         the same on CUDA cores, kept as a cross-check selectable through abs_set_launch)
 //   k_fwd2          Z = sum of partials + b1, bf16(H), partial logits per 32 hidden units; the last CTA of
 //                   each group of 8 ("last CTA done" ticket) sums the group's partial logits in a fixed order
 //   k_bwd           every CTA: logits = sum of group partials + b2, softmax, dL (CTA 0: db2 += ...); then
@@ -29,13 +26,12 @@
 //                   accumulators, finished tiles leave by TMA store (a worker's first gradient of an iteration)
 //                   or TMA reduce-add; 128 x 64 or 128 x 128 tiles
 //   k_dw1_regs      one 128 x 64 tile per CTA, the accumulator tile prefetched into registers, K-batched
-//   k_dw1_tcgen05   one tile per CTA, the accumulator tile by TMA load / add in shared memory / TMA store
-//                   (or TMA reduce-add); the first version, kept selectable
 #include <cuda.h>
 
 #include <cstdio>
 
 #include "abs_internal.h"
+#include "bulk_copy.cuh"
 
 namespace abs_sgd {
 
@@ -43,7 +39,7 @@ namespace {
 
 constexpr int kMB = 64;          // samples per micro-batch = K of the dW1 contraction
 constexpr int kOutPad = 16;      // logits / dL rows are padded to 16 columns
-constexpr int kSplitK = 4;       // forward GEMM: d_in is split into at most this many partial sums
+constexpr int kSplitK = 4;       // forward GEMM: d_in is split into at most this many partial sums (stride of zpart)
 constexpr int kHB = 32;          // hidden units per CTA in k_fwd2 / k_bwd
 constexpr int kGroup = 8;        // CTAs per first-level group of the logit reduction
 constexpr int kMaxBatch = kMlpMaxBatch;   // micro-batches one call may carry (grid dimension of the front kernels)
@@ -59,81 +55,40 @@ __device__ __forceinline__ uint32_t pack_bf16x2(float a, float b) {
 // Also copies the labels, so that the caller's buffers are read by this kernel only (the rest of
 // the gradient may run on another stream after the caller's stream has moved on).
 // --------------------------------------------------------------------------------------------
-__global__ void __launch_bounds__(256) k_cast_x(const float* __restrict__ x, const int32_t* __restrict__ y,
+template <bool kBf16In>   // the caller's X already holds bf16 values: copied (and transposed) as they are
+__global__ void __launch_bounds__(256) k_cast_x(const void* __restrict__ x_in, const int32_t* __restrict__ y,
                                                 __nv_bfloat16* __restrict__ xb, __nv_bfloat16* __restrict__ xtb,
                                                 int32_t* __restrict__ ycopy, int d_in) {
     __shared__ __nv_bfloat16 tile[16][kMB + 8];
     const int c0 = blockIdx.x * 16;
+    pdl_wait();
+    pdl_trigger();
     if (blockIdx.x == 0 && threadIdx.x < kMB) ycopy[blockIdx.y * kMB + threadIdx.x] = y[blockIdx.y * kMB + threadIdx.x];
-    x += (size_t)blockIdx.y * kMB * d_in;      // micro-batch blockIdx.y of the call
-    xb += (size_t)blockIdx.y * kMB * d_in;
+    const size_t mb_off = (size_t)blockIdx.y * kMB * d_in;   // micro-batch blockIdx.y of the call
+    xb += mb_off;
     xtb += (size_t)blockIdx.y * d_in * kMB;
     {
         const int r = threadIdx.x / 4, q = threadIdx.x % 4;
-        const float4 v = *reinterpret_cast<const float4*>(x + (size_t)r * d_in + c0 + 4 * q);
+        const size_t at = (size_t)r * d_in + c0 + 4 * q;
         uint2 pk;
-        pk.x = pack_bf16x2(v.x, v.y);
-        pk.y = pack_bf16x2(v.z, v.w);
-        *reinterpret_cast<uint2*>(xb + (size_t)r * d_in + c0 + 4 * q) = pk;
-        tile[4 * q + 0][r] = __float2bfloat16_rn(v.x);
-        tile[4 * q + 1][r] = __float2bfloat16_rn(v.y);
-        tile[4 * q + 2][r] = __float2bfloat16_rn(v.z);
-        tile[4 * q + 3][r] = __float2bfloat16_rn(v.w);
+        if (kBf16In) {
+            pk = *reinterpret_cast<const uint2*>(static_cast<const __nv_bfloat16*>(x_in) + mb_off + at);
+        } else {
+            const float4 v = *reinterpret_cast<const float4*>(static_cast<const float*>(x_in) + mb_off + at);
+            pk.x = pack_bf16x2(v.x, v.y);
+            pk.y = pack_bf16x2(v.z, v.w);
+        }
+        *reinterpret_cast<uint2*>(xb + at) = pk;
+        tile[4 * q + 0][r] = __ushort_as_bfloat16((unsigned short)(pk.x & 0xFFFFu));
+        tile[4 * q + 1][r] = __ushort_as_bfloat16((unsigned short)(pk.x >> 16));
+        tile[4 * q + 2][r] = __ushort_as_bfloat16((unsigned short)(pk.y & 0xFFFFu));
+        tile[4 * q + 3][r] = __ushort_as_bfloat16((unsigned short)(pk.y >> 16));
     }
     __syncthreads();
     {
         const int c = threadIdx.x / 16, r4 = (threadIdx.x % 16) * 4;
         uint2 pk = *reinterpret_cast<const uint2*>(&tile[c][r4]);
         *reinterpret_cast<uint2*>(xtb + (size_t)(c0 + c) * kMB + r4) = pk;
-    }
-}
-
-// --------------------------------------------------------------------------------------------
-// Forward GEMM, CUDA cores (cross-check):  zpart[s][h][r] = sum_{k in split s} W1b[k][h] * xb[r][k]
-// CTA tile: 64 hidden x 64 samples, 256 threads, 4x4 outputs per thread; gridDim.y = number of splits.
-// --------------------------------------------------------------------------------------------
-__global__ void __launch_bounds__(256) k_fwd1(const __nv_bfloat16* __restrict__ w1b, const __nv_bfloat16* __restrict__ xb,
-                                              float* __restrict__ zpart, int d_in, int d_h) {
-    constexpr int KT = 32;
-    __shared__ float sw[KT][64 + 4];   // [k][h]
-    __shared__ float sx[KT][64 + 4];   // [k][r]
-    const int h0 = blockIdx.x * 64;
-    const int s = blockIdx.y;
-    xb += (size_t)blockIdx.z * kMB * d_in;                   // micro-batch blockIdx.z of the call
-    zpart += (size_t)blockIdx.z * kSplitK * d_h * kMB;
-    const int k_per = d_in / (int)gridDim.y;
-    const int kbeg = s * k_per, kend = kbeg + k_per;
-    const int th = threadIdx.x / 16, tr = threadIdx.x % 16;   // 16 x 16 threads, 4 h x 4 r each
-    float acc[4][4] = {};
-    for (int k0 = kbeg; k0 < kend; k0 += KT) {
-        for (int e = threadIdx.x; e < KT * 64; e += 256) {
-            const int k = e / 64, h = e % 64;
-            sw[k][h] = bf16_to_f(w1b[(size_t)(k0 + k) * d_h + h0 + h]);
-        }
-        for (int e = threadIdx.x; e < KT * 64; e += 256) {
-            const int r = e / KT, k = e % KT;
-            sx[k][r] = bf16_to_f(xb[(size_t)r * d_in + k0 + k]);
-        }
-        __syncthreads();
-#pragma unroll 8
-        for (int k = 0; k < KT; ++k) {
-            float a[4], b[4];
-#pragma unroll
-            for (int i = 0; i < 4; ++i) a[i] = sw[k][th * 4 + i];
-#pragma unroll
-            for (int j = 0; j < 4; ++j) b[j] = sx[k][tr * 4 + j];
-#pragma unroll
-            for (int i = 0; i < 4; ++i)
-#pragma unroll
-                for (int j = 0; j < 4; ++j) acc[i][j] = fmaf(a[i], b[j], acc[i][j]);
-        }
-        __syncthreads();
-    }
-    float* out = zpart + (size_t)s * d_h * kMB;
-#pragma unroll
-    for (int i = 0; i < 4; ++i) {
-        float4 v = make_float4(acc[i][0], acc[i][1], acc[i][2], acc[i][3]);
-        *reinterpret_cast<float4*>(out + (size_t)(h0 + th * 4 + i) * kMB + tr * 4) = v;
     }
 }
 
@@ -171,6 +126,10 @@ __global__ void __launch_bounds__(256) k_fwd2(const float* zpart, int nsplit, co
         float z[8];
 #pragma unroll
         for (int j = 0; j < 8; ++j) z[j] = b1[h_beg + g * 8 + j];
+        // up to here only parameters were read (published before the call started); zpart comes from the
+        // forward GEMM just ahead on the stream
+        pdl_wait();
+        pdl_trigger();
         for (int s = 0; s < nsplit; ++s)
 #pragma unroll
             for (int j = 0; j < 8; ++j) z[j] += zpart[((size_t)s * d_h + h_beg + g * 8 + j) * kMB + r];
@@ -244,6 +203,12 @@ __global__ void __launch_bounds__(256) k_bwd(const __nv_bfloat16* hbt, const flo
     gpart += (size_t)jb * n_groups * kMB * kOutPad;
     y += (size_t)jb * kMB;
     const int r = threadIdx.x % kMB, g = threadIdx.x / kMB;
+    for (int e = threadIdx.x; e < kHB * kOutPad; e += 256) {   // parameters: published before the call started
+        const int hl = e / kOutPad, o = e % kOutPad;
+        sw2[hl][o] = o < d_out ? bf16_to_f(w2b[(size_t)(h_beg + hl) * d_out + o]) : 0.f;
+    }
+    pdl_wait();                                      // hbt and gpart come from k_fwd2, just ahead on the stream
+    pdl_trigger();
     float hv[8];                                     // issued first: independent of the logit sums below
 #pragma unroll
     for (int j = 0; j < 8; ++j) hv[j] = bf16_to_f(hbt[(size_t)(h_beg + g * 8 + j) * kMB + r]);
@@ -281,10 +246,6 @@ __global__ void __launch_bounds__(256) k_bwd(const __nv_bfloat16* hbt, const flo
             sdl32[rr][o] = gl;
             sdl[rr][o] = bf16_to_f(__float2bfloat16_rn(gl));
         }
-    }
-    for (int e = threadIdx.x; e < kHB * kOutPad; e += 256) {
-        const int hl = e / kOutPad, o = e % kOutPad;
-        sw2[hl][o] = o < d_out ? bf16_to_f(w2b[(size_t)(h_beg + hl) * d_out + o]) : 0.f;
     }
     __syncthreads();
     float db2 = 0.f;                                 // CTA column 0, thread o < d_out: sum_r dL[r][o]
@@ -356,31 +317,6 @@ __global__ void __launch_bounds__(256) k_bwd(const __nv_bfloat16* hbt, const flo
 // ============================================================================================
 // tcgen05 / TMA / mbarrier helpers
 // ============================================================================================
-constexpr uint32_t kSpinLimit = 1u << 22;
-
-__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
-
-__device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
-    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count) : "memory");
-}
-__device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, uint32_t bytes) {
-    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
-    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
-}
-// Bounded wait: gives up after kSpinLimit polls and reports failure instead of hanging.
-__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity) {
-    const uint32_t addr = smem_u32(bar);
-    for (uint32_t it = 0; it < kSpinLimit; ++it) {
-        uint32_t ok;
-        asm volatile(
-            "{\n .reg .pred p;\n mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n selp.u32 %0, 1, 0, p;\n}\n"
-            : "=r"(ok) : "r"(addr), "r"(parity) : "memory");
-        if (ok) return true;
-    }
-    return false;
-}
 __device__ __forceinline__ void tma_load_2d(void* dst, const CUtensorMap* tm, int x, int y, uint64_t* bar) {
     asm volatile(
         "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
@@ -461,123 +397,16 @@ __device__ __forceinline__ void panel_row_update(float* panel, int row, const ui
 }
 
 // ============================================================================================
-// dW1 = X^T dZ on tcgen05.  One CTA per 128 x kDwN output tile; K = 64 = four UMMA steps.
+// dW1 = X^T dZ on tcgen05, 128 x 64 output tiles; one micro-batch is K = 64 = four UMMA steps.
 // ============================================================================================
 constexpr int kTileM = 128;
 constexpr int kDwN = 64;
 constexpr int kPanels = kDwN / 32;
 
-struct DwSmem {
-    alignas(1024) uint8_t a[kTileM * 128];            // A tile  [128 m][64 k] bf16, swizzled rows
-    alignas(1024) uint8_t b[kDwN * 128];              // B tile  [kDwN n][64 k] bf16
-    alignas(1024) float c[kPanels][kTileM * 32];      // accumulator tile as column panels [128][32] fp32, swizzled rows
-    alignas(8) uint64_t bar_ab;
-    uint64_t bar_c;
-    uint64_t bar_mma;
-    uint32_t tmem_base;
-    uint32_t failed;
-};
-
-template <bool kReduce>
-__global__ void __launch_bounds__(128) k_dw1_tcgen05(const __grid_constant__ CUtensorMap tm_xt,
-                                                     const __grid_constant__ CUtensorMap tm_dzt,
-                                                     const __grid_constant__ CUtensorMap tm_acc, int store,
-                                                     int* status) {
-    // store != 0: the accumulator slice is known to hold nothing yet (a worker's first gradient of the
-    // iteration): the tile is not read, the product is stored instead of added.
-    extern __shared__ uint8_t smem_raw[];
-    DwSmem& s = *reinterpret_cast<DwSmem*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
-    const int warp = threadIdx.x / 32;
-    const bool load_c = !kReduce && !store;
-    const int n0 = blockIdx.x * kDwN;     // hidden offset
-    const int m0 = blockIdx.y * kTileM;   // input-feature offset
-
-    if (warp == 0) {
-        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&s.tmem_base)), "r"(kDwN) : "memory");
-        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
-    }
-    if (threadIdx.x == 0) {
-        mbar_init(&s.bar_ab, 1);
-        mbar_init(&s.bar_c, 1);
-        mbar_init(&s.bar_mma, 1);
-        s.failed = 0;
-        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-    }
-    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
-    __syncthreads();
-    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-    const uint32_t tmem = s.tmem_base;
-
-    if (threadIdx.x == 0) {
-        mbar_expect_tx(&s.bar_ab, kTileM * 128 + kDwN * 128);
-        tma_load_2d(s.a, &tm_xt, 0, m0, &s.bar_ab);
-        tma_load_2d(s.b, &tm_dzt, 0, n0, &s.bar_ab);
-        if (load_c) {   // the accumulator tile streams in while the MMA runs
-            mbar_expect_tx(&s.bar_c, kTileM * kDwN * 4);
-#pragma unroll
-            for (int p = 0; p < kPanels; ++p) tma_load_2d(s.c[p], &tm_acc, n0 + p * 32, m0, &s.bar_c);
-        }
-        if (mbar_wait(&s.bar_ab, 0)) {
-            asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-            const uint64_t da = umma_desc_k_sw128(smem_u32(s.a));
-            const uint64_t db = umma_desc_k_sw128(smem_u32(s.b));
-            constexpr uint32_t idesc = umma_idesc_bf16(kTileM, kDwN);
-#pragma unroll
-            for (int k = 0; k < kMB / 16; ++k)   // K advances by 16 bf16 = 32 bytes: +2 in the address field
-                umma_bf16(tmem, da + 2 * k, db + 2 * k, idesc, k > 0);
-            umma_commit(&s.bar_mma);
-        } else {
-            s.failed = 1;
-        }
-    }
-    __syncwarp();
-
-    bool ok = mbar_wait(&s.bar_mma, 0);
-    if (load_c) ok = mbar_wait(&s.bar_c, 0) && ok;
-    ok = __all_sync(0xffffffffu, ok);
-    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-    if (ok) {
-        const int row = threadIdx.x;                    // TMEM lane = output row
-#pragma unroll 1
-        for (int p = 0; p < kPanels; ++p) {
-            uint32_t v[32];
-            tmem_ld_32(tmem + ((uint32_t)(warp * 32) << 16) + (uint32_t)(p * 32), v);
-            if (load_c) panel_row_update<true>(s.c[p], row, v);
-            else panel_row_update<false>(s.c[p], row, v);
-        }
-        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // smem writes -> visible to the TMA engine
-    } else {
-        s.failed = 1;
-    }
-    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
-    __syncthreads();
-    if (threadIdx.x == 0) {
-        if (!s.failed) {
-#pragma unroll
-            for (int p = 0; p < kPanels; ++p) {
-                if (kReduce && !store) tma_reduce_add_2d(&tm_acc, s.c[p], n0 + p * 32, m0);
-                else tma_store_2d(&tm_acc, s.c[p], n0 + p * 32, m0);
-            }
-            asm volatile("cp.async.bulk.commit_group;" ::: "memory");
-            // shared memory may be released once the engine has read it; the global writes complete on their own
-            asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
-        } else {
-            atomicExch(status, ABS_ETIMEOUT);
-            // give copies that may still be in flight a bounded chance to land before smem is released
-            mbar_wait(&s.bar_ab, 0);
-            if (load_c) mbar_wait(&s.bar_c, 0);
-        }
-    }
-    __syncthreads();
-    if (warp == 0) {
-        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(kDwN) : "memory");
-    }
-}
-
 // ============================================================================================
-// dW1 with a register-prefetched accumulator tile, optionally K-batched.  Same tile as
-// k_dw1_tcgen05, but the fp32 accumulator tile never goes through TMA: every thread loads its
-// 8 float4 of the tile with plain coalesced loads at kernel entry (all in flight while the
+// dW1 with a register-prefetched accumulator tile, optionally K-batched.  One CTA per tile; the fp32
+// accumulator tile never goes through TMA: every thread loads its 8 float4 of the tile with plain
+// coalesced loads at kernel entry (all in flight while the kernel ahead on the stream finishes, the
 // operands arrive and the MMAs run), the TMEM result is transposed through a padded shared-memory
 // tile, and the sums go back with coalesced stores.
 // K batching: the operands of nb (1..kMaxBatch) micro-batches are stacked along K, so one launch
@@ -620,7 +449,10 @@ __global__ void __launch_bounds__(256) k_dw1_regs(const __grid_constant__ CUtens
 #pragma unroll
     for (int k = 0; k < kPer; ++k) {
         const int e = threadIdx.x + 256 * k;
-        c[k] = store ? make_float4(0.f, 0.f, 0.f, 0.f) : gbase[(size_t)(e / kC4) * ld4 + (e % kC4)];   // store: see k_dw1_tcgen05
+        // store: the slice holds nothing yet (a worker's first gradient of the iteration), so it is not read.
+        // These loads stand in front of pdl_wait(): the slice was last written by a kernel at least two places
+        // ahead on this stream (the previous dW1 of this worker) or by work ordered before the whole call.
+        c[k] = store ? make_float4(0.f, 0.f, 0.f, 0.f) : gbase[(size_t)(e / kC4) * ld4 + (e % kC4)];
     }
 
     if (warp == 0) {
@@ -637,6 +469,8 @@ __global__ void __launch_bounds__(256) k_dw1_regs(const __grid_constant__ CUtens
     __syncthreads();
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
     const uint32_t tmem = s.tmem_base;
+    pdl_wait();      // dzt comes from k_bwd, just ahead on the stream
+    pdl_trigger();
 
     if (threadIdx.x == 0) {
         mbar_expect_tx(&s.bar_ab, nb * kDwOperandBytes);
@@ -770,6 +604,8 @@ __global__ void __launch_bounds__(192) k_dw1_ring(const __grid_constant__ CUtens
     __syncthreads();
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
     const uint32_t tmem = s.tmem_base;
+    pdl_wait();      // dzt comes from k_bwd, just ahead on the stream
+    pdl_trigger();
 
     if (warp == 0) {
         if (lane == 0) {                             // ---- TMA producer
@@ -938,6 +774,8 @@ __global__ void __launch_bounds__(128) k_fwd1_tcgen05(const __grid_constant__ CU
     __syncthreads();
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
     const uint32_t tmem = s.tmem_base;
+    pdl_wait();      // xb comes from k_cast_x, just ahead (possibly on another stream, then ordered by an event)
+    pdl_trigger();
 
     if (warp == 0 && lane == 0) {                    // ---- TMA producer
         for (int kb = 0; kb < nk; ++kb) {
@@ -1011,248 +849,6 @@ __global__ void __launch_bounds__(128) k_fwd1_tcgen05(const __grid_constant__ CU
     }
 }
 
-// ============================================================================================
-// Forward, fused:  k_fwd1_tcgen05 + k_fwd2 in one kernel.  The CTAs that hold the K splits of one
-// 128-hidden tile form a thread-block cluster (1 x nsplit x 1).  Each runs the same TMA -> MMA
-// pipeline as k_fwd1_tcgen05, then parks its partial accumulator [128][64 NB] in its own shared
-// memory (the pipeline stages are free by then); after a cluster barrier, CTA rank q adds up rows
-// [q 128/nsplit, (q+1) 128/nsplit) of all nsplit partials through distributed shared memory, in
-// rank order (fixed summation order), and does k_fwd2's work for those hidden units: bias, ReLU,
-// bf16 H -> hbt, partial logits -> lpart, group ticket -> gpart.  The split-K partials never
-// leave the SMs (k_fwd1_tcgen05 writes and k_fwd2 re-reads 4 bytes x nsplit per element of Z).
-// ============================================================================================
-__device__ __forceinline__ float4 ld_dsmem_f4(uint32_t local_addr, uint32_t rank) {
-    uint32_t remote;
-    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(remote) : "r"(local_addr), "r"(rank));
-    float4 v;
-    asm volatile("ld.shared::cluster.v4.f32 {%0,%1,%2,%3}, [%4];" : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "r"(remote));
-    return v;
-}
-__device__ __forceinline__ void cluster_sync_all() {
-    asm volatile("barrier.cluster.arrive.release.aligned;\n barrier.cluster.wait.acquire.aligned;" ::: "memory");
-}
-
-template <int NB>
-__global__ void __launch_bounds__(128) k_fwd_fused(const __grid_constant__ CUtensorMap tm_w1,
-                                                   const __grid_constant__ CUtensorMap tm_xb, const float* __restrict__ b1,
-                                                   const __nv_bfloat16* __restrict__ w2b, __nv_bfloat16* hbt, float* lpart,
-                                                   float* gpart, unsigned int* tickets, int d_in, int d_h, int d_out,
-                                                   int* status) {
-    constexpr int kFwdStages = FwdCfg<NB>::kStages, kFwdStageBytes = FwdCfg<NB>::kStageBytes;
-    constexpr int kTmemCols = FwdCfg<NB>::kTmemCols;
-    constexpr int kPitch = 64 * NB + 4;              // floats per row of the parked partial (conflict-free float4 rows)
-    static_assert(128 * kPitch * 4 <= kFwdStages * kFwdStageBytes, "the parked partial must fit into the stages");
-    extern __shared__ uint8_t smem_raw[];
-    FwdSmem<NB>& s = *reinterpret_cast<FwdSmem<NB>*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
-    __shared__ float sh[kHB][kMB + 1];
-    __shared__ float sw2[kHB][kOutPad];
-    __shared__ unsigned int s_last[2 * kMaxBatch];
-    const int warp = threadIdx.x / 32, lane = threadIdx.x % 32;
-    const int h0 = blockIdx.x * 128;
-    const int nsplit = gridDim.y;                    // = cluster size
-    const int split = blockIdx.y;
-    const int k_per = d_in / nsplit;
-    const int kbeg = split * k_per;
-    const int nk = k_per / 64;                       // pipeline steps of 64 k
-    uint32_t rank;
-    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(rank));
-
-    if (warp == 0) {
-        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&s.tmem_base)), "r"(kTmemCols) : "memory");
-        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
-    }
-    if (threadIdx.x == 0) {
-        for (int i = 0; i < kFwdStages; ++i) {
-            mbar_init(&s.full[i], 1);
-            mbar_init(&s.empty[i], 1);
-        }
-        mbar_init(&s.done, 1);
-        s.failed = 0;
-        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-    }
-    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
-    __syncthreads();
-    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-    const uint32_t tmem = s.tmem_base;
-
-    if (warp == 0 && lane == 0) {                    // ---- TMA producer
-        for (int kb = 0; kb < nk; ++kb) {
-            const int st = kb % kFwdStages;
-            if (kb >= kFwdStages && !mbar_wait(&s.empty[st], ((kb / kFwdStages) - 1) & 1)) { s.failed = 1; break; }
-            mbar_expect_tx(&s.full[st], kFwdStageBytes);
-            const int k0 = kbeg + kb * 64;
-            tma_load_2d(s.stage[st], &tm_w1, h0, k0, &s.full[st]);
-            tma_load_2d(s.stage[st] + 8192, &tm_w1, h0 + 64, k0, &s.full[st]);
-#pragma unroll
-            for (int jb = 0; jb < NB; ++jb)
-                tma_load_2d(s.stage[st] + 16384 + jb * 8192, &tm_xb, k0, jb * kMB, &s.full[st]);
-        }
-    } else if (warp == 1 && lane == 0) {             // ---- MMA issuer
-        constexpr uint32_t idesc = umma_idesc_bf16(128, 64 * NB) | (1u << 15);   // A is MN-major
-        bool ok = true;
-        for (int kb = 0; kb < nk && ok; ++kb) {
-            const int st = kb % kFwdStages;
-            ok = mbar_wait(&s.full[st], (kb / kFwdStages) & 1);
-            if (!ok) break;
-            asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-            const uint32_t a0 = smem_u32(s.stage[st]);
-            const uint64_t db = umma_desc_k_sw128(a0 + 16384);
-#pragma unroll
-            for (int k = 0; k < 4; ++k)
-                umma_bf16(tmem, umma_desc_mn_sw128(a0 + k * 2048, 8192), db + 2 * k, idesc, (kb > 0 || k > 0));
-            umma_commit(&s.empty[st]);
-        }
-        if (ok) umma_commit(&s.done);
-        else s.failed = 1;
-    }
-    __syncwarp();
-
-    bool ok = mbar_wait(&s.done, 0);
-    ok = __all_sync(0xffffffffu, ok);
-    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-    float* red = reinterpret_cast<float*>(s.stage[0]);   // every load has landed, every MMA has completed
-    if (ok) {
-        const int row = warp * 32 + lane;            // TMEM lane = hidden unit within the tile
-#pragma unroll 1
-        for (int p = 0; p < 2 * NB; ++p) {
-            uint32_t v[32];
-            tmem_ld_32(tmem + ((uint32_t)(warp * 32) << 16) + (uint32_t)(p * 32), v);
-#pragma unroll
-            for (int j = 0; j < 8; ++j)
-                *reinterpret_cast<float4*>(red + row * kPitch + p * 32 + 4 * j) =
-                    make_float4(__uint_as_float(v[4 * j]), __uint_as_float(v[4 * j + 1]), __uint_as_float(v[4 * j + 2]),
-                                __uint_as_float(v[4 * j + 3]));
-        }
-    } else if (threadIdx.x == 0) {
-        atomicExch(status, ABS_ETIMEOUT);
-        for (int i = 0; i < kFwdStages; ++i) mbar_wait(&s.full[i], 0);   // bounded chance for copies in flight to land
-    }
-    __syncwarp();
-    // From here on every CTA of the cluster takes the same path (also after a failed wait: its numbers are
-    // then meaningless and the status word says so), so that both cluster barriers and every ticket are met.
-    cluster_sync_all();
-    {
-        const int rows_per_rank = 128 / nsplit, n_chunk = rows_per_rank / kHB;   // 32 (64) rows = 1 (2) chunks of 32
-        const int n_cta2 = d_h / kHB, n_groups = (n_cta2 + kGroup - 1) / kGroup; // chunk = what one k_fwd2 CTA handles
-        const uint32_t red_addr = smem_u32(red);
-        for (int ch = 0; ch < n_chunk; ++ch) {
-            const int hl0 = (int)rank * rows_per_rank + ch * kHB;                 // first tile row of the chunk
-            const int cta2 = (h0 + hl0) / kHB;
-            for (int e = threadIdx.x; e < kHB * kOutPad; e += 128) {
-                const int hl = e / kOutPad, o = e % kOutPad;
-                sw2[hl][o] = o < d_out ? bf16_to_f(w2b[(size_t)(h0 + hl0 + hl) * d_out + o]) : 0.f;
-            }
-#pragma unroll 1
-            for (int jb = 0; jb < NB; ++jb) {
-                // Z = sum over the K splits (rank order) + b1 ; H = bf16(relu(Z)) -> hbt and sh.
-                // All 4 x nsplit remote loads of a thread are issued before the first add.
-                float4 part[4][kSplitK];
-#pragma unroll
-                for (int k = 0; k < 4; ++k) {
-                    const int hl = threadIdx.x / 16 + 8 * k, r4 = (threadIdx.x % 16) * 4;
-                    const uint32_t off = red_addr + (uint32_t)(((hl0 + hl) * kPitch + jb * kMB + r4) * 4);
-#pragma unroll
-                    for (int sp = 0; sp < kSplitK; ++sp)
-                        if (sp < nsplit) part[k][sp] = ld_dsmem_f4(off, (uint32_t)sp);
-                }
-#pragma unroll
-                for (int k = 0; k < 4; ++k) {
-                    const int hl = threadIdx.x / 16 + 8 * k, r4 = (threadIdx.x % 16) * 4;
-                    const int h = h0 + hl0 + hl;
-                    const float bias = b1[h];
-                    float4 z = make_float4(bias, bias, bias, bias);
-#pragma unroll
-                    for (int sp = 0; sp < kSplitK; ++sp)
-                        if (sp < nsplit) { z.x += part[k][sp].x; z.y += part[k][sp].y; z.z += part[k][sp].z; z.w += part[k][sp].w; }
-                    const __nv_bfloat16 q0 = __float2bfloat16_rn(z.x > 0.f ? z.x : 0.f), q1 = __float2bfloat16_rn(z.y > 0.f ? z.y : 0.f);
-                    const __nv_bfloat16 q2 = __float2bfloat16_rn(z.z > 0.f ? z.z : 0.f), q3 = __float2bfloat16_rn(z.w > 0.f ? z.w : 0.f);
-                    uint2 pk;
-                    pk.x = (uint32_t)__bfloat16_as_ushort(q0) | ((uint32_t)__bfloat16_as_ushort(q1) << 16);
-                    pk.y = (uint32_t)__bfloat16_as_ushort(q2) | ((uint32_t)__bfloat16_as_ushort(q3) << 16);
-                    *reinterpret_cast<uint2*>(hbt + ((size_t)jb * d_h + h) * kMB + r4) = pk;
-                    sh[hl][r4 + 0] = bf16_to_f(q0); sh[hl][r4 + 1] = bf16_to_f(q1);
-                    sh[hl][r4 + 2] = bf16_to_f(q2); sh[hl][r4 + 3] = bf16_to_f(q3);
-                }
-                __syncthreads();
-                {   // partial logits of these 32 hidden units: thread = (sample r, 8 of the 16 padded outputs)
-                    const int r = threadIdx.x / 2, og = threadIdx.x % 2;
-                    float a[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
-#pragma unroll 8
-                    for (int hl = 0; hl < kHB; ++hl) {
-                        const float hv = sh[hl][r];
-#pragma unroll
-                        for (int j = 0; j < 8; ++j) a[j] = fmaf(hv, sw2[hl][8 * og + j], a[j]);
-                    }
-                    float4* dst = reinterpret_cast<float4*>(lpart + ((size_t)jb * n_cta2 + cta2) * (kMB * kOutPad)) + r * 4 + og * 2;
-                    dst[0] = make_float4(a[0], a[1], a[2], a[3]);
-                    dst[1] = make_float4(a[4], a[5], a[6], a[7]);
-                }
-                __syncthreads();                     // sh is rewritten by the next micro-batch
-            }
-            __syncthreads();                         // sw2 is rewritten by the next chunk
-        }
-        // ---- group tickets (one per chunk and micro-batch), as in k_fwd2
-        __threadfence();
-        __syncthreads();
-        const int n_units = n_chunk * NB;
-        if ((int)threadIdx.x < n_units) {
-            const int ch = threadIdx.x / NB, jb = threadIdx.x % NB;
-            const int cta2 = (h0 + (int)rank * rows_per_rank + ch * kHB) / kHB;
-            const int group = cta2 / kGroup, g_count = min(kGroup, n_cta2 - group * kGroup);
-            s_last[threadIdx.x] = (atomicAdd(&tickets[(size_t)jb * n_groups + group], 1u) == (unsigned)(g_count - 1));
-        }
-        __syncthreads();
-        for (int u = 0; u < n_units; ++u) {
-            if (!s_last[u]) continue;
-            __threadfence();
-            const int ch = u / NB, jb = u % NB;
-            const int cta2 = (h0 + (int)rank * rows_per_rank + ch * kHB) / kHB;
-            const int group = cta2 / kGroup, g_first = group * kGroup, g_count = min(kGroup, n_cta2 - g_first);
-            const float4* lp = reinterpret_cast<const float4*>(lpart + (size_t)jb * n_cta2 * (kMB * kOutPad));
-            float4* gp = reinterpret_cast<float4*>(gpart + ((size_t)jb * n_groups + group) * (kMB * kOutPad));
-            for (int i = threadIdx.x; i < kMB * kOutPad / 4; i += 128) {
-                float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-                for (int c = 0; c < g_count; ++c) {
-                    const float4 v = __ldcg(lp + (size_t)(g_first + c) * (kMB * kOutPad / 4) + i);
-                    acc.x += v.x; acc.y += v.y; acc.z += v.z; acc.w += v.w;
-                }
-                gp[i] = acc;
-            }
-            if (threadIdx.x == 0) tickets[(size_t)jb * n_groups + group] = 0u;   // ready for the next launch
-        }
-    }
-    cluster_sync_all();                              // nobody leaves while its shared memory may still be read
-    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
-    __syncthreads();
-    if (warp == 0) {
-        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(kTmemCols) : "memory");
-    }
-}
-
-template <int NB>
-cudaError_t fwd_fused_set_attr() {
-    return cudaFuncSetAttribute(k_fwd_fused<NB>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(FwdSmem<NB>) + 1024);
-}
-// Launch with the nsplit CTAs of a hidden tile as one thread-block cluster.
-template <int NB>
-cudaError_t fwd_fused_launch(int n_tiles, int nsplit, cudaStream_t stream, const CUtensorMap& tw, const CUtensorMap& tx,
-                             const float* b1, const __nv_bfloat16* w2b, __nv_bfloat16* hbt, float* lpart, float* gpart,
-                             unsigned int* tickets, int d_in, int d_h, int d_out, int* status) {
-    cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3(n_tiles, nsplit, 1);
-    cfg.blockDim = dim3(128, 1, 1);
-    cfg.dynamicSmemBytes = sizeof(FwdSmem<NB>) + 1024;
-    cfg.stream = stream;
-    cudaLaunchAttribute attr[1];
-    attr[0].id = cudaLaunchAttributeClusterDimension;
-    attr[0].val.clusterDim.x = 1;
-    attr[0].val.clusterDim.y = nsplit;
-    attr[0].val.clusterDim.z = 1;
-    cfg.attrs = attr;
-    cfg.numAttrs = 1;
-    return cudaLaunchKernelEx(&cfg, k_fwd_fused<NB>, tw, tx, b1, w2b, hbt, lpart, gpart, tickets, d_in, d_h, d_out, status);
-}
-
 template <int NB>
 cudaError_t fwd1_set_attr() {
     cudaError_t e = cudaFuncSetAttribute(k_fwd1_tcgen05<NB, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
@@ -1261,15 +857,6 @@ cudaError_t fwd1_set_attr() {
     return cudaFuncSetAttribute(k_fwd1_tcgen05<NB, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                 (int)sizeof(FwdSmem<NB, true>) + 1024);
 }
-template <int NB>
-void fwd1_launch(dim3 grid, cudaStream_t stream, bool light, const CUtensorMap& tw, const CUtensorMap& tx, float* zpart,
-                 int d_in, int d_h, int* status) {
-    if (light)
-        k_fwd1_tcgen05<NB, true><<<grid, 128, sizeof(FwdSmem<NB, true>) + 1024, stream>>>(tw, tx, zpart, d_in, d_h, status);
-    else
-        k_fwd1_tcgen05<NB, false><<<grid, 128, sizeof(FwdSmem<NB, false>) + 1024, stream>>>(tw, tx, zpart, d_in, d_h, status);
-}
-
 // ---- host helpers --------------------------------------------------------------------------
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
@@ -1379,19 +966,10 @@ cudaError_t mlp_scratch_init(MlpScratch* s, const MlpDims& d, void* base, __nv_b
     if (e == cudaSuccess)
         e = cudaFuncSetAttribute(k_dw1_regs, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                  dw_regs_buf_bytes(kMaxBatch) + (int)sizeof(DwRegCtl) + 1024);
-    if (e == cudaSuccess)
-        e = fwd1_set_attr<1>();
-        if (e == cudaSuccess) e = fwd1_set_attr<2>();
-        if (e == cudaSuccess) e = fwd1_set_attr<3>();
-        if (e == cudaSuccess) e = fwd1_set_attr<4>();
-        if (e == cudaSuccess) e = fwd_fused_set_attr<1>();
-        if (e == cudaSuccess) e = fwd_fused_set_attr<2>();
-        if (e == cudaSuccess) e = fwd_fused_set_attr<3>();
-        if (e == cudaSuccess) e = fwd_fused_set_attr<4>();
-    if (e == cudaSuccess)
-        e = cudaFuncSetAttribute(k_dw1_tcgen05<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(DwSmem) + 1024);
-    if (e == cudaSuccess)
-        e = cudaFuncSetAttribute(k_dw1_tcgen05<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(DwSmem) + 1024);
+    if (e == cudaSuccess) e = fwd1_set_attr<1>();
+    if (e == cudaSuccess) e = fwd1_set_attr<2>();
+    if (e == cudaSuccess) e = fwd1_set_attr<3>();
+    if (e == cudaSuccess) e = fwd1_set_attr<4>();
     if (e != cudaSuccess) *err = "cudaFuncSetAttribute(tcgen05 kernels)";
     return e;
 }
@@ -1404,113 +982,112 @@ cudaError_t mlp_make_acc_tmap(void* tmap_out, const MlpDims& d, float* acc_row) 
                : cudaErrorInvalidValue;
 }
 
-cudaError_t launch_mlp_cast(const MlpDims& d, const MlpScratch& s, int slot0, int nb, const float* x_dev, const int32_t* y_dev,
-                            cudaStream_t stream, MlpMark mark, void* user) {
-    mark(user, ABS_K_MLP_FWD, 0, stream);
+cudaError_t launch_mlp_cast(const MlpDims& d, const MlpScratch& s, int slot0, int nb, const void* x_dev, bool x_is_bf16,
+                            const int32_t* y_dev, cudaStream_t stream, bool chained, MlpMark mark, void* user) {
+    mark(user, ABS_K_MLP_FWD, -1, stream);   // part 0 of the forward class: the cast
     // micro-batch j of the call goes to slot slot0 + j of the scratch set
-    k_cast_x<<<dim3(d.d_in / 16, nb), 256, 0, stream>>>(x_dev, y_dev, s.xb + (size_t)slot0 * kMB * d.d_in,
-                                                        s.xtb + (size_t)slot0 * d.d_in * kMB, s.ycopy + slot0 * kMB, d.d_in);
-    return cudaGetLastError();
+    __nv_bfloat16* xb = s.xb + (size_t)slot0 * kMB * d.d_in;
+    __nv_bfloat16* xtb = s.xtb + (size_t)slot0 * d.d_in * kMB;
+    int32_t* yc = s.ycopy + slot0 * kMB;
+    const dim3 grid(d.d_in / 16, nb);
+    const cudaError_t e = x_is_bf16 ? launch_kernel(k_cast_x<true>, grid, 256, 0, stream, chained, x_dev, y_dev, xb, xtb, yc, d.d_in)
+                                    : launch_kernel(k_cast_x<false>, grid, 256, 0, stream, chained, x_dev, y_dev, xb, xtb, yc, d.d_in);
+    mark(user, ABS_K_MLP_FWD, 1, stream);
+    return e;
+}
+
+template <int NB>
+cudaError_t fwd1_launch(dim3 grid, cudaStream_t stream, bool chained, bool light, const CUtensorMap& tw, const CUtensorMap& tx,
+                        float* zpart, int d_in, int d_h, int* status) {
+    if (light)
+        return launch_kernel(k_fwd1_tcgen05<NB, true>, grid, 128, sizeof(FwdSmem<NB, true>) + 1024, stream, chained, tw, tx, zpart,
+                             d_in, d_h, status);
+    return launch_kernel(k_fwd1_tcgen05<NB, false>, grid, 128, sizeof(FwdSmem<NB, false>) + 1024, stream, chained, tw, tx, zpart,
+                         d_in, d_h, status);
 }
 
 cudaError_t launch_mlp_front(const MlpDims& d, const MlpScratch& s, const float* x_pub, const __nv_bfloat16* shadow,
                              int shadow_idx, int nb, bool store, float* acc_row, int32_t* cnt, int variant,
-                             cudaStream_t stream, MlpMark mark, void* user) {
+                             cudaStream_t stream, int chain, MlpMark mark, void* user) {
     const size_t o_b1 = (size_t)d.d_in * d.d_hidden, o_w2 = o_b1 + d.d_hidden, o_b2 = o_w2 + (size_t)d.d_hidden * d.d_out;
     cudaError_t e;
     const unsigned n_cta = d.d_hidden / kHB;
     const bool light = (variant & kMlpLightBit) != 0;
 
-    // every K split must be a whole number of 64-wide pipeline steps (d_in is a multiple of 128)
-    const int nsplit = (d.d_in % (64 * kSplitK) == 0) ? kSplitK : 2;
-    const CUtensorMap* tw = reinterpret_cast<const CUtensorMap*>(&s.tmap_w1[shadow_idx]);
-    const CUtensorMap* tx = reinterpret_cast<const CUtensorMap*>(&s.tmap_xb);
-    if ((variant & 64) && !(variant & 2)) {
-        // one kernel: forward GEMM, split-K sum through the cluster's shared memory, bias / ReLU / logits.  Same
-        // bits as the two-kernel path; measured slower when several workers' calls overlap (its 128 CTAs keep a
-        // whole SM's shared memory each while 128 threads do the epilogue work), so it is not the default.
-        const int n_tiles = d.d_hidden / 128;
-        const float* b1 = x_pub + o_b1;
-        const __nv_bfloat16* w2b = shadow + o_w2;
-        switch (nb) {
-            case 1: e = fwd_fused_launch<1>(n_tiles, nsplit, stream, *tw, *tx, b1, w2b, s.hbt, s.lpart, s.gpart, s.tickets, d.d_in, d.d_hidden, d.d_out, s.status); break;
-            case 2: e = fwd_fused_launch<2>(n_tiles, nsplit, stream, *tw, *tx, b1, w2b, s.hbt, s.lpart, s.gpart, s.tickets, d.d_in, d.d_hidden, d.d_out, s.status); break;
-            case 3: e = fwd_fused_launch<3>(n_tiles, nsplit, stream, *tw, *tx, b1, w2b, s.hbt, s.lpart, s.gpart, s.tickets, d.d_in, d.d_hidden, d.d_out, s.status); break;
-            default: e = fwd_fused_launch<4>(n_tiles, nsplit, stream, *tw, *tx, b1, w2b, s.hbt, s.lpart, s.gpart, s.tickets, d.d_in, d.d_hidden, d.d_out, s.status); break;
-        }
-        if (e != cudaSuccess) return e;
-    } else {
-        if (variant & 2) {
-            k_fwd1<<<dim3(d.d_hidden / 64, nsplit, nb), 256, 0, stream>>>(shadow, s.xb, s.zpart, d.d_in, d.d_hidden);
-        } else {
-            const dim3 grid(d.d_hidden / 128, nsplit);
-            switch (nb) {                                // the nb micro-batches are stacked along N of one GEMM
-                case 1: fwd1_launch<1>(grid, stream, light, *tw, *tx, s.zpart, d.d_in, d.d_hidden, s.status); break;
-                case 2: fwd1_launch<2>(grid, stream, light, *tw, *tx, s.zpart, d.d_in, d.d_hidden, s.status); break;
-                case 3: fwd1_launch<3>(grid, stream, light, *tw, *tx, s.zpart, d.d_in, d.d_hidden, s.status); break;
-                default: fwd1_launch<4>(grid, stream, light, *tw, *tx, s.zpart, d.d_in, d.d_hidden, s.status); break;
-            }
-        }
-        k_fwd2<<<dim3(n_cta, nb), 256, 0, stream>>>(s.zpart, nsplit, x_pub + o_b1, shadow + o_w2, s.hbt, s.lpart, s.gpart,
-                                                    s.tickets, d.d_hidden, d.d_out);
+    // every K split must be a whole number of 64-wide pipeline steps (d_in is a multiple of 128).  Eight splits (256
+    // CTAs, two per SM) measured slower than four: 34.7 against 33.4 us per micro-batch, 16.7 against 15.5 batched.
+    int nsplit = kSplitK;
+    while (nsplit > 1 && d.d_in % (64 * nsplit) != 0) nsplit /= 2;
+    const CUtensorMap& tw = *reinterpret_cast<const CUtensorMap*>(&s.tmap_w1[shadow_idx]);
+    const CUtensorMap& tx = *reinterpret_cast<const CUtensorMap*>(&s.tmap_xb);
+    const dim3 grid(d.d_hidden / 128, nsplit);
+    mark(user, ABS_K_MLP_FWD, -2, stream);       // part 1: the forward GEMM
+    switch (nb) {                                // the nb micro-batches are stacked along N of one GEMM
+        case 1: e = fwd1_launch<1>(grid, stream, (chain & kChainFwd1) != 0, light, tw, tx, s.zpart, d.d_in, d.d_hidden, s.status); break;
+        case 2: e = fwd1_launch<2>(grid, stream, (chain & kChainFwd1) != 0, light, tw, tx, s.zpart, d.d_in, d.d_hidden, s.status); break;
+        case 3: e = fwd1_launch<3>(grid, stream, (chain & kChainFwd1) != 0, light, tw, tx, s.zpart, d.d_in, d.d_hidden, s.status); break;
+        default: e = fwd1_launch<4>(grid, stream, (chain & kChainFwd1) != 0, light, tw, tx, s.zpart, d.d_in, d.d_hidden, s.status); break;
     }
-    mark(user, ABS_K_MLP_FWD, ((variant & 64) && !(variant & 2)) ? 2 : 3, stream);   // launches of the group, the cast included
-    if ((e = cudaGetLastError()) != cudaSuccess) return e;
+    mark(user, ABS_K_MLP_FWD, 1, stream);
+    if (e != cudaSuccess) return e;
+    mark(user, ABS_K_MLP_FWD, -3, stream);       // part 2: bias, ReLU, partial logits
+    const float* zp = s.zpart;
+    const float* b1 = x_pub + o_b1;
+    const __nv_bfloat16* w2b = shadow + o_w2;
+    e = launch_kernel(k_fwd2, dim3(n_cta, nb), 256, 0, stream, (chain & kChainFwd2) != 0, zp, nsplit, b1, w2b, s.hbt, s.lpart, s.gpart, s.tickets,
+                      d.d_hidden, d.d_out);
+    mark(user, ABS_K_MLP_FWD, 1, stream);
+    if (e != cudaSuccess) return e;
 
-    mark(user, ABS_K_MLP_BWD, 0, stream);
+    mark(user, ABS_K_MLP_BWD, -1, stream);
     const int n_groups = (n_cta + kGroup - 1) / kGroup;
-    k_bwd<<<dim3(n_cta, nb), 256, 0, stream>>>(s.hbt, s.gpart, n_groups, x_pub + o_b2, s.ycopy, shadow + o_w2, s.dzt, s.bpart,
-                                               s.tickets_b, acc_row + o_b1, acc_row + o_w2, acc_row + o_b2, cnt, d.d_hidden,
-                                               d.d_out, store ? 1 : 0);
+    const __nv_bfloat16* hbt = s.hbt;
+    const float* gpart = s.gpart;
+    const float* b2 = x_pub + o_b2;
+    const int32_t* yc = s.ycopy;
+    e = launch_kernel(k_bwd, dim3(n_cta, nb), 256, 0, stream, (chain & kChainBwd) != 0, hbt, gpart, n_groups, b2, yc, w2b, s.dzt, s.bpart,
+                      s.tickets_b, acc_row + o_b1, acc_row + o_w2, acc_row + o_b2, cnt, d.d_hidden, d.d_out, store ? 1 : 0);
     mark(user, ABS_K_MLP_BWD, 1, stream);
-    return cudaGetLastError();
+    return e;
+}
+
+template <int kN, bool kLight>
+cudaError_t dw1_ring_launch(const MlpDims& d, const MlpScratch& s, const CUtensorMap& ta, const CUtensorMap& tb,
+                            const CUtensorMap& tc, int nb, int st, cudaStream_t stream, bool chained) {
+    const int n_tiles_n = d.d_hidden / kN, n_tiles = n_tiles_n * (d.d_in / kTileM);
+    const int ctas = n_tiles < s.num_sms ? n_tiles : s.num_sms;
+    return launch_kernel(k_dw1_ring<kN, kLight>, ctas, 192, sizeof(DwRingSmem<kN, kLight>) + 1024, stream, chained, ta, tb, tc,
+                         n_tiles_n, n_tiles, d.d_in, d.d_hidden, nb, st, s.status);
 }
 
 cudaError_t launch_mlp_dw1(const MlpDims& d, const MlpScratch& s, float* acc_row, const void* acc_tmap, int nb, bool store,
-                           int variant, cudaStream_t stream, MlpMark mark, void* user) {
+                           int variant, cudaStream_t stream, bool chained, MlpMark mark, void* user) {
     const int st = store ? 1 : 0;
     const bool light = (variant & kMlpLightBit) != 0;
-    mark(user, ABS_K_MLP_DW1, 0, stream);
-    const dim3 grid(d.d_hidden / kDwN, d.d_in / kTileM);
-    const CUtensorMap* ta = reinterpret_cast<const CUtensorMap*>(&s.tmap_xt);
-    const CUtensorMap* tb = reinterpret_cast<const CUtensorMap*>(&s.tmap_dzt);
-    const CUtensorMap* tc = reinterpret_cast<const CUtensorMap*>(acc_tmap);
-    // Which kernel: bits 4 (ring), 8 (register prefetch), 16 (TMA load + add + store), 1 (TMA reduce-add) force
-    // one; otherwise the measured best for the case: the persistent ring kernel when the tile is stored (it
-    // never reads the accumulator) and for K-batched adds, the register-prefetch kernel for single adds.
-    int kind = (variant & 4) ? 4 : (variant & 8) ? 8 : (variant & 16) ? 16 : (variant & 1) ? 1 : 0;
+    mark(user, ABS_K_MLP_DW1, -1, stream);
+    const CUtensorMap& ta = *reinterpret_cast<const CUtensorMap*>(&s.tmap_xt);
+    const CUtensorMap& tb = *reinterpret_cast<const CUtensorMap*>(&s.tmap_dzt);
+    const CUtensorMap& tc = *reinterpret_cast<const CUtensorMap*>(acc_tmap);
+    // Which kernel: bit 4 (ring) or 8 (register prefetch) forces one; otherwise the measured best for the case: the
+    // persistent ring kernel when the tile is stored (it never reads the accumulator) and for K-batched adds, the
+    // register-prefetch kernel for single adds.
+    int kind = (variant & 4) ? 4 : (variant & 8) ? 8 : 0;
     if (kind == 0) kind = (store || nb > 1) ? 4 : 8;
-    if ((kind == 16 || kind == 1) && nb > 1) kind = 8;   // the one-tile-per-CTA TMA kernels are not K-batched
+    cudaError_t e;
     if (kind == 4) {
-        if (nb > 1 && !(variant & 32)) {   // K-batched: 128 x 128 tiles (bit 5 keeps 128 x 64)
-            const int n_tiles_n = d.d_hidden / 128, n_tiles = n_tiles_n * (d.d_in / kTileM);
-            const int ctas = n_tiles < s.num_sms ? n_tiles : s.num_sms;
-            if (light)
-                k_dw1_ring<128, true><<<ctas, 192, sizeof(DwRingSmem<128, true>) + 1024, stream>>>(*ta, *tb, *tc, n_tiles_n, n_tiles,
-                                                                                                 d.d_in, d.d_hidden, nb, st, s.status);
-            else
-                k_dw1_ring<128, false><<<ctas, 192, sizeof(DwRingSmem<128, false>) + 1024, stream>>>(*ta, *tb, *tc, n_tiles_n, n_tiles,
-                                                                                                   d.d_in, d.d_hidden, nb, st, s.status);
-        } else {
-            const int n_tiles_n = d.d_hidden / kDwN, n_tiles = n_tiles_n * (d.d_in / kTileM);
-            const int ctas = n_tiles < s.num_sms ? n_tiles : s.num_sms;
-            if (light)
-                k_dw1_ring<64, true><<<ctas, 192, sizeof(DwRingSmem<64, true>) + 1024, stream>>>(*ta, *tb, *tc, n_tiles_n, n_tiles,
-                                                                                               d.d_in, d.d_hidden, nb, st, s.status);
-            else
-                k_dw1_ring<64, false><<<ctas, 192, sizeof(DwRingSmem<64, false>) + 1024, stream>>>(*ta, *tb, *tc, n_tiles_n, n_tiles,
-                                                                                                 d.d_in, d.d_hidden, nb, st, s.status);
-        }
-    } else if (kind == 8) {
-        const size_t smem = dw_regs_buf_bytes(nb) + sizeof(DwRegCtl) + 1024;
-        k_dw1_regs<<<grid, 256, smem, stream>>>(*ta, *tb, acc_row, d.d_in, d.d_hidden, nb, st, s.status);
-    } else if (kind == 1) {
-        k_dw1_tcgen05<true><<<grid, 128, sizeof(DwSmem) + 1024, stream>>>(*ta, *tb, *tc, st, s.status);
+        if (nb > 1 && !(variant & 32))     // K-batched: 128 x 128 tiles (bit 32 keeps 128 x 64)
+            e = light ? dw1_ring_launch<128, true>(d, s, ta, tb, tc, nb, st, stream, chained)
+                      : dw1_ring_launch<128, false>(d, s, ta, tb, tc, nb, st, stream, chained);
+        else
+            e = light ? dw1_ring_launch<64, true>(d, s, ta, tb, tc, nb, st, stream, chained)
+                      : dw1_ring_launch<64, false>(d, s, ta, tb, tc, nb, st, stream, chained);
     } else {
-        k_dw1_tcgen05<false><<<grid, 128, sizeof(DwSmem) + 1024, stream>>>(*ta, *tb, *tc, st, s.status);
+        const size_t smem = dw_regs_buf_bytes(nb) + sizeof(DwRegCtl) + 1024;
+        e = launch_kernel(k_dw1_regs, dim3(d.d_hidden / kDwN, d.d_in / kTileM), 256, smem, stream, chained, ta, tb, acc_row, d.d_in,
+                          d.d_hidden, nb, st, s.status);
     }
     mark(user, ABS_K_MLP_DW1, 1, stream);
-    return cudaGetLastError();
+    return e;
 }
 
 }  // namespace abs_sgd

@@ -61,6 +61,19 @@ extern "C" int abs_sync_step_noalloc(float* x_dev, float* v_dev, float* acc_dev,
     if ((reinterpret_cast<uintptr_t>(x_dev) | reinterpret_cast<uintptr_t>(v_dev) | reinterpret_cast<uintptr_t>(acc_dev)) & 15)
         return ABS_EINVAL;
     if (reinterpret_cast<uintptr_t>(cnt_dev) & 3) return ABS_EINVAL;
+    // The built-in array and the launch belong to the CURRENT device: the caller's buffers must live there too.
+    // (A query of the pointer's attributes allocates nothing.)
+    {
+        int dev = -1;
+        if (cudaGetDevice(&dev) != cudaSuccess) return ABS_ECUDA;
+        const void* bufs[4] = {x_dev, v_dev, acc_dev, cnt_dev};
+        for (const void* b : bufs) {
+            cudaPointerAttributes at{};
+            if (cudaPointerGetAttributes(&at, b) != cudaSuccess) { cudaGetLastError(); return ABS_EINVAL; }
+            if ((at.type != cudaMemoryTypeDevice && at.type != cudaMemoryTypeManaged) || (at.type == cudaMemoryTypeDevice && at.device != dev))
+                return ABS_EINVAL;
+        }
+    }
 
     unsigned int* scratch = nullptr;
     int num_sms = 0;
@@ -87,5 +100,8 @@ extern "C" int abs_sync_step_noalloc(float* x_dev, float* v_dev, float* acc_dev,
     a.disp_scale = 0.0f;
     a.shadow = nullptr;
     a.zero_acc = 1;
-    return abs_sgd::launch_sync(a, 0, num_sms, s) == cudaSuccess ? ABS_OK : ABS_ECUDA;
+    // Always the load/store form of the kernel: its bulk-copy form has bounded waits whose time-out is reported
+    // through a context (abs_check), which this entry point does not have.
+    a.plain_only = 1;
+    return abs_sgd::launch_sync(a, 0, num_sms, s, false) == cudaSuccess ? ABS_OK : ABS_ECUDA;
 }

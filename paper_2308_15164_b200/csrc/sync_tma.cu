@@ -16,6 +16,7 @@
 // bounded: on a time-out the thread records ABS_ETIMEOUT in the status word and raises the CTA's abort flag, every
 // role stops taking tiles, the loader waits (bounded) for the copies it armed, and the CTA returns.
 #include "abs_internal.h"
+#include "bulk_copy.cuh"
 
 namespace abs_sgd {
 
@@ -27,7 +28,6 @@ constexpr int kConsumers = 128;
 constexpr int kLoaderTid = kConsumers, kSenderTid = kConsumers + 32;
 constexpr int kThreads = kConsumers + 64;
 constexpr int kMaxStages = 4;
-constexpr uint32_t kSpinLimit = 1u << 22;
 constexpr int kCtlBytes = 256;
 
 struct Ctl {
@@ -36,27 +36,6 @@ struct Ctl {
 };
 static_assert(sizeof(Ctl) <= kCtlBytes, "control block");
 
-__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
-__device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
-    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count) : "memory");
-}
-__device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, uint32_t bytes) {
-    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
-    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
-}
-__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity) {
-    const uint32_t addr = smem_u32(bar);
-    for (uint32_t it = 0; it < kSpinLimit; ++it) {
-        uint32_t ok;
-        asm volatile(
-            "{\n .reg .pred p;\n mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n selp.u32 %0, 1, 0, p;\n}\n"
-            : "=r"(ok) : "r"(addr), "r"(parity) : "memory");
-        if (ok) return true;
-    }
-    return false;
-}
 // global -> shared, bytes and both addresses multiples of 16; read-once data: evict-first in L2
 __device__ __forceinline__ void bulk_load(void* dst_smem, const void* src, uint32_t bytes, uint64_t* bar, uint64_t policy) {
     asm volatile(
@@ -85,7 +64,6 @@ __global__ void __launch_bounds__(kThreads) k_sync_tma(const SyncArgs a, const i
     const size_t stage_bytes = (size_t)(W + 2) * kTileBytes + kTileBytes / 2;
     const int tid = threadIdx.x;
 
-    if (tid < W) s_cnt[tid] = a.cnt[tid];
     for (int i = tid; i < kTileElems / 4; i += kThreads) zero_tile[i] = make_float4(0.f, 0.f, 0.f, 0.f);
     if (tid == 0) {
         for (int s = 0; s < n_stages; ++s) {
@@ -97,6 +75,9 @@ __global__ void __launch_bounds__(kThreads) k_sync_tma(const SyncArgs a, const i
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // the zero tile is read by the copy engine
+    pdl_wait();      // set-up above overlaps the tail of the kernel ahead on the stream; its counters and rows are read below
+    pdl_trigger();
+    if (tid < W) s_cnt[tid] = a.cnt[tid];
     __syncthreads();
 
     long long B = 0;
@@ -253,16 +234,7 @@ __global__ void k_bounded_wait_selftest(int* status, uint32_t polls) {
     if (threadIdx.x == 0) {
         mbar_init(&bar, 1);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-        const uint32_t addr = smem_u32(&bar);
-        bool done = false;
-        for (uint32_t it = 0; it < polls && !done; ++it) {
-            uint32_t ok;
-            asm volatile(
-                "{\n .reg .pred p;\n mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n selp.u32 %0, 1, 0, p;\n}\n"
-                : "=r"(ok) : "r"(addr), "r"(0u) : "memory");
-            done = ok != 0;
-        }
-        if (!done) *status = ABS_ETIMEOUT;
+        if (!mbar_wait(&bar, 0u, polls)) *status = ABS_ETIMEOUT;
     }
 }
 
@@ -273,7 +245,7 @@ cudaError_t launch_bounded_wait_selftest(int* status, cudaStream_t stream) {
     return cudaGetLastError();
 }
 
-cudaError_t launch_sync_tma(const SyncArgs& a, int num_sms, cudaStream_t stream) {
+cudaError_t launch_sync_tma(const SyncArgs& a, int num_sms, cudaStream_t stream, bool chained) {
     if (a.W < 1 || a.W > kSyncTmaMaxW || a.norm_out) return cudaErrorNotSupported;
     const size_t stage_bytes = (size_t)(a.W + 2) * kTileBytes + kTileBytes / 2;
     const size_t fixed = kCtlBytes + kTileBytes;
@@ -305,8 +277,7 @@ cudaError_t launch_sync_tma(const SyncArgs& a, int num_sms, cudaStream_t stream)
     unsigned long long grid = (unsigned long long)num_sms * ctas;
     if (grid > n_tiles) grid = n_tiles;
     if (grid == 0) grid = 1;
-    k_sync_tma<<<(unsigned)grid, kThreads, smem, stream>>>(a, stages, lazy);
-    return cudaGetLastError();
+    return launch_kernel(k_sync_tma, (unsigned)grid, kThreads, smem, stream, chained, a, stages, lazy);
 }
 
 }  // namespace abs_sgd

@@ -137,13 +137,22 @@ class GlobalStep:
         self._token = torch.zeros(1, dtype=torch.int32, device=eng.device)
         dist.barrier(group=group)
 
-    def sync_step(self):
+    def sync_step(self, timed: bool = False):
+        """One end of iteration.  timed=True returns a CUDA event pair on stream_sync around this rank's fused
+        kernel (between the two exchanges)."""
         eng = self.eng
         counts = eng.global_begin()
         exchange_counts(counts, eng.stream_sync, self.group)          # exchange A: all b_i, everywhere
+        ev = None
+        if timed:
+            ev = (torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True))
+            ev[0].record(eng.stream_sync)
         eng.global_step()
+        if timed:
+            ev[1].record(eng.stream_sync)
         exchange_counts(self._token, eng.stream_sync, self.group)     # exchange B: every rank's kernel is done
         eng.global_end()
+        return ev
 
     def close(self):
         self.eng.synchronize()

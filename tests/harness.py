@@ -12,7 +12,7 @@ TOL_F32 = 1e-5          # max |x_gpu - x_oracle| <= TOL_F32 * max |x_oracle|   (
 TOL_BF16 = 2e-3         # same bound for runs whose gradients come from bf16-operand GEMMs
 
 
-def oracle_run(wl, x0, pool, columns=None, lambda_dc=0.0, oracle_cls=None, lr_schedule=None):
+def oracle_run(wl, x0, pool, columns=None, lambda_dc=0.0, oracle_cls=None, lr_schedule=None, every_iteration=True):
     """Run the oracle over the workload (optionally restricted to `columns` of the parameter
     vector -- the path is element-wise, so a column subset evolves independently).
     Returns dict(xs=[x_1, x_2, ...], consumed=[...], states=[(cnt, cur, t) after each sync])."""
@@ -36,7 +36,8 @@ def oracle_run(wl, x0, pool, columns=None, lambda_dc=0.0, oracle_cls=None, lr_sc
                     g = g[columns]
             o.accumulate(i, g)
         o.sync_step()
-        xs.append(o.params().copy())
+        if every_iteration or t == wl.T - 1:           # (full-size runs keep the final parameters only)
+            xs.append(o.params().copy())
         states.append(o.counters())
     return dict(xs=xs, consumed=[np.asarray(c) for c in o.consumed], states=states, v=np.asarray(o.v).copy())
 

@@ -36,7 +36,7 @@ def test_every_declared_symbol_is_exported(B):
     assert {"abs_init", "abs_accumulate", "abs_accumulate_mlp", "abs_sync_step", "abs_params"} <= set(names)
     for n in names:
         assert hasattr(B.lib, n), f"{n} declared in include/ but not exported"
-        assert n in B._sig or n.endswith("_noalloc"), f"{n} has no binding signature"
+        assert n in B._sig, f"{n} has no binding signature"
 
 
 def test_workspace_bytes_host_side(B):
@@ -52,7 +52,8 @@ def test_workspace_bytes_host_side(B):
 
 
 @pytest.mark.parametrize("kw", [
-    dict(P=0, W=2), dict(P=16, W=0), dict(P=16, W=65), dict(P=16, W=2, grad_dtype=7), dict(P=16, W=2, flags=64),
+    dict(P=0, W=2), dict(P=16, W=0), dict(P=16, W=65), dict(P=16, W=2, grad_dtype=7), dict(P=16, W=2, flags=128),
+    dict(P=16, W=2, flags=64), dict(P=16, W=2, flags=16),
     dict(P=16, W=2, lr=float("nan")), dict(P=16, W=2, flags=1, stream_acc=5, stream_sync=5),
     dict(P=16, W=2, flags=2, mlp=(100, 128, 10, 64)), dict(P=16, W=2, flags=2, mlp=(128, 128, 10, 64)),
     dict(P=128 * 128 + 128 + 1280 + 10, W=2, flags=2, mlp=(128, 128, 10, 32)),

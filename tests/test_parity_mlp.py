@@ -5,10 +5,17 @@ Bars: every gradient tensor within 2e-3 * max|ref| element-wise and 2e-3 in Frob
 bf16-emulating oracle evaluated at the same parameters; end-of-run parameters within
 2e-3 * max|param|; counters bit-exact.
 
-The ReLU gate [Z > 0] is a discrete decision taken on a floating-point number.  The GPU
-accumulates Z in fp32, the oracle in fp64, so for the handful of pre-activations with
-|Z| < 1e-4 (fp32 accumulation error is ~1e-6 here) either gate value is a valid outcome.  Those
-hidden units are compared against every valid outcome; all others are compared strictly."""
+Two decisions of the path are discrete and taken on floating-point numbers; the GPU takes them on fp32
+values, the oracle on fp64 ones, so where the number sits within rounding error of the threshold both
+outcomes are valid and the comparison has to allow for either:
+  * the ReLU gate [Z > 0]: for the handful of pre-activations with |Z| < 1e-4 (fp32 accumulation error is ~1e-6
+    here) either gate value is a valid outcome.  Those hidden units are compared against every valid outcome;
+  * the rounding of dZ to bf16 in front of dW1 = X^T dZ: an entry within 1e-6 (relative; the fp32 evaluation of dH is
+    good to ~1e-7) of the midpoint between two bf16 numbers may be rounded either way, and a whole row of dZ when
+    one of the row's dL entries sits that close to a midpoint (dH = dL W2^T then moves by a fraction of a bf16
+    unit).  One bf16 unit of ONE of the 64 terms of an entry of dW1 can exceed 2e-3 of the tensor's maximum, so the
+    element-wise bar carries, for exactly those entries, the allowance |X[r, i]| * ulp_bf16(dZ[r, h]) summed over
+    the undecided (r, h) -- zero for every other entry, which is compared at the plain bar."""
 
 import itertools
 
@@ -24,22 +31,57 @@ TOL = 2e-3
 TAU = 1e-4
 
 
-def _engine(wl, x0, pipelined=False, epilogue=0, overwrite_first=False):
+def _engine(wl, x0, pipelined=False, epilogue=0, overwrite_first=False, x_bf16=False):
     import torch
 
     from paper_2308_15164_b200 import binding as B
 
     d = wl.mlp
     eng = B.AbsSgd(torch.from_numpy(x0).cuda(), wl.W, wl.lr, wl.momentum, wl.weight_decay,
-                   pipelined=pipelined, mlp=(d.d_in, d.d_hidden, d.d_out, d.mb), overwrite_first=overwrite_first)
+                   pipelined=pipelined, mlp=(d.d_in, d.d_hidden, d.d_out, d.mb), overwrite_first=overwrite_first,
+                   mlp_x_bf16=x_bf16)
     eng.set_launch(B.K_MLP_DW1, epilogue)
     return eng
 
 
-def _close(got, ref, what):
+def _close(got, ref, what, allow=None):
     scale = np.abs(ref).max()
-    assert np.abs(got - ref).max() <= TOL * scale, f"{what}: max err {np.abs(got - ref).max():.3e} vs {TOL}*{scale:.3e}"
+    err = np.abs(got - ref)
+    if allow is None:
+        assert err.max() <= TOL * scale, f"{what}: max err {err.max():.3e} vs {TOL}*{scale:.3e}"
+    else:
+        over = err - (TOL * scale + allow)
+        assert over.max() <= 0.0, f"{what}: max err {err.max():.3e} vs {TOL}*{scale:.3e} (+ allowance {allow.flat[over.argmax()]:.3e})"
     assert np.linalg.norm(got - ref) <= TOL * np.linalg.norm(ref), f"{what}: Frobenius"
+
+
+def _bf16_ulp(a):
+    """Spacing of the bf16 numbers around |a| (8 significant bits)."""
+    a = np.abs(a)
+    out = np.zeros_like(a)
+    nz = a > 0
+    out[nz] = 2.0 ** (np.floor(np.log2(a[nz])) - 7)
+    return out
+
+
+def _near_midpoint(a, rel=1e-6):
+    """Entries whose rounding to bf16 an fp32 evaluation of the same quantity may take the other way: within
+    rel * |a| of the midpoint between two neighbouring bf16 numbers."""
+    a = np.abs(a)
+    ulp = _bf16_ulp(a)
+    out = np.zeros(a.shape, dtype=bool)
+    nz = ulp > 0
+    mid = np.floor(a[nz] / ulp[nz]) * ulp[nz] + 0.5 * ulp[nz]
+    out[nz] = np.abs(a[nz] - mid) <= rel * a[nz]
+    return out
+
+
+def _dw1_allowance(aux):
+    """[d_in, d_hidden]: by how much an entry of dW1 = X^T bf16(dZ) may move through undecided bf16 roundings of dZ
+    (see the module docstring).  Zero wherever no undecided entry contributes."""
+    dZ = np.where(aux["Z"] > 0.0, aux["dH"], 0.0)
+    undecided = _near_midpoint(dZ) | _near_midpoint(aux["dL"]).any(axis=1)[:, None]
+    return np.abs(aux["X"]).T @ (_bf16_ulp(dZ) * undecided)
 
 
 def _check_gradient(got_flat, params, X, y, dims):
@@ -54,10 +96,11 @@ def _check_gradient(got_flat, params, X, y, dims):
     clear = np.setdiff1d(np.arange(d_h), amb_cols)
     _close(gW2, dW2, "dW2")
     _close(gb2, db2, "db2")
-    _close(gW1[:, clear], dW1[:, clear], "dW1")
+    allow = _dw1_allowance(aux)
+    _close(gW1[:, clear], dW1[:, clear], "dW1", allow[:, clear])
     _close(gb1[clear], db1[clear], "db1")
     # undecided gates: the column must equal the reference with some subset of them inverted
-    sW1, sb1 = TOL * np.abs(dW1).max(), TOL * np.abs(db1).max()
+    sW1, sb1 = TOL * np.abs(dW1).max() + allow.max(), TOL * np.abs(db1).max()
     for h in amb_cols:
         rows = [int(r) for r, hh in amb if hh == h]
         assert len(rows) <= 4
@@ -75,9 +118,7 @@ def _check_gradient(got_flat, params, X, y, dims):
     return len(amb)
 
 
-@pytest.mark.parametrize("epilogue", [0, 16, 1, 2, 64, 4, 8],
-                         ids=["auto", "tma-load-add-store", "tma-reduce", "cuda-core-forward", "cluster-fused-forward",
-                              "persistent-ring-dw1", "register-prefetch-dw1"])
+@pytest.mark.parametrize("epilogue", [0, 4, 8, 128], ids=["auto", "persistent-ring-dw1", "register-prefetch-dw1", "deep-pipelines"])
 @pytest.mark.parametrize("small", [True, False], ids=["384x512", "3072x4096"])
 def test_single_microbatch_gradient(small, epilogue):
     wl = wlm.config(4, small=small)
@@ -176,6 +217,160 @@ def _oracle_training(wl, x0, xs, ys):
     return o.params(), states, o.consumed
 
 
+def _oracle_gradients(p, xs, ys, calls, wl, pool):
+    """The oracle's gradients (fp32, as they enter the accumulators) and pre-activations of one iteration's
+    micro-batches, all evaluated at the parameters p.  The micro-batches are independent, so they are computed on
+    a few host threads (NumPy releases the interpreter lock inside its loops); the oracle itself is untouched."""
+    d = wl.mlp
+
+    def one(call):
+        i, k, c = call
+        _, g, aux = mlp_loss_and_grad(p, xs[c % wl.mlp_pool], ys[c % wl.mlp_pool], d.d_in, d.d_hidden, d.d_out, mode="bf16")
+        und = set(int(h) for _, h in np.argwhere(np.abs(aux["Z"]) < TAU))
+        return g.astype(np.float32), und, _dw1_allowance(aux).astype(np.float32)
+
+    return list(pool.map(one, calls))
+
+
+@pytest.mark.slow
+@pytest.mark.parametrize("small", [True, False], ids=["384x512", "3072x4096"])
+def test_workload4_full_length(small):
+    """Workload 4 as stated (3072-4096-10, W = 4, b_i ~ U{1..8}, lr 0.05, momentum 0.9, 50 iterations: 872
+    micro-batches), and its small form.
+
+    With these hyper-parameters the run is unstable -- the oracle's own loss climbs from 3 to above 20 -- and a
+    relative perturbation of 1e-6 of the gradients (fp32 rounding) has grown to several 1e-3 of the parameter
+    scale by iteration 50 in the oracle alone.  End-of-run parameters therefore cannot separate a correct fp32
+    accumulation from a wrong one at the 2e-3 bar; what is compared instead:
+      (a) every one of the 50 iterations on its own: a context started FROM THE ORACLE'S parameters x_t computes
+          that iteration's micro-batch gradients; each worker's accumulator must match the oracle's accumulator of
+          the same iteration, tensor by tensor, at the 2e-3 bars (hidden units with an undecided ReLU gate apart);
+      (b) the free-running library over all 50 iterations, eager and pipelined: bit-identical to each other,
+          counters and consumed b_i bit-exact against the oracle, parameters within 2e-3 of the oracle's while the
+          amplification is still small (iterations 1..8) and within a coarse sanity bound at the end."""
+    import concurrent.futures
+
+    import torch
+
+    from paper_2308_15164_b200 import binding as B
+
+    wl = wlm.config(4, small=small)
+    assert wl.T == 50
+    d = wl.mlp
+    dims = (d.d_in, d.d_hidden, d.d_out)
+    x0 = wlm.params0(wl)
+    xs, ys = wlm.mlp_batches(wl)
+    xs_d, ys_d = torch.from_numpy(xs).cuda(), torch.from_numpy(ys).cuda()
+    torch.cuda.synchronize()
+    o = AbsSgdOracle(x0, wl.W, wl.lr, wl.momentum, wl.weight_decay)
+    ref_xs, ref_states = [], []
+    worst = 0.0
+    with concurrent.futures.ThreadPoolExecutor(4) as pool:
+        for t, calls in enumerate(wlm.iter_calls(wl)):
+            p = o.params()                                # all micro-batches of iteration t see x_t
+            res = _oracle_gradients(p, xs, ys, calls, wl, pool)
+            und = [set() for _ in range(wl.W)]
+            allow = [0.0] * wl.W
+            for (i, k, c), (g, u, al) in zip(calls, res):
+                o.accumulate(i, g)
+                und[i] |= u
+                allow[i] = allow[i] + al
+            # (a) this iteration on the library, started from the oracle's x_t
+            eng = B.AbsSgd(torch.from_numpy(p).cuda(), wl.W, wl.lr, wl.momentum, wl.weight_decay,
+                           mlp=(d.d_in, d.d_hidden, d.d_out, d.mb))
+            for (i, k, c) in calls:
+                eng.accumulate_mlp(i, xs_d[c % wl.mlp_pool], ys_d[c % wl.mlp_pool])
+            eng.check()
+            assert np.array_equal(eng.counters()[0][0], o.cnt[o.cur])
+            for i in range(wl.W):
+                if o.cnt[o.cur, i] == 0:
+                    continue
+                got = eng.accumulator(0, i).cpu().numpy()
+                want = o.acc[o.cur, i]
+                clear = np.setdiff1d(np.arange(d.d_hidden), sorted(und[i]))
+                gW1, gb1, gW2, gb2 = mlp_split(got, *dims)
+                wW1, wb1, wW2, wb2 = mlp_split(want, *dims)
+                _close(gW2, wW2, f"iteration {t} worker {i} dW2"); _close(gb2, wb2, f"iteration {t} worker {i} db2")
+                _close(gW1[:, clear], wW1[:, clear], f"iteration {t} worker {i} dW1", allow[i][:, clear])
+                _close(gb1[clear], wb1[clear], f"iteration {t} worker {i} db1")
+                worst = max(worst, float(np.abs(gW1[:, clear] - wW1[:, clear]).max() / np.abs(wW1).max()))
+                if und[i]:
+                    u = sorted(und[i])
+                    assert np.abs(gW1[:, u] - wW1[:, u]).max() <= 0.2 * np.abs(wW1).max()
+            eng.destroy()
+            o.sync_step()
+            ref_xs.append(o.params())
+            ref_states.append(o.counters())
+    ref = ref_xs[-1]
+    assert np.abs(ref - x0).max() > 1e-2 * np.abs(x0).max()
+    print(f"workload 4 ({'small' if small else 'full size'}): worst per-iteration dW1 deviation {worst:.2e} of max|dW1|")
+    # (b) the free-running library
+    outs = []
+    for pipelined in (False, True):
+        eng = _engine(wl, x0, pipelined=pipelined)
+        states, early = [], 0.0
+        for t, calls in enumerate(wlm.iter_calls(wl)):
+            for (i, k, c) in calls:
+                eng.accumulate_mlp(i, xs_d[c % wl.mlp_pool], ys_d[c % wl.mlp_pool])
+            eng.sync_step()
+            states.append(eng.counters())
+            if t < 8:
+                got_t = eng.params_host()
+                err = np.abs(got_t.astype(np.float64) - ref_xs[t]).max() / np.abs(ref_xs[t]).max()
+                assert err <= TOL, f"pipelined={pipelined}, x_{t + 1}: {err:.3e}"
+                early = max(early, err)
+        eng.check()
+        got = eng.params_host()
+        consumed = [eng.consumed(s) for s in range(len(states))]
+        eng.destroy()
+        end = np.abs(got.astype(np.float64) - ref).max() / np.abs(ref).max()
+        print(f"  free run, pipelined={pipelined}: x_1..x_8 within {early:.2e}, x_50 within {end:.2e} of max|x|")
+        assert end <= 0.1, "the free run left the oracle's neighbourhood altogether"
+        for (c1, cur1, t1), (c2, cur2, t2) in zip(states, ref_states):
+            assert np.array_equal(c1, c2) and (cur1, t1) == (cur2, t2)
+        for a, b in zip(consumed, o.consumed):
+            assert np.array_equal(a, b)
+        outs.append(got)
+    assert np.array_equal(outs[0], outs[1]), "eager and pipelined runs must be bit-identical"
+
+
+@pytest.mark.parametrize("n", [1, 3])
+@pytest.mark.parametrize("small", [True, False], ids=["384x512", "3072x4096"])
+def test_bf16_x_input(small, n):
+    """ABS_FLAG_MLP_X_BF16: the caller hands over X as bf16 values.  They enter the GEMMs as they are, so the
+    accumulator equals, bit for bit, that of an fp32 call fed the same (bf16-representable) values, and matches
+    the oracle evaluated on them."""
+    import torch
+
+    wl = wlm.config(4, small=small)
+    d = wl.mlp
+    dims = (d.d_in, d.d_hidden, d.d_out)
+    x0 = wlm.params0(wl)
+    xs, ys = wlm.mlp_batches(wl)
+    bits = wlm.f32_to_bf16_bits(xs[30:30 + n])                      # input preparation: X given as bf16
+    x_as_f32 = wlm.bf16_bits_to_f32(bits)
+    xb_d = torch.from_numpy(bits.view(np.int16)).cuda().view(torch.bfloat16).contiguous()
+    xf_d = torch.from_numpy(x_as_f32).cuda().contiguous()
+    y_d = torch.from_numpy(ys[30:30 + n]).cuda().contiguous()
+    torch.cuda.synchronize()
+    outs = []
+    for x_bf16, xd in ((True, xb_d), (False, xf_d)):
+        eng = _engine(wl, x0, x_bf16=x_bf16)
+        if n == 1:
+            eng.accumulate_mlp(2, xd, y_d)
+            eng.accumulate_mlp(2, xd, y_d)                          # second call: the adding path
+        else:
+            eng.accumulate_mlp_batch(2, n, xd, y_d)
+            eng.accumulate_mlp_batch(2, n, xd, y_d)
+        eng.check()
+        assert eng.counters()[0][0].tolist() == [0, 0, 2 * n, 0]
+        outs.append(eng.accumulator(0, 2).cpu().numpy())
+        eng.destroy()
+    assert np.array_equal(outs[0], outs[1])
+    if n == 1:
+        _check_gradient(outs[0] * 0.5, x0, x_as_f32[0], ys[30], dims)   # g + g = 2 g exactly in fp32
+
+
 @pytest.mark.parametrize("small,T", [(True, 12), (False, 5)], ids=["384x512-T12", "3072x4096-T5"])
 def test_training_run_matches_oracle(small, T):
     wl = wlm.config(4, small=small, T=T)
@@ -224,15 +419,17 @@ def test_batched_microbatches_match_the_sum_of_gradients(small, n, epilogue):
     assert eng.counters()[0][0].tolist() == [0, 0, 0, n]
     want = np.zeros(wl.P)
     undecided = set()
+    allow = 0.0
     for j in range(n):
         _, g, aux = mlp_loss_and_grad(x0, xs[b0 + j], ys[b0 + j], *dims, mode="bf16")
         want += g
         undecided |= set(int(h) for _, h in np.argwhere(np.abs(aux["Z"]) < TAU))
+        allow = allow + _dw1_allowance(aux)
     clear = np.setdiff1d(np.arange(d.d_hidden), sorted(undecided))
     gW1, gb1, gW2, gb2 = mlp_split(got, *dims)
     wW1, wb1, wW2, wb2 = mlp_split(want, *dims)
     _close(gW2, wW2, "dW2"); _close(gb2, wb2, "db2")
-    _close(gW1[:, clear], wW1[:, clear], "dW1"); _close(gb1[clear], wb1[clear], "db1")
+    _close(gW1[:, clear], wW1[:, clear], "dW1", allow[:, clear]); _close(gb1[clear], wb1[clear], "db1")
     # hidden units with an undecided ReLU gate: bounded by the contribution of those few gates
     if undecided:
         u = sorted(undecided)
@@ -321,30 +518,3 @@ def test_mixed_calls_idle_workers_and_batches(pipelined, overwrite_first):
     assert np.abs(got.astype(np.float64) - ref).max() <= TOL * np.abs(ref).max()
     for a, b in zip(consumed, o.consumed):
         assert np.array_equal(a, b)
-
-
-@pytest.mark.parametrize("n", [1, 2, 3, 4])
-@pytest.mark.parametrize("small", [True, False], ids=["384x512", "3072x4096"])
-def test_cluster_fused_forward_is_bit_identical_to_the_two_kernel_forward(small, n):
-    """The cluster kernel adds the K-split partial sums in the same order as k_fwd2 does: same H, same logits,
-    hence the same accumulator bits."""
-    import torch
-
-    wl = wlm.config(4, small=small)
-    x0 = wlm.params0(wl)
-    rng = np.random.default_rng(3)
-    d = wl.mlp
-    o_w1, o_b1, o_w2, o_b2 = d.offsets
-    x0[o_b1:o_w2] = rng.standard_normal(d.d_hidden).astype(np.float32) * 0.1
-    xs, ys = wlm.mlp_batches(wl)
-    xd, yd = torch.from_numpy(xs[20:20 + n]).cuda().contiguous(), torch.from_numpy(ys[20:20 + n]).cuda().contiguous()
-    torch.cuda.synchronize()
-    outs = []
-    for variant in (0, 64):
-        eng = _engine(wl, x0, epilogue=variant)
-        eng.accumulate_mlp_batch(1, n, xd, yd)
-        eng.accumulate_mlp_batch(1, n, xd, yd)
-        eng.check()
-        outs.append(eng.accumulator(0, 1).cpu().numpy())
-        eng.destroy()
-    assert np.array_equal(outs[0], outs[1])

@@ -94,6 +94,26 @@ def test_full_size_sampled_columns(cfg, T):
     _check(wl, True, columns=cols, every_iteration=False)
 
 
+@pytest.mark.slow
+@pytest.mark.parametrize("cfg,T", [(2, 100), (3, 200), (5, 20)])
+def test_full_size_every_element(cfg, T):
+    """Workloads 2, 3 and 5 at their full size and length in the bench's launch configuration (pipelined), EVERY
+    parameter compared with the oracle -- its C form, which the CPU suite holds to the NumPy oracle within 1e-7
+    and which runs the full vectors in tens of seconds on the host cores."""
+    from oracle.c_oracle import AbsSgdOracleC
+
+    wl = wlm.config(cfg, T=T)
+    x0 = wlm.params0(wl)
+    pool = wlm.grad_pool(wl)
+    ref = H.oracle_run(wl, x0, pool, oracle_cls=AbsSgdOracleC, every_iteration=False)
+    got = H.gpu_run(wl, x0, pool, True, every_iteration=False)
+    H.assert_states_equal(got, ref)
+    assert got["xs"][-1].shape == (wl.P,)
+    rel = H.assert_params_close(got["xs"][-1], ref["xs"][-1], what=f"{wl.name} x_T, all {wl.P} parameters")
+    assert np.abs(ref["xs"][-1] - x0).max() > 1e-3 * np.abs(x0).max()      # the run moved the parameters
+    print(f"workload {cfg}: max |x_gpu - x_oracle| / max|x| = {rel:.2e} over {wl.P} parameters")
+
+
 # ------------------------------------------------------------------ edge cases
 @pytest.mark.parametrize("P", [1, 3, 4, 5, 255, 256, 257, 1023, 4097, 65537])
 @pytest.mark.parametrize("dtype", ["f32", "bf16"])
