@@ -258,7 +258,7 @@ def run_ours(args):
     sampler = ClockSampler(local_rank)
     secs_w, _, _ = timed(eng, max(args.steps // 10, 2), args.warmup)      # warm-up (outside the clock samples)
     est = secs_w / max(args.steps // 10, 2)
-    repeats = int(min(max(1, np.ceil(MIN_TIMED_SECONDS / max(est * args.steps, 1e-9))), 200))
+    repeats = int(min(max(1, np.ceil(args.min_seconds / max(est * args.steps, 1e-9))), 200))
     repeats = int(D.reduce_max(float(repeats), dev))                      # the same count on every rank
     sampler.start()
     regions = [timed(eng, args.steps, 0) for _ in range(repeats)]
@@ -367,7 +367,7 @@ def run_ours(args):
         "config": {"workload": WORKLOAD, "mode": "pipelined (two streams)", "l2": "inputs larger than L2: gradient pool "
                    "748 MB cycled, accumulators 374 MB", "parallelism": f"replicas x{world}", "bytes_per_step": step_bytes},
         "timing": {"repeats": repeats, "what": f"the {args.steps}-step region repeated {repeats} times (at least "
-                   f"{MIN_TIMED_SECONDS} s in all); ms_per_step and value are the median repetition",
+                   f"{args.min_seconds} s in all); ms_per_step and value are the median repetition",
                    "ms_per_step_min": secs_all[0] / args.steps * 1e3, "ms_per_step_max": secs_all[-1] / args.steps * 1e3,
                    "us_per_step_x_sm_mhz": (ms_step * 1e3 * clocks["sm_mhz"]) if clocks["sm_mhz"] else None},
         "frac_of_measured_hbm": value / world / peaks["hbm_gbs"],
@@ -541,10 +541,11 @@ def run_other_workloads(B, wlm, dev):
     return out
 
 
-def run_sync_curve(B, dev, peaks, P=11_689_512):
-    """The fused step alone on the GPU (eager mode, an event pair around every launch) for several worker
-    counts W, every worker active: GB/s on its algorithmic bytes (8 W + 16) P.  For W <= 2 the accumulators
-    written just before partly sit in the 126 MB L2, so those two points are optimistic."""
+def run_sync_curve(B, dev, peaks, P=25_557_032):
+    """The fused step alone on the GPU (eager mode, an event pair around every launch -- the pairs keep the launch
+    from being chained to the kernel ahead, so every figure includes the kernel's own ramp and tail) for several
+    worker counts W, every worker active: GB/s on its algorithmic bytes (8 W + 16) P, at the size of workload 3's
+    vector.  For W = 1 the accumulator written just before partly sits in the 126 MB L2: that point is optimistic."""
     import torch
 
     out = {"P": P, "unit": "GB/s on (8*W + 16) * P bytes", "peak": peaks["hbm_gbs"]}
@@ -561,7 +562,8 @@ def run_sync_curve(B, dev, peaks, P=11_689_512):
                     eng.sync_step()
             n, ms = eng.kernel_stats(B.K_SYNC)
             eng.profile(False)
-        out[str(W)] = {"us": ms / n * 1e3, "gbs": (8 * W + 16) * P / (ms / n) / 1e6}
+        gbs = (8 * W + 16) * P / (ms / n) / 1e6
+        out[str(W)] = {"us": ms / n * 1e3, "gbs": gbs, "frac_of_measured_hbm": gbs / peaks["hbm_gbs"]}
         eng.check(); eng.destroy()
     return out
 
@@ -802,8 +804,9 @@ def run_mlp(B, wlm, dev, peaks, iters=12):
             run(True)
             st = {nm: eng.kernel_stats(k) for nm, k in (("fwd", B.K_MLP_FWD), ("bwd", B.K_MLP_BWD), ("dw1", B.K_MLP_DW1),
                                                         ("sync", B.K_SYNC))}
-            us = {nm: v[1] / max(v[0], 1) * 1e3 for nm, v in st.items()}
             _, n_calls, n_stored, _ = mlp_run_bytes(sched, d, wl.P, max_batch, overwrite_first)
+            us = {nm: v[1] / max(v[0], 1) * 1e3 for nm, v in st.items()}
+            us["fwd"] = st["fwd"][1] / n_calls * 1e3      # three timed kernels per call: cast, forward GEMM, bias / ReLU / logits
             dw1_bytes = ((4 * n_stored + 8 * (n_calls - n_stored)) * w1 + n_mb * 2 * d.mb * (d.d_in + d.d_hidden)) / n_calls
             res.update({"us_cast_fwd1_fwd2_per_call": us["fwd"], "us_bwd_per_call": us["bwd"], "us_dw1_per_call": us["dw1"],
                         "us_sync": us["sync"], "calls": n_calls, "calls_that_store": n_stored,
@@ -931,6 +934,8 @@ def main():
     ap.add_argument("--steps", type=int, default=1000)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--min-seconds", type=float, default=MIN_TIMED_SECONDS,
+                    help="the --steps-long timed region is repeated until this much time has been measured (0: once)")
     ap.add_argument("--sections", default="e2e,cpu,mlp,tiny,schedules,batch_curve,sync_curve,global",
                     help="extra measurements after the timed region (drop them for a profiler's launch list)")
     args = ap.parse_args()
