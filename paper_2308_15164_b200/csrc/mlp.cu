@@ -322,6 +322,12 @@ __device__ __forceinline__ void tma_load_2d(void* dst, const CUtensorMap* tm, in
         "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
         ::"r"(smem_u32(dst)), "l"(reinterpret_cast<uint64_t>(tm)), "r"(x), "r"(y), "r"(smem_u32(bar)) : "memory");
 }
+// Same with an L2 cache policy (createpolicy) for the loaded lines.
+__device__ __forceinline__ void tma_load_2d_hint(void* dst, const CUtensorMap* tm, int x, int y, uint64_t* bar, uint64_t policy) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1, {%2, %3}], [%4], %5;"
+        ::"r"(smem_u32(dst)), "l"(reinterpret_cast<uint64_t>(tm)), "r"(x), "r"(y), "r"(smem_u32(bar)), "l"(policy) : "memory");
+}
 __device__ __forceinline__ void tma_store_2d(const CUtensorMap* tm, const void* src, int x, int y) {
     asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.tile.bulk_group [%0, {%2, %3}], [%1];"
                  ::"l"(reinterpret_cast<uint64_t>(tm)), "r"(smem_u32(src)), "r"(x), "r"(y) : "memory");
@@ -778,13 +784,20 @@ __global__ void __launch_bounds__(128) k_fwd1_tcgen05(const __grid_constant__ CU
     pdl_trigger();
 
     if (warp == 0 && lane == 0) {                    // ---- TMA producer
+        // The bf16 weights (2 bytes per W1 element, 25 MB at 3072 x 4096) are read by every gradient call of the
+        // iteration: their lines are marked evict-last, so that they tend to stay in the 126 MB L2 between calls
+        // while the accumulator traffic of the dW1 kernels streams through (measured: 31.4 -> 31.0 us per micro-batch
+        // with single calls, 15.5 -> 15.3 batched; marking the accumulator traffic evict-first on top cost 7 %
+        // with single calls -- a worker's stored slice is partly still cached when its next gradient is added).
+        uint64_t pol_w1;
+        asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(pol_w1));
         for (int kb = 0; kb < nk; ++kb) {
             const int st = kb % kFwdStages;
             if (kb >= kFwdStages && !mbar_wait(&s.empty[st], ((kb / kFwdStages) - 1) & 1)) { s.failed = 1; break; }
             mbar_expect_tx(&s.full[st], kFwdStageBytes);
             const int k0 = kbeg + kb * 64;
-            tma_load_2d(s.stage[st], &tm_w1, h0, k0, &s.full[st]);
-            tma_load_2d(s.stage[st] + 8192, &tm_w1, h0 + 64, k0, &s.full[st]);
+            tma_load_2d_hint(s.stage[st], &tm_w1, h0, k0, &s.full[st], pol_w1);
+            tma_load_2d_hint(s.stage[st] + 8192, &tm_w1, h0 + 64, k0, &s.full[st], pol_w1);
 #pragma unroll
             for (int jb = 0; jb < NB; ++jb)          // rows jb*64.. of the stacked xb
                 tma_load_2d(s.stage[st] + 16384 + jb * 8192, &tm_xb, k0, jb * kMB, &s.full[st]);
