@@ -41,6 +41,8 @@ NVLINK_MEASURED_GBS = 770.0        # peer copy, per direction and GPU, measured 
 WORKLOAD = ("cfg2 resnet18-sized static heterogeneity: P=11689512 fp32 (62 tensors), W=4, b=(2,2,4,8), lr=0.1 mu=0.9 "
             "wd=5e-4; one step = one iteration = 16 accumulate + 1 fused sync step")
 MIN_TIMED_SECONDS = 1.0            # the --steps-long region is repeated until this much time has been measured
+DEFAULT_SECTIONS = "e2e,cpu,mlp,tiny,schedules,batch_curve,sync_curve,global"
+GLOBAL_STEP_DEADLINE_S = 180       # multi-GPU section: see run_ours
 
 
 def measured_peaks():
@@ -391,17 +393,45 @@ def run_ours(args):
     }
 
     sections = args.sections.split(",")
-    if world > 1 or "global_step" in sections:
-        # Step 1 across the GPUs of this job (every rank takes part; rank 0 reports)
-        try:
-            line["global_step"] = run_global_step(B, D, wlm, wl, dev, rank, world, rows, min(args.steps, 50), peaks)
-        except Exception as exc:                       # the replica figure above stands on its own
-            line["global_step"] = {"error": f"{type(exc).__name__}: {exc}"}
+    if world > 1 and args.sections == DEFAULT_SECTIONS:
+        sections = ["e2e", "cpu"]                      # the other GPUs of the job are held while rank 0 measures alone
     if rank == 0:
         if "e2e" in sections:
             line["e2e"] = run_e2e(B, wlm, wl, x0_d, pool, order, step_bytes, min(args.steps, 10))
         if "cpu" in sections:
             line["cpu_baseline"] = run_cpu_baseline(wlm, wl, x0, pool, order, step_bytes)
+    if world > 1 or "global_step" in sections:
+        # Step 1 across the GPUs of this job (every rank takes part; rank 0 reports).  Nothing here may cost the
+        # line above: an exception is reported inside the object, and if the section has not ended by its deadline
+        # (a rank that never arrived at a collective) every rank leaves -- rank 0 after printing the line without it.
+        # At that point no kernel of this section can be in flight: the fused kernels are launched behind the
+        # collective that every rank has to join.
+        finished = threading.Event()
+
+        def watchdog():
+            if finished.wait(GLOBAL_STEP_DEADLINE_S):
+                return
+            if rank == 0:
+                line["global_step"] = {"error": f"no result within {GLOBAL_STEP_DEADLINE_S} s; left out"}
+                print(json.dumps(line), flush=True)
+            os._exit(0)
+
+        threading.Thread(target=watchdog, daemon=True).start()
+        try:
+            if world == 1:                             # asked for on one GPU: a process group of one rank
+                import torch.distributed as tdist
+
+                if not tdist.is_initialized():
+                    os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+                    os.environ.setdefault("MASTER_PORT", "29512")
+                    os.environ.setdefault("NCCL_NVLS_ENABLE", "0")
+                    tdist.init_process_group(backend="nccl", rank=0, world_size=1, device_id=dev)
+            D.barrier(dev)
+            line["global_step"] = run_global_step(B, D, wlm, wl, dev, rank, world, rows, min(args.steps, 50), peaks)
+        except Exception as exc:                       # the replica figure above stands on its own
+            line["global_step"] = {"error": f"{type(exc).__name__}: {exc}"}
+        finished.set()
+    if rank == 0:
         del pool_d
         torch.cuda.empty_cache()
         if "mlp" in sections:
@@ -938,7 +968,7 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--min-seconds", type=float, default=MIN_TIMED_SECONDS,
                     help="the --steps-long timed region is repeated until this much time has been measured (0: once)")
-    ap.add_argument("--sections", default="e2e,cpu,mlp,tiny,schedules,batch_curve,sync_curve,global",
+    ap.add_argument("--sections", default=DEFAULT_SECTIONS,
                     help="extra measurements after the timed region (drop them for a profiler's launch list)")
     args = ap.parse_args()
     if args.warmup < 3:
