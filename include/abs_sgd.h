@@ -168,10 +168,11 @@ int abs_accumulate_host(abs_ctx *ctx, uint32_t worker, const void *grad_host);
  * int32 class indices in [0, mlp_out).  GEMM operands are rounded to bf16 (nearest even) with fp32 accumulation;
  * dW1 = X^T dZ runs on the tcgen05 tensor cores and its epilogue adds into the accumulator.
  * Needs ABS_FLAG_MLP.  x_dev and y_dev are read by the first kernel only, which is enqueued on stream_acc
- * (they may be reused by later work on that stream).  The remaining kernels run on an internal stream of
- * the worker (workers compute concurrently, as in the paper; calls of one worker stay in call order), which
- * starts after everything enqueued on stream_acc so far; abs_sync_step, abs_wait, abs_check, abs_accumulate,
- * abs_accumulate_host and abs_accumulator make stream_acc wait for all of them. */
+ * (they may be reused by later work on that stream).  The remaining kernels run on internal streams of
+ * the worker (workers compute concurrently, as in the paper; what a worker's calls add to its row is added in call
+ * order; the dW1 GEMM of a single call runs on a second stream of the worker, so that the worker's next call can
+ * start beside it), which start after everything enqueued on stream_acc so far; abs_sync_step, abs_wait, abs_check,
+ * abs_accumulate, abs_accumulate_host and abs_accumulator make stream_acc wait for all of them. */
 int abs_accumulate_mlp(abs_ctx *ctx, uint32_t worker, const void *x_dev, const int32_t *y_dev);
 
 /* n (1..4) consecutive reference batches of one worker in one call: the same computation as n calls of
