@@ -124,7 +124,10 @@ typedef struct abs_config {
                                  micro-batch.  Flat layout: W1 [in,hidden] row-major, b1 [hidden],
                                  W2 [hidden,out] row-major, b2 [out]; P must equal their total.
                                  Limits: in % 128 == 0, hidden % 128 == 0, out <= 16, mb == 64.      */
-    void *stream_acc;         /* cudaStream_t for Step 2 work (accumulation); NULL = default stream   */
+    void *stream_acc;         /* cudaStream_t for Step 2 work (accumulation); NULL = default stream.  With
+                                 ABS_FLAG_MLP a high-priority stream is worth having: the first kernel of
+                                 every gradient call runs there and should not queue behind earlier calls'
+                                 dW1 GEMMs (which the library runs at the lowest priority)              */
     void *stream_sync;        /* cudaStream_t for Step 1 work when ABS_FLAG_PIPELINED; must then
                                  differ from stream_acc                                               */
 } abs_config;
@@ -170,8 +173,8 @@ int abs_accumulate_host(abs_ctx *ctx, uint32_t worker, const void *grad_host);
  * Needs ABS_FLAG_MLP.  x_dev and y_dev are read by the first kernel only, which is enqueued on stream_acc
  * (they may be reused by later work on that stream).  The remaining kernels run on internal streams of
  * the worker (workers compute concurrently, as in the paper; what a worker's calls add to its row is added in call
- * order; the dW1 GEMM of a single call runs on a second stream of the worker, so that the worker's next call can
- * start beside it), which start after everything enqueued on stream_acc so far; abs_sync_step, abs_wait, abs_check,
+ * order; the dW1 GEMM of a call runs on a second, lowest-priority stream of the worker, so that the worker's next
+ * call can start beside it), which start after everything enqueued on stream_acc so far; abs_sync_step, abs_wait, abs_check,
  * abs_accumulate, abs_accumulate_host and abs_accumulator make stream_acc wait for all of them. */
 int abs_accumulate_mlp(abs_ctx *ctx, uint32_t worker, const void *x_dev, const int32_t *y_dev);
 

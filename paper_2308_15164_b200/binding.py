@@ -145,7 +145,10 @@ class AbsSgd:
         assert params0.is_cuda and params0.dtype == torch.float32 and params0.is_contiguous()
         self.device = params0.device
         self.P, self.W = params0.numel(), W
-        self.stream_acc = stream_acc or torch.cuda.Stream(device=self.device)
+        # An MLP context's own stream_acc is a high-priority stream: the operand cast of a gradient call runs there and
+        # would otherwise queue behind the thousands of CTAs of earlier calls' dW1 GEMMs.  (Streaming contexts keep
+        # the default priority: their accumulate kernels must not starve the fused step on stream_sync.)
+        self.stream_acc = stream_acc or torch.cuda.Stream(device=self.device, priority=-1 if mlp else 0)
         self.stream_sync = stream_sync or (torch.cuda.Stream(device=self.device) if pipelined else None)
         flags = (FLAG_PIPELINED if pipelined else 0) | (FLAG_MLP if mlp else 0) | (FLAG_HOST_INPUT if host_input else 0) | (FLAG_OVERWRITE_FIRST if overwrite_first else 0) | (FLAG_MLP_COALESCE if mlp_coalesce else 0) | (FLAG_GRAD_NORM if grad_norm else 0) | (FLAG_MLP_X_BF16 if mlp_x_bf16 else 0)
         self.cfg = make_config(self.P, W, lr, momentum, weight_decay, lambda_dc, grad_dtype, flags, mlp,

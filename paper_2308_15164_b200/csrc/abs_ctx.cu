@@ -160,12 +160,14 @@ struct abs_ctx {
     // in its own scratch set, taken round-robin.
     MlpScratch mlp_scratch[kMlpSets]{};
     cudaStream_t s_w[kMlpStreams] = {};
-    // The dW1 GEMM of a call runs on a second stream of the worker, one priority level below: the worker's next
-    // call (forward, loss, backward: short, latency-bound kernels that only touch the bias / W2 slices of the row)
-    // overlaps it, and the short kernels of every worker get free CTA slots before the HBM-bound GEMMs.
+    // The dW1 GEMM of a call runs on a second stream of the worker, at the lowest priority: the worker's next call
+    // (forward, loss, backward: short, latency-bound kernels that only touch the bias / W2 slices of the row)
+    // overlaps it, and the short kernels of every worker get free CTA slots before the HBM-bound GEMMs, whose
+    // thousands of CTAs would otherwise keep them queueing (timeline with four workers' calls in flight: a 3 us
+    // cast kernel took 23 us on average, `k_fwd2` 23 against 5).  Measured on 3072-4096-10, W = 4: single calls
+    // 31.1 -> 30.0 us per micro-batch, batch calls 15.4 -> 14.6.
     cudaStream_t s_d[kMlpStreams] = {};
     cudaEvent_t ev_front[kMlpStreams] = {};        // front kernels of the newest call on s_w[k] have finished
-    bool gemm_on_d[kMlpStreams] = {};              // where the newest dW1 of worker stream k was enqueued
     int n_wstreams = 0;
     cudaEvent_t ev_fork = nullptr;                 // stream_acc -> worker stream (re-recorded per call)
     cudaEvent_t ev_set_done[kMlpSets] = {};        // last use of a scratch set has finished
@@ -391,17 +393,11 @@ int run_mlp_group(abs_ctx* c, uint32_t worker, int set, int n, bool first, bool 
     CK(launch_mlp_front(c->mlp_dims, sc, c->x(c->pub), c->shadow(c->pub), c->pub, n, first, c->acc(c->cur, worker),
                         c->cnt(c->cur, worker), variant, s_run, c->mlp_chain(serial, n), mlp_mark, c));
     cudaStream_t s_gemm = s_run;
-    // Single calls: dW1 on the worker's second stream (measured on 3072-4096-10, W = 4: 32.2 -> 31.3 us per
-    // micro-batch); K-batched calls keep it behind their front kernels (15.6 against 16.0 us).
-    const bool split = !serial && n == 1;
-    if (split) s_gemm = c->s_d[k];
-    if (!serial && c->w_outstanding[k] && c->gemm_on_d[k] != split)   // the worker's previous dW1 ran on the other stream
-        CK(cudaStreamWaitEvent(s_gemm, c->ev_w_done[k], 0));
-    if (split) {
+    if (!serial) {   // dW1 on the worker's second (lowest-priority) stream, behind the front kernels of this call
+        s_gemm = c->s_d[k];
         CK(cudaEventRecord(c->ev_front[k], s_run));
         CK(cudaStreamWaitEvent(s_gemm, c->ev_front[k], 0));
     }
-    if (!serial) c->gemm_on_d[k] = split;
     // On its own stream the kernel ahead of this dW1 is the worker's previous dW1, which writes the same slice:
     // never chained there (the register-prefetch kernel reads the slice in front of its wait).
     CK(launch_mlp_dw1(c->mlp_dims, sc, c->acc(c->cur, worker), &c->acc_tmaps[(size_t)c->cur * c->cfg.W + worker], n,
@@ -558,8 +554,7 @@ int abs_init(abs_ctx** out, const abs_config* cfg, void* workspace_dev, size_t w
         if ((e = cudaDeviceGetStreamPriorityRange(&prio_lo, &prio_hi)) != cudaSuccess) return bail(e, "cudaDeviceGetStreamPriorityRange");
         for (int k = 0; k < c->n_wstreams; ++k) {
             if ((e = cudaStreamCreateWithPriority(&c->s_w[k], cudaStreamNonBlocking, prio_hi)) != cudaSuccess) return bail(e, "cudaStreamCreate");
-            const int prio_gemm = prio_hi < prio_lo ? prio_hi + 1 : prio_hi;   // (numerically lower = higher priority)
-            if ((e = cudaStreamCreateWithPriority(&c->s_d[k], cudaStreamNonBlocking, prio_gemm)) != cudaSuccess) return bail(e, "cudaStreamCreate");
+            if ((e = cudaStreamCreateWithPriority(&c->s_d[k], cudaStreamNonBlocking, prio_lo)) != cudaSuccess) return bail(e, "cudaStreamCreate");
             if ((e = cudaEventCreateWithFlags(&c->ev_w_done[k], cudaEventDisableTiming)) != cudaSuccess) return bail(e, "cudaEventCreate");
             if ((e = cudaEventCreateWithFlags(&c->ev_front[k], cudaEventDisableTiming)) != cudaSuccess) return bail(e, "cudaEventCreate");
         }

@@ -4,6 +4,8 @@
     python -m paper_2308_15164_b200.profile_case accumulate [--P 11689512] [--W 4] [--iters 3] [--bf16]
     python -m paper_2308_15164_b200.profile_case mlp        [--iters 2] [--batch 4] [--calls 2]
     python -m paper_2308_15164_b200.profile_case global     [--P 25557032] [--ranks 4] [--W 2] [--iters 2]
+    python -m paper_2308_15164_b200.profile_case timeline   [--iters 3] [--batch 4]     (no profiler: prints the library's
+                                                            own timeline of the MLP workload's kernels)
 
 Each case keeps its working set larger than the 126 MB L2 but to a few hundred MB, launches the
 kernel of interest a handful of times and exits, so that a multi-pass capture ends by itself.
@@ -21,7 +23,7 @@ import torch
 
 def main(argv=None):
     ap = argparse.ArgumentParser()
-    ap.add_argument("case", choices=["sync", "accumulate", "mlp", "global"])
+    ap.add_argument("case", choices=["sync", "accumulate", "mlp", "global", "timeline"])
     ap.add_argument("--P", type=int, default=11_689_512)
     ap.add_argument("--W", type=int, default=4)
     ap.add_argument("--iters", type=int, default=3)
@@ -38,6 +40,8 @@ def main(argv=None):
 
     dev = torch.device("cuda:0")
     torch.cuda.set_device(dev)
+    if args.case == "timeline":
+        return timeline(args, B, wlm, dev)
     if args.case == "global":
         from . import dist as D
 
@@ -91,6 +95,61 @@ def main(argv=None):
         eng.check()
         eng.destroy()
     print("done", args.case)
+    return 0
+
+
+def timeline(args, B, wlm, dev):
+    """Workload 4 (3072-4096-10, W = 4, b_i ~ U{1..8}), pipelined, with every worker's calls on its own streams:
+    six warm-up iterations, then `--iters` iterations with abs_profile(ctx, 2); prints every timed kernel's span
+    (start, stop, stream) and, per kernel, the mean duration while the workers' calls overlap."""
+    wl = wlm.config(4, T=6 + args.iters)
+    d = wl.mlp
+    x0 = torch.from_numpy(wlm.params0(wl)).to(dev)
+    xs, ys = wlm.mlp_batches(wl)
+    xs_d, ys_d = torch.from_numpy(xs).to(dev), torch.from_numpy(ys).to(dev)
+    sched = wlm.schedule(wl)
+    eng = B.AbsSgd(x0, wl.W, wl.lr, wl.momentum, pipelined=True, mlp=(d.d_in, d.d_hidden, d.d_out, d.mb))
+    torch.cuda.synchronize()
+    n = 0
+
+    def run(rows):
+        nonlocal n
+        with torch.cuda.stream(eng.stream_acc):
+            for b_row in rows:
+                if args.batch > 1:
+                    for i, b in enumerate(b_row):
+                        left = int(b)
+                        while left > 0:
+                            k = min(args.batch, left)
+                            lo = (n * 7) % (wl.mlp_pool - args.batch)
+                            eng.accumulate_mlp_batch(i, k, xs_d[lo:lo + k], ys_d[lo:lo + k]); left -= k; n += k
+                else:
+                    for (i, k) in wlm.call_order(b_row):
+                        eng.accumulate_mlp(i, xs_d[n % wl.mlp_pool], ys_d[n % wl.mlp_pool]); n += 1
+                eng.sync_step()
+            eng.wait()
+        torch.cuda.synchronize()
+
+    run(sched[:6])
+    eng.profile(2)
+    run(sched[6:])
+    spans = eng.profile_timeline()
+    eng.profile(False)
+    names = {("mlp_fwd", 0): "cast", ("mlp_fwd", 1): "forward GEMM", ("mlp_fwd", 2): "bias/ReLU/logits", ("mlp_bwd", 0): "backward",
+             ("mlp_dw1", 0): "dW1", ("sync", 0): "fused step"}
+    print(f"b of the timed iterations: {sched[6:].tolist()}; calls of up to {args.batch} micro-batches")
+    stat = {}
+    for (cls, part, stream, t0, t1) in sorted(spans, key=lambda r: r[3]):
+        nm = names.get((cls, part), cls)
+        print(f"  {t0:9.1f} .. {t1:9.1f} us  ({t1 - t0:6.1f})  stream {stream:2d}  {nm}")
+        stat.setdefault(nm, []).append(t1 - t0)
+    last = max(t1 for (_, _, _, _, t1) in spans)
+    print(f"{len(spans)} spans over {last:.1f} us")
+    for nm, v in stat.items():
+        print(f"  {nm:18s} n = {len(v):3d}  mean {np.mean(v):6.1f} us  min {np.min(v):6.1f}  max {np.max(v):6.1f}")
+    eng.check()
+    eng.destroy()
+    print("done timeline")
     return 0
 
 

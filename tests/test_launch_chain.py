@@ -150,7 +150,7 @@ def test_timeline_of_the_timed_launches():
     assert set(by[("mlp_fwd", 0)]) == {0}                       # the cast reads the caller's buffers: stream_acc
     assert set(by[("sync", 0)]) == {1}                          # Step 1 on stream_sync
     assert set(by[("mlp_fwd", 1)]) <= {2, 3, 4, 5}              # the workers' own streams
-    assert set(by[("mlp_dw1", 0)]) <= {10, 11, 12, 13}          # dW1 of single calls: the workers' second streams
+    assert set(by[("mlp_dw1", 0)]) <= {10, 11, 12, 13}          # dW1: the workers' second streams
     n_st, ms = eng.kernel_stats(B.K_MLP_DW1)
     assert n_st == n and ms > 0
     eng.check()
