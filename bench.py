@@ -748,13 +748,15 @@ def run_tiny(B, wlm, dev, iters=2000):
     return out
 
 
-def mlp_run_bytes(sched, d, P, max_batch, overwrite_first):
+def mlp_run_bytes(sched, d, P, max_batch, overwrite_first, defer=False):
     """Algorithmic HBM bytes of an MLP run over the schedule `sched` [T, W] when every worker hands over its b_i
     micro-batches in calls of up to `max_batch`: per call the bf16 weights are streamed once (2 bytes per W1
     element) and the W1 slice of the accumulator is written (4 bytes per element: the worker's first call of the
     iteration stores) or read and written (8: later calls add); per micro-batch the bf16 operands of dW1; per
     iteration the fused step, (8 W_act + 16 + 2) bytes per parameter (the 2: the bf16 copy of the new weights;
-    4 W_act + 18 when the step does not write zeros).  Returns (bytes, calls, stored calls, micro-batches)."""
+    4 W_act + 18 when the step does not write zeros).  defer (ABS_FLAG_MLP_DEFER): the slice is written once per active
+    worker and iteration (4 bytes per element), never read by a gradient call, and the operands are written by the
+    call and read by that one contraction.  Returns (bytes, calls, stored calls, micro-batches)."""
     w1 = d.d_in * d.d_hidden
     total = calls = stored = mbs = 0
     prev_active = 0
@@ -765,7 +767,10 @@ def mlp_run_bytes(sched, d, P, max_batch, overwrite_first):
             left, first = int(b), True
             while left > 0:
                 n = min(max_batch, left)
-                total += 2 * w1 + (4 if first else 8) * w1 + n * 2 * d.mb * (d.d_in + d.d_hidden)
+                if defer:
+                    total += 2 * w1 + (4 * w1 if first else 0) + 2 * n * 2 * d.mb * (d.d_in + d.d_hidden)
+                else:
+                    total += 2 * w1 + (4 if first else 8) * w1 + n * 2 * d.mb * (d.d_in + d.d_hidden)
                 calls += 1; stored += 1 if first else 0; mbs += n
                 left -= n; first = False
         prev_active = int(sum(1 for b in b_row if b > 0))
@@ -797,9 +802,9 @@ def run_mlp(B, wlm, dev, peaks, iters=12):
     out = {"workload": "cfg4 mlp 3072-4096-10, mb=64, W=4, b_i~U{1..8}, pipelined", "iterations": iters,
            "dw1_flop_per_microbatch": flop}
 
-    def run_case(max_batch, variant=0, coalesce=False, overwrite_first=False, serial=0):
+    def run_case(max_batch, variant=0, coalesce=False, overwrite_first=False, serial=0, defer=False):
         eng = B.AbsSgd(x0_d, wl.W, wl.lr, wl.momentum, wl.weight_decay, pipelined=True, mlp=(d.d_in, d.d_hidden, d.d_out, d.mb),
-                       mlp_coalesce=coalesce, overwrite_first=overwrite_first)
+                       mlp_coalesce=coalesce, overwrite_first=overwrite_first, mlp_defer=defer)
         eng.set_launch(B.K_MLP_DW1, variant)
         eng.set_launch(B.K_MLP_FWD, serial)
 
@@ -847,7 +852,7 @@ def run_mlp(B, wlm, dev, peaks, iters=12):
                         "dw1_bytes_per_call": dw1_bytes, "dw1_hbm_gbs": dw1_bytes / us["dw1"] / 1e3,
                         "dw1_frac_of_hbm": dw1_bytes / us["dw1"] / 1e3 / peaks["hbm_gbs"]})
         else:
-            nbytes, n_calls, n_stored, _ = mlp_run_bytes(sched, d, wl.P, 4 if coalesce else max_batch, overwrite_first)
+            nbytes, n_calls, n_stored, _ = mlp_run_bytes(sched, d, wl.P, 4 if coalesce else max_batch, overwrite_first, defer)
             floor_us = nbytes / peaks["hbm_gbs"] / 1e3 / n_mb
             res.update({"algorithmic_bytes_per_microbatch": nbytes / n_mb, "hbm_floor_us_per_microbatch": floor_us,
                         "frac_of_hbm_floor": floor_us / res["us_per_microbatch"]})
@@ -859,7 +864,12 @@ def run_mlp(B, wlm, dev, peaks, iters=12):
                      ("single_calls_gathered_by_the_library", dict(max_batch=1, coalesce=True)),
                      ("batch_calls_up_to_4", dict(max_batch=4)),
                      ("batch_calls_up_to_4_overwrite_first", dict(max_batch=4, overwrite_first=True)),
-                     ("batch_calls_up_to_4_deep_pipelines", dict(max_batch=4, variant=128))):
+                     ("batch_calls_up_to_4_deep_pipelines", dict(max_batch=4, variant=128)),
+                     # ABS_FLAG_MLP_DEFER: one dW1 contraction per worker and iteration (K = 64 b_i)
+                     ("deferred_single_calls", dict(max_batch=1, defer=True)),
+                     ("deferred_single_calls_gathered_by_the_library", dict(max_batch=1, coalesce=True, defer=True)),
+                     ("deferred_batch_calls_up_to_4", dict(max_batch=4, defer=True)),
+                     ("deferred_batch_calls_up_to_4_overwrite_first", dict(max_batch=4, defer=True, overwrite_first=True))):
         out[name] = run_case(**kw)
     for name, kw in (("single_calls", dict(max_batch=1)), ("single_calls_ring_dw1", dict(max_batch=1, variant=4)),
                      ("batch_calls_up_to_4", dict(max_batch=4)), ("batch_calls_up_to_4_tile_per_cta_dw1", dict(max_batch=4, variant=8))):

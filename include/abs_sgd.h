@@ -96,6 +96,23 @@ extern "C" {
 #define ABS_FLAG_MLP_X_BF16 64u   /* with ABS_FLAG_MLP: abs_accumulate_mlp* take x_dev as bf16 values ([mlp_mb, mlp_in] row-major,
                                      2 bytes each) instead of fp32; they enter the GEMMs as they are (no rounding step) */
 
+#define ABS_FLAG_MLP_DEFER 128u   /* with ABS_FLAG_MLP: the layer-1 weight gradient is formed once per worker and iteration
+                                     instead of once per call.  Within an iteration every gradient is evaluated at the
+                                     same x_t (Algorithm 1, Step 2), so the worker's sum of micro-batch gradients
+                                     sum_j X_j^T dZ_j is ONE contraction over its stacked micro-batches (K = 64 b_i).  A
+                                     gradient call then runs forward, loss and layer-2 backward as usual (bias and W2
+                                     slices of the row, b_i) and only leaves its dW1 operands -- bf16(X)^T and bf16(dZ)^T,
+                                     (mlp_in + mlp_hidden) * 128 bytes -- in the accumulator set's operand pool; the
+                                     W1 slice of the row is written when the iteration ends (abs_sync_step /
+                                     abs_global_begin), or earlier when something reads or adds to the row
+                                     (abs_accumulator, abs_accumulate*, abs_wait, abs_check, abs_state_export,
+                                     abs_set_launch) or the pool (max(32, 16 W) micro-batches, at most 128) is full.
+                                     The row then holds the same sum as without the flag to fp32 rounding (one fp32
+                                     accumulation over K = 64 b_i instead of b_i rounded additions).  Per micro-batch
+                                     the accumulator traffic of 8 mlp_in mlp_hidden bytes (read + write of the slice)
+                                     becomes 4 mlp_in mlp_hidden / b_i (one write per worker and iteration).  Combines
+                                     with every other flag.                                                       */
+
 #define ABS_MAX_WORKERS 64u
 #define ABS_MAX_RANKS   16u   /* GPUs taking part in abs_global_* (n_ranks * W <= ABS_MAX_WORKERS)        */
 #define ABS_IPC_HANDLE_BYTES 64

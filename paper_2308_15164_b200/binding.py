@@ -26,7 +26,7 @@ lib = ctypes.CDLL(LIB_PATH)
 
 OK, EINVAL, ESTATE, ECUDA, ENOMEM, ETIMEOUT, ELIMIT = 0, -1, -2, -3, -4, -5, -6
 GRAD_F32, GRAD_BF16 = 0, 1
-FLAG_PIPELINED, FLAG_MLP, FLAG_HOST_INPUT, FLAG_OVERWRITE_FIRST, FLAG_MLP_COALESCE, FLAG_GRAD_NORM, FLAG_MLP_X_BF16 = 1, 2, 4, 8, 16, 32, 64
+FLAG_PIPELINED, FLAG_MLP, FLAG_HOST_INPUT, FLAG_OVERWRITE_FIRST, FLAG_MLP_COALESCE, FLAG_GRAD_NORM, FLAG_MLP_X_BF16, FLAG_MLP_DEFER = 1, 2, 4, 8, 16, 32, 64, 128
 K_ACCUMULATE, K_SYNC, K_MLP_FWD, K_MLP_BWD, K_MLP_DW1, K_CHAIN = range(6)
 MAX_WORKERS, MAX_RANKS, IPC_HANDLE_BYTES = 64, 16, 64
 KERNEL_NAMES = ["accumulate", "sync", "mlp_fwd", "mlp_bwd", "mlp_dw1"]
@@ -140,7 +140,7 @@ class AbsSgd:
 
     def __init__(self, params0: torch.Tensor, W: int, lr: float, momentum=0.0, weight_decay=0.0, lambda_dc=0.0,
                  grad_dtype=GRAD_F32, pipelined=False, mlp=None, host_input=False, overwrite_first=False,
-                 mlp_coalesce=False, grad_norm=False, mlp_x_bf16=False, stream_acc: Optional[torch.cuda.Stream] = None, stream_sync: Optional[torch.cuda.Stream] = None,
+                 mlp_coalesce=False, grad_norm=False, mlp_x_bf16=False, mlp_defer=False, stream_acc: Optional[torch.cuda.Stream] = None, stream_sync: Optional[torch.cuda.Stream] = None,
                  workspace: Optional[torch.Tensor] = None):
         assert params0.is_cuda and params0.dtype == torch.float32 and params0.is_contiguous()
         self.device = params0.device
@@ -150,7 +150,7 @@ class AbsSgd:
         # the default priority: their accumulate kernels must not starve the fused step on stream_sync.)
         self.stream_acc = stream_acc or torch.cuda.Stream(device=self.device, priority=-1 if mlp else 0)
         self.stream_sync = stream_sync or (torch.cuda.Stream(device=self.device) if pipelined else None)
-        flags = (FLAG_PIPELINED if pipelined else 0) | (FLAG_MLP if mlp else 0) | (FLAG_HOST_INPUT if host_input else 0) | (FLAG_OVERWRITE_FIRST if overwrite_first else 0) | (FLAG_MLP_COALESCE if mlp_coalesce else 0) | (FLAG_GRAD_NORM if grad_norm else 0) | (FLAG_MLP_X_BF16 if mlp_x_bf16 else 0)
+        flags = (FLAG_PIPELINED if pipelined else 0) | (FLAG_MLP if mlp else 0) | (FLAG_HOST_INPUT if host_input else 0) | (FLAG_OVERWRITE_FIRST if overwrite_first else 0) | (FLAG_MLP_COALESCE if mlp_coalesce else 0) | (FLAG_GRAD_NORM if grad_norm else 0) | (FLAG_MLP_X_BF16 if mlp_x_bf16 else 0) | (FLAG_MLP_DEFER if mlp_defer else 0)
         self.cfg = make_config(self.P, W, lr, momentum, weight_decay, lambda_dc, grad_dtype, flags, mlp,
                                self.stream_acc.cuda_stream, self.stream_sync.cuda_stream if self.stream_sync else 0)
         nbytes = abs_workspace_bytes(self.cfg)

@@ -33,6 +33,8 @@ struct Layout {
     size_t P_pad = 0;
     size_t off_x[2] = {0, 0}, off_v = 0, off_acc = 0, off_cnt = 0, off_ticket = 0, off_log = 0, off_gcnt = 0;
     size_t off_shadow[2] = {0, 0}, off_mlp = 0, off_stage[2] = {0, 0}, off_norm_part = 0, off_norm_log = 0;
+    size_t off_pool[2] = {0, 0};
+    int pool_cap = 0;
     size_t norm_slots = 0;
     size_t total = 0;
 };
@@ -44,8 +46,9 @@ bool config_ok(const abs_config* c, std::string* why) {
     if (c->W == 0 || c->W > ABS_MAX_WORKERS) return fail("W must be in 1..64");
     if (c->grad_dtype != ABS_GRAD_F32 && c->grad_dtype != ABS_GRAD_BF16) return fail("unknown grad_dtype");
     if (c->flags & ~(ABS_FLAG_PIPELINED | ABS_FLAG_MLP | ABS_FLAG_HOST_INPUT | ABS_FLAG_OVERWRITE_FIRST | ABS_FLAG_MLP_COALESCE |
-                     ABS_FLAG_GRAD_NORM | ABS_FLAG_MLP_X_BF16))
+                     ABS_FLAG_GRAD_NORM | ABS_FLAG_MLP_X_BF16 | ABS_FLAG_MLP_DEFER))
         return fail("unknown flag bits");
+    if ((c->flags & ABS_FLAG_MLP_DEFER) && !(c->flags & ABS_FLAG_MLP)) return fail("ABS_FLAG_MLP_DEFER needs ABS_FLAG_MLP");
     if ((c->flags & ABS_FLAG_MLP_COALESCE) && !(c->flags & ABS_FLAG_MLP)) return fail("ABS_FLAG_MLP_COALESCE needs ABS_FLAG_MLP");
     if ((c->flags & ABS_FLAG_MLP_X_BF16) && !(c->flags & ABS_FLAG_MLP)) return fail("ABS_FLAG_MLP_X_BF16 needs ABS_FLAG_MLP");
     if (!std::isfinite(c->lr) || !std::isfinite(c->momentum) || !std::isfinite(c->weight_decay) ||
@@ -84,6 +87,12 @@ Layout make_layout(const abs_config& c) {
         L.off_shadow[1] = pipe ? take(L.P_pad * 2) : L.off_shadow[0];
         MlpDims d{(int)c.mlp_in, (int)c.mlp_hidden, (int)c.mlp_out, (int)c.mlp_mb};
         L.off_mlp = take((size_t)kMlpSets * mlp_scratch_bytes(d));
+        if (c.flags & ABS_FLAG_MLP_DEFER) {
+            // room for 16 micro-batches per worker and iteration before the operands are contracted early
+            L.pool_cap = (int)std::min<uint32_t>(std::max<uint32_t>(16 * c.W, 32), kMlpMaxSlots);
+            L.off_pool[0] = take(mlp_pool_bytes(d, L.pool_cap));
+            L.off_pool[1] = take(mlp_pool_bytes(d, L.pool_cap));
+        }
     }
     if (c.flags & ABS_FLAG_HOST_INPUT) {
         const size_t es = c.grad_dtype == ABS_GRAD_BF16 ? 2 : 4;
@@ -186,6 +195,15 @@ struct abs_ctx {
     uint64_t pend_age[kMaxW] = {}; // order in which the pending groups were opened
     uint64_t pend_clock = 0;
     std::vector<TmapBytes> acc_tmaps;   // [2][W]: TMA descriptor of each accumulator row's W1 slice
+    // ABS_FLAG_MLP_DEFER: the dW1 operands of every gradient call of an iteration stay in the accumulator set's
+    // operand pool; a worker's dW1 = sum_j X_j^T dZ_j is contracted in ONE launch (K = 64 b_i) when the iteration
+    // ends, when something reads or adds to its accumulator row, or when the pool is full.
+    bool defer = false;
+    MlpPool pool[2]{};
+    int pool_n[2] = {0, 0};                   // slots handed out (bump allocation; back to 0 when the iteration ends)
+    std::vector<int16_t> pool_owner[2];       // worker whose micro-batch sits in the slot; -1: none (contracted, or never used)
+    int pend_pool0[kMaxW] = {};               // first pool slot of a waiting group (ABS_FLAG_MLP_COALESCE)
+    bool w1_touched[2][kMaxW] = {};           // the row's W1 slice has been written in the set's current iteration
 
     // multi-GPU mode (abs_global_*): every rank's workspace as mapped in this process
     uint32_t n_ranks = 0, rank = 0;
@@ -310,11 +328,12 @@ void mlp_mark(void* user, int kernel_class, int n, cudaStream_t stream);
 
 int flush_all(abs_ctx* c);
 int flush_worker(abs_ctx* c, uint32_t worker);
+int settle_all(abs_ctx* c);
 
 // stream_acc waits (on the device) for every gradient kernel enqueued so far on the worker streams (waiting
-// micro-batch groups are started first).
+// micro-batch groups are started and pooled dW1 operands contracted first).
 int join_workers(abs_ctx* c) {
-    if (int rc = flush_all(c)) return rc;
+    if (int rc = settle_all(c)) return rc;
     for (int k = 0; k < c->n_wstreams; ++k)
         if (c->w_outstanding[k]) {
             CK(cudaStreamWaitEvent(c->s_acc, c->ev_w_done[k], 0));
@@ -352,9 +371,15 @@ int launch_fused(abs_ctx* c, uint32_t set, int in, int out, uint64_t log_step, c
     }
     // Beside the MLP's gradient kernels (pipelined mode) the bulk-copy form is the better neighbour: it holds six
     // warps per SM instead of every thread slot.  Measured on the 3072-4096-10 workload with batch calls: 16.9
-    // against 17.5 us per micro-batch, although alone on the GPU it is the slower one at W = 4.
+    // against 17.5 us per micro-batch, although alone on the GPU it is the slower one at W = 4.  There it runs
+    // as one CTA per SM with four stages (110 KB at W = 4) instead of two CTAs with three (168 KB), so that a
+    // forward-GEMM or dW1 CTA still fits on the SM (single calls 32.4 -> 32.0 us, batch calls 15.8 -> 15.4; with
+    // ABS_FLAG_MLP_DEFER 17.1 -> 16.6 and 14.9 -> 14.2 for gathered calls).
     int shape = c->ctas_per_sm[ABS_K_SYNC];
-    if (shape == 0 && c->mlp && c->pipelined) shape = -2;
+    if (shape == 0 && c->mlp && c->pipelined) {
+        shape = -2;
+        a.tma_one_cta = 4;
+    }
     {
         Timed tm(c, ABS_K_SYNC, stream);
         CK(launch_sync(a, shape, c->num_sms, stream, c->chained()));
@@ -376,7 +401,7 @@ int take_scratch_set(abs_ctx* c, bool serial, int* out) {
 // Forward, loss, backward and dW1 of the n micro-batches that sit, cast, in slots 0..n-1 of scratch set `set`,
 // on the worker's internal stream (which first waits for everything enqueued on stream_acc so far, the casts
 // included).  deferred: the casts were launched, and counted, by earlier calls.
-int run_mlp_group(abs_ctx* c, uint32_t worker, int set, int n, bool first, bool deferred) {
+int run_mlp_group(abs_ctx* c, uint32_t worker, int set, int n, bool first, int pool0) {
     const int k = (int)(worker % (uint32_t)c->n_wstreams);
     int variant = c->ctas_per_sm[ABS_K_MLP_DW1];
     const bool serial = c->ctas_per_sm[ABS_K_MLP_FWD] == 1;
@@ -389,9 +414,22 @@ int run_mlp_group(abs_ctx* c, uint32_t worker, int set, int n, bool first, bool 
         CK(cudaEventRecord(c->ev_fork, c->s_acc));
         CK(cudaStreamWaitEvent(s_run, c->ev_fork, 0));
     }
-    (void)deferred;
+    __nv_bfloat16* dzt_out = nullptr;
+    if (c->defer) dzt_out = c->pool[c->cur].dzt + (size_t)pool0 * c->mlp_dims.d_hidden * c->mlp_dims.mb;
     CK(launch_mlp_front(c->mlp_dims, sc, c->x(c->pub), c->shadow(c->pub), c->pub, n, first, c->acc(c->cur, worker),
-                        c->cnt(c->cur, worker), variant, s_run, c->mlp_chain(serial, n), mlp_mark, c));
+                        c->cnt(c->cur, worker), dzt_out, variant, s_run, c->mlp_chain(serial, n), mlp_mark, c));
+    if (c->defer) {   // the call ends here: its dW1 operands stay in the pool
+        for (int j = 0; j < n; ++j) c->pool_owner[c->cur][pool0 + j] = (int16_t)worker;
+        if (serial) {
+            for (bool& u : c->set_used) u = false;
+        } else {
+            CK(cudaEventRecord(c->ev_set_done[set], s_run));
+            CK(cudaEventRecord(c->ev_w_done[k], s_run));
+            c->set_used[set] = true;
+            c->w_outstanding[k] = true;
+        }
+        return ABS_OK;
+    }
     cudaStream_t s_gemm = s_run;
     if (!serial) {   // dW1 on the worker's second (lowest-priority) stream, behind the front kernels of this call
         s_gemm = c->s_d[k];
@@ -400,8 +438,10 @@ int run_mlp_group(abs_ctx* c, uint32_t worker, int set, int n, bool first, bool 
     }
     // On its own stream the kernel ahead of this dW1 is the worker's previous dW1, which writes the same slice:
     // never chained there (the register-prefetch kernel reads the slice in front of its wait).
-    CK(launch_mlp_dw1(c->mlp_dims, sc, c->acc(c->cur, worker), &c->acc_tmaps[(size_t)c->cur * c->cfg.W + worker], n,
-                      first, variant, s_gemm, serial && (c->mlp_chain(serial, n) & kChainDw1) != 0, mlp_mark, c));
+    CK(launch_mlp_dw1(c->mlp_dims, sc, nullptr, nullptr, c->acc(c->cur, worker),
+                      &c->acc_tmaps[(size_t)c->cur * c->cfg.W + worker], n, first, variant, s_gemm,
+                      serial && (c->mlp_chain(serial, n) & kChainDw1) != 0, mlp_mark, c));
+    c->w1_touched[c->cur][worker] = true;
     if (serial) {
         for (bool& u : c->set_used) u = false;
     } else {
@@ -421,7 +461,7 @@ int flush_worker(abs_ctx* c, uint32_t worker) {
     c->pend_n[worker] = 0;
     c->set_reserved[set] = false;
     c->n_reserved -= 1;
-    return run_mlp_group(c, worker, set, n, c->pend_first[worker], true);
+    return run_mlp_group(c, worker, set, n, c->pend_first[worker], c->pend_pool0[worker]);
 }
 
 int flush_all(abs_ctx* c) {
@@ -435,6 +475,75 @@ int flush_all(abs_ctx* c) {
     }
 }
 
+// ABS_FLAG_MLP_DEFER: dW1 of the worker's micro-batches waiting in the current set's operand pool, one launch
+// (K = 64 per micro-batch), stored into -- or, if the W1 slice of its row was written earlier in the iteration,
+// added to -- the accumulator row.  Runs behind the worker's front kernels, on its second stream.
+int contract_worker(abs_ctx* c, uint32_t worker) {
+    const uint32_t set = c->cur;
+    MlpSlots sl{};
+    int n = 0;
+    for (int q = 0; q < c->pool_n[set]; ++q)
+        if (c->pool_owner[set][q] == (int16_t)worker) {
+            sl.s[n++] = (uint16_t)q;
+            c->pool_owner[set][q] = -1;
+        }
+    if (n == 0) return ABS_OK;
+    const int k = (int)(worker % (uint32_t)c->n_wstreams);
+    const bool serial = c->ctas_per_sm[ABS_K_MLP_FWD] == 1;
+    int variant = c->ctas_per_sm[ABS_K_MLP_DW1];
+    // light form beside the other workers' kernels, as for per-call dW1 (measured: batch calls 13.6 -> 13.1 us)
+    if (!serial && c->cfg.W > 1 && !(variant & 128)) variant |= kMlpLightBit;
+    cudaStream_t s_gemm = c->s_acc;
+    if (!serial) {
+        s_gemm = c->s_d[k];
+        CK(cudaEventRecord(c->ev_front[k], c->s_w[k]));
+        CK(cudaStreamWaitEvent(s_gemm, c->ev_front[k], 0));
+    }
+    const bool store = !c->w1_touched[set][worker];
+    CK(launch_mlp_dw1(c->mlp_dims, c->mlp_scratch[0], &c->pool[set], &sl, c->acc(set, worker),
+                      &c->acc_tmaps[(size_t)set * c->cfg.W + worker], n, store, variant, s_gemm, false, mlp_mark, c));
+    c->w1_touched[set][worker] = true;
+    if (!serial) {
+        CK(cudaEventRecord(c->ev_w_done[k], s_gemm));
+        c->w_outstanding[k] = true;
+    }
+    return ABS_OK;
+}
+
+// Every gradient enqueued so far is on its way into the accumulator rows: waiting groups are started and
+// (ABS_FLAG_MLP_DEFER) the pooled dW1 operands contracted.
+int settle_all(abs_ctx* c) {
+    if (int rc = flush_all(c)) return rc;
+    if (!c->defer) return ABS_OK;
+    for (uint32_t i = 0; i < c->cfg.W; ++i)
+        if (int rc = contract_worker(c, i)) return rc;
+    return ABS_OK;
+}
+
+// n consecutive free slots of the current set's operand pool.  A full pool is emptied first: everything in it is
+// contracted, and stream_acc (so every later kernel that writes a slot) waits for those launches.
+int take_pool_slots(abs_ctx* c, int n, int* slot0) {
+    const uint32_t set = c->cur;
+    if (c->pool_n[set] + n > c->pool[set].cap) {
+        if (int rc = settle_all(c)) return rc;
+        for (int k = 0; k < c->n_wstreams; ++k)
+            if (c->w_outstanding[k]) {
+                CK(cudaStreamWaitEvent(c->s_acc, c->ev_w_done[k], 0));
+                c->w_outstanding[k] = false;
+            }
+        c->pool_n[set] = 0;
+    }
+    *slot0 = c->pool_n[set];
+    c->pool_n[set] += n;
+    return ABS_OK;
+}
+
+// The iteration of set `closing` has ended (its gradients are settled); `opening` starts a new one.
+void turn_sets(abs_ctx* c, uint32_t closing, uint32_t opening) {
+    c->pool_n[closing] = 0;
+    for (uint32_t i = 0; i < c->cfg.W; ++i) c->w1_touched[opening][i] = false;
+}
+
 // One micro-batch of `worker` joins its waiting group: cast now (the caller's buffers are free again once
 // stream_acc has passed this point), everything else when the group runs.
 int coalesce_one(abs_ctx* c, uint32_t worker, const void* x_dev, const int32_t* y_dev) {
@@ -446,6 +555,8 @@ int coalesce_one(abs_ctx* c, uint32_t worker, const void* x_dev, const int32_t* 
             if (int rc = flush_worker(c, (uint32_t)oldest)) return rc;
         }
         int set = 0;
+        if (c->defer)   // the group's dW1 operands sit in consecutive pool slots (unused ones stay empty)
+            if (int rc = take_pool_slots(c, kMlpMaxBatch, &c->pend_pool0[worker])) return rc;
         if (int rc = take_scratch_set(c, false, &set)) return rc;
         c->set_reserved[set] = true;
         c->n_reserved += 1;
@@ -454,7 +565,9 @@ int coalesce_one(abs_ctx* c, uint32_t worker, const void* x_dev, const int32_t* 
         c->pend_age[worker] = ++c->pend_clock;
     }
     const int slot = c->pend_n[worker];
-    CK(launch_mlp_cast(c->mlp_dims, c->mlp_scratch[c->pend_set[worker]], slot, 1, x_dev, c->x_bf16(), y_dev, c->s_acc,
+    __nv_bfloat16* xtb_out = nullptr;
+    if (c->defer) xtb_out = c->pool[c->cur].xtb + (size_t)(c->pend_pool0[worker] + slot) * c->mlp_dims.d_in * c->mlp_dims.mb;
+    CK(launch_mlp_cast(c->mlp_dims, c->mlp_scratch[c->pend_set[worker]], slot, 1, x_dev, c->x_bf16(), y_dev, xtb_out, c->s_acc,
                        (c->mlp_chain(false, 1) & kChainCast) != 0, mlp_mark, c));
     c->pend_n[worker] = slot + 1;
     c->h_cnt[(size_t)c->cur * c->cfg.W + worker] += 1;
@@ -498,6 +611,7 @@ int abs_init(abs_ctx** out, const abs_config* cfg, void* workspace_dev, size_t w
     c->pipelined = cfg->flags & ABS_FLAG_PIPELINED;
     c->mlp = cfg->flags & ABS_FLAG_MLP;
     c->coalesce = cfg->flags & ABS_FLAG_MLP_COALESCE;
+    c->defer = cfg->flags & ABS_FLAG_MLP_DEFER;
     c->h_cnt.assign((size_t)2 * cfg->W, 0);
     c->lr_now = cfg->lr;
     c->lr_prev_call = cfg->lr;
@@ -546,6 +660,12 @@ int abs_init(abs_ctx** out, const abs_config* cfg, void* workspace_dev, size_t w
                 return bail(e, "cudaMemsetAsync");
             if ((e = cudaEventCreateWithFlags(&c->ev_set_done[k], cudaEventDisableTiming)) != cudaSuccess) return bail(e, "cudaEventCreate");
         }
+        if (c->defer)
+            for (int k = 0; k < 2; ++k) {
+                if ((e = mlp_pool_init(&c->pool[k], c->mlp_dims, L.pool_cap, c->ws + L.off_pool[k])) != cudaSuccess)
+                    return bail(e, "cuTensorMapEncodeTiled(operand pool)");
+                c->pool_owner[k].assign((size_t)L.pool_cap, (int16_t)-1);
+            }
         if ((e = cudaEventCreateWithFlags(&c->ev_fork, cudaEventDisableTiming)) != cudaSuccess) return bail(e, "cudaEventCreate");
         c->n_wstreams = (int)std::min<uint32_t>(cfg->W, kMlpStreams);
         // Highest priority: the short, dependent gradient kernels get free CTA slots before the long HBM-bound
@@ -592,6 +712,7 @@ int abs_accumulate(abs_ctx* c, uint32_t worker, const void* grad_dev) {
                              c->ctas_per_sm[ABS_K_ACCUMULATE], c->num_sms, c->s_acc, c->chained()));
     }
     c->launches += 1;
+    c->w1_touched[c->cur][worker] = true;
     c->h_cnt[(size_t)c->cur * c->cfg.W + worker] += 1;
     return ABS_OK;
 }
@@ -615,6 +736,7 @@ int abs_accumulate_batch(abs_ctx* c, uint32_t worker, uint32_t n, const void* co
                                    first, c->ctas_per_sm[ABS_K_ACCUMULATE], c->num_sms, c->s_acc, c->chained()));
     }
     c->launches += 1;
+    c->w1_touched[c->cur][worker] = true;
     c->h_cnt[(size_t)c->cur * c->cfg.W + worker] += (int32_t)n;
     return ABS_OK;
 }
@@ -643,6 +765,7 @@ int abs_accumulate_host(abs_ctx* c, uint32_t worker, const void* grad_host) {
     CK(cudaEventRecord(c->ev_stage_free[k], c->s_acc));
     c->stage_used[k] = true;
     c->launches += 1;
+    c->w1_touched[c->cur][worker] = true;
     c->h_cnt[(size_t)c->cur * c->cfg.W + worker] += 1;
     return ABS_OK;
 }
@@ -663,15 +786,20 @@ int abs_accumulate_mlp_batch(abs_ctx* c, uint32_t worker, uint32_t n, const void
     if (serial) {
         if (int rc = join_workers(c)) return rc;
     }
-    int set = 0;
+    int set = 0, pool0 = 0;
+    __nv_bfloat16* xtb_out = nullptr;
+    if (c->defer) {
+        if (int rc = take_pool_slots(c, (int)n, &pool0)) return rc;
+        xtb_out = c->pool[c->cur].xtb + (size_t)pool0 * c->mlp_dims.d_in * c->mlp_dims.mb;
+    }
     if (int rc = take_scratch_set(c, serial, &set)) return rc;
     // A worker's first gradient of an iteration finds its accumulator row empty (all zero, or -- with
     // ABS_FLAG_OVERWRITE_FIRST -- stale): it is stored, not added, and dW1 skips reading the 4 d_in d_hidden
     // bytes of the slice.  0 + g = g, so the default mode's results do not change.
     const bool first = c->h_cnt[(size_t)c->cur * c->cfg.W + worker] == 0;
-    CK(launch_mlp_cast(c->mlp_dims, c->mlp_scratch[set], 0, (int)n, x_dev, c->x_bf16(), y_dev, c->s_acc,
+    CK(launch_mlp_cast(c->mlp_dims, c->mlp_scratch[set], 0, (int)n, x_dev, c->x_bf16(), y_dev, xtb_out, c->s_acc,
                        (c->mlp_chain(serial, (int)n) & kChainCast) != 0, mlp_mark, c));
-    if (int rc = run_mlp_group(c, worker, set, (int)n, first, false)) return rc;
+    if (int rc = run_mlp_group(c, worker, set, (int)n, first, pool0)) return rc;
     c->h_cnt[(size_t)c->cur * c->cfg.W + worker] += (int32_t)n;
     return ABS_OK;
 }
@@ -683,7 +811,7 @@ int abs_accumulate_mlp(abs_ctx* c, uint32_t worker, const void* x_dev, const int
 int abs_sync_step(abs_ctx* c) {
     if (!live(c)) return ABS_ESTATE;
     if (c->n_ranks != 0) return invalid(c, "context is in multi-GPU mode: end iterations with abs_global_begin / _step / _end");
-    if (int rc = flush_all(c)) return rc;   // every gradient of iteration t is under way before the iteration ends
+    if (int rc = settle_all(c)) return rc;   // every gradient of iteration t is under way before the iteration ends
     const uint32_t W = c->cfg.W;
     const uint32_t d = c->cur ^ 1;   // the delayed set (filled during iteration t-1)
     if (!c->pipelined) {
@@ -740,6 +868,7 @@ int abs_sync_step(abs_ctx* c) {
     }
     // Logical state (Algorithm 1: clear the consumed set, swap roles, t = t + 1).
     for (uint32_t i = 0; i < W; ++i) c->h_cnt[(size_t)d * W + i] = 0;
+    turn_sets(c, c->cur, d);
     c->lr_prev_call = c->lr_now;
     c->cur = d;
     c->t += 1;
@@ -793,7 +922,7 @@ int abs_global_begin(abs_ctx* c, int32_t** counts_dev, uint32_t* n_counts) {
     if (c->n_ranks == 0) return invalid(c, "abs_global_attach has not been called");
     if (c->global_phase != 0) return invalid(c, "abs_global_begin / _step / _end must be called in that order");
     if (!counts_dev || !n_counts) return invalid(c, "output pointer is NULL");
-    if (int rc = flush_all(c)) return rc;
+    if (int rc = settle_all(c)) return rc;
     const uint32_t W = c->cfg.W;
     // Publish x_{t+1}: the kernels launched one call ago, on every rank, have all finished (ev_sync_done was
     // recorded behind the caller's closing barrier).
@@ -855,6 +984,7 @@ int abs_global_step(abs_ctx* c) {
     // Logical state (Algorithm 1: clear the consumed set, swap roles, t = t + 1).
     const uint32_t d = c->cur ^ 1;
     for (uint32_t i = 0; i < W; ++i) c->h_cnt[(size_t)d * W + i] = 0;
+    turn_sets(c, c->cur, d);
     c->lr_prev_call = c->lr_now;
     c->cur = d;
     c->t += 1;
@@ -1024,7 +1154,7 @@ int abs_wait(abs_ctx* c) {
 
 int abs_check(abs_ctx* c) {
     if (!live(c)) return ABS_ESTATE;
-    if (int rc = flush_all(c)) return rc;
+    if (int rc = settle_all(c)) return rc;
     if (c->pipelined) CK(cudaStreamSynchronize(c->s_sync));
     for (int k = 0; k < c->n_wstreams; ++k) {
         CK(cudaStreamSynchronize(c->s_w[k]));
@@ -1079,7 +1209,7 @@ bool same_config(const abs_config& a, const abs_config& b) {
 
 // Everything enqueued so far has finished (waiting micro-batch groups are started first).
 int drain(abs_ctx* c) {
-    if (int rc = flush_all(c)) return rc;
+    if (int rc = settle_all(c)) return rc;
     if (c->pipelined) CK(cudaStreamSynchronize(c->s_sync));
     for (int k = 0; k < c->n_wstreams; ++k) {
         CK(cudaStreamSynchronize(c->s_w[k]));
@@ -1152,6 +1282,10 @@ int abs_state_import(abs_ctx* c, const void* src_host, size_t bytes) {
     c->disp_scale = h.disp_scale;
     c->global_prev_lr = h.global_prev_lr;
     for (size_t k = 0; k < c->h_cnt.size(); ++k) c->h_cnt[k] = h.h_cnt[k];
+    for (uint32_t set = 0; set < 2; ++set) {   // a row that has received gradients may hold some in its W1 slice
+        c->pool_n[set] = 0;
+        for (uint32_t i = 0; i < c->cfg.W; ++i) c->w1_touched[set][i] = c->h_cnt[(size_t)set * c->cfg.W + i] > 0;
+    }
     if (c->mlp) {   // the bf16 copies are a function of the parameters: rebuild them
         CK(launch_cast_bf16(c->x(0), c->shadow(0), c->L.P_pad, c->num_sms, c->s_acc));
         c->launches += 1;
@@ -1181,7 +1315,7 @@ int abs_set_launch(abs_ctx* c, int kernel_class, int ctas_per_sm) {
         return invalid(c, "unknown bits in the ABS_K_MLP_DW1 mask");
     if (kernel_class == ABS_K_CHAIN && (ctas_per_sm < 0 || ctas_per_sm > 1)) return invalid(c, "ABS_K_CHAIN takes 0 or 1");
     if (kernel_class == ABS_K_MLP_FWD && (ctas_per_sm < 0 || ctas_per_sm > 1)) return invalid(c, "ABS_K_MLP_FWD takes 0 or 1");
-    if (int rc = flush_all(c)) return rc;
+    if (int rc = settle_all(c)) return rc;
     c->ctas_per_sm[kernel_class] = ctas_per_sm;
     return ABS_OK;
 }

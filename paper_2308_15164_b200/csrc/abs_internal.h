@@ -72,6 +72,7 @@ struct SyncArgs {
     unsigned int norm_slots;  // slots in norm_part
     int overlapped;           // the launch runs beside the next iteration's accumulate kernels (pipelined mode)
     int* status;              // optional device status word (ABS_ETIMEOUT if a bounded wait of the bulk-copy kernel ran out)
+    int tma_one_cta;          // bulk-copy form: 0 = as many CTAs per SM as its budget holds; n > 0 = one CTA per SM with n stages
     int plain_only;           // 1: never the bulk-copy form (a caller without a status word to report its time-outs through)
 };
 // n (1..kMaxAccBatch) gradients of one worker added in one pass over its accumulator row, in list order.
@@ -134,6 +135,12 @@ constexpr int kMlpSets = 8;      // scratch sets, one per call in flight, taken 
 struct MlpDims {
     int d_in, d_hidden, d_out, mb;
 };
+// Micro-batches one dW1 launch may contract (K = 64 per micro-batch) and the slots of the stacked operand
+// tensors that hold them, in contraction order.
+constexpr int kMlpMaxSlots = 128;
+struct MlpSlots {
+    uint16_t s[kMlpMaxSlots];
+};
 struct alignas(64) TmapBytes {   // storage for one CUtensorMap (encoded on the host, passed by value to kernels)
     unsigned char b[128];
 };
@@ -156,6 +163,16 @@ struct MlpScratch {      // device pointers carved from the workspace (all hidde
     TmapBytes tmap_xt, tmap_dzt;   // dW1 operands
     TmapBytes tmap_xb, tmap_w1[2]; // forward GEMM operands (W1 of each bf16 shadow copy)
 };
+// ABS_FLAG_MLP_DEFER: the dW1 operands of an accumulator set's gradient calls are kept (bf16(X)^T and bf16(dZ)^T,
+// (d_in + d_hidden) * 128 bytes per micro-batch) in `cap` slots instead of being contracted call by call.
+struct MlpPool {
+    __nv_bfloat16* xtb;  // [cap][d_in][mb]
+    __nv_bfloat16* dzt;  // [cap][d_hidden][mb]
+    int cap;
+    TmapBytes tmap_xt, tmap_dzt;
+};
+size_t mlp_pool_bytes(const MlpDims& d, int cap);
+cudaError_t mlp_pool_init(MlpPool* p, const MlpDims& d, int cap, void* base);
 size_t mlp_scratch_bytes(const MlpDims& d);
 // Lays the scratch out at `base` (1024-B aligned) and encodes the operand TMA descriptors (host call).
 cudaError_t mlp_scratch_init(MlpScratch* s, const MlpDims& d, void* base, __nv_bfloat16* shadow0,
@@ -173,17 +190,23 @@ cudaError_t mlp_make_acc_tmap(void* tmap_out, const MlpDims& d, float* acc_row);
 // one call -- forward class: 0 cast, 1 forward GEMM, 2 bias / ReLU / logits), mark(user, kernel_class, n, stream)
 // after its n launches.
 typedef void (*MlpMark)(void* user, int kernel_class, int n, cudaStream_t stream);
+// xtb_out / dzt_out: where bf16(X)^T / bf16(dZ)^T of the call's nb micro-batches go ([nb][d_in][mb] /
+// [nb][d_hidden][mb]); nullptr: slots slot0.. / 0.. of the scratch set.
 cudaError_t launch_mlp_cast(const MlpDims& d, const MlpScratch& s, int slot0, int nb, const void* x_dev, bool x_is_bf16,
-                            const int32_t* y_dev, cudaStream_t stream, bool chained, MlpMark mark, void* user);
+                            const int32_t* y_dev, __nv_bfloat16* xtb_out, cudaStream_t stream, bool chained, MlpMark mark,
+                            void* user);
 cudaError_t launch_mlp_front(const MlpDims& d, const MlpScratch& s, const float* x_pub, const __nv_bfloat16* shadow,
-                             int shadow_idx, int nb, bool store, float* acc_row, int32_t* cnt, int variant,
-                             cudaStream_t stream, int chain, MlpMark mark, void* user);
+                             int shadow_idx, int nb, bool store, float* acc_row, int32_t* cnt, __nv_bfloat16* dzt_out,
+                             int variant, cudaStream_t stream, int chain, MlpMark mark, void* user);
 // nb: a call may carry up to kMlpMaxBatch micro-batches (x_dev [nb][mb][d_in], y_dev [nb][mb]): the front kernels
 // take them as an extra grid dimension, and ONE dW1 launch contracts them with K = 64 nb (the accumulator slice is
 // read and written once).
 // store: the accumulator row holds nothing yet (the worker's first gradient of the iteration): front and dw1
 // store their results instead of adding them, and dw1 does not read the accumulator slice at all.
-cudaError_t launch_mlp_dw1(const MlpDims& d, const MlpScratch& s, float* acc_row, const void* acc_tmap, int nb, bool store,
-                           int variant, cudaStream_t stream, bool chained, MlpMark mark, void* user);
+// pool: the operands are those of a deferred-operand pool, micro-batch j in slot slots->s[j] (nb <= kMlpMaxSlots);
+// nullptr: slots 0..nb-1 of the scratch set (nb <= kMlpMaxBatch).
+cudaError_t launch_mlp_dw1(const MlpDims& d, const MlpScratch& s, const MlpPool* pool, const MlpSlots* slots, float* acc_row,
+                           const void* acc_tmap, int nb, bool store, int variant, cudaStream_t stream, bool chained,
+                           MlpMark mark, void* user);
 
 }  // namespace abs_sgd

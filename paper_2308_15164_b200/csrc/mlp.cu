@@ -418,7 +418,7 @@ constexpr int kPanels = kDwN / 32;
 // K batching: the operands of nb (1..kMaxBatch) micro-batches are stacked along K, so one launch
 // computes  acc += sum_j X_j^T dZ_j  (K = 64 nb) and the accumulator slice is read and written once
 // for nb micro-batches instead of nb times -- the kernel is bound by that traffic, not by the MMAs.
-// Operand j lives at row offset j*d_in (X^T) / j*d_h (dZ^T) of the stacked operand tensors.
+// Operand j lives in slot sl.s[j] of the stacked operand tensors: row offset slot*d_in (X^T) / slot*d_h (dZ^T).
 // 256 threads: warps 0-3 read TMEM columns 0..31 of their lane quarter, warps 4-7 columns 32..63.
 // ============================================================================================
 constexpr int kDwPitch = kDwN + 4;   // floats per row of the staging tile (pitch 272 B: conflict-free float4 rows)
@@ -438,8 +438,9 @@ __host__ __device__ constexpr int dw_regs_buf_bytes(int nb) {
 }
 
 __global__ void __launch_bounds__(256) k_dw1_regs(const __grid_constant__ CUtensorMap tm_xt,
-                                                  const __grid_constant__ CUtensorMap tm_dzt, float* acc_w1, int d_in,
-                                                  int ld, int nb, int store, int* status) {
+                                                  const __grid_constant__ CUtensorMap tm_dzt,
+                                                  const __grid_constant__ MlpSlots sl, float* acc_w1, int d_in, int ld,
+                                                  int nb, int store, int* status) {
     extern __shared__ uint8_t smem_raw[];
     uint8_t* buf = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
     DwRegCtl& s = *reinterpret_cast<DwRegCtl*>(buf + dw_regs_buf_bytes(nb));
@@ -481,8 +482,8 @@ __global__ void __launch_bounds__(256) k_dw1_regs(const __grid_constant__ CUtens
     if (threadIdx.x == 0) {
         mbar_expect_tx(&s.bar_ab, nb * kDwOperandBytes);
         for (int j = 0; j < nb; ++j) {
-            tma_load_2d(buf + j * kDwOperandBytes, &tm_xt, 0, j * d_in + m0, &s.bar_ab);
-            tma_load_2d(buf + j * kDwOperandBytes + kTileM * 128, &tm_dzt, 0, j * ld + n0, &s.bar_ab);
+            tma_load_2d(buf + j * kDwOperandBytes, &tm_xt, 0, (int)sl.s[j] * d_in + m0, &s.bar_ab);
+            tma_load_2d(buf + j * kDwOperandBytes + kTileM * 128, &tm_dzt, 0, (int)sl.s[j] * ld + n0, &s.bar_ab);
         }
         if (mbar_wait(&s.bar_ab, 0)) {
             asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
@@ -579,7 +580,8 @@ struct DwRingSmem {
 template <int kN, bool kLight = false>
 __global__ void __launch_bounds__(192) k_dw1_ring(const __grid_constant__ CUtensorMap tm_xt,
                                                   const __grid_constant__ CUtensorMap tm_dzt,
-                                                  const __grid_constant__ CUtensorMap tm_acc, int n_tiles_n, int n_tiles,
+                                                  const __grid_constant__ CUtensorMap tm_acc,
+                                                  const __grid_constant__ MlpSlots sl, int n_tiles_n, int n_tiles,
                                                   int d_in, int ld, int nb, int store, int* status) {
     constexpr int kRingOps = DwRingCfg<kN, kLight>::kOps, kSlotBytes = DwRingCfg<kN, kLight>::kSlotBytes;
     constexpr int kRingC = DwRingCfg<kN, kLight>::kC;
@@ -623,10 +625,11 @@ __global__ void __launch_bounds__(192) k_dw1_ring(const __grid_constant__ CUtens
                     const int st = q % kRingOps;
                     if (q >= kRingOps && !mbar_wait(&s.op_empty[st], ((q / kRingOps) - 1) & 1)) { s.failed = 1; break; }
                     mbar_expect_tx(&s.op_full[st], kSlotBytes);
-                    tma_load_2d(s.op[st], &tm_xt, 0, j * d_in + m0, &s.op_full[st]);
+                    const int slot = (int)sl.s[j];   // where micro-batch j of the contraction sits in the stacked operands
+                    tma_load_2d(s.op[st], &tm_xt, 0, slot * d_in + m0, &s.op_full[st]);
 #pragma unroll
                     for (int b = 0; b < kHalves; ++b)   // 64-row boxes, 8 KB apart: one K-major B operand of kN rows
-                        tma_load_2d(s.op[st] + kTileM * 128 + b * (kDwN * 128), &tm_dzt, 0, j * ld + n0 + b * kDwN, &s.op_full[st]);
+                        tma_load_2d(s.op[st] + kTileM * 128 + b * (kDwN * 128), &tm_dzt, 0, slot * ld + n0 + b * kDwN, &s.op_full[st]);
                 }
             }
         }
@@ -987,6 +990,23 @@ cudaError_t mlp_scratch_init(MlpScratch* s, const MlpDims& d, void* base, __nv_b
     return e;
 }
 
+size_t mlp_pool_bytes(const MlpDims& d, int cap) {
+    return align_up((size_t)cap * d.d_in * kMB * 2, 1024) + align_up((size_t)cap * d.d_hidden * kMB * 2, 1024);
+}
+
+cudaError_t mlp_pool_init(MlpPool* p, const MlpDims& d, int cap, void* base) {
+    p->cap = cap;
+    p->xtb = static_cast<__nv_bfloat16*>(base);
+    p->dzt = reinterpret_cast<__nv_bfloat16*>(static_cast<char*>(base) + align_up((size_t)cap * d.d_in * kMB * 2, 1024));
+    // same boxes as the scratch sets' operands: slot j at rows [j*d_in, (j+1)*d_in) of X^T, [j*d_h, (j+1)*d_h) of dZ^T
+    if (!encode_2d(reinterpret_cast<CUtensorMap*>(&p->tmap_xt), CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, p->xtb,
+                   (uint64_t)cap * d.d_in, kMB, kTileM, kMB) ||
+        !encode_2d(reinterpret_cast<CUtensorMap*>(&p->tmap_dzt), CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, p->dzt,
+                   (uint64_t)cap * d.d_hidden, kMB, kDwN, kMB))
+        return cudaErrorInvalidValue;
+    return cudaSuccess;
+}
+
 cudaError_t mlp_make_acc_tmap(void* tmap_out, const MlpDims& d, float* acc_row) {
     // W1 slice of a worker's accumulator: [d_in][d_hidden] fp32 at offset 0 of the flat row.
     return encode_2d(reinterpret_cast<CUtensorMap*>(tmap_out), CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, acc_row, d.d_in,
@@ -996,11 +1016,12 @@ cudaError_t mlp_make_acc_tmap(void* tmap_out, const MlpDims& d, float* acc_row) 
 }
 
 cudaError_t launch_mlp_cast(const MlpDims& d, const MlpScratch& s, int slot0, int nb, const void* x_dev, bool x_is_bf16,
-                            const int32_t* y_dev, cudaStream_t stream, bool chained, MlpMark mark, void* user) {
+                            const int32_t* y_dev, __nv_bfloat16* xtb_out, cudaStream_t stream, bool chained, MlpMark mark,
+                            void* user) {
     mark(user, ABS_K_MLP_FWD, -1, stream);   // part 0 of the forward class: the cast
     // micro-batch j of the call goes to slot slot0 + j of the scratch set
     __nv_bfloat16* xb = s.xb + (size_t)slot0 * kMB * d.d_in;
-    __nv_bfloat16* xtb = s.xtb + (size_t)slot0 * d.d_in * kMB;
+    __nv_bfloat16* xtb = xtb_out ? xtb_out : s.xtb + (size_t)slot0 * d.d_in * kMB;
     int32_t* yc = s.ycopy + slot0 * kMB;
     const dim3 grid(d.d_in / 16, nb);
     const cudaError_t e = x_is_bf16 ? launch_kernel(k_cast_x<true>, grid, 256, 0, stream, chained, x_dev, y_dev, xb, xtb, yc, d.d_in)
@@ -1020,8 +1041,8 @@ cudaError_t fwd1_launch(dim3 grid, cudaStream_t stream, bool chained, bool light
 }
 
 cudaError_t launch_mlp_front(const MlpDims& d, const MlpScratch& s, const float* x_pub, const __nv_bfloat16* shadow,
-                             int shadow_idx, int nb, bool store, float* acc_row, int32_t* cnt, int variant,
-                             cudaStream_t stream, int chain, MlpMark mark, void* user) {
+                             int shadow_idx, int nb, bool store, float* acc_row, int32_t* cnt, __nv_bfloat16* dzt_out,
+                             int variant, cudaStream_t stream, int chain, MlpMark mark, void* user) {
     const size_t o_b1 = (size_t)d.d_in * d.d_hidden, o_w2 = o_b1 + d.d_hidden, o_b2 = o_w2 + (size_t)d.d_hidden * d.d_out;
     cudaError_t e;
     const unsigned n_cta = d.d_hidden / kHB;
@@ -1058,7 +1079,8 @@ cudaError_t launch_mlp_front(const MlpDims& d, const MlpScratch& s, const float*
     const float* gpart = s.gpart;
     const float* b2 = x_pub + o_b2;
     const int32_t* yc = s.ycopy;
-    e = launch_kernel(k_bwd, dim3(n_cta, nb), 256, 0, stream, (chain & kChainBwd) != 0, hbt, gpart, n_groups, b2, yc, w2b, s.dzt, s.bpart,
+    e = launch_kernel(k_bwd, dim3(n_cta, nb), 256, 0, stream, (chain & kChainBwd) != 0, hbt, gpart, n_groups, b2, yc, w2b,
+                      dzt_out ? dzt_out : s.dzt, s.bpart,
                       s.tickets_b, acc_row + o_b1, acc_row + o_w2, acc_row + o_b2, cnt, d.d_hidden, d.d_out, store ? 1 : 0);
     mark(user, ABS_K_MLP_BWD, 1, stream);
     return e;
@@ -1066,38 +1088,47 @@ cudaError_t launch_mlp_front(const MlpDims& d, const MlpScratch& s, const float*
 
 template <int kN, bool kLight>
 cudaError_t dw1_ring_launch(const MlpDims& d, const MlpScratch& s, const CUtensorMap& ta, const CUtensorMap& tb,
-                            const CUtensorMap& tc, int nb, int st, cudaStream_t stream, bool chained) {
+                            const CUtensorMap& tc, const MlpSlots& sl, int nb, int st, cudaStream_t stream, bool chained) {
     const int n_tiles_n = d.d_hidden / kN, n_tiles = n_tiles_n * (d.d_in / kTileM);
     const int ctas = n_tiles < s.num_sms ? n_tiles : s.num_sms;
     return launch_kernel(k_dw1_ring<kN, kLight>, ctas, 192, sizeof(DwRingSmem<kN, kLight>) + 1024, stream, chained, ta, tb, tc,
-                         n_tiles_n, n_tiles, d.d_in, d.d_hidden, nb, st, s.status);
+                         sl, n_tiles_n, n_tiles, d.d_in, d.d_hidden, nb, st, s.status);
 }
 
-cudaError_t launch_mlp_dw1(const MlpDims& d, const MlpScratch& s, float* acc_row, const void* acc_tmap, int nb, bool store,
-                           int variant, cudaStream_t stream, bool chained, MlpMark mark, void* user) {
+cudaError_t launch_mlp_dw1(const MlpDims& d, const MlpScratch& s, const MlpPool* pool, const MlpSlots* slots, float* acc_row,
+                           const void* acc_tmap, int nb, bool store, int variant, cudaStream_t stream, bool chained,
+                           MlpMark mark, void* user) {
     const int st = store ? 1 : 0;
     const bool light = (variant & kMlpLightBit) != 0;
+    if (nb < 1 || nb > (pool ? kMlpMaxSlots : kMaxBatch) || (pool && !slots)) return cudaErrorInvalidValue;
     mark(user, ABS_K_MLP_DW1, -1, stream);
-    const CUtensorMap& ta = *reinterpret_cast<const CUtensorMap*>(&s.tmap_xt);
-    const CUtensorMap& tb = *reinterpret_cast<const CUtensorMap*>(&s.tmap_dzt);
+    const CUtensorMap& ta = *reinterpret_cast<const CUtensorMap*>(pool ? &pool->tmap_xt : &s.tmap_xt);
+    const CUtensorMap& tb = *reinterpret_cast<const CUtensorMap*>(pool ? &pool->tmap_dzt : &s.tmap_dzt);
     const CUtensorMap& tc = *reinterpret_cast<const CUtensorMap*>(acc_tmap);
+    MlpSlots sl;
+    if (pool) {
+        sl = *slots;
+    } else {
+        for (int j = 0; j < kMlpMaxSlots; ++j) sl.s[j] = (uint16_t)(j < kMaxBatch ? j : 0);
+    }
     // Which kernel: bit 4 (ring) or 8 (register prefetch) forces one; otherwise the measured best for the case: the
     // persistent ring kernel when the tile is stored (it never reads the accumulator) and for K-batched adds, the
     // register-prefetch kernel for single adds.
     int kind = (variant & 4) ? 4 : (variant & 8) ? 8 : 0;
     if (kind == 0) kind = (store || nb > 1) ? 4 : 8;
+    if (nb > kMaxBatch) kind = 4;          // the register-prefetch kernel holds every operand in shared memory at once
     cudaError_t e;
     if (kind == 4) {
         if (nb > 1 && !(variant & 32))     // K-batched: 128 x 128 tiles (bit 32 keeps 128 x 64)
-            e = light ? dw1_ring_launch<128, true>(d, s, ta, tb, tc, nb, st, stream, chained)
-                      : dw1_ring_launch<128, false>(d, s, ta, tb, tc, nb, st, stream, chained);
+            e = light ? dw1_ring_launch<128, true>(d, s, ta, tb, tc, sl, nb, st, stream, chained)
+                      : dw1_ring_launch<128, false>(d, s, ta, tb, tc, sl, nb, st, stream, chained);
         else
-            e = light ? dw1_ring_launch<64, true>(d, s, ta, tb, tc, nb, st, stream, chained)
-                      : dw1_ring_launch<64, false>(d, s, ta, tb, tc, nb, st, stream, chained);
+            e = light ? dw1_ring_launch<64, true>(d, s, ta, tb, tc, sl, nb, st, stream, chained)
+                      : dw1_ring_launch<64, false>(d, s, ta, tb, tc, sl, nb, st, stream, chained);
     } else {
         const size_t smem = dw_regs_buf_bytes(nb) + sizeof(DwRegCtl) + 1024;
-        e = launch_kernel(k_dw1_regs, dim3(d.d_hidden / kDwN, d.d_in / kTileM), 256, smem, stream, chained, ta, tb, acc_row, d.d_in,
-                          d.d_hidden, nb, st, s.status);
+        e = launch_kernel(k_dw1_regs, dim3(d.d_hidden / kDwN, d.d_in / kTileM), 256, smem, stream, chained, ta, tb, sl, acc_row,
+                          d.d_in, d.d_hidden, nb, st, s.status);
     }
     mark(user, ABS_K_MLP_DW1, 1, stream);
     return e;

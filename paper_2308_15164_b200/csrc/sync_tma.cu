@@ -260,6 +260,12 @@ cudaError_t launch_sync_tma(const SyncArgs& a, int num_sms, cudaStream_t stream,
     int stages = (int)((budget_sm / ctas - fixed) / stage_bytes);
     if (stages > kMaxStages) stages = kMaxStages;
     if (stages < 2) stages = 2;
+    if (a.tma_one_cta > 0) {   // the caller wants room left on the SM for another kernel's CTA
+        ctas = 1;
+        stages = a.tma_one_cta > kMaxStages ? kMaxStages : a.tma_one_cta;
+        while (stages > 2 && fixed + (size_t)stages * stage_bytes > budget_sm / 2 + stage_bytes) --stages;
+        if (stages < 2) stages = 2;
+    }
     if (fixed + (size_t)stages * stage_bytes > whole) return cudaErrorNotSupported;
     const int lazy = stages >= 3 ? 1 : 0;
     const size_t smem = fixed + (size_t)stages * stage_bytes;

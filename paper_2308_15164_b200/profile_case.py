@@ -4,7 +4,7 @@
     python -m paper_2308_15164_b200.profile_case accumulate [--P 11689512] [--W 4] [--iters 3] [--bf16]
     python -m paper_2308_15164_b200.profile_case mlp        [--iters 2] [--batch 4] [--calls 2]
     python -m paper_2308_15164_b200.profile_case global     [--P 25557032] [--ranks 4] [--W 2] [--iters 2]
-    python -m paper_2308_15164_b200.profile_case timeline   [--iters 3] [--batch 4]     (no profiler: prints the library's
+    python -m paper_2308_15164_b200.profile_case timeline   [--iters 3] [--batch 4] [--defer]   (no profiler: prints the library's
                                                             own timeline of the MLP workload's kernels)
 
 Each case keeps its working set larger than the 126 MB L2 but to a few hundred MB, launches the
@@ -33,6 +33,7 @@ def main(argv=None):
     ap.add_argument("--batch", type=int, default=1, help="mlp: reference batches per call (1..4)")
     ap.add_argument("--ranks", type=int, default=4, help="global: ranks emulated in this process (W = workers per rank)")
     ap.add_argument("--calls", type=int, default=1, help="mlp: calls per worker and iteration (the first one stores)")
+    ap.add_argument("--defer", action="store_true", help="mlp, timeline: ABS_FLAG_MLP_DEFER (one dW1 contraction per worker and iteration)")
     args = ap.parse_args(argv)
 
     from . import binding as B
@@ -79,7 +80,8 @@ def main(argv=None):
         x0 = torch.from_numpy(wlm.params0(wl)).to(dev)
         xs, ys = wlm.mlp_batches(wl)
         xs_d, ys_d = torch.from_numpy(xs[:8]).to(dev), torch.from_numpy(ys[:8]).to(dev)
-        eng = B.AbsSgd(x0, wl.W, wl.lr, wl.momentum, pipelined=args.pipelined, mlp=(d.d_in, d.d_hidden, d.d_out, d.mb))
+        eng = B.AbsSgd(x0, wl.W, wl.lr, wl.momentum, pipelined=args.pipelined, mlp=(d.d_in, d.d_hidden, d.d_out, d.mb),
+                       mlp_defer=args.defer)
         eng.set_launch(B.K_MLP_DW1, args.epilogue)
         torch.cuda.synchronize()
         c = 0
@@ -108,7 +110,7 @@ def timeline(args, B, wlm, dev):
     xs, ys = wlm.mlp_batches(wl)
     xs_d, ys_d = torch.from_numpy(xs).to(dev), torch.from_numpy(ys).to(dev)
     sched = wlm.schedule(wl)
-    eng = B.AbsSgd(x0, wl.W, wl.lr, wl.momentum, pipelined=True, mlp=(d.d_in, d.d_hidden, d.d_out, d.mb))
+    eng = B.AbsSgd(x0, wl.W, wl.lr, wl.momentum, pipelined=True, mlp=(d.d_in, d.d_hidden, d.d_out, d.mb), mlp_defer=args.defer)
     torch.cuda.synchronize()
     n = 0
 

@@ -52,8 +52,8 @@ def test_workspace_bytes_host_side(B):
 
 
 @pytest.mark.parametrize("kw", [
-    dict(P=0, W=2), dict(P=16, W=0), dict(P=16, W=65), dict(P=16, W=2, grad_dtype=7), dict(P=16, W=2, flags=128),
-    dict(P=16, W=2, flags=64), dict(P=16, W=2, flags=16),
+    dict(P=0, W=2), dict(P=16, W=0), dict(P=16, W=65), dict(P=16, W=2, grad_dtype=7), dict(P=16, W=2, flags=256),
+    dict(P=16, W=2, flags=128), dict(P=16, W=2, flags=64), dict(P=16, W=2, flags=16),
     dict(P=16, W=2, lr=float("nan")), dict(P=16, W=2, flags=1, stream_acc=5, stream_sync=5),
     dict(P=16, W=2, flags=2, mlp=(100, 128, 10, 64)), dict(P=16, W=2, flags=2, mlp=(128, 128, 10, 64)),
     dict(P=128 * 128 + 128 + 1280 + 10, W=2, flags=2, mlp=(128, 128, 10, 32)),

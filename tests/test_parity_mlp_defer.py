@@ -1,0 +1,262 @@
+"""GPU parity of ABS_FLAG_MLP_DEFER: the layer-1 weight gradient of a worker is contracted once per iteration,
+over all its micro-batches (every gradient of an iteration is evaluated at the same x_t: Algorithm 1, Step 2),
+instead of once per call.  Checked against the CPU oracle, through the C ABI, at the bars of the per-call path
+(2e-3 of the tensor maximum element-wise and 2e-3 in Frobenius norm; counters bit-exact):
+
+  * a worker's accumulator row after several single and batch calls (read through abs_accumulator, which makes
+    the library contract what is waiting) against the oracle's sum of gradients;
+  * reading the row in the middle of an iteration and going on (the second contraction adds to the first);
+  * more micro-batches in one iteration than the operand pool holds (early contraction);
+  * whole training runs -- eager, pipelined, with gathered calls, in overwrite-first mode -- against the oracle run,
+    eager and pipelined bit-identical;
+  * gradient vectors (abs_accumulate) and MLP calls mixed within an iteration, idle workers;
+  * export / import in the middle of an iteration."""
+
+import numpy as np
+import pytest
+
+from oracle.abs_oracle import AbsSgdOracle, mlp_loss_and_grad
+from paper_2308_15164_b200 import workloads as wlm
+
+pytestmark = pytest.mark.gpu
+
+TOL = 2e-3
+
+
+def _engine(wl, x0, W=None, pipelined=False, coalesce=False, overwrite_first=False, defer=True):
+    import torch
+
+    from paper_2308_15164_b200 import binding as B
+
+    d = wl.mlp
+    return B.AbsSgd(torch.from_numpy(x0).cuda(), W or wl.W, wl.lr, wl.momentum, wl.weight_decay, pipelined=pipelined,
+                    mlp=(d.d_in, d.d_hidden, d.d_out, d.mb), overwrite_first=overwrite_first, mlp_coalesce=coalesce,
+                    mlp_defer=defer)
+
+
+def _grad(p, xs, ys, c, wl):
+    d = wl.mlp
+    return mlp_loss_and_grad(p, xs[c % wl.mlp_pool], ys[c % wl.mlp_pool], d.d_in, d.d_hidden, d.d_out, mode="bf16")[1].astype(np.float32)
+
+
+def _close_row(got, ref, wl, what):
+    """Tensor by tensor (W1, b1, W2, b2 slices of the flat row)."""
+    d = wl.mlp
+    o = [0, d.d_in * d.d_hidden, d.d_in * d.d_hidden + d.d_hidden, d.d_in * d.d_hidden + d.d_hidden + d.d_hidden * d.d_out, wl.P]
+    for name, lo, hi in zip(("dW1", "db1", "dW2", "db2"), o[:-1], o[1:]):
+        g, r = got[lo:hi].astype(np.float64), ref[lo:hi].astype(np.float64)
+        assert np.abs(g - r).max() <= TOL * np.abs(r).max(), f"{what}: {name} max err {np.abs(g - r).max():.3e} vs {TOL}*{np.abs(r).max():.3e}"
+        assert np.linalg.norm(g - r) <= TOL * np.linalg.norm(r), f"{what}: {name} Frobenius"
+
+
+@pytest.mark.parametrize("small", [True, False], ids=["384x512", "3072x4096"])
+def test_row_after_several_calls_and_a_read_in_the_middle(small):
+    import torch
+
+    wl = wlm.config(4, small=small, T=1)
+    x0 = wlm.params0(wl)
+    xs, ys = wlm.mlp_batches(wl)
+    xs_d, ys_d = torch.from_numpy(xs).cuda(), torch.from_numpy(ys).cuda()
+    eng = _engine(wl, x0)
+    # worker 2: 1 + 3 + 1 micro-batches; worker 0: 2; workers 1, 3 idle
+    plan = [(2, 1), (0, 2), (2, 3), (2, 1)]
+    ref = {0: np.zeros(wl.P, np.float32), 2: np.zeros(wl.P, np.float32)}
+    c = 0
+    for (i, n) in plan:
+        eng.accumulate_mlp_batch(i, n, xs_d[c:c + n], ys_d[c:c + n]) if n > 1 else eng.accumulate_mlp(i, xs_d[c], ys_d[c])
+        for j in range(n):
+            ref[i] = ref[i] + _grad(x0, xs, ys, c + j, wl)
+        c += n
+    cur = eng.counters()[1]
+    for i in (0, 2):
+        _close_row(eng.accumulator(cur, i).cpu().numpy(), ref[i], wl, f"worker {i}")
+    for i in (1, 3):
+        assert not eng.accumulator(cur, i).any()
+    # the iteration goes on: what comes now is added to what the read made the library contract
+    for (i, n) in [(2, 2), (1, 1)]:
+        eng.accumulate_mlp_batch(i, n, xs_d[c:c + n], ys_d[c:c + n]) if n > 1 else eng.accumulate_mlp(i, xs_d[c], ys_d[c])
+        for j in range(n):
+            ref[i] = ref.get(i, np.zeros(wl.P, np.float32)) + _grad(x0, xs, ys, c + j, wl)
+        c += n
+    for i in (0, 1, 2):
+        _close_row(eng.accumulator(cur, i).cpu().numpy(), ref[i], wl, f"worker {i}, second read")
+    assert eng.counters()[0][cur].tolist() == [2, 1, 7, 0]
+    eng.check()
+    eng.destroy()
+
+
+@pytest.mark.parametrize("calls", ["single", "batches-of-3"])
+def test_more_microbatches_than_the_pool_holds(calls):
+    """W = 2: the pool holds 32 micro-batches; 45 arrive in one iteration (worker 0: 30, worker 1: 15)."""
+    import torch
+
+    wl = wlm.config(4, small=True, T=1)
+    x0 = wlm.params0(wl)
+    xs, ys = wlm.mlp_batches(wl)
+    xs_d, ys_d = torch.from_numpy(xs).cuda(), torch.from_numpy(ys).cuda()
+    o = AbsSgdOracle(x0, 2, wl.lr, wl.momentum, wl.weight_decay)
+    eng = _engine(wl, x0, W=2, pipelined=True)
+    step = 1 if calls == "single" else 3
+    c = 0
+    for rnd in range(15 // step):
+        for i, n in ((0, 2 * step), (1, step)):
+            for lo in range(0, n, step):
+                at = c % (wl.mlp_pool - step)
+                if step == 1:
+                    eng.accumulate_mlp(i, xs_d[at], ys_d[at])
+                else:
+                    eng.accumulate_mlp_batch(i, step, xs_d[at:at + step], ys_d[at:at + step])
+                for j in range(step):
+                    o.accumulate(i, _grad(x0, xs, ys, at + j, wl))
+                c += step
+    cur = eng.counters()[1]
+    assert eng.counters()[0][cur].tolist() == [30, 15]
+    for _ in range(3):
+        eng.sync_step(); o.sync_step()
+    eng.check()
+    got = eng.params_host()
+    ref = o.params()
+    assert np.abs(ref - x0).max() > 1e-4
+    assert np.abs(got.astype(np.float64) - ref).max() <= TOL * np.abs(ref).max()
+    assert np.array_equal(eng.consumed(1), np.array([30, 15]))
+    eng.destroy()
+
+
+def _run(wl, x0, xs_d, ys_d, **kw):
+    eng = _engine(wl, x0, **kw)
+    states = []
+    for t, calls in enumerate(wlm.iter_calls(wl)):
+        for (i, k, c) in calls:
+            eng.accumulate_mlp(i, xs_d[c % wl.mlp_pool], ys_d[c % wl.mlp_pool])
+        eng.sync_step()
+        states.append(eng.counters())
+    eng.check()
+    out = eng.params_host()
+    consumed = [eng.consumed(s) for s in range(len(states))]
+    eng.destroy()
+    return out, states, consumed
+
+
+@pytest.mark.parametrize("small,T", [(True, 12), (False, 5)], ids=["384x512-T12", "3072x4096-T5"])
+def test_training_run_matches_oracle(small, T):
+    import torch
+
+    wl = wlm.config(4, small=small, T=T)
+    d = wl.mlp
+    x0 = wlm.params0(wl)
+    xs, ys = wlm.mlp_batches(wl)
+    xs_d, ys_d = torch.from_numpy(xs).cuda(), torch.from_numpy(ys).cuda()
+    o = AbsSgdOracle(x0, wl.W, wl.lr, wl.momentum, wl.weight_decay)
+    ref_states = []
+    for calls in wlm.iter_calls(wl):
+        p = o.params()
+        for (i, k, c) in calls:
+            o.accumulate(i, _grad(p, xs, ys, c, wl))
+        o.sync_step()
+        ref_states.append(o.counters())
+    ref = o.params()
+    assert np.abs(ref - x0).max() > 1e-4
+    outs = {}
+    for name, kw in (("eager", dict()), ("pipelined", dict(pipelined=True)), ("gathered", dict(pipelined=True, coalesce=True)),
+                     ("overwrite-first", dict(pipelined=True, overwrite_first=True)), ("per-call", dict(pipelined=True, defer=False))):
+        got, states, consumed = _run(wl, x0, xs_d, ys_d, **kw)
+        err = np.abs(got.astype(np.float64) - ref).max()
+        assert err <= TOL * np.abs(ref).max(), f"{name}: {err:.3e}"
+        for (c1, cur1, t1), (c2, cur2, t2) in zip(states, ref_states):
+            assert np.array_equal(c1, c2) and (cur1, t1) == (cur2, t2)
+        for a, b in zip(consumed, o.consumed):
+            assert np.array_equal(a, b)
+        outs[name] = got
+    assert np.array_equal(outs["eager"], outs["pipelined"]), "eager and pipelined runs must be bit-identical"
+    assert np.array_equal(outs["overwrite-first"], outs["pipelined"]), "overwrite-first mode must give the same parameters"
+    # against the per-call path only the order of the fp32 additions differs
+    assert np.abs(outs["pipelined"] - outs["per-call"]).max() <= 1e-4 * np.abs(ref).max()
+
+
+_MIXED = [
+    [(0, "mlp", 1), (1, "vec", 1), (0, "mlp", 2), (3, "mlp", 4)],
+    [(2, "vec", 2), (2, "mlp", 3), (0, "mlp", 1), (2, "vec", 1), (2, "mlp", 1)],
+    [],
+    [(1, "mlp", 2), (1, "mlp", 2), (3, "vec", 1)],
+    [(0, "mlp", 4), (1, "mlp", 4), (2, "mlp", 4), (3, "mlp", 4)],
+]
+
+
+@pytest.mark.parametrize("overwrite_first", [False, True], ids=["clear-in-sync", "overwrite-first"])
+@pytest.mark.parametrize("pipelined", [False, True], ids=["eager", "pipelined"])
+def test_gradient_vectors_and_mlp_calls_mixed(pipelined, overwrite_first):
+    import torch
+
+    wl = wlm.config(4, small=True, T=len(_MIXED))
+    x0 = wlm.params0(wl)
+    xs, ys = wlm.mlp_batches(wl)
+    vec = np.random.default_rng(11).standard_normal((3, wl.P)).astype(np.float32) * 1e-3
+    o = AbsSgdOracle(x0, wl.W, wl.lr, wl.momentum, wl.weight_decay)
+    eng = _engine(wl, x0, pipelined=pipelined, overwrite_first=overwrite_first)
+    xs_d, ys_d = torch.from_numpy(xs).cuda(), torch.from_numpy(ys).cuda()
+    vec_d = [torch.from_numpy(vec[j]).cuda() for j in range(3)]
+    c = 0
+    for t, calls in enumerate(_MIXED + [[], []]):
+        p = o.params()
+        for (i, kind, n) in calls:
+            lo = c % (wl.mlp_pool - 4)
+            if kind == "mlp":
+                eng.accumulate_mlp_batch(i, n, xs_d[lo:lo + n], ys_d[lo:lo + n])
+                for j in range(n):
+                    o.accumulate(i, _grad(p, xs, ys, lo + j, wl))
+            else:
+                for j in range(n):
+                    eng.accumulate(i, vec_d[(c + j) % 3])
+                    o.accumulate(i, vec[(c + j) % 3])
+            c += n
+        eng.sync_step(); o.sync_step()
+        cnt, cur, tt = eng.counters()
+        assert np.array_equal(cnt, o.counters()[0]) and (cur, tt) == o.counters()[1:]
+    eng.check()
+    got = eng.params_host()
+    ref = o.params()
+    assert np.abs(ref - x0).max() > 1e-5
+    assert np.abs(got.astype(np.float64) - ref).max() <= TOL * np.abs(ref).max()
+    for s, b in enumerate(o.consumed):
+        assert np.array_equal(eng.consumed(s), b)
+    eng.destroy()
+
+
+def test_export_in_the_middle_of_an_iteration_and_resume_in_a_fresh_context():
+    import torch
+
+    wl = wlm.config(4, small=True, T=4)
+    x0 = wlm.params0(wl)
+    xs, ys = wlm.mlp_batches(wl)
+    xs_d, ys_d = torch.from_numpy(xs).cuda(), torch.from_numpy(ys).cuda()
+    its = list(wlm.iter_calls(wl))
+
+    def feed(eng, calls):
+        for (i, k, c) in calls:
+            eng.accumulate_mlp(i, xs_d[c % wl.mlp_pool], ys_d[c % wl.mlp_pool])
+
+    a = _engine(wl, x0, pipelined=True)
+    for calls in its[:2]:
+        feed(a, calls); a.sync_step()
+    half = len(its[2]) // 2
+    feed(a, its[2][:half])
+    blob = a.state_export()                      # the operands waiting in the pool are contracted into the rows first
+    b = _engine(wl, (x0 * 0.5).astype(np.float32), pipelined=True)
+    b.state_import(blob)
+    for eng in (a, b):
+        feed(eng, its[2][half:]); eng.sync_step()
+        feed(eng, its[3]); eng.sync_step(); eng.sync_step()
+        eng.check()
+    assert np.array_equal(a.params_host(), b.params_host())
+    assert np.array_equal(a.momentum().cpu().numpy(), b.momentum().cpu().numpy())
+    assert np.array_equal(a.counters()[0], b.counters()[0])
+    # and the run as a whole still follows the oracle
+    o = AbsSgdOracle(x0, wl.W, wl.lr, wl.momentum, wl.weight_decay)
+    for calls in its:
+        p = o.params()
+        for (i, k, c) in calls:
+            o.accumulate(i, _grad(p, xs, ys, c, wl))
+        o.sync_step()
+    o.sync_step()
+    assert np.abs(a.params_host().astype(np.float64) - o.params()).max() <= TOL * np.abs(o.params()).max()
+    a.destroy(); b.destroy()
