@@ -110,8 +110,15 @@ extern "C" {
                                      The row then holds the same sum as without the flag to fp32 rounding (one fp32
                                      accumulation over K = 64 b_i instead of b_i rounded additions).  Per micro-batch
                                      the accumulator traffic of 8 mlp_in mlp_hidden bytes (read + write of the slice)
-                                     becomes 4 mlp_in mlp_hidden / b_i (one write per worker and iteration).  Combines
-                                     with every other flag.                                                       */
+                                     becomes 4 mlp_in mlp_hidden / b_i (one write per worker and iteration).  When the
+                                     iteration ends with the W1 slice of every row untouched (the usual case: gradient
+                                     calls only, nothing read in between; single-GPU steps without ABS_FLAG_GRAD_NORM,
+                                     mlp_hidden a multiple of 128) not even that is written: abs_sync_step forms the
+                                     weighted average of the W1 slice as ONE contraction over all micro-batches of all
+                                     workers, (sum_j X_j^T dZ_j) / B, inside the kernel that applies the update, and
+                                     runs the row-based fused step on the bias / W2 part of the vector only (the rows'
+                                     W1 slices then stay as they are: zero, or stale with ABS_FLAG_OVERWRITE_FIRST).
+                                     Combines with every other flag.                                              */
 
 #define ABS_MAX_WORKERS 64u
 #define ABS_MAX_RANKS   16u   /* GPUs taking part in abs_global_* (n_ranks * W <= ABS_MAX_WORKERS)        */
@@ -283,6 +290,8 @@ int abs_selftest_timeout(abs_ctx *ctx);
  *                  128 = forward GEMM and ring dW1 kernel always with their deep pipelines, which take a whole
  *                  SM's shared memory (default: with W > 1, outside serial mode, their light forms of about
  *                  100 KB, so that CTAs of different workers' calls share an SM; same results bit for bit).
+ *   ABS_K_MLP_BWD  1 = with ABS_FLAG_MLP_DEFER: the fused step never works from the pooled operands; every
+ *                  iteration's dW1 is contracted into the rows first (see the flag).
  *   ABS_K_MLP_FWD  1 = serial mode: every kernel of a gradient call runs on stream_acc instead of the
  *                  worker's internal stream (for per-kernel timing).
  *   ABS_K_CHAIN    0 = consecutive kernels of a stream are chained by programmatic dependent launch: the next

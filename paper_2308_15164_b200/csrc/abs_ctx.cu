@@ -204,6 +204,13 @@ struct abs_ctx {
     std::vector<int16_t> pool_owner[2];       // worker whose micro-batch sits in the slot; -1: none (contracted, or never used)
     int pend_pool0[kMaxW] = {};               // first pool slot of a waiting group (ABS_FLAG_MLP_COALESCE)
     bool w1_touched[2][kMaxW] = {};           // the row's W1 slice has been written in the set's current iteration
+    // A set whose iteration ended with every W1 slice untouched is not contracted row by row: its fused step forms
+    // the weighted average of the W1 slice straight from the pooled operands (k_sync_w1) and runs the row-based
+    // kernel on the rest of the vector only.
+    bool fused_pending[2] = {false, false};
+    MlpSlots fused_slots[2]{};
+    int fused_n[2] = {0, 0};
+    TmapBytes tm_x[2]{}, tm_v{}, tm_shadow[2]{};   // W1 slices of the parameter buffers, the momentum and the bf16 copies
 
     // multi-GPU mode (abs_global_*): every rank's workspace as mapped in this process
     uint32_t n_ranks = 0, rank = 0;
@@ -329,6 +336,7 @@ void mlp_mark(void* user, int kernel_class, int n, cudaStream_t stream);
 int flush_all(abs_ctx* c);
 int flush_worker(abs_ctx* c, uint32_t worker);
 int settle_all(abs_ctx* c);
+int contract_pending_sets(abs_ctx* c);
 
 // stream_acc waits (on the device) for every gradient kernel enqueued so far on the worker streams (waiting
 // micro-batch groups are started and pooled dW1 operands contracted first).
@@ -379,6 +387,32 @@ int launch_fused(abs_ctx* c, uint32_t set, int in, int out, uint64_t log_step, c
     if (shape == 0 && c->mlp && c->pipelined) {
         shape = -2;
         a.tma_one_cta = 4;
+    }
+    if (c->fused_pending[set]) {
+        // W1 slice: weighted average and update straight from the set's pooled operands; the rest of the vector
+        // (b1, W2, b2) by the row-based kernel, which also logs and clears the counters.
+        float B = 0.f;
+        for (uint32_t i = 0; i < c->cfg.W; ++i) B += (float)c->h_cnt[(size_t)set * c->cfg.W + i];
+        const size_t w1 = (size_t)c->mlp_dims.d_in * c->mlp_dims.d_hidden;
+        a.x_in += w1;
+        a.x_out += w1;
+        a.v += w1;
+        a.acc += w1;
+        a.shadow += w1;
+        a.n_vec = (c->L.P_pad - w1) / 4;
+        a.plain_only = 1;
+        {
+            Timed tm(c, ABS_K_SYNC, stream);
+            CK(launch_mlp_sync_w1(c->mlp_dims, c->mlp_scratch[0], c->pool[set], c->fused_slots[set], c->fused_n[set], &c->tm_x[in],
+                                  &c->tm_x[out], &c->tm_v, &c->tm_shadow[out], B, a.lr, a.mu, a.wd, a.lambda_dc, a.disp_scale, stream,
+                                  c->chained()));
+            CK(launch_sync(a, 0, c->num_sms, stream, c->chained()));
+        }
+        c->launches += 2;
+        c->fused_pending[set] = false;
+        for (int q = 0; q < c->pool_n[set]; ++q) c->pool_owner[set][q] = -1;
+        c->pool_n[set] = 0;
+        return ABS_OK;
     }
     {
         Timed tm(c, ABS_K_SYNC, stream);
@@ -478,8 +512,7 @@ int flush_all(abs_ctx* c) {
 // ABS_FLAG_MLP_DEFER: dW1 of the worker's micro-batches waiting in the current set's operand pool, one launch
 // (K = 64 per micro-batch), stored into -- or, if the W1 slice of its row was written earlier in the iteration,
 // added to -- the accumulator row.  Runs behind the worker's front kernels, on its second stream.
-int contract_worker(abs_ctx* c, uint32_t worker) {
-    const uint32_t set = c->cur;
+int contract_worker(abs_ctx* c, uint32_t set, uint32_t worker) {
     MlpSlots sl{};
     int n = 0;
     for (int q = 0; q < c->pool_n[set]; ++q)
@@ -514,9 +547,47 @@ int contract_worker(abs_ctx* c, uint32_t worker) {
 // (ABS_FLAG_MLP_DEFER) the pooled dW1 operands contracted.
 int settle_all(abs_ctx* c) {
     if (int rc = flush_all(c)) return rc;
-    if (!c->defer) return ABS_OK;
+    if (!c->defer || c->fused_pending[c->cur]) return ABS_OK;   // (pending: the set's fused step works from the pool)
     for (uint32_t i = 0; i < c->cfg.W; ++i)
-        if (int rc = contract_worker(c, i)) return rc;
+        if (int rc = contract_worker(c, c->cur, i)) return rc;
+    return ABS_OK;
+}
+
+// A set that waits for its fused step with its W1 gradients still in pooled form (eager mode: until the next
+// abs_sync_step) is needed row by row after all: contract it.
+int contract_pending_sets(abs_ctx* c) {
+    for (uint32_t set = 0; set < 2; ++set)
+        if (c->fused_pending[set]) {
+            c->fused_pending[set] = false;
+            for (uint32_t i = 0; i < c->cfg.W; ++i)
+                if (int rc = contract_worker(c, set, i)) return rc;
+            c->pool_n[set] = 0;
+        }
+    return ABS_OK;
+}
+
+// End of the current set's iteration: its waiting groups are started, and its pooled dW1 operands are either left
+// for the fused step (every W1 slice of the set untouched: the step then works from the operands, see
+// fused_pending) or contracted into the rows.
+int close_iteration(abs_ctx* c) {
+    if (int rc = flush_all(c)) return rc;
+    if (!c->defer) return ABS_OK;
+    const uint32_t set = c->cur;
+    bool fuse = c->n_ranks == 0 && !c->grad_norm() && c->mlp_dims.d_hidden % 128 == 0 && c->ctas_per_sm[ABS_K_MLP_BWD] != 1;
+    for (uint32_t i = 0; i < c->cfg.W && fuse; ++i) fuse = !c->w1_touched[set][i];
+    int n = 0;
+    if (fuse) {
+        for (int q = 0; q < c->pool_n[set]; ++q)
+            if (c->pool_owner[set][q] >= 0) c->fused_slots[set].s[n++] = (uint16_t)q;
+        fuse = n > 0;
+    }
+    if (!fuse) {
+        if (int rc = settle_all(c)) return rc;
+        c->pool_n[set] = 0;
+        return ABS_OK;
+    }
+    c->fused_pending[set] = true;
+    c->fused_n[set] = n;
     return ABS_OK;
 }
 
@@ -538,9 +609,10 @@ int take_pool_slots(abs_ctx* c, int n, int* slot0) {
     return ABS_OK;
 }
 
-// The iteration of set `closing` has ended (its gradients are settled); `opening` starts a new one.
+// The iteration of set `closing` has ended (its gradients are settled); `opening` starts a new one (its pool is
+// empty: what it held was contracted, or consumed by its fused step, before the set could become current again).
 void turn_sets(abs_ctx* c, uint32_t closing, uint32_t opening) {
-    c->pool_n[closing] = 0;
+    (void)closing;
     for (uint32_t i = 0; i < c->cfg.W; ++i) c->w1_touched[opening][i] = false;
 }
 
@@ -665,6 +737,10 @@ int abs_init(abs_ctx** out, const abs_config* cfg, void* workspace_dev, size_t w
                 if ((e = mlp_pool_init(&c->pool[k], c->mlp_dims, L.pool_cap, c->ws + L.off_pool[k])) != cudaSuccess)
                     return bail(e, "cuTensorMapEncodeTiled(operand pool)");
                 c->pool_owner[k].assign((size_t)L.pool_cap, (int16_t)-1);
+                if ((e = mlp_make_acc_tmap(&c->tm_x[k], c->mlp_dims, c->x(k))) != cudaSuccess ||
+                    (e = mlp_make_shadow_tmap(&c->tm_shadow[k], c->mlp_dims, c->shadow(k))) != cudaSuccess ||
+                    (e = mlp_make_acc_tmap(&c->tm_v, c->mlp_dims, c->v())) != cudaSuccess)
+                    return bail(e, "cuTensorMapEncodeTiled(parameters)");
             }
         if ((e = cudaEventCreateWithFlags(&c->ev_fork, cudaEventDisableTiming)) != cudaSuccess) return bail(e, "cudaEventCreate");
         c->n_wstreams = (int)std::min<uint32_t>(cfg->W, kMlpStreams);
@@ -811,7 +887,7 @@ int abs_accumulate_mlp(abs_ctx* c, uint32_t worker, const void* x_dev, const int
 int abs_sync_step(abs_ctx* c) {
     if (!live(c)) return ABS_ESTATE;
     if (c->n_ranks != 0) return invalid(c, "context is in multi-GPU mode: end iterations with abs_global_begin / _step / _end");
-    if (int rc = settle_all(c)) return rc;   // every gradient of iteration t is under way before the iteration ends
+    if (int rc = close_iteration(c)) return rc;   // every gradient of iteration t is under way before the iteration ends
     const uint32_t W = c->cfg.W;
     const uint32_t d = c->cur ^ 1;   // the delayed set (filled during iteration t-1)
     if (!c->pipelined) {
@@ -923,6 +999,7 @@ int abs_global_begin(abs_ctx* c, int32_t** counts_dev, uint32_t* n_counts) {
     if (c->global_phase != 0) return invalid(c, "abs_global_begin / _step / _end must be called in that order");
     if (!counts_dev || !n_counts) return invalid(c, "output pointer is NULL");
     if (int rc = settle_all(c)) return rc;
+    c->pool_n[c->cur] = 0;
     const uint32_t W = c->cfg.W;
     // Publish x_{t+1}: the kernels launched one call ago, on every rank, have all finished (ev_sync_done was
     // recorded behind the caller's closing barrier).
@@ -1077,6 +1154,7 @@ int abs_momentum(abs_ctx* c, const float** v_dev_out) {
 int abs_accumulator(abs_ctx* c, uint32_t set, uint32_t worker, const float** acc_dev_out) {
     if (!live(c)) return ABS_ESTATE;
     if (set > 1 || worker >= c->cfg.W || !acc_dev_out) return invalid(c, "bad set / worker / output pointer");
+    if (int rc = contract_pending_sets(c)) return rc;
     if (int rc = join_workers(c)) return rc;
     *acc_dev_out = c->acc(set, worker);
     return ABS_OK;
@@ -1209,6 +1287,7 @@ bool same_config(const abs_config& a, const abs_config& b) {
 
 // Everything enqueued so far has finished (waiting micro-batch groups are started first).
 int drain(abs_ctx* c) {
+    if (int rc = contract_pending_sets(c)) return rc;
     if (int rc = settle_all(c)) return rc;
     if (c->pipelined) CK(cudaStreamSynchronize(c->s_sync));
     for (int k = 0; k < c->n_wstreams; ++k) {
@@ -1284,6 +1363,7 @@ int abs_state_import(abs_ctx* c, const void* src_host, size_t bytes) {
     for (size_t k = 0; k < c->h_cnt.size(); ++k) c->h_cnt[k] = h.h_cnt[k];
     for (uint32_t set = 0; set < 2; ++set) {   // a row that has received gradients may hold some in its W1 slice
         c->pool_n[set] = 0;
+        c->fused_pending[set] = false;
         for (uint32_t i = 0; i < c->cfg.W; ++i) c->w1_touched[set][i] = c->h_cnt[(size_t)set * c->cfg.W + i] > 0;
     }
     if (c->mlp) {   // the bf16 copies are a function of the parameters: rebuild them

@@ -179,6 +179,15 @@ cudaError_t mlp_scratch_init(MlpScratch* s, const MlpDims& d, void* base, __nv_b
                              __nv_bfloat16* shadow1, const char** err);
 // TMA descriptor of the W1 slice of one worker's accumulator row (fp32 [d_in][d_hidden]).
 cudaError_t mlp_make_acc_tmap(void* tmap_out, const MlpDims& d, float* acc_row);
+// W1 slice of a bf16 copy of the parameters, as a TMA descriptor (boxes of 128 rows x 64 columns).
+cudaError_t mlp_make_shadow_tmap(void* tmap_out, const MlpDims& d, __nv_bfloat16* shadow);
+// Step 1 + update of the W1 slice straight from the pooled operands of the set's nb micro-batches (slots): the
+// weighted average is (sum_j X_j^T dZ_j) / B.  tm_*: descriptors from mlp_make_acc_tmap (x_in, x_out, v: fp32 vectors)
+// and mlp_make_shadow_tmap (bf16 copy of x_out, or nullptr).  Needs d_hidden % 128 == 0.
+cudaError_t launch_mlp_sync_w1(const MlpDims& d, const MlpScratch& s, const MlpPool& pool, const MlpSlots& slots, int nb,
+                               const void* tm_x_in, const void* tm_x_out, const void* tm_v, const void* tm_shadow,
+                               float B, float lr, float mu, float wd, float lambda_dc, float disp_scale, cudaStream_t stream,
+                               bool chained);
 // The gradient of a call is enqueued in three parts so that the caller can put them on different streams:
 //   cast:  the only part that reads the caller's x_dev / y_dev (bf16 copies and labels into this scratch set);
 //   front: forward GEMM, loss, layer-2 backward (writes dzt of this scratch set; adds db2, db1, dW2 into

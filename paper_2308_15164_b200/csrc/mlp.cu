@@ -384,6 +384,15 @@ __device__ __forceinline__ void tmem_ld_32(uint32_t taddr, uint32_t (&v)[32]) {
         : "r"(taddr) : "memory");
     asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
 }
+// 16 consecutive fp32 columns of this thread's TMEM lane.
+__device__ __forceinline__ void tmem_ld_16(uint32_t taddr, uint32_t (&v)[16]) {
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
+        : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]), "=r"(v[8]),
+          "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15])
+        : "r"(taddr) : "memory");
+    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+}
 // Adds the 32 TMEM values of one row into that row of a swizzled [128][32] fp32 panel in shared
 // memory (row = 128 bytes; 16-byte chunk j sits at position j ^ (row % 8), as the TMA box wrote it).
 template <bool kAdd>
@@ -720,6 +729,229 @@ __global__ void __launch_bounds__(192) k_dw1_ring(const __grid_constant__ CUtens
 }
 
 // ============================================================================================
+// Step 1 + update for the W1 slice straight from the pooled dW1 operands (ABS_FLAG_MLP_DEFER).
+// When no accumulator row's W1 slice was written during the iteration, sum_i G_t^i restricted to W1 is
+// sum over ALL micro-batches of the iteration of X_j^T dZ_j: one contraction with K = 64 B, whose tiles feed
+// the update directly -- the slices are never written, read or cleared:
+//     g = (sum_j X_j^T dZ_j) * (1 / B);  Eq. 6;  + wd x;  v = mu v + g;  x' = x - lr v;  bf16(x') -> shadow
+// Same roles as k_dw1_ring with 128 x 128 tiles (warp 0: operand TMA producer, warp 1: MMA issuer, two TMEM
+// accumulators).  The eight epilogue warps take a finished tile in four panels of 32 columns: the x and v
+// panels ([128][32] fp32, swizzled rows) arrive by TMA in a ring of kStepE stages whose loads the epilogue's own
+// leader thread issues two panels ahead (self-paced: the operand producer never waits for the epilogue and
+// cannot be what the epilogue waits for); each thread updates its row in place, the bf16 copy goes into a
+// [128][64] panel shared by two steps, and the leader sends everything back with TMA stores.
+// HBM traffic: 18 bytes per W1 element (x, v read; x', v, bf16 x' written) + the operands once (they stay in
+// L2 between tiles), against (8 W_act + 18) for the row-based step plus 4 W_act for the contractions.
+// ============================================================================================
+constexpr int kStepN = 128;      // tile width
+constexpr int kStepOps = 3;      // operand slots of 32 KB
+constexpr int kStepE = 3;        // epilogue stages: [x panel 16 KB | v panel 16 KB]
+constexpr int kStepEpiThreads = 256;   // eight epilogue warps: two per TMEM lane quarter, 16 columns of a panel each
+constexpr int kStepSlotBytes = kTileM * 128 + kStepN * 128;
+constexpr int kPanelBytes = kTileM * 32 * 4;
+
+struct StepSmem {
+    alignas(1024) uint8_t op[kStepOps][kStepSlotBytes];
+    alignas(1024) uint8_t ep[kStepE][2 * kPanelBytes];
+    alignas(1024) uint8_t sh[2][kTileM * 128];          // bf16 copy, [128 rows][64 columns], swizzled 128-byte rows
+    alignas(8) uint64_t op_full[kStepOps];
+    uint64_t op_empty[kStepOps];
+    uint64_t acc_full[2];
+    uint64_t acc_empty[2];
+    uint64_t ep_full[kStepE];
+    uint32_t tmem_base;
+    uint32_t failed;
+    uint32_t stop[2];
+};
+
+struct W1StepCoef {
+    float inv_B;         // 1 / B, B = sum_i b_i of the set
+    float lr, mu, wd, lambda_dc, disp_scale;
+};
+
+__global__ void __launch_bounds__(64 + kStepEpiThreads) k_sync_w1(const __grid_constant__ CUtensorMap tm_xt,
+                                                 const __grid_constant__ CUtensorMap tm_dzt,
+                                                 const __grid_constant__ CUtensorMap tm_x_in,
+                                                 const __grid_constant__ CUtensorMap tm_x_out,
+                                                 const __grid_constant__ CUtensorMap tm_v,
+                                                 const __grid_constant__ CUtensorMap tm_shadow,
+                                                 const __grid_constant__ MlpSlots sl, int n_tiles_n, int n_tiles, int d_in,
+                                                 int ld, int nb, W1StepCoef cf, int has_shadow, int* status) {
+    extern __shared__ uint8_t smem_raw[];
+    StepSmem& s = *reinterpret_cast<StepSmem*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+    const int warp = threadIdx.x / 32, lane = threadIdx.x % 32;
+    const int my_tiles = (n_tiles - (int)blockIdx.x + (int)gridDim.x - 1) / (int)gridDim.x;
+    const int my_panels = my_tiles * 4;
+
+    if (warp == 1) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&s.tmem_base)), "r"(2 * kStepN) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    if (threadIdx.x == 0) {
+        for (int i = 0; i < kStepOps; ++i) {
+            mbar_init(&s.op_full[i], 1);
+            mbar_init(&s.op_empty[i], 1);
+        }
+        for (int i = 0; i < 2; ++i) {
+            mbar_init(&s.acc_full[i], 1);
+            mbar_init(&s.acc_empty[i], kStepEpiThreads);
+        }
+        for (int i = 0; i < kStepE; ++i) mbar_init(&s.ep_full[i], 1);
+        s.failed = 0;
+        s.stop[0] = s.stop[1] = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    const uint32_t tmem = s.tmem_base;
+    pdl_wait();      // the operands come from the gradient kernels, x and v from the previous step
+    pdl_trigger();
+
+    if (warp == 0) {
+        if (lane == 0) {                             // ---- operand producer
+            int q = 0;
+            for (int i = 0; i < my_tiles && !s.failed; ++i) {
+                const int t = (int)blockIdx.x + i * (int)gridDim.x;
+                const int n0 = (t % n_tiles_n) * kStepN, m0 = (t / n_tiles_n) * kTileM;
+                for (int j = 0; j < nb; ++j, ++q) {
+                    const int st = q % kStepOps;
+                    if (q >= kStepOps && !mbar_wait(&s.op_empty[st], ((q / kStepOps) - 1) & 1)) { s.failed = 1; break; }
+                    mbar_expect_tx(&s.op_full[st], kStepSlotBytes);
+                    const int slot = (int)sl.s[j];
+                    tma_load_2d(s.op[st], &tm_xt, 0, slot * d_in + m0, &s.op_full[st]);
+                    tma_load_2d(s.op[st] + kTileM * 128, &tm_dzt, 0, slot * ld + n0, &s.op_full[st]);
+                    tma_load_2d(s.op[st] + kTileM * 128 + kDwN * 128, &tm_dzt, 0, slot * ld + n0 + kDwN, &s.op_full[st]);
+                }
+            }
+        }
+    } else if (warp == 1) {
+        if (lane == 0) {                             // ---- MMA issuer
+            constexpr uint32_t idesc = umma_idesc_bf16(kTileM, kStepN);
+            int q = 0;
+            bool ok = true;
+            for (int i = 0; i < my_tiles && ok; ++i) {
+                const int ab = i & 1;
+                if (i >= 2 && !mbar_wait(&s.acc_empty[ab], ((i / 2) - 1) & 1)) { ok = false; break; }
+                for (int j = 0; j < nb; ++j, ++q) {
+                    const int st = q % kStepOps;
+                    if (!mbar_wait(&s.op_full[st], (q / kStepOps) & 1)) { ok = false; break; }
+                    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                    const uint32_t a0 = smem_u32(s.op[st]);
+                    const uint64_t da = umma_desc_k_sw128(a0), db = umma_desc_k_sw128(a0 + kTileM * 128);
+#pragma unroll
+                    for (int k = 0; k < kMB / 16; ++k) umma_bf16(tmem + ab * kStepN, da + 2 * k, db + 2 * k, idesc, (j > 0 || k > 0));
+                    umma_commit(&s.op_empty[st]);
+                }
+                if (ok) umma_commit(&s.acc_full[ab]);
+            }
+            if (!ok) s.failed = 1;
+        }
+    } else {                                         // ---- epilogue warps 2..9
+        // A warp may read the TMEM lanes of its quarter (warp % 4) only; warps 2-5 take columns 0..15 of a panel,
+        // warps 6-9 columns 16..31, so every scheduler of the SM has two warps to issue from.
+        const int qd = warp % 4, half = (warp - 2) / 4;
+        const int row = qd * 32 + lane;
+        const int sw = row & 7;
+        const bool leader = (threadIdx.x == 64);
+        auto panel_coords = [&](int e, int* col, int* m0) {
+            const int t = (int)blockIdx.x + (e >> 2) * (int)gridDim.x;
+            *col = (t % n_tiles_n) * kStepN + (e & 3) * 32;
+            *m0 = (t / n_tiles_n) * kTileM;
+        };
+        auto load_panels = [&](int e) {              // leader only: x and v panels of step e into stage e % kStepE
+            int col, m0;
+            panel_coords(e, &col, &m0);
+            const int st = e % kStepE;
+            mbar_expect_tx(&s.ep_full[st], 2 * kPanelBytes);
+            tma_load_2d(s.ep[st], &tm_x_in, col, m0, &s.ep_full[st]);
+            tma_load_2d(s.ep[st] + kPanelBytes, &tm_v, col, m0, &s.ep_full[st]);
+        };
+        if (leader)
+            for (int e = 0; e < kStepE - 1 && e < my_panels; ++e) load_panels(e);
+        const float c_dc = -cf.lambda_dc * cf.disp_scale;
+        bool stopped = false;
+        for (int e = 0; e < my_panels && !stopped; ++e) {
+            const int i = e >> 2, p = e & 3, ab = i & 1, st = e % kStepE;
+            bool ok = true;
+            if (p == 0) ok = mbar_wait(&s.acc_full[ab], (i / 2) & 1);
+            ok = mbar_wait(&s.ep_full[st], (e / kStepE) & 1) && ok;
+            ok = __all_sync(0xffffffffu, ok);
+            if (!ok) s.failed = 1;
+            if (ok) {
+                uint32_t acc[16];
+                asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                tmem_ld_16(tmem + ((uint32_t)(qd * 32) << 16) + (uint32_t)(ab * kStepN + p * 32 + half * 16), acc);
+                if (p == 3) {                        // the accumulator is in registers: the tile after next may use it
+                    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+                    mbar_arrive(&s.acc_empty[ab]);
+                }
+                float4* xrow = reinterpret_cast<float4*>(s.ep[st]) + row * 8;
+                float4* vrow = reinterpret_cast<float4*>(s.ep[st] + kPanelBytes) + row * 8;
+                uint8_t* shrow = s.sh[(e >> 1) & 1] + row * 128;
+                float4 x[4], v[4];
+#pragma unroll
+                for (int jj = 0; jj < 4; ++jj) {
+                    const int j = half * 4 + jj;     // 16-byte chunk of the panel row
+                    x[jj] = xrow[j ^ sw];
+                    v[jj] = vrow[j ^ sw];
+                }
+#pragma unroll
+                for (int jj = 0; jj < 4; ++jj) {
+                    const int j = half * 4 + jj;
+                    float gx = __uint_as_float(acc[4 * jj]) * cf.inv_B, gy = __uint_as_float(acc[4 * jj + 1]) * cf.inv_B;
+                    float gz = __uint_as_float(acc[4 * jj + 2]) * cf.inv_B, gw = __uint_as_float(acc[4 * jj + 3]) * cf.inv_B;
+                    if (cf.lambda_dc != 0.0f) {      // Eq. 6 with x_t - x_{t-1} = -disp_scale * v
+                        gx += c_dc * gx * gx * v[jj].x; gy += c_dc * gy * gy * v[jj].y;
+                        gz += c_dc * gz * gz * v[jj].z; gw += c_dc * gw * gw * v[jj].w;
+                    }
+                    gx += cf.wd * x[jj].x; gy += cf.wd * x[jj].y; gz += cf.wd * x[jj].z; gw += cf.wd * x[jj].w;
+                    v[jj].x = cf.mu * v[jj].x + gx; v[jj].y = cf.mu * v[jj].y + gy;
+                    v[jj].z = cf.mu * v[jj].z + gz; v[jj].w = cf.mu * v[jj].w + gw;
+                    x[jj].x -= cf.lr * v[jj].x; x[jj].y -= cf.lr * v[jj].y; x[jj].z -= cf.lr * v[jj].z; x[jj].w -= cf.lr * v[jj].w;
+                    xrow[j ^ sw] = x[jj];
+                    vrow[j ^ sw] = v[jj];
+                    // columns 4j..4j+3 of panel p = bf16 elements (p & 1) * 32 + 4j.. of the 64-column copy row
+                    uint2 pk;
+                    pk.x = pack_bf16x2(x[jj].x, x[jj].y);
+                    pk.y = pack_bf16x2(x[jj].z, x[jj].w);
+                    const int chunk = (p & 1) * 4 + (j >> 1);
+                    *reinterpret_cast<uint2*>(shrow + ((chunk ^ sw) << 4) + ((j & 1) << 3)) = pk;
+                }
+            }
+            if (leader) s.stop[e & 1] = *reinterpret_cast<volatile uint32_t*>(&s.failed);
+            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // smem writes -> visible to the TMA engine
+            asm volatile("bar.sync 1, %0;" ::"n"(kStepEpiThreads) : "memory");
+            if (*reinterpret_cast<volatile uint32_t*>(&s.stop[e & 1])) { stopped = true; break; }
+            if (leader) {
+                int col, m0;
+                panel_coords(e, &col, &m0);
+                tma_store_2d(&tm_x_out, s.ep[st], col, m0);
+                tma_store_2d(&tm_v, s.ep[st] + kPanelBytes, col, m0);
+                if ((p & 1) && has_shadow) tma_store_2d(&tm_shadow, s.sh[(e >> 1) & 1], col - 32, m0);
+                asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+                // the stores of step e-1 have read their stage: it takes the panels of step e + kStepE - 1
+                asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory");
+                if (e + kStepE - 1 < my_panels) load_panels(e + kStepE - 1);
+            }
+        }
+        if (leader) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
+    }
+    __syncwarp();
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    if (threadIdx.x == 0 && s.failed) {
+        atomicExch(status, ABS_ETIMEOUT);
+        for (int i = 0; i < kStepOps; ++i) mbar_wait(&s.op_full[i], 0);   // bounded chance for copies in flight to land
+        for (int i = 0; i < kStepE; ++i) mbar_wait(&s.ep_full[i], 0);
+    }
+    __syncthreads();
+    if (warp == 1) {
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(2 * kStepN) : "memory");
+    }
+}
+
+// ============================================================================================
 // Forward GEMM on tcgen05:  zpart[s][h][r] = sum_{k in split s} W1b[k][h] * xb[r][k]
 //   D [M = 128 hidden][N = 64 samples] += A B^T with
 //   A = W1b^T tile: stored [k][h] with h contiguous, i.e. an MN-major operand.  A TMA box of
@@ -1005,6 +1237,39 @@ cudaError_t mlp_pool_init(MlpPool* p, const MlpDims& d, int cap, void* base) {
                    (uint64_t)cap * d.d_hidden, kMB, kDwN, kMB))
         return cudaErrorInvalidValue;
     return cudaSuccess;
+}
+
+cudaError_t mlp_make_shadow_tmap(void* tmap_out, const MlpDims& d, __nv_bfloat16* shadow) {
+    // W1 slice of a bf16 copy of the parameters: [d_in][d_hidden] bf16, boxes of 128 rows x 64 columns
+    return encode_2d(reinterpret_cast<CUtensorMap*>(tmap_out), CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, shadow, d.d_in, d.d_hidden,
+                     kTileM, 64)
+               ? cudaSuccess
+               : cudaErrorInvalidValue;
+}
+
+cudaError_t launch_mlp_sync_w1(const MlpDims& d, const MlpScratch& s, const MlpPool& pool, const MlpSlots& slots, int nb,
+                               const void* tm_x_in, const void* tm_x_out, const void* tm_v, const void* tm_shadow,
+                               float B, float lr, float mu, float wd, float lambda_dc, float disp_scale, cudaStream_t stream,
+                               bool chained) {
+    if (nb < 1 || nb > kMlpMaxSlots || d.d_hidden % kStepN != 0) return cudaErrorInvalidValue;
+    static bool opted_in[64] = {};
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    if (dev < 0 || dev >= 64 || !opted_in[dev]) {
+        e = cudaFuncSetAttribute(k_sync_w1, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(StepSmem) + 1024);
+        if (e != cudaSuccess) return e;
+        if (dev >= 0 && dev < 64) opted_in[dev] = true;
+    }
+    const int n_tiles_n = d.d_hidden / kStepN, n_tiles = n_tiles_n * (d.d_in / kTileM);
+    const int ctas = n_tiles < s.num_sms ? n_tiles : s.num_sms;
+    const W1StepCoef cf{1.0f / B, lr, mu, wd, lambda_dc, disp_scale};
+    const CUtensorMap& shadow_map = *reinterpret_cast<const CUtensorMap*>(tm_shadow ? tm_shadow : tm_x_out);
+    return launch_kernel(k_sync_w1, ctas, 64 + kStepEpiThreads, sizeof(StepSmem) + 1024, stream, chained,
+                         *reinterpret_cast<const CUtensorMap*>(&pool.tmap_xt), *reinterpret_cast<const CUtensorMap*>(&pool.tmap_dzt),
+                         *reinterpret_cast<const CUtensorMap*>(tm_x_in), *reinterpret_cast<const CUtensorMap*>(tm_x_out),
+                         *reinterpret_cast<const CUtensorMap*>(tm_v), shadow_map, slots, n_tiles_n, n_tiles, d.d_in, d.d_hidden, nb,
+                         cf, tm_shadow ? 1 : 0, s.status);
 }
 
 cudaError_t mlp_make_acc_tmap(void* tmap_out, const MlpDims& d, float* acc_row) {

@@ -10,7 +10,10 @@ instead of once per call.  Checked against the CPU oracle, through the C ABI, at
   * whole training runs -- eager, pipelined, with gathered calls, in overwrite-first mode -- against the oracle run,
     eager and pipelined bit-identical;
   * gradient vectors (abs_accumulate) and MLP calls mixed within an iteration, idle workers;
-  * export / import in the middle of an iteration."""
+  * export / import in the middle of an iteration;
+  * the two forms of the deferred step -- W1 slice updated straight from the pooled operands (one contraction over
+    all micro-batches inside the update kernel) or from the rows (per-worker contractions first) -- against each
+    other after the same iterations, with and without Eq. 6."""
 
 import numpy as np
 import pytest
@@ -122,8 +125,12 @@ def test_more_microbatches_than_the_pool_holds(calls):
     eng.destroy()
 
 
-def _run(wl, x0, xs_d, ys_d, **kw):
+def _run(wl, x0, xs_d, ys_d, rows_only=False, **kw):
+    from paper_2308_15164_b200 import binding as B
+
     eng = _engine(wl, x0, **kw)
+    if rows_only:                                    # the fused step never works from the pooled operands
+        eng.set_launch(B.K_MLP_BWD, 1)
     states = []
     for t, calls in enumerate(wlm.iter_calls(wl)):
         for (i, k, c) in calls:
@@ -158,7 +165,8 @@ def test_training_run_matches_oracle(small, T):
     assert np.abs(ref - x0).max() > 1e-4
     outs = {}
     for name, kw in (("eager", dict()), ("pipelined", dict(pipelined=True)), ("gathered", dict(pipelined=True, coalesce=True)),
-                     ("overwrite-first", dict(pipelined=True, overwrite_first=True)), ("per-call", dict(pipelined=True, defer=False))):
+                     ("overwrite-first", dict(pipelined=True, overwrite_first=True)), ("per-call", dict(pipelined=True, defer=False)),
+                     ("rows-only", dict(pipelined=True, rows_only=True)), ("rows-only-eager", dict(rows_only=True))):
         got, states, consumed = _run(wl, x0, xs_d, ys_d, **kw)
         err = np.abs(got.astype(np.float64) - ref).max()
         assert err <= TOL * np.abs(ref).max(), f"{name}: {err:.3e}"
@@ -169,8 +177,51 @@ def test_training_run_matches_oracle(small, T):
         outs[name] = got
     assert np.array_equal(outs["eager"], outs["pipelined"]), "eager and pipelined runs must be bit-identical"
     assert np.array_equal(outs["overwrite-first"], outs["pipelined"]), "overwrite-first mode must give the same parameters"
-    # against the per-call path only the order of the fp32 additions differs
+    assert np.array_equal(outs["rows-only"], outs["rows-only-eager"])
+    # against the per-call path, and between the two forms of the deferred step, only the order of the fp32 additions
+    # differs (and 1 / B is multiplied by instead of divided by)
     assert np.abs(outs["pipelined"] - outs["per-call"]).max() <= 1e-4 * np.abs(ref).max()
+    assert np.abs(outs["rows-only"] - outs["per-call"]).max() <= 1e-4 * np.abs(ref).max()
+
+
+@pytest.mark.parametrize("lambda_dc", [0.0, 0.3], ids=["plain", "eq6"])
+@pytest.mark.parametrize("small", [True, False], ids=["384x512", "3072x4096"])
+def test_one_step_from_the_pooled_operands_against_the_step_from_the_rows(small, lambda_dc):
+    """The same three iterations with the W1 slice updated straight from the pooled operands (one contraction over all
+    micro-batches, inside the update kernel) and from the rows (per-worker contractions, then the row-based fused
+    step): parameters, momentum and the next iteration's gradients (which read the bf16 copy of the new weights)
+    agree to fp32 rounding, element by element."""
+    import torch
+
+    from paper_2308_15164_b200 import binding as B
+
+    wl = wlm.config(4, small=small, T=3)
+    d = wl.mlp
+    x0 = wlm.params0(wl)
+    xs, ys = wlm.mlp_batches(wl)
+    xs_d, ys_d = torch.from_numpy(xs).cuda(), torch.from_numpy(ys).cuda()
+    res = []
+    for rows_only in (False, True):
+        eng = B.AbsSgd(torch.from_numpy(x0).cuda(), wl.W, wl.lr, wl.momentum, 1e-3, lambda_dc, pipelined=True,
+                       mlp=(d.d_in, d.d_hidden, d.d_out, d.mb), mlp_defer=True)
+        if rows_only:
+            eng.set_launch(B.K_MLP_BWD, 1)
+        for t, calls in enumerate(wlm.iter_calls(wl)):
+            for (i, k, c) in calls:
+                eng.accumulate_mlp(i, xs_d[c % wl.mlp_pool], ys_d[c % wl.mlp_pool])
+            eng.sync_step()
+        eng.sync_step()
+        eng.wait(); eng.synchronize(); eng.check()
+        x, v = eng.params_host().copy(), eng.momentum().cpu().numpy().copy()
+        eng.accumulate_mlp(1, xs_d[5], ys_d[5])      # a gradient at the new parameters: reads their bf16 copy
+        g = eng.accumulator(eng.counters()[1], 1).cpu().numpy().copy()
+        res.append((x, v, g))
+        eng.destroy()
+    (xa, va, ga), (xb, vb, gb) = res
+    assert np.abs(xa - x0).max() > 1e-4
+    assert np.abs(xa - xb).max() <= 2e-6 * np.abs(xb).max()
+    assert np.abs(va - vb).max() <= 2e-5 * np.abs(vb).max()
+    assert np.abs(ga - gb).max() <= TOL * np.abs(gb).max()
 
 
 _MIXED = [
