@@ -748,27 +748,31 @@ def run_tiny(B, wlm, dev, iters=2000):
     return out
 
 
-def mlp_run_bytes(sched, d, P, max_batch, overwrite_first, defer=False):
+def mlp_run_bytes(sched, d, P, max_batch, overwrite_first, defer=None):
     """Algorithmic HBM bytes of an MLP run over the schedule `sched` [T, W] when every worker hands over its b_i
     micro-batches in calls of up to `max_batch`: per call the bf16 weights are streamed once (2 bytes per W1
     element) and the W1 slice of the accumulator is written (4 bytes per element: the worker's first call of the
     iteration stores) or read and written (8: later calls add); per micro-batch the bf16 operands of dW1; per
     iteration the fused step, (8 W_act + 16 + 2) bytes per parameter (the 2: the bf16 copy of the new weights;
-    4 W_act + 18 when the step does not write zeros).  defer (ABS_FLAG_MLP_DEFER): the slice is written once per active
-    worker and iteration (4 bytes per element), never read by a gradient call, and the operands are written by the
-    call and read by that one contraction.  Returns (bytes, calls, stored calls, micro-batches)."""
+    4 W_act + 18 when the step does not write zeros).
+    defer = "rows" (ABS_FLAG_MLP_DEFER with the rows written): the slice is written once per active worker and
+    iteration (4 bytes per element), never read by a gradient call, and the operands are written by the call and read
+    by that one contraction.  defer = "pool" (Step 1 from the pooled operands): no accumulator traffic for W1 at all;
+    the step moves 18 bytes per W1 element and the row-based amount on the rest of the vector.
+    Returns (bytes, calls, stored calls, micro-batches)."""
     w1 = d.d_in * d.d_hidden
     total = calls = stored = mbs = 0
     prev_active = 0
     for b_row in sched:
         if prev_active:
-            total += ((4 if overwrite_first else 8) * prev_active + 18) * P
+            row_based = ((4 if overwrite_first else 8) * prev_active + 18)
+            total += 18 * w1 + row_based * (P - w1) if defer == "pool" else row_based * P
         for b in b_row:
             left, first = int(b), True
             while left > 0:
                 n = min(max_batch, left)
                 if defer:
-                    total += 2 * w1 + (4 * w1 if first else 0) + 2 * n * 2 * d.mb * (d.d_in + d.d_hidden)
+                    total += 2 * w1 + (4 * w1 if first and defer == "rows" else 0) + 2 * n * 2 * d.mb * (d.d_in + d.d_hidden)
                 else:
                     total += 2 * w1 + (4 if first else 8) * w1 + n * 2 * d.mb * (d.d_in + d.d_hidden)
                 calls += 1; stored += 1 if first else 0; mbs += n
@@ -802,11 +806,13 @@ def run_mlp(B, wlm, dev, peaks, iters=12):
     out = {"workload": "cfg4 mlp 3072-4096-10, mb=64, W=4, b_i~U{1..8}, pipelined", "iterations": iters,
            "dw1_flop_per_microbatch": flop}
 
-    def run_case(max_batch, variant=0, coalesce=False, overwrite_first=False, serial=0, defer=False):
+    def run_case(max_batch, variant=0, coalesce=False, overwrite_first=False, serial=0, defer=None):
         eng = B.AbsSgd(x0_d, wl.W, wl.lr, wl.momentum, wl.weight_decay, pipelined=True, mlp=(d.d_in, d.d_hidden, d.d_out, d.mb),
-                       mlp_coalesce=coalesce, overwrite_first=overwrite_first, mlp_defer=defer)
+                       mlp_coalesce=coalesce, overwrite_first=overwrite_first, mlp_defer=defer is not None)
         eng.set_launch(B.K_MLP_DW1, variant)
         eng.set_launch(B.K_MLP_FWD, serial)
+        if defer == "rows":
+            eng.set_launch(B.K_MLP_BWD, 1)
 
         def run(profile):
             eng.profile(profile)
@@ -865,11 +871,14 @@ def run_mlp(B, wlm, dev, peaks, iters=12):
                      ("batch_calls_up_to_4", dict(max_batch=4)),
                      ("batch_calls_up_to_4_overwrite_first", dict(max_batch=4, overwrite_first=True)),
                      ("batch_calls_up_to_4_deep_pipelines", dict(max_batch=4, variant=128)),
-                     # ABS_FLAG_MLP_DEFER: one dW1 contraction per worker and iteration (K = 64 b_i)
-                     ("deferred_single_calls", dict(max_batch=1, defer=True)),
-                     ("deferred_single_calls_gathered_by_the_library", dict(max_batch=1, coalesce=True, defer=True)),
-                     ("deferred_batch_calls_up_to_4", dict(max_batch=4, defer=True)),
-                     ("deferred_batch_calls_up_to_4_overwrite_first", dict(max_batch=4, defer=True, overwrite_first=True))):
+                     # ABS_FLAG_MLP_DEFER: Step 1 of the W1 slice straight from the pooled dW1 operands (one contraction
+                     # over all micro-batches of the iteration inside the update kernel) ...
+                     ("deferred_single_calls", dict(max_batch=1, defer="pool")),
+                     ("deferred_single_calls_gathered_by_the_library", dict(max_batch=1, coalesce=True, defer="pool")),
+                     ("deferred_batch_calls_up_to_4", dict(max_batch=4, defer="pool")),
+                     # ... or one dW1 contraction per worker and iteration into the rows (K = 64 b_i), then the row-based step
+                     ("deferred_rows_single_calls", dict(max_batch=1, defer="rows")),
+                     ("deferred_rows_batch_calls_up_to_4", dict(max_batch=4, defer="rows"))):
         out[name] = run_case(**kw)
     for name, kw in (("single_calls", dict(max_batch=1)), ("single_calls_ring_dw1", dict(max_batch=1, variant=4)),
                      ("batch_calls_up_to_4", dict(max_batch=4)), ("batch_calls_up_to_4_tile_per_cta_dw1", dict(max_batch=4, variant=8))):

@@ -96,29 +96,30 @@ extern "C" {
 #define ABS_FLAG_MLP_X_BF16 64u   /* with ABS_FLAG_MLP: abs_accumulate_mlp* take x_dev as bf16 values ([mlp_mb, mlp_in] row-major,
                                      2 bytes each) instead of fp32; they enter the GEMMs as they are (no rounding step) */
 
-#define ABS_FLAG_MLP_DEFER 128u   /* with ABS_FLAG_MLP: the layer-1 weight gradient is formed once per worker and iteration
-                                     instead of once per call.  Within an iteration every gradient is evaluated at the
-                                     same x_t (Algorithm 1, Step 2), so the worker's sum of micro-batch gradients
-                                     sum_j X_j^T dZ_j is ONE contraction over its stacked micro-batches (K = 64 b_i).  A
-                                     gradient call then runs forward, loss and layer-2 backward as usual (bias and W2
-                                     slices of the row, b_i) and only leaves its dW1 operands -- bf16(X)^T and bf16(dZ)^T,
-                                     (mlp_in + mlp_hidden) * 128 bytes -- in the accumulator set's operand pool; the
-                                     W1 slice of the row is written when the iteration ends (abs_sync_step /
-                                     abs_global_begin), or earlier when something reads or adds to the row
-                                     (abs_accumulator, abs_accumulate*, abs_wait, abs_check, abs_state_export,
-                                     abs_set_launch) or the pool (max(32, 16 W) micro-batches, at most 128) is full.
-                                     The row then holds the same sum as without the flag to fp32 rounding (one fp32
-                                     accumulation over K = 64 b_i instead of b_i rounded additions).  Per micro-batch
-                                     the accumulator traffic of 8 mlp_in mlp_hidden bytes (read + write of the slice)
-                                     becomes 4 mlp_in mlp_hidden / b_i (one write per worker and iteration).  When the
-                                     iteration ends with the W1 slice of every row untouched (the usual case: gradient
-                                     calls only, nothing read in between; single-GPU steps without ABS_FLAG_GRAD_NORM,
-                                     mlp_hidden a multiple of 128) not even that is written: abs_sync_step forms the
-                                     weighted average of the W1 slice as ONE contraction over all micro-batches of all
-                                     workers, (sum_j X_j^T dZ_j) / B, inside the kernel that applies the update, and
-                                     runs the row-based fused step on the bias / W2 part of the vector only (the rows'
-                                     W1 slices then stay as they are: zero, or stale with ABS_FLAG_OVERWRITE_FIRST).
-                                     Combines with every other flag.                                              */
+#define ABS_FLAG_MLP_DEFER 128u   /* with ABS_FLAG_MLP: a gradient call no longer touches its worker's accumulator row.
+                                     Within an iteration every gradient is evaluated at the same x_t (Algorithm 1,
+                                     Step 2), so a worker's sum of micro-batch gradients is ONE contraction over its
+                                     stacked micro-batches, sum_j X_j^T dZ_j with K = 64 b_i, and may be formed late.
+                                     A call runs forward, loss and layer-2 backward, bumps b_i, and leaves in the
+                                     accumulator set's operand pool (about (3 mlp_in + 2 mlp_hidden) * 128 bytes per
+                                     micro-batch) its dW1 operands bf16(X)^T, bf16(dZ)^T and its own db1 | dW2 | db2.
+                                     Calls therefore need no order among themselves, not even those of one worker:
+                                     they are spread over the library's internal streams call by call (results do not
+                                     depend on that: every later sum runs in call order).  The rows are written when
+                                     somebody needs them: when a row is read or added to (abs_accumulator,
+                                     abs_accumulate*, abs_wait, abs_check, abs_state_export, abs_set_launch,
+                                     abs_global_begin) or the pool (max(32, 16 W) micro-batches, at most 128) is full.
+                                     At the end of an iteration (abs_sync_step) they are usually not written at all:
+                                     when no row of the set was written during the iteration (gradient calls only;
+                                     single-GPU step without ABS_FLAG_GRAD_NORM, mlp_hidden a multiple of 128) the step
+                                     forms the weighted average of the W1 slice as one contraction over ALL micro-batches
+                                     of all workers, (sum_j X_j^T dZ_j) / B, inside the kernel that applies the update,
+                                     and runs the row-based fused step on the bias / W2 part of the vector only (the
+                                     rows' W1 slices then stay as they are: zero, or stale with
+                                     ABS_FLAG_OVERWRITE_FIRST).  Otherwise the rows are completed first and the
+                                     row-based step runs.  Either way the result equals that of the per-call path to
+                                     fp32 rounding (one fp32 accumulation over K instead of rounded additions into the
+                                     row).  Combines with every other flag.                                         */
 
 #define ABS_MAX_WORKERS 64u
 #define ABS_MAX_RANKS   16u   /* GPUs taking part in abs_global_* (n_ranks * W <= ABS_MAX_WORKERS)        */
@@ -290,8 +291,8 @@ int abs_selftest_timeout(abs_ctx *ctx);
  *                  128 = forward GEMM and ring dW1 kernel always with their deep pipelines, which take a whole
  *                  SM's shared memory (default: with W > 1, outside serial mode, their light forms of about
  *                  100 KB, so that CTAs of different workers' calls share an SM; same results bit for bit).
- *   ABS_K_MLP_BWD  1 = with ABS_FLAG_MLP_DEFER: the fused step never works from the pooled operands; every
- *                  iteration's dW1 is contracted into the rows first (see the flag).
+ *   ABS_K_MLP_BWD  1 = with ABS_FLAG_MLP_DEFER: the step never works from the pooled operands; every iteration's
+ *                  rows are completed first (see the flag).
  *   ABS_K_MLP_FWD  1 = serial mode: every kernel of a gradient call runs on stream_acc instead of the
  *                  worker's internal stream (for per-kernel timing).
  *   ABS_K_CHAIN    0 = consecutive kernels of a stream are chained by programmatic dependent launch: the next

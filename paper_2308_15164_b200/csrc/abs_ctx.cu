@@ -203,12 +203,18 @@ struct abs_ctx {
     int pool_n[2] = {0, 0};                   // slots handed out (bump allocation; back to 0 when the iteration ends)
     std::vector<int16_t> pool_owner[2];       // worker whose micro-batch sits in the slot; -1: none (contracted, or never used)
     int pend_pool0[kMaxW] = {};               // first pool slot of a waiting group (ABS_FLAG_MLP_COALESCE)
+    // In this mode a call adds nothing to its worker's row, so calls need no order among themselves: call after call
+    // takes the next of the kMlpStreams internal streams (and that stream's scratch set), whoever the worker is.
+    int rr_stream = 0;
+    bool d_outstanding[kMlpStreams] = {};     // contractions enqueued on s_d[k] since stream_acc last waited for it
+    cudaEvent_t ev_d_done[kMlpStreams] = {};
     bool w1_touched[2][kMaxW] = {};           // the row's W1 slice has been written in the set's current iteration
     // A set whose iteration ended with every W1 slice untouched is not contracted row by row: its fused step forms
     // the weighted average of the W1 slice straight from the pooled operands (k_sync_w1) and runs the row-based
     // kernel on the rest of the vector only.
     bool fused_pending[2] = {false, false};
     MlpSlots fused_slots[2]{};
+    uint8_t fused_owner[2][kMlpMaxSlots] = {};
     int fused_n[2] = {0, 0};
     TmapBytes tm_x[2]{}, tm_v{}, tm_shadow[2]{};   // W1 slices of the parameter buffers, the momentum and the bf16 copies
 
@@ -340,14 +346,27 @@ int contract_pending_sets(abs_ctx* c);
 
 // stream_acc waits (on the device) for every gradient kernel enqueued so far on the worker streams (waiting
 // micro-batch groups are started and pooled dW1 operands contracted first).
+// `stream` waits (on the device) for everything enqueued so far on the internal streams.  Per-call mode records
+// ev_w_done behind every call; deferred mode records here, once per wait instead of once per call.
+int wait_for_workers(abs_ctx* c, cudaStream_t stream, bool clear) {
+    for (int k = 0; k < c->n_wstreams; ++k) {
+        if (c->w_outstanding[k]) {
+            if (c->defer) CK(cudaEventRecord(c->ev_w_done[k], c->s_w[k]));
+            CK(cudaStreamWaitEvent(stream, c->ev_w_done[k], 0));
+            if (clear) c->w_outstanding[k] = false;
+        }
+        if (c->d_outstanding[k]) {
+            CK(cudaEventRecord(c->ev_d_done[k], c->s_d[k]));
+            CK(cudaStreamWaitEvent(stream, c->ev_d_done[k], 0));
+            if (clear) c->d_outstanding[k] = false;
+        }
+    }
+    return ABS_OK;
+}
+
 int join_workers(abs_ctx* c) {
     if (int rc = settle_all(c)) return rc;
-    for (int k = 0; k < c->n_wstreams; ++k)
-        if (c->w_outstanding[k]) {
-            CK(cudaStreamWaitEvent(c->s_acc, c->ev_w_done[k], 0));
-            c->w_outstanding[k] = false;
-        }
-    return ABS_OK;
+    return wait_for_workers(c, c->s_acc, true);
 }
 
 // Launch the fused Step-1 kernel on `set`, reading x[in] and writing x[out], on `stream`.
@@ -403,12 +422,14 @@ int launch_fused(abs_ctx* c, uint32_t set, int in, int out, uint64_t log_step, c
         a.plain_only = 1;
         {
             Timed tm(c, ABS_K_SYNC, stream);
+            CK(launch_mlp_gather_small(c->mlp_dims, c->pool[set], c->fused_slots[set], c->fused_owner[set], c->fused_n[set], 0,
+                                       (int)c->cfg.W, 0ull, c->acc(set, 0), c->L.P_pad, stream, c->chained()));
             CK(launch_mlp_sync_w1(c->mlp_dims, c->mlp_scratch[0], c->pool[set], c->fused_slots[set], c->fused_n[set], &c->tm_x[in],
-                                  &c->tm_x[out], &c->tm_v, &c->tm_shadow[out], B, a.lr, a.mu, a.wd, a.lambda_dc, a.disp_scale, stream,
-                                  c->chained()));
+                                  &c->tm_x[out], &c->tm_v, &c->tm_shadow[out], B, a.lr, a.mu, a.wd, a.lambda_dc, a.disp_scale,
+                                  0, stream, c->chained()));
             CK(launch_sync(a, 0, c->num_sms, stream, c->chained()));
         }
-        c->launches += 2;
+        c->launches += 3;
         c->fused_pending[set] = false;
         for (int q = 0; q < c->pool_n[set]; ++q) c->pool_owner[set][q] = -1;
         c->pool_n[set] = 0;
@@ -436,34 +457,38 @@ int take_scratch_set(abs_ctx* c, bool serial, int* out) {
 // on the worker's internal stream (which first waits for everything enqueued on stream_acc so far, the casts
 // included).  deferred: the casts were launched, and counted, by earlier calls.
 int run_mlp_group(abs_ctx* c, uint32_t worker, int set, int n, bool first, int pool0) {
-    const int k = (int)(worker % (uint32_t)c->n_wstreams);
+    int k = (int)(worker % (uint32_t)c->n_wstreams);
     int variant = c->ctas_per_sm[ABS_K_MLP_DW1];
     const bool serial = c->ctas_per_sm[ABS_K_MLP_FWD] == 1;
     // With several workers' calls in flight the forward GEMM and the ring dW1 kernel run in their light
     // shared-memory configurations (a CTA of each fits on one SM); alone, the deep pipelines are faster.
     if (!serial && c->cfg.W > 1 && !(variant & 128)) variant |= kMlpLightBit;
+    if (c->defer) {
+        // The next internal stream and its own scratch set (calls on one stream are ordered, so the set needs no
+        // guard); what crosses streams -- bf16(X), labels, the dW1 operands, the small partial gradients -- sits
+        // in the call's pool slots.  The call ends with k_bwd.
+        k = serial ? 0 : c->rr_stream;
+        if (!serial) c->rr_stream = (c->rr_stream + 1) % c->n_wstreams;
+        cudaStream_t s_run = serial ? c->s_acc : c->s_w[k];
+        if (!serial) {
+            CK(cudaEventRecord(c->ev_fork, c->s_acc));
+            CK(cudaStreamWaitEvent(s_run, c->ev_fork, 0));
+        }
+        CK(launch_mlp_front(c->mlp_dims, c->mlp_scratch[k], c->x(c->pub), c->shadow(c->pub), c->pub, n, first,
+                            c->acc(c->cur, worker), c->cnt(c->cur, worker), &c->pool[c->cur], pool0, variant, s_run,
+                            c->mlp_chain(serial, n), mlp_mark, c));
+        for (int j = 0; j < n; ++j) c->pool_owner[c->cur][pool0 + j] = (int16_t)worker;
+        if (!serial) c->w_outstanding[k] = true;
+        return ABS_OK;
+    }
     const MlpScratch& sc = c->mlp_scratch[set];
     cudaStream_t s_run = serial ? c->s_acc : c->s_w[k];
     if (!serial) {
         CK(cudaEventRecord(c->ev_fork, c->s_acc));
         CK(cudaStreamWaitEvent(s_run, c->ev_fork, 0));
     }
-    __nv_bfloat16* dzt_out = nullptr;
-    if (c->defer) dzt_out = c->pool[c->cur].dzt + (size_t)pool0 * c->mlp_dims.d_hidden * c->mlp_dims.mb;
     CK(launch_mlp_front(c->mlp_dims, sc, c->x(c->pub), c->shadow(c->pub), c->pub, n, first, c->acc(c->cur, worker),
-                        c->cnt(c->cur, worker), dzt_out, variant, s_run, c->mlp_chain(serial, n), mlp_mark, c));
-    if (c->defer) {   // the call ends here: its dW1 operands stay in the pool
-        for (int j = 0; j < n; ++j) c->pool_owner[c->cur][pool0 + j] = (int16_t)worker;
-        if (serial) {
-            for (bool& u : c->set_used) u = false;
-        } else {
-            CK(cudaEventRecord(c->ev_set_done[set], s_run));
-            CK(cudaEventRecord(c->ev_w_done[k], s_run));
-            c->set_used[set] = true;
-            c->w_outstanding[k] = true;
-        }
-        return ABS_OK;
-    }
+                        c->cnt(c->cur, worker), nullptr, 0, variant, s_run, c->mlp_chain(serial, n), mlp_mark, c));
     cudaStream_t s_gemm = s_run;
     if (!serial) {   // dW1 on the worker's second (lowest-priority) stream, behind the front kernels of this call
         s_gemm = c->s_d[k];
@@ -493,7 +518,7 @@ int flush_worker(abs_ctx* c, uint32_t worker) {
     if (n == 0) return ABS_OK;
     const int set = c->pend_set[worker];
     c->pend_n[worker] = 0;
-    c->set_reserved[set] = false;
+    if (!c->defer) c->set_reserved[set] = false;
     c->n_reserved -= 1;
     return run_mlp_group(c, worker, set, n, c->pend_first[worker], c->pend_pool0[worker]);
 }
@@ -514,9 +539,11 @@ int flush_all(abs_ctx* c) {
 // added to -- the accumulator row.  Runs behind the worker's front kernels, on its second stream.
 int contract_worker(abs_ctx* c, uint32_t set, uint32_t worker) {
     MlpSlots sl{};
+    uint8_t owners[kMlpMaxSlots];
     int n = 0;
     for (int q = 0; q < c->pool_n[set]; ++q)
         if (c->pool_owner[set][q] == (int16_t)worker) {
+            owners[n] = (uint8_t)worker;
             sl.s[n++] = (uint16_t)q;
             c->pool_owner[set][q] = -1;
         }
@@ -527,19 +554,24 @@ int contract_worker(abs_ctx* c, uint32_t set, uint32_t worker) {
     // light form beside the other workers' kernels, as for per-call dW1 (measured: batch calls 13.6 -> 13.1 us)
     if (!serial && c->cfg.W > 1 && !(variant & 128)) variant |= kMlpLightBit;
     cudaStream_t s_gemm = c->s_acc;
-    if (!serial) {
+    if (!serial) {   // the worker's calls ran on any of the internal streams; stream_acc may have waited for some already
         s_gemm = c->s_d[k];
-        CK(cudaEventRecord(c->ev_front[k], c->s_w[k]));
-        CK(cudaStreamWaitEvent(s_gemm, c->ev_front[k], 0));
+        CK(cudaEventRecord(c->ev_fork, c->s_acc));
+        CK(cudaStreamWaitEvent(s_gemm, c->ev_fork, 0));
+        for (int j = 0; j < c->n_wstreams; ++j)
+            if (c->w_outstanding[j]) {
+                CK(cudaEventRecord(c->ev_front[j], c->s_w[j]));
+                CK(cudaStreamWaitEvent(s_gemm, c->ev_front[j], 0));
+            }
     }
-    const bool store = !c->w1_touched[set][worker];
+    const bool keep = c->w1_touched[set][worker];   // the row was written earlier in the iteration: add to it
+    CK(launch_mlp_gather_small(c->mlp_dims, c->pool[set], sl, owners, n, (int)worker, 1, keep ? (1ull << worker) : 0ull,
+                               c->acc(set, 0), c->L.P_pad, s_gemm, false));
+    c->launches += 1;
     CK(launch_mlp_dw1(c->mlp_dims, c->mlp_scratch[0], &c->pool[set], &sl, c->acc(set, worker),
-                      &c->acc_tmaps[(size_t)set * c->cfg.W + worker], n, store, variant, s_gemm, false, mlp_mark, c));
+                      &c->acc_tmaps[(size_t)set * c->cfg.W + worker], n, !keep, variant, s_gemm, false, mlp_mark, c));
     c->w1_touched[set][worker] = true;
-    if (!serial) {
-        CK(cudaEventRecord(c->ev_w_done[k], s_gemm));
-        c->w_outstanding[k] = true;
-    }
+    if (!serial) c->d_outstanding[k] = true;
     return ABS_OK;
 }
 
@@ -578,7 +610,10 @@ int close_iteration(abs_ctx* c) {
     int n = 0;
     if (fuse) {
         for (int q = 0; q < c->pool_n[set]; ++q)
-            if (c->pool_owner[set][q] >= 0) c->fused_slots[set].s[n++] = (uint16_t)q;
+            if (c->pool_owner[set][q] >= 0) {
+                c->fused_owner[set][n] = (uint8_t)c->pool_owner[set][q];
+                c->fused_slots[set].s[n++] = (uint16_t)q;
+            }
         fuse = n > 0;
     }
     if (!fuse) {
@@ -597,11 +632,7 @@ int take_pool_slots(abs_ctx* c, int n, int* slot0) {
     const uint32_t set = c->cur;
     if (c->pool_n[set] + n > c->pool[set].cap) {
         if (int rc = settle_all(c)) return rc;
-        for (int k = 0; k < c->n_wstreams; ++k)
-            if (c->w_outstanding[k]) {
-                CK(cudaStreamWaitEvent(c->s_acc, c->ev_w_done[k], 0));
-                c->w_outstanding[k] = false;
-            }
+        if (int rc = wait_for_workers(c, c->s_acc, true)) return rc;
         c->pool_n[set] = 0;
     }
     *slot0 = c->pool_n[set];
@@ -620,26 +651,28 @@ void turn_sets(abs_ctx* c, uint32_t closing, uint32_t opening) {
 // stream_acc has passed this point), everything else when the group runs.
 int coalesce_one(abs_ctx* c, uint32_t worker, const void* x_dev, const int32_t* y_dev) {
     if (c->pend_n[worker] == 0) {
-        if (c->n_reserved >= kMlpSets / 2) {   // keep half of the scratch sets for groups that are running
-            int oldest = -1;
-            for (uint32_t i = 0; i < c->cfg.W; ++i)
-                if (c->pend_n[i] && (oldest < 0 || c->pend_age[i] < c->pend_age[oldest])) oldest = (int)i;
-            if (int rc = flush_worker(c, (uint32_t)oldest)) return rc;
-        }
-        int set = 0;
-        if (c->defer)   // the group's dW1 operands sit in consecutive pool slots (unused ones stay empty)
+        if (c->defer) {   // the group waits in consecutive pool slots (unused ones stay empty)
             if (int rc = take_pool_slots(c, kMlpMaxBatch, &c->pend_pool0[worker])) return rc;
-        if (int rc = take_scratch_set(c, false, &set)) return rc;
-        c->set_reserved[set] = true;
+            c->pend_set[worker] = 0;
+        } else {
+            if (c->n_reserved >= kMlpSets / 2) {   // keep half of the scratch sets for groups that are running
+                int oldest = -1;
+                for (uint32_t i = 0; i < c->cfg.W; ++i)
+                    if (c->pend_n[i] && (oldest < 0 || c->pend_age[i] < c->pend_age[oldest])) oldest = (int)i;
+                if (int rc = flush_worker(c, (uint32_t)oldest)) return rc;
+            }
+            int set = 0;
+            if (int rc = take_scratch_set(c, false, &set)) return rc;
+            c->set_reserved[set] = true;
+            c->pend_set[worker] = set;
+        }
         c->n_reserved += 1;
-        c->pend_set[worker] = set;
         c->pend_first[worker] = c->h_cnt[(size_t)c->cur * c->cfg.W + worker] == 0;
         c->pend_age[worker] = ++c->pend_clock;
     }
     const int slot = c->pend_n[worker];
-    __nv_bfloat16* xtb_out = nullptr;
-    if (c->defer) xtb_out = c->pool[c->cur].xtb + (size_t)(c->pend_pool0[worker] + slot) * c->mlp_dims.d_in * c->mlp_dims.mb;
-    CK(launch_mlp_cast(c->mlp_dims, c->mlp_scratch[c->pend_set[worker]], slot, 1, x_dev, c->x_bf16(), y_dev, xtb_out, c->s_acc,
+    CK(launch_mlp_cast(c->mlp_dims, c->mlp_scratch[c->pend_set[worker]], c->defer ? c->pend_pool0[worker] + slot : slot, 1, x_dev,
+                       c->x_bf16(), y_dev, c->defer ? &c->pool[c->cur] : nullptr, c->s_acc,
                        (c->mlp_chain(false, 1) & kChainCast) != 0, mlp_mark, c));
     c->pend_n[worker] = slot + 1;
     c->h_cnt[(size_t)c->cur * c->cfg.W + worker] += 1;
@@ -743,7 +776,7 @@ int abs_init(abs_ctx** out, const abs_config* cfg, void* workspace_dev, size_t w
                     return bail(e, "cuTensorMapEncodeTiled(parameters)");
             }
         if ((e = cudaEventCreateWithFlags(&c->ev_fork, cudaEventDisableTiming)) != cudaSuccess) return bail(e, "cudaEventCreate");
-        c->n_wstreams = (int)std::min<uint32_t>(cfg->W, kMlpStreams);
+        c->n_wstreams = c->defer ? kMlpStreams : (int)std::min<uint32_t>(cfg->W, kMlpStreams);
         // Highest priority: the short, dependent gradient kernels get free CTA slots before the long HBM-bound
         // fused step that runs beside them on stream_sync and would otherwise fill every slot with its own CTAs.
         int prio_lo = 0, prio_hi = 0;
@@ -753,6 +786,7 @@ int abs_init(abs_ctx** out, const abs_config* cfg, void* workspace_dev, size_t w
             if ((e = cudaStreamCreateWithPriority(&c->s_d[k], cudaStreamNonBlocking, prio_lo)) != cudaSuccess) return bail(e, "cudaStreamCreate");
             if ((e = cudaEventCreateWithFlags(&c->ev_w_done[k], cudaEventDisableTiming)) != cudaSuccess) return bail(e, "cudaEventCreate");
             if ((e = cudaEventCreateWithFlags(&c->ev_front[k], cudaEventDisableTiming)) != cudaSuccess) return bail(e, "cudaEventCreate");
+            if ((e = cudaEventCreateWithFlags(&c->ev_d_done[k], cudaEventDisableTiming)) != cudaSuccess) return bail(e, "cudaEventCreate");
         }
         c->acc_tmaps.resize((size_t)2 * cfg->W);
         for (uint32_t set = 0; set < 2; ++set)
@@ -863,18 +897,17 @@ int abs_accumulate_mlp_batch(abs_ctx* c, uint32_t worker, uint32_t n, const void
         if (int rc = join_workers(c)) return rc;
     }
     int set = 0, pool0 = 0;
-    __nv_bfloat16* xtb_out = nullptr;
     if (c->defer) {
         if (int rc = take_pool_slots(c, (int)n, &pool0)) return rc;
-        xtb_out = c->pool[c->cur].xtb + (size_t)pool0 * c->mlp_dims.d_in * c->mlp_dims.mb;
+    } else if (int rc = take_scratch_set(c, serial, &set)) {
+        return rc;
     }
-    if (int rc = take_scratch_set(c, serial, &set)) return rc;
     // A worker's first gradient of an iteration finds its accumulator row empty (all zero, or -- with
     // ABS_FLAG_OVERWRITE_FIRST -- stale): it is stored, not added, and dW1 skips reading the 4 d_in d_hidden
     // bytes of the slice.  0 + g = g, so the default mode's results do not change.
     const bool first = c->h_cnt[(size_t)c->cur * c->cfg.W + worker] == 0;
-    CK(launch_mlp_cast(c->mlp_dims, c->mlp_scratch[set], 0, (int)n, x_dev, c->x_bf16(), y_dev, xtb_out, c->s_acc,
-                       (c->mlp_chain(serial, (int)n) & kChainCast) != 0, mlp_mark, c));
+    CK(launch_mlp_cast(c->mlp_dims, c->mlp_scratch[set], c->defer ? pool0 : 0, (int)n, x_dev, c->x_bf16(), y_dev,
+                       c->defer ? &c->pool[c->cur] : nullptr, c->s_acc, (c->mlp_chain(serial, (int)n) & kChainCast) != 0, mlp_mark, c));
     if (int rc = run_mlp_group(c, worker, set, (int)n, first, pool0)) return rc;
     c->h_cnt[(size_t)c->cur * c->cfg.W + worker] += (int32_t)n;
     return ABS_OK;
@@ -925,8 +958,7 @@ int abs_sync_step(abs_ctx* c) {
         CK(cudaStreamWaitEvent(c->s_sync, c->ev_acc_done, 0));
         // Step 1 needs every gradient of iteration t; stream_acc does not: the workers go straight on with
         // iteration t+1 (other accumulator set, other parameter buffer), each behind its own previous call only.
-        for (int k = 0; k < c->n_wstreams; ++k)
-            if (c->w_outstanding[k]) CK(cudaStreamWaitEvent(c->s_sync, c->ev_w_done[k], 0));
+        if (int rc = wait_for_workers(c, c->s_sync, false)) return rc;
         if (B > 0) {
             const int out = c->pub ^ 1;
             int rc = launch_fused(c, c->cur, c->pub, out, c->t + 1, c->s_sync);
@@ -1010,8 +1042,7 @@ int abs_global_begin(abs_ctx* c, int32_t** counts_dev, uint32_t* n_counts) {
     }
     CK(cudaEventRecord(c->ev_acc_done, c->s_acc));
     CK(cudaStreamWaitEvent(c->s_sync, c->ev_acc_done, 0));
-    for (int k = 0; k < c->n_wstreams; ++k)
-        if (c->w_outstanding[k]) CK(cudaStreamWaitEvent(c->s_sync, c->ev_w_done[k], 0));
+    if (int rc = wait_for_workers(c, c->s_sync, false)) return rc;
     // This rank's b_i into its slots of the exchange vector (zeros elsewhere: the caller's sum over ranks then
     // is a gather); the device counters of the set are cleared here, the kernel reads the exchanged copy.
     CK(launch_global_counts(c->gcnt(), c->cnt(c->cur, 0), (int)(c->rank * W), (int)W, (int)(c->n_ranks * W), c->s_sync));
@@ -1297,7 +1328,7 @@ int drain(abs_ctx* c) {
     if (c->s_copy) CK(cudaStreamSynchronize(c->s_copy));
     CK(cudaStreamSynchronize(c->s_acc));
     if (c->pipelined) CK(cudaStreamSynchronize(c->s_sync));
-    for (int k = 0; k < c->n_wstreams; ++k) c->w_outstanding[k] = false;
+    for (int k = 0; k < c->n_wstreams; ++k) c->w_outstanding[k] = c->d_outstanding[k] = false;
     return ABS_OK;
 }
 }  // namespace
@@ -1395,6 +1426,7 @@ int abs_set_launch(abs_ctx* c, int kernel_class, int ctas_per_sm) {
         return invalid(c, "unknown bits in the ABS_K_MLP_DW1 mask");
     if (kernel_class == ABS_K_CHAIN && (ctas_per_sm < 0 || ctas_per_sm > 1)) return invalid(c, "ABS_K_CHAIN takes 0 or 1");
     if (kernel_class == ABS_K_MLP_FWD && (ctas_per_sm < 0 || ctas_per_sm > 1)) return invalid(c, "ABS_K_MLP_FWD takes 0 or 1");
+    if (kernel_class == ABS_K_MLP_BWD && (ctas_per_sm < 0 || ctas_per_sm > 1)) return invalid(c, "ABS_K_MLP_BWD takes 0 or 1");
     if (int rc = settle_all(c)) return rc;
     c->ctas_per_sm[kernel_class] = ctas_per_sm;
     return ABS_OK;
@@ -1462,6 +1494,7 @@ int abs_destroy(abs_ctx* c) {
     for (int k = 0; k < c->n_wstreams; ++k)
         if (c->s_d[k]) { cudaStreamSynchronize(c->s_d[k]); cudaStreamDestroy(c->s_d[k]); }
     for (cudaEvent_t e : c->ev_front) if (e) cudaEventDestroy(e);
+    for (cudaEvent_t e : c->ev_d_done) if (e) cudaEventDestroy(e);
     for (cudaEvent_t e : c->ev_set_done) if (e) cudaEventDestroy(e);
     for (cudaEvent_t e : c->ev_w_done) if (e) cudaEventDestroy(e);
     if (c->ev_fork) cudaEventDestroy(c->ev_fork);

@@ -165,11 +165,18 @@ struct MlpScratch {      // device pointers carved from the workspace (all hidde
 };
 // ABS_FLAG_MLP_DEFER: the dW1 operands of an accumulator set's gradient calls are kept (bf16(X)^T and bf16(dZ)^T,
 // (d_in + d_hidden) * 128 bytes per micro-batch) in `cap` slots instead of being contracted call by call.
+// A slot also holds what else a call hands from one of its kernels to the next across streams -- bf16(X) for the
+// forward GEMM, the labels -- and the micro-batch's db1 | dW2 | db2 (laid out like the row behind W1): in this
+// mode a call adds nothing to the row, so calls of one worker need no order among themselves.
 struct MlpPool {
     __nv_bfloat16* xtb;  // [cap][d_in][mb]
     __nv_bfloat16* dzt;  // [cap][d_hidden][mb]
+    __nv_bfloat16* xb;   // [cap][mb][d_in]
+    int32_t* ycopy;      // [cap][mb]
+    float* part;         // [cap][part_stride]: db1 [d_hidden] | dW2 [d_hidden][d_out] | db2 [d_out]
+    size_t part_stride;  // floats
     int cap;
-    TmapBytes tmap_xt, tmap_dzt;
+    TmapBytes tmap_xt, tmap_dzt, tmap_xb;
 };
 size_t mlp_pool_bytes(const MlpDims& d, int cap);
 cudaError_t mlp_pool_init(MlpPool* p, const MlpDims& d, int cap, void* base);
@@ -183,11 +190,11 @@ cudaError_t mlp_make_acc_tmap(void* tmap_out, const MlpDims& d, float* acc_row);
 cudaError_t mlp_make_shadow_tmap(void* tmap_out, const MlpDims& d, __nv_bfloat16* shadow);
 // Step 1 + update of the W1 slice straight from the pooled operands of the set's nb micro-batches (slots): the
 // weighted average is (sum_j X_j^T dZ_j) / B.  tm_*: descriptors from mlp_make_acc_tmap (x_in, x_out, v: fp32 vectors)
-// and mlp_make_shadow_tmap (bf16 copy of x_out, or nullptr).  Needs d_hidden % 128 == 0.
+// and mlp_make_shadow_tmap (bf16 copy of x_out, or nullptr).  Needs d_hidden % 128 == 0.  max_ctas > 0 caps the grid.
 cudaError_t launch_mlp_sync_w1(const MlpDims& d, const MlpScratch& s, const MlpPool& pool, const MlpSlots& slots, int nb,
                                const void* tm_x_in, const void* tm_x_out, const void* tm_v, const void* tm_shadow,
-                               float B, float lr, float mu, float wd, float lambda_dc, float disp_scale, cudaStream_t stream,
-                               bool chained);
+                               float B, float lr, float mu, float wd, float lambda_dc, float disp_scale, int max_ctas,
+                               cudaStream_t stream, bool chained);
 // The gradient of a call is enqueued in three parts so that the caller can put them on different streams:
 //   cast:  the only part that reads the caller's x_dev / y_dev (bf16 copies and labels into this scratch set);
 //   front: forward GEMM, loss, layer-2 backward (writes dzt of this scratch set; adds db2, db1, dW2 into
@@ -199,14 +206,21 @@ cudaError_t launch_mlp_sync_w1(const MlpDims& d, const MlpScratch& s, const MlpP
 // one call -- forward class: 0 cast, 1 forward GEMM, 2 bias / ReLU / logits), mark(user, kernel_class, n, stream)
 // after its n launches.
 typedef void (*MlpMark)(void* user, int kernel_class, int n, cudaStream_t stream);
-// xtb_out / dzt_out: where bf16(X)^T / bf16(dZ)^T of the call's nb micro-batches go ([nb][d_in][mb] /
-// [nb][d_hidden][mb]); nullptr: slots slot0.. / 0.. of the scratch set.
+// pool (ABS_FLAG_MLP_DEFER): the cast writes into pool slots slot0.. instead of the scratch set's; the front kernels
+// read them there (pool_slot0..), leave bf16(dZ)^T and the micro-batches' db1 | dW2 | db2 there and add nothing to
+// acc_row (only cnt is bumped, atomically).
 cudaError_t launch_mlp_cast(const MlpDims& d, const MlpScratch& s, int slot0, int nb, const void* x_dev, bool x_is_bf16,
-                            const int32_t* y_dev, __nv_bfloat16* xtb_out, cudaStream_t stream, bool chained, MlpMark mark,
+                            const int32_t* y_dev, const MlpPool* pool, cudaStream_t stream, bool chained, MlpMark mark,
                             void* user);
 cudaError_t launch_mlp_front(const MlpDims& d, const MlpScratch& s, const float* x_pub, const __nv_bfloat16* shadow,
-                             int shadow_idx, int nb, bool store, float* acc_row, int32_t* cnt, __nv_bfloat16* dzt_out,
-                             int variant, cudaStream_t stream, int chain, MlpMark mark, void* user);
+                             int shadow_idx, int nb, bool store, float* acc_row, int32_t* cnt, const MlpPool* pool,
+                             int pool_slot0, int variant, cudaStream_t stream, int chain, MlpMark mark, void* user);
+// Bias / W2 part of the rows of workers first_worker .. first_worker + n_workers - 1 of one accumulator set from the
+// pooled per-micro-batch partials: row = (keep_mask bit ? row : 0) + sum of the partials of the worker's slots
+// (owners[q] = worker of slots.s[q]), in list order.
+cudaError_t launch_mlp_gather_small(const MlpDims& d, const MlpPool& pool, const MlpSlots& slots, const uint8_t* owners, int n,
+                                    int first_worker, int n_workers, unsigned long long keep_mask, float* acc_set,
+                                    size_t row_stride, cudaStream_t stream, bool chained);
 // nb: a call may carry up to kMlpMaxBatch micro-batches (x_dev [nb][mb][d_in], y_dev [nb][mb]): the front kernels
 // take them as an extra grid dimension, and ONE dW1 launch contracts them with K = 64 nb (the accumulator slice is
 // read and written once).

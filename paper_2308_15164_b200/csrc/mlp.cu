@@ -189,7 +189,7 @@ __global__ void __launch_bounds__(256) k_bwd(const __nv_bfloat16* hbt, const flo
                                              const float* __restrict__ b2, const int32_t* y,
                                              const __nv_bfloat16* __restrict__ w2b, __nv_bfloat16* dzt, float* bpart,
                                              unsigned int* tickets_b, float* acc_b1, float* acc_w2, float* acc_b2,
-                                             int32_t* cnt, int d_h, int d_out, int store) {
+                                             int32_t* cnt, int d_h, int d_out, int store, float* part, size_t part_stride) {
     __shared__ float sdl[kMB][kOutPad + 1];     // bf16(dL) as float
     __shared__ float sdl32[kMB][kOutPad + 1];   // dL unrounded (CTA 0: db2)
     __shared__ float sw2[kHB][kOutPad];
@@ -279,6 +279,18 @@ __global__ void __launch_bounds__(256) k_bwd(const __nv_bfloat16* hbt, const flo
             if (slot == 0) c += sdz[hl][rr];
         }
         const int h = h_beg + hl;
+        if (part) {
+            // Deferred form: nothing is added to the row here.  Every micro-batch leaves its own db1 | dW2 | db2 (laid
+            // out like the row behind W1) in its pool slot; k_gather_small adds them up, in slot order, when the
+            // iteration ends -- so calls of one worker need no order among themselves.
+            float* mine = part + (size_t)jb * part_stride;
+            if (slot < d_out) mine[d_h + (size_t)h * d_out + slot] = a;
+            if (slot + 8 < d_out) mine[d_h + (size_t)h * d_out + slot + 8] = b;
+            if (slot == 0) mine[h] = c;
+            if (blockIdx.x == 0 && threadIdx.x < d_out) mine[d_h + (size_t)d_h * d_out + threadIdx.x] = db2;
+            if (blockIdx.x == 0 && jb == 0 && threadIdx.x == 0) atomicAdd(cnt, nb);   // M_t^i += nb * M_r
+            return;
+        }
         if (nb > 1) {
             // Several micro-batches add into the same accumulator entries: every CTA parks its partial sums, and
             // the last of the nb CTAs of this hidden chunk ("last CTA done" ticket) adds them up in micro-batch
@@ -311,6 +323,36 @@ __global__ void __launch_bounds__(256) k_bwd(const __nv_bfloat16* hbt, const flo
             if (blockIdx.x == 0 && threadIdx.x < d_out) acc_b2[threadIdx.x] += db2;
         }
         if (blockIdx.x == 0 && threadIdx.x == 0) cnt[0] += nb;   // M_t^i += nb * M_r
+    }
+}
+
+// --------------------------------------------------------------------------------------------
+// k_gather_small (ABS_FLAG_MLP_DEFER): the bias / W2 part of worker rows from the per-micro-batch partials that
+// k_bwd left in the pool.  Worker w = first_worker + blockIdx.y:
+//     row_w[o_small + t] = (keep_w ? row_w[o_small + t] : 0) + sum over the slots owned by w, in list order, of part[slot][t]
+// Workers without slots in the list are left alone.
+// --------------------------------------------------------------------------------------------
+struct GatherList {
+    MlpSlots slots;                  // pool slots, in contraction order
+    uint8_t owner[kMlpMaxSlots];     // worker that owns each of them
+};
+__global__ void __launch_bounds__(256) k_gather_small(const float* __restrict__ part, size_t part_stride,
+                                                      const __grid_constant__ GatherList gl, int n, int first_worker,
+                                                      unsigned long long keep_mask, float* acc, size_t row_stride,
+                                                      size_t o_small, int n_small) {
+    const int w = first_worker + blockIdx.y;
+    pdl_wait();
+    pdl_trigger();
+    bool any = false;
+    for (int q = 0; q < n; ++q) any = any || gl.owner[q] == w;
+    if (!any) return;
+    float* row = acc + (size_t)w * row_stride + o_small;
+    const bool keep = (keep_mask >> w) & 1ull;
+    for (int t = blockIdx.x * 256 + threadIdx.x; t < n_small; t += gridDim.x * 256) {
+        float a = keep ? row[t] : 0.f;
+        for (int q = 0; q < n; ++q)
+            if (gl.owner[q] == w) a += part[(size_t)gl.slots.s[q] * part_stride + t];
+        row[t] = a;
     }
 }
 
@@ -986,7 +1028,7 @@ struct FwdSmem {
 template <int NB, bool kLight = false>
 __global__ void __launch_bounds__(128) k_fwd1_tcgen05(const __grid_constant__ CUtensorMap tm_w1,
                                                       const __grid_constant__ CUtensorMap tm_xb, float* __restrict__ zpart,
-                                                      int d_in, int d_h, int* status) {
+                                                      int d_in, int d_h, int xb_row0, int* status) {
     constexpr int kFwdStages = FwdCfg<NB, kLight>::kStages, kFwdStageBytes = FwdCfg<NB, kLight>::kStageBytes;
     constexpr int kTmemCols = FwdCfg<NB, kLight>::kTmemCols;
     extern __shared__ uint8_t smem_raw[];
@@ -1034,8 +1076,8 @@ __global__ void __launch_bounds__(128) k_fwd1_tcgen05(const __grid_constant__ CU
             tma_load_2d_hint(s.stage[st], &tm_w1, h0, k0, &s.full[st], pol_w1);
             tma_load_2d_hint(s.stage[st] + 8192, &tm_w1, h0 + 64, k0, &s.full[st], pol_w1);
 #pragma unroll
-            for (int jb = 0; jb < NB; ++jb)          // rows jb*64.. of the stacked xb
-                tma_load_2d(s.stage[st] + 16384 + jb * 8192, &tm_xb, k0, jb * kMB, &s.full[st]);
+            for (int jb = 0; jb < NB; ++jb)          // rows xb_row0 + jb*64.. of the stacked xb
+                tma_load_2d(s.stage[st] + 16384 + jb * 8192, &tm_xb, k0, xb_row0 + jb * kMB, &s.full[st]);
         }
     } else if (warp == 1 && lane == 0) {             // ---- MMA issuer
         constexpr uint32_t idesc = umma_idesc_bf16(128, 64 * NB) | (1u << 15);   // A is MN-major
@@ -1222,14 +1264,33 @@ cudaError_t mlp_scratch_init(MlpScratch* s, const MlpDims& d, void* base, __nv_b
     return e;
 }
 
+namespace {
+size_t pool_part_stride(const MlpDims& d) {   // floats per slot: db1 | dW2 | db2, padded to whole 128-byte lines
+    return align_up((size_t)d.d_hidden + (size_t)d.d_hidden * d.d_out + d.d_out, 32);
+}
+}  // namespace
+
 size_t mlp_pool_bytes(const MlpDims& d, int cap) {
-    return align_up((size_t)cap * d.d_in * kMB * 2, 1024) + align_up((size_t)cap * d.d_hidden * kMB * 2, 1024);
+    return 2 * align_up((size_t)cap * d.d_in * kMB * 2, 1024) + align_up((size_t)cap * d.d_hidden * kMB * 2, 1024) +
+           align_up((size_t)cap * kMB * 4, 1024) + align_up((size_t)cap * pool_part_stride(d) * 4, 1024);
 }
 
 cudaError_t mlp_pool_init(MlpPool* p, const MlpDims& d, int cap, void* base) {
     p->cap = cap;
-    p->xtb = static_cast<__nv_bfloat16*>(base);
-    p->dzt = reinterpret_cast<__nv_bfloat16*>(static_cast<char*>(base) + align_up((size_t)cap * d.d_in * kMB * 2, 1024));
+    char* at = static_cast<char*>(base);
+    p->xtb = reinterpret_cast<__nv_bfloat16*>(at);
+    at += align_up((size_t)cap * d.d_in * kMB * 2, 1024);
+    p->dzt = reinterpret_cast<__nv_bfloat16*>(at);
+    at += align_up((size_t)cap * d.d_hidden * kMB * 2, 1024);
+    p->xb = reinterpret_cast<__nv_bfloat16*>(at);
+    at += align_up((size_t)cap * d.d_in * kMB * 2, 1024);
+    p->ycopy = reinterpret_cast<int32_t*>(at);
+    at += align_up((size_t)cap * kMB * 4, 1024);
+    p->part = reinterpret_cast<float*>(at);
+    p->part_stride = pool_part_stride(d);
+    if (!encode_2d(reinterpret_cast<CUtensorMap*>(&p->tmap_xb), CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, p->xb, (uint64_t)cap * kMB,
+                   d.d_in, kMB, 64))
+        return cudaErrorInvalidValue;
     // same boxes as the scratch sets' operands: slot j at rows [j*d_in, (j+1)*d_in) of X^T, [j*d_h, (j+1)*d_h) of dZ^T
     if (!encode_2d(reinterpret_cast<CUtensorMap*>(&p->tmap_xt), CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, p->xtb,
                    (uint64_t)cap * d.d_in, kMB, kTileM, kMB) ||
@@ -1237,6 +1298,20 @@ cudaError_t mlp_pool_init(MlpPool* p, const MlpDims& d, int cap, void* base) {
                    (uint64_t)cap * d.d_hidden, kMB, kDwN, kMB))
         return cudaErrorInvalidValue;
     return cudaSuccess;
+}
+
+cudaError_t launch_mlp_gather_small(const MlpDims& d, const MlpPool& pool, const MlpSlots& slots, const uint8_t* owners, int n,
+                                    int first_worker, int n_workers, unsigned long long keep_mask, float* acc_set,
+                                    size_t row_stride, cudaStream_t stream, bool chained) {
+    if (n < 1 || n > kMlpMaxSlots || n_workers < 1) return cudaErrorInvalidValue;
+    GatherList gl;
+    gl.slots = slots;
+    for (int q = 0; q < kMlpMaxSlots; ++q) gl.owner[q] = q < n ? owners[q] : (uint8_t)255;
+    const int n_small = d.d_hidden + d.d_hidden * d.d_out + d.d_out;
+    const size_t o_small = (size_t)d.d_in * d.d_hidden;
+    const float* part = pool.part;
+    return launch_kernel(k_gather_small, dim3((n_small + 255) / 256, n_workers), 256, 0, stream, chained, part, pool.part_stride, gl, n,
+                         first_worker, keep_mask, acc_set, row_stride, o_small, n_small);
 }
 
 cudaError_t mlp_make_shadow_tmap(void* tmap_out, const MlpDims& d, __nv_bfloat16* shadow) {
@@ -1249,8 +1324,8 @@ cudaError_t mlp_make_shadow_tmap(void* tmap_out, const MlpDims& d, __nv_bfloat16
 
 cudaError_t launch_mlp_sync_w1(const MlpDims& d, const MlpScratch& s, const MlpPool& pool, const MlpSlots& slots, int nb,
                                const void* tm_x_in, const void* tm_x_out, const void* tm_v, const void* tm_shadow,
-                               float B, float lr, float mu, float wd, float lambda_dc, float disp_scale, cudaStream_t stream,
-                               bool chained) {
+                               float B, float lr, float mu, float wd, float lambda_dc, float disp_scale, int max_ctas,
+                               cudaStream_t stream, bool chained) {
     if (nb < 1 || nb > kMlpMaxSlots || d.d_hidden % kStepN != 0) return cudaErrorInvalidValue;
     static bool opted_in[64] = {};
     int dev = 0;
@@ -1262,7 +1337,8 @@ cudaError_t launch_mlp_sync_w1(const MlpDims& d, const MlpScratch& s, const MlpP
         if (dev >= 0 && dev < 64) opted_in[dev] = true;
     }
     const int n_tiles_n = d.d_hidden / kStepN, n_tiles = n_tiles_n * (d.d_in / kTileM);
-    const int ctas = n_tiles < s.num_sms ? n_tiles : s.num_sms;
+    int ctas = n_tiles < s.num_sms ? n_tiles : s.num_sms;
+    if (max_ctas > 0 && ctas > max_ctas) ctas = max_ctas;
     const W1StepCoef cf{1.0f / B, lr, mu, wd, lambda_dc, disp_scale};
     const CUtensorMap& shadow_map = *reinterpret_cast<const CUtensorMap*>(tm_shadow ? tm_shadow : tm_x_out);
     return launch_kernel(k_sync_w1, ctas, 64 + kStepEpiThreads, sizeof(StepSmem) + 1024, stream, chained,
@@ -1281,13 +1357,13 @@ cudaError_t mlp_make_acc_tmap(void* tmap_out, const MlpDims& d, float* acc_row) 
 }
 
 cudaError_t launch_mlp_cast(const MlpDims& d, const MlpScratch& s, int slot0, int nb, const void* x_dev, bool x_is_bf16,
-                            const int32_t* y_dev, __nv_bfloat16* xtb_out, cudaStream_t stream, bool chained, MlpMark mark,
+                            const int32_t* y_dev, const MlpPool* pool, cudaStream_t stream, bool chained, MlpMark mark,
                             void* user) {
     mark(user, ABS_K_MLP_FWD, -1, stream);   // part 0 of the forward class: the cast
-    // micro-batch j of the call goes to slot slot0 + j of the scratch set
-    __nv_bfloat16* xb = s.xb + (size_t)slot0 * kMB * d.d_in;
-    __nv_bfloat16* xtb = xtb_out ? xtb_out : s.xtb + (size_t)slot0 * d.d_in * kMB;
-    int32_t* yc = s.ycopy + slot0 * kMB;
+    // micro-batch j of the call goes to slot slot0 + j of the scratch set, or of the pool
+    __nv_bfloat16* xb = (pool ? pool->xb : s.xb) + (size_t)slot0 * kMB * d.d_in;
+    __nv_bfloat16* xtb = (pool ? pool->xtb : s.xtb) + (size_t)slot0 * d.d_in * kMB;
+    int32_t* yc = (pool ? pool->ycopy : s.ycopy) + slot0 * kMB;
     const dim3 grid(d.d_in / 16, nb);
     const cudaError_t e = x_is_bf16 ? launch_kernel(k_cast_x<true>, grid, 256, 0, stream, chained, x_dev, y_dev, xb, xtb, yc, d.d_in)
                                     : launch_kernel(k_cast_x<false>, grid, 256, 0, stream, chained, x_dev, y_dev, xb, xtb, yc, d.d_in);
@@ -1297,17 +1373,17 @@ cudaError_t launch_mlp_cast(const MlpDims& d, const MlpScratch& s, int slot0, in
 
 template <int NB>
 cudaError_t fwd1_launch(dim3 grid, cudaStream_t stream, bool chained, bool light, const CUtensorMap& tw, const CUtensorMap& tx,
-                        float* zpart, int d_in, int d_h, int* status) {
+                        float* zpart, int d_in, int d_h, int xb_row0, int* status) {
     if (light)
         return launch_kernel(k_fwd1_tcgen05<NB, true>, grid, 128, sizeof(FwdSmem<NB, true>) + 1024, stream, chained, tw, tx, zpart,
-                             d_in, d_h, status);
+                             d_in, d_h, xb_row0, status);
     return launch_kernel(k_fwd1_tcgen05<NB, false>, grid, 128, sizeof(FwdSmem<NB, false>) + 1024, stream, chained, tw, tx, zpart,
-                         d_in, d_h, status);
+                         d_in, d_h, xb_row0, status);
 }
 
 cudaError_t launch_mlp_front(const MlpDims& d, const MlpScratch& s, const float* x_pub, const __nv_bfloat16* shadow,
-                             int shadow_idx, int nb, bool store, float* acc_row, int32_t* cnt, __nv_bfloat16* dzt_out,
-                             int variant, cudaStream_t stream, int chain, MlpMark mark, void* user) {
+                             int shadow_idx, int nb, bool store, float* acc_row, int32_t* cnt, const MlpPool* pool,
+                             int pool_slot0, int variant, cudaStream_t stream, int chain, MlpMark mark, void* user) {
     const size_t o_b1 = (size_t)d.d_in * d.d_hidden, o_w2 = o_b1 + d.d_hidden, o_b2 = o_w2 + (size_t)d.d_hidden * d.d_out;
     cudaError_t e;
     const unsigned n_cta = d.d_hidden / kHB;
@@ -1318,14 +1394,15 @@ cudaError_t launch_mlp_front(const MlpDims& d, const MlpScratch& s, const float*
     int nsplit = kSplitK;
     while (nsplit > 1 && d.d_in % (64 * nsplit) != 0) nsplit /= 2;
     const CUtensorMap& tw = *reinterpret_cast<const CUtensorMap*>(&s.tmap_w1[shadow_idx]);
-    const CUtensorMap& tx = *reinterpret_cast<const CUtensorMap*>(&s.tmap_xb);
+    const CUtensorMap& tx = *reinterpret_cast<const CUtensorMap*>(pool ? &pool->tmap_xb : &s.tmap_xb);
+    const int xb_row0 = pool ? pool_slot0 * kMB : 0;
     const dim3 grid(d.d_hidden / 128, nsplit);
     mark(user, ABS_K_MLP_FWD, -2, stream);       // part 1: the forward GEMM
     switch (nb) {                                // the nb micro-batches are stacked along N of one GEMM
-        case 1: e = fwd1_launch<1>(grid, stream, (chain & kChainFwd1) != 0, light, tw, tx, s.zpart, d.d_in, d.d_hidden, s.status); break;
-        case 2: e = fwd1_launch<2>(grid, stream, (chain & kChainFwd1) != 0, light, tw, tx, s.zpart, d.d_in, d.d_hidden, s.status); break;
-        case 3: e = fwd1_launch<3>(grid, stream, (chain & kChainFwd1) != 0, light, tw, tx, s.zpart, d.d_in, d.d_hidden, s.status); break;
-        default: e = fwd1_launch<4>(grid, stream, (chain & kChainFwd1) != 0, light, tw, tx, s.zpart, d.d_in, d.d_hidden, s.status); break;
+        case 1: e = fwd1_launch<1>(grid, stream, (chain & kChainFwd1) != 0, light, tw, tx, s.zpart, d.d_in, d.d_hidden, xb_row0, s.status); break;
+        case 2: e = fwd1_launch<2>(grid, stream, (chain & kChainFwd1) != 0, light, tw, tx, s.zpart, d.d_in, d.d_hidden, xb_row0, s.status); break;
+        case 3: e = fwd1_launch<3>(grid, stream, (chain & kChainFwd1) != 0, light, tw, tx, s.zpart, d.d_in, d.d_hidden, xb_row0, s.status); break;
+        default: e = fwd1_launch<4>(grid, stream, (chain & kChainFwd1) != 0, light, tw, tx, s.zpart, d.d_in, d.d_hidden, xb_row0, s.status); break;
     }
     mark(user, ABS_K_MLP_FWD, 1, stream);
     if (e != cudaSuccess) return e;
@@ -1343,10 +1420,13 @@ cudaError_t launch_mlp_front(const MlpDims& d, const MlpScratch& s, const float*
     const __nv_bfloat16* hbt = s.hbt;
     const float* gpart = s.gpart;
     const float* b2 = x_pub + o_b2;
-    const int32_t* yc = s.ycopy;
-    e = launch_kernel(k_bwd, dim3(n_cta, nb), 256, 0, stream, (chain & kChainBwd) != 0, hbt, gpart, n_groups, b2, yc, w2b,
-                      dzt_out ? dzt_out : s.dzt, s.bpart,
-                      s.tickets_b, acc_row + o_b1, acc_row + o_w2, acc_row + o_b2, cnt, d.d_hidden, d.d_out, store ? 1 : 0);
+    const int32_t* yc = pool ? pool->ycopy + (size_t)pool_slot0 * kMB : s.ycopy;
+    __nv_bfloat16* dzt = pool ? pool->dzt + (size_t)pool_slot0 * d.d_hidden * kMB : s.dzt;
+    float* part = pool ? pool->part + (size_t)pool_slot0 * pool->part_stride : nullptr;
+    const size_t part_stride = pool ? pool->part_stride : 0;
+    e = launch_kernel(k_bwd, dim3(n_cta, nb), 256, 0, stream, (chain & kChainBwd) != 0, hbt, gpart, n_groups, b2, yc, w2b, dzt, s.bpart,
+                      s.tickets_b, acc_row + o_b1, acc_row + o_w2, acc_row + o_b2, cnt, d.d_hidden, d.d_out, store ? 1 : 0, part,
+                      part_stride);
     mark(user, ABS_K_MLP_BWD, 1, stream);
     return e;
 }

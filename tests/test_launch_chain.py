@@ -59,7 +59,7 @@ def test_chained_and_plain_launches_give_the_same_bits_streaming(cfg, T, batch, 
     assert not np.array_equal(a[0], wlm.params0(wlm.config(cfg, small=True, T=T)))
 
 
-def _mlp_run(chain, mode, serial, pipelined):
+def _mlp_run(chain, mode, serial, pipelined, defer=False):
     import torch
 
     from paper_2308_15164_b200 import binding as B
@@ -70,7 +70,7 @@ def _mlp_run(chain, mode, serial, pipelined):
     dev = torch.device("cuda:0")
     xs_d, ys_d = torch.from_numpy(xs).to(dev), torch.from_numpy(ys).to(dev)
     eng = B.AbsSgd(torch.from_numpy(wlm.params0(wl)).to(dev), wl.W, wl.lr, wl.momentum, wl.weight_decay, pipelined=pipelined,
-                   mlp=(d.d_in, d.d_hidden, d.d_out, d.mb), mlp_coalesce=(mode == "gathered"))
+                   mlp=(d.d_in, d.d_hidden, d.d_out, d.mb), mlp_coalesce=(mode == "gathered"), mlp_defer=defer)
     eng.set_launch(B.K_CHAIN, chain)
     eng.set_launch(B.K_MLP_FWD, serial)
     torch.cuda.synchronize()
@@ -93,14 +93,15 @@ def _mlp_run(chain, mode, serial, pipelined):
     return x
 
 
+@pytest.mark.parametrize("defer", [False, True], ids=["per-call-dw1", "deferred-dw1"])
 @pytest.mark.parametrize("mode", ["single", "gathered", "batch"])
 @pytest.mark.parametrize("serial", [0, 1], ids=["worker-streams", "one-stream"])
-def test_chained_and_plain_launches_give_the_same_bits_mlp(mode, serial):
+def test_chained_and_plain_launches_give_the_same_bits_mlp(mode, serial, defer):
     if mode == "gathered" and serial:
         pytest.skip("serial mode runs every call at once: nothing to gather")
     for pipelined in (False, True):
-        a = _mlp_run(0, mode, serial, pipelined)
-        b = _mlp_run(1, mode, serial, pipelined)
+        a = _mlp_run(0, mode, serial, pipelined, defer)
+        b = _mlp_run(1, mode, serial, pipelined, defer)
         assert np.array_equal(a, b), f"pipelined={pipelined}"
 
 
@@ -111,9 +112,9 @@ def test_set_launch_rejects_unknown_values():
 
     eng = B.AbsSgd(torch.zeros(1024, device="cuda"), 2, 0.1)
     for cls, val in ((B.K_CHAIN, 2), (B.K_CHAIN, -1), (B.K_MLP_DW1, 1), (B.K_MLP_DW1, 64), (B.K_MLP_DW1, 256),
-                     (B.K_MLP_FWD, 2), (B.K_SYNC, -3), (6, 0), (-1, 0)):
+                     (B.K_MLP_FWD, 2), (B.K_MLP_BWD, 2), (B.K_SYNC, -3), (6, 0), (-1, 0)):
         assert B.lib.abs_set_launch(eng._h, cls, val) == B.EINVAL, (cls, val)
-    for cls, val in ((B.K_CHAIN, 1), (B.K_CHAIN, 0), (B.K_MLP_DW1, 4 | 32 | 128), (B.K_MLP_DW1, 8), (B.K_SYNC, -2), (B.K_ACCUMULATE, 4)):
+    for cls, val in ((B.K_CHAIN, 1), (B.K_CHAIN, 0), (B.K_MLP_DW1, 4 | 32 | 128), (B.K_MLP_DW1, 8), (B.K_SYNC, -2), (B.K_ACCUMULATE, 4), (B.K_MLP_BWD, 1)):
         assert B.lib.abs_set_launch(eng._h, cls, val) == B.OK, (cls, val)
     eng.destroy()
 
