@@ -79,3 +79,32 @@ def test_mlp_batches_and_sample_columns():
     assert x.shape == (64, 64, 384) and y.shape == (64, 64) and y.min() == 0 and y.max() == 9
     idx = wl.sample_columns(25_557_032)
     assert idx[0] == 0 and idx[-1] == 25_557_031 and np.all(np.diff(idx) > 0)
+
+
+def test_bench_byte_model_of_the_mlp_runs():
+    """bench.mlp_run_bytes on a schedule small enough to add up by hand (d_in = d_hidden = 128, 10 outputs)."""
+    import importlib.util
+    import os
+
+    spec = importlib.util.spec_from_file_location("bench_module", os.path.join(os.path.dirname(os.path.dirname(__file__)), "bench.py"))
+    bench = importlib.util.module_from_spec(spec)
+    spec.loader.exec_module(bench)
+    d = wl.MlpDims(128, 128, 10, 64)
+    w1, P = 128 * 128, d.P
+    ops = 2 * 64 * (128 + 128)                         # bf16 X^T and dZ^T of one micro-batch
+    sched = [[3, 0], [1, 2]]                           # two iterations, two workers
+    # per-call mode, single calls: worker 0 stores once and adds twice; the second iteration's step applies the first's set
+    total, calls, stored, mbs = bench.mlp_run_bytes(sched, d, P, 1, False)
+    assert (calls, stored, mbs) == (6, 3, 6)
+    assert total == 6 * 2 * w1 + (3 * 4 + 3 * 8) * w1 + 6 * ops + (8 * 1 + 18) * P
+    # batch calls of up to 4: one call per active worker and iteration, all of them store
+    total4, calls4, stored4, _ = bench.mlp_run_bytes(sched, d, P, 4, False)
+    assert (calls4, stored4) == (3, 3)
+    assert total4 == 3 * 2 * w1 + 3 * 4 * w1 + 6 * ops + (8 * 1 + 18) * P
+    # deferred, rows written: the slice once per active worker and iteration, operands written and read
+    rows, _, _, _ = bench.mlp_run_bytes(sched, d, P, 1, False, "rows")
+    assert rows == 6 * 2 * w1 + 3 * 4 * w1 + 2 * 6 * ops + (8 * 1 + 18) * P
+    # deferred, Step 1 from the pool: no accumulator traffic for W1; 18 bytes per W1 element in the step
+    pool, _, _, _ = bench.mlp_run_bytes(sched, d, P, 1, False, "pool")
+    assert pool == 6 * 2 * w1 + 2 * 6 * ops + 18 * w1 + (8 * 1 + 18) * (P - w1)
+    assert pool < rows < total
