@@ -37,7 +37,7 @@ UNIT = "GB/s"
 HBM_NOMINAL_GBS = 8000.0
 HBM_FALLBACK_GBS = 6650.0
 NVLINK_MEASURED_GBS = 770.0        # peer copy, per direction and GPU, measured on this machine
-# the same string in both arms: the workload the benchmark's metric is quoted on
+# the same string in both arms: the workload the headline metric is quoted on
 WORKLOAD = ("cfg2 resnet18-sized static heterogeneity: P=11689512 fp32 (62 tensors), W=4, b=(2,2,4,8), lr=0.1 mu=0.9 "
             "wd=5e-4; one step = one iteration = 16 accumulate + 1 fused sync step")
 MIN_TIMED_SECONDS = 1.0            # the --steps-long region is repeated until this much time has been measured

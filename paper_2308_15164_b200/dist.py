@@ -34,7 +34,7 @@ def init(backend: str, timeout_s: float = 0.0) -> Tuple[int, int, int]:
         os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
         os.environ.setdefault("MASTER_PORT", "29511")
         # the collectives of this package carry a few integers: in-switch reduction buys nothing, and a rank that
-        # leaves while its memory is bound to a multicast object is worse than one that simply leaves
+        # leaves while its memory is bound to an NVLink-switch reduction group is worse than one that simply leaves
         os.environ.setdefault("NCCL_NVLS_ENABLE", "0")
         kw = dict(timeout=datetime.timedelta(seconds=timeout_s)) if timeout_s > 0 else {}
         dist.init_process_group(backend=backend, rank=rank, world_size=world, **kw)
