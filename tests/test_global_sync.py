@@ -227,10 +227,13 @@ def test_call_order_and_mode_errors():
         e.destroy()
 
 
-def test_mlp_gradients_computed_on_two_ranks_match_one_context_and_oracle():
+@pytest.mark.parametrize("defer", [False, True], ids=["per-call-dw1", "deferred-dw1"])
+def test_mlp_gradients_computed_on_two_ranks_match_one_context_and_oracle(defer):
     """Workload 4 (small layer sizes): every rank computes its workers' MLP gradients at x_t (single and batch
     calls) -- the fused kernel must also refresh every rank's bf16 copy of the weights, which the next forward
-    pass reads."""
+    pass reads.  With ABS_FLAG_MLP_DEFER the ranks complete their rows when the iteration ends (one contraction per
+    worker); the one-GPU context they are compared with bit for bit does the same (its step from the pooled
+    operands would sum in another order)."""
     import torch
 
     from oracle.abs_oracle import AbsSgdOracle, mlp_loss_and_grad
@@ -250,8 +253,10 @@ def test_mlp_gradients_computed_on_two_ranks_match_one_context_and_oracle():
     x0_d = torch.from_numpy(x0).to(dev)
     torch.cuda.synchronize()
     mlp = (d.d_in, d.d_hidden, d.d_out, d.mb)
-    one = B.AbsSgd(x0_d, wl.W, wl.lr, wl.momentum, wl.weight_decay, pipelined=True, mlp=mlp)
-    ranks = [B.AbsSgd(x0_d, Wl, wl.lr, wl.momentum, wl.weight_decay, pipelined=True, mlp=mlp) for _ in range(G)]
+    one = B.AbsSgd(x0_d, wl.W, wl.lr, wl.momentum, wl.weight_decay, pipelined=True, mlp=mlp, mlp_defer=defer)
+    if defer:
+        one.set_launch(B.K_MLP_BWD, 1)
+    ranks = [B.AbsSgd(x0_d, Wl, wl.lr, wl.momentum, wl.weight_decay, pipelined=True, mlp=mlp, mlp_defer=defer) for _ in range(G)]
     grp = D.LocalRanks(ranks)
     ref = AbsSgdOracle(x0, wl.W, wl.lr, wl.momentum, wl.weight_decay)
     for t, b_row in enumerate(sched):
