@@ -311,3 +311,42 @@ def test_export_in_the_middle_of_an_iteration_and_resume_in_a_fresh_context():
     o.sync_step()
     assert np.abs(a.params_host().astype(np.float64) - o.params()).max() <= TOL * np.abs(o.params()).max()
     a.destroy(); b.destroy()
+
+
+def test_eager_mode_reading_a_closed_set_that_still_waits_in_pooled_form():
+    """Eager mode applies a set one call after its iteration ended; until then its W1 gradients wait in pooled form.
+    Reading the closed set's rows (abs_accumulator) or exporting the state makes the library complete the rows
+    first; the step that follows then runs row-based and the run still follows the oracle."""
+    import torch
+
+    wl = wlm.config(4, small=True, T=3)
+    x0 = wlm.params0(wl)
+    xs, ys = wlm.mlp_batches(wl)
+    xs_d, ys_d = torch.from_numpy(xs).cuda(), torch.from_numpy(ys).cuda()
+    its = list(wlm.iter_calls(wl))
+    o = AbsSgdOracle(x0, wl.W, wl.lr, wl.momentum, wl.weight_decay)
+    eng = _engine(wl, x0, pipelined=False)
+    for t, calls in enumerate(its):
+        p = o.params()
+        sums = {}
+        for (i, k, c) in calls:
+            g = _grad(p, xs, ys, c, wl)
+            o.accumulate(i, g)
+            sums[i] = sums.get(i, 0) + g
+            eng.accumulate_mlp(i, xs_d[c % wl.mlp_pool], ys_d[c % wl.mlp_pool])
+        closed = eng.counters()[1]
+        eng.sync_step(); o.sync_step()               # the set just filled is now closed and waits for the next call
+        if t == 0:
+            for i, s in sums.items():
+                _close_row(eng.accumulator(closed, i).cpu().numpy(), s, wl, f"closed set, worker {i}")
+        elif t == 1:
+            blob = eng.state_export()
+            assert blob.nbytes > 0
+    eng.sync_step(); o.sync_step()
+    eng.check()
+    ref = o.params()
+    assert np.abs(ref - x0).max() > 1e-4
+    assert np.abs(eng.params_host().astype(np.float64) - ref).max() <= TOL * np.abs(ref).max()
+    for s in range(len(its) + 1):
+        assert np.array_equal(eng.consumed(s), o.consumed[s])
+    eng.destroy()
