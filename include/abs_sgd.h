@@ -114,9 +114,8 @@ extern "C" {
                                      single-GPU step without ABS_FLAG_GRAD_NORM, mlp_hidden a multiple of 128) the step
                                      forms the weighted average of the W1 slice as one contraction over ALL micro-batches
                                      of all workers, (sum_j X_j^T dZ_j) / B, inside the kernel that applies the update,
-                                     and runs the row-based fused step on the bias / W2 part of the vector only (the
-                                     rows' W1 slices then stay as they are: zero, or stale with
-                                     ABS_FLAG_OVERWRITE_FIRST).  Otherwise the rows are completed first and the
+                                     and the bias / W2 part from the pooled per-micro-batch partials (the rows then
+                                     stay as they are: zero, or stale with ABS_FLAG_OVERWRITE_FIRST).  Otherwise the rows are completed first and the
                                      row-based step runs.  Either way the result equals that of the per-call path to
                                      fp32 rounding (one fp32 accumulation over K instead of rounded additions into the
                                      row).  Combines with every other flag.                                         */

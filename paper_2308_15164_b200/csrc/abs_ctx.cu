@@ -214,7 +214,6 @@ struct abs_ctx {
     // kernel on the rest of the vector only.
     bool fused_pending[2] = {false, false};
     MlpSlots fused_slots[2]{};
-    uint8_t fused_owner[2][kMlpMaxSlots] = {};
     int fused_n[2] = {0, 0};
     TmapBytes tm_x[2]{}, tm_v{}, tm_shadow[2]{};   // W1 slices of the parameter buffers, the momentum and the bf16 copies
 
@@ -408,28 +407,21 @@ int launch_fused(abs_ctx* c, uint32_t set, int in, int out, uint64_t log_step, c
         a.tma_one_cta = 4;
     }
     if (c->fused_pending[set]) {
-        // W1 slice: weighted average and update straight from the set's pooled operands; the rest of the vector
-        // (b1, W2, b2) by the row-based kernel, which also logs and clears the counters.
+        // Weighted average and update straight from the set's pool: the bias / W2 part from the per-micro-batch
+        // partials (a small kernel, which also logs and clears the counters), the W1 slice from the dW1 operands.
+        // No accumulator row is read or written.
         float B = 0.f;
         for (uint32_t i = 0; i < c->cfg.W; ++i) B += (float)c->h_cnt[(size_t)set * c->cfg.W + i];
-        const size_t w1 = (size_t)c->mlp_dims.d_in * c->mlp_dims.d_hidden;
-        a.x_in += w1;
-        a.x_out += w1;
-        a.v += w1;
-        a.acc += w1;
-        a.shadow += w1;
-        a.n_vec = (c->L.P_pad - w1) / 4;
-        a.plain_only = 1;
         {
             Timed tm(c, ABS_K_SYNC, stream);
-            CK(launch_mlp_gather_small(c->mlp_dims, c->pool[set], c->fused_slots[set], c->fused_owner[set], c->fused_n[set], 0,
-                                       (int)c->cfg.W, 0ull, c->acc(set, 0), c->L.P_pad, stream, c->chained()));
+            CK(launch_mlp_sync_small(c->mlp_dims, c->pool[set], c->fused_slots[set], c->fused_n[set], a.x_in, a.x_out, a.v, a.shadow,
+                                     B, a.lr, a.mu, a.wd, a.lambda_dc, a.disp_scale, a.cnt, a.log_row, (int)c->cfg.W, stream,
+                                     c->chained()));
             CK(launch_mlp_sync_w1(c->mlp_dims, c->mlp_scratch[0], c->pool[set], c->fused_slots[set], c->fused_n[set], &c->tm_x[in],
                                   &c->tm_x[out], &c->tm_v, &c->tm_shadow[out], B, a.lr, a.mu, a.wd, a.lambda_dc, a.disp_scale,
                                   0, stream, c->chained()));
-            CK(launch_sync(a, 0, c->num_sms, stream, c->chained()));
         }
-        c->launches += 3;
+        c->launches += 2;
         c->fused_pending[set] = false;
         for (int q = 0; q < c->pool_n[set]; ++q) c->pool_owner[set][q] = -1;
         c->pool_n[set] = 0;
@@ -610,10 +602,7 @@ int close_iteration(abs_ctx* c) {
     int n = 0;
     if (fuse) {
         for (int q = 0; q < c->pool_n[set]; ++q)
-            if (c->pool_owner[set][q] >= 0) {
-                c->fused_owner[set][n] = (uint8_t)c->pool_owner[set][q];
-                c->fused_slots[set].s[n++] = (uint16_t)q;
-            }
+            if (c->pool_owner[set][q] >= 0) c->fused_slots[set].s[n++] = (uint16_t)q;
         fuse = n > 0;
     }
     if (!fuse) {

@@ -195,6 +195,12 @@ cudaError_t launch_mlp_sync_w1(const MlpDims& d, const MlpScratch& s, const MlpP
                                const void* tm_x_in, const void* tm_x_out, const void* tm_v, const void* tm_shadow,
                                float B, float lr, float mu, float wd, float lambda_dc, float disp_scale, int max_ctas,
                                cudaStream_t stream, bool chained);
+// The same step for the rest of the vector (b1, W2, b2) from the pooled per-micro-batch partials; also moves the
+// set's device counters cnt[0..W) into log_row and clears them.  x_in, x_out, v, shadow_out: whole flat vectors.
+cudaError_t launch_mlp_sync_small(const MlpDims& d, const MlpPool& pool, const MlpSlots& slots, int nb, const float* x_in,
+                                  float* x_out, float* v, __nv_bfloat16* shadow_out, float B, float lr, float mu, float wd,
+                                  float lambda_dc, float disp_scale, int32_t* cnt, int32_t* log_row, int W, cudaStream_t stream,
+                                  bool chained);
 // The gradient of a call is enqueued in three parts so that the caller can put them on different streams:
 //   cast:  the only part that reads the caller's x_dev / y_dev (bf16 copies and labels into this scratch set);
 //   front: forward GEMM, loss, layer-2 backward (writes dzt of this scratch set; adds db2, db1, dW2 into

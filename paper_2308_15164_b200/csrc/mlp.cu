@@ -993,6 +993,37 @@ __global__ void __launch_bounds__(64 + kStepEpiThreads) k_sync_w1(const __grid_c
     }
 }
 
+// The bias / W2 part of the same step (everything behind W1 in the flat vector), straight from the pooled
+// per-micro-batch partials: sum_i G_t^i restricted to that part is the sum over all slots of db1 | dW2 | db2, added
+// here in slot order, then the same update.  One thread per parameter; CTA 0 also moves the device counters b_i of
+// the set into the consumed-count log and clears them (nothing in this step reads them: B comes from the host).
+__global__ void __launch_bounds__(256) k_sync_small_pooled(const float* __restrict__ part, size_t part_stride,
+                                                           const __grid_constant__ MlpSlots sl, int n,
+                                                           const float* x_in, float* x_out, float* v,
+                                                           __nv_bfloat16* shadow, int n_small, W1StepCoef cf, int32_t* cnt,
+                                                           int32_t* log_row, int W) {
+    const int t = blockIdx.x * 256 + threadIdx.x;
+    pdl_wait();
+    pdl_trigger();
+    if (t < n_small) {
+        float sum = 0.f;
+        for (int q = 0; q < n; ++q) sum += part[(size_t)sl.s[q] * part_stride + t];
+        float g = sum * cf.inv_B;
+        float vv = v[t], x = x_in[t];
+        if (cf.lambda_dc != 0.0f) g += (-cf.lambda_dc * cf.disp_scale) * g * g * vv;   // Eq. 6
+        g += cf.wd * x;
+        vv = cf.mu * vv + g;
+        x -= cf.lr * vv;
+        v[t] = vv;
+        x_out[t] = x;
+        if (shadow) shadow[t] = __float2bfloat16_rn(x);
+    }
+    if (blockIdx.x == 0 && threadIdx.x < W) {
+        log_row[threadIdx.x] = cnt[threadIdx.x];
+        cnt[threadIdx.x] = 0;
+    }
+}
+
 // ============================================================================================
 // Forward GEMM on tcgen05:  zpart[s][h][r] = sum_{k in split s} W1b[k][h] * xb[r][k]
 //   D [M = 128 hidden][N = 64 samples] += A B^T with
@@ -1320,6 +1351,20 @@ cudaError_t mlp_make_shadow_tmap(void* tmap_out, const MlpDims& d, __nv_bfloat16
                      kTileM, 64)
                ? cudaSuccess
                : cudaErrorInvalidValue;
+}
+
+cudaError_t launch_mlp_sync_small(const MlpDims& d, const MlpPool& pool, const MlpSlots& slots, int nb, const float* x_in,
+                                  float* x_out, float* v, __nv_bfloat16* shadow_out, float B, float lr, float mu, float wd,
+                                  float lambda_dc, float disp_scale, int32_t* cnt, int32_t* log_row, int W, cudaStream_t stream,
+                                  bool chained) {
+    if (nb < 1 || nb > kMlpMaxSlots) return cudaErrorInvalidValue;
+    const size_t w1 = (size_t)d.d_in * d.d_hidden;
+    const int n_small = d.d_hidden + d.d_hidden * d.d_out + d.d_out;
+    const W1StepCoef cf{1.0f / B, lr, mu, wd, lambda_dc, disp_scale};
+    const float* part = pool.part;
+    const float* xi = x_in + w1;
+    return launch_kernel(k_sync_small_pooled, (n_small + 255) / 256, 256, 0, stream, chained, part, pool.part_stride, slots, nb, xi,
+                         x_out + w1, v + w1, shadow_out ? shadow_out + w1 : nullptr, n_small, cf, cnt, log_row, W);
 }
 
 cudaError_t launch_mlp_sync_w1(const MlpDims& d, const MlpScratch& s, const MlpPool& pool, const MlpSlots& slots, int nb,
