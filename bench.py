@@ -871,11 +871,13 @@ def run_mlp(B, wlm, dev, peaks, iters=12):
                      ("batch_calls_up_to_4", dict(max_batch=4)),
                      ("batch_calls_up_to_4_overwrite_first", dict(max_batch=4, overwrite_first=True)),
                      ("batch_calls_up_to_4_deep_pipelines", dict(max_batch=4, variant=128)),
+                     ("batch_calls_up_to_8", dict(max_batch=8)),
                      # ABS_FLAG_MLP_DEFER: Step 1 of the W1 slice straight from the pooled dW1 operands (one contraction
                      # over all micro-batches of the iteration inside the update kernel) ...
                      ("deferred_single_calls", dict(max_batch=1, defer="pool")),
                      ("deferred_single_calls_gathered_by_the_library", dict(max_batch=1, coalesce=True, defer="pool")),
                      ("deferred_batch_calls_up_to_4", dict(max_batch=4, defer="pool")),
+                     ("deferred_batch_calls_up_to_8", dict(max_batch=8, defer="pool")),
                      # ... or one dW1 contraction per worker and iteration into the rows (K = 64 b_i), then the row-based step
                      ("deferred_rows_single_calls", dict(max_batch=1, defer="rows")),
                      ("deferred_rows_batch_calls_up_to_4", dict(max_batch=4, defer="rows"))):

@@ -202,7 +202,7 @@ int abs_accumulate_host(abs_ctx *ctx, uint32_t worker, const void *grad_host);
  * abs_accumulate, abs_accumulate_host and abs_accumulator make stream_acc wait for all of them. */
 int abs_accumulate_mlp(abs_ctx *ctx, uint32_t worker, const void *x_dev, const int32_t *y_dev);
 
-/* n (1..4) consecutive reference batches of one worker in one call: the same computation as n calls of
+/* n (1..8) consecutive reference batches of one worker in one call: the same computation as n calls of
  * abs_accumulate_mlp (forward, loss and backward of every micro-batch at x_t; b_i += n), but the n dW1
  * products are contracted by ONE tcgen05 GEMM with K = 64 n, so the worker's fp32 accumulator slice is
  * read and written once instead of n times -- that traffic, not the MMAs, bounds the kernel.  The sum

@@ -187,7 +187,7 @@ struct abs_ctx {
     // ABS_FLAG_MLP_COALESCE: single calls of a worker wait, already cast into consecutive slots of one scratch
     // set, until four have gathered (or something needs the accumulator), then run as one batch call.
     bool coalesce = false;
-    int pend_n[kMaxW] = {};        // micro-batches of worker i waiting (0..kMlpMaxBatch)
+    int pend_n[kMaxW] = {};        // micro-batches of worker i waiting (0..kMlpGatherMax)
     int pend_set[kMaxW] = {};      // scratch set that holds them
     bool pend_first[kMaxW] = {};   // they open the worker's iteration (the row holds nothing yet)
     bool set_reserved[kMlpSets] = {};
@@ -641,7 +641,7 @@ void turn_sets(abs_ctx* c, uint32_t closing, uint32_t opening) {
 int coalesce_one(abs_ctx* c, uint32_t worker, const void* x_dev, const int32_t* y_dev) {
     if (c->pend_n[worker] == 0) {
         if (c->defer) {   // the group waits in consecutive pool slots (unused ones stay empty)
-            if (int rc = take_pool_slots(c, kMlpMaxBatch, &c->pend_pool0[worker])) return rc;
+            if (int rc = take_pool_slots(c, kMlpGatherMax, &c->pend_pool0[worker])) return rc;
             c->pend_set[worker] = 0;
         } else {
             if (c->n_reserved >= kMlpSets / 2) {   // keep half of the scratch sets for groups that are running
@@ -665,7 +665,7 @@ int coalesce_one(abs_ctx* c, uint32_t worker, const void* x_dev, const int32_t* 
                        (c->mlp_chain(false, 1) & kChainCast) != 0, mlp_mark, c));
     c->pend_n[worker] = slot + 1;
     c->h_cnt[(size_t)c->cur * c->cfg.W + worker] += 1;
-    if (c->pend_n[worker] == kMlpMaxBatch) return flush_worker(c, worker);
+    if (c->pend_n[worker] == kMlpGatherMax) return flush_worker(c, worker);
     return ABS_OK;
 }
 
@@ -873,7 +873,7 @@ int abs_accumulate_mlp_batch(abs_ctx* c, uint32_t worker, uint32_t n, const void
     if (!live(c)) return ABS_ESTATE;
     if (!c->mlp) return invalid(c, "context was created without ABS_FLAG_MLP");
     if (worker >= c->cfg.W) return invalid(c, "worker index out of range");
-    if (n == 0 || n > (uint32_t)kMlpMaxBatch) return invalid(c, "n must be in 1..4");
+    if (n == 0 || n > (uint32_t)kMlpMaxBatch) return invalid(c, "n must be in 1..8");
     if (!x_dev || (reinterpret_cast<uintptr_t>(x_dev) & 15)) return invalid(c, "x pointer must be non-NULL and 16-byte aligned");
     if (!y_dev || (reinterpret_cast<uintptr_t>(y_dev) & 3)) return invalid(c, "y pointer must be non-NULL and 4-byte aligned");
     const bool serial = c->ctas_per_sm[ABS_K_MLP_FWD] == 1;   // measurement aid: everything on stream_acc

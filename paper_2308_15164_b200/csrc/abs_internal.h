@@ -123,7 +123,8 @@ cudaError_t launch_global_counts(int32_t* gcnt, int32_t* cnt, int own_lo, int W_
 cudaError_t launch_cast_bf16(const float* src, __nv_bfloat16* dst, size_t n, int num_sms, cudaStream_t stream);
 
 // ---- MLP micro-batch gradient (Step 2 with the gradient computed on the device) ----------
-constexpr int kMlpMaxBatch = 4;
+constexpr int kMlpMaxBatch = 8;     // micro-batches one gradient call may carry
+constexpr int kMlpGatherMax = 4;    // micro-batches ABS_FLAG_MLP_COALESCE gathers into one group
 // Internal bit of the `variant` argument below (set by the context, never by abs_set_launch): forward GEMM and ring
 // dW1 kernel in their light shared-memory configurations, so that CTAs of different workers' calls share an SM.
 constexpr int kMlpLightBit = 256;

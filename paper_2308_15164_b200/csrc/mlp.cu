@@ -1041,9 +1041,10 @@ __global__ void __launch_bounds__(256) k_sync_small_pooled(const float* __restri
 // kLight: 2 - 3 stages (72 - 96 KB) instead of 4 - 6, so that a dW1 CTA of another worker's call fits beside it.
 template <int NB, bool kLight = false>
 struct FwdCfg {
-    static constexpr int kStages = kLight ? (NB <= 2 ? 3 : 2) : (NB <= 2 ? 6 : (NB == 3 ? 5 : 4));   // <= 200 KB of stages
     static constexpr int kStageBytes = 2 * 8192 + NB * 8192;              // two A boxes + NB B boxes
-    static constexpr int kTmemCols = NB == 1 ? 64 : (NB == 2 ? 128 : 256);   // power of two >= 64 NB
+    // <= 200 KB of stages (deep) / about 100 KB (light; 160 KB for more than four micro-batches)
+    static constexpr int kStages = kLight ? (NB <= 2 ? 3 : 2) : (NB <= 2 ? 6 : (NB == 3 ? 5 : (NB == 4 ? 4 : (NB <= 6 ? 3 : 2))));
+    static constexpr int kTmemCols = NB == 1 ? 64 : (NB == 2 ? 128 : (NB <= 4 ? 256 : 512));   // power of two >= 64 NB
 };
 
 template <int NB, bool kLight = false>
@@ -1111,7 +1112,11 @@ __global__ void __launch_bounds__(128) k_fwd1_tcgen05(const __grid_constant__ CU
                 tma_load_2d(s.stage[st] + 16384 + jb * 8192, &tm_xb, k0, xb_row0 + jb * kMB, &s.full[st]);
         }
     } else if (warp == 1 && lane == 0) {             // ---- MMA issuer
-        constexpr uint32_t idesc = umma_idesc_bf16(128, 64 * NB) | (1u << 15);   // A is MN-major
+        // N of one instruction is at most 256: the first four micro-batches go into TMEM columns 0..255, the
+        // others (NB > 4) into columns 256.. with a second instruction per K step.
+        constexpr int kN0 = NB <= 4 ? 64 * NB : 256, kN1 = NB <= 4 ? 0 : 64 * (NB - 4);
+        constexpr uint32_t idesc = umma_idesc_bf16(128, kN0) | (1u << 15);   // A is MN-major
+        constexpr uint32_t idesc1 = umma_idesc_bf16(128, kN1 > 0 ? kN1 : 64) | (1u << 15);
         bool ok = true;
         for (int kb = 0; kb < nk && ok; ++kb) {
             const int st = kb % kFwdStages;
@@ -1121,8 +1126,12 @@ __global__ void __launch_bounds__(128) k_fwd1_tcgen05(const __grid_constant__ CU
             const uint32_t a0 = smem_u32(s.stage[st]);
             const uint64_t db = umma_desc_k_sw128(a0 + 16384);
 #pragma unroll
-            for (int k = 0; k < 4; ++k)
+            for (int k = 0; k < 4; ++k) {
                 umma_bf16(tmem, umma_desc_mn_sw128(a0 + k * 2048, 8192), db + 2 * k, idesc, (kb > 0 || k > 0));
+                if (kN1 > 0)
+                    umma_bf16(tmem + 256, umma_desc_mn_sw128(a0 + k * 2048, 8192), umma_desc_k_sw128(a0 + 16384 + 4 * 8192) + 2 * k,
+                              idesc1, (kb > 0 || k > 0));
+            }
             umma_commit(&s.empty[st]);               // frees the stage once these MMAs have read it
         }
         if (ok) umma_commit(&s.done);
@@ -1291,6 +1300,10 @@ cudaError_t mlp_scratch_init(MlpScratch* s, const MlpDims& d, void* base, __nv_b
     if (e == cudaSuccess) e = fwd1_set_attr<2>();
     if (e == cudaSuccess) e = fwd1_set_attr<3>();
     if (e == cudaSuccess) e = fwd1_set_attr<4>();
+    if (e == cudaSuccess) e = fwd1_set_attr<5>();
+    if (e == cudaSuccess) e = fwd1_set_attr<6>();
+    if (e == cudaSuccess) e = fwd1_set_attr<7>();
+    if (e == cudaSuccess) e = fwd1_set_attr<8>();
     if (e != cudaSuccess) *err = "cudaFuncSetAttribute(tcgen05 kernels)";
     return e;
 }
@@ -1436,7 +1449,10 @@ cudaError_t launch_mlp_front(const MlpDims& d, const MlpScratch& s, const float*
 
     // every K split must be a whole number of 64-wide pipeline steps (d_in is a multiple of 128).  Eight splits (256
     // CTAs, two per SM) measured slower than four: 34.7 against 33.4 us per micro-batch, 16.7 against 15.5 batched.
-    int nsplit = kSplitK;
+    // A call of several micro-batches has enough MMA work per CTA with two splits, and every split costs the
+    // call 2 x 1 MB of partial sums per micro-batch (measured, batch calls of up to 4 / 8: 14.5 -> 13.8 / 13.0 -> 12.3 us
+    // per micro-batch; with ABS_FLAG_MLP_DEFER 9.5 -> 9.0 / 9.5 -> 8.8; one split was no better than two).
+    int nsplit = nb == 1 ? kSplitK : 2;
     while (nsplit > 1 && d.d_in % (64 * nsplit) != 0) nsplit /= 2;
     const CUtensorMap& tw = *reinterpret_cast<const CUtensorMap*>(&s.tmap_w1[shadow_idx]);
     const CUtensorMap& tx = *reinterpret_cast<const CUtensorMap*>(pool ? &pool->tmap_xb : &s.tmap_xb);
@@ -1447,7 +1463,12 @@ cudaError_t launch_mlp_front(const MlpDims& d, const MlpScratch& s, const float*
         case 1: e = fwd1_launch<1>(grid, stream, (chain & kChainFwd1) != 0, light, tw, tx, s.zpart, d.d_in, d.d_hidden, xb_row0, s.status); break;
         case 2: e = fwd1_launch<2>(grid, stream, (chain & kChainFwd1) != 0, light, tw, tx, s.zpart, d.d_in, d.d_hidden, xb_row0, s.status); break;
         case 3: e = fwd1_launch<3>(grid, stream, (chain & kChainFwd1) != 0, light, tw, tx, s.zpart, d.d_in, d.d_hidden, xb_row0, s.status); break;
-        default: e = fwd1_launch<4>(grid, stream, (chain & kChainFwd1) != 0, light, tw, tx, s.zpart, d.d_in, d.d_hidden, xb_row0, s.status); break;
+        case 4: e = fwd1_launch<4>(grid, stream, (chain & kChainFwd1) != 0, light, tw, tx, s.zpart, d.d_in, d.d_hidden, xb_row0, s.status); break;
+        case 5: e = fwd1_launch<5>(grid, stream, (chain & kChainFwd1) != 0, light, tw, tx, s.zpart, d.d_in, d.d_hidden, xb_row0, s.status); break;
+        case 6: e = fwd1_launch<6>(grid, stream, (chain & kChainFwd1) != 0, light, tw, tx, s.zpart, d.d_in, d.d_hidden, xb_row0, s.status); break;
+        case 7: e = fwd1_launch<7>(grid, stream, (chain & kChainFwd1) != 0, light, tw, tx, s.zpart, d.d_in, d.d_hidden, xb_row0, s.status); break;
+        case 8: e = fwd1_launch<8>(grid, stream, (chain & kChainFwd1) != 0, light, tw, tx, s.zpart, d.d_in, d.d_hidden, xb_row0, s.status); break;
+        default: return cudaErrorInvalidValue;
     }
     mark(user, ABS_K_MLP_FWD, 1, stream);
     if (e != cudaSuccess) return e;

@@ -88,3 +88,33 @@ def test_a_wait_that_runs_out_is_reported_and_leaves_the_context_usable():
     got = eng.params_host()
     assert np.allclose(got, 1.0 - 0.1 * 2.0, rtol=0, atol=1e-6)
     eng.destroy()
+
+
+def test_mlp_batch_call_argument_checks():
+    """abs_accumulate_mlp_batch takes 1..8 micro-batches, aligned non-null device pointers and a worker in range;
+    a rejected call launches nothing and counts nothing."""
+    import torch
+
+    from paper_2308_15164_b200 import binding as B
+    from paper_2308_15164_b200 import workloads as wlm
+
+    wl = wlm.config(4, small=True)
+    d = wl.mlp
+    x0 = torch.from_numpy(wlm.params0(wl)).cuda()
+    x = torch.zeros((9, d.mb, d.d_in), device="cuda")
+    y = torch.zeros((9, d.mb), dtype=torch.int32, device="cuda")
+    for defer in (False, True):
+        eng = B.AbsSgd(x0, wl.W, wl.lr, mlp=(d.d_in, d.d_hidden, d.d_out, d.mb), mlp_defer=defer)
+        h = eng._h
+        n0 = eng.launch_count()
+        assert B.lib.abs_accumulate_mlp_batch(h, 0, 0, x.data_ptr(), y.data_ptr()) == B.EINVAL
+        assert B.lib.abs_accumulate_mlp_batch(h, 0, 9, x.data_ptr(), y.data_ptr()) == B.EINVAL
+        assert B.lib.abs_accumulate_mlp_batch(h, wl.W, 1, x.data_ptr(), y.data_ptr()) == B.EINVAL
+        assert B.lib.abs_accumulate_mlp_batch(h, 0, 1, None, y.data_ptr()) == B.EINVAL
+        assert B.lib.abs_accumulate_mlp_batch(h, 0, 1, x.data_ptr() + 4, y.data_ptr()) == B.EINVAL
+        assert B.lib.abs_accumulate_mlp_batch(h, 0, 1, x.data_ptr(), None) == B.EINVAL
+        assert eng.launch_count() == n0 and not eng.counters()[0].any()
+        assert B.lib.abs_accumulate_mlp_batch(h, 0, 8, x.data_ptr(), y.data_ptr()) == B.OK
+        assert eng.counters()[0][eng.counters()[1]].tolist() == [8, 0, 0, 0]
+        eng.check()
+        eng.destroy()

@@ -415,7 +415,7 @@ def test_training_run_matches_oracle(small, T):
 
 
 @pytest.mark.parametrize("epilogue", [0, 8, 4, 36], ids=["auto", "tile-per-cta", "persistent-ring-128x128", "persistent-ring-128x64"])
-@pytest.mark.parametrize("n", [2, 3, 4])
+@pytest.mark.parametrize("n", [2, 3, 4, 5, 8])
 @pytest.mark.parametrize("small", [True, False], ids=["384x512", "3072x4096"])
 def test_batched_microbatches_match_the_sum_of_gradients(small, n, epilogue):
     """abs_accumulate_mlp_batch: n reference batches of one worker contracted by one K = 64 n GEMM give the sum
@@ -452,13 +452,20 @@ def test_batched_microbatches_match_the_sum_of_gradients(small, n, epilogue):
     if undecided:
         u = sorted(undecided)
         assert np.abs(gW1[:, u] - wW1[:, u]).max() <= 0.2 * np.abs(wW1).max()
-    # and the same data through n single calls agrees to fp32 rounding of the sums
+    # and the same data through n single calls: a batch call forms Z from two split-K partial sums, a single call
+    # from four, so Z agrees to fp32 rounding only, and an H or dZ entry that sits within that of a bf16 rounding
+    # midpoint may round the other way (valid either way, as against the oracle): one bf16 unit of one of the
+    # 64 n terms of a dW1 column, and -- through the logits -- a last-digit change of that sample's dL row.  The two
+    # paths therefore agree at half the bar against the oracle element-wise and a quarter of it in norm (measured:
+    # 6e-4 and 1e-4), not to fp32 rounding.
     eng2 = _engine(wl, x0, epilogue=epilogue)
     for j in range(n):
         eng2.accumulate_mlp(3, xd[j], yd[j])
     eng2.check()
     single = eng2.accumulator(0, 3).cpu().numpy().astype(np.float64)
-    assert np.abs(got - single).max() <= 1e-5 * np.abs(single).max()
+    diff = np.abs(got - single)
+    assert diff.max() <= 1e-3 * np.abs(single).max()
+    assert np.linalg.norm(got - single) <= 5e-4 * np.linalg.norm(single)
     # a second call on the same worker takes the adding path: the row doubles
     eng.accumulate_mlp_batch(3, n, xd, yd)
     eng.check()
