@@ -445,9 +445,9 @@ int take_scratch_set(abs_ctx* c, bool serial, int* out) {
     return ABS_OK;
 }
 
-// Forward, loss, backward and dW1 of the n micro-batches that sit, cast, in slots 0..n-1 of scratch set `set`,
-// on the worker's internal stream (which first waits for everything enqueued on stream_acc so far, the casts
-// included).  deferred: the casts were launched, and counted, by earlier calls.
+// Forward, loss, backward and dW1 of the n micro-batches that sit, cast, in slots 0..n-1 of scratch set `set`
+// (ABS_FLAG_MLP_DEFER: in pool slots pool0.. of the current accumulator set, and without the dW1), on an internal
+// stream, which first waits for everything enqueued on stream_acc so far, the casts included.
 int run_mlp_group(abs_ctx* c, uint32_t worker, int set, int n, bool first, int pool0) {
     int k = (int)(worker % (uint32_t)c->n_wstreams);
     int variant = c->ctas_per_sm[ABS_K_MLP_DW1];
