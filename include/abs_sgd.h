@@ -118,7 +118,8 @@ extern "C" {
                                      stay as they are: zero, or stale with ABS_FLAG_OVERWRITE_FIRST).  Otherwise the rows are completed first and the
                                      row-based step runs.  Either way the result equals that of the per-call path to
                                      fp32 rounding (one fp32 accumulation over K instead of rounded additions into the
-                                     row).  Combines with every other flag.                                         */
+                                     row).  Combines with every other flag; with ABS_FLAG_MLP_COALESCE single calls are
+                                     gathered four at a time whoever their workers are.                             */
 
 #define ABS_MAX_WORKERS 64u
 #define ABS_MAX_RANKS   16u   /* GPUs taking part in abs_global_* (n_ranks * W <= ABS_MAX_WORKERS)        */

@@ -202,10 +202,12 @@ struct abs_ctx {
     MlpPool pool[2]{};
     int pool_n[2] = {0, 0};                   // slots handed out (bump allocation; back to 0 when the iteration ends)
     std::vector<int16_t> pool_owner[2];       // worker whose micro-batch sits in the slot; -1: none (contracted, or never used)
-    int pend_pool0[kMaxW] = {};               // first pool slot of a waiting group (ABS_FLAG_MLP_COALESCE)
     // In this mode a call adds nothing to its worker's row, so calls need no order among themselves: call after call
     // takes the next of the kMlpStreams internal streams (and that stream's scratch set), whoever the worker is.
     int rr_stream = 0;
+    // ... and ABS_FLAG_MLP_COALESCE gathers single calls into one group whoever their workers are
+    int grp_n = 0, grp_pool0 = 0;
+    MlpWorkers grp_workers{};
     bool d_outstanding[kMlpStreams] = {};     // contractions enqueued on s_d[k] since stream_acc last waited for it
     cudaEvent_t ev_d_done[kMlpStreams] = {};
     bool w1_touched[2][kMaxW] = {};           // the row's W1 slice has been written in the set's current iteration
@@ -448,7 +450,7 @@ int take_scratch_set(abs_ctx* c, bool serial, int* out) {
 // Forward, loss, backward and dW1 of the n micro-batches that sit, cast, in slots 0..n-1 of scratch set `set`
 // (ABS_FLAG_MLP_DEFER: in pool slots pool0.. of the current accumulator set, and without the dW1), on an internal
 // stream, which first waits for everything enqueued on stream_acc so far, the casts included.
-int run_mlp_group(abs_ctx* c, uint32_t worker, int set, int n, bool first, int pool0) {
+int run_mlp_group(abs_ctx* c, uint32_t worker, int set, int n, bool first, int pool0, const MlpWorkers* mixed = nullptr) {
     int k = (int)(worker % (uint32_t)c->n_wstreams);
     int variant = c->ctas_per_sm[ABS_K_MLP_DW1];
     const bool serial = c->ctas_per_sm[ABS_K_MLP_FWD] == 1;
@@ -466,10 +468,12 @@ int run_mlp_group(abs_ctx* c, uint32_t worker, int set, int n, bool first, int p
             CK(cudaEventRecord(c->ev_fork, c->s_acc));
             CK(cudaStreamWaitEvent(s_run, c->ev_fork, 0));
         }
+        MlpWorkers wk{};
+        for (int j = 0; j < n; ++j) wk.w[j] = mixed ? mixed->w[j] : (uint8_t)worker;
         CK(launch_mlp_front(c->mlp_dims, c->mlp_scratch[k], c->x(c->pub), c->shadow(c->pub), c->pub, n, first,
-                            c->acc(c->cur, worker), c->cnt(c->cur, worker), &c->pool[c->cur], pool0, variant, s_run,
+                            c->acc(c->cur, worker), c->cnt(c->cur, 0), &c->pool[c->cur], pool0, &wk, variant, s_run,
                             c->mlp_chain(serial, n), mlp_mark, c));
-        for (int j = 0; j < n; ++j) c->pool_owner[c->cur][pool0 + j] = (int16_t)worker;
+        for (int j = 0; j < n; ++j) c->pool_owner[c->cur][pool0 + j] = (int16_t)wk.w[j];
         if (!serial) c->w_outstanding[k] = true;
         return ABS_OK;
     }
@@ -480,7 +484,7 @@ int run_mlp_group(abs_ctx* c, uint32_t worker, int set, int n, bool first, int p
         CK(cudaStreamWaitEvent(s_run, c->ev_fork, 0));
     }
     CK(launch_mlp_front(c->mlp_dims, sc, c->x(c->pub), c->shadow(c->pub), c->pub, n, first, c->acc(c->cur, worker),
-                        c->cnt(c->cur, worker), nullptr, 0, variant, s_run, c->mlp_chain(serial, n), mlp_mark, c));
+                        c->cnt(c->cur, worker), nullptr, 0, nullptr, variant, s_run, c->mlp_chain(serial, n), mlp_mark, c));
     cudaStream_t s_gemm = s_run;
     if (!serial) {   // dW1 on the worker's second (lowest-priority) stream, behind the front kernels of this call
         s_gemm = c->s_d[k];
@@ -510,12 +514,17 @@ int flush_worker(abs_ctx* c, uint32_t worker) {
     if (n == 0) return ABS_OK;
     const int set = c->pend_set[worker];
     c->pend_n[worker] = 0;
-    if (!c->defer) c->set_reserved[set] = false;
+    c->set_reserved[set] = false;
     c->n_reserved -= 1;
-    return run_mlp_group(c, worker, set, n, c->pend_first[worker], c->pend_pool0[worker]);
+    return run_mlp_group(c, worker, set, n, c->pend_first[worker], 0);
 }
 
 int flush_all(abs_ctx* c) {
+    if (c->grp_n > 0) {   // deferred mode: the one group of gathered single calls
+        const int n = c->grp_n;
+        c->grp_n = 0;
+        if (int rc = run_mlp_group(c, c->grp_workers.w[0], 0, n, false, c->grp_pool0, &c->grp_workers)) return rc;
+    }
     if (c->n_reserved == 0) return ABS_OK;
     for (;;) {   // oldest group first: the order does not change results (rows are independent), only timing
         int best = -1;
@@ -639,11 +648,22 @@ void turn_sets(abs_ctx* c, uint32_t closing, uint32_t opening) {
 // One micro-batch of `worker` joins its waiting group: cast now (the caller's buffers are free again once
 // stream_acc has passed this point), everything else when the group runs.
 int coalesce_one(abs_ctx* c, uint32_t worker, const void* x_dev, const int32_t* y_dev) {
+    if (c->defer) {
+        // Deferred calls are independent of their workers: ONE group gathers the next kMlpGatherMax single calls,
+        // whoever makes them, in consecutive pool slots (slots a group leaves unused stay empty).  (Groups of eight
+        // measured slower than groups of four: 10.8 against 10.1 us per micro-batch -- the forward GEMM of a group
+        // starts later and the last group of an iteration holds the step back longer.)
+        if (c->grp_n == 0)
+            if (int rc = take_pool_slots(c, kMlpGatherMax, &c->grp_pool0)) return rc;
+        CK(launch_mlp_cast(c->mlp_dims, c->mlp_scratch[0], c->grp_pool0 + c->grp_n, 1, x_dev, c->x_bf16(), y_dev, &c->pool[c->cur],
+                           c->s_acc, (c->mlp_chain(false, 1) & kChainCast) != 0, mlp_mark, c));
+        c->grp_workers.w[c->grp_n++] = (uint8_t)worker;
+        c->h_cnt[(size_t)c->cur * c->cfg.W + worker] += 1;
+        if (c->grp_n == kMlpGatherMax) return flush_all(c);
+        return ABS_OK;
+    }
     if (c->pend_n[worker] == 0) {
-        if (c->defer) {   // the group waits in consecutive pool slots (unused ones stay empty)
-            if (int rc = take_pool_slots(c, kMlpGatherMax, &c->pend_pool0[worker])) return rc;
-            c->pend_set[worker] = 0;
-        } else {
+        {
             if (c->n_reserved >= kMlpSets / 2) {   // keep half of the scratch sets for groups that are running
                 int oldest = -1;
                 for (uint32_t i = 0; i < c->cfg.W; ++i)
@@ -660,8 +680,7 @@ int coalesce_one(abs_ctx* c, uint32_t worker, const void* x_dev, const int32_t* 
         c->pend_age[worker] = ++c->pend_clock;
     }
     const int slot = c->pend_n[worker];
-    CK(launch_mlp_cast(c->mlp_dims, c->mlp_scratch[c->pend_set[worker]], c->defer ? c->pend_pool0[worker] + slot : slot, 1, x_dev,
-                       c->x_bf16(), y_dev, c->defer ? &c->pool[c->cur] : nullptr, c->s_acc,
+    CK(launch_mlp_cast(c->mlp_dims, c->mlp_scratch[c->pend_set[worker]], slot, 1, x_dev, c->x_bf16(), y_dev, nullptr, c->s_acc,
                        (c->mlp_chain(false, 1) & kChainCast) != 0, mlp_mark, c));
     c->pend_n[worker] = slot + 1;
     c->h_cnt[(size_t)c->cur * c->cfg.W + worker] += 1;

@@ -142,6 +142,9 @@ constexpr int kMlpMaxSlots = 128;
 struct MlpSlots {
     uint16_t s[kMlpMaxSlots];
 };
+struct MlpWorkers {      // worker of each micro-batch of a pooled gradient call
+    uint8_t w[8];
+};
 struct alignas(64) TmapBytes {   // storage for one CUtensorMap (encoded on the host, passed by value to kernels)
     unsigned char b[128];
 };
@@ -215,13 +218,14 @@ cudaError_t launch_mlp_sync_small(const MlpDims& d, const MlpPool& pool, const M
 typedef void (*MlpMark)(void* user, int kernel_class, int n, cudaStream_t stream);
 // pool (ABS_FLAG_MLP_DEFER): the cast writes into pool slots slot0.. instead of the scratch set's; the front kernels
 // read them there (pool_slot0..), leave bf16(dZ)^T and the micro-batches' db1 | dW2 | db2 there and add nothing to
-// acc_row (only cnt is bumped, atomically).
+// acc_row; cnt is then the counter array of the whole set, and micro-batch j bumps cnt[workers->w[j]], atomically.
 cudaError_t launch_mlp_cast(const MlpDims& d, const MlpScratch& s, int slot0, int nb, const void* x_dev, bool x_is_bf16,
                             const int32_t* y_dev, const MlpPool* pool, cudaStream_t stream, bool chained, MlpMark mark,
                             void* user);
 cudaError_t launch_mlp_front(const MlpDims& d, const MlpScratch& s, const float* x_pub, const __nv_bfloat16* shadow,
                              int shadow_idx, int nb, bool store, float* acc_row, int32_t* cnt, const MlpPool* pool,
-                             int pool_slot0, int variant, cudaStream_t stream, int chain, MlpMark mark, void* user);
+                             int pool_slot0, const MlpWorkers* workers, int variant, cudaStream_t stream, int chain, MlpMark mark,
+                             void* user);
 // Bias / W2 part of the rows of workers first_worker .. first_worker + n_workers - 1 of one accumulator set from the
 // pooled per-micro-batch partials: row = (keep_mask bit ? row : 0) + sum of the partials of the worker's slots
 // (owners[q] = worker of slots.s[q]), in list order.

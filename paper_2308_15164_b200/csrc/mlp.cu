@@ -189,7 +189,8 @@ __global__ void __launch_bounds__(256) k_bwd(const __nv_bfloat16* hbt, const flo
                                              const float* __restrict__ b2, const int32_t* y,
                                              const __nv_bfloat16* __restrict__ w2b, __nv_bfloat16* dzt, float* bpart,
                                              unsigned int* tickets_b, float* acc_b1, float* acc_w2, float* acc_b2,
-                                             int32_t* cnt, int d_h, int d_out, int store, float* part, size_t part_stride) {
+                                             int32_t* cnt, int d_h, int d_out, int store, float* part, size_t part_stride,
+                                             MlpWorkers wk) {
     __shared__ float sdl[kMB][kOutPad + 1];     // bf16(dL) as float
     __shared__ float sdl32[kMB][kOutPad + 1];   // dL unrounded (CTA 0: db2)
     __shared__ float sw2[kHB][kOutPad];
@@ -288,7 +289,9 @@ __global__ void __launch_bounds__(256) k_bwd(const __nv_bfloat16* hbt, const flo
             if (slot + 8 < d_out) mine[d_h + (size_t)h * d_out + slot + 8] = b;
             if (slot == 0) mine[h] = c;
             if (blockIdx.x == 0 && threadIdx.x < d_out) mine[d_h + (size_t)d_h * d_out + threadIdx.x] = db2;
-            if (blockIdx.x == 0 && jb == 0 && threadIdx.x == 0) atomicAdd(cnt, nb);   // M_t^i += nb * M_r
+            // M_t^i += M_r for the worker this micro-batch belongs to (cnt: the set's counters; a gathered group may
+            // hold micro-batches of several workers)
+            if (blockIdx.x == 0 && threadIdx.x == 0) atomicAdd(cnt + wk.w[jb], 1);
             return;
         }
         if (nb > 1) {
@@ -1441,7 +1444,8 @@ cudaError_t fwd1_launch(dim3 grid, cudaStream_t stream, bool chained, bool light
 
 cudaError_t launch_mlp_front(const MlpDims& d, const MlpScratch& s, const float* x_pub, const __nv_bfloat16* shadow,
                              int shadow_idx, int nb, bool store, float* acc_row, int32_t* cnt, const MlpPool* pool,
-                             int pool_slot0, int variant, cudaStream_t stream, int chain, MlpMark mark, void* user) {
+                             int pool_slot0, const MlpWorkers* workers, int variant, cudaStream_t stream, int chain, MlpMark mark,
+                             void* user) {
     const size_t o_b1 = (size_t)d.d_in * d.d_hidden, o_w2 = o_b1 + d.d_hidden, o_b2 = o_w2 + (size_t)d.d_hidden * d.d_out;
     cudaError_t e;
     const unsigned n_cta = d.d_hidden / kHB;
@@ -1492,7 +1496,7 @@ cudaError_t launch_mlp_front(const MlpDims& d, const MlpScratch& s, const float*
     const size_t part_stride = pool ? pool->part_stride : 0;
     e = launch_kernel(k_bwd, dim3(n_cta, nb), 256, 0, stream, (chain & kChainBwd) != 0, hbt, gpart, n_groups, b2, yc, w2b, dzt, s.bpart,
                       s.tickets_b, acc_row + o_b1, acc_row + o_w2, acc_row + o_b2, cnt, d.d_hidden, d.d_out, store ? 1 : 0, part,
-                      part_stride);
+                      part_stride, workers ? *workers : MlpWorkers{});
     mark(user, ABS_K_MLP_BWD, 1, stream);
     return e;
 }

@@ -350,3 +350,34 @@ def test_eager_mode_reading_a_closed_set_that_still_waits_in_pooled_form():
     for s in range(len(its) + 1):
         assert np.array_equal(eng.consumed(s), o.consumed[s])
     eng.destroy()
+
+
+def test_gathered_single_calls_of_several_workers_share_a_group():
+    """ABS_FLAG_MLP_COALESCE with ABS_FLAG_MLP_DEFER gathers consecutive single calls four at a time whoever their
+    workers are: every worker's b_i and row must still be its own."""
+    import torch
+
+    wl = wlm.config(4, small=True, T=1)
+    x0 = wlm.params0(wl)
+    xs, ys = wlm.mlp_batches(wl)
+    xs_d, ys_d = torch.from_numpy(xs).cuda(), torch.from_numpy(ys).cuda()
+    eng = _engine(wl, x0, pipelined=True, coalesce=True)
+    order = [2, 0, 2, 3, 3, 0, 2, 2, 0, 3, 2]        # 11 calls: two full groups and one of three; worker 1 idle
+    ref = {}
+    for c, i in enumerate(order):
+        eng.accumulate_mlp(i, xs_d[c], ys_d[c])
+        ref[i] = ref.get(i, 0) + _grad(x0, xs, ys, c, wl)
+    cur = eng.counters()[1]
+    assert eng.counters()[0][cur].tolist() == [3, 0, 5, 3]
+    for i, want in ref.items():
+        _close_row(eng.accumulator(cur, i).cpu().numpy(), want, wl, f"worker {i}")
+    assert not eng.accumulator(cur, 1).any()
+    o = AbsSgdOracle(x0, wl.W, wl.lr, wl.momentum, wl.weight_decay)
+    for c, i in enumerate(order):
+        o.accumulate(i, _grad(x0, xs, ys, c, wl))
+    for _ in range(2):
+        eng.sync_step(); o.sync_step()
+    eng.check()
+    assert np.array_equal(eng.consumed(1), np.array([3, 0, 5, 3]))
+    assert np.abs(eng.params_host().astype(np.float64) - o.params()).max() <= TOL * np.abs(o.params()).max()
+    eng.destroy()
