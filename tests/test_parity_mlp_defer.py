@@ -381,3 +381,39 @@ def test_gathered_single_calls_of_several_workers_share_a_group():
     assert np.array_equal(eng.consumed(1), np.array([3, 0, 5, 3]))
     assert np.abs(eng.params_host().astype(np.float64) - o.params()).max() <= TOL * np.abs(o.params()).max()
     eng.destroy()
+
+
+@pytest.mark.parametrize("defer", [False, True], ids=["per-call-dw1", "deferred-dw1"])
+@pytest.mark.parametrize("shape", [(128, 128, 10), (256, 128, 3), (128, 384, 16)])
+def test_smallest_layer_sizes(shape, defer):
+    """One tile in one or both directions, one and sixteen outputs: three iterations against the oracle."""
+    import dataclasses
+
+    import torch
+
+    from paper_2308_15164_b200 import binding as B
+
+    d_in, d_h, d_out = shape
+    dims = wlm.MlpDims(d_in, d_h, d_out, 64)
+    wl = dataclasses.replace(wlm.config(4, small=True, T=3), mlp=dims, P=dims.P)
+    x0 = wlm.params0(wl)
+    xs, ys = wlm.mlp_batches(wl)
+    xs_d, ys_d = torch.from_numpy(xs).cuda(), torch.from_numpy(ys).cuda()
+    o = AbsSgdOracle(x0, wl.W, wl.lr, wl.momentum, wl.weight_decay)
+    eng = B.AbsSgd(torch.from_numpy(x0).cuda(), wl.W, wl.lr, wl.momentum, wl.weight_decay, pipelined=True,
+                   mlp=(d_in, d_h, d_out, 64), mlp_defer=defer)
+    for t, calls in enumerate(wlm.iter_calls(wl)):
+        p = o.params()
+        for (i, k, c) in calls:
+            g = mlp_loss_and_grad(p, xs[c % wl.mlp_pool], ys[c % wl.mlp_pool], d_in, d_h, d_out, mode="bf16")[1].astype(np.float32)
+            o.accumulate(i, g)
+            eng.accumulate_mlp(i, xs_d[c % wl.mlp_pool], ys_d[c % wl.mlp_pool])
+        eng.sync_step(); o.sync_step()
+    eng.sync_step(); o.sync_step()
+    eng.check()
+    ref = o.params()
+    assert np.abs(ref - x0).max() > 1e-4
+    assert np.abs(eng.params_host().astype(np.float64) - ref).max() <= TOL * np.abs(ref).max()
+    for s in range(4):
+        assert np.array_equal(eng.consumed(s), o.consumed[s])
+    eng.destroy()
