@@ -417,3 +417,48 @@ def test_smallest_layer_sizes(shape, defer):
     for s in range(4):
         assert np.array_equal(eng.consumed(s), o.consumed[s])
     eng.destroy()
+
+
+@pytest.mark.parametrize("mode", ["deferred", "deferred-gathered", "deferred-rows", "per-call"])
+def test_twelve_workers(mode):
+    """W = 12 (more workers than internal streams; the row-based step in its chunked form), two of them idle."""
+    import dataclasses
+
+    import torch
+
+    from paper_2308_15164_b200 import binding as B
+
+    W = 12
+    wl = dataclasses.replace(wlm.config(4, small=True, T=3), W=W)
+    d = wl.mlp
+    x0 = wlm.params0(wl)
+    xs, ys = wlm.mlp_batches(wl)
+    xs_d, ys_d = torch.from_numpy(xs).cuda(), torch.from_numpy(ys).cuda()
+    rng = np.random.default_rng(5)
+    sched = rng.integers(0, 4, size=(3, W))
+    sched[:, 3] = 0; sched[:, 7] = 0
+    o = AbsSgdOracle(x0, W, wl.lr, wl.momentum, wl.weight_decay)
+    eng = B.AbsSgd(torch.from_numpy(x0).cuda(), W, wl.lr, wl.momentum, wl.weight_decay, pipelined=True,
+                   mlp=(d.d_in, d.d_hidden, d.d_out, d.mb), mlp_defer=mode != "per-call", mlp_coalesce=mode == "deferred-gathered")
+    if mode == "deferred-rows":
+        eng.set_launch(B.K_MLP_BWD, 1)
+    c = 0
+    for t in range(3):
+        p = o.params()
+        for k in range(int(sched[t].max())):          # round-robin over the workers, as they would arrive
+            for i in range(W):
+                if k < sched[t, i]:
+                    o.accumulate(i, _grad(p, xs, ys, c, wl))
+                    eng.accumulate_mlp(i, xs_d[c % wl.mlp_pool], ys_d[c % wl.mlp_pool])
+                    c += 1
+        eng.sync_step(); o.sync_step()
+        cnt, cur, tt = eng.counters()
+        assert np.array_equal(cnt, o.counters()[0])
+    eng.sync_step(); o.sync_step()
+    eng.check()
+    ref = o.params()
+    assert np.abs(ref - x0).max() > 1e-4
+    assert np.abs(eng.params_host().astype(np.float64) - ref).max() <= TOL * np.abs(ref).max()
+    for s in range(4):
+        assert np.array_equal(eng.consumed(s), o.consumed[s])
+    eng.destroy()
