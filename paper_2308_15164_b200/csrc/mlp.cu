@@ -26,6 +26,12 @@
 //                   accumulators, finished tiles leave by TMA store (a worker's first gradient of an iteration)
 //                   or TMA reduce-add; 128 x 64 or 128 x 128 tiles
 //   k_dw1_regs      one 128 x 64 tile per CTA, the accumulator tile prefetched into registers, K-batched
+// Deferred mode (all gradients of an iteration are evaluated at the same x_t, so the sums may be formed late): a
+// call stops after k_bwd and leaves bf16(X)^T, bf16(dZ)^T and its db1 | dW2 | db2 in pool slots; then
+//   k_sync_w1            Step 1 + update of the W1 slice: ONE contraction over all pooled micro-batches of the
+//                        iteration, the update as its epilogue (no accumulator row involved)
+//   k_sync_small_pooled  the same step for b1, W2, b2 from the pooled partials
+//   k_gather_small, k_dw1_ring over a slot list: the rows themselves, when somebody needs them
 #include <cuda.h>
 
 #include <cstdio>
