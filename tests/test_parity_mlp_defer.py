@@ -462,3 +462,49 @@ def test_twelve_workers(mode):
     for s in range(4):
         assert np.array_equal(eng.consumed(s), o.consumed[s])
     eng.destroy()
+
+
+def test_learning_rate_schedule_eq6_and_weight_decay_in_the_pooled_step():
+    """gamma_t changing every iteration, Eq. 6 and weight decay through the step that works from the pooled operands
+    (the rate travels with the gradients: the set of iteration t is applied with the rate in effect when it ended),
+    eager and pipelined, against the oracle."""
+    import torch
+
+    from paper_2308_15164_b200 import binding as B
+
+    T = 6
+    wl = wlm.config(4, small=True, T=T)
+    d = wl.mlp
+    x0 = wlm.params0(wl)
+    xs, ys = wlm.mlp_batches(wl)
+    xs_d, ys_d = torch.from_numpy(xs).cuda(), torch.from_numpy(ys).cuda()
+    lrs = [0.05, 0.02, 0.08, 0.01, 0.04, 0.03, 0.03]
+    lam, wd = 0.3, 1e-3
+    o = AbsSgdOracle(x0, wl.W, lrs[0], wl.momentum, wd, lam)
+    its = list(wlm.iter_calls(wl))
+    for t, calls in enumerate(its):
+        o.lr = lrs[t]
+        p = o.params()
+        for (i, k, c) in calls:
+            o.accumulate(i, _grad(p, xs, ys, c, wl))
+        o.sync_step()
+    o.lr = lrs[T]
+    o.sync_step()
+    ref = o.params()
+    assert np.abs(ref - x0).max() > 1e-4
+    outs = []
+    for pipelined in (False, True):
+        eng = B.AbsSgd(torch.from_numpy(x0).cuda(), wl.W, lrs[0], wl.momentum, wd, lam, pipelined=pipelined,
+                       mlp=(d.d_in, d.d_hidden, d.d_out, d.mb), mlp_defer=True)
+        for t, calls in enumerate(its):
+            eng.set_lr(lrs[t + 1])                   # gamma_{t+1}: supplied one iteration ahead
+            for (i, k, c) in calls:
+                eng.accumulate_mlp(i, xs_d[c % wl.mlp_pool], ys_d[c % wl.mlp_pool])
+            eng.sync_step()
+        eng.sync_step()
+        eng.check()
+        got = eng.params_host()
+        assert np.abs(got.astype(np.float64) - ref).max() <= TOL * np.abs(ref).max(), f"pipelined={pipelined}"
+        outs.append(got)
+        eng.destroy()
+    assert np.array_equal(outs[0], outs[1])
