@@ -436,6 +436,9 @@ def run_ours(args):
         torch.cuda.empty_cache()
         if "mlp" in sections:
             line["mlp"] = run_mlp(B, wlm, dev, peaks)
+            # the section's headline rows once more, side by side (us per micro-batch of the whole pipelined run)
+            line["mlp_us_per_microbatch"] = {k: round(v["us_per_microbatch"], 2) for k, v in line["mlp"].items()
+                                             if isinstance(v, dict) and not k.startswith("serial_")}
         if "tiny" in sections:
             line["tiny"] = run_tiny(B, wlm, dev)
         if "schedules" in sections:
