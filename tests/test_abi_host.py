@@ -123,3 +123,30 @@ def test_multi_gpu_entry_points_reject_bad_arguments_on_the_host(B):
     assert B.lib.abs_ipc_export(None, None, None) == B.EINVAL
     assert B.lib.abs_ipc_open(None, 0, None) == B.EINVAL
     assert B.lib.abs_ipc_close(None, 0) == B.EINVAL
+
+
+def test_workspace_of_the_deferred_mlp_mode_grows_by_its_operand_pools(B):
+    """ABS_FLAG_MLP_DEFER adds one operand pool per accumulator set: max(32, 16 W) slots, at most 128, of
+    (3 d_in + 2 d_hidden) * 128 bytes of bf16 operands, the labels and the micro-batch's db1 | dW2 | db2."""
+    d_in, d_h, d_out = 256, 384, 10
+    P = d_in * d_h + d_h + d_h * d_out + d_out
+
+    def extra(W):
+        kw = dict(P=P, W=W, lr=0.1, mlp=(d_in, d_h, d_out, 64))
+        plain = B.abs_workspace_bytes(B.make_config(flags=B.FLAG_MLP, **kw))
+        defer = B.abs_workspace_bytes(B.make_config(flags=B.FLAG_MLP | B.FLAG_MLP_DEFER, **kw))
+        assert plain > 0 and defer > plain
+        return defer - plain
+
+    def up(v, a):
+        return (v + a - 1) // a * a
+
+    def pools(cap):
+        part = up(d_h + d_h * d_out + d_out, 32) * 4
+        one = 2 * up(cap * d_in * 64 * 2, 1024) + up(cap * d_h * 64 * 2, 1024) + up(cap * 64 * 4, 1024) + up(cap * part, 1024)
+        return 2 * up(one, 4096)
+
+    assert extra(1) == pools(32)
+    assert extra(4) == pools(64)
+    assert extra(8) == pools(128)
+    assert extra(40) == pools(128)                   # capped
