@@ -871,8 +871,7 @@ __global__ void __launch_bounds__(64 + kStepEpiThreads) k_sync_w1(const __grid_c
                     mbar_expect_tx(&s.op_full[st], kStepSlotBytes);
                     const int slot = (int)sl.s[j];
                     tma_load_2d(s.op[st], &tm_xt, 0, slot * d_in + m0, &s.op_full[st]);
-                    tma_load_2d(s.op[st] + kTileM * 128, &tm_dzt, 0, slot * ld + n0, &s.op_full[st]);
-                    tma_load_2d(s.op[st] + kTileM * 128 + kDwN * 128, &tm_dzt, 0, slot * ld + n0 + kDwN, &s.op_full[st]);
+                    tma_load_2d(s.op[st] + kTileM * 128, &tm_dzt, 0, slot * ld + n0, &s.op_full[st]);   // one 128-row box
                 }
             }
         }
@@ -1342,7 +1341,9 @@ cudaError_t mlp_pool_init(MlpPool* p, const MlpDims& d, int cap, void* base) {
     p->part = reinterpret_cast<float*>(at);
     p->part_stride = pool_part_stride(d);
     if (!encode_2d(reinterpret_cast<CUtensorMap*>(&p->tmap_xb), CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, p->xb, (uint64_t)cap * kMB,
-                   d.d_in, kMB, 64))
+                   d.d_in, kMB, 64) ||
+        !encode_2d(reinterpret_cast<CUtensorMap*>(&p->tmap_dzt128), CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, p->dzt,
+                   (uint64_t)cap * d.d_hidden, kMB, kStepN, kMB))
         return cudaErrorInvalidValue;
     // same boxes as the scratch sets' operands: slot j at rows [j*d_in, (j+1)*d_in) of X^T, [j*d_h, (j+1)*d_h) of dZ^T
     if (!encode_2d(reinterpret_cast<CUtensorMap*>(&p->tmap_xt), CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, p->xtb,
@@ -1409,7 +1410,7 @@ cudaError_t launch_mlp_sync_w1(const MlpDims& d, const MlpScratch& s, const MlpP
     const W1StepCoef cf{1.0f / B, lr, mu, wd, lambda_dc, disp_scale};
     const CUtensorMap& shadow_map = *reinterpret_cast<const CUtensorMap*>(tm_shadow ? tm_shadow : tm_x_out);
     return launch_kernel(k_sync_w1, ctas, 64 + kStepEpiThreads, sizeof(StepSmem) + 1024, stream, chained,
-                         *reinterpret_cast<const CUtensorMap*>(&pool.tmap_xt), *reinterpret_cast<const CUtensorMap*>(&pool.tmap_dzt),
+                         *reinterpret_cast<const CUtensorMap*>(&pool.tmap_xt), *reinterpret_cast<const CUtensorMap*>(&pool.tmap_dzt128),
                          *reinterpret_cast<const CUtensorMap*>(tm_x_in), *reinterpret_cast<const CUtensorMap*>(tm_x_out),
                          *reinterpret_cast<const CUtensorMap*>(tm_v), shadow_map, slots, n_tiles_n, n_tiles, d.d_in, d.d_hidden, nb,
                          cf, tm_shadow ? 1 : 0, s.status);
