@@ -160,6 +160,8 @@ struct MlpScratch {      // device pointers carved from the workspace (all hidde
     float* bpart;        // [4][d_hidden/32][4][256] partial dW2 / db1 / db2 sums of k_bwd, per micro-batch of a call
     unsigned int* tickets_b;  // [d_hidden/32]     "last CTA done" tickets of k_bwd (zero between launches)
     unsigned int* tickets;  // [groups]           "last CTA done" tickets of the logit reduction (zero between launches)
+    unsigned int* tickets2; // [4]                second level of that reduction, one per micro-batch of a call
+    float* dlbuf;        // [4][2][mb][16]        dL of each micro-batch: unrounded, and rounded to bf16
     int* status;         // device status word: ABS_ETIMEOUT if a bounded wait ran out
     void* zero_from;     // region that must be zero before first use (tickets + status) ...
     size_t zero_bytes;   // ... and its size

@@ -102,13 +102,15 @@ __global__ void __launch_bounds__(256) k_cast_x(const void* __restrict__ x_in, c
 // k_fwd2: per CTA 32 hidden units x 64 samples.
 //   phase 1 (thread = sample r, 8 hidden units): Z = sum_s zpart + b1 ; hb = bf16(relu(Z)) -> hbt
 //   phase 2 (thread = sample r, 4 logits):        partial logits of these 32 hidden units -> lpart[cta]
-//   tail: the last CTA of each group of 8 sums the group's partials (fixed order) -> gpart[group].
-//         The remaining sum over the groups is cheap (n_groups x 4 KB) and is done by every CTA of k_bwd.
-// tickets[0 .. n_groups) are the group tickets: all zero on entry and reset before exit.
+//   tail: the last CTA of each group of 8 sums the group's partials (fixed order) -> gpart[group]; the last group
+//         to finish sums the group partials (fixed order), adds b2 and forms dL once for the micro-batch -> dlbuf.
+// tickets[0 .. n_groups) are the group tickets, tickets2[0] the second level's: all zero on entry, reset before exit.
 // --------------------------------------------------------------------------------------------
 __global__ void __launch_bounds__(256) k_fwd2(const float* zpart, int nsplit, const float* __restrict__ b1,
                                               const __nv_bfloat16* __restrict__ w2b, __nv_bfloat16* hbt,
-                                              float* lpart, float* gpart, unsigned int* tickets, int d_h, int d_out) {
+                                              float* lpart, float* gpart, unsigned int* tickets, int d_h, int d_out,
+                                              const float* __restrict__ b2, const int32_t* y, float* dlbuf,
+                                              unsigned int* tickets2) {
     __shared__ float sh[kHB][kMB + 1];
     __shared__ float sw2[kHB][kOutPad];
     __shared__ unsigned int s_last;
@@ -121,6 +123,9 @@ __global__ void __launch_bounds__(256) k_fwd2(const float* zpart, int nsplit, co
         lpart += (size_t)j * n_cta * kMB * kOutPad;
         gpart += (size_t)j * n_groups * kMB * kOutPad;
         tickets += (size_t)j * n_groups;
+        y += (size_t)j * kMB;
+        dlbuf += (size_t)j * 2 * kMB * kOutPad;
+        tickets2 += j;
     }
 
     for (int e = threadIdx.x; e < kHB * kOutPad; e += 256) {
@@ -179,50 +184,20 @@ __global__ void __launch_bounds__(256) k_fwd2(const float* zpart, int nsplit, co
         reinterpret_cast<float4*>(gpart)[(size_t)group * (kMB * kOutPad / 4) + threadIdx.x] = acc;
     }
     if (threadIdx.x == 0) tickets[group] = 0u;   // ready for the next launch
-}
-
-// --------------------------------------------------------------------------------------------
-// k_bwd: per CTA 32 hidden units x 64 samples.
-//   prologue (every CTA, identical result): logits = sum over groups of gpart + b2 (fixed order);
-//            dL = (softmax - onehot)/mb, 4 lanes per sample row (max and sum by shuffles); CTA 0 also adds
-//            db2 = sum_r dL
-//   phase 1 (thread = sample r, 8 hidden units): dH = sum_o bf16(dL)[r][o] W2b[h][o]; dZ = dH * [H > 0]
-//            (H > 0 exactly when Z > 0); dzt[h][r] = bf16(dZ)
-//   phase 2 (thread = hidden unit, 2 outputs): dW2[h][o] += sum_r bf16(H)[h][r] bf16(dL)[r][o],
-//            db1[h] += sum_r dZ[h][r]   (fixed summation order over r)
-// --------------------------------------------------------------------------------------------
-__global__ void __launch_bounds__(256) k_bwd(const __nv_bfloat16* hbt, const float* gpart, int n_groups,
-                                             const float* __restrict__ b2, const int32_t* y,
-                                             const __nv_bfloat16* __restrict__ w2b, __nv_bfloat16* dzt, float* bpart,
-                                             unsigned int* tickets_b, float* acc_b1, float* acc_w2, float* acc_b2,
-                                             int32_t* cnt, int d_h, int d_out, int store, float* part, size_t part_stride,
-                                             MlpWorkers wk) {
-    __shared__ float sdl[kMB][kOutPad + 1];     // bf16(dL) as float
-    __shared__ float sdl32[kMB][kOutPad + 1];   // dL unrounded (CTA 0: db2)
-    __shared__ float sw2[kHB][kOutPad];
-    __shared__ float sh[kHB][kMB + 1];
-    __shared__ float sdz[kHB][kMB + 1];
-    __shared__ unsigned int s_last;
-    const int h_beg = blockIdx.x * kHB;
-    const int jb = blockIdx.y, nb = gridDim.y;       // micro-batch of this CTA, micro-batches in the call
-    hbt += (size_t)jb * d_h * kMB;
-    dzt += (size_t)jb * d_h * kMB;
-    gpart += (size_t)jb * n_groups * kMB * kOutPad;
-    y += (size_t)jb * kMB;
-    const int r = threadIdx.x % kMB, g = threadIdx.x / kMB;
-    for (int e = threadIdx.x; e < kHB * kOutPad; e += 256) {   // parameters: published before the call started
-        const int hl = e / kOutPad, o = e % kOutPad;
-        sw2[hl][o] = o < d_out ? bf16_to_f(w2b[(size_t)(h_beg + hl) * d_out + o]) : 0.f;
-    }
-    pdl_wait();                                      // hbt and gpart come from k_fwd2, just ahead on the stream
-    pdl_trigger();
-    float hv[8];                                     // issued first: independent of the logit sums below
-#pragma unroll
-    for (int j = 0; j < 8; ++j) hv[j] = bf16_to_f(hbt[(size_t)(h_beg + g * 8 + j) * kMB + r]);
+    // ---- second level: the last group to finish sums the group partials (fixed order), adds b2 and forms
+    //      dL = (softmax - onehot) / mb once for the micro-batch: dlbuf[0] unrounded (db2), dlbuf[1] rounded to bf16.
+    //      (Every k_bwd CTA used to do this for itself: n_groups x 4 KB of L2 reads per CTA.)
+    const int n_groups = (n_cta + kGroup - 1) / kGroup;
+    __threadfence();
+    __syncthreads();
+    if (threadIdx.x == 0) s_last = (atomicAdd(tickets2, 1u) == (unsigned)(n_groups - 1));
+    __syncthreads();
+    if (!s_last) return;
+    __threadfence();
     {
         float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
         for (int c = 0; c < n_groups; ++c) {
-            const float4 v = reinterpret_cast<const float4*>(gpart)[(size_t)c * (kMB * kOutPad / 4) + threadIdx.x];
+            const float4 v = __ldcg(reinterpret_cast<const float4*>(gpart) + (size_t)c * (kMB * kOutPad / 4) + threadIdx.x);
             acc.x += v.x; acc.y += v.y; acc.z += v.z; acc.w += v.w;
         }
         // softmax and dL on the registers that hold the sums: 4 adjacent lanes share a sample row
@@ -246,13 +221,60 @@ __global__ void __launch_bounds__(256) k_bwd(const __nv_bfloat16* hbt, const flo
         den += __shfl_xor_sync(0xffffffffu, den, 1);
         den += __shfl_xor_sync(0xffffffffu, den, 2);
         const int yr = y[rr];
+        float gl[4], gb[4];
 #pragma unroll
         for (int j = 0; j < 4; ++j) {
             const int o = 4 * og + j;
-            const float gl = o < d_out ? (l[j] / den - (o == yr ? 1.f : 0.f)) * (1.0f / kMB) : 0.f;
-            sdl32[rr][o] = gl;
-            sdl[rr][o] = bf16_to_f(__float2bfloat16_rn(gl));
+            gl[j] = o < d_out ? (l[j] / den - (o == yr ? 1.f : 0.f)) * (1.0f / kMB) : 0.f;
+            gb[j] = bf16_to_f(__float2bfloat16_rn(gl[j]));
         }
+        reinterpret_cast<float4*>(dlbuf)[threadIdx.x] = make_float4(gl[0], gl[1], gl[2], gl[3]);
+        reinterpret_cast<float4*>(dlbuf + kMB * kOutPad)[threadIdx.x] = make_float4(gb[0], gb[1], gb[2], gb[3]);
+    }
+    if (threadIdx.x == 0) *tickets2 = 0u;
+}
+
+// --------------------------------------------------------------------------------------------
+// k_bwd: per CTA 32 hidden units x 64 samples.
+//   prologue: dL = (softmax - onehot)/mb of the micro-batch as k_fwd2's last CTA left it (unrounded and rounded
+//            to bf16); CTA 0 also adds db2 = sum_r dL
+//   phase 1 (thread = sample r, 8 hidden units): dH = sum_o bf16(dL)[r][o] W2b[h][o]; dZ = dH * [H > 0]
+//            (H > 0 exactly when Z > 0); dzt[h][r] = bf16(dZ)
+//   phase 2 (thread = hidden unit, 2 outputs): dW2[h][o] += sum_r bf16(H)[h][r] bf16(dL)[r][o],
+//            db1[h] += sum_r dZ[h][r]   (fixed summation order over r)
+// --------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(256) k_bwd(const __nv_bfloat16* hbt, const float* dlbuf,
+                                             const __nv_bfloat16* __restrict__ w2b, __nv_bfloat16* dzt, float* bpart,
+                                             unsigned int* tickets_b, float* acc_b1, float* acc_w2, float* acc_b2,
+                                             int32_t* cnt, int d_h, int d_out, int store, float* part, size_t part_stride,
+                                             MlpWorkers wk) {
+    __shared__ float sdl[kMB][kOutPad + 1];     // bf16(dL) as float
+    __shared__ float sdl32[kMB][kOutPad + 1];   // dL unrounded (CTA 0: db2)
+    __shared__ float sw2[kHB][kOutPad];
+    __shared__ float sh[kHB][kMB + 1];
+    __shared__ float sdz[kHB][kMB + 1];
+    __shared__ unsigned int s_last;
+    const int h_beg = blockIdx.x * kHB;
+    const int jb = blockIdx.y, nb = gridDim.y;       // micro-batch of this CTA, micro-batches in the call
+    hbt += (size_t)jb * d_h * kMB;
+    dzt += (size_t)jb * d_h * kMB;
+    const int r = threadIdx.x % kMB, g = threadIdx.x / kMB;
+    for (int e = threadIdx.x; e < kHB * kOutPad; e += 256) {   // parameters: published before the call started
+        const int hl = e / kOutPad, o = e % kOutPad;
+        sw2[hl][o] = o < d_out ? bf16_to_f(w2b[(size_t)(h_beg + hl) * d_out + o]) : 0.f;
+    }
+    pdl_wait();                                      // hbt and dL come from k_fwd2, just ahead on the stream
+    pdl_trigger();
+    float hv[8];
+#pragma unroll
+    for (int j = 0; j < 8; ++j) hv[j] = bf16_to_f(hbt[(size_t)(h_beg + g * 8 + j) * kMB + r]);
+    {   // dL of the micro-batch, formed once by k_fwd2: [0] unrounded (db2), [1] rounded to bf16
+        const float* dl = dlbuf + (size_t)jb * 2 * kMB * kOutPad;
+        const int rr = threadIdx.x / 4, og = threadIdx.x % 4;
+        const float4 a = reinterpret_cast<const float4*>(dl)[threadIdx.x];
+        const float4 b = reinterpret_cast<const float4*>(dl + kMB * kOutPad)[threadIdx.x];
+        sdl32[rr][4 * og + 0] = a.x; sdl32[rr][4 * og + 1] = a.y; sdl32[rr][4 * og + 2] = a.z; sdl32[rr][4 * og + 3] = a.w;
+        sdl[rr][4 * og + 0] = b.x; sdl[rr][4 * og + 1] = b.y; sdl[rr][4 * og + 2] = b.z; sdl[rr][4 * og + 3] = b.w;
     }
     __syncthreads();
     float db2 = 0.f;                                 // CTA column 0, thread o < d_out: sum_r dL[r][o]
@@ -1242,7 +1264,8 @@ size_t layout_scratch(MlpScratch* s, const MlpDims& d, char* base) {
     char* gpart = take((size_t)kMaxBatch * n_groups * kMB * kOutPad * 4);
     char* bpart = take((size_t)kMaxBatch * n_cta * 4 * 256 * 4);
     char* ycopy = take((size_t)kMaxBatch * kMB * 4);
-    char* tickets = take((size_t)(kMaxBatch * n_groups + n_cta) * 4);   // k_fwd2 group tickets, then k_bwd chunk tickets
+    char* dlbuf = take((size_t)kMaxBatch * 2 * kMB * kOutPad * 4);
+    char* tickets = take((size_t)(kMaxBatch * n_groups + n_cta + kMaxBatch) * 4);   // k_fwd2 group tickets, k_bwd chunk tickets, k_fwd2 second level
     char* status = take(256);
     if (s) {
         s->xb = reinterpret_cast<__nv_bfloat16*>(xb);
@@ -1254,6 +1277,8 @@ size_t layout_scratch(MlpScratch* s, const MlpDims& d, char* base) {
         s->gpart = reinterpret_cast<float*>(gpart);
         s->tickets = reinterpret_cast<unsigned int*>(tickets);
         s->tickets_b = reinterpret_cast<unsigned int*>(tickets) + kMaxBatch * n_groups;
+        s->tickets2 = reinterpret_cast<unsigned int*>(tickets) + kMaxBatch * n_groups + n_cta;
+        s->dlbuf = reinterpret_cast<float*>(dlbuf);
         s->bpart = reinterpret_cast<float*>(bpart);
         s->ycopy = reinterpret_cast<int32_t*>(ycopy);
         s->status = reinterpret_cast<int*>(status);
@@ -1487,21 +1512,20 @@ cudaError_t launch_mlp_front(const MlpDims& d, const MlpScratch& s, const float*
     const float* zp = s.zpart;
     const float* b1 = x_pub + o_b1;
     const __nv_bfloat16* w2b = shadow + o_w2;
+    const float* b2 = x_pub + o_b2;
+    const int32_t* yc = pool ? pool->ycopy + (size_t)pool_slot0 * kMB : s.ycopy;
     e = launch_kernel(k_fwd2, dim3(n_cta, nb), 256, 0, stream, (chain & kChainFwd2) != 0, zp, nsplit, b1, w2b, s.hbt, s.lpart, s.gpart, s.tickets,
-                      d.d_hidden, d.d_out);
+                      d.d_hidden, d.d_out, b2, yc, s.dlbuf, s.tickets2);
     mark(user, ABS_K_MLP_FWD, 1, stream);
     if (e != cudaSuccess) return e;
 
     mark(user, ABS_K_MLP_BWD, -1, stream);
-    const int n_groups = (n_cta + kGroup - 1) / kGroup;
     const __nv_bfloat16* hbt = s.hbt;
-    const float* gpart = s.gpart;
-    const float* b2 = x_pub + o_b2;
-    const int32_t* yc = pool ? pool->ycopy + (size_t)pool_slot0 * kMB : s.ycopy;
+    const float* dlbuf = s.dlbuf;
     __nv_bfloat16* dzt = pool ? pool->dzt + (size_t)pool_slot0 * d.d_hidden * kMB : s.dzt;
     float* part = pool ? pool->part + (size_t)pool_slot0 * pool->part_stride : nullptr;
     const size_t part_stride = pool ? pool->part_stride : 0;
-    e = launch_kernel(k_bwd, dim3(n_cta, nb), 256, 0, stream, (chain & kChainBwd) != 0, hbt, gpart, n_groups, b2, yc, w2b, dzt, s.bpart,
+    e = launch_kernel(k_bwd, dim3(n_cta, nb), 256, 0, stream, (chain & kChainBwd) != 0, hbt, dlbuf, w2b, dzt, s.bpart,
                       s.tickets_b, acc_row + o_b1, acc_row + o_w2, acc_row + o_b2, cnt, d.d_hidden, d.d_out, store ? 1 : 0, part,
                       part_stride, workers ? *workers : MlpWorkers{});
     mark(user, ABS_K_MLP_BWD, 1, stream);
