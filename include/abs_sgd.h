@@ -292,7 +292,8 @@ int abs_selftest_timeout(abs_ctx *ctx);
  *                  SM's shared memory (default: with W > 1, outside serial mode, their light forms of about
  *                  100 KB, so that CTAs of different workers' calls share an SM; same results bit for bit).
  *   ABS_K_MLP_BWD  1 = with ABS_FLAG_MLP_DEFER: the step never works from the pooled operands; every iteration's
- *                  rows are completed first (see the flag).
+ *                  rows are completed first (see the flag).  2 = the pooled step keeps 128 x 128 tiles (default:
+ *                  128 x 256 where mlp_hidden is a multiple of 256).
  *   ABS_K_MLP_FWD  1 = serial mode: every kernel of a gradient call runs on stream_acc instead of the
  *                  worker's internal stream (for per-kernel timing).
  *   ABS_K_CHAIN    0 = consecutive kernels of a stream are chained by programmatic dependent launch: the next

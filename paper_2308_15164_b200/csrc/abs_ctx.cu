@@ -421,7 +421,7 @@ int launch_fused(abs_ctx* c, uint32_t set, int in, int out, uint64_t log_step, c
                                      c->chained()));
             CK(launch_mlp_sync_w1(c->mlp_dims, c->mlp_scratch[0], c->pool[set], c->fused_slots[set], c->fused_n[set], &c->tm_x[in],
                                   &c->tm_x[out], &c->tm_v, &c->tm_shadow[out], B, a.lr, a.mu, a.wd, a.lambda_dc, a.disp_scale,
-                                  0, stream, c->chained()));
+                                  c->ctas_per_sm[ABS_K_MLP_BWD] == 2 ? -128 : 0, stream, c->chained()));
         }
         c->launches += 2;
         c->fused_pending[set] = false;
@@ -1434,7 +1434,7 @@ int abs_set_launch(abs_ctx* c, int kernel_class, int ctas_per_sm) {
         return invalid(c, "unknown bits in the ABS_K_MLP_DW1 mask");
     if (kernel_class == ABS_K_CHAIN && (ctas_per_sm < 0 || ctas_per_sm > 1)) return invalid(c, "ABS_K_CHAIN takes 0 or 1");
     if (kernel_class == ABS_K_MLP_FWD && (ctas_per_sm < 0 || ctas_per_sm > 1)) return invalid(c, "ABS_K_MLP_FWD takes 0 or 1");
-    if (kernel_class == ABS_K_MLP_BWD && (ctas_per_sm < 0 || ctas_per_sm > 1)) return invalid(c, "ABS_K_MLP_BWD takes 0 or 1");
+    if (kernel_class == ABS_K_MLP_BWD && (ctas_per_sm < 0 || ctas_per_sm > 2)) return invalid(c, "ABS_K_MLP_BWD takes 0, 1 or 2");
     if (int rc = settle_all(c)) return rc;
     c->ctas_per_sm[kernel_class] = ctas_per_sm;
     return ABS_OK;

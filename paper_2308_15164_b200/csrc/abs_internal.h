@@ -183,7 +183,7 @@ struct MlpPool {
     size_t part_stride;  // floats
     int cap;
     TmapBytes tmap_xt, tmap_dzt, tmap_xb;
-    TmapBytes tmap_dzt128;   // dZ^T in boxes of 128 rows (one TMA copy per operand slot of k_sync_w1)
+    TmapBytes tmap_dzt128, tmap_dzt256;   // dZ^T in boxes of 128 / 256 rows (one TMA copy per operand slot of k_sync_w1)
 };
 size_t mlp_pool_bytes(const MlpDims& d, int cap);
 cudaError_t mlp_pool_init(MlpPool* p, const MlpDims& d, int cap, void* base);

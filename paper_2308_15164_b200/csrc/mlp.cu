@@ -816,19 +816,26 @@ __global__ void __launch_bounds__(192) k_dw1_ring(const __grid_constant__ CUtens
 // HBM traffic: 18 bytes per W1 element (x, v read; x', v, bf16 x' written) + the operands once (they stay in
 // L2 between tiles), against (8 W_act + 18) for the row-based step plus 4 W_act for the contractions.
 // ============================================================================================
-constexpr int kStepN = 128;      // tile width
-constexpr int kStepOps = 3;      // operand slots of 32 KB
 constexpr int kStepE = 3;        // epilogue stages: [x panel 16 KB | v panel 16 KB]
 constexpr int kStepEpiThreads = 256;   // eight epilogue warps: two per TMEM lane quarter, 16 columns of a panel each
-constexpr int kStepSlotBytes = kTileM * 128 + kStepN * 128;
 constexpr int kPanelBytes = kTileM * 32 * 4;
+// kN: tile width.  128: three operand slots of 32 KB.  256 (d_hidden a multiple of 256): two slots of 48 KB -- the
+// same bytes in flight, a quarter less operand traffic from L2 per output element (the X^T tile serves twice the
+// columns), all 512 TMEM columns for the two accumulators.
+template <int kN>
+struct StepCfg {
+    static constexpr int kOps = kN == 128 ? 3 : 2;
+    static constexpr int kSlotBytes = kTileM * 128 + kN * 128;
+    static constexpr int kPP = kN / 32;              // epilogue panels per tile
+};
 
+template <int kN>
 struct StepSmem {
-    alignas(1024) uint8_t op[kStepOps][kStepSlotBytes];
+    alignas(1024) uint8_t op[StepCfg<kN>::kOps][StepCfg<kN>::kSlotBytes];
     alignas(1024) uint8_t ep[kStepE][2 * kPanelBytes];
     alignas(1024) uint8_t sh[2][kTileM * 128];          // bf16 copy, [128 rows][64 columns], swizzled 128-byte rows
-    alignas(8) uint64_t op_full[kStepOps];
-    uint64_t op_empty[kStepOps];
+    alignas(8) uint64_t op_full[StepCfg<kN>::kOps];
+    uint64_t op_empty[StepCfg<kN>::kOps];
     uint64_t acc_full[2];
     uint64_t acc_empty[2];
     uint64_t ep_full[kStepE];
@@ -842,6 +849,7 @@ struct W1StepCoef {
     float lr, mu, wd, lambda_dc, disp_scale;
 };
 
+template <int kN>
 __global__ void __launch_bounds__(64 + kStepEpiThreads) k_sync_w1(const __grid_constant__ CUtensorMap tm_xt,
                                                  const __grid_constant__ CUtensorMap tm_dzt,
                                                  const __grid_constant__ CUtensorMap tm_x_in,
@@ -851,10 +859,12 @@ __global__ void __launch_bounds__(64 + kStepEpiThreads) k_sync_w1(const __grid_c
                                                  const __grid_constant__ MlpSlots sl, int n_tiles_n, int n_tiles, int d_in,
                                                  int ld, int nb, W1StepCoef cf, int has_shadow, int* status) {
     extern __shared__ uint8_t smem_raw[];
-    StepSmem& s = *reinterpret_cast<StepSmem*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+    constexpr int kStepOps = StepCfg<kN>::kOps, kStepSlotBytes = StepCfg<kN>::kSlotBytes, kPP = StepCfg<kN>::kPP;
+    constexpr int kStepN = kN;
+    StepSmem<kN>& s = *reinterpret_cast<StepSmem<kN>*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
     const int warp = threadIdx.x / 32, lane = threadIdx.x % 32;
     const int my_tiles = (n_tiles - (int)blockIdx.x + (int)gridDim.x - 1) / (int)gridDim.x;
-    const int my_panels = my_tiles * 4;
+    const int my_panels = my_tiles * (kN / 32);
 
     if (warp == 1) {
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&s.tmem_base)), "r"(2 * kStepN) : "memory");
@@ -893,7 +903,7 @@ __global__ void __launch_bounds__(64 + kStepEpiThreads) k_sync_w1(const __grid_c
                     mbar_expect_tx(&s.op_full[st], kStepSlotBytes);
                     const int slot = (int)sl.s[j];
                     tma_load_2d(s.op[st], &tm_xt, 0, slot * d_in + m0, &s.op_full[st]);
-                    tma_load_2d(s.op[st] + kTileM * 128, &tm_dzt, 0, slot * ld + n0, &s.op_full[st]);   // one 128-row box
+                    tma_load_2d(s.op[st] + kTileM * 128, &tm_dzt, 0, slot * ld + n0, &s.op_full[st]);   // one box of kN rows
                 }
             }
         }
@@ -927,8 +937,8 @@ __global__ void __launch_bounds__(64 + kStepEpiThreads) k_sync_w1(const __grid_c
         const int sw = row & 7;
         const bool leader = (threadIdx.x == 64);
         auto panel_coords = [&](int e, int* col, int* m0) {
-            const int t = (int)blockIdx.x + (e >> 2) * (int)gridDim.x;
-            *col = (t % n_tiles_n) * kStepN + (e & 3) * 32;
+            const int t = (int)blockIdx.x + (e / kPP) * (int)gridDim.x;
+            *col = (t % n_tiles_n) * kStepN + (e % kPP) * 32;
             *m0 = (t / n_tiles_n) * kTileM;
         };
         auto load_panels = [&](int e) {              // leader only: x and v panels of step e into stage e % kStepE
@@ -944,7 +954,7 @@ __global__ void __launch_bounds__(64 + kStepEpiThreads) k_sync_w1(const __grid_c
         const float c_dc = -cf.lambda_dc * cf.disp_scale;
         bool stopped = false;
         for (int e = 0; e < my_panels && !stopped; ++e) {
-            const int i = e >> 2, p = e & 3, ab = i & 1, st = e % kStepE;
+            const int i = e / kPP, p = e % kPP, ab = i & 1, st = e % kStepE;
             bool ok = true;
             if (p == 0) ok = mbar_wait(&s.acc_full[ab], (i / 2) & 1);
             ok = mbar_wait(&s.ep_full[st], (e / kStepE) & 1) && ok;
@@ -954,7 +964,7 @@ __global__ void __launch_bounds__(64 + kStepEpiThreads) k_sync_w1(const __grid_c
                 uint32_t acc[16];
                 asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
                 tmem_ld_16(tmem + ((uint32_t)(qd * 32) << 16) + (uint32_t)(ab * kStepN + p * 32 + half * 16), acc);
-                if (p == 3) {                        // the accumulator is in registers: the tile after next may use it
+                if (p == kPP - 1) {                  // the accumulator is in registers: the tile after next may use it
                     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
                     mbar_arrive(&s.acc_empty[ab]);
                 }
@@ -1368,7 +1378,10 @@ cudaError_t mlp_pool_init(MlpPool* p, const MlpDims& d, int cap, void* base) {
     if (!encode_2d(reinterpret_cast<CUtensorMap*>(&p->tmap_xb), CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, p->xb, (uint64_t)cap * kMB,
                    d.d_in, kMB, 64) ||
         !encode_2d(reinterpret_cast<CUtensorMap*>(&p->tmap_dzt128), CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, p->dzt,
-                   (uint64_t)cap * d.d_hidden, kMB, kStepN, kMB))
+                   (uint64_t)cap * d.d_hidden, kMB, 128, kMB) ||
+        (d.d_hidden % 256 == 0 &&
+         !encode_2d(reinterpret_cast<CUtensorMap*>(&p->tmap_dzt256), CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, p->dzt,
+                    (uint64_t)cap * d.d_hidden, kMB, 256, kMB)))
         return cudaErrorInvalidValue;
     // same boxes as the scratch sets' operands: slot j at rows [j*d_in, (j+1)*d_in) of X^T, [j*d_h, (j+1)*d_h) of dZ^T
     if (!encode_2d(reinterpret_cast<CUtensorMap*>(&p->tmap_xt), CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, p->xtb,
@@ -1415,30 +1428,44 @@ cudaError_t launch_mlp_sync_small(const MlpDims& d, const MlpPool& pool, const M
                          x_out + w1, v + w1, shadow_out ? shadow_out + w1 : nullptr, n_small, cf, cnt, log_row, W);
 }
 
-cudaError_t launch_mlp_sync_w1(const MlpDims& d, const MlpScratch& s, const MlpPool& pool, const MlpSlots& slots, int nb,
-                               const void* tm_x_in, const void* tm_x_out, const void* tm_v, const void* tm_shadow,
-                               float B, float lr, float mu, float wd, float lambda_dc, float disp_scale, int max_ctas,
-                               cudaStream_t stream, bool chained) {
-    if (nb < 1 || nb > kMlpMaxSlots || d.d_hidden % kStepN != 0) return cudaErrorInvalidValue;
+namespace {
+template <int kN>
+cudaError_t sync_w1_launch(const MlpDims& d, const MlpScratch& s, const TmapBytes& tm_a, const TmapBytes& tm_b, const MlpSlots& slots,
+                           int nb, const void* tm_x_in, const void* tm_x_out, const void* tm_v, const void* tm_shadow,
+                           const W1StepCoef& cf, int max_ctas, cudaStream_t stream, bool chained) {
     static bool opted_in[64] = {};
     int dev = 0;
     cudaError_t e = cudaGetDevice(&dev);
     if (e != cudaSuccess) return e;
     if (dev < 0 || dev >= 64 || !opted_in[dev]) {
-        e = cudaFuncSetAttribute(k_sync_w1, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(StepSmem) + 1024);
+        e = cudaFuncSetAttribute(k_sync_w1<kN>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(StepSmem<kN>) + 1024);
         if (e != cudaSuccess) return e;
         if (dev >= 0 && dev < 64) opted_in[dev] = true;
     }
-    const int n_tiles_n = d.d_hidden / kStepN, n_tiles = n_tiles_n * (d.d_in / kTileM);
+    const int n_tiles_n = d.d_hidden / kN, n_tiles = n_tiles_n * (d.d_in / kTileM);
     int ctas = n_tiles < s.num_sms ? n_tiles : s.num_sms;
     if (max_ctas > 0 && ctas > max_ctas) ctas = max_ctas;
-    const W1StepCoef cf{1.0f / B, lr, mu, wd, lambda_dc, disp_scale};
     const CUtensorMap& shadow_map = *reinterpret_cast<const CUtensorMap*>(tm_shadow ? tm_shadow : tm_x_out);
-    return launch_kernel(k_sync_w1, ctas, 64 + kStepEpiThreads, sizeof(StepSmem) + 1024, stream, chained,
-                         *reinterpret_cast<const CUtensorMap*>(&pool.tmap_xt), *reinterpret_cast<const CUtensorMap*>(&pool.tmap_dzt128),
+    return launch_kernel(k_sync_w1<kN>, ctas, 64 + kStepEpiThreads, sizeof(StepSmem<kN>) + 1024, stream, chained,
+                         *reinterpret_cast<const CUtensorMap*>(&tm_a), *reinterpret_cast<const CUtensorMap*>(&tm_b),
                          *reinterpret_cast<const CUtensorMap*>(tm_x_in), *reinterpret_cast<const CUtensorMap*>(tm_x_out),
                          *reinterpret_cast<const CUtensorMap*>(tm_v), shadow_map, slots, n_tiles_n, n_tiles, d.d_in, d.d_hidden, nb,
                          cf, tm_shadow ? 1 : 0, s.status);
+}
+}  // namespace
+
+cudaError_t launch_mlp_sync_w1(const MlpDims& d, const MlpScratch& s, const MlpPool& pool, const MlpSlots& slots, int nb,
+                               const void* tm_x_in, const void* tm_x_out, const void* tm_v, const void* tm_shadow,
+                               float B, float lr, float mu, float wd, float lambda_dc, float disp_scale, int max_ctas,
+                               cudaStream_t stream, bool chained) {
+    if (nb < 1 || nb > kMlpMaxSlots || d.d_hidden % 128 != 0) return cudaErrorInvalidValue;
+    const W1StepCoef cf{1.0f / B, lr, mu, wd, lambda_dc, disp_scale};
+    // 128 x 256 tiles where the layer allows them and there are enough of them to go round
+    if (d.d_hidden % 256 == 0 && max_ctas != -128)
+        return sync_w1_launch<256>(d, s, pool.tmap_xt, pool.tmap_dzt256, slots, nb, tm_x_in, tm_x_out, tm_v, tm_shadow, cf, max_ctas,
+                                   stream, chained);
+    return sync_w1_launch<128>(d, s, pool.tmap_xt, pool.tmap_dzt128, slots, nb, tm_x_in, tm_x_out, tm_v, tm_shadow, cf,
+                               max_ctas < 0 ? 0 : max_ctas, stream, chained);
 }
 
 cudaError_t mlp_make_acc_tmap(void* tmap_out, const MlpDims& d, float* acc_row) {

@@ -112,9 +112,9 @@ def test_set_launch_rejects_unknown_values():
 
     eng = B.AbsSgd(torch.zeros(1024, device="cuda"), 2, 0.1)
     for cls, val in ((B.K_CHAIN, 2), (B.K_CHAIN, -1), (B.K_MLP_DW1, 1), (B.K_MLP_DW1, 64), (B.K_MLP_DW1, 256),
-                     (B.K_MLP_FWD, 2), (B.K_MLP_BWD, 2), (B.K_SYNC, -3), (6, 0), (-1, 0)):
+                     (B.K_MLP_FWD, 2), (B.K_MLP_BWD, 3), (B.K_SYNC, -3), (6, 0), (-1, 0)):
         assert B.lib.abs_set_launch(eng._h, cls, val) == B.EINVAL, (cls, val)
-    for cls, val in ((B.K_CHAIN, 1), (B.K_CHAIN, 0), (B.K_MLP_DW1, 4 | 32 | 128), (B.K_MLP_DW1, 8), (B.K_SYNC, -2), (B.K_ACCUMULATE, 4), (B.K_MLP_BWD, 1)):
+    for cls, val in ((B.K_CHAIN, 1), (B.K_CHAIN, 0), (B.K_MLP_DW1, 4 | 32 | 128), (B.K_MLP_DW1, 8), (B.K_SYNC, -2), (B.K_ACCUMULATE, 4), (B.K_MLP_BWD, 1), (B.K_MLP_BWD, 2)):
         assert B.lib.abs_set_launch(eng._h, cls, val) == B.OK, (cls, val)
     eng.destroy()
 

@@ -201,11 +201,11 @@ def test_one_step_from_the_pooled_operands_against_the_step_from_the_rows(small,
     xs, ys = wlm.mlp_batches(wl)
     xs_d, ys_d = torch.from_numpy(xs).cuda(), torch.from_numpy(ys).cuda()
     res = []
-    for rows_only in (False, True):
+    for knob in (0, 1, 2):                           # pooled step (128 x 256 tiles), rows first, pooled step with 128 x 128 tiles
         eng = B.AbsSgd(torch.from_numpy(x0).cuda(), wl.W, wl.lr, wl.momentum, 1e-3, lambda_dc, pipelined=True,
                        mlp=(d.d_in, d.d_hidden, d.d_out, d.mb), mlp_defer=True)
-        if rows_only:
-            eng.set_launch(B.K_MLP_BWD, 1)
+        if knob:
+            eng.set_launch(B.K_MLP_BWD, knob)
         for t, calls in enumerate(wlm.iter_calls(wl)):
             for (i, k, c) in calls:
                 eng.accumulate_mlp(i, xs_d[c % wl.mlp_pool], ys_d[c % wl.mlp_pool])
@@ -217,11 +217,13 @@ def test_one_step_from_the_pooled_operands_against_the_step_from_the_rows(small,
         g = eng.accumulator(eng.counters()[1], 1).cpu().numpy().copy()
         res.append((x, v, g))
         eng.destroy()
-    (xa, va, ga), (xb, vb, gb) = res
+    (xa, va, ga), (xb, vb, gb), (xc, vc, gc) = res
     assert np.abs(xa - x0).max() > 1e-4
     assert np.abs(xa - xb).max() <= 2e-6 * np.abs(xb).max()
     assert np.abs(va - vb).max() <= 2e-5 * np.abs(vb).max()
     assert np.abs(ga - gb).max() <= TOL * np.abs(gb).max()
+    # the two tile widths contract the same operands in the same order: the same bits
+    assert np.array_equal(xa, xc) and np.array_equal(va, vc) and np.array_equal(ga, gc)
 
 
 _MIXED = [
