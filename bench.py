@@ -438,7 +438,7 @@ def run_ours(args):
             line["mlp"] = run_mlp(B, wlm, dev, peaks)
             # the section's headline rows once more, side by side (us per micro-batch of the whole pipelined run)
             line["mlp_us_per_microbatch"] = {k: round(v["us_per_microbatch"], 2) for k, v in line["mlp"].items()
-                                             if isinstance(v, dict) and not k.startswith("serial_")}
+                                             if isinstance(v, dict) and "us_per_microbatch" in v and not k.startswith("serial_")}
         if "tiny" in sections:
             line["tiny"] = run_tiny(B, wlm, dev)
         if "schedules" in sections:
@@ -885,6 +885,36 @@ def run_mlp(B, wlm, dev, peaks, iters=12):
                      ("deferred_rows_single_calls", dict(max_batch=1, defer="rows")),
                      ("deferred_rows_batch_calls_up_to_4", dict(max_batch=4, defer="rows"))):
         out[name] = run_case(**kw)
+    # The deferred mode's step alone on the GPU (k_sync_small_pooled + k_sync_w1, the library's event pair around
+    # them), 18 micro-batches pooled per iteration (the workload's mean): against the bytes it has to move --
+    # 18 per W1 element (x, v in; x', v, bf16 x' out), the pooled operands once, the bias / W2 part.
+    def pooled_step(n_mb=18, iters=8):
+        eng = B.AbsSgd(x0_d, wl.W, wl.lr, wl.momentum, wl.weight_decay, pipelined=True, mlp=(d.d_in, d.d_hidden, d.d_out, d.mb),
+                       mlp_defer=True)
+
+        def run(k):
+            n = 0
+            with torch.cuda.stream(eng.stream_acc):
+                for _ in range(k):
+                    for j in range(n_mb):
+                        eng.accumulate_mlp(j % wl.W, xp[n % wl.mlp_pool], yp[n % wl.mlp_pool]); n += 1
+                    eng.sync_step(); eng.wait()
+                    eng.stream_acc.synchronize()
+            torch.cuda.synchronize()
+
+        run(2)
+        eng.profile(True)
+        run(iters)
+        ns, ms = eng.kernel_stats(B.K_SYNC)
+        eng.profile(False)
+        eng.check(); eng.destroy()
+        us = ms / ns * 1e3
+        nbytes = 18 * w1 + n_mb * 2 * d.mb * (d.d_in + d.d_hidden) + (n_mb + 18) * (wl.P - w1)
+        return {"microbatches_pooled": n_mb, "us": us, "algorithmic_bytes": nbytes, "gbs": nbytes / us / 1e3,
+                "frac_of_measured_hbm": nbytes / us / 1e3 / peaks["hbm_gbs"],
+                "contraction_tflops": 2.0 * w1 * d.mb * n_mb / us / 1e6}
+
+    out["deferred_step_alone"] = pooled_step()
     for name, kw in (("single_calls", dict(max_batch=1)), ("single_calls_ring_dw1", dict(max_batch=1, variant=4)),
                      ("batch_calls_up_to_4", dict(max_batch=4)), ("batch_calls_up_to_4_tile_per_cta_dw1", dict(max_batch=4, variant=8))):
         out["serial_" + name] = run_case(serial=1, **kw)
