@@ -200,7 +200,9 @@ int abs_accumulate_host(abs_ctx *ctx, uint32_t worker, const void *grad_host);
  * the worker (workers compute concurrently, as in the paper; what a worker's calls add to its row is added in call
  * order; the dW1 GEMM of a call runs on a second, lowest-priority stream of the worker, so that the worker's next
  * call can start beside it), which start after everything enqueued on stream_acc so far; abs_sync_step, abs_wait, abs_check,
- * abs_accumulate, abs_accumulate_host and abs_accumulator make stream_acc wait for all of them. */
+ * abs_accumulate, abs_accumulate_host and abs_accumulator make stream_acc wait for all of them.  With
+ * ABS_FLAG_MLP_DEFER a call adds nothing to the row and launches no dW1 kernel (see the flag): calls are then spread
+ * over the internal streams whoever their workers are. */
 int abs_accumulate_mlp(abs_ctx *ctx, uint32_t worker, const void *x_dev, const int32_t *y_dev);
 
 /* n (1..8) consecutive reference batches of one worker in one call: the same computation as n calls of
