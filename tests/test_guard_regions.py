@@ -31,7 +31,8 @@ def _make(x0_d, W, wl, dev, **kw):
     from paper_2308_15164_b200 import binding as B
 
     flags = (B.FLAG_PIPELINED if kw.get("pipelined") else 0) | (B.FLAG_MLP if kw.get("mlp") else 0) | \
-            (B.FLAG_OVERWRITE_FIRST if kw.get("overwrite_first") else 0) | (B.FLAG_MLP_COALESCE if kw.get("mlp_coalesce") else 0)
+            (B.FLAG_OVERWRITE_FIRST if kw.get("overwrite_first") else 0) | (B.FLAG_MLP_COALESCE if kw.get("mlp_coalesce") else 0) | \
+            (B.FLAG_MLP_DEFER if kw.get("mlp_defer") else 0)
     gd = kw.get("grad_dtype", B.GRAD_F32)
     cfg = B.make_config(x0_d.numel(), W, wl.lr, wl.momentum, wl.weight_decay, 0.0, gd, flags, kw.get("mlp"), 1, 2 if kw.get("pipelined") else 0)
     g = Guarded(B.abs_workspace_bytes(cfg), dev)
@@ -98,3 +99,44 @@ def test_mlp_and_multi_gpu_paths_stay_inside_their_workspaces():
     assert pairs[0][1].intact()
     for e in ranks:
         e.destroy()
+
+
+@pytest.mark.parametrize("pipelined", [False, True], ids=["eager", "pipelined"])
+def test_deferred_mlp_mode_stays_inside_its_workspace(pipelined):
+    """ABS_FLAG_MLP_DEFER: the operand pools are the last regions of the workspace, right in front of the upper guard.
+    Single, gathered and batch calls (up to eight micro-batches), a pool that overflows, the step from the pooled
+    operands and the one from the rows, a read of the rows and an export."""
+    import torch
+
+    from paper_2308_15164_b200 import binding as B
+
+    dev = torch.device("cuda:0")
+    wl = wlm.config(4, small=True, T=3)
+    d = wl.mlp
+    mlp = (d.d_in, d.d_hidden, d.d_out, d.mb)
+    x0 = torch.from_numpy(wlm.params0(wl)).to(dev)
+    xs, ys = wlm.mlp_batches(wl)
+    xs_d, ys_d = torch.from_numpy(xs).to(dev), torch.from_numpy(ys).to(dev)
+    torch.cuda.synchronize()
+    for coalesce in (False, True):
+        eng, g = _make(x0, 2, wl, dev, pipelined=pipelined, mlp=mlp, mlp_defer=True, mlp_coalesce=coalesce)
+        for t in range(4):
+            if t == 2:
+                eng.set_launch(B.K_MLP_BWD, 1)       # rows first from here on
+            for i in range(2):
+                for k in range(3):
+                    eng.accumulate_mlp(i, xs_d[(t + i + k) % 8], ys_d[(t + i + k) % 8])
+                eng.accumulate_mlp_batch(i, 8, xs_d[8:16], ys_d[8:16])
+                eng.accumulate_mlp_batch(i, 5, xs_d[3:8], ys_d[3:8])
+            if t == 1:                               # 32 slots: this iteration overflows the pool
+                for k in range(6):
+                    eng.accumulate_mlp(k % 2, xs_d[k], ys_d[k])
+                eng.accumulator(eng.counters()[1], 0)
+            eng.sync_step()
+        eng.check()
+        eng.synchronize()
+        assert g.intact(), coalesce
+        blob = eng.state_export()
+        eng.state_import(blob)
+        assert g.intact()
+        eng.destroy()
