@@ -510,3 +510,41 @@ def test_learning_rate_schedule_eq6_and_weight_decay_in_the_pooled_step():
         outs.append(got)
         eng.destroy()
     assert np.array_equal(outs[0], outs[1])
+
+
+@pytest.mark.parametrize("pipelined", [False, True], ids=["eager", "pipelined"])
+def test_one_worker(pipelined):
+    """W = 1 (every kernel chained, deep pipelines): single and batch calls over three iterations against the oracle."""
+    import dataclasses
+
+    import torch
+
+    from paper_2308_15164_b200 import binding as B
+
+    wl = dataclasses.replace(wlm.config(4, small=True, T=3), W=1)
+    d = wl.mlp
+    x0 = wlm.params0(wl)
+    xs, ys = wlm.mlp_batches(wl)
+    xs_d, ys_d = torch.from_numpy(xs).cuda(), torch.from_numpy(ys).cuda()
+    o = AbsSgdOracle(x0, 1, wl.lr, wl.momentum, wl.weight_decay)
+    eng = B.AbsSgd(torch.from_numpy(x0).cuda(), 1, wl.lr, wl.momentum, wl.weight_decay, pipelined=pipelined,
+                   mlp=(d.d_in, d.d_hidden, d.d_out, d.mb), mlp_defer=True)
+    c = 0
+    for t, plan in enumerate([(1, 3, 1), (8,), (2, 1, 1, 5)]):
+        p = o.params()
+        for n in plan:
+            if n == 1:
+                eng.accumulate_mlp(0, xs_d[c], ys_d[c])
+            else:
+                eng.accumulate_mlp_batch(0, n, xs_d[c:c + n], ys_d[c:c + n])
+            for j in range(n):
+                o.accumulate(0, _grad(p, xs, ys, c + j, wl))
+            c += n
+        eng.sync_step(); o.sync_step()
+    eng.sync_step(); o.sync_step()
+    eng.check()
+    ref = o.params()
+    assert np.abs(ref - x0).max() > 1e-4
+    assert np.abs(eng.params_host().astype(np.float64) - ref).max() <= TOL * np.abs(ref).max()
+    assert [int(eng.consumed(s)[0]) for s in range(4)] == [0, 5, 8, 9]
+    eng.destroy()
