@@ -214,6 +214,14 @@ int abs_accumulate_mlp(abs_ctx *ctx, uint32_t worker, const void *x_dev, const i
  * y_dev: [n][mlp_mb] int32. */
 int abs_accumulate_mlp_batch(abs_ctx *ctx, uint32_t worker, uint32_t n, const void *x_dev, const int32_t *y_dev);
 
+/* The same call for n (1..8) reference batches that are NOT adjacent in memory: x_devs[j] / y_devs[j] point to
+ * micro-batch j ([mlp_mb, mlp_in] and [mlp_mb], aligned as for abs_accumulate_mlp); the two pointer arrays are host
+ * memory and are read before the call returns.  One cast launch reads all n buffers (on stream_acc, like every
+ * gradient call's first kernel); from there on the call is abs_accumulate_mlp_batch over the same micro-batches
+ * in list order, bit for bit. */
+int abs_accumulate_mlp_list(abs_ctx *ctx, uint32_t worker, uint32_t n, const void *const *x_devs,
+                            const int32_t *const *y_devs);
+
 /* Algorithm 1, Step 1 + compensation + "Update parameters" + t = t + 1 (see the file header).
  * Without ABS_FLAG_PIPELINED the fused kernel runs on stream_acc.  With it, the call makes
  * x_{t+1} (computed by the kernel launched one call earlier on stream_sync) visible to

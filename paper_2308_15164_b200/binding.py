@@ -62,6 +62,7 @@ _sig = {
     "abs_accumulate_host": (ctypes.c_int, [_vp, _u32, _vp]),
     "abs_accumulate_mlp": (ctypes.c_int, [_vp, _u32, _vp, _vp]),
     "abs_accumulate_mlp_batch": (ctypes.c_int, [_vp, _u32, _u32, _vp, _vp]),
+    "abs_accumulate_mlp_list": (ctypes.c_int, [_vp, _u32, _u32, ctypes.POINTER(ctypes.c_void_p), ctypes.POINTER(ctypes.c_void_p)]),
     "abs_sync_step": (ctypes.c_int, [_vp]),
     "abs_params": (ctypes.c_int, [_vp, ctypes.POINTER(_vp)]),
     "abs_params_host": (ctypes.c_int, [_vp, _vp]),
@@ -190,6 +191,14 @@ class AbsSgd:
 
     def accumulate_mlp_batch(self, worker: int, n: int, x, y):
         self._ck(lib.abs_accumulate_mlp_batch(self._h, worker, n, _ptr(x), _ptr(y)))
+
+    def accumulate_mlp_list(self, worker: int, xs, ys):
+        """n separate micro-batches (tensors or raw device addresses) in one call."""
+        n = len(xs)
+        assert n == len(ys)
+        xa = (ctypes.c_void_p * n)(*[_ptr(x) for x in xs])
+        ya = (ctypes.c_void_p * n)(*[_ptr(y) for y in ys])
+        self._ck(lib.abs_accumulate_mlp_list(self._h, worker, n, xa, ya))
 
     def sync_step(self):
         self._ck(lib.abs_sync_step(self._h))

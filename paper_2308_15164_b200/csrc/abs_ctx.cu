@@ -655,7 +655,7 @@ int coalesce_one(abs_ctx* c, uint32_t worker, const void* x_dev, const int32_t* 
         // starts later and the last group of an iteration holds the step back longer.)
         if (c->grp_n == 0)
             if (int rc = take_pool_slots(c, kMlpGatherMax, &c->grp_pool0)) return rc;
-        CK(launch_mlp_cast(c->mlp_dims, c->mlp_scratch[0], c->grp_pool0 + c->grp_n, 1, x_dev, c->x_bf16(), y_dev, &c->pool[c->cur],
+        CK(launch_mlp_cast(c->mlp_dims, c->mlp_scratch[0], c->grp_pool0 + c->grp_n, 1, &x_dev, c->x_bf16(), &y_dev, &c->pool[c->cur],
                            c->s_acc, (c->mlp_chain(false, 1) & kChainCast) != 0, mlp_mark, c));
         c->grp_workers.w[c->grp_n++] = (uint8_t)worker;
         c->h_cnt[(size_t)c->cur * c->cfg.W + worker] += 1;
@@ -680,7 +680,7 @@ int coalesce_one(abs_ctx* c, uint32_t worker, const void* x_dev, const int32_t* 
         c->pend_age[worker] = ++c->pend_clock;
     }
     const int slot = c->pend_n[worker];
-    CK(launch_mlp_cast(c->mlp_dims, c->mlp_scratch[c->pend_set[worker]], slot, 1, x_dev, c->x_bf16(), y_dev, nullptr, c->s_acc,
+    CK(launch_mlp_cast(c->mlp_dims, c->mlp_scratch[c->pend_set[worker]], slot, 1, &x_dev, c->x_bf16(), &y_dev, nullptr, c->s_acc,
                        (c->mlp_chain(false, 1) & kChainCast) != 0, mlp_mark, c));
     c->pend_n[worker] = slot + 1;
     c->h_cnt[(size_t)c->cur * c->cfg.W + worker] += 1;
@@ -888,15 +888,18 @@ int abs_accumulate_host(abs_ctx* c, uint32_t worker, const void* grad_host) {
     return ABS_OK;
 }
 
-int abs_accumulate_mlp_batch(abs_ctx* c, uint32_t worker, uint32_t n, const void* x_dev, const int32_t* y_dev) {
+int abs_accumulate_mlp_list(abs_ctx* c, uint32_t worker, uint32_t n, const void* const* x_devs, const int32_t* const* y_devs) {
     if (!live(c)) return ABS_ESTATE;
     if (!c->mlp) return invalid(c, "context was created without ABS_FLAG_MLP");
     if (worker >= c->cfg.W) return invalid(c, "worker index out of range");
     if (n == 0 || n > (uint32_t)kMlpMaxBatch) return invalid(c, "n must be in 1..8");
-    if (!x_dev || (reinterpret_cast<uintptr_t>(x_dev) & 15)) return invalid(c, "x pointer must be non-NULL and 16-byte aligned");
-    if (!y_dev || (reinterpret_cast<uintptr_t>(y_dev) & 3)) return invalid(c, "y pointer must be non-NULL and 4-byte aligned");
+    if (!x_devs || !y_devs) return invalid(c, "pointer list is NULL");
+    for (uint32_t j = 0; j < n; ++j) {
+        if (!x_devs[j] || (reinterpret_cast<uintptr_t>(x_devs[j]) & 15)) return invalid(c, "x pointer must be non-NULL and 16-byte aligned");
+        if (!y_devs[j] || (reinterpret_cast<uintptr_t>(y_devs[j]) & 3)) return invalid(c, "y pointer must be non-NULL and 4-byte aligned");
+    }
     const bool serial = c->ctas_per_sm[ABS_K_MLP_FWD] == 1;   // measurement aid: everything on stream_acc
-    if (c->coalesce && n == 1 && !serial) return coalesce_one(c, worker, x_dev, y_dev);
+    if (c->coalesce && n == 1 && !serial) return coalesce_one(c, worker, x_devs[0], y_devs[0]);
     if (int rc = flush_worker(c, worker)) return rc;           // the worker's row is added to in call order
     // Only the cast kernel reads the caller's buffers; it runs on stream_acc, in call order.  The rest of the
     // call (forward, loss, backward, dW1) runs on the worker's internal stream, so that the latency chains of
@@ -914,11 +917,28 @@ int abs_accumulate_mlp_batch(abs_ctx* c, uint32_t worker, uint32_t n, const void
     // ABS_FLAG_OVERWRITE_FIRST -- stale): it is stored, not added, and dW1 skips reading the 4 d_in d_hidden
     // bytes of the slice.  0 + g = g, so the default mode's results do not change.
     const bool first = c->h_cnt[(size_t)c->cur * c->cfg.W + worker] == 0;
-    CK(launch_mlp_cast(c->mlp_dims, c->mlp_scratch[set], c->defer ? pool0 : 0, (int)n, x_dev, c->x_bf16(), y_dev,
+    CK(launch_mlp_cast(c->mlp_dims, c->mlp_scratch[set], c->defer ? pool0 : 0, (int)n, x_devs, c->x_bf16(), y_devs,
                        c->defer ? &c->pool[c->cur] : nullptr, c->s_acc, (c->mlp_chain(serial, (int)n) & kChainCast) != 0, mlp_mark, c));
     if (int rc = run_mlp_group(c, worker, set, (int)n, first, pool0)) return rc;
     c->h_cnt[(size_t)c->cur * c->cfg.W + worker] += (int32_t)n;
     return ABS_OK;
+}
+
+int abs_accumulate_mlp_batch(abs_ctx* c, uint32_t worker, uint32_t n, const void* x_dev, const int32_t* y_dev) {
+    if (!live(c)) return ABS_ESTATE;
+    if (!c->mlp) return invalid(c, "context was created without ABS_FLAG_MLP");
+    if (n == 0 || n > (uint32_t)kMlpMaxBatch) return invalid(c, "n must be in 1..8");
+    if (!x_dev || (reinterpret_cast<uintptr_t>(x_dev) & 15)) return invalid(c, "x pointer must be non-NULL and 16-byte aligned");
+    if (!y_dev || (reinterpret_cast<uintptr_t>(y_dev) & 3)) return invalid(c, "y pointer must be non-NULL and 4-byte aligned");
+    // micro-batch j at x_dev + j * mb * mlp_in elements, y_dev + j * mb
+    const void* xs[kMlpMaxBatch];
+    const int32_t* ys[kMlpMaxBatch];
+    const size_t es = c->x_bf16() ? 2 : 4;
+    for (uint32_t j = 0; j < n; ++j) {
+        xs[j] = static_cast<const char*>(x_dev) + (size_t)j * c->mlp_dims.mb * c->mlp_dims.d_in * es;
+        ys[j] = y_dev + (size_t)j * c->mlp_dims.mb;
+    }
+    return abs_accumulate_mlp_list(c, worker, n, xs, ys);
 }
 
 int abs_accumulate_mlp(abs_ctx* c, uint32_t worker, const void* x_dev, const int32_t* y_dev) {

@@ -222,8 +222,9 @@ typedef void (*MlpMark)(void* user, int kernel_class, int n, cudaStream_t stream
 // pool (ABS_FLAG_MLP_DEFER): the cast writes into pool slots slot0.. instead of the scratch set's; the front kernels
 // read them there (pool_slot0..), leave bf16(dZ)^T and the micro-batches' db1 | dW2 | db2 there and add nothing to
 // acc_row; cnt is then the counter array of the whole set, and micro-batch j bumps cnt[workers->w[j]], atomically.
-cudaError_t launch_mlp_cast(const MlpDims& d, const MlpScratch& s, int slot0, int nb, const void* x_dev, bool x_is_bf16,
-                            const int32_t* y_dev, const MlpPool* pool, cudaStream_t stream, bool chained, MlpMark mark,
+// x_devs / y_devs: the caller's buffers of the nb micro-batches (one pointer each; they need not be adjacent).
+cudaError_t launch_mlp_cast(const MlpDims& d, const MlpScratch& s, int slot0, int nb, const void* const* x_devs, bool x_is_bf16,
+                            const int32_t* const* y_devs, const MlpPool* pool, cudaStream_t stream, bool chained, MlpMark mark,
                             void* user);
 cudaError_t launch_mlp_front(const MlpDims& d, const MlpScratch& s, const float* x_pub, const __nv_bfloat16* shadow,
                              int shadow_idx, int nb, bool store, float* acc_row, int32_t* cnt, const MlpPool* pool,

@@ -61,16 +61,21 @@ __device__ __forceinline__ uint32_t pack_bf16x2(float a, float b) {
 // Also copies the labels, so that the caller's buffers are read by this kernel only (the rest of
 // the gradient may run on another stream after the caller's stream has moved on).
 // --------------------------------------------------------------------------------------------
+struct CastList {          // the caller's buffers of the micro-batches of a call (contiguous or not)
+    const void* x[kMlpMaxBatch];
+    const int32_t* y[kMlpMaxBatch];
+};
 template <bool kBf16In>   // the caller's X already holds bf16 values: copied (and transposed) as they are
-__global__ void __launch_bounds__(256) k_cast_x(const void* __restrict__ x_in, const int32_t* __restrict__ y,
+__global__ void __launch_bounds__(256) k_cast_x(const __grid_constant__ CastList in,
                                                 __nv_bfloat16* __restrict__ xb, __nv_bfloat16* __restrict__ xtb,
                                                 int32_t* __restrict__ ycopy, int d_in) {
     __shared__ __nv_bfloat16 tile[16][kMB + 8];
     const int c0 = blockIdx.x * 16;
     pdl_wait();
     pdl_trigger();
-    if (blockIdx.x == 0 && threadIdx.x < kMB) ycopy[blockIdx.y * kMB + threadIdx.x] = y[blockIdx.y * kMB + threadIdx.x];
-    const size_t mb_off = (size_t)blockIdx.y * kMB * d_in;   // micro-batch blockIdx.y of the call
+    const void* x_in = in.x[blockIdx.y];                     // micro-batch blockIdx.y of the call
+    if (blockIdx.x == 0 && threadIdx.x < kMB) ycopy[blockIdx.y * kMB + threadIdx.x] = in.y[blockIdx.y][threadIdx.x];
+    const size_t mb_off = (size_t)blockIdx.y * kMB * d_in;
     xb += mb_off;
     xtb += (size_t)blockIdx.y * d_in * kMB;
     {
@@ -78,9 +83,9 @@ __global__ void __launch_bounds__(256) k_cast_x(const void* __restrict__ x_in, c
         const size_t at = (size_t)r * d_in + c0 + 4 * q;
         uint2 pk;
         if (kBf16In) {
-            pk = *reinterpret_cast<const uint2*>(static_cast<const __nv_bfloat16*>(x_in) + mb_off + at);
+            pk = *reinterpret_cast<const uint2*>(static_cast<const __nv_bfloat16*>(x_in) + at);
         } else {
-            const float4 v = *reinterpret_cast<const float4*>(static_cast<const float*>(x_in) + mb_off + at);
+            const float4 v = *reinterpret_cast<const float4*>(static_cast<const float*>(x_in) + at);
             pk.x = pack_bf16x2(v.x, v.y);
             pk.y = pack_bf16x2(v.z, v.w);
         }
@@ -1476,17 +1481,23 @@ cudaError_t mlp_make_acc_tmap(void* tmap_out, const MlpDims& d, float* acc_row) 
                : cudaErrorInvalidValue;
 }
 
-cudaError_t launch_mlp_cast(const MlpDims& d, const MlpScratch& s, int slot0, int nb, const void* x_dev, bool x_is_bf16,
-                            const int32_t* y_dev, const MlpPool* pool, cudaStream_t stream, bool chained, MlpMark mark,
+cudaError_t launch_mlp_cast(const MlpDims& d, const MlpScratch& s, int slot0, int nb, const void* const* x_devs, bool x_is_bf16,
+                            const int32_t* const* y_devs, const MlpPool* pool, cudaStream_t stream, bool chained, MlpMark mark,
                             void* user) {
+    if (nb < 1 || nb > kMaxBatch) return cudaErrorInvalidValue;
+    CastList in{};
+    for (int j = 0; j < nb; ++j) {
+        in.x[j] = x_devs[j];
+        in.y[j] = y_devs[j];
+    }
     mark(user, ABS_K_MLP_FWD, -1, stream);   // part 0 of the forward class: the cast
     // micro-batch j of the call goes to slot slot0 + j of the scratch set, or of the pool
     __nv_bfloat16* xb = (pool ? pool->xb : s.xb) + (size_t)slot0 * kMB * d.d_in;
     __nv_bfloat16* xtb = (pool ? pool->xtb : s.xtb) + (size_t)slot0 * d.d_in * kMB;
     int32_t* yc = (pool ? pool->ycopy : s.ycopy) + slot0 * kMB;
     const dim3 grid(d.d_in / 16, nb);
-    const cudaError_t e = x_is_bf16 ? launch_kernel(k_cast_x<true>, grid, 256, 0, stream, chained, x_dev, y_dev, xb, xtb, yc, d.d_in)
-                                    : launch_kernel(k_cast_x<false>, grid, 256, 0, stream, chained, x_dev, y_dev, xb, xtb, yc, d.d_in);
+    const cudaError_t e = x_is_bf16 ? launch_kernel(k_cast_x<true>, grid, 256, 0, stream, chained, in, xb, xtb, yc, d.d_in)
+                                    : launch_kernel(k_cast_x<false>, grid, 256, 0, stream, chained, in, xb, xtb, yc, d.d_in);
     mark(user, ABS_K_MLP_FWD, 1, stream);
     return e;
 }

@@ -548,3 +548,80 @@ def test_one_worker(pipelined):
     assert np.abs(eng.params_host().astype(np.float64) - ref).max() <= TOL * np.abs(ref).max()
     assert [int(eng.consumed(s)[0]) for s in range(4)] == [0, 5, 8, 9]
     eng.destroy()
+
+
+@pytest.mark.parametrize("defer", [False, True], ids=["per-call-dw1", "deferred-dw1"])
+def test_list_call_equals_the_batch_call_bit_for_bit(defer):
+    """abs_accumulate_mlp_list over n separate buffers = abs_accumulate_mlp_batch over the same micro-batches laid
+    out contiguously: same kernels behind one cast launch, same bits (rows, counters, parameters after the steps)."""
+    import torch
+
+    from paper_2308_15164_b200 import binding as B
+
+    wl = wlm.config(4, small=True, T=2)
+    d = wl.mlp
+    x0 = wlm.params0(wl)
+    xs, ys = wlm.mlp_batches(wl)
+    xs_d, ys_d = torch.from_numpy(xs).cuda(), torch.from_numpy(ys).cuda()
+    plan = [(0, [3, 9, 1]), (2, [5]), (0, [7, 2, 11, 4, 6, 8, 10, 12]), (3, [13, 14])]   # worker, pool indices (scattered)
+    outs = []
+    for form in ("list", "batch"):
+        eng = B.AbsSgd(torch.from_numpy(x0).cuda(), wl.W, wl.lr, wl.momentum, wl.weight_decay, pipelined=True,
+                       mlp=(d.d_in, d.d_hidden, d.d_out, d.mb), mlp_defer=defer)
+        for t in range(2):
+            for (i, idx) in plan:
+                if form == "list":
+                    eng.accumulate_mlp_list(i, [xs_d[j] for j in idx], [ys_d[j] for j in idx])
+                else:
+                    xc = torch.stack([xs_d[j] for j in idx]).contiguous()
+                    yc = torch.stack([ys_d[j] for j in idx]).contiguous()
+                    torch.cuda.synchronize()
+                    eng.accumulate_mlp_batch(i, len(idx), xc, yc)
+                    eng.synchronize()                # xc / yc go out of scope: their reads must have happened
+            if t == 1:
+                cur = eng.counters()[1]
+                rows = [eng.accumulator(cur, i).cpu().numpy().copy() for i in range(wl.W)]
+            eng.sync_step()
+        eng.sync_step()
+        eng.check()
+        outs.append((rows, eng.params_host().copy(), [eng.consumed(s).copy() for s in range(3)]))
+        eng.destroy()
+    (ra, xa, ca), (rb, xb, cb) = outs
+    assert np.abs(xa - x0).max() > 1e-5
+    assert np.array_equal(xa, xb)
+    for a, b in zip(ra, rb):
+        assert np.array_equal(a, b)
+    for a, b in zip(ca, cb):
+        assert np.array_equal(a, b)
+    assert ca[1].tolist() == [11, 0, 1, 2]
+
+
+def test_list_call_argument_checks():
+    import ctypes
+
+    import torch
+
+    from paper_2308_15164_b200 import binding as B
+
+    wl = wlm.config(4, small=True)
+    d = wl.mlp
+    x = torch.zeros((2, d.mb, d.d_in), device="cuda")
+    y = torch.zeros((2, d.mb), dtype=torch.int32, device="cuda")
+    eng = B.AbsSgd(torch.from_numpy(wlm.params0(wl)).cuda(), wl.W, wl.lr, mlp=(d.d_in, d.d_hidden, d.d_out, d.mb))
+    n0 = eng.launch_count()
+    xa = (ctypes.c_void_p * 2)(x[0].data_ptr(), x[1].data_ptr())
+    ya = (ctypes.c_void_p * 2)(y[0].data_ptr(), y[1].data_ptr())
+    bad = (ctypes.c_void_p * 2)(x[0].data_ptr(), None)
+    mis = (ctypes.c_void_p * 2)(x[0].data_ptr(), x[1].data_ptr() + 4)
+    f = B.lib.abs_accumulate_mlp_list
+    assert f(eng._h, 0, 0, xa, ya) == B.EINVAL
+    assert f(eng._h, 0, 9, xa, ya) == B.EINVAL
+    assert f(eng._h, wl.W, 2, xa, ya) == B.EINVAL
+    assert f(eng._h, 0, 2, None, ya) == B.EINVAL
+    assert f(eng._h, 0, 2, bad, ya) == B.EINVAL
+    assert f(eng._h, 0, 2, mis, ya) == B.EINVAL
+    assert f(eng._h, 0, 2, xa, bad) == B.EINVAL
+    assert eng.launch_count() == n0 and not eng.counters()[0].any()
+    assert f(eng._h, 0, 2, xa, ya) == B.OK
+    eng.check()
+    eng.destroy()
