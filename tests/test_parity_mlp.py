@@ -265,7 +265,10 @@ def test_workload4_full_length(small):
           entry element-wise (_close_trajectory; hidden units with an undecided ReLU gate apart);
       (b) the free-running library over all 50 iterations, eager and pipelined: bit-identical to each other,
           counters and consumed b_i bit-exact against the oracle, parameters within 2e-3 of the oracle's while the
-          amplification is still small (iterations 1..8) and within a coarse sanity bound at the end."""
+          amplification is still small (iterations 1..8) and within a coarse sanity bound at the end.
+    Both with and without ABS_FLAG_MLP_DEFER (against the same oracle run): with it, in (a) the rows are what
+    abs_accumulator makes the library contract from the pooled operands (one contraction per worker over its
+    micro-batches of the iteration), in (b) every step works straight from the pool."""
     import concurrent.futures
 
     import torch
@@ -292,29 +295,30 @@ def test_workload4_full_length(small):
                 o.accumulate(i, g)
                 und[i] |= u
             # (a) this iteration on the library, started from the oracle's x_t
-            eng = B.AbsSgd(torch.from_numpy(p).cuda(), wl.W, wl.lr, wl.momentum, wl.weight_decay,
-                           mlp=(d.d_in, d.d_hidden, d.d_out, d.mb))
-            for (i, k, c) in calls:
-                eng.accumulate_mlp(i, xs_d[c % wl.mlp_pool], ys_d[c % wl.mlp_pool])
-            eng.check()
-            assert np.array_equal(eng.counters()[0][0], o.cnt[o.cur])
-            for i in range(wl.W):
-                if o.cnt[o.cur, i] == 0:
-                    continue
-                got = eng.accumulator(0, i).cpu().numpy()
-                want = o.acc[o.cur, i]
-                clear = np.setdiff1d(np.arange(d.d_hidden), sorted(und[i]))
-                gW1, gb1, gW2, gb2 = mlp_split(got, *dims)
-                wW1, wb1, wW2, wb2 = mlp_split(want, *dims)
-                _close_trajectory(gW2, wW2, f"iteration {t} worker {i} dW2")
-                _close_trajectory(gb2, wb2, f"iteration {t} worker {i} db2")
-                e_max, e_fro = _close_trajectory(gW1[:, clear], wW1[:, clear], f"iteration {t} worker {i} dW1")
-                _close_trajectory(gb1[clear], wb1[clear], f"iteration {t} worker {i} db1")
-                worst, worst_fro = max(worst, float(e_max)), max(worst_fro, float(e_fro))
-                if und[i]:
-                    u = sorted(und[i])
-                    assert np.abs(gW1[:, u] - wW1[:, u]).max() <= 0.2 * np.abs(wW1).max()
-            eng.destroy()
+            for defer in (False, True):
+                eng = B.AbsSgd(torch.from_numpy(p).cuda(), wl.W, wl.lr, wl.momentum, wl.weight_decay,
+                               mlp=(d.d_in, d.d_hidden, d.d_out, d.mb), mlp_defer=defer)
+                for (i, k, c) in calls:
+                    eng.accumulate_mlp(i, xs_d[c % wl.mlp_pool], ys_d[c % wl.mlp_pool])
+                eng.check()
+                assert np.array_equal(eng.counters()[0][0], o.cnt[o.cur])
+                for i in range(wl.W):
+                    if o.cnt[o.cur, i] == 0:
+                        continue
+                    got = eng.accumulator(0, i).cpu().numpy()
+                    want = o.acc[o.cur, i]
+                    clear = np.setdiff1d(np.arange(d.d_hidden), sorted(und[i]))
+                    gW1, gb1, gW2, gb2 = mlp_split(got, *dims)
+                    wW1, wb1, wW2, wb2 = mlp_split(want, *dims)
+                    _close_trajectory(gW2, wW2, f"iteration {t} worker {i} dW2 (defer={defer})")
+                    _close_trajectory(gb2, wb2, f"iteration {t} worker {i} db2")
+                    e_max, e_fro = _close_trajectory(gW1[:, clear], wW1[:, clear], f"iteration {t} worker {i} dW1 (defer={defer})")
+                    _close_trajectory(gb1[clear], wb1[clear], f"iteration {t} worker {i} db1")
+                    worst, worst_fro = max(worst, float(e_max)), max(worst_fro, float(e_fro))
+                    if und[i]:
+                        u = sorted(und[i])
+                        assert np.abs(gW1[:, u] - wW1[:, u]).max() <= 0.2 * np.abs(wW1).max()
+                eng.destroy()
             o.sync_step()
             ref_xs.append(o.params())
             ref_states.append(o.counters())
@@ -323,33 +327,35 @@ def test_workload4_full_length(small):
     print(f"workload 4 ({'small' if small else 'full size'}): worst per-iteration dW1 deviation {worst:.2e} of max|dW1|, "
           f"{worst_fro:.2e} in Frobenius norm")
     # (b) the free-running library
-    outs = []
-    for pipelined in (False, True):
-        eng = _engine(wl, x0, pipelined=pipelined)
-        states, early = [], 0.0
-        for t, calls in enumerate(wlm.iter_calls(wl)):
-            for (i, k, c) in calls:
-                eng.accumulate_mlp(i, xs_d[c % wl.mlp_pool], ys_d[c % wl.mlp_pool])
-            eng.sync_step()
-            states.append(eng.counters())
-            if t < 8:
-                got_t = eng.params_host()
-                err = np.abs(got_t.astype(np.float64) - ref_xs[t]).max() / np.abs(ref_xs[t]).max()
-                assert err <= TOL, f"pipelined={pipelined}, x_{t + 1}: {err:.3e}"
-                early = max(early, err)
-        eng.check()
-        got = eng.params_host()
-        consumed = [eng.consumed(s) for s in range(len(states))]
-        eng.destroy()
-        end = np.abs(got.astype(np.float64) - ref).max() / np.abs(ref).max()
-        print(f"  free run, pipelined={pipelined}: x_1..x_8 within {early:.2e}, x_50 within {end:.2e} of max|x|")
-        assert end <= 0.1, "the free run left the oracle's neighbourhood altogether"
-        for (c1, cur1, t1), (c2, cur2, t2) in zip(states, ref_states):
-            assert np.array_equal(c1, c2) and (cur1, t1) == (cur2, t2)
-        for a, b in zip(consumed, o.consumed):
-            assert np.array_equal(a, b)
-        outs.append(got)
-    assert np.array_equal(outs[0], outs[1]), "eager and pipelined runs must be bit-identical"
+    for defer in (False, True):
+        outs = []
+        for pipelined in (False, True):
+            eng = B.AbsSgd(torch.from_numpy(x0).cuda(), wl.W, wl.lr, wl.momentum, wl.weight_decay, pipelined=pipelined,
+                           mlp=(d.d_in, d.d_hidden, d.d_out, d.mb), mlp_defer=defer)
+            states, early = [], 0.0
+            for t, calls in enumerate(wlm.iter_calls(wl)):
+                for (i, k, c) in calls:
+                    eng.accumulate_mlp(i, xs_d[c % wl.mlp_pool], ys_d[c % wl.mlp_pool])
+                eng.sync_step()
+                states.append(eng.counters())
+                if t < 8:
+                    got_t = eng.params_host()
+                    err = np.abs(got_t.astype(np.float64) - ref_xs[t]).max() / np.abs(ref_xs[t]).max()
+                    assert err <= TOL, f"pipelined={pipelined}, x_{t + 1}: {err:.3e}"
+                    early = max(early, err)
+            eng.check()
+            got = eng.params_host()
+            consumed = [eng.consumed(s) for s in range(len(states))]
+            eng.destroy()
+            end = np.abs(got.astype(np.float64) - ref).max() / np.abs(ref).max()
+            print(f"  free run, defer={defer}, pipelined={pipelined}: x_1..x_8 within {early:.2e}, x_50 within {end:.2e} of max|x|")
+            assert end <= 0.1, "the free run left the oracle's neighbourhood altogether"
+            for (c1, cur1, t1), (c2, cur2, t2) in zip(states, ref_states):
+                assert np.array_equal(c1, c2) and (cur1, t1) == (cur2, t2)
+            for a, b in zip(consumed, o.consumed):
+                assert np.array_equal(a, b)
+            outs.append(got)
+        assert np.array_equal(outs[0], outs[1]), "eager and pipelined runs must be bit-identical"
 
 
 @pytest.mark.parametrize("n", [1, 3])
