@@ -625,3 +625,34 @@ def test_list_call_argument_checks():
     assert f(eng._h, 0, 2, xa, ya) == B.OK
     eng.check()
     eng.destroy()
+
+
+def test_bf16_inputs_in_deferred_mode():
+    """ABS_FLAG_MLP_X_BF16 with ABS_FLAG_MLP_DEFER: X handed over as bf16 values gives the same bits as the same
+    values handed over as fp32 (the cast copies them as they are), single, batch and list calls."""
+    import torch
+
+    from paper_2308_15164_b200 import binding as B
+
+    wl = wlm.config(4, small=True, T=2)
+    d = wl.mlp
+    x0 = wlm.params0(wl)
+    xs, ys = wlm.mlp_batches(wl)
+    xb = torch.from_numpy(xs).cuda().to(torch.bfloat16)          # the values both runs see
+    xf = xb.to(torch.float32)
+    ys_d = torch.from_numpy(ys).cuda()
+    outs = []
+    for x_bf16, xd in ((True, xb), (False, xf)):
+        eng = B.AbsSgd(torch.from_numpy(x0).cuda(), wl.W, wl.lr, wl.momentum, wl.weight_decay, pipelined=True,
+                       mlp=(d.d_in, d.d_hidden, d.d_out, d.mb), mlp_defer=True, mlp_x_bf16=x_bf16)
+        for t in range(2):
+            eng.accumulate_mlp(0, xd[3], ys_d[3])
+            eng.accumulate_mlp_batch(1, 3, xd[4:7], ys_d[4:7])
+            eng.accumulate_mlp_list(2, [xd[9], xd[1]], [ys_d[9], ys_d[1]])
+            eng.sync_step()
+        eng.sync_step()
+        eng.check()
+        outs.append(eng.params_host().copy())
+        eng.destroy()
+    assert np.abs(outs[0] - x0).max() > 1e-5
+    assert np.array_equal(outs[0], outs[1])
