@@ -656,3 +656,34 @@ def test_bf16_inputs_in_deferred_mode():
         eng.destroy()
     assert np.abs(outs[0] - x0).max() > 1e-5
     assert np.array_equal(outs[0], outs[1])
+
+
+def test_gradient_norm_flag_in_deferred_mode():
+    """ABS_FLAG_GRAD_NORM with ABS_FLAG_MLP_DEFER: the norm is formed by the row-based step, so every iteration's rows
+    are completed first; |Gbar|^2 and the parameters follow the oracle."""
+    import torch
+
+    from paper_2308_15164_b200 import binding as B
+
+    wl = wlm.config(4, small=True, T=3)
+    d = wl.mlp
+    x0 = wlm.params0(wl)
+    xs, ys = wlm.mlp_batches(wl)
+    xs_d, ys_d = torch.from_numpy(xs).cuda(), torch.from_numpy(ys).cuda()
+    o = AbsSgdOracle(x0, wl.W, wl.lr, wl.momentum, wl.weight_decay)
+    eng = B.AbsSgd(torch.from_numpy(x0).cuda(), wl.W, wl.lr, wl.momentum, wl.weight_decay, pipelined=True,
+                   mlp=(d.d_in, d.d_hidden, d.d_out, d.mb), mlp_defer=True, grad_norm=True)
+    for t, calls in enumerate(wlm.iter_calls(wl)):
+        p = o.params()
+        for (i, k, c) in calls:
+            o.accumulate(i, _grad(p, xs, ys, c, wl))
+            eng.accumulate_mlp(i, xs_d[c % wl.mlp_pool], ys_d[c % wl.mlp_pool])
+        eng.sync_step(); o.sync_step()
+    eng.sync_step(); o.sync_step()
+    eng.check()
+    assert np.abs(eng.params_host().astype(np.float64) - o.params()).max() <= TOL * np.abs(o.params()).max()
+    for s in range(1, 4):
+        want = o.gnorm2[s]
+        assert want > 0
+        assert abs(eng.grad_norm2(s) - want) <= 2 * TOL * want, (s, eng.grad_norm2(s), want)
+    eng.destroy()
